@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the LIME ranking-inference hot path on B200.
+
+One "step" = one batch through the online path: ragged offsets -> history gather -> n XOR layers (link states)
+-> candidate scoring.  The offline candidate->link precompute is timed separately (the paper caches it).
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N --steps K --warmup W
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2510_18239_b200 import synth  # noqa: E402
+
+METRIC = "candidate_scores_per_sec"
+UNIT = "candidates/s"
+ROTATE = 4                      # input sets rotated between steps so that no step is served from L2
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12      # 148 SMs x 128 FP32 lanes x FMA x max SM clock
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+# ----------------------------------------------------------------------------- algorithmic work per kernel and step
+def kernel_models(wl: synth.Workload, total_tokens: int):
+    """name -> (bound, algorithmic units per step, unit).  Bytes: what the stage must move; flops: what it must
+    compute (2 per multiply-add), for all launches of that kernel in one step."""
+    es = 4 if wl.dtype == synth.F32 else 2
+    d, ell, H, n, f = wl.d, wl.ell, wl.H, wl.n_layers, wl.dff
+    BC, BL, N = wl.B * wl.C, wl.B * wl.ell, total_tokens
+    hist_proj = sum((3 if j < n - 1 else 2) for j in range(n)) * 2.0 * N * d * d
+    link_proj = (ell + (n - 1) * BL) * 3 * 2.0 * d * d
+    glu = 4.0 * d * f * (BL * n + N * (n - 1))
+    down = 2.0 * d * f * (BL * n + N * (n - 1))
+    m = {
+        "k_score": ("hbm", BC * (es * ell + es * d + 4.0), "B"),
+        "k_gather": ("hbm", N * (4.0 + 2 * es * d), "B"),
+        "k_linear_simt_ln": ("alu", hist_proj + link_proj, "flop"),
+        "k_linear_simt_glu": ("alu", glu, "flop"),
+        "k_linear_simt": ("alu", down, "flop"),
+        "k_attn_link": ("alu", 4.0 * ell * d * N * n, "flop"),
+        "k_attn_hist": ("alu", 4.0 * ell * d * N * (n - 1), "flop"),
+    }
+    return m
+
+
+def model_for(name, models):
+    best = None
+    for k in models:
+        if name.startswith(k) and (best is None or len(k) > len(best)):
+            best = k
+    return models.get(best) if best else None
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            p = [x.strip() for x in ln.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(wl, inp, users, budget_s=None):
+    """Time the fp64 oracle (as it stands) on `users` of the batch: gather + encode + precompute + score."""
+    from oracle import lime_oracle as O
+    from tests import lime_helpers as Hh
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    table64_rows = {}
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(inp["lengths"])
+
+    class LazyTable:                      # widen only the rows the sample touches (the table is GBs)
+        shape = inp["table"].shape
+        dtype = np.float64
+
+        def __getitem__(self, key):
+            i = key[0] if isinstance(key, tuple) else key
+            r = table64_rows.get(i)
+            if r is None:
+                r = synth.storage_to_f64(inp["table"][i], wl.dtype)
+                table64_rows[i] = r
+            return r
+
+    tab = LazyTable()
+    done, t0 = 0, time.perf_counter()
+    for b in users:
+        Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg)
+        done += 1
+        if budget_s is not None and time.perf_counter() - t0 > budget_s:
+            break
+    return done, time.perf_counter() - t0
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, wl):
+    """--impl reference: the oracle, timed on host cores; each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = synth.make_inputs(wl, seed=0)
+    users_per_step = max(1, min(wl.B, 2))
+    for _ in range(args.warmup):
+        oracle_sample(wl, inp, range(1))
+    times = []
+    for s in range(args.steps):
+        users = [(s * users_per_step + u) % wl.B for u in range(users_per_step)]
+        _, dt = oracle_sample(wl, inp, users)
+        times.append(dt)
+    total = sum(times)
+    value = users_per_step * wl.C * args.steps / total
+    sample = f"{users_per_step} users x {wl.C} candidates per step (gather+encode+precompute+score), fp64 numpy"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(wl),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl):
+    return {"workload": wl.name, "B": wl.B, "N": wl.n_max if not wl.ragged else [wl.n_min, wl.n_max], "d": wl.d, "H": wl.H,
+            "ell": wl.ell, "n_layers": wl.n_layers, "C": wl.C, "V": wl.V, "zipf_s": wl.zipf_s,
+            "l2": f"{ROTATE} rotating input sets per step slot (candidate streams total > 126 MB L2)"}
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_18239_b200 import binding as Bd
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    # inputs: one model (table, links, weights) per rank; ROTATE request sets; users are sharded across ranks with
+    # a fixed per-GPU batch (weak scaling, no collective on the data path)
+    inp = synth.make_inputs(wl, seed=rank)
+    dt = Bd.LIME_F32 if wl.dtype == synth.F32 else Bd.LIME_BF16
+    lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff)
+    table = Bd.to_device(inp["table"], wl.dtype, dev)
+    links = Bd.to_device(inp["links"], wl.dtype, dev)
+    wts = {k: Bd.to_device(inp[k], wl.dtype, dev) for k in ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")}
+    lime.set_weights(links, [{k: wts[k][j] for k in wts} for j in range(wl.n_layers)])
+
+    sets, host_sets = [], []
+    pre_ms = []
+    for r in range(ROTATE):
+        lengths = synth.history_lengths(rank * 100 + r, wl.B, wl.n_min, wl.n_max)
+        total = int(lengths.sum())
+        hist_ids = synth.zipf_ids(rank * 100 + r, "hist_ids", total, wl.V, wl.zipf_s) if wl.zipf_s else inp["hist_ids"]
+        cand_ids = synth.uniform_ids(rank * 100 + r, "cand_ids", wl.B * wl.C, wl.V) if wl.zipf_s else inp["cand_ids"]
+        s = dict(lengths=torch.from_numpy(lengths).to(dev), hist_ids=torch.from_numpy(hist_ids).to(dev),
+                 cand_ids=torch.from_numpy(cand_ids).to(dev), total=total)
+        s["T"] = lime.gather_history(table, s["cand_ids"])
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s["W"] = lime.precompute_candidate_links(s["T"])          # warm
+        e0.record()
+        s["W"] = lime.precompute_candidate_links(s["T"])
+        e1.record()
+        torch.cuda.synchronize()
+        pre_ms.append(e0.elapsed_time(e1))
+        sets.append(s)
+        host_sets.append(dict(lengths=torch.from_numpy(lengths).pin_memory(), hist_ids=torch.from_numpy(hist_ids).pin_memory(),
+                              cand_ids=torch.from_numpy(cand_ids).pin_memory(), total=total))
+    max_total = max(s["total"] for s in sets)
+    off = torch.empty(wl.B + 1, dtype=torch.int32, device=dev)
+    hist = torch.empty((max_total, wl.d), dtype=lime.tdtype, device=dev)
+    ls = torch.empty((wl.B, wl.ell, wl.d), dtype=lime.tdtype, device=dev)
+    logits = torch.empty(wl.B * wl.C, dtype=torch.float32, device=dev)
+    ws = lime.workspace(wl.B, max_total)
+    ctx = lime.ctx
+
+    def step(i):
+        s = sets[i % ROTATE]
+        h = hist[: s["total"]]
+        Bd.lime_lengths_to_offsets(ctx, s["lengths"], off)
+        Bd.lime_gather_history(ctx, table, s["hist_ids"], h)
+        Bd.lime_encode_user(ctx, h, off, wl.B, None, ls, ws)
+        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    cap = 64 * args.steps + 64
+    Bd.lime_profile_start(cap)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for i in range(args.steps):
+        step(i)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    barrier()
+    records, launches = Bd.lime_profile_stop(cap)
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = ev[0].elapsed_time(ev[-1])
+    step_ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * wl.B * wl.C * args.steps / (total_ms * 1e-3)
+
+    # end to end through the C ABI from host buffers: request = (lengths, history ids, candidate ids) in pinned host
+    # memory; the corpus-level caches (table, phi(T L^t) for every item) are resident, as in the paper's serving flow
+    w_corpus = lime.precompute_candidate_links(table)
+    d_len = torch.empty(wl.B, dtype=torch.int32, device=dev)
+    d_hid = torch.empty(max_total, dtype=torch.int32, device=dev)
+    d_cid = torch.empty(wl.B * wl.C, dtype=torch.int32, device=dev)
+    Tbuf = torch.empty((wl.B * wl.C, wl.d), dtype=lime.tdtype, device=dev)
+    Wbuf = torch.empty((wl.B * wl.C, wl.ell), dtype=lime.tdtype, device=dev)
+    h_logits = torch.empty(wl.B * wl.C, dtype=torch.float32).pin_memory()
+    lime_w = Bd.Lime(wl.ell, 1, 1, 1, dtype=dt, gated_mlp=False)       # row gather of the [V x ell] weight cache
+
+    def e2e_step(i):
+        hs = host_sets[i % ROTATE]
+        n = hs["total"]
+        d_len.copy_(hs["lengths"], non_blocking=True)
+        d_hid[:n].copy_(hs["hist_ids"], non_blocking=True)
+        d_cid.copy_(hs["cand_ids"], non_blocking=True)
+        h = hist[:n]
+        Bd.lime_lengths_to_offsets(ctx, d_len, off)
+        Bd.lime_gather_history(ctx, table, d_hid[:n], h)
+        Bd.lime_encode_user(ctx, h, off, wl.B, None, ls, ws)
+        Bd.lime_gather_history(ctx, table, d_cid, Tbuf)
+        Bd.lime_gather_history(lime_w.ctx, w_corpus, d_cid, Wbuf)
+        Bd.lime_score_candidates(ctx, ls, wl.B, Wbuf, Tbuf, None, wl.C, wl.B * wl.C, None, logits)
+        h_logits.copy_(logits, non_blocking=True)
+        return 4 * (wl.B + n + wl.B * wl.C), 4 * wl.B * wl.C
+
+    for i in range(min(3, args.warmup)):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h2d = d2h = 0
+    e0.record()
+    for i in range(args.steps):
+        a, b = e2e_step(i)
+        h2d += a
+        d2h += b
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * wl.B * wl.C * args.steps / (e2e_ms * 1e-3)
+
+    if rank == 0:
+        pk = peaks()
+        avg_tokens = int(sum(s["total"] for s in sets) / ROTATE)
+        models = kernel_models(wl, avg_tokens)
+        agg = {}
+        for name, ms in records:
+            a = agg.setdefault(name, [0, 0.0])
+            a[0] += 1
+            a[1] += ms
+        ksum = sum(v[1] for v in agg.values()) or 1.0
+        kernels = []
+        for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
+            per_step_ms = ms / args.steps
+            entry = {"kernel": name, "launches_per_step": cnt / args.steps, "ms_per_step": per_step_ms, "share": ms / ksum}
+            mdl = model_for(name, models)
+            if mdl and per_step_ms > 0:
+                bound, units, unit = mdl
+                if bound == "hbm":
+                    ach = units / (per_step_ms * 1e-3) / 1e9
+                    entry.update(bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"])
+                else:
+                    ach = units / (per_step_ms * 1e-3) / 1e12
+                    peak = FP32_ALU_TFLOPS if bound == "alu" else pk["bf16_tflops_sustained"]
+                    entry.update(bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
+            kernels.append(entry)
+        dom = next((k for k in kernels if "bound" in k), None)
+        roofline = None
+        if dom:
+            roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
+                        "unit": dom["unit"], "frac": dom["frac"], "traffic": None,
+                        "peak_source": pk["source"] if dom["bound"] != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"}
+        score = next((k for k in kernels if k["kernel"].startswith("k_score")), None)
+
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget)
+            cpu = {"value": n_done * wl.C / dt_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                   "sample": f"first {n_done} users x {wl.C} candidates of the same workload, {dt_s:.1f} s "
+                             "(gather+encode+precompute+score, fp64 numpy)"}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": total_ms / args.steps, "p50_batch_latency_ms": step_ms[len(step_ms) // 2],
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == synth.BF16 else "f32",
+                "data": "synthetic", "config": workload_config(wl), "clocks": clocks,
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
+                        "ms_per_step": e2e_ms / args.steps},
+                "gpu_launches": launches, "roofline": roofline, "scoring_roofline": score, "kernels": kernels[:12],
+                "precompute": {"ms": statistics.median(pre_ms), "candidates": wl.B * wl.C,
+                               "candidates_per_s": wl.B * wl.C / (statistics.median(pre_ms) * 1e-3)},
+                "cpu_baseline": cpu, "peaks": pk}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="bf16_baseline")
+    ap.add_argument("--C", type=int, default=0, help="override candidates per user (candidate sweep)")
+    ap.add_argument("--N", type=int, default=0, help="override history length (history sweep)")
+    ap.add_argument("--B", type=int, default=0)
+    ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = synth.named_workloads()[args.workload]
+    if args.C:
+        wl = wl.replace(C=args.C)
+    if args.N:
+        wl = wl.replace(n_min=args.N, n_max=args.N)
+    if args.B:
+        wl = wl.replace(B=args.B)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

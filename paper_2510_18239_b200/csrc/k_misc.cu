@@ -1,0 +1,169 @@
+// Ragged bookkeeping, the history-embedding gather and small elementwise helpers.
+#include "lime_common.cuh"
+
+namespace lime {
+
+// ----------------------------------------------------------------------------- block-wide exclusive scan
+// One block of 1024 threads walks the array in slabs of 1024 with a running carry. B is at most a few
+// thousand users per batch, so a single block is latency-optimal (one launch, no inter-block traffic).
+template <typename F>
+__device__ __forceinline__ void block_exclusive_scan(int n, int32_t* out, F value_at) {
+  __shared__ int32_t warp_tot[32];
+  __shared__ int32_t carry_s;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int32_t v = (i < n) ? value_at(i) : 0;
+    int32_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+      int32_t w = (lane < (int)(blockDim.x >> 5)) ? warp_tot[lane] : 0;
+      int32_t wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int32_t t = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += t;
+      }
+      warp_tot[lane] = wi - w;  // exclusive prefix of warp totals
+    }
+    __syncthreads();
+    const int32_t carry = carry_s;
+    if (i < n) out[i] = carry + warp_tot[wid] + incl - v;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_s = carry + warp_tot[wid] + incl;  // last thread holds the slab total
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) out[n] = carry_s;
+}
+
+__global__ void __launch_bounds__(1024) k_offsets(const int32_t* __restrict__ len, int B, int32_t* __restrict__ off) {
+  block_exclusive_scan(B, off, [&](int i) { return max(len[i], 0); });
+}
+
+__global__ void __launch_bounds__(1024)
+k_tile_schedule(const int32_t* __restrict__ off, int B, int tile, int32_t* __restrict__ tile_start) {
+  block_exclusive_scan(B, tile_start, [&](int i) {
+    int n = off[i + 1] - off[i];
+    return n > 0 ? (n + tile - 1) / tile : 0;
+  });
+}
+
+lime_status launch_offsets(const int32_t* len, int B, int32_t* off, cudaStream_t st) {
+  ProfScope _p("k_offsets", st);
+  k_offsets<<<1, 1024, 0, st>>>(len, B, off);
+  LIME_LAUNCH_CHECK("k_offsets");
+  return LIME_OK;
+}
+
+lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st) {
+  ProfScope _p("k_tile_schedule", st);
+  k_tile_schedule<<<1, 1024, 0, st>>>(off, B, tile, tile_start);
+  LIME_LAUNCH_CHECK("k_tile_schedule");
+  return LIME_OK;
+}
+
+// ----------------------------------------------------------------------------- gather
+// out[t, :] = table[ids[t], :].  Rows are 16-byte multiples (d % 8 == 0 for both dtypes), so a row moves as
+// uint4 words: `LANES` consecutive threads own one row and each moves row_vec / LANES words, giving fully
+// coalesced 128-bit loads and stores.  Reads of hot (Zipf head) rows hit L2; the stream is write-dominated.
+template <int LANES>
+__global__ void __launch_bounds__(256)
+k_gather(const uint4* __restrict__ table, int64_t V, int row_vec, const int32_t* __restrict__ ids, int64_t total,
+         uint4* __restrict__ out, int32_t* __restrict__ dev_flag) {
+  const int rows_per_block = blockDim.x / LANES;
+  const int sub = threadIdx.x % LANES;
+  const int64_t stride = (int64_t)gridDim.x * rows_per_block;
+  for (int64_t t = (int64_t)blockIdx.x * rows_per_block + threadIdx.x / LANES; t < total; t += stride) {
+    const int32_t id = __ldg(ids + t);
+    const bool ok = id >= 0 && (int64_t)id < V;
+    uint4* dst = out + t * row_vec;
+    if (ok) {
+      const uint4* src = table + (int64_t)id * row_vec;
+      for (int v = sub; v < row_vec; v += LANES) dst[v] = __ldg(src + v);
+    } else {
+      for (int v = sub; v < row_vec; v += LANES) dst[v] = make_uint4(0, 0, 0, 0);
+      if (sub == 0 && dev_flag != nullptr) atomicMin(dev_flag, (int32_t)min(t, (int64_t)INT32_MAX));
+    }
+  }
+}
+
+lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const int32_t* ids, int64_t total,
+                          void* out, int32_t* dev_flag, cudaStream_t st) {
+  if (total == 0) return LIME_OK;
+  const int es = dtype == LIME_F32 ? 4 : 2;
+  const int row_vec = d * es / 16;
+  const int threads = 256;
+  // enough lanes per row that each thread moves 1-2 words
+  int lanes = row_vec >= 32 ? 32 : (row_vec >= 16 ? 16 : (row_vec >= 8 ? 8 : 4));
+  const int rows_per_block = threads / lanes;
+  int64_t blocks = (total + rows_per_block - 1) / rows_per_block;
+  const int64_t cap = (int64_t)kSMs * 16;
+  if (blocks > cap) blocks = cap;
+  ProfScope _p("k_gather", st);
+  const uint4* tb = (const uint4*)table;
+  uint4* o = (uint4*)out;
+  switch (lanes) {
+    case 32: k_gather<32><<<(int)blocks, threads, 0, st>>>(tb, V, row_vec, ids, total, o, dev_flag); break;
+    case 16: k_gather<16><<<(int)blocks, threads, 0, st>>>(tb, V, row_vec, ids, total, o, dev_flag); break;
+    case 8:  k_gather<8><<<(int)blocks, threads, 0, st>>>(tb, V, row_vec, ids, total, o, dev_flag); break;
+    default: k_gather<4><<<(int)blocks, threads, 0, st>>>(tb, V, row_vec, ids, total, o, dev_flag); break;
+  }
+  LIME_LAUNCH_CHECK("k_gather");
+  return LIME_OK;
+}
+
+// ----------------------------------------------------------------------------- elementwise helpers
+template <typename T>
+__global__ void k_cast_rows(const float* __restrict__ in, int64_t n, T* __restrict__ out) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    Store<T>::st(out + i, in[i]);
+}
+template <typename T>
+__global__ void k_widen(const T* __restrict__ in, int64_t n, float* __restrict__ out) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    out[i] = Store<T>::ld(in + i);
+}
+__global__ void k_axpy(const float* __restrict__ x, float* __restrict__ y, int64_t n, int zero_first) {
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    y[i] = (zero_first ? 0.0f : y[i]) + x[i];
+}
+
+static inline int ew_blocks(int64_t n) {
+  int64_t b = (n + 255) / 256;
+  const int64_t cap = (int64_t)kSMs * 8;
+  return (int)(b > cap ? cap : (b < 1 ? 1 : b));
+}
+
+lime_status launch_cast_rows(const float* in, int64_t n, void* out, int dtype, cudaStream_t st) {
+  if (n == 0) return LIME_OK;
+  ProfScope _p("k_cast_rows", st);
+  if (dtype == LIME_F32) k_cast_rows<float><<<ew_blocks(n), 256, 0, st>>>(in, n, (float*)out);
+  else k_cast_rows<__nv_bfloat16><<<ew_blocks(n), 256, 0, st>>>(in, n, (__nv_bfloat16*)out);
+  LIME_LAUNCH_CHECK("k_cast_rows");
+  return LIME_OK;
+}
+lime_status launch_widen(const void* in, int dtype, float* out, int64_t n, cudaStream_t st) {
+  if (n == 0) return LIME_OK;
+  ProfScope _p("k_widen", st);
+  if (dtype == LIME_F32) k_widen<float><<<ew_blocks(n), 256, 0, st>>>((const float*)in, n, out);
+  else k_widen<__nv_bfloat16><<<ew_blocks(n), 256, 0, st>>>((const __nv_bfloat16*)in, n, out);
+  LIME_LAUNCH_CHECK("k_widen");
+  return LIME_OK;
+}
+lime_status launch_axpy(const float* x, float* y, int64_t n, int zero_first, cudaStream_t st) {
+  if (n == 0) return LIME_OK;
+  ProfScope _p("k_axpy", st);
+  k_axpy<<<ew_blocks(n), 256, 0, st>>>(x, y, n, zero_first);
+  LIME_LAUNCH_CHECK("k_axpy");
+  return LIME_OK;
+}
+
+}  // namespace lime

@@ -1,0 +1,398 @@
+// C-ABI entry points: argument validation, workspace carving and launch sequencing.  No arithmetic of the
+// method lives here; every step runs in the kernels of this directory.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "lime_common.cuh"
+
+namespace lime {
+
+static thread_local char g_err[256] = "";
+
+lime_status cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_err, sizeof(g_err), "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
+  return LIME_CUDA_ERROR;
+}
+
+// ---- per-kernel event timing (process-wide, single-threaded use) -------------------------------------------
+struct ProfState {
+  bool open = false;
+  int capacity = 0, count = 0;
+  cudaEvent_t* ev = nullptr;      // 2 per record
+  const char** names = nullptr;
+};
+static ProfState g_prof;
+
+ProfScope::ProfScope(const char* name, cudaStream_t s) : slot(-1), st(s) {
+  if (!g_prof.open || g_prof.count >= g_prof.capacity) return;
+  slot = g_prof.count++;
+  g_prof.names[slot] = name;
+  cudaEventRecord(g_prof.ev[2 * slot], st);
+}
+ProfScope::~ProfScope() {
+  if (slot >= 0) cudaEventRecord(g_prof.ev[2 * slot + 1], st);
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+static inline int elem_size(int dtype) { return dtype == LIME_F32 ? 4 : 2; }
+
+// Tokens per work item of the link<-history attention: a power of two in [64, 1024] giving a few items per SM.
+static int pick_chunk(int64_t total_tokens) {
+  int64_t target = total_tokens / (4 * kSMs);
+  int c = 64;
+  while (c < 1024 && c < target) c <<= 1;
+  return c;
+}
+constexpr int kHistTile = 128;  // tokens per block of the history<-links attention
+
+struct Workspace {
+  // history rows, storage dtype
+  void *S, *Q, *K, *V, *U;
+  // link rows, fp32
+  float *T, *QT, *KT, *VT, *AT, *UT, *LP, *LS32;
+  int32_t *chunk_start, *tile_start;
+  float *part_m, *part_s, *part_acc;
+  int chunk, n_chunk_upper, n_tile_upper;
+  size_t bytes;
+};
+
+static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
+  Workspace w;
+  const lime_config& g = c->cfg;
+  const size_t es = elem_size(g.dtype);
+  size_t o = 0;
+  char* p = static_cast<char*>(base);
+  auto take = [&](size_t nbytes) { void* r = p ? p + o : nullptr; o += align_up(nbytes); return r; };
+  const size_t hd = (size_t)total * g.d * es, hf = (size_t)total * c->d_ff * es;
+  w.S = take(hd); w.Q = take(hd); w.K = take(hd); w.V = take(hd); w.U = take(hf);
+  const size_t ld = (size_t)B * g.ell * g.d * 4, lf = (size_t)B * g.ell * c->d_ff * 4;
+  w.T = (float*)take(ld); w.QT = (float*)take(ld); w.KT = (float*)take(ld); w.VT = (float*)take(ld);
+  w.AT = (float*)take(ld); w.UT = (float*)take(lf); w.LP = (float*)take(ld); w.LS32 = (float*)take(ld);
+  w.chunk_start = (int32_t*)take((size_t)(B + 1) * 4);
+  w.tile_start = (int32_t*)take((size_t)(B + 1) * 4);
+  w.chunk = pick_chunk(total);
+  w.n_chunk_upper = (int)((total + w.chunk - 1) / w.chunk + B);
+  w.n_tile_upper = (int)((total + kHistTile - 1) / kHistTile + B);
+  const size_t rows = (size_t)w.n_chunk_upper * g.H * g.ell;
+  w.part_m = (float*)take(rows * 4);
+  w.part_s = (float*)take(rows * 4);
+  w.part_acc = (float*)take(rows * c->d_h * 4);
+  w.bytes = o;
+  return w;
+}
+
+// One XOR layer on a carved workspace (see lime_xor_layer in lime.h for the contract).
+static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B,
+                                  int64_t total, const float* links_in, int links_shared, void* hist_out,
+                                  float* links_out, const Workspace& w, bool schedules_ready, cudaStream_t st) {
+  const lime_config& g = c->cfg;
+  lime_status s;
+  const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
+
+  // link rows: Q[T], K[T], V[T] = LN(T) W_{Q,K,V}
+  LinearArgs la{};
+  la.X = links_in; la.x_dtype = LIME_F32; la.M = link_rows; la.K = g.d; la.N = g.d;
+  la.W[0] = c->w.Wq[layer]; la.W[1] = c->w.Wk[layer]; la.W[2] = c->w.Wv[layer]; la.w_dtype = g.dtype;
+  la.Y[0] = w.QT; la.Y[1] = w.KT; la.Y[2] = w.VT; la.y_dtype = LIME_F32; la.n_out = 3;
+  la.ln = g.ln; la.ln_eps = c->ln_eps;
+  if ((s = launch_linear_simt(la, st)) != LIME_OK) return s;
+
+  // history rows: K[S], V[S] (and Q[S] when the history is updated) = LN(S) W
+  LinearArgs lh{};
+  lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
+  lh.W[0] = c->w.Wk[layer]; lh.W[1] = c->w.Wv[layer]; lh.W[2] = c->w.Wq[layer];
+  lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = hist_out ? 3 : 2;
+  lh.ln = g.ln; lh.ln_eps = c->ln_eps;
+  if ((s = launch_linear_simt(lh, st)) != LIME_OK) return s;
+
+  if (!schedules_ready) {
+    if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
+    if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
+  }
+
+  // O[T] = phi(Q[T] K[S]^T) V[S]
+  AttnLinkArgs al{};
+  al.QT = w.QT; al.qt_user_stride = links_shared ? 0 : (int64_t)g.ell * g.d;
+  al.KS = w.K; al.VS = w.V; al.s_dtype = g.dtype; al.off = off; al.B = B; al.total = total;
+  al.ell = g.ell; al.d = g.d; al.H = g.H; al.phi = g.phi; al.scale = c->attn_scale;
+  al.chunk = w.chunk; al.chunk_start = w.chunk_start; al.n_chunk_upper = w.n_chunk_upper;
+  al.part_m = w.part_m; al.part_s = w.part_s; al.part_acc = w.part_acc; al.AT = w.AT;
+  if ((s = launch_attn_link_simt(al, st)) != LIME_OK) return s;
+  if ((s = launch_attn_link_merge(al, st)) != LIME_OK) return s;
+
+  // links_out = GatedMLP(O[T])
+  const int64_t BL = (int64_t)B * g.ell;
+  if (g.gated_mlp) {
+    LinearArgs lg{};
+    lg.X = w.AT; lg.x_dtype = LIME_F32; lg.M = BL; lg.K = g.d; lg.N = c->d_ff; lg.w_dtype = g.dtype;
+    lg.W[0] = c->w.Wg[layer]; lg.W[1] = c->w.Wu[layer]; lg.Y[0] = w.UT; lg.y_dtype = LIME_F32; lg.n_out = 1; lg.glu = 1;
+    if ((s = launch_linear_simt(lg, st)) != LIME_OK) return s;
+    LinearArgs lo{};
+    lo.X = w.UT; lo.x_dtype = LIME_F32; lo.M = BL; lo.K = c->d_ff; lo.N = g.d; lo.w_dtype = g.dtype;
+    lo.W[0] = c->w.Wo[layer]; lo.Y[0] = links_out; lo.y_dtype = LIME_F32; lo.n_out = 1;
+    if ((s = launch_linear_simt(lo, st)) != LIME_OK) return s;
+  } else {
+    if ((s = launch_axpy(w.AT, links_out, BL * g.d, 1, st)) != LIME_OK) return s;
+  }
+
+  if (hist_out) {
+    // O[S] = phi(Q[S] K[T]^T) V[T], written over Q[S]; then hist_out = GatedMLP(O[S])
+    AttnHistArgs ah{};
+    ah.QS = w.Q; ah.AS = w.Q; ah.s_dtype = g.dtype; ah.KT = w.KT; ah.VT = w.VT;
+    ah.t_user_stride = links_shared ? 0 : (int64_t)g.ell * g.d;
+    ah.off = off; ah.B = B; ah.total = total; ah.ell = g.ell; ah.d = g.d; ah.H = g.H; ah.phi = g.phi;
+    ah.scale = c->attn_scale; ah.tile = kHistTile; ah.tile_start = w.tile_start; ah.n_tile_upper = w.n_tile_upper;
+    if ((s = launch_attn_hist_simt(ah, st)) != LIME_OK) return s;
+    if (g.gated_mlp) {
+      LinearArgs lg{};
+      lg.X = w.Q; lg.x_dtype = g.dtype; lg.M = total; lg.K = g.d; lg.N = c->d_ff; lg.w_dtype = g.dtype;
+      lg.W[0] = c->w.Wg[layer]; lg.W[1] = c->w.Wu[layer]; lg.Y[0] = w.U; lg.y_dtype = g.dtype; lg.n_out = 1; lg.glu = 1;
+      if ((s = launch_linear_simt(lg, st)) != LIME_OK) return s;
+      LinearArgs lo{};
+      lo.X = w.U; lo.x_dtype = g.dtype; lo.M = total; lo.K = c->d_ff; lo.N = g.d; lo.w_dtype = g.dtype;
+      lo.W[0] = c->w.Wo[layer]; lo.Y[0] = hist_out; lo.y_dtype = g.dtype; lo.n_out = 1;
+      if ((s = launch_linear_simt(lo, st)) != LIME_OK) return s;
+    } else if (total > 0) {
+      LIME_CUDA(cudaMemcpyAsync(hist_out, w.Q, (size_t)total * g.d * elem_size(g.dtype), cudaMemcpyDeviceToDevice, st));
+    }
+  }
+  return LIME_OK;
+}
+
+static lime_status check_layer_weights(const Ctx* c, int layer) {
+  if (c->cfg.gated_mlp && (!c->w.Wg[layer] || !c->w.Wu[layer] || !c->w.Wo[layer])) return LIME_INVALID_ARG;
+  return LIME_OK;
+}
+
+}  // namespace lime
+
+using namespace lime;
+
+extern "C" {
+
+const char* lime_last_cuda_error(void) { return g_err; }
+const char* lime_version(void) { return "lime-b200 0.1 sm_100a"; }
+
+lime_status lime_profile_start(int32_t capacity) {
+  if (capacity <= 0 || g_prof.open) return LIME_INVALID_ARG;
+  g_prof.ev = new (std::nothrow) cudaEvent_t[2 * (size_t)capacity];
+  g_prof.names = new (std::nothrow) const char*[capacity];
+  if (!g_prof.ev || !g_prof.names) return LIME_INVALID_ARG;
+  for (int i = 0; i < 2 * capacity; ++i) {
+    cudaError_t e = cudaEventCreate(&g_prof.ev[i]);
+    if (e != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(g_prof.ev[j]);
+      delete[] g_prof.ev; delete[] g_prof.names;
+      g_prof = ProfState();
+      return cuda_fail(e, "lime_profile_start");
+    }
+  }
+  g_prof.capacity = capacity; g_prof.count = 0; g_prof.open = true;
+  return LIME_OK;
+}
+
+lime_status lime_profile_stop(char* names, size_t names_bytes, float* ms, int32_t ms_capacity, int32_t* count) {
+  if (!g_prof.open || !count) return LIME_INVALID_ARG;
+  g_prof.open = false;
+  lime_status ret = LIME_OK;
+  const int n = g_prof.count < ms_capacity ? g_prof.count : ms_capacity;
+  size_t pos = 0;
+  if (names && names_bytes) names[0] = 0;
+  for (int i = 0; i < n; ++i) {
+    cudaError_t e = cudaEventSynchronize(g_prof.ev[2 * i + 1]);
+    float t = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]);
+    if (e != cudaSuccess) ret = cuda_fail(e, "lime_profile_stop");
+    if (ms) ms[i] = t;
+    if (names) {
+      const size_t len = strlen(g_prof.names[i]);
+      if (pos + len + 2 <= names_bytes) {
+        memcpy(names + pos, g_prof.names[i], len);
+        pos += len;
+        names[pos++] = '\n';
+        names[pos] = 0;
+      }
+    }
+  }
+  *count = g_prof.count;
+  for (int i = 0; i < 2 * g_prof.capacity; ++i) cudaEventDestroy(g_prof.ev[i]);
+  delete[] g_prof.ev; delete[] g_prof.names;
+  g_prof = ProfState();
+  return ret;
+}
+
+lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
+  if (!cfg || !out) return LIME_INVALID_ARG;
+  *out = nullptr;
+  const lime_config& g = *cfg;
+  if (g.d <= 0 || g.H <= 0 || g.ell <= 0 || g.n_layers <= 0 || g.d_ff < 0) return LIME_INVALID_ARG;
+  if (g.dtype != LIME_F32 && g.dtype != LIME_BF16) return LIME_INVALID_ARG;
+  if (g.phi != LIME_PHI_SOFTMAX && g.phi != LIME_PHI_SILU) return LIME_INVALID_ARG;
+  if (g.attn_scale < 0.f || g.cand_scale < 0.f || g.ln_eps < 0.f) return LIME_INVALID_ARG;
+  const int d_ff = g.d_ff ? g.d_ff : g.d;
+  if (g.d % 8 || d_ff % 8 || g.d % g.H || g.d / g.H > 128 || g.ell > 256 || g.n_layers > LIME_MAX_LAYERS ||
+      g.d > 1024 || d_ff > 1024)
+    return LIME_UNSUPPORTED_SHAPE;
+  // a user's K[T], V[T] (fp32) must fit in one SM's shared memory for the history<-links attention
+  if (sizeof(float) * ((size_t)2 * g.ell * (g.d + 1) + 4 * (size_t)g.d) > 200 * 1024) return LIME_UNSUPPORTED_SHAPE;
+  Ctx* c = new (std::nothrow) Ctx();
+  if (!c) return LIME_INVALID_ARG;
+  c->cfg = g;
+  memset(&c->w, 0, sizeof(c->w));
+  c->have_weights = false;
+  c->d_ff = d_ff;
+  c->d_h = g.d / g.H;
+  c->attn_scale = g.attn_scale > 0.f ? g.attn_scale : 1.0f / sqrtf((float)c->d_h);
+  c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
+  c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
+  c->keff = nullptr; c->links32 = nullptr;
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
+  if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
+  if (e != cudaSuccess) {
+    if (c->keff) cudaFree(c->keff);
+    delete c;
+    return cuda_fail(e, "lime_create");
+  }
+  *out = reinterpret_cast<lime_ctx*>(c);
+  return LIME_OK;
+}
+
+lime_status lime_destroy(lime_ctx* ctx) {
+  if (!ctx) return LIME_OK;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  cudaFree(c->keff);
+  cudaFree(c->links32);
+  delete c;
+  return LIME_OK;
+}
+
+lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream) {
+  if (!ctx || !w || !w->links) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  const lime_config& g = c->cfg;
+  if (!aligned16(w->links)) return LIME_INVALID_ARG;
+  for (int j = 0; j < g.n_layers; ++j) {
+    const void* ps[6] = {w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], w->Wo[j]};
+    for (const void* p : ps) if (!aligned16(p)) return LIME_INVALID_ARG;
+    if (g.gated_mlp && (!w->Wg[j] || !w->Wu[j] || !w->Wo[j])) return LIME_INVALID_ARG;
+  }
+  if (!aligned16(w->cand_Wq) || !aligned16(w->cand_Wk) || !aligned16(w->cand_Wv)) return LIME_INVALID_ARG;
+  c->w = *w;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  lime_status s = launch_widen(w->links, g.dtype, c->links32, (int64_t)g.ell * g.d, st);
+  if (s != LIME_OK) return s;
+  s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_scale, c->keff, st);
+  if (s != LIME_OK) return s;
+  c->have_weights = true;
+  return LIME_OK;
+}
+
+size_t lime_workspace_bytes(const lime_ctx* ctx, int32_t B, int64_t total_tokens) {
+  if (!ctx || B < 0 || total_tokens < 0 || total_tokens > 0x7fffffffLL) return 0;
+  const Ctx* c = reinterpret_cast<const Ctx*>(ctx);
+  return carve(c, nullptr, B, total_tokens).bytes + 256;
+}
+
+lime_status lime_lengths_to_offsets(lime_ctx* ctx, const int32_t* len, int32_t B, int32_t* off, void* stream) {
+  if (!ctx || !off || B < 0 || (B > 0 && !len)) return LIME_INVALID_ARG;
+  return launch_offsets(len, B, off, static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_gather_history(lime_ctx* ctx, const void* table, int64_t V, const int32_t* ids, int64_t total_tokens,
+                                void* out, int32_t* dev_flag, void* stream) {
+  if (!ctx || total_tokens < 0 || V < 0) return LIME_INVALID_ARG;
+  if (total_tokens == 0) return LIME_OK;
+  if (!table || !ids || !out || !aligned16(table) || !aligned16(out)) return LIME_INVALID_ARG;
+  const Ctx* c = reinterpret_cast<const Ctx*>(ctx);
+  return launch_gather(c->cfg.dtype, table, V, c->cfg.d, ids, total_tokens, out, dev_flag,
+                       static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb, int64_t M, void* out_w, void* stream) {
+  if (!ctx || M < 0) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_weights) return LIME_NOT_READY;
+  if (M == 0) return LIME_OK;
+  if (!cand_emb || !out_w || !aligned16(cand_emb) || !aligned16(out_w)) return LIME_INVALID_ARG;
+  return launch_precompute(c->cfg.dtype, cand_emb, M, c->cfg.d, c->cfg.ell, c->keff, out_w,
+                           static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hist_in, const int32_t* off, int32_t B,
+                           int64_t total_tokens, const float* links_in, int32_t links_shared, void* hist_out,
+                           float* links_out, void* ws, size_t ws_bytes, void* stream) {
+  if (!ctx || B < 0 || total_tokens < 0 || total_tokens > 0x7fffffffLL) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_weights) return LIME_NOT_READY;
+  if (layer < 0 || layer >= c->cfg.n_layers) return LIME_INVALID_ARG;
+  if (B == 0) return LIME_OK;
+  if (!off || !links_in || !links_out || !ws || (total_tokens > 0 && !hist_in)) return LIME_INVALID_ARG;
+  if (!aligned16(hist_in) || !aligned16(hist_out) || !aligned16(links_in) || !aligned16(links_out)) return LIME_INVALID_ARG;
+  if (check_layer_weights(c, layer) != LIME_OK) return LIME_INVALID_ARG;
+  char* base = reinterpret_cast<char*>(align_up(reinterpret_cast<uintptr_t>(ws)));
+  const size_t pad = base - static_cast<char*>(ws);
+  Workspace w = carve(c, base, B, total_tokens);
+  if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
+  return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false,
+                        static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off, int32_t B, int64_t total_tokens,
+                             const float* link_ctx, void* link_states, void* ws, size_t ws_bytes, void* stream) {
+  if (!ctx || B < 0 || total_tokens < 0 || total_tokens > 0x7fffffffLL) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_weights) return LIME_NOT_READY;
+  if (B == 0) return LIME_OK;
+  if (!off || !link_states || !ws || (total_tokens > 0 && !hist)) return LIME_INVALID_ARG;
+  if (!aligned16(hist) || !aligned16(link_ctx) || !aligned16(link_states)) return LIME_INVALID_ARG;
+  const lime_config& g = c->cfg;
+  for (int j = 0; j < g.n_layers; ++j)
+    if (check_layer_weights(c, j) != LIME_OK) return LIME_INVALID_ARG;
+  char* base = reinterpret_cast<char*>(align_up(reinterpret_cast<uintptr_t>(ws)));
+  const size_t pad = base - static_cast<char*>(ws);
+  Workspace w = carve(c, base, B, total_tokens);
+  if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  lime_status s;
+  if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
+  if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
+  const int64_t BLd = (int64_t)B * g.ell * g.d;
+  for (int j = 0; j < g.n_layers; ++j) {
+    const bool last = j == g.n_layers - 1;
+    const float* lin = j == 0 ? (link_ctx ? link_ctx : c->links32) : w.T;
+    const int shared = (j == 0 && !link_ctx) ? 1 : 0;
+    s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true, st);
+    if (s != LIME_OK) return s;
+    if ((s = launch_axpy(w.T, w.LP, BLd, j == 0, st)) != LIME_OK) return s;   // L^P = sum_j T^j  (Eq. 8)
+  }
+  // link states = L^P W_V^c (Eq. 4's values), stored as the run's dtype
+  const float* src = w.LP;
+  if (c->w.cand_Wv) {
+    LinearArgs lv{};
+    lv.X = w.LP; lv.x_dtype = LIME_F32; lv.M = (int64_t)B * g.ell; lv.K = g.d; lv.N = g.d; lv.w_dtype = g.dtype;
+    lv.W[0] = c->w.cand_Wv; lv.Y[0] = w.LS32; lv.y_dtype = LIME_F32; lv.n_out = 1;
+    if ((s = launch_linear_simt(lv, st)) != LIME_OK) return s;
+    src = w.LS32;
+  }
+  return launch_cast_rows(src, BLd, link_states, g.dtype, st);
+}
+
+lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
+                                  const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
+                                  const int32_t* cand_ids, float* logits, void* stream) {
+  if (!ctx || B < 0 || C < 0 || total_cands < 0 || total_cands > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (!cand_off && total_cands != (int64_t)B * C) return LIME_INVALID_ARG;
+  if (B == 0 || total_cands == 0) return LIME_OK;
+  if (!link_states || !cand_w || !cand_emb || !logits) return LIME_INVALID_ARG;
+  if (!aligned16(link_states) || !aligned16(cand_w) || !aligned16(cand_emb)) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  ScoreArgs a{};
+  a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->cfg.ell; a.d = c->cfg.d;
+  a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
+  return launch_score_simt(a, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

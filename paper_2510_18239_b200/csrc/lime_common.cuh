@@ -1,0 +1,152 @@
+// Shared declarations of the CUDA side of the LIME hot path (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lime.h"
+
+namespace lime {
+
+constexpr int kSMs = 148;  // B200: 2 dies x 74 SMs; grids of persistent kernels are sized from this
+
+// ----------------------------------------------------------------------------- storage helpers
+template <typename T> struct Store;
+template <> struct Store<float> {
+  static __device__ __forceinline__ float ld(const float* p) { return *p; }
+  static __device__ __forceinline__ void st(float* p, float v) { *p = v; }
+};
+template <> struct Store<__nv_bfloat16> {
+  static __device__ __forceinline__ float ld(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+  static __device__ __forceinline__ void st(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Largest b in [0, B) with start[b] <= x, for a non-decreasing start[0..B] (start[0] = 0).
+__device__ __forceinline__ int upper_user(const int32_t* __restrict__ start, int B, int x) {
+  int lo = 0, hi = B;  // invariant: start[lo] <= x, answer in [lo, hi)
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (start[mid] <= x) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
+// ----------------------------------------------------------------------------- context
+struct Ctx {
+  lime_config cfg;
+  lime_weights w;
+  bool have_weights;
+  int device;
+  float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
+  float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
+  float attn_scale, cand_scale, ln_eps;
+  int d_ff, d_h;
+};
+
+// record a CUDA error for lime_last_cuda_error(); returns LIME_CUDA_ERROR
+lime_status cuda_fail(cudaError_t e, const char* where);
+#define LIME_CUDA(expr)                                          \
+  do {                                                           \
+    cudaError_t _e = (expr);                                     \
+    if (_e != cudaSuccess) return ::lime::cuda_fail(_e, #expr);  \
+  } while (0)
+#define LIME_LAUNCH_CHECK(name)                                  \
+  do {                                                           \
+    cudaError_t _e = cudaGetLastError();                         \
+    if (_e != cudaSuccess) return ::lime::cuda_fail(_e, name);   \
+  } while (0)
+
+// ----------------------------------------------------------------------------- per-kernel event timing
+// While a profile is open (lime_profile_start .. lime_profile_stop) every launcher brackets its kernel with two
+// CUDA events on the launching stream.  Closed, a scope costs one predictable branch.
+struct ProfScope {
+  ProfScope(const char* name, cudaStream_t st);
+  ~ProfScope();
+  int slot;
+  cudaStream_t st;
+};
+
+// ----------------------------------------------------------------------------- kernel launchers (host)
+// Each returns LIME_OK or a status; all launch on `st` and never synchronise.
+
+lime_status launch_offsets(const int32_t* len, int B, int32_t* off, cudaStream_t st);
+
+lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const int32_t* ids, int64_t total,
+                          void* out, int32_t* dev_flag, cudaStream_t st);
+
+// tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B  (work list of per-user token tiles)
+lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st);
+
+// Y[r, n] (+)= epilogue( LN?(X[r, :]) . W[:, n] ) for up to three weight matrices sharing X.
+struct LinearArgs {
+  const void* X; int x_dtype;   // [M x K], lime_dtype
+  int64_t M; int K; int N;      // every W is [K x N], stored w_dtype; a NULL W means identity (K == N)
+  const void* W[3]; int w_dtype;
+  void* Y[3]; int y_dtype;      // outputs [M x N] each (ldy = N)
+  int n_out;                    // 1..3 (ignored when glu)
+  int ln; float ln_eps;         // LayerNorm rows of X first
+  int glu;                      // 1: Y[0] = SiLU(X W[0]) * (X W[1])
+  int accumulate;               // 1: Y[0] += result (y_dtype must be F32, n_out == 1)
+  const float* also_add_to;     // unused (reserved)
+};
+lime_status launch_linear_simt(const LinearArgs& a, cudaStream_t st);
+
+// link <- history attention partials: per (user, chunk of `chunk` tokens, head, link row): running max, sum,
+// un-normalised weighted values.
+struct AttnLinkArgs {
+  const float* QT; int64_t qt_user_stride;   // [B x ell x d] fp32 (stride 0: shared)
+  const void* KS; const void* VS; int s_dtype; // [total x d]
+  const int32_t* off; int B; int64_t total;
+  int ell, d, H; int phi; float scale;
+  int chunk; const int32_t* chunk_start; int n_chunk_upper;  // work list from launch_tile_schedule(tile = chunk)
+  float* part_m; float* part_s; float* part_acc;             // [n_chunk_upper x H x ell], same, [.. x d_h]
+  float* AT;                                                  // out [B x ell x d] fp32
+};
+lime_status launch_attn_link_simt(const AttnLinkArgs& a, cudaStream_t st);
+lime_status launch_attn_link_merge(const AttnLinkArgs& a, cudaStream_t st);
+
+// history <- links attention: AS[t, :] = phi(Q[S]_t K[T]^T) V[T] per head, over the ell links of t's user
+struct AttnHistArgs {
+  const void* QS; void* AS; int s_dtype;     // [total x d]; AS may alias QS
+  const float* KT; const float* VT; int64_t t_user_stride;  // [B x ell x d] fp32
+  const int32_t* off; int B; int64_t total;
+  int ell, d, H; int phi; float scale;
+  int tile; const int32_t* tile_start; int n_tile_upper;
+};
+lime_status launch_attn_hist_simt(const AttnHistArgs& a, cudaStream_t st);
+
+// out[r, :] (storage dtype) = in[r, :] fp32, optionally accumulate into acc fp32 first
+lime_status launch_cast_rows(const float* in, int64_t n, void* out, int dtype, cudaStream_t st);
+lime_status launch_axpy(const float* x, float* y, int64_t n, int zero_first, cudaStream_t st);
+lime_status launch_widen(const void* in, int dtype, float* out, int64_t n, cudaStream_t st);
+
+// candidate -> link weights: W[c, :] = softmax_l( <T_c, keff_l> )  (keff already carries cand_scale)
+lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int ell, const float* keff,
+                              void* out_w, cudaStream_t st);
+// keff = ((L Wk) Wq^T) * scale, fp32 [ell x d]
+lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, float scale,
+                        float* keff, cudaStream_t st);
+
+struct ScoreArgs {
+  const void* LS; const void* W; const void* T; int dtype;
+  int B; int ell, d;
+  const int32_t* cand_off; int C; int64_t total;
+  const int32_t* cand_ids;
+  float* logits;
+};
+lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);
+
+}  // namespace lime

@@ -1,0 +1,300 @@
+"""Parity of the CUDA library (through the C ABI) against the fp64 CPU oracle, element by element, on the same
+seeded inputs.  Tolerances: bit-exact for offsets and gathered rows; logits max-abs <= 1e-4 on the fp32 path and
+<= 2e-2 with bf16 storage (plus a relative bound against the spread of the oracle's logits, because logits of the
+synthetic workloads are small and the absolute bound alone would be vacuous)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lime_oracle as O
+from paper_2510_18239_b200 import synth
+from tests import lime_helpers as Hh
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+REL_BF16 = 6e-2     # max-abs error / std(oracle logits), bf16 storage of history rows through n layers
+
+
+def _lib():
+    from paper_2510_18239_b200 import binding
+    return binding
+
+
+def small(dtype, **kw):
+    base = dict(name="small", B=3, n_min=40, n_max=40, d=32, H=2, ell=8, n_layers=2, C=24, dtype=dtype, V=500,
+                zipf_s=1.1, table_std=1.0, link_std=1.0)
+    base.update(kw)
+    return synth.Workload(**base)
+
+
+# ----------------------------------------------------------------------------- offsets / gather: bit exact
+@pytest.mark.parametrize("B", [0, 1, 2, 31, 1000, 1024, 1025, 5000])
+def test_offsets_bit_exact(B):
+    Bd = _lib()
+    lime = Bd.Lime(32, 2, 8, 1, dtype=Bd.LIME_F32)
+    r = np.random.default_rng(B)
+    lengths = r.integers(0, 4097, size=B).astype(np.int32)
+    if B > 4:
+        lengths[r.integers(0, B, size=B // 4)] = 0
+    off = lime.lengths_to_offsets(torch.from_numpy(lengths).cuda())
+    want = O.lengths_to_offsets(lengths)
+    assert off.dtype == torch.int32
+    assert np.array_equal(off.cpu().numpy().astype(np.int64), want)
+
+
+@pytest.mark.parametrize("dtype,d", [(synth.F32, 8), (synth.F32, 64), (synth.BF16, 8), (synth.BF16, 128),
+                                     (synth.BF16, 256), (synth.BF16, 1024)])
+def test_gather_bit_exact_and_bad_ids(dtype, d):
+    Bd = _lib()
+    V, n = 777, 5001
+    lime = Bd.Lime(d, 1 if d < 128 else d // 128, 4, 1, dtype=Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16)
+    table = synth.normal_storage(1, "t", (V, d), 1.0, dtype)
+    ids = synth.zipf_ids(1, "i", n, V, 1.1)
+    ids[17] = -1
+    ids[4000] = V
+    ids[4500] = 2 ** 31 - 1
+    flag = torch.full((1,), 2 ** 31 - 1, dtype=torch.int32, device="cuda")
+    out = lime.gather_history(Bd.to_device(table, dtype), torch.from_numpy(ids).cuda(), flag)
+    got = out.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == synth.BF16 else out.cpu().numpy()
+    ok = (ids >= 0) & (ids < V)
+    want = np.zeros((n, d), dtype=table.dtype)
+    want[ok] = O.gather_history(table, ids[ok])
+    assert np.array_equal(got.view(np.uint8), want.view(np.uint8))
+    assert int(flag.item()) == 17
+    # empty gather is legal
+    assert lime.gather_history(Bd.to_device(table, dtype), torch.zeros(0, dtype=torch.int32, device="cuda")).shape == (0, d)
+
+
+# ----------------------------------------------------------------------------- candidate side
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("ell,d,M", [(1, 8, 5), (8, 64, 300), (32, 128, 1000), (64, 256, 257), (33, 40, 64)])
+@pytest.mark.parametrize("proj", [False, True])
+def test_precompute_matches_oracle(dtype, ell, d, M, proj):
+    Bd = _lib()
+    dt = Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16
+    lime = Bd.Lime(d, max(1, d // 128), ell, 1, dtype=dt, gated_mlp=False)
+    links = synth.normal_storage(2, "l", (ell, d), 1.0, dtype)
+    T = synth.normal_storage(2, "c", (M, d), 1.0, dtype)
+    cand_np = {}
+    if proj:
+        cand_np = {"Wq": synth.normal_storage(2, "cq", (d, d), d ** -0.5, dtype),
+                   "Wk": synth.normal_storage(2, "ck", (d, d), d ** -0.5, dtype)}
+    lime.set_weights(Bd.to_device(links, dtype), [{}], {k: Bd.to_device(v, dtype) for k, v in cand_np.items()})
+    W = lime.precompute_candidate_links(Bd.to_device(T, dtype))
+    cfg = O.OracleConfig(d=d, H=1, ell=ell, n_layers=1)
+    want = O.precompute_candidate_links(synth.storage_to_f64(T, dtype), synth.storage_to_f64(links, dtype), cfg,
+                                        synth.storage_to_f64(cand_np["Wq"], dtype) if proj else None,
+                                        synth.storage_to_f64(cand_np["Wk"], dtype) if proj else None)
+    got = Hh.to_f64(W)
+    assert got.shape == want.shape
+    tol = 2e-5 if dtype == synth.F32 else 4e-3          # bf16 output rounding: 2^-9 relative on weights <= 1
+    assert np.abs(got - want).max() <= tol
+    assert np.abs(got.sum(axis=1) - 1.0).max() <= (1e-5 if dtype == synth.F32 else 1e-2)
+
+
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("B,C,ell,d", [(1, 1, 1, 8), (3, 50, 8, 64), (2, 300, 32, 128), (2, 129, 64, 256), (5, 77, 33, 40)])
+def test_score_matches_oracle_on_same_inputs(dtype, B, C, ell, d):
+    Bd = _lib()
+    dt = Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16
+    lime = Bd.Lime(d, max(1, d // 128), ell, 1, dtype=dt, gated_mlp=False)
+    LS = synth.normal_storage(3, "ls", (B, ell, d), 1.0, dtype)
+    T = synth.normal_storage(3, "t", (B * C, d), 1.0, dtype)
+    Wraw = np.abs(synth.storage_to_f64(synth.normal_storage(3, "w", (B * C, ell), 1.0, synth.F32), synth.F32)) + 0.01
+    Wst = synth.to_storage(Wraw / Wraw.sum(axis=1, keepdims=True), dtype)
+    logits = lime.score_candidates(Bd.to_device(LS, dtype), Bd.to_device(Wst, dtype), Bd.to_device(T, dtype), C=C)
+    W64, T64, LS64 = (synth.storage_to_f64(x, dtype) for x in (Wst, T, LS))
+    want = np.concatenate([O.score_candidates(W64[b * C:(b + 1) * C], LS64[b], T64[b * C:(b + 1) * C]) for b in range(B)])
+    err = np.abs(Hh.to_f64(logits) - want).max()
+    assert err <= 1e-4 * max(1.0, np.abs(want).max()), err      # same stored inputs: only fp32 accumulation differs
+
+
+def test_score_ragged_offsets_ids_and_empty_users():
+    Bd = _lib()
+    dtype, ell, d = synth.BF16, 16, 64
+    lime = Bd.Lime(d, 1, ell, 1, dtype=Bd.LIME_BF16, gated_mlp=False)
+    counts = np.array([5, 0, 130, 1, 0, 64, 63], dtype=np.int64)
+    B, total = counts.size, int(counts.sum())
+    off = O.lengths_to_offsets(counts)
+    corpus = 400
+    LS = synth.normal_storage(4, "ls", (B, ell, d), 1.0, dtype)
+    Tc = synth.normal_storage(4, "t", (corpus, d), 1.0, dtype)
+    Wc = synth.to_storage(O.softmax_rows(np.random.default_rng(4).normal(size=(corpus, ell))), dtype)
+    ids = synth.uniform_ids(4, "ids", total, corpus)
+    logits = lime.score_candidates(Bd.to_device(LS, dtype), Bd.to_device(Wc, dtype), Bd.to_device(Tc, dtype),
+                                   cand_off=torch.from_numpy(off.astype(np.int32)).cuda(),
+                                   cand_ids=torch.from_numpy(ids).cuda(), total_cands=total)
+    W64, T64, LS64 = (synth.storage_to_f64(x, dtype) for x in (Wc, Tc, LS))
+    want = np.concatenate([O.score_candidates(W64[ids[off[b]:off[b + 1]]], LS64[b], T64[ids[off[b]:off[b + 1]]])
+                           for b in range(B)])
+    assert np.abs(Hh.to_f64(logits) - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+
+
+# ----------------------------------------------------------------------------- XOR layer and encode
+def _oracle_batch(wl, inp, phi=O.SOFTMAX, ln=True, gated_mlp=True, cand_np=None):
+    cfg = Hh.oracle_config(wl, phi=phi, ln=ln, gated_mlp=gated_mlp)
+    layers = Hh.oracle_layers(inp, wl, gated_mlp)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(inp["lengths"])
+    cand_w = None
+    if cand_np:
+        cand_w = {k + "_c": synth.storage_to_f64(v, wl.dtype) for k, v in cand_np.items()}
+    logits, LS = [], []
+    for b in range(wl.B):
+        lg, ls, _ = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg, cand_w=cand_w)
+        logits.append(lg)
+        LS.append(ls)
+    return np.concatenate(logits), np.stack(LS)
+
+
+def _check_logits(got, want, dtype):
+    err = np.abs(got - want).max()
+    spread = want.std()
+    if dtype == synth.F32:
+        assert err <= TOL_F32, (err, spread)
+    else:
+        # 2e-2 absolute for logits of order one or smaller; stress cases with larger logits scale it by max|logit|
+        # (bf16 storage carries 2^-9 relative rounding per stored value)
+        assert err <= TOL_BF16 * max(1.0, np.abs(want).max()), (err, spread)
+        assert err <= REL_BF16 * max(spread, 1e-6) + 1e-4, (err, spread)
+
+
+@pytest.mark.parametrize("N", [0, 1, 2, 31, 63, 64, 65, 127, 129, 300])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_xor_layer_history_lengths(N, dtype):
+    """One XOR layer, both directions, against the oracle for history lengths around the tile sizes."""
+    Bd = _lib()
+    wl = small(dtype, B=2, n_min=N, n_max=N, n_layers=1, ell=8, d=32, H=2)
+    inp = synth.make_inputs(wl, seed=N)
+    dev = Hh.DeviceBatch(wl, inp)
+    L = dev.lime
+    off = L.lengths_to_offsets(dev.lengths)
+    hist = L.gather_history(dev.table, dev.hist_ids)
+    links32 = dev.links.float().contiguous()
+    hist_out = torch.empty_like(hist)
+    links_out = torch.empty((wl.B, wl.ell, wl.d), dtype=torch.float32, device="cuda")
+    Bd.lime_xor_layer(L.ctx, 0, hist, off, wl.B, links32, True, hist_out, links_out, L.workspace(wl.B, hist.shape[0]))
+    cfg = Hh.oracle_config(wl)
+    lw = Hh.oracle_layers(inp, wl)[0]
+    table64, links64 = synth.storage_to_f64(inp["table"], dtype), synth.storage_to_f64(inp["links"], dtype)
+    tol = 2e-4 if dtype == synth.F32 else 4e-2
+    for b in range(wl.B):
+        E = O.gather_history(table64, inp["hist_ids"][b * N:(b + 1) * N])
+        S_next, T_next = O.xor_layer(E, links64, lw, cfg)
+        assert np.abs(Hh.to_f64(links_out[b]) - T_next).max() <= tol
+        if N:
+            assert np.abs(Hh.to_f64(hist_out[b * N:(b + 1) * N]) - S_next).max() <= tol
+    if N == 0:
+        assert torch.count_nonzero(links_out).item() == 0
+
+
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("ell,d,H", [(1, 8, 1), (8, 64, 2), (32, 128, 4), (64, 128, 4), (64, 256, 8), (33, 40, 5)])
+def test_encode_and_score_shapes(dtype, ell, d, H):
+    wl = small(dtype, B=3, n_min=5, n_max=150, d=d, H=H, ell=ell, n_layers=2, C=40, V=700, table_std=0.5)
+    inp = synth.make_inputs(wl, seed=ell + d)
+    out = Hh.DeviceBatch(wl, inp).run()
+    want_logits, want_ls = _oracle_batch(wl, inp)
+    assert np.array_equal(out["off"].cpu().numpy(), O.lengths_to_offsets(inp["lengths"]))
+    ls_tol = 2e-4 if dtype == synth.F32 else 5e-2
+    assert np.abs(Hh.to_f64(out["link_states"]) - want_ls).max() <= ls_tol * max(1.0, np.abs(want_ls).max())
+    _check_logits(Hh.to_f64(out["logits"]), want_logits, dtype)
+
+
+@pytest.mark.parametrize("phi,ln,gated", [(O.SOFTMAX, False, False), (O.SILU, True, True), (O.SILU, False, False),
+                                          (O.SOFTMAX, True, False)])
+def test_profiles_core_and_silu(phi, ln, gated):
+    Bd = _lib()
+    wl = small(synth.F32, B=2, n_min=0, n_max=90, n_layers=3, table_std=0.7)
+    inp = synth.make_inputs(wl, seed=5)
+    inp["lengths"][0] = 0                                   # an empty history in the batch
+    inp["hist_ids"] = inp["hist_ids"][: int(inp["lengths"].sum())]
+    dev = Hh.DeviceBatch(wl, inp, phi=Bd.LIME_PHI_SILU if phi == O.SILU else Bd.LIME_PHI_SOFTMAX, ln=ln, gated_mlp=gated)
+    out = dev.run()
+    want_logits, want_ls = _oracle_batch(wl, inp, phi=phi, ln=ln, gated_mlp=gated)
+    assert np.abs(Hh.to_f64(out["link_states"]) - want_ls).max() <= 2e-4 * max(1.0, np.abs(want_ls).max())
+    _check_logits(Hh.to_f64(out["logits"]), want_logits, synth.F32)
+
+
+def test_candidate_side_projections_and_link_context():
+    Bd = _lib()
+    wl = small(synth.F32, B=2, n_min=30, n_max=60, n_layers=2)
+    inp = synth.make_inputs(wl, seed=6)
+    cand_np = {k: synth.normal_storage(6, "c" + k, (wl.d, wl.d), wl.d ** -0.5, wl.dtype) for k in ("Wq", "Wk", "Wv")}
+    out = Hh.DeviceBatch(wl, inp, cand=cand_np).run()
+    want_logits, want_ls = _oracle_batch(wl, inp, cand_np=cand_np)
+    assert np.abs(Hh.to_f64(out["link_states"]) - want_ls).max() <= 2e-4 * max(1.0, np.abs(want_ls).max())
+    _check_logits(Hh.to_f64(out["logits"]), want_logits, synth.F32)
+    # per-user contextualised links L^C (Eq. 2's output) instead of the shared L
+    dev = Hh.DeviceBatch(wl, inp)
+    LC = synth.normal_storage(7, "lc", (wl.B, wl.ell, wl.d), 1.0, synth.F32)
+    off = dev.lime.lengths_to_offsets(dev.lengths)
+    hist = dev.lime.gather_history(dev.table, dev.hist_ids)
+    ls = dev.lime.encode_user(hist, off, torch.from_numpy(LC).cuda())
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    offh = O.lengths_to_offsets(inp["lengths"])
+    for b in range(wl.B):
+        E = O.gather_history(table64, inp["hist_ids"][offh[b]:offh[b + 1]])
+        LP, _ = O.encode_user(E, LC[b].astype(np.float64), layers, cfg)
+        assert np.abs(Hh.to_f64(ls[b]) - LP).max() <= 2e-4 * max(1.0, np.abs(LP).max())
+
+
+# ----------------------------------------------------------------------------- the named workloads
+def test_config1_tiny_fp32_full_parity():
+    wl = synth.named_workloads()["tiny_fp32"]
+    inp = synth.make_inputs(wl, seed=0)
+    out = Hh.DeviceBatch(wl, inp).run()
+    want_logits, want_ls = _oracle_batch(wl, inp)
+    got = Hh.to_f64(out["logits"])
+    assert got.shape == (wl.B * wl.C,)
+    _check_logits(got, want_logits, synth.F32)
+    assert np.abs(got - want_logits).max() <= 1e-3 * want_logits.std()     # fp32 path is far inside 1e-4
+
+
+def _sampled_parity(wl, seed, users, n_cand=64):
+    inp = synth.make_inputs(wl, seed=seed)
+    out = Hh.DeviceBatch(wl, inp).run()
+    torch.cuda.synchronize()
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(inp["lengths"])
+    assert np.array_equal(out["off"].cpu().numpy(), off)
+    # gathered rows: bit exact on a sample of tokens
+    r = np.random.default_rng(seed)
+    tok = r.integers(0, off[-1], size=512)
+    got_rows = out["hist"][torch.from_numpy(tok).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got_rows, inp["table"][inp["hist_ids"][tok]])
+    got_all, want_all = [], []
+    for b in users:
+        rows = np.sort(r.choice(wl.C, size=min(n_cand, wl.C), replace=False))
+        lg, _, _ = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg, cand_rows=rows)
+        got_all.append(Hh.to_f64(out["logits"][b * wl.C:(b + 1) * wl.C])[rows])
+        want_all.append(lg)
+    _check_logits(np.concatenate(got_all), np.concatenate(want_all), wl.dtype)
+
+
+def test_config2_bf16_baseline_sampled():
+    wl = synth.named_workloads()["bf16_baseline"]
+    _sampled_parity(wl, seed=0, users=[0, 1, 100, 255])
+
+
+def test_config3_candidate_sweep_sampled():
+    wl = synth.named_workloads()["candidate_sweep"].replace(C=4096)
+    _sampled_parity(wl, seed=0, users=[0, 63])
+
+
+def test_config4_long_history_sampled():
+    wl = synth.named_workloads()["long_history"].replace(n_min=4096, n_max=4096, B=8)
+    _sampled_parity(wl, seed=0, users=[0, 7])
+
+
+def test_config5_production_ragged_sampled():
+    wl = synth.named_workloads()["production_ragged"].replace(B=32, V=200_000, C=512)
+    inp_len = synth.history_lengths(0, wl.B, wl.n_min, wl.n_max)
+    users = [int(np.argmin(inp_len)), int(np.argmax(inp_len))]
+    _sampled_parity(wl, seed=0, users=users)
