@@ -76,15 +76,24 @@ def model_for(name, models):
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
+    """nvidia-smi sampled every 50 ms; start() early (it takes a second to come up), then mark() the timed region."""
+
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
+        self.t0 = self.t1 = None
+
+    def mark(self, begin: bool):
+        if begin:
+            self.t0 = time.time()
+        else:
+            self.t1 = time.time()
 
     def start(self):
         q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except Exception:
@@ -92,7 +101,7 @@ class ClockSampler:
 
     def _read(self):
         for ln in self.proc.stdout:
-            self.lines.append(ln.strip())
+            self.lines.append((time.time(), ln.strip()))
 
     def stop(self):
         if not self.proc:
@@ -103,7 +112,10 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for ln in self.lines:
+        inside = [ln for (ts, ln) in self.lines if self.t0 is None or (self.t0 - 0.05 <= ts <= (self.t1 or ts) + 0.1)]
+        if not inside:
+            inside = [ln for (_, ln) in self.lines[-3:]]
+        for ln in inside:
             p = [x.strip() for x in ln.split(",")]
             if len(p) < 7:
                 continue
@@ -254,22 +266,23 @@ def run_ours(args, wl):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        step(i)
-    barrier()
-
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for i in range(args.warmup):
+        step(i)
+    barrier()
     cap = 64 * args.steps + 64
     Bd.lime_profile_start(cap)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
+    sampler.mark(True)
     ev[0].record()
     for i in range(args.steps):
         step(i)
         ev[i + 1].record()
     torch.cuda.synchronize()
+    sampler.mark(False)
     barrier()
     records, launches = Bd.lime_profile_stop(cap)
     clocks = sampler.stop() if rank == 0 else None
@@ -385,8 +398,8 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="bf16_baseline")
     ap.add_argument("--C", type=int, default=0, help="override candidates per user (candidate sweep)")

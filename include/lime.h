@@ -47,7 +47,8 @@ typedef enum lime_status {
   LIME_UNSUPPORTED_SHAPE = 2,   /* d, H, ell, d_ff outside what the kernels are built for                */
   LIME_WORKSPACE_TOO_SMALL = 3,
   LIME_CUDA_ERROR = 4,          /* a CUDA runtime/driver call failed; see lime_last_cuda_error()         */
-  LIME_NOT_READY = 5            /* weights not set                                                        */
+  LIME_NOT_READY = 5,           /* weights not set                                                        */
+  LIME_DEVICE_TIMEOUT = 6       /* a bounded wait inside a kernel gave up; outputs of that call are invalid */
 } lime_status;
 
 typedef enum lime_dtype { LIME_F32 = 0, LIME_BF16 = 1 } lime_dtype;
@@ -150,6 +151,13 @@ LIME_API lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int
 LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
                                   const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
                                   const int32_t* cand_ids, float* logits, void* stream);
+
+/* Health check.  The tensor-core kernels synchronise their warps through mbarriers with bounded waits (2 s); a wait
+ * that gives up records a non-zero code in a device word of the context and the kernel exits cleanly (no trap, no
+ * hang) with its outputs undefined.  lime_device_status SYNCHRONISES the device (a blocking copy of that word),
+ * writes the code to *code (host), clears it, and returns LIME_DEVICE_TIMEOUT if it was set, else LIME_OK.
+ * The paper has no counterpart; codes: 1 producer, 2-3 MMA issuer, 4 epilogue waits of the scorer. */
+LIME_API lime_status lime_device_status(lime_ctx* ctx, int32_t* code);
 
 /* Per-kernel timing for benchmarks (the paper reports latency only end to end, App. F; this breaks a call down).
  * Between lime_profile_start(capacity) and lime_profile_stop every kernel this library launches is bracketed by two

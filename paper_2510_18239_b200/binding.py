@@ -46,7 +46,7 @@ class lime_weights(ctypes.Structure):
 
 EXPORTS = ("lime_create", "lime_destroy", "lime_set_weights", "lime_workspace_bytes", "lime_lengths_to_offsets",
            "lime_gather_history", "lime_precompute_candidate_links", "lime_xor_layer", "lime_encode_user",
-           "lime_score_candidates", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
+           "lime_score_candidates", "lime_device_status", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
            "lime_version")
 
 _lib_handle = None
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_xor_layer.argtypes = [vp, i32, vp, vp, i32, i64, vp, i32, vp, vp, vp, sz, vp]
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.lime_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     lib.lime_profile_start.argtypes = [i32]
     lib.lime_profile_stop.argtypes = [ctypes.c_char_p, sz, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
     for name in EXPORTS:
@@ -166,6 +167,15 @@ def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: t
     _check(load_library().lime_score_candidates(ctx, _ptr(link_states), B, _ptr(cand_w), _ptr(cand_emb), _ptr(cand_off),
                                                 C, total_cands, _ptr(cand_ids), _ptr(logits), _stream()),
            "lime_score_candidates")
+
+
+def lime_device_status(ctx: int) -> int:
+    """Synchronises; raises LimeError(LIME_DEVICE_TIMEOUT) if a bounded in-kernel wait gave up, else returns 0."""
+    code = ctypes.c_int32(0)
+    st = load_library().lime_device_status(ctx, ctypes.byref(code))
+    if st != 0:
+        raise LimeError(st, "lime_device_status", f"wait code {code.value}")
+    return int(code.value)
 
 
 def lime_profile_start(capacity: int = 4096) -> None:

@@ -247,12 +247,16 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->attn_scale = g.attn_scale > 0.f ? g.attn_scale : 1.0f / sqrtf((float)c->d_h);
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
-  c->keff = nullptr; c->links32 = nullptr;
+  c->keff = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
+  if (e == cudaSuccess) e = cudaMalloc(&c->dev_err, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemset(c->dev_err, 0, sizeof(int));
   if (e != cudaSuccess) {
     if (c->keff) cudaFree(c->keff);
+    if (c->links32) cudaFree(c->links32);
+    if (c->dev_err) cudaFree(c->dev_err);
     delete c;
     return cuda_fail(e, "lime_create");
   }
@@ -265,6 +269,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   Ctx* c = reinterpret_cast<Ctx*>(ctx);
   cudaFree(c->keff);
   cudaFree(c->links32);
+  cudaFree(c->dev_err);
   delete c;
   return LIME_OK;
 }
@@ -392,7 +397,21 @@ lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_
   ScoreArgs a{};
   a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->cfg.ell; a.d = c->cfg.d;
   a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
+  if (score_tc_supported(a)) return launch_score_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   return launch_score_simt(a, static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_device_status(lime_ctx* ctx, int32_t* code) {
+  if (!ctx || !code) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  int v = 0;
+  LIME_CUDA(cudaMemcpy(&v, c->dev_err, sizeof(int), cudaMemcpyDeviceToHost));
+  *code = v;
+  if (v != 0) {
+    LIME_CUDA(cudaMemset(c->dev_err, 0, sizeof(int)));
+    return LIME_DEVICE_TIMEOUT;
+  }
+  return LIME_OK;
 }
 
 }  // extern "C"

@@ -52,6 +52,7 @@ struct Ctx {
   int device;
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
+  int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
   int d_ff, d_h;
 };
@@ -148,5 +149,8 @@ struct ScoreArgs {
   float* logits;
 };
 lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);
+// bf16 streaming scorer on tcgen05 tensor cores (fixed C per user, dense rows, ell in {16,32,64,128}, d % 64 == 0)
+bool score_tc_supported(const ScoreArgs& a);
+lime_status launch_score_tc(const ScoreArgs& a, int* err, cudaStream_t st);
 
 }  // namespace lime

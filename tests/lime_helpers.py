@@ -67,6 +67,7 @@ class DeviceBatch:
         cand = L.gather_history(self.table, self.cand_ids)
         W = L.precompute_candidate_links(cand)
         logits = L.score_candidates(ls, W, cand, C=self.wl.C)
+        self.Bd.lime_device_status(L.ctx)      # synchronises; raises if a bounded in-kernel wait gave up
         return dict(off=off, hist=hist, link_states=ls, cand=cand, W=W, logits=logits)
 
 

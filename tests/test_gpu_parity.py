@@ -95,7 +95,9 @@ def test_precompute_matches_oracle(dtype, ell, d, M, proj):
 
 
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
-@pytest.mark.parametrize("B,C,ell,d", [(1, 1, 1, 8), (3, 50, 8, 64), (2, 300, 32, 128), (2, 129, 64, 256), (5, 77, 33, 40)])
+@pytest.mark.parametrize("B,C,ell,d", [(1, 1, 1, 8), (3, 50, 8, 64), (2, 300, 32, 128), (2, 129, 64, 256), (5, 77, 33, 40),
+                                       (1, 128, 16, 64), (7, 1, 32, 128), (3, 2048, 32, 128), (160, 130, 64, 128),
+                                       (2, 1000, 128, 64), (300, 16, 32, 128)])
 def test_score_matches_oracle_on_same_inputs(dtype, B, C, ell, d):
     Bd = _lib()
     dt = Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16
@@ -105,6 +107,7 @@ def test_score_matches_oracle_on_same_inputs(dtype, B, C, ell, d):
     Wraw = np.abs(synth.storage_to_f64(synth.normal_storage(3, "w", (B * C, ell), 1.0, synth.F32), synth.F32)) + 0.01
     Wst = synth.to_storage(Wraw / Wraw.sum(axis=1, keepdims=True), dtype)
     logits = lime.score_candidates(Bd.to_device(LS, dtype), Bd.to_device(Wst, dtype), Bd.to_device(T, dtype), C=C)
+    assert Bd.lime_device_status(lime.ctx) == 0
     W64, T64, LS64 = (synth.storage_to_f64(x, dtype) for x in (Wst, T, LS))
     want = np.concatenate([O.score_candidates(W64[b * C:(b + 1) * C], LS64[b], T64[b * C:(b + 1) * C]) for b in range(B)])
     err = np.abs(Hh.to_f64(logits) - want).max()
