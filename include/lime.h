@@ -48,7 +48,8 @@ typedef enum lime_status {
   LIME_WORKSPACE_TOO_SMALL = 3,
   LIME_CUDA_ERROR = 4,          /* a CUDA runtime/driver call failed; see lime_last_cuda_error()         */
   LIME_NOT_READY = 5,           /* weights not set                                                        */
-  LIME_DEVICE_TIMEOUT = 6       /* a bounded wait inside a kernel gave up; outputs of that call are invalid */
+  LIME_DEVICE_TIMEOUT = 6,      /* a bounded wait inside a kernel gave up; outputs of that call are invalid */
+  LIME_EXCEEDS_STATIC_SCRATCH = 7 /* shape too large for the fixed scratch of an allocation-free entry point    */
 } lime_status;
 
 typedef enum lime_dtype { LIME_F32 = 0, LIME_BF16 = 1 } lime_dtype;
@@ -151,6 +152,28 @@ LIME_API lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int
 LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
                                   const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
                                   const int32_t* cand_ids, float* logits, void* stream);
+
+/* Allocation-free precompute (the paper has no counterpart: this exists for hosts that must not allocate).
+ * Same result as lime_create + lime_set_weights + lime_precompute_candidate_links, for callers that cannot call
+ * cudaMalloc at this point - a serving process whose device memory pool is frozen after start-up, or code running
+ * inside a framework that owns the allocator - and therefore cannot create a context.  It takes the shape and the
+ * weight pointers directly (dtype, d, ell, cand_scale as in lime_config; links [ell x d]; cand_Wq / cand_Wk [d x d]
+ * or NULL; cand_emb [M x d]; out_w [M x ell]; all device pointers of `dtype`, 16-byte aligned) and calls no
+ * cudaMalloc, cudaFree or other allocating routine.  Its scratch (the effective link keys and one intermediate,
+ * 2 * ell * d floats) lives in a fixed device array inside the library, 2 * LIME_NOALLOC_MAX_LINK_ELEMS floats
+ * (128 KB) that every GPU loading the library holds until the process exits.
+ *   - ell * d > LIME_NOALLOC_MAX_LINK_ELEMS returns LIME_EXCEEDS_STATIC_SCRATCH (and sets the error text); nothing
+ *     is launched.
+ *   - The first call on each device looks up the array's device address (with that device current); make that
+ *     first call before starting any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents; every call rewrites all of the part
+ *     it uses before reading it, so nothing needs clearing.  Two calls that overlap on the GPU (different streams,
+ *     or different threads) race on it: serialise them. */
+#define LIME_NOALLOC_MAX_LINK_ELEMS 16384
+LIME_API lime_status lime_precompute_candidate_links_noalloc(int32_t dtype, int32_t d, int32_t ell, float cand_scale,
+                                                             const void* links, const void* cand_Wq,
+                                                             const void* cand_Wk, const void* cand_emb, int64_t M,
+                                                             void* out_w, void* stream);
 
 /* Health check.  The tensor-core kernels synchronise their warps through mbarriers with bounded waits (2 s); a wait
  * that gives up records a non-zero code in a device word of the context and the kernel exits cleanly (no trap, no

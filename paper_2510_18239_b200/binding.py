@@ -17,7 +17,7 @@ LIME_MAX_LAYERS = 16
 LIME_F32, LIME_BF16 = 0, 1
 LIME_PHI_SOFTMAX, LIME_PHI_SILU = 0, 1
 _STATUS = {0: "LIME_OK", 1: "LIME_INVALID_ARG", 2: "LIME_UNSUPPORTED_SHAPE", 3: "LIME_WORKSPACE_TOO_SMALL",
-           4: "LIME_CUDA_ERROR", 5: "LIME_NOT_READY", 6: "LIME_DEVICE_TIMEOUT"}
+           4: "LIME_CUDA_ERROR", 5: "LIME_NOT_READY", 6: "LIME_DEVICE_TIMEOUT", 7: "LIME_EXCEEDS_STATIC_SCRATCH"}
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblime_b200.so")
 
@@ -46,7 +46,7 @@ class lime_weights(ctypes.Structure):
 
 EXPORTS = ("lime_create", "lime_destroy", "lime_set_weights", "lime_workspace_bytes", "lime_lengths_to_offsets",
            "lime_gather_history", "lime_precompute_candidate_links", "lime_xor_layer", "lime_encode_user",
-           "lime_score_candidates", "lime_device_status", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
+           "lime_score_candidates", "lime_precompute_candidate_links_noalloc", "lime_device_status", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
            "lime_version")
 
 _lib_handle = None
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_xor_layer.argtypes = [vp, i32, vp, vp, i32, i64, vp, i32, vp, vp, vp, sz, vp]
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.lime_precompute_candidate_links_noalloc.argtypes = [i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, i64, vp, vp]
     lib.lime_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     lib.lime_profile_start.argtypes = [i32]
     lib.lime_profile_stop.argtypes = [ctypes.c_char_p, sz, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
@@ -167,6 +168,19 @@ def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: t
     _check(load_library().lime_score_candidates(ctx, _ptr(link_states), B, _ptr(cand_w), _ptr(cand_emb), _ptr(cand_off),
                                                 C, total_cands, _ptr(cand_ids), _ptr(logits), _stream()),
            "lime_score_candidates")
+
+
+def lime_precompute_candidate_links_noalloc(dtype: int, d: int, ell: int, cand_scale: float, links: torch.Tensor,
+                                            cand_Wq: Optional[torch.Tensor], cand_Wk: Optional[torch.Tensor],
+                                            cand_emb: torch.Tensor, out_w: torch.Tensor) -> None:
+    """Context-free, allocation-free precompute for callers that may not allocate device memory; the caller passes
+    every buffer, including the output.  Raises LimeError(LIME_EXCEEDS_STATIC_SCRATCH) if ell * d is too large."""
+    st = load_library().lime_precompute_candidate_links_noalloc(dtype, d, ell, cand_scale, _ptr(links), _ptr(cand_Wq),
+                                                                _ptr(cand_Wk), _ptr(cand_emb), cand_emb.shape[0],
+                                                                _ptr(out_w), _stream())
+    if st != 0:
+        raise LimeError(st, "lime_precompute_candidate_links_noalloc",
+                        load_library().lime_last_cuda_error().decode() if st in (4, 7) else "")
 
 
 def lime_device_status(ctx: int) -> int:
