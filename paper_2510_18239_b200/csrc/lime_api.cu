@@ -54,6 +54,9 @@ struct Workspace {
   float *T, *QT, *KT, *VT, *AT, *UT, *LP, *LS32;
   int32_t *chunk_start, *tile_start;
   float *part_m, *part_s, *part_acc;
+  // tensor-core path: folded link-side operands (bf16) and their row sums
+  void *Q2, *K2, *G2t, *U2t;
+  float *cQ, *cK;
   int chunk, n_chunk_upper, n_tile_upper;
   size_t bytes;
 };
@@ -79,6 +82,10 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.part_m = (float*)take(rows * 4);
   w.part_s = (float*)take(rows * 4);
   w.part_acc = (float*)take(rows * c->d_h * 4);
+  const size_t HL = (size_t)g.H * g.ell;
+  w.Q2 = take((size_t)B * HL * g.d * 2); w.K2 = take((size_t)B * HL * g.d * 2);
+  w.G2t = take((size_t)B * c->d_ff * HL * 2); w.U2t = take((size_t)B * c->d_ff * HL * 2);
+  w.cQ = (float*)take((size_t)B * HL * 4); w.cK = (float*)take((size_t)B * HL * 4);
   w.bytes = o;
   return w;
 }
@@ -103,7 +110,9 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   LinearArgs lh{};
   lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
   lh.W[0] = c->w.Wk[layer]; lh.W[1] = c->w.Wv[layer]; lh.W[2] = c->w.Wq[layer];
-  lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = hist_out ? 3 : 2;
+  const bool tc_hist = hist_out && c->WoT[layer] &&
+                       hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
+  lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = (hist_out && !tc_hist) ? 3 : 2;
   lh.ln = g.ln; lh.ln_eps = c->ln_eps;
   if ((s = launch_linear_simt(lh, st)) != LIME_OK) return s;
 
@@ -137,7 +146,21 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
     if ((s = launch_axpy(w.AT, links_out, BL * g.d, 1, st)) != LIME_OK) return s;
   }
 
-  if (hist_out) {
+  if (tc_hist) {
+    // tensor-core path: fold W_Q into the link keys and W_g / W_u into the link values, then one fused kernel
+    LinkPrepArgs lp{};
+    lp.QT = w.QT; lp.KT = w.KT; lp.VT = w.VT; lp.users = links_shared ? 1 : B; lp.shared = links_shared;
+    lp.ell = g.ell; lp.d = g.d; lp.H = g.H; lp.f = c->d_ff; lp.scale = c->attn_scale;
+    lp.Wq = c->w.Wq[layer]; lp.Wk = c->w.Wk[layer]; lp.Wg = c->w.Wg[layer]; lp.Wu = c->w.Wu[layer];
+    lp.K2 = w.K2; lp.cK = w.cK; lp.G2t = w.G2t; lp.U2t = w.U2t;
+    if ((s = launch_link_prep(lp, st)) != LIME_OK) return s;
+    HistUpdateArgs hu{};
+    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
+    hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
+    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = g.ln; hu.ln_eps = c->ln_eps;
+    hu.err = c->dev_err;
+    if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
+  } else if (hist_out) {
     // O[S] = phi(Q[S] K[T]^T) V[T], written over Q[S]; then hist_out = GatedMLP(O[S])
     AttnHistArgs ah{};
     ah.QS = w.Q; ah.AS = w.Q; ah.s_dtype = g.dtype; ah.KT = w.KT; ah.VT = w.VT;
@@ -248,6 +271,7 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
@@ -270,6 +294,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   cudaFree(c->keff);
   cudaFree(c->links32);
   cudaFree(c->dev_err);
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) cudaFree(c->WoT[j]);
   delete c;
   return LIME_OK;
 }
@@ -291,6 +316,13 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
   if (s != LIME_OK) return s;
   s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_scale, c->keff, st);
   if (s != LIME_OK) return s;
+  // tensor-core path: W_o as a K-major B operand ([d x d_ff], contraction index contiguous)
+  if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) {
+    for (int j = 0; j < g.n_layers; ++j) {
+      if (!c->WoT[j]) LIME_CUDA(cudaMalloc(&c->WoT[j], (size_t)g.d * c->d_ff * 2));
+      if ((s = launch_transpose_bf16(w->Wo[j], c->d_ff, g.d, c->WoT[j], st)) != LIME_OK) return s;
+    }
+  }
   c->have_weights = true;
   return LIME_OK;
 }

@@ -52,6 +52,7 @@ struct Ctx {
   int device;
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
+  void* WoT[LIME_MAX_LAYERS];  // W_o transposed [d x d_ff] bf16 per layer (tensor-core path), or NULL
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
   int d_ff, d_h;
@@ -152,5 +153,28 @@ lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);
 // bf16 streaming scorer on tcgen05 tensor cores (fixed C per user, dense rows, ell in {16,32,64,128}, d % 64 == 0)
 bool score_tc_supported(const ScoreArgs& a);
 lime_status launch_score_tc(const ScoreArgs& a, int* err, cudaStream_t st);
+
+// ---- tensor-core XOR layer (bf16, d = d_ff = 128, H * ell = 128) ----------------------------------------------
+struct LinkPrepArgs {
+  const float *QT, *KT, *VT;     // [users x ell x d] fp32 projected link rows (users = 1 when shared)
+  int users, shared, ell, d, H, f;
+  float scale;
+  const void *Wq, *Wk, *Wg, *Wu; // layer weights (bf16; Wq / Wk may be NULL = identity)
+  void* Q2; float* cQ;           // out (nullable pair): folded link queries [users x H*ell x d] bf16 and their row sums
+  void* K2; float* cK;           // out (nullable group): folded link keys, row sums,
+  void* G2t; void* U2t;          //   folded gate / up operands [users x f x H*ell] bf16
+};
+lime_status launch_link_prep(const LinkPrepArgs& a, cudaStream_t st);
+lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, cudaStream_t st);
+
+struct HistUpdateArgs {
+  const void* hist_in; void* hist_out; int64_t total;
+  const void *K2, *G2t, *U2t; const float* cK; const void* WoT;   // WoT [d x f] bf16 (W_o transposed)
+  const int32_t* off; const int32_t* tile_start; int B, n_tile_upper;
+  int ell, shared, ln; float ln_eps;
+  int* err;
+};
+bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
+lime_status launch_hist_update_tc(const HistUpdateArgs& a, cudaStream_t st);
 
 }  // namespace lime

@@ -194,6 +194,47 @@ def test_xor_layer_history_lengths(N, dtype):
         assert torch.count_nonzero(links_out).item() == 0
 
 
+@pytest.mark.parametrize("ell,H", [(32, 4), (16, 8), (64, 2)])
+@pytest.mark.parametrize("lengths", [[1], [127, 128, 129], [0, 300, 5, 0, 1000], [256] * 40])
+@pytest.mark.parametrize("shared_links", [True, False])
+def test_xor_layer_tensor_core_path(ell, H, lengths, shared_links):
+    """One XOR layer at the shapes the fused tensor-core kernels serve (bf16, d = 128, H * ell = 128), ragged
+    histories around the 128-token tile, shared and per-user link rows."""
+    Bd = _lib()
+    B = len(lengths)
+    wl = small(synth.BF16, B=B, n_min=0, n_max=1, d=128, H=H, ell=ell, n_layers=1, V=3000, table_std=0.05)
+    inp = synth.make_inputs(wl, seed=ell + B)
+    inp["lengths"] = np.asarray(lengths, dtype=np.int32)
+    total = int(sum(lengths))
+    inp["hist_ids"] = synth.zipf_ids(3, "h", total, wl.V, 1.1)
+    dev = Hh.DeviceBatch(wl, inp)
+    L = dev.lime
+    off = L.lengths_to_offsets(dev.lengths)
+    hist = L.gather_history(dev.table, dev.hist_ids)
+    if shared_links:
+        links_np = synth.storage_to_f64(inp["links"], wl.dtype)[None].repeat(B, axis=0)
+        links32 = dev.links.float().contiguous()
+    else:
+        links_np = np.random.default_rng(9).normal(size=(B, ell, wl.d)).astype(np.float32).astype(np.float64)
+        links32 = torch.from_numpy(links_np.astype(np.float32)).cuda()
+    hist_out = torch.zeros_like(hist)
+    links_out = torch.empty((B, ell, wl.d), dtype=torch.float32, device="cuda")
+    Bd.lime_xor_layer(L.ctx, 0, hist, off, B, links32, shared_links, hist_out if total else None, links_out,
+                      L.workspace(B, total))
+    assert Bd.lime_device_status(L.ctx) == 0
+    cfg = Hh.oracle_config(wl)
+    lw = Hh.oracle_layers(inp, wl)[0]
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    offh = O.lengths_to_offsets(lengths)
+    for b in range(B):
+        E = O.gather_history(table64, inp["hist_ids"][offh[b]:offh[b + 1]])
+        S_next, T_next = O.xor_layer(E, links_np[b], lw, cfg)
+        assert np.abs(Hh.to_f64(links_out[b]) - T_next).max() <= 4e-2 * max(1.0, np.abs(T_next).max())
+        if lengths[b]:
+            got = Hh.to_f64(hist_out[offh[b]:offh[b + 1]])
+            assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
+
+
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 @pytest.mark.parametrize("ell,d,H", [(1, 8, 1), (8, 64, 2), (32, 128, 4), (64, 128, 4), (64, 256, 8), (33, 40, 5)])
 def test_encode_and_score_shapes(dtype, ell, d, H):
