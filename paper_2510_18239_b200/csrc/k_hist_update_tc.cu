@@ -43,6 +43,19 @@ struct HistUpdateParams {
 // address of 16-byte chunk `c` (0..7) of row r inside a 128B-swizzled [rows x 64 bf16] sub-tile
 __device__ __forceinline__ uint32_t sw128_chunk(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
 
+// user of tile t, cached: the tile ranges of consecutive tiles are the same user most of the time
+struct TileUser {
+  int b = -1, lo = 0, hi = 0;
+  __device__ __forceinline__ int of(const int32_t* __restrict__ tile_start, int B, int t) {
+    if (t < lo || t >= hi) {
+      b = upper_user(tile_start, B, t);
+      lo = tile_start[b];
+      hi = tile_start[b + 1];
+    }
+    return b;
+  }
+};
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -101,8 +114,9 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + HU_OFF_WO + kb * HU_SUB, &tmWo, kb * 64, 0, wo_full, pol_keep);
       int cur_user = -1, seg = 0, it = 0;
       bool ok = true;
+      TileUser tu;
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int b = upper_user(p.tile_start, p.B, t);
+        const int b = tu.of(p.tile_start, p.B, t);
         if (b != cur_user) {
           if (seg > 0 && !mbar_wait(uops_empty, (uint32_t)(seg - 1) & 1u, p.err, 11)) { ok = false; break; }
           const int urow = p.shared ? 0 : b;
@@ -117,7 +131,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
         const int s = it & 1;
         if (!mbar_wait(&x_empty[s], ((uint32_t)(it >> 1) & 1u) ^ 1u, p.err, 12)) { ok = false; break; }
-        const int row0 = p.off[b] + (t - p.tile_start[b]) * HU_TILE;
+        const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
         mbar_arrive_expect_tx(&x_full[s], HU_X_STAGE);
         for (int kb = 0; kb < 2; ++kb)
           tma_load_2d_hint(smem + HU_OFF_X + s * HU_X_STAGE + kb * HU_SUB, &tmX, kb * 64, row0, &x_full[s], pol_stream);
@@ -136,8 +150,9 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       const uint32_t sbase = smem_u32(smem);
       int cur_user = -1, seg = 0, it = 0;
       bool ok = mbar_wait(wo_full, 0, p.err, 21);
+      TileUser tu;
       for (int t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int b = upper_user(p.tile_start, p.B, t);
+        const int b = tu.of(p.tile_start, p.B, t);
         const uint32_t tp = (uint32_t)it & 1u;
         if (b != cur_user) {
           if (!mbar_wait(uops_full, (uint32_t)seg & 1u, p.err, 22)) break;
@@ -166,7 +181,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
         mma_commit(gu_full);
         // the user's operands are free once the last tile of the segment has issued its MMAs on them
-        const bool last_of_user = (t + 1 == t_end) || (upper_user(p.tile_start, p.B, t + 1) != b);
+        const bool last_of_user = (t + 1 == t_end) || (t + 1 >= tu.hi);
         if (last_of_user) mma_commit(uops_empty);
         // 5. S' = U . W_o
         if (!mbar_wait(u_ready, tp, p.err, 25)) break;
@@ -189,8 +204,9 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     float* ck_s = reinterpret_cast<float*>(smem + HU_OFF_CK) + (warp - 2) * HU_HL;   // this warp's own copy
     int cur_user = -1, it = 0;
     constexpr int H = HU_HL / ELL;
+    TileUser tu;
     for (int t = t_begin; t < t_end; ++t, ++it) {
-      const int b = upper_user(p.tile_start, p.B, t);
+      const int b = tu.of(p.tile_start, p.B, t);
       const uint32_t tp = (uint32_t)it & 1u;
       const int s = it & 1;
       if (b != cur_user) {
@@ -199,7 +215,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         __syncwarp();
         cur_user = b;
       }
-      const int row0 = p.off[b] + (t - p.tile_start[b]) * HU_TILE;
+      const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
       const bool valid = row0 + (int)r < p.off[b + 1];
       // LayerNorm statistics of this thread's token from the staged tile (two passes, rotated chunk order)
       if (!mbar_wait(&x_full[s], (uint32_t)(it >> 1) & 1u, p.err, 31)) break;

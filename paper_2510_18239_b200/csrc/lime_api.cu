@@ -76,12 +76,14 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.chunk_start = (int32_t*)take((size_t)(B + 1) * 4);
   w.tile_start = (int32_t*)take((size_t)(B + 1) * 4);
   w.chunk = pick_chunk(total);
+  const bool tc_link = link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi);
+  if (tc_link && w.chunk < 512) w.chunk = 512;   // one CTA per chunk: amortise its set-up over >= 4 token tiles
   w.n_chunk_upper = (int)((total + w.chunk - 1) / w.chunk + B);
   w.n_tile_upper = (int)((total + kHistTile - 1) / kHistTile + B);
   const size_t rows = (size_t)w.n_chunk_upper * g.H * g.ell;
   w.part_m = (float*)take(rows * 4);
   w.part_s = (float*)take(rows * 4);
-  w.part_acc = (float*)take(rows * c->d_h * 4);
+  w.part_acc = (float*)take(rows * (tc_link ? g.d : c->d_h) * 4);
   const size_t HL = (size_t)g.H * g.ell;
   w.Q2 = take((size_t)B * HL * g.d * 2); w.K2 = take((size_t)B * HL * g.d * 2);
   w.G2t = take((size_t)B * c->d_ff * HL * 2); w.U2t = take((size_t)B * c->d_ff * HL * 2);
@@ -106,22 +108,47 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   la.ln = g.ln; la.ln_eps = c->ln_eps;
   if ((s = launch_linear_simt(la, st)) != LIME_OK) return s;
 
-  // history rows: K[S], V[S] (and Q[S] when the history is updated) = LN(S) W
-  LinearArgs lh{};
-  lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
-  lh.W[0] = c->w.Wk[layer]; lh.W[1] = c->w.Wv[layer]; lh.W[2] = c->w.Wq[layer];
+  // history rows: K[S], V[S], Q[S] = LN(S) W, only for the directions that run on CUDA cores (the tensor-core
+  // kernels contract against the stored history and never materialise them)
   const bool tc_hist = hist_out && c->WoT[layer] &&
                        hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
-  lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = (hist_out && !tc_hist) ? 3 : 2;
-  lh.ln = g.ln; lh.ln_eps = c->ln_eps;
-  if ((s = launch_linear_simt(lh, st)) != LIME_OK) return s;
+  const bool tc_link = link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi);
+  {
+    LinearArgs lh{};
+    lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
+    lh.ln = g.ln; lh.ln_eps = c->ln_eps;
+    int n = 0;
+    if (!tc_link) { lh.W[n] = c->w.Wk[layer]; lh.Y[n++] = w.K; lh.W[n] = c->w.Wv[layer]; lh.Y[n++] = w.V; }
+    if (hist_out && !tc_hist) { lh.W[n] = c->w.Wq[layer]; lh.Y[n++] = w.Q; }
+    lh.n_out = n;
+    if (n > 0 && (s = launch_linear_simt(lh, st)) != LIME_OK) return s;
+  }
 
   if (!schedules_ready) {
     if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
     if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
   }
 
+  if (tc_link || tc_hist) {
+    // fold the history-side projections into the link rows (see k_link_prep.cu)
+    LinkPrepArgs lp{};
+    lp.QT = w.QT; lp.KT = w.KT; lp.VT = w.VT; lp.users = links_shared ? 1 : B; lp.shared = links_shared;
+    lp.ell = g.ell; lp.d = g.d; lp.H = g.H; lp.f = c->d_ff; lp.scale = c->attn_scale;
+    lp.Wq = c->w.Wq[layer]; lp.Wk = c->w.Wk[layer]; lp.Wg = c->w.Wg[layer]; lp.Wu = c->w.Wu[layer];
+    if (tc_link) { lp.Q2 = w.Q2; lp.cQ = w.cQ; }
+    if (tc_hist) { lp.K2 = w.K2; lp.cK = w.cK; lp.G2t = w.G2t; lp.U2t = w.U2t; }
+    if ((s = launch_link_prep(lp, st)) != LIME_OK) return s;
+  }
+
   // O[T] = phi(Q[T] K[S]^T) V[S]
+  if (tc_link) {
+    LinkAttnArgs la2{};
+    la2.hist = hist_in; la2.total = total; la2.Q2 = w.Q2; la2.cQ = w.cQ; la2.Wv = c->w.Wv[layer]; la2.off = off;
+    la2.chunk_start = w.chunk_start; la2.B = B; la2.chunk = w.chunk; la2.n_chunk_upper = w.n_chunk_upper;
+    la2.ell = g.ell; la2.d = g.d; la2.H = g.H; la2.shared = links_shared; la2.ln = g.ln; la2.ln_eps = c->ln_eps;
+    la2.part_m = w.part_m; la2.part_s = w.part_s; la2.part_acc = w.part_acc; la2.AT = w.AT; la2.err = c->dev_err;
+    if ((s = launch_link_attn_tc(la2, st)) != LIME_OK) return s;
+  } else {
   AttnLinkArgs al{};
   al.QT = w.QT; al.qt_user_stride = links_shared ? 0 : (int64_t)g.ell * g.d;
   al.KS = w.K; al.VS = w.V; al.s_dtype = g.dtype; al.off = off; al.B = B; al.total = total;
@@ -130,6 +157,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   al.part_m = w.part_m; al.part_s = w.part_s; al.part_acc = w.part_acc; al.AT = w.AT;
   if ((s = launch_attn_link_simt(al, st)) != LIME_OK) return s;
   if ((s = launch_attn_link_merge(al, st)) != LIME_OK) return s;
+  }
 
   // links_out = GatedMLP(O[T])
   const int64_t BL = (int64_t)B * g.ell;
@@ -147,13 +175,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   }
 
   if (tc_hist) {
-    // tensor-core path: fold W_Q into the link keys and W_g / W_u into the link values, then one fused kernel
-    LinkPrepArgs lp{};
-    lp.QT = w.QT; lp.KT = w.KT; lp.VT = w.VT; lp.users = links_shared ? 1 : B; lp.shared = links_shared;
-    lp.ell = g.ell; lp.d = g.d; lp.H = g.H; lp.f = c->d_ff; lp.scale = c->attn_scale;
-    lp.Wq = c->w.Wq[layer]; lp.Wk = c->w.Wk[layer]; lp.Wg = c->w.Wg[layer]; lp.Wu = c->w.Wu[layer];
-    lp.K2 = w.K2; lp.cK = w.cK; lp.G2t = w.G2t; lp.U2t = w.U2t;
-    if ((s = launch_link_prep(lp, st)) != LIME_OK) return s;
+    // scores, per-head softmax, value mix and GatedMLP in one fused tensor-core kernel
     HistUpdateArgs hu{};
     hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
     hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;

@@ -167,6 +167,19 @@ struct LinkPrepArgs {
 lime_status launch_link_prep(const LinkPrepArgs& a, cudaStream_t st);
 lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, cudaStream_t st);
 
+struct LinkAttnArgs {
+  const void* hist; int64_t total;          // [total x d] bf16
+  const void* Q2; const float* cQ;          // folded link queries [users x H*ell x d] bf16 and their row sums
+  const void* Wv;                           // [d x d] bf16 or NULL (identity)
+  const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
+  int ell, d, H, shared, ln; float ln_eps;
+  float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
+  float* AT;                                // out [B x ell x d] fp32
+  int* err;
+};
+bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi);
+lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st);
+
 struct HistUpdateArgs {
   const void* hist_in; void* hist_out; int64_t total;
   const void *K2, *G2t, *U2t; const float* cK; const void* WoT;   // WoT [d x f] bf16 (W_o transposed)

@@ -153,6 +153,19 @@ __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, float (&v)[16]) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const float (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15]))
+      : "memory");
+}
+
 // ----------------------------------------------------------------------------- tcgen05.mma (bf16 x bf16 -> fp32)
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both operands K-major unless flagged, M x N tile.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_major = false, bool b_mn_major = false) {
@@ -175,6 +188,20 @@ __device__ __forceinline__ uint64_t make_sdesc_k_sw128(uint32_t smem_addr) {
   d |= (uint64_t)(1024 >> 4) << 32;                    // stride byte offset: 8 rows x 128 B
   d |= (uint64_t)1 << 46;                              // descriptor version (Blackwell)
   d |= (uint64_t)2 << 61;                              // layout: 128-byte swizzle
+  return d;
+}
+
+// Shared-memory matrix descriptor for an MN-major bf16 operand held as [K rows x 64 MN elements] 128B-swizzled
+// sub-tiles (a row-major [K x MN] matrix loaded by TMA in 64-column boxes): 8 K-rows are 1024 B apart (stride
+// offset), the next 64 MN elements live `mn_chunk_bytes` further (leading offset = distance between sub-tiles).
+// Stepping K by 16 rows advances the start address by 2048 bytes.
+__device__ __forceinline__ uint64_t make_sdesc_mn_sw128(uint32_t smem_addr, uint32_t mn_chunk_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((mn_chunk_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
   return d;
 }
 

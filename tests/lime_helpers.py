@@ -12,8 +12,9 @@ from paper_2510_18239_b200 import synth
 LAYER_KEYS = ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")
 
 
-def oracle_config(wl: synth.Workload, phi=O.SOFTMAX, ln=True, gated_mlp=True) -> O.OracleConfig:
-    return O.OracleConfig(d=wl.d, H=wl.H, ell=wl.ell, n_layers=wl.n_layers, phi=phi, ln=ln, gated_mlp=gated_mlp)
+def oracle_config(wl: synth.Workload, phi=O.SOFTMAX, ln=True, gated_mlp=True, attn_scale=None) -> O.OracleConfig:
+    return O.OracleConfig(d=wl.d, H=wl.H, ell=wl.ell, n_layers=wl.n_layers, phi=phi, ln=ln, gated_mlp=gated_mlp,
+                          attn_scale=attn_scale)
 
 
 def oracle_layers(inp: Dict[str, np.ndarray], wl: synth.Workload, gated_mlp=True) -> List[Dict[str, np.ndarray]]:
@@ -41,13 +42,15 @@ def oracle_user(inp, wl, b: int, off: np.ndarray, table64: np.ndarray, links64: 
 class DeviceBatch:
     """Device-side mirror of one synthetic batch plus a configured library context."""
 
-    def __init__(self, wl: synth.Workload, inp: Dict[str, np.ndarray], phi=0, ln=True, gated_mlp=True, cand=None):
+    def __init__(self, wl: synth.Workload, inp: Dict[str, np.ndarray], phi=0, ln=True, gated_mlp=True, cand=None,
+                 attn_scale=0.0):
         import torch
         from paper_2510_18239_b200 import binding as Bd
         self.Bd = Bd
         self.wl = wl
         dt = Bd.LIME_F32 if wl.dtype == synth.F32 else Bd.LIME_BF16
-        self.lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff, phi=phi, ln=ln, gated_mlp=gated_mlp)
+        self.lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff, phi=phi, ln=ln, gated_mlp=gated_mlp,
+                            attn_scale=attn_scale)
         self.table = Bd.to_device(inp["table"], wl.dtype)
         self.links = Bd.to_device(inp["links"], wl.dtype)
         self.w = {k: Bd.to_device(inp[k], wl.dtype) for k in LAYER_KEYS}

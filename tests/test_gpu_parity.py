@@ -235,6 +235,49 @@ def test_xor_layer_tensor_core_path(ell, H, lengths, shared_links):
             assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
 
 
+@pytest.mark.parametrize("ln", [True, False])
+def test_link_attention_running_max_is_raised_mid_history(ln):
+    """History whose later tiles score far higher than the first one for half of the link rows (the second 128 tokens
+    are the negated first 128, so every score flips sign), with a large softmax scale: the online softmax of the
+    tensor-core kernel must raise its reference maximum and rescale its accumulator, and still match the oracle."""
+    Bd = _lib()
+    n, d, ell, H = 128 * 3 + 37, 128, 32, 4
+    wl = small(synth.BF16, B=2, n_min=n, n_max=n, d=d, H=H, ell=ell, n_layers=1, V=2 * n, table_std=1.0)
+    inp = synth.make_inputs(wl, seed=21)
+    r = np.random.default_rng(21)
+    base = r.normal(size=(1, d))
+    rows = np.concatenate([base + 0.05 * r.normal(size=(128, d)), -base + 0.05 * r.normal(size=(128, d)),
+                           r.normal(size=(n - 256, d))])
+    table = np.concatenate([rows, rows[::-1]])                # user 1 sees the same tokens in reverse order
+    inp["table"] = synth.to_storage(table, synth.BF16)
+    inp["hist_ids"] = np.arange(2 * n, dtype=np.int32)
+    scale = 1.0
+    dev = Hh.DeviceBatch(wl, inp, ln=ln, attn_scale=scale)
+    L = dev.lime
+    off = L.lengths_to_offsets(dev.lengths)
+    hist = L.gather_history(dev.table, dev.hist_ids)
+    links_out = torch.empty((2, ell, d), dtype=torch.float32, device="cuda")
+    Bd.lime_xor_layer(L.ctx, 0, hist, off, 2, dev.links.float().contiguous(), True, None, links_out, L.workspace(2, 2 * n))
+    assert Bd.lime_device_status(L.ctx) == 0
+    cfg = Hh.oracle_config(wl, ln=ln, attn_scale=scale)
+    lw = Hh.oracle_layers(inp, wl)[0]
+    table64, links64 = synth.storage_to_f64(inp["table"], synth.BF16), synth.storage_to_f64(inp["links"], synth.BF16)
+    outs = []
+    for b in range(2):
+        E = table64[b * n:(b + 1) * n]
+        # the flip really produces large jumps of the per-row maximum between the first two tiles
+        Xn = O.layer_norm(E) if ln else E
+        sc = ((O.layer_norm(links64) if ln else links64) @ lw["Wq"])[:, :d // H] @ (Xn @ lw["Wk"])[:, :d // H].T * scale
+        if b == 0:
+            assert (sc[:, 128:256].max(axis=1) - sc[:, :128].max(axis=1) > 8).sum() >= 4
+        _, T_next = O.xor_layer(E, links64, lw, cfg, need_history=False)
+        got = Hh.to_f64(links_out[b])
+        assert np.abs(got - T_next).max() <= 4e-2 * max(1.0, np.abs(T_next).max()), np.abs(got - T_next).max()
+        outs.append(got)
+    # same multiset of tokens in another order: same result up to rounding (no positional term)
+    assert np.abs(outs[0] - outs[1]).max() <= 4e-2 * max(1.0, np.abs(outs[0]).max())
+
+
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 @pytest.mark.parametrize("ell,d,H", [(1, 8, 1), (8, 64, 2), (32, 128, 4), (64, 128, 4), (64, 256, 8), (33, 40, 5)])
 def test_encode_and_score_shapes(dtype, ell, d, H):
