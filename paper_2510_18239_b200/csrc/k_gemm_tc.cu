@@ -1,0 +1,238 @@
+// Link-row algebra of the XOR layers as tcgen05 GEMMs (bf16 in, fp32 accumulate in TMEM).
+//
+// The B*ell link rows of a layer go through three dense contractions per layer (weights folded once at set-up,
+// see k_link_prep.cu):
+//   PREP   LN(T) [rows x d] . Wprep [d x 4*H*128]  -> folded queries Q2, folded keys K2 (+ their row sums) and the
+//          folded gate / up operands G2t, U2t that the streaming kernels contract against the history (Eq. 7)
+//   GLU    Ohat [rows x H*d] . [Mvg | Mvu] [H*d x 2f] -> SiLU(gate) * up      (value projection + GatedMLP input, Eq. 5)
+//   F32    U [rows x f] . W_o [f x d]               -> link rows of the layer's output, fp32  (Eq. 8 terms)
+// One CTA per 128-row x N_TILE output tile: warp 0 streams K blocks of A and B with TMA through a stage ring,
+// warp 1 issues the MMAs, warps 2-5 (one thread per output row = TMEM lane) run the epilogue.
+#include "lime_common.cuh"
+#include "tc_common.cuh"
+
+namespace lime {
+
+constexpr int GM_THREADS = 192, GM_MAX_STAGES = 6;
+constexpr uint32_t GM_SUB = 128 * 128;    // [128 rows x 64 bf16]
+
+enum { GM_EPI_PREP = 0, GM_EPI_GLU = 1, GM_EPI_F32 = 2 };
+
+struct GemmParams {
+  int64_t M;            // valid rows of A / C
+  int kblocks;          // K / 64
+  int stages;
+  // PREP
+  int ell, H, shared_rows;          // rows are (user, link): user = row / ell
+  __nv_bfloat16 *Q2, *K2, *G2t, *U2t;
+  float *cQ, *cK;
+  // GLU: out bf16 [M x 128]; F32: out fp32 [M x n_total]
+  void* out;
+  int n_total;
+  int* err;
+};
+
+__device__ __forceinline__ uint32_t gm_pack(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int EPI, int NT>
+__global__ void __launch_bounds__(GM_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+  using namespace tc;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (threadIdx.x == 0) atomicCAS(p.err, 0, 92);
+    return;
+  }
+  constexpr uint32_t B_SUB = (uint32_t)NT * 128;
+  constexpr uint32_t STAGE = GM_SUB + B_SUB;
+  const int S = p.stages;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + GM_MAX_STAGES;
+  uint64_t* acc_full = bars + 2 * GM_MAX_STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * GM_MAX_STAGES + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 128, nt = blockIdx.y;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(acc_full, 1);
+    fence_barrier_init();
+    prefetch_tmap(&tmA); prefetch_tmap(&tmB);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, NT); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_last();
+      bool ok = true;
+      int kb = 0;
+      for (; kb < p.kblocks; ++kb) {
+        const int s = kb % S;
+        if (!mbar_wait(&empty[s], ((uint32_t)(kb / S) & 1u) ^ 1u, p.err, 71)) { ok = false; break; }
+        uint8_t* st = smem + (size_t)s * STAGE;
+        mbar_arrive_expect_tx(&full[s], STAGE);
+        tma_load_2d_hint(st, &tmA, kb * 64, m0, &full[s], pol);
+        tma_load_2d_hint(st + GM_SUB, &tmB, kb * 64, nt * NT, &full[s], pol);
+        if (NT == 256) tma_load_2d_hint(st + GM_SUB + GM_SUB, &tmB, kb * 64, nt * NT + 128, &full[s], pol);
+      }
+      if (!ok || *(volatile int*)p.err != 0)
+        for (int j = 0; j < kb && j < S; ++j) mbar_wait_quiet(&full[(kb - 1 - j) % S], (uint32_t)((kb - 1 - j) / S) & 1u);
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(128, NT);
+      const uint32_t sbase = smem_u32(smem);
+      bool ok = true;
+      for (int kb = 0; kb < p.kblocks && ok; ++kb) {
+        const int s = kb % S;
+        if (!mbar_wait(&full[s], (uint32_t)(kb / S) & 1u, p.err, 72)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_bf16_ss(tmem_base, make_sdesc_k_sw128(sbase + s * STAGE + k * 32),
+                      make_sdesc_k_sw128(sbase + s * STAGE + GM_SUB + k * 32), idesc, (kb | k) != 0);
+        mma_commit(&empty[s]);
+      }
+      if (ok) mma_commit(acc_full);
+    }
+  } else {
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const int64_t row = (int64_t)m0 + r;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    if (mbar_wait(acc_full, 0, p.err, 73)) {
+      tc_fence_after();
+      const bool valid = row < p.M;
+      if (EPI == GM_EPI_PREP) {
+        // n-tile -> (segment, head); row -> (user, link)
+        const int seg = nt / p.H, h = nt % p.H;
+        const int64_t u = row / p.ell;
+        const int l = (int)(row % p.ell);
+        const int HL = p.H * p.ell;
+        if (seg < 2) {
+          __nv_bfloat16* dst = (seg == 0 ? p.Q2 : p.K2) + ((u * HL) + h * p.ell + l) * 128;
+          float rs = 0.f;
+#pragma unroll
+          for (int c = 0; c < 128; c += 16) {
+            float v[16];
+            tmem_ld_32x16(lane_addr + c, v);
+            tmem_wait_ld();
+            uint4 o0, o1;
+            o0.x = gm_pack(v[0], v[1]); o0.y = gm_pack(v[2], v[3]); o0.z = gm_pack(v[4], v[5]); o0.w = gm_pack(v[6], v[7]);
+            o1.x = gm_pack(v[8], v[9]); o1.y = gm_pack(v[10], v[11]); o1.z = gm_pack(v[12], v[13]); o1.w = gm_pack(v[14], v[15]);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) rs += __bfloat162float(__float2bfloat16_rn(v[j]));   // sum of what is stored
+            if (valid) {
+              *reinterpret_cast<uint4*>(dst + c) = o0;
+              *reinterpret_cast<uint4*>(dst + c + 8) = o1;
+            }
+          }
+          if (valid) (seg == 0 ? p.cQ : p.cK)[u * HL + h * p.ell + l] = rs;
+        } else {
+          // transposed store: out[user][n][(h,l)]
+          __nv_bfloat16* dst = (seg == 2 ? p.G2t : p.U2t) + u * 128 * HL + h * p.ell + l;
+#pragma unroll
+          for (int c = 0; c < 128; c += 16) {
+            float v[16];
+            tmem_ld_32x16(lane_addr + c, v);
+            tmem_wait_ld();
+            if (valid) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) dst[(int64_t)(c + j) * HL] = __float2bfloat16_rn(v[j]);
+            }
+          }
+        }
+      } else if (EPI == GM_EPI_GLU) {
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row * 128;
+#pragma unroll
+        for (int c = 0; c < 128; c += 16) {
+          float g[16], u[16];
+          tmem_ld_32x16(lane_addr + c, g);
+          tmem_ld_32x16(lane_addr + 128 + c, u);
+          tmem_wait_ld();
+          float y[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) y[j] = silu_f(g[j]) * u[j];
+          if (valid) {
+            uint4 o0, o1;
+            o0.x = gm_pack(y[0], y[1]); o0.y = gm_pack(y[2], y[3]); o0.z = gm_pack(y[4], y[5]); o0.w = gm_pack(y[6], y[7]);
+            o1.x = gm_pack(y[8], y[9]); o1.y = gm_pack(y[10], y[11]); o1.z = gm_pack(y[12], y[13]); o1.w = gm_pack(y[14], y[15]);
+            *reinterpret_cast<uint4*>(dst + c) = o0;
+            *reinterpret_cast<uint4*>(dst + c + 8) = o1;
+          }
+        }
+      } else {
+        float* dst = reinterpret_cast<float*>(p.out) + row * p.n_total + (int64_t)nt * NT;
+#pragma unroll
+        for (int c = 0; c < NT; c += 16) {
+          float v[16];
+          tmem_ld_32x16(lane_addr + c, v);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(dst + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, NT);
+  }
+}
+
+template <int EPI, int NT>
+static lime_status launch_gemm(const void* A, int64_t M, int K, const void* Bt, int n_rows_b, int n_tiles, GemmParams p,
+                               const char* name, cudaStream_t st) {
+  if (M == 0) return LIME_OK;
+  CUtensorMap tmA, tmB;
+  if (!make_tmap_bf16_sw128(&tmA, A, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128) ||
+      !make_tmap_bf16_sw128(&tmB, Bt, (uint64_t)n_rows_b, (uint64_t)K, (uint64_t)K, 128))
+    return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+  constexpr size_t stage = GM_SUB + (size_t)NT * 128;
+  p.M = M; p.kblocks = K / 64;
+  p.stages = p.kblocks < 4 ? p.kblocks : 4;
+  const size_t smem = p.stages * stage + 256;
+  LIME_CUDA(cudaFuncSetAttribute(k_gemm_tc<EPI, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  ProfScope _p(name, st);
+  dim3 grid((unsigned)((M + 127) / 128), (unsigned)n_tiles);
+  k_gemm_tc<EPI, NT><<<grid, GM_THREADS, smem, st>>>(tmA, tmB, p);
+  LIME_LAUNCH_CHECK(name);
+  return LIME_OK;
+}
+
+lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st) {
+  GemmParams p{};
+  p.ell = a.ell; p.H = a.H; p.Q2 = (__nv_bfloat16*)a.Q2; p.K2 = (__nv_bfloat16*)a.K2; p.G2t = (__nv_bfloat16*)a.G2t;
+  p.U2t = (__nv_bfloat16*)a.U2t; p.cQ = a.cQ; p.cK = a.cK; p.err = a.err;
+  // segments: Q2 | K2 | G2 | U2, H n-tiles each; the last layer needs only the queries
+  const int n_tiles = (a.need_hist ? 4 : 1) * a.H;
+  return launch_gemm<GM_EPI_PREP, 128>(a.A, a.M, 128, a.Bt, 4 * a.H * 128, n_tiles, p, "k_gemm_tc_prep", st);
+}
+
+lime_status launch_gemm_glu(const LinkGemmArgs& a, cudaStream_t st) {
+  GemmParams p{};
+  p.out = a.out; p.err = a.err;
+  return launch_gemm<GM_EPI_GLU, 256>(a.A, a.M, a.K, a.Bt, 256, 1, p, "k_gemm_tc_glu", st);
+}
+
+lime_status launch_gemm_f32(const LinkGemmArgs& a, cudaStream_t st) {
+  GemmParams p{};
+  p.out = a.out; p.n_total = 128; p.err = a.err;
+  return launch_gemm<GM_EPI_F32, 128>(a.A, a.M, a.K, a.Bt, 128, 1, p, "k_gemm_tc_f32", st);
+}
+
+}  // namespace lime

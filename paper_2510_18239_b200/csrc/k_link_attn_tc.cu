@@ -9,7 +9,7 @@
 //                         s_ij = rstd_j * (raw_ij - mu_j * rowsum(Q2)_i)
 //   acc    [HL x d]    += P' [HL x 128] . X_tile            P'_ij = p_ij * rstd_j;  the mean term sum_j P'_ij mu_j is
 //                                                           a per-row scalar subtracted from every column at the end
-//   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (merge kernel, also combines the chunks of a user)
+//   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (chunks merged in k_link_prep.cu, W_V folded into the GEMM after)
 // HL = H * ell stacked (head, link) rows = 128 TMEM lanes; thread i of the softmax warps owns row i: an online
 // softmax whose reference maximum is only raised when the true maximum exceeds it by more than 8 (then the
 // accumulator row is rescaled in TMEM), so most tiles need no correction pass.
@@ -301,59 +301,12 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   }
 }
 
-// Combine the chunks of a user (log-sum-exp weights), normalise, and apply W_V of the row's head:
-//   AT[b, l, h*d_h + k] = sum_i ( sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c ) * Wv[i, h*d_h + k]
-// grid (B, H); block 256.
-__global__ void __launch_bounds__(256)
-k_link_attn_merge_fold(const int32_t* __restrict__ chunk_start, int ell, int d, int H, const float* __restrict__ part_m,
-                       const float* __restrict__ part_s, const float* __restrict__ part_acc,
-                       const __nv_bfloat16* __restrict__ Wv, float* __restrict__ AT) {
-  extern __shared__ float sm[];
-  const int b = blockIdx.x, h = blockIdx.y, d_h = d / H, HL = H * ell;
-  float* Os = sm;                        // [ell][d] merged, normalised accumulator rows of head h
-  const int c0 = chunk_start[b], c1 = chunk_start[b + 1];
-  for (int i = threadIdx.x; i < ell * d; i += blockDim.x) {
-    const int l = i / d, k = i % d;
-    const int row = h * ell + l;
-    float out = 0.f;
-    if (c1 > c0) {
-      float M = -INFINITY;
-      for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
-      float S = 0.f, O = 0.f;
-      for (int c = c0; c < c1; ++c) {
-        const float w = __expf(part_m[(int64_t)c * HL + row] - M);
-        S = fmaf(part_s[(int64_t)c * HL + row], w, S);
-        O = fmaf(part_acc[((int64_t)c * HL + row) * d + k], w, O);
-      }
-      out = O / S;
-    }
-    Os[i] = out;
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < ell * d_h; i += blockDim.x) {
-    const int l = i / d_h, k = i % d_h;
-    float acc = 0.f;
-    if (Wv) {
-      for (int j = 0; j < d; ++j) acc = fmaf(Os[l * d + j], __bfloat162float(Wv[(int64_t)j * d + h * d_h + k]), acc);
-    } else {
-      acc = Os[l * d + h * d_h + k];
-    }
-    AT[((int64_t)b * ell + l) * d + h * d_h + k] = acc;
-  }
-}
-
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi) {
   return dtype == LIME_BF16 && d == LA_D && H * ell == LA_HL && phi == LIME_PHI_SOFTMAX;
 }
 
 lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
-  if (a.n_chunk_upper <= 0 || a.total == 0) {
-    if (a.B > 0) {
-      // no history at all: every user's attention output is zero
-      LIME_CUDA(cudaMemsetAsync(a.AT, 0, sizeof(float) * (size_t)a.B * a.ell * a.d, st));
-    }
-    return LIME_OK;
-  }
+  if (a.n_chunk_upper <= 0 || a.total == 0) return LIME_OK;   // no history: the merge step writes zeros
   CUtensorMap tmX, tmQ2;
   const uint64_t users = a.shared ? 1 : (uint64_t)a.B;
   if (!make_tmap_bf16_sw128(&tmX, a.hist, (uint64_t)a.total, LA_D, LA_D, LA_TILE) ||
@@ -367,14 +320,6 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
     ProfScope _p("k_link_attn_tc", st);
     k_link_attn_tc<<<a.n_chunk_upper, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
     LIME_LAUNCH_CHECK("k_link_attn_tc");
-  }
-  const size_t smem = sizeof(float) * (size_t)a.ell * a.d;
-  {
-    ProfScope _p("k_link_attn_merge_fold", st);
-    dim3 grid(a.B, a.H);
-    k_link_attn_merge_fold<<<grid, 256, smem, st>>>(a.chunk_start, a.ell, a.d, a.H, a.part_m, a.part_s, a.part_acc,
-                                                    (const __nv_bfloat16*)a.Wv, a.AT);
-    LIME_LAUNCH_CHECK("k_link_attn_merge_fold");
   }
   return LIME_OK;
 }

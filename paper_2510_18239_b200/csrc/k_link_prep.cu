@@ -1,80 +1,123 @@
-// Link-side operand preparation for the tensor-core XOR layer kernels.
+// Link-side preparation for the tensor-core XOR layer kernels.
 //
 // Both attention directions of Eq. 7 touch the history only through LN(S): K[S] = LN(S) W_K, V[S] = LN(S) W_V,
-// Q[S] = LN(S) W_Q.  Because the link side is tiny (ell rows per user), the projections are folded into it, so
-// that the streaming kernels contract directly against the stored history rows and never materialise Q/K/V of
-// the history:
-//   links <- history scores   Q[T]_h K[S]_h^T = Q2_(h,l) . LN(S)^T     Q2[(h,l), :] = scale * Q[T]_{l,h} W_{K,h}^T
-//   history <- links scores   Q[S]_h K[T]_h^T = LN(S) . K2_(h,l)^T     K2[(h,l), :] = scale * K[T]_{l,h} W_{Q,h}^T
-//   GatedMLP input O[S] W_g = P . G2,  O[S] W_u = P . U2               G2[(h,l), :] = V[T]_{l,h} W_g[h rows, :]
-// (h, l) = head-major stacked link rows, H*ell of them.  Outputs are bf16 in the layouts the MMA operands want.
+// Q[S] = LN(S) W_Q.  Because the link side is tiny (ell rows per user), the history-side projections are folded
+// into it, so that the streaming kernels contract directly against the stored history rows and never materialise
+// Q/K/V of the history.  With That = LN(T) the link rows entering the layer and (h, l) the head-major stacked rows:
+//   links <- history scores  Q[T]_h K[S]_h^T = Q2_(h,l) . LN(S)^T    Q2_(h,l) = That_l (scale W_{Q,h} W_{K,h}^T)
+//   history <- links scores  Q[S]_h K[T]_h^T = LN(S) . K2_(h,l)^T    K2_(h,l) = That_l (scale W_{K,h} W_{Q,h}^T)
+//   GatedMLP input           O[S] W_g = P . G2,  O[S] W_u = P . U2   G2_(h,l) = That_l (W_{V,h} W_g[h rows, :])
+//   link rows                O[T] W_g = sum_h Ohat_(h,l) (W_{V,h} W_g[h rows, :])        (same folded matrices)
+// The bracketed products depend on the weights only and are formed once, here, at lime_set_weights time.
 #include "lime_common.cuh"
 
 namespace lime {
 
-// out[(h,l), i] = scale * sum_{k < d_h} A[l, h*d_h + k] * W[i, h*d_h + k]      (W row-major [d_out x d], NULL = I)
-// grid (users, H), block 256.  A fp32 [ell x d] per user.
-__global__ void __launch_bounds__(256)
-k_fold_rows(const float* __restrict__ A, int64_t a_user_stride, const __nv_bfloat16* __restrict__ W, int ell, int d,
-            int H, int d_out, float scale, __nv_bfloat16* __restrict__ out, int64_t out_user_stride) {
-  extern __shared__ float smem[];
+__device__ __forceinline__ float w_at(const __nv_bfloat16* W, int r, int c, int ld) {
+  return W ? __bfloat162float(W[(int64_t)r * ld + c]) : (r == c ? 1.f : 0.f);
+}
+
+// WprepT [4*H*128 x d]  (B operand of the PREP GEMM: output column major, contraction index j contiguous)
+// WpostT [2f x H*d]     (B operand of the GLU GEMM on link rows)
+__global__ void k_fold_weights(const __nv_bfloat16* __restrict__ Wq, const __nv_bfloat16* __restrict__ Wk,
+                               const __nv_bfloat16* __restrict__ Wv, const __nv_bfloat16* __restrict__ Wg,
+                               const __nv_bfloat16* __restrict__ Wu, int d, int H, int f, float scale,
+                               __nv_bfloat16* __restrict__ WprepT, __nv_bfloat16* __restrict__ WpostT) {
   const int d_h = d / H;
-  float* As = smem;                      // [ell][d_h]
-  float* Ws = As + ell * d_h;            // [d_out][d_h + 1]
-  const int u = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  const float* a = A + (int64_t)u * a_user_stride;
-  for (int i = tid; i < ell * d_h; i += blockDim.x) As[i] = a[(i / d_h) * d + h * d_h + (i % d_h)];
-  for (int i = tid; i < d_out * d_h; i += blockDim.x) {
-    const int r = i / d_h, k = i % d_h;
-    Ws[r * (d_h + 1) + k] = W ? __bfloat162float(W[(int64_t)r * d + h * d_h + k]) : (r == h * d_h + k ? 1.f : 0.f);
-  }
-  __syncthreads();
-  __nv_bfloat16* o = out + (int64_t)u * out_user_stride + (int64_t)h * ell * d_out;
-  for (int i = tid; i < ell * d_out; i += blockDim.x) {
-    const int l = i / d_out, r = i % d_out;
+  const int n_prep = 4 * H * 128 * d, n_post = 2 * f * H * d;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < n_prep + n_post; idx += gridDim.x * blockDim.x) {
     float acc = 0.f;
-    const float* ar = As + l * d_h;
-    const float* wr = Ws + r * (d_h + 1);
-    for (int k = 0; k < d_h; ++k) acc = fmaf(ar[k], wr[k], acc);
-    o[(int64_t)l * d_out + r] = __float2bfloat16_rn(acc * scale);
+    if (idx < n_prep) {
+      const int R = idx / d, j = idx % d;
+      const int seg = R / (H * 128), h = (R / 128) % H, i = R % 128;
+      for (int k = h * d_h; k < (h + 1) * d_h; ++k) {
+        if (seg == 0) acc = fmaf(w_at(Wq, j, k, d), w_at(Wk, i, k, d), acc);
+        else if (seg == 1) acc = fmaf(w_at(Wk, j, k, d), w_at(Wq, i, k, d), acc);
+        else if (seg == 2) acc = fmaf(w_at(Wv, j, k, d), __bfloat162float(Wg[(int64_t)k * f + i]), acc);
+        else acc = fmaf(w_at(Wv, j, k, d), __bfloat162float(Wu[(int64_t)k * f + i]), acc);
+      }
+      if (seg < 2) acc *= scale;
+      WprepT[idx] = __float2bfloat16_rn(acc);
+    } else {
+      const int e = idx - n_prep;
+      const int R = e / (H * d), c = e % (H * d);
+      const int n = R % f, h = c / d, i = c % d;
+      const __nv_bfloat16* Wx = R < f ? Wg : Wu;
+      for (int k = h * d_h; k < (h + 1) * d_h; ++k) acc = fmaf(w_at(Wv, i, k, d), __bfloat162float(Wx[(int64_t)k * f + n]), acc);
+      WpostT[e] = __float2bfloat16_rn(acc);
+    }
   }
 }
 
-// outT[n, (h,l)] = sum_{k < d_h} A[l, h*d_h + k] * W[h*d_h + k, n]             (W row-major [d x f])
-// i.e. the transposed fold, stored [f x H*ell] so that (h,l) is the contiguous (contraction) index.
-__global__ void __launch_bounds__(256)
-k_fold_cols_t(const float* __restrict__ A, int64_t a_user_stride, const __nv_bfloat16* __restrict__ W, int ell, int d,
-              int H, int f, __nv_bfloat16* __restrict__ outT, int64_t out_user_stride) {
-  extern __shared__ float smem[];
-  const int d_h = d / H;
-  float* As = smem;                      // [ell][d_h + 1]
-  float* Ws = As + ell * (d_h + 1);      // [d_h][f]
-  const int u = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  const float* a = A + (int64_t)u * a_user_stride;
-  for (int i = tid; i < ell * d_h; i += blockDim.x) As[(i / d_h) * (d_h + 1) + (i % d_h)] = a[(i / d_h) * d + h * d_h + (i % d_h)];
-  for (int i = tid; i < d_h * f; i += blockDim.x) Ws[i] = __bfloat162float(W[(int64_t)(h * d_h + i / f) * f + (i % f)]);
-  __syncthreads();
-  const int HL = H * ell;
-  __nv_bfloat16* o = outT + (int64_t)u * out_user_stride;
-  for (int i = tid; i < ell * f; i += blockDim.x) {
-    const int n = i / ell, l = i % ell;
-    float acc = 0.f;
-    const float* ar = As + l * (d_h + 1);
-    for (int k = 0; k < d_h; ++k) acc = fmaf(ar[k], Ws[k * f + n], acc);
-    o[(int64_t)n * HL + h * ell + l] = __float2bfloat16_rn(acc);
-  }
+lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,
+                                int H, int f, float scale, void* WprepT, void* WpostT, cudaStream_t st) {
+  ProfScope _p("k_fold_weights", st);
+  k_fold_weights<<<kSMs * 2, 256, 0, st>>>((const __nv_bfloat16*)Wq, (const __nv_bfloat16*)Wk, (const __nv_bfloat16*)Wv,
+                                           (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, d, H, f, scale,
+                                           (__nv_bfloat16*)WprepT, (__nv_bfloat16*)WpostT);
+  LIME_LAUNCH_CHECK("k_fold_weights");
+  return LIME_OK;
 }
 
-// sums[r] = sum_i bf16 X[r, i]  (of the rounded values, so that the LayerNorm fold cancels exactly what the MMA sees)
+// out[r, :] = bf16( LN(T[r, :]) )  (or bf16(T) when ln == 0); one warp per row
 __global__ void __launch_bounds__(256)
-k_rowsum_bf16(const __nv_bfloat16* __restrict__ X, int64_t rows, int cols, float* __restrict__ sums) {
+k_ln_rows_bf16(const float* __restrict__ T, int64_t rows, int d, int ln, float eps, __nv_bfloat16* __restrict__ out) {
   const int lane = threadIdx.x & 31;
   const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= rows) return;
-  float s = 0.f;
-  for (int i = lane; i < cols; i += 32) s += __bfloat162float(X[r * cols + i]);
-  s = warp_sum(s);
-  if (lane == 0) sums[r] = s;
+  const float* x = T + r * d;
+  float mu = 0.f, rstd = 1.f;
+  if (ln) {
+    float s = 0.f;
+    for (int k = lane; k < d; k += 32) s += x[k];
+    mu = warp_sum(s) / (float)d;
+    float v = 0.f;
+    for (int k = lane; k < d; k += 32) { const float c = x[k] - mu; v = fmaf(c, c, v); }
+    rstd = rsqrtf(warp_sum(v) / (float)d + eps);
+  }
+  for (int k = lane; k < d; k += 32) out[r * d + k] = __float2bfloat16_rn((x[k] - mu) * rstd);
+}
+
+lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, float eps, void* out, cudaStream_t st) {
+  if (rows == 0) return LIME_OK;
+  ProfScope _p("k_ln_rows_bf16", st);
+  k_ln_rows_bf16<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(T, rows, d, ln, eps, (__nv_bfloat16*)out);
+  LIME_LAUNCH_CHECK("k_ln_rows_bf16");
+  return LIME_OK;
+}
+
+// Combine the chunks of a user with log-sum-exp weights and normalise:
+//   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = exp(m_c - max_c m_c)
+// grid (B * H * ell), block d threads.  A user without history gets zeros.
+__global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H,
+                                       const float* __restrict__ part_m, const float* __restrict__ part_s,
+                                       const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
+  const int HL = H * ell;
+  const int u = blockIdx.x / HL, row = blockIdx.x % HL, h = row / ell, l = row % ell;
+  const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
+  const int i = threadIdx.x;
+  float out = 0.f;
+  if (c1 > c0) {
+    float M = -INFINITY;
+    for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
+    float S = 0.f, O = 0.f;
+    for (int c = c0; c < c1; ++c) {
+      const float w = __expf(part_m[(int64_t)c * HL + row] - M);
+      S = fmaf(part_s[(int64_t)c * HL + row], w, S);
+      O = fmaf(part_acc[((int64_t)c * HL + row) * d + i], w, O);
+    }
+    out = O / S;
+  }
+  Ohat[((int64_t)u * ell + l) * (H * d) + h * d + i] = __float2bfloat16_rn(out);
+}
+
+lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
+                                        const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
+  if (B == 0) return LIME_OK;
+  ProfScope _p("k_link_attn_merge_norm", st);
+  k_link_attn_merge_norm<<<B * H * ell, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
+  return LIME_OK;
 }
 
 // W [rows x cols] -> WT [cols x rows]  (bf16), set-up time only
@@ -97,36 +140,6 @@ lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, c
   dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
   k_transpose_bf16<<<grid, block, 0, st>>>((const __nv_bfloat16*)W, rows, cols, (__nv_bfloat16*)WT);
   LIME_LAUNCH_CHECK("k_transpose_bf16");
-  return LIME_OK;
-}
-
-lime_status launch_link_prep(const LinkPrepArgs& a, cudaStream_t st) {
-  const int d_h = a.d / a.H, HL = a.H * a.ell;
-  dim3 grid(a.users, a.H);
-  const size_t smem_rows = sizeof(float) * ((size_t)a.ell * d_h + (size_t)a.d * (d_h + 1));
-  const size_t smem_cols = sizeof(float) * ((size_t)a.ell * (d_h + 1) + (size_t)d_h * a.f);
-  if (smem_rows > 200 * 1024 || smem_cols > 200 * 1024) return LIME_UNSUPPORTED_SHAPE;
-  ProfScope _p("k_link_prep", st);
-  LIME_CUDA(cudaFuncSetAttribute(k_fold_rows, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_rows));
-  LIME_CUDA(cudaFuncSetAttribute(k_fold_cols_t, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_cols));
-  const int64_t ustride = a.shared ? 0 : (int64_t)a.ell * a.d;
-  if (a.Q2) {
-    k_fold_rows<<<grid, 256, smem_rows, st>>>(a.QT, ustride, (const __nv_bfloat16*)a.Wk, a.ell, a.d, a.H, a.d, a.scale,
-                                              (__nv_bfloat16*)a.Q2, (int64_t)HL * a.d);
-    k_rowsum_bf16<<<(unsigned)(((int64_t)a.users * HL + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)a.Q2,
-                                                                              (int64_t)a.users * HL, a.d, a.cQ);
-  }
-  if (a.K2) {
-    k_fold_rows<<<grid, 256, smem_rows, st>>>(a.KT, ustride, (const __nv_bfloat16*)a.Wq, a.ell, a.d, a.H, a.d, a.scale,
-                                              (__nv_bfloat16*)a.K2, (int64_t)HL * a.d);
-    k_rowsum_bf16<<<(unsigned)(((int64_t)a.users * HL + 7) / 8), 256, 0, st>>>((const __nv_bfloat16*)a.K2,
-                                                                              (int64_t)a.users * HL, a.d, a.cK);
-    k_fold_cols_t<<<grid, 256, smem_cols, st>>>(a.VT, ustride, (const __nv_bfloat16*)a.Wg, a.ell, a.d, a.H, a.f,
-                                                (__nv_bfloat16*)a.G2t, (int64_t)a.f * HL);
-    k_fold_cols_t<<<grid, 256, smem_cols, st>>>(a.VT, ustride, (const __nv_bfloat16*)a.Wu, a.ell, a.d, a.H, a.f,
-                                                (__nv_bfloat16*)a.U2t, (int64_t)a.f * HL);
-  }
-  LIME_LAUNCH_CHECK("k_link_prep");
   return LIME_OK;
 }
 

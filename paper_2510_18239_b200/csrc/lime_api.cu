@@ -57,6 +57,7 @@ struct Workspace {
   // tensor-core path: folded link-side operands (bf16) and their row sums
   void *Q2, *K2, *G2t, *U2t;
   float *cQ, *cK;
+  void *That, *Ohat, *UTb;   // LN(T) [B*ell x d], merged attention rows [B*ell x H*d], GLU output [B*ell x d_ff] (bf16)
   int chunk, n_chunk_upper, n_tile_upper;
   size_t bytes;
 };
@@ -88,8 +89,59 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.Q2 = take((size_t)B * HL * g.d * 2); w.K2 = take((size_t)B * HL * g.d * 2);
   w.G2t = take((size_t)B * c->d_ff * HL * 2); w.U2t = take((size_t)B * c->d_ff * HL * 2);
   w.cQ = (float*)take((size_t)B * HL * 4); w.cK = (float*)take((size_t)B * HL * 4);
+  w.That = take((size_t)B * g.ell * g.d * 2); w.Ohat = take((size_t)B * g.ell * g.H * g.d * 2);
+  w.UTb = take((size_t)B * g.ell * c->d_ff * 2);
   w.bytes = o;
   return w;
+}
+
+// True when the whole layer runs on the tensor-core kernels (bf16, d = d_ff = 128, H * ell = 128, softmax, GatedMLP).
+static bool layer_on_tensor_cores(const Ctx* c, int layer) {
+  const lime_config& g = c->cfg;
+  return c->WoT[layer] && c->WprepT[layer] && c->WpostT[layer] && link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi) &&
+         hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
+}
+
+// One XOR layer, tensor-core path: three link-row GEMMs around the two streaming attention kernels.
+static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B, int64_t total,
+                                const float* links_in, int links_shared, void* hist_out, float* links_out,
+                                const Workspace& w, cudaStream_t st) {
+  const lime_config& g = c->cfg;
+  lime_status s;
+  const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
+  const int64_t BL = (int64_t)B * g.ell;
+  // LN(T) -> bf16, then one GEMM gives every folded link-side operand of both attention directions
+  if ((s = launch_ln_rows_bf16(links_in, link_rows, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
+  LinkGemmArgs gp{};
+  gp.A = w.That; gp.M = link_rows; gp.K = g.d; gp.Bt = c->WprepT[layer]; gp.ell = g.ell; gp.H = g.H;
+  gp.need_hist = hist_out != nullptr; gp.Q2 = w.Q2; gp.K2 = w.K2; gp.G2t = w.G2t; gp.U2t = w.U2t; gp.cQ = w.cQ; gp.cK = w.cK;
+  gp.err = c->dev_err;
+  if ((s = launch_gemm_prep(gp, st)) != LIME_OK) return s;
+  // O[T]: links attend over the stored history (keys = values = history rows), chunks merged and normalised
+  LinkAttnArgs la{};
+  la.hist = hist_in; la.total = total; la.Q2 = w.Q2; la.cQ = w.cQ; la.off = off; la.chunk_start = w.chunk_start; la.B = B;
+  la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = links_shared;
+  la.ln = g.ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.err = c->dev_err;
+  if ((s = launch_link_attn_tc(la, st)) != LIME_OK) return s;
+  if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
+    return s;
+  // links_out = GatedMLP(O[T]) with W_V folded into the gate / up weights
+  LinkGemmArgs gg{};
+  gg.A = w.Ohat; gg.M = BL; gg.K = g.H * g.d; gg.Bt = c->WpostT[layer]; gg.out = w.UTb; gg.err = c->dev_err;
+  if ((s = launch_gemm_glu(gg, st)) != LIME_OK) return s;
+  LinkGemmArgs go{};
+  go.A = w.UTb; go.M = BL; go.K = c->d_ff; go.Bt = c->WoT[layer]; go.out = links_out; go.err = c->dev_err;
+  if ((s = launch_gemm_f32(go, st)) != LIME_OK) return s;
+  if (hist_out) {
+    // history attends back over the links; scores, per-head softmax, value mix and GatedMLP in one fused kernel
+    HistUpdateArgs hu{};
+    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
+    hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
+    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = g.ln; hu.ln_eps = c->ln_eps;
+    hu.err = c->dev_err;
+    if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
+  }
+  return LIME_OK;
 }
 
 // One XOR layer on a carved workspace (see lime_xor_layer in lime.h for the contract).
@@ -98,6 +150,14 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
                                   float* links_out, const Workspace& w, bool schedules_ready, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
+  if (!schedules_ready) {
+    if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
+    if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
+  }
+  if (layer_on_tensor_cores(c, layer))
+    return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, st);
+
+  // ---- generic path on CUDA cores (fp32 storage, other shapes, SiLU attention, no GatedMLP) ----
   const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
 
   // link rows: Q[T], K[T], V[T] = LN(T) W_{Q,K,V}
@@ -108,47 +168,15 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   la.ln = g.ln; la.ln_eps = c->ln_eps;
   if ((s = launch_linear_simt(la, st)) != LIME_OK) return s;
 
-  // history rows: K[S], V[S], Q[S] = LN(S) W, only for the directions that run on CUDA cores (the tensor-core
-  // kernels contract against the stored history and never materialise them)
-  const bool tc_hist = hist_out && c->WoT[layer] &&
-                       hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
-  const bool tc_link = link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi);
-  {
-    LinearArgs lh{};
-    lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
-    lh.ln = g.ln; lh.ln_eps = c->ln_eps;
-    int n = 0;
-    if (!tc_link) { lh.W[n] = c->w.Wk[layer]; lh.Y[n++] = w.K; lh.W[n] = c->w.Wv[layer]; lh.Y[n++] = w.V; }
-    if (hist_out && !tc_hist) { lh.W[n] = c->w.Wq[layer]; lh.Y[n++] = w.Q; }
-    lh.n_out = n;
-    if (n > 0 && (s = launch_linear_simt(lh, st)) != LIME_OK) return s;
-  }
-
-  if (!schedules_ready) {
-    if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
-    if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
-  }
-
-  if (tc_link || tc_hist) {
-    // fold the history-side projections into the link rows (see k_link_prep.cu)
-    LinkPrepArgs lp{};
-    lp.QT = w.QT; lp.KT = w.KT; lp.VT = w.VT; lp.users = links_shared ? 1 : B; lp.shared = links_shared;
-    lp.ell = g.ell; lp.d = g.d; lp.H = g.H; lp.f = c->d_ff; lp.scale = c->attn_scale;
-    lp.Wq = c->w.Wq[layer]; lp.Wk = c->w.Wk[layer]; lp.Wg = c->w.Wg[layer]; lp.Wu = c->w.Wu[layer];
-    if (tc_link) { lp.Q2 = w.Q2; lp.cQ = w.cQ; }
-    if (tc_hist) { lp.K2 = w.K2; lp.cK = w.cK; lp.G2t = w.G2t; lp.U2t = w.U2t; }
-    if ((s = launch_link_prep(lp, st)) != LIME_OK) return s;
-  }
+  // history rows: K[S], V[S] (and Q[S] when the history is updated) = LN(S) W
+  LinearArgs lh{};
+  lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
+  lh.W[0] = c->w.Wk[layer]; lh.W[1] = c->w.Wv[layer]; lh.W[2] = c->w.Wq[layer];
+  lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = hist_out ? 3 : 2;
+  lh.ln = g.ln; lh.ln_eps = c->ln_eps;
+  if ((s = launch_linear_simt(lh, st)) != LIME_OK) return s;
 
   // O[T] = phi(Q[T] K[S]^T) V[S]
-  if (tc_link) {
-    LinkAttnArgs la2{};
-    la2.hist = hist_in; la2.total = total; la2.Q2 = w.Q2; la2.cQ = w.cQ; la2.Wv = c->w.Wv[layer]; la2.off = off;
-    la2.chunk_start = w.chunk_start; la2.B = B; la2.chunk = w.chunk; la2.n_chunk_upper = w.n_chunk_upper;
-    la2.ell = g.ell; la2.d = g.d; la2.H = g.H; la2.shared = links_shared; la2.ln = g.ln; la2.ln_eps = c->ln_eps;
-    la2.part_m = w.part_m; la2.part_s = w.part_s; la2.part_acc = w.part_acc; la2.AT = w.AT; la2.err = c->dev_err;
-    if ((s = launch_link_attn_tc(la2, st)) != LIME_OK) return s;
-  } else {
   AttnLinkArgs al{};
   al.QT = w.QT; al.qt_user_stride = links_shared ? 0 : (int64_t)g.ell * g.d;
   al.KS = w.K; al.VS = w.V; al.s_dtype = g.dtype; al.off = off; al.B = B; al.total = total;
@@ -157,7 +185,6 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   al.part_m = w.part_m; al.part_s = w.part_s; al.part_acc = w.part_acc; al.AT = w.AT;
   if ((s = launch_attn_link_simt(al, st)) != LIME_OK) return s;
   if ((s = launch_attn_link_merge(al, st)) != LIME_OK) return s;
-  }
 
   // links_out = GatedMLP(O[T])
   const int64_t BL = (int64_t)B * g.ell;
@@ -174,15 +201,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
     if ((s = launch_axpy(w.AT, links_out, BL * g.d, 1, st)) != LIME_OK) return s;
   }
 
-  if (tc_hist) {
-    // scores, per-head softmax, value mix and GatedMLP in one fused tensor-core kernel
-    HistUpdateArgs hu{};
-    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
-    hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
-    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = g.ln; hu.ln_eps = c->ln_eps;
-    hu.err = c->dev_err;
-    if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
-  } else if (hist_out) {
+  if (hist_out) {
     // O[S] = phi(Q[S] K[T]^T) V[T], written over Q[S]; then hist_out = GatedMLP(O[S])
     AttnHistArgs ah{};
     ah.QS = w.Q; ah.AS = w.Q; ah.s_dtype = g.dtype; ah.KT = w.KT; ah.VT = w.VT;
@@ -293,7 +312,7 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
-  for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = nullptr;
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
@@ -316,7 +335,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   cudaFree(c->keff);
   cudaFree(c->links32);
   cudaFree(c->dev_err);
-  for (int j = 0; j < LIME_MAX_LAYERS; ++j) cudaFree(c->WoT[j]);
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); }
   delete c;
   return LIME_OK;
 }
@@ -338,11 +357,18 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
   if (s != LIME_OK) return s;
   s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_scale, c->keff, st);
   if (s != LIME_OK) return s;
-  // tensor-core path: W_o as a K-major B operand ([d x d_ff], contraction index contiguous)
-  if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) {
+  // tensor-core path: per layer, W_o as a K-major B operand ([d x d_ff], contraction index contiguous) and the
+  // weight-only products that fold the history-side projections into the link rows
+  if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) &&
+      link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi)) {
     for (int j = 0; j < g.n_layers; ++j) {
       if (!c->WoT[j]) LIME_CUDA(cudaMalloc(&c->WoT[j], (size_t)g.d * c->d_ff * 2));
+      if (!c->WprepT[j]) LIME_CUDA(cudaMalloc(&c->WprepT[j], (size_t)4 * g.H * 128 * g.d * 2));
+      if (!c->WpostT[j]) LIME_CUDA(cudaMalloc(&c->WpostT[j], (size_t)2 * c->d_ff * g.H * g.d * 2));
       if ((s = launch_transpose_bf16(w->Wo[j], c->d_ff, g.d, c->WoT[j], st)) != LIME_OK) return s;
+      if ((s = launch_fold_weights(w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], g.d, g.H, c->d_ff, c->attn_scale,
+                                   c->WprepT[j], c->WpostT[j], st)) != LIME_OK)
+        return s;
     }
   }
   c->have_weights = true;

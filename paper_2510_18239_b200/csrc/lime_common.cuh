@@ -52,7 +52,9 @@ struct Ctx {
   int device;
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
-  void* WoT[LIME_MAX_LAYERS];  // W_o transposed [d x d_ff] bf16 per layer (tensor-core path), or NULL
+  void* WoT[LIME_MAX_LAYERS];    // tensor-core path, per layer (NULL otherwise): W_o transposed [d x d_ff] bf16,
+  void* WprepT[LIME_MAX_LAYERS]; //   folded PREP operand [4*H*128 x d], folded link-row GLU operand [2*d_ff x H*d]
+  void* WpostT[LIME_MAX_LAYERS];
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
   int d_ff, d_h;
@@ -155,26 +157,30 @@ bool score_tc_supported(const ScoreArgs& a);
 lime_status launch_score_tc(const ScoreArgs& a, int* err, cudaStream_t st);
 
 // ---- tensor-core XOR layer (bf16, d = d_ff = 128, H * ell = 128) ----------------------------------------------
-struct LinkPrepArgs {
-  const float *QT, *KT, *VT;     // [users x ell x d] fp32 projected link rows (users = 1 when shared)
-  int users, shared, ell, d, H, f;
-  float scale;
-  const void *Wq, *Wk, *Wg, *Wu; // layer weights (bf16; Wq / Wk may be NULL = identity)
-  void* Q2; float* cQ;           // out (nullable pair): folded link queries [users x H*ell x d] bf16 and their row sums
-  void* K2; float* cK;           // out (nullable group): folded link keys, row sums,
-  void* G2t; void* U2t;          //   folded gate / up operands [users x f x H*ell] bf16
-};
-lime_status launch_link_prep(const LinkPrepArgs& a, cudaStream_t st);
+lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,
+                                int H, int f, float scale, void* WprepT, void* WpostT, cudaStream_t st);
+lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, float eps, void* out, cudaStream_t st);
+lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
+                                        const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st);
 lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, cudaStream_t st);
+
+// link-row GEMMs on tensor cores (k_gemm_tc.cu); A [M x K] bf16 row-major, Bt [N x K] bf16 (weights, pre-folded)
+struct LinkGemmArgs {
+  const void* A; int64_t M; int K; const void* Bt; void* out;
+  int ell, H, need_hist;                       // PREP: rows are (user, link); need_hist = also K2 / G2t / U2t
+  void *Q2, *K2, *G2t, *U2t; float *cQ, *cK;   // PREP outputs
+  int* err;
+};
+lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st);
+lime_status launch_gemm_glu(const LinkGemmArgs& a, cudaStream_t st);
+lime_status launch_gemm_f32(const LinkGemmArgs& a, cudaStream_t st);
 
 struct LinkAttnArgs {
   const void* hist; int64_t total;          // [total x d] bf16
   const void* Q2; const float* cQ;          // folded link queries [users x H*ell x d] bf16 and their row sums
-  const void* Wv;                           // [d x d] bf16 or NULL (identity)
   const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
   int ell, d, H, shared, ln; float ln_eps;
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
-  float* AT;                                // out [B x ell x d] fp32
   int* err;
 };
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi);
