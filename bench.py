@@ -45,25 +45,50 @@ def peaks():
 
 # ----------------------------------------------------------------------------- algorithmic work per kernel and step
 def kernel_models(wl: synth.Workload, total_tokens: int):
-    """name -> (bound, algorithmic units per step, unit).  Bytes: what the stage must move; flops: what it must
-    compute (2 per multiply-add), for all launches of that kernel in one step."""
+    """name -> dict(bytes=, flops=) : algorithmic work of ALL launches of that kernel in one step.  Bytes are what
+    the stage must move through HBM (inputs read once, outputs written once, scratch excluded); flops what it must
+    compute (2 per multiply-add).  A kernel with both is bounded by whichever floor (bytes / HBM peak, flops /
+    tensor peak) is longer."""
     es = 4 if wl.dtype == synth.F32 else 2
     d, ell, H, n, f = wl.d, wl.ell, wl.H, wl.n_layers, wl.dff
-    BC, BL, N = wl.B * wl.C, wl.B * wl.ell, total_tokens
+    BC, BL, N, HL = wl.B * wl.C, wl.B * wl.ell, total_tokens, wl.H * wl.ell
     hist_proj = sum((3 if j < n - 1 else 2) for j in range(n)) * 2.0 * N * d * d
     link_proj = (ell + (n - 1) * BL) * 3 * 2.0 * d * d
     glu = 4.0 * d * f * (BL * n + N * (n - 1))
     down = 2.0 * d * f * (BL * n + N * (n - 1))
-    m = {
-        "k_score": ("hbm", BC * (es * ell + es * d + 4.0), "B"),
-        "k_gather": ("hbm", N * (4.0 + 2 * es * d), "B"),
-        "k_linear_simt_ln": ("alu", hist_proj + link_proj, "flop"),
-        "k_linear_simt_glu": ("alu", glu, "flop"),
-        "k_linear_simt": ("alu", down, "flop"),
-        "k_attn_link": ("alu", 4.0 * ell * d * N * n, "flop"),
-        "k_attn_hist": ("alu", 4.0 * ell * d * N * (n - 1), "flop"),
+    return {
+        "k_score": dict(bytes=BC * (es * ell + es * d + 4.0)),
+        "k_gather": dict(bytes=N * (4.0 + 2 * es * d)),
+        "k_precompute": dict(bytes=BC * es * (d + ell)),
+        # fused tensor-core layer kernels: history rows read once per direction, written once by the update
+        "k_link_attn_tc": dict(bytes=n * N * d * es, flops=n * 4.0 * HL * d * N, pipe="tensor"),
+        "k_hist_update_tc": dict(bytes=(n - 1) * 2.0 * N * d * es, flops=(n - 1) * 2.0 * N * (HL * d + 2 * HL * f + f * d),
+                                 pipe="tensor"),
+        # CUDA-core path (fp32 storage and shapes the tensor-core kernels do not serve)
+        "k_linear_simt_ln": dict(flops=hist_proj + link_proj, pipe="alu"),
+        "k_linear_simt_glu": dict(flops=glu, pipe="alu"),
+        "k_linear_simt": dict(flops=down, pipe="alu"),
+        "k_attn_link": dict(flops=4.0 * ell * d * N * n, pipe="alu"),
+        "k_attn_hist": dict(flops=4.0 * ell * d * N * (n - 1), pipe="alu"),
     }
-    return m
+
+
+def roofline_entry(mdl, ms, pk):
+    """Achieved rate of `ms` milliseconds of kernel time against the roofline that bounds it."""
+    t = ms * 1e-3
+    floors = {}
+    if "bytes" in mdl:
+        floors["hbm"] = mdl["bytes"] / (pk["hbm_gbs"] * 1e9)
+    if "flops" in mdl:
+        peak = FP32_ALU_TFLOPS if mdl.get("pipe") == "alu" else pk["bf16_tflops_sustained"]
+        floors["alu" if mdl.get("pipe") == "alu" else "tensor"] = mdl["flops"] / (peak * 1e12)
+    bound = max(floors, key=floors.get)
+    if bound == "hbm":
+        ach = mdl["bytes"] / t / 1e9
+        return dict(bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"])
+    peak = FP32_ALU_TFLOPS if bound == "alu" else pk["bf16_tflops_sustained"]
+    ach = mdl["flops"] / t / 1e12
+    return dict(bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
 
 
 def model_for(name, models):
@@ -176,8 +201,9 @@ def run_reference(args, wl):
     if rank != 0:
         return
     inp = synth.make_inputs(wl, seed=0)
-    users_per_step = max(1, min(wl.B, 2))
-    for _ in range(args.warmup):
+    _, t_user = oracle_sample(wl, inp, range(1))          # calibrates the per-step sample; also the first warm-up
+    users_per_step = 2 if (wl.B >= 2 and 2 * t_user * args.steps < 120.0) else 1
+    for _ in range(max(0, args.warmup - 1)):
         oracle_sample(wl, inp, range(1))
     times = []
     for s in range(args.steps):
@@ -202,6 +228,28 @@ def workload_config(wl):
 
 
 # ----------------------------------------------------------------------------- the CUDA arm
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels captured with ncu, keyed by
+# kernel and workload, with the hash of the kernel's source at capture time: once the source changes the figure
+# is stale and the bench reports null.
+NCU_TRAFFIC = {}
+
+
+def source_hash(rel):
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2510_18239_b200", "csrc", rel), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:16]
+
+
+def ncu_traffic(kernel, wl):
+    rec = NCU_TRAFFIC.get((kernel, wl.name, wl.B, wl.C))
+    if not rec:
+        return None
+    try:
+        return rec["bytes"] if source_hash(rec["source"]) == rec["sha"] else None
+    except OSError:
+        return None
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -235,16 +283,22 @@ def run_ours(args, wl):
         s = dict(lengths=torch.from_numpy(lengths).to(dev), hist_ids=torch.from_numpy(hist_ids).to(dev),
                  cand_ids=torch.from_numpy(cand_ids).to(dev), total=total)
         s["T"] = lime.gather_history(table, s["cand_ids"])
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s["W"] = lime.precompute_candidate_links(s["T"])          # warm
-        e0.record()
         s["W"] = lime.precompute_candidate_links(s["T"])
-        e1.record()
-        torch.cuda.synchronize()
-        pre_ms.append(e0.elapsed_time(e1))
         sets.append(s)
         host_sets.append(dict(lengths=torch.from_numpy(lengths).pin_memory(), hist_ids=torch.from_numpy(hist_ids).pin_memory(),
                               cand_ids=torch.from_numpy(cand_ids).pin_memory(), total=total))
+    # offline stage, timed on its own: one launch per input set, back to back, sets rotated (inputs > L2 in all)
+    wscratch = torch.empty_like(sets[0]["W"])
+    for s in sets:
+        Bd.lime_precompute_candidate_links(lime.ctx, s["T"], wscratch)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pre_reps = 5 * ROTATE
+    e0.record()
+    for i in range(pre_reps):
+        Bd.lime_precompute_candidate_links(lime.ctx, sets[i % ROTATE]["T"], wscratch)
+    e1.record()
+    torch.cuda.synchronize()
+    pre_ms = e0.elapsed_time(e1) / pre_reps
     max_total = max(s["total"] for s in sets)
     off = torch.empty(wl.B + 1, dtype=torch.int32, device=dev)
     hist = torch.empty((max_total, wl.d), dtype=lime.tdtype, device=dev)
@@ -272,8 +326,8 @@ def run_ours(args, wl):
     for i in range(args.warmup):
         step(i)
     barrier()
-    cap = 64 * args.steps + 64
-    Bd.lime_profile_start(cap)
+
+    # ---- timed region: exactly `steps` steps, device-timed, nothing but the library's launches in between
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
     sampler.mark(True)
@@ -284,7 +338,6 @@ def run_ours(args, wl):
     torch.cuda.synchronize()
     sampler.mark(False)
     barrier()
-    records, launches = Bd.lime_profile_stop(cap)
     clocks = sampler.stop() if rank == 0 else None
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))
@@ -294,8 +347,35 @@ def run_ours(args, wl):
         total_ms = float(t.item())
     value = world * wl.B * wl.C * args.steps / (total_ms * 1e-3)
 
-    # end to end through the C ABI from host buffers: request = (lengths, history ids, candidate ids) in pinned host
-    # memory; the corpus-level caches (table, phi(T L^t) for every item) are resident, as in the paper's serving flow
+    # ---- the same steps again with every launch of the library bracketed by CUDA events on its stream: per-kernel
+    #      launch durations and the launch count of one step (the brackets add gaps, so this pass is not `value`)
+    prof_steps = min(args.steps, 100)
+    cap = 64 * prof_steps + 64
+    Bd.lime_profile_start(cap)
+    for i in range(prof_steps):
+        step(i)
+    torch.cuda.synchronize()
+    records, launches = Bd.lime_profile_stop(cap)
+    launches_per_step = launches / prof_steps
+
+    # ---- the scoring kernel alone, back to back over the rotating input sets (burst figure: no event brackets
+    #      or neighbouring kernels inside the interval)
+    score_reps = max(20, min(200, args.steps))
+    for i in range(ROTATE):
+        s = sets[i]
+        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(score_reps):
+        s = sets[i % ROTATE]
+        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+    e1.record()
+    torch.cuda.synchronize()
+    score_alone_ms = e0.elapsed_time(e1) / score_reps
+
+    # ---- end to end through the C ABI from host buffers: request = (lengths, history ids, candidate ids) in pinned
+    #      host memory; the corpus-level caches (table, phi(T L^t) for every item) are resident, as in the paper's
+    #      serving flow; logits come back to pinned host memory
     w_corpus = lime.precompute_candidate_links(table)
     d_len = torch.empty(wl.B, dtype=torch.int32, device=dev)
     d_hid = torch.empty(max_total, dtype=torch.int32, device=dev)
@@ -321,10 +401,9 @@ def run_ours(args, wl):
         h_logits.copy_(logits, non_blocking=True)
         return 4 * (wl.B + n + wl.B * wl.C), 4 * wl.B * wl.C
 
-    for i in range(min(3, args.warmup)):
+    for i in range(3):
         e2e_step(i)
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h2d = d2h = 0
     e0.record()
     for i in range(args.steps):
@@ -340,6 +419,7 @@ def run_ours(args, wl):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_ms = float(t.item())
     e2e_value = world * wl.B * wl.C * args.steps / (e2e_ms * 1e-3)
+    Bd.lime_device_status(ctx)          # raises if any bounded in-kernel wait gave up during the run
 
     if rank == 0:
         pk = peaks()
@@ -353,26 +433,34 @@ def run_ours(args, wl):
         ksum = sum(v[1] for v in agg.values()) or 1.0
         kernels = []
         for name, (cnt, ms) in sorted(agg.items(), key=lambda kv: -kv[1][1]):
-            per_step_ms = ms / args.steps
-            entry = {"kernel": name, "launches_per_step": cnt / args.steps, "ms_per_step": per_step_ms, "share": ms / ksum}
+            per_step_ms = ms / prof_steps
+            entry = {"kernel": name, "launches_per_step": cnt / prof_steps, "ms_per_step": per_step_ms, "share": ms / ksum}
             mdl = model_for(name, models)
             if mdl and per_step_ms > 0:
-                bound, units, unit = mdl
-                if bound == "hbm":
-                    ach = units / (per_step_ms * 1e-3) / 1e9
-                    entry.update(bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"])
-                else:
-                    ach = units / (per_step_ms * 1e-3) / 1e12
-                    peak = FP32_ALU_TFLOPS if bound == "alu" else pk["bf16_tflops_sustained"]
-                    entry.update(bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
+                entry.update(roofline_entry(mdl, per_step_ms, pk))
             kernels.append(entry)
+
+        def roof(k, ms=None, how="CUDA events around each launch inside the step"):
+            mdl = model_for(k["kernel"], models)
+            r = dict(kernel=k["kernel"], **roofline_entry(mdl, ms if ms is not None else k["ms_per_step"], pk))
+            r["traffic"] = ncu_traffic(k["kernel"], wl)
+            r["peak_source"] = ("derived: 148 SM x 128 lanes x 2 x 1.965 GHz" if r["bound"] == "alu" else
+                                f"{pk['source']} ({'copy bandwidth' if r['bound'] == 'hbm' else 'sustained bf16 GEMM'})")
+            r["timing"] = how
+            r["share_of_step"] = k["share"]
+            return r
+
         dom = next((k for k in kernels if "bound" in k), None)
-        roofline = None
-        if dom:
-            roofline = {"kernel": dom["kernel"], "bound": dom["bound"], "achieved": dom["achieved"], "peak": dom["peak"],
-                        "unit": dom["unit"], "frac": dom["frac"], "traffic": None,
-                        "peak_source": pk["source"] if dom["bound"] != "alu" else "derived: 148 SM x 128 lanes x 2 x 1.965 GHz"}
+        roofline = roof(dom) if dom else None
         score = next((k for k in kernels if k["kernel"].startswith("k_score")), None)
+        scoring = None
+        if score:
+            scoring = roof(score, score_alone_ms, f"{score_reps} back-to-back launches over {ROTATE} rotating input sets, CUDA events")
+            scoring["ms_alone"] = score_alone_ms
+            scoring["ms_in_step"] = score["ms_per_step"]
+            scoring["frac_in_step"] = score.get("frac")
+            if roofline and roofline["kernel"] == score["kernel"]:
+                roofline = scoring
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
@@ -386,9 +474,10 @@ def run_ours(args, wl):
                 "data": "synthetic", "config": workload_config(wl), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps},
-                "gpu_launches": launches, "roofline": roofline, "scoring_roofline": score, "kernels": kernels[:12],
-                "precompute": {"ms": statistics.median(pre_ms), "candidates": wl.B * wl.C,
-                               "candidates_per_s": wl.B * wl.C / (statistics.median(pre_ms) * 1e-3)},
+                "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roofline, "scoring_roofline": scoring,
+                "kernels": kernels[:14],
+                "precompute": {"ms": pre_ms, "candidates": wl.B * wl.C, "candidates_per_s": wl.B * wl.C / (pre_ms * 1e-3),
+                               **roofline_entry(models["k_precompute"], pre_ms, pk)},
                 "cpu_baseline": cpu, "peaks": pk}
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -398,7 +487,7 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="bf16_baseline")
