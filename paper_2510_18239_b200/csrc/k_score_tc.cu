@@ -5,11 +5,12 @@
 // The contraction T.LS^T is a real dense GEMM (25-50 flop per streamed byte, more than the CUDA cores can
 // sustain at HBM rate), so it runs as tcgen05.mma with the accumulator in TMEM; what remains per candidate is an
 // ell-term dot product with the cached weight row.  The kernel is a persistent, warp-specialised stream:
-//   warp 0    : TMA producer  - candidate tile [128 x d] (+ the user's link states when the stage holds another
-//                               user's) into a ring of 128B-swizzled shared-memory stages
+//   warp 0    : TMA producer  - candidate tile [128 x d], its cached weight rows [128 x ell] (+ the user's link
+//                               states when the stage holds another user's) into a ring of shared-memory stages
 //   warp 1    : MMA issuer    - d/16 tcgen05.mma (M=128, N=ell, K=16) per tile into one of two TMEM accumulators
-//   warps 2-5 : epilogue      - thread r owns candidate row r of the tile (TMEM lane r): prefetches its weight row
-//                               with 128-bit loads, reads the accumulator row with tcgen05.ld, writes one logit
+//   warps 2-5 : epilogue      - thread r owns candidate row r of the tile (TMEM lane r): takes its weight row from
+//                               the stage, reads the accumulator row with tcgen05.ld, writes one logit
+// Every HBM stream is therefore prefetched a whole ring ahead of its use; no warp waits on a global load.
 // HBM traffic per candidate is the algorithmic minimum: its weight row, its embedding row, one fp32 logit.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
@@ -21,7 +22,6 @@ constexpr int SCT_THREADS = 192;
 constexpr int SCT_MAX_STAGES = 8;
 
 struct ScoreTcParams {
-  const __nv_bfloat16* W;
   float* logits;
   int B, C, d;
   int tiles_per_user, n_tiles;
@@ -31,7 +31,8 @@ struct ScoreTcParams {
 
 template <int ELL>
 __global__ void __launch_bounds__(SCT_THREADS, 1)
-k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmLS, const ScoreTcParams p) {
+k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmLS,
+           const __grid_constant__ CUtensorMap tmW, const ScoreTcParams p) {
   using namespace tc;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -39,7 +40,8 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
   const int KB = p.d / 64;                       // 64-element (128-byte) K blocks
   const uint32_t t_bytes = (uint32_t)KB * SCT_TILE * 128;
   const uint32_t ls_bytes = (uint32_t)KB * ELL * 128;
-  const uint32_t stage_bytes = t_bytes + ls_bytes;
+  constexpr uint32_t w_bytes = (uint32_t)SCT_TILE * ELL * 2;     // weight rows, not swizzled: row r at r * ELL * 2
+  const uint32_t stage_bytes = t_bytes + ls_bytes + w_bytes;
   const int S = p.stages;
 
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)S * stage_bytes);
@@ -56,11 +58,12 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
   const int t_end = (int)(((int64_t)(blockIdx.x + 1) * p.n_tiles) / gridDim.x);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 5); }   // MMA commit + 4 epilogue warps
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full[b], 1); mbar_init(&tmem_empty[b], 4); }
     fence_barrier_init();
     prefetch_tmap(&tmT);
     prefetch_tmap(&tmLS);
+    prefetch_tmap(&tmW);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TMEM_COLS);
@@ -92,9 +95,10 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
         for (int q = 0; q < SCT_MAX_STAGES; ++q)
           if (q == s) { load_ls = stage_user[q] != b; stage_user[q] = b; }
         uint8_t* st = smem + (size_t)s * stage_bytes;
-        mbar_arrive_expect_tx(&full[s], t_bytes + (load_ls ? ls_bytes : 0u));
+        mbar_arrive_expect_tx(&full[s], t_bytes + w_bytes + (load_ls ? ls_bytes : 0u));
         for (int kb = 0; kb < KB; ++kb)
           tma_load_2d_hint(st + (size_t)kb * SCT_TILE * 128, &tmT, kb * 64, row0, &full[s], pol_stream);
+        tma_load_2d_hint(st + t_bytes + ls_bytes, &tmW, 0, row0, &full[s], pol_stream);
         if (load_ls)
           for (int kb = 0; kb < KB; ++kb)
             tma_load_2d_hint(st + t_bytes + (size_t)kb * ELL * 128, &tmLS, kb * 64, b * ELL, &full[s], pol_keep);
@@ -147,36 +151,41 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
       const int c0 = (t % p.tiles_per_user) * SCT_TILE;
       const bool valid = c0 + r < p.C;
       const int64_t grow = (int64_t)b * p.C + c0 + r;
+      const int s = it % S;
+      if (!mbar_wait(&full[s], (uint32_t)(it / S) & 1u, p.err, 5)) break;
       uint4 w[ELL / 8];
-      if (valid) {
-        const uint4* wp = reinterpret_cast<const uint4*>(p.W + grow * ELL);
+      {
+        const uint4* wp = reinterpret_cast<const uint4*>(smem + (size_t)s * stage_bytes + t_bytes + ls_bytes) + r * (ELL / 8);
 #pragma unroll
-        for (int i = 0; i < ELL / 8; ++i) w[i] = __ldcs(wp + i);     // streamed once: evict-first
-      } else {
-#pragma unroll
-        for (int i = 0; i < ELL / 8; ++i) w[i] = make_uint4(0, 0, 0, 0);
+        for (int i = 0; i < ELL / 8; ++i) w[i] = wp[i];
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty[s]);       // this warp has taken its rows out of the stage
       if (!mbar_wait(&tmem_full[buf], bph, p.err, 4)) break;
       tc_fence_after();
-      float acc = 0.f;
+      // dot of the weight row with the accumulator row, CH columns per TMEM load, four independent partial sums
+      constexpr int CH = ELL >= 32 ? 32 : 16;
+      float acc4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int c = 0; c < ELL; c += 16) {
-        float v[16];
-        tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * ELL + c), v);
+      for (int c = 0; c < ELL; c += CH) {
+        float v[CH];
+        const uint32_t ta = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * ELL + c);
+        if constexpr (CH == 32) tmem_ld_32x32(ta, v); else tmem_ld_32x16(ta, v);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < CH / 8; ++i) {
           const uint4 u = w[c / 8 + i];
           const uint32_t uu[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float lo = __uint_as_float(uu[j] << 16);
             const float hi = __uint_as_float(uu[j] & 0xffff0000u);
-            acc = fmaf(lo, v[i * 8 + 2 * j], acc);
-            acc = fmaf(hi, v[i * 8 + 2 * j + 1], acc);
+            acc4[j] = fmaf(lo, v[i * 8 + 2 * j], acc4[j]);
+            acc4[j] = fmaf(hi, v[i * 8 + 2 * j + 1], acc4[j]);
           }
         }
       }
+      const float acc = (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[buf]);
@@ -194,7 +203,7 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
 
 // Shared-memory budget: S stages of (candidate tile + link states) + barriers + alignment slack.
 static int score_tc_stages(int ell, int d, size_t* smem_bytes) {
-  const size_t stage = (size_t)(d / 64) * (SCT_TILE + ell) * 128;
+  const size_t stage = (size_t)(d / 64) * (SCT_TILE + ell) * 128 + (size_t)SCT_TILE * ell * 2;
   const size_t fixed = 1024 + 2 * SCT_MAX_STAGES * 8 + 4 * 8 + 16;
   int S = (int)((226 * 1024 - fixed) / stage);
   if (S > SCT_MAX_STAGES) S = SCT_MAX_STAGES;
@@ -215,19 +224,20 @@ template <int ELL>
 static lime_status launch_score_tc_t(const ScoreArgs& a, int* err, cudaStream_t st) {
   size_t smem;
   const int S = score_tc_stages(ELL, a.d, &smem);
-  CUtensorMap tmT, tmLS;
+  CUtensorMap tmT, tmLS, tmW;
   if (!make_tmap_bf16_sw128(&tmT, a.T, (uint64_t)a.total, (uint64_t)a.d, (uint64_t)a.d, SCT_TILE) ||
-      !make_tmap_bf16_sw128(&tmLS, a.LS, (uint64_t)a.B * ELL, (uint64_t)a.d, (uint64_t)a.d, ELL))
+      !make_tmap_bf16_sw128(&tmLS, a.LS, (uint64_t)a.B * ELL, (uint64_t)a.d, (uint64_t)a.d, ELL) ||
+      !make_tmap_bf16_plain(&tmW, a.W, (uint64_t)a.total, ELL, ELL, SCT_TILE))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   ScoreTcParams p;
-  p.W = (const __nv_bfloat16*)a.W; p.logits = a.logits; p.B = a.B; p.C = a.C; p.d = a.d;
+  p.logits = a.logits; p.B = a.B; p.C = a.C; p.d = a.d;
   p.tiles_per_user = (a.C + SCT_TILE - 1) / SCT_TILE;
   p.n_tiles = p.tiles_per_user * a.B;
   p.stages = S; p.err = err;
   int grid = p.n_tiles < kSMs ? p.n_tiles : kSMs;
   LIME_CUDA(cudaFuncSetAttribute(k_score_tc<ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   ProfScope _p("k_score_tc", st);
-  k_score_tc<ELL><<<grid, SCT_THREADS, smem, st>>>(tmT, tmLS, p);
+  k_score_tc<ELL><<<grid, SCT_THREADS, smem, st>>>(tmT, tmLS, tmW, p);
   LIME_LAUNCH_CHECK("k_score_tc");
   return LIME_OK;
 }

@@ -311,15 +311,17 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->attn_scale = g.attn_scale > 0.f ? g.attn_scale : 1.0f / sqrtf((float)c->d_h);
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
-  c->keff = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
+  c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
+  if (e == cudaSuccess) e = cudaMalloc(&c->keff_hl, 2 * (size_t)2 * g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->dev_err, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->dev_err, 0, sizeof(int));
   if (e != cudaSuccess) {
     if (c->keff) cudaFree(c->keff);
+    if (c->keff_hl) cudaFree(c->keff_hl);
     if (c->links32) cudaFree(c->links32);
     if (c->dev_err) cudaFree(c->dev_err);
     delete c;
@@ -333,6 +335,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   if (!ctx) return LIME_OK;
   Ctx* c = reinterpret_cast<Ctx*>(ctx);
   cudaFree(c->keff);
+  cudaFree(c->keff_hl);
   cudaFree(c->links32);
   cudaFree(c->dev_err);
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); }
@@ -357,6 +360,8 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
   if (s != LIME_OK) return s;
   s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_scale, c->keff, st);
   if (s != LIME_OK) return s;
+  if (precompute_tc_supported(g.dtype, g.d, g.ell) && (s = launch_keff_split(c->keff, g.ell, g.d, c->keff_hl, st)) != LIME_OK)
+    return s;
   // tensor-core path: per layer, W_o as a K-major B operand ([d x d_ff], contraction index contiguous) and the
   // weight-only products that fold the history-side projections into the link rows
   if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) &&
@@ -402,6 +407,9 @@ lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb,
   if (!c->have_weights) return LIME_NOT_READY;
   if (M == 0) return LIME_OK;
   if (!cand_emb || !out_w || !aligned16(cand_emb) || !aligned16(out_w)) return LIME_INVALID_ARG;
+  if (precompute_tc_supported(c->cfg.dtype, c->cfg.d, c->cfg.ell))
+    return launch_precompute_tc(cand_emb, M, c->cfg.d, c->cfg.ell, c->keff_hl, out_w, c->dev_err,
+                                static_cast<cudaStream_t>(stream));
   return launch_precompute(c->cfg.dtype, cand_emb, M, c->cfg.d, c->cfg.ell, c->keff, out_w,
                            static_cast<cudaStream_t>(stream));
 }

@@ -51,6 +51,7 @@ struct Ctx {
   bool have_weights;
   int device;
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
+  void* keff_hl;    // [2 ell x d] bf16: keff split into a rounded part and its remainder (tensor-core precompute)
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
   void* WoT[LIME_MAX_LAYERS];    // tensor-core path, per layer (NULL otherwise): W_o transposed [d x d_ff] bf16,
   void* WprepT[LIME_MAX_LAYERS]; //   folded PREP operand [4*H*128 x d], folded link-row GLU operand [2*d_ff x H*d]
@@ -143,6 +144,12 @@ lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int
 // keff = ((L Wk) Wq^T) * scale, fp32 [ell x d]
 lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, float scale,
                         float* keff, cudaStream_t st);
+
+// bf16 precompute on tcgen05 tensor cores (ell in {16,32,64,128}, d % 64 == 0); keff_hl from launch_keff_split
+bool precompute_tc_supported(int dtype, int d, int ell);
+lime_status launch_keff_split(const float* keff, int ell, int d, void* keff_hl, cudaStream_t st);
+lime_status launch_precompute_tc(const void* cand, int64_t M, int d, int ell, const void* keff_hl, void* out_w, int* err,
+                                 cudaStream_t st);
 
 struct ScoreArgs {
   const void* LS; const void* W; const void* T; int dtype;

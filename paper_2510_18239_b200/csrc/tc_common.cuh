@@ -226,5 +226,8 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 // 128-byte swizzle.  Returns false if the driver entry point is unavailable or the encode fails.
 bool make_tmap_bf16_sw128(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
                           uint32_t box_rows);
+// Row-major bf16 matrix [rows x cols], cols <= 256, box [box_rows x cols] (whole rows), no swizzle.
+bool make_tmap_bf16_plain(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                          uint32_t box_rows);
 
 }  // namespace lime

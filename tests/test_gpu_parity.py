@@ -94,6 +94,31 @@ def test_precompute_matches_oracle(dtype, ell, d, M, proj):
     assert np.abs(got.sum(axis=1) - 1.0).max() <= (1e-5 if dtype == synth.F32 else 1e-2)
 
 
+@pytest.mark.parametrize("ell,d,M", [(16, 64, 148 * 128 * 9 + 77), (32, 128, 148 * 128 * 5 + 1), (128, 64, 30000),
+                                     (64, 256, 148 * 128 * 3 + 127)])
+def test_precompute_tensor_core_many_tiles(ell, d, M):
+    """bf16 precompute at sizes where every persistent CTA walks several tiles and wraps its stage ring, with a ragged
+    last tile; all rows against the oracle."""
+    Bd = _lib()
+    lime = Bd.Lime(d, max(1, d // 128), ell, 1, dtype=Bd.LIME_BF16, gated_mlp=False)
+    links = synth.normal_storage(5, "l", (ell, d), 1.0, synth.BF16)
+    T = synth.normal_storage(5, "c", (M, d), 1.0, synth.BF16)
+    Wq = synth.normal_storage(5, "cq", (d, d), d ** -0.5, synth.BF16)
+    lime.set_weights(Bd.to_device(links, synth.BF16), [{}], {"Wq": Bd.to_device(Wq, synth.BF16)})
+    W = lime.precompute_candidate_links(Bd.to_device(T, synth.BF16))
+    assert Bd.lime_device_status(lime.ctx) == 0
+    cfg = O.OracleConfig(d=d, H=1, ell=ell, n_layers=1)
+    T64, L64, Wq64 = (synth.storage_to_f64(x, synth.BF16) for x in (T, links, Wq))
+    s = (T64 @ Wq64) @ L64.T * cfg.c_scale                  # the oracle's definition, evaluated for all rows at once
+    e = np.exp(s - s.max(axis=1, keepdims=True))
+    want = e / e.sum(axis=1, keepdims=True)
+    rows = np.random.default_rng(0).integers(0, M, size=50)
+    assert np.abs(want[rows] - O.precompute_candidate_links(T64[rows], L64, cfg, Wq64, None)).max() < 1e-12
+    got = Hh.to_f64(W)
+    assert np.abs(got - want).max() <= 4e-3
+    assert np.abs(got.sum(axis=1) - 1.0).max() <= 1e-2
+
+
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 @pytest.mark.parametrize("B,C,ell,d", [(1, 1, 1, 8), (3, 50, 8, 64), (2, 300, 32, 128), (2, 129, 64, 256), (5, 77, 33, 40),
                                        (1, 128, 16, 64), (7, 1, 32, 128), (3, 2048, 32, 128), (160, 130, 64, 128),
