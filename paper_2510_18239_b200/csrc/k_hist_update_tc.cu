@@ -5,37 +5,51 @@
 // fused per 128-token tile into three chained tensor-core contractions whose operands never leave the SM:
 //   1. scores  [128 x HL]  = X_tile [128 x d] . K2^T               (K2 = folded link keys, see k_link_prep.cu)
 //      LayerNorm is applied afterwards as s = rstd_t * (raw - mu_t * rowsum(K2)), exact for the bf16 operands
-//   2. per-head softmax over the ell links of each token (one thread per token, registers only) -> P (bf16, smem)
+//   2. per-head softmax over the ell links of each token (registers only) -> P (bf16, smem)
 //   3. [gate | up] [128 x 2f] = P [128 x HL] . [G2 | U2]           (value mix and first GatedMLP layer folded)
 //   4. U = SiLU(gate) * up (bf16, smem)       5. S' = U [128 x f] . W_o [f x d]  -> bf16 rows to global
-// HL = H * ell stacked (head, link) rows.  Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 one
-// thread per token row (TMEM lane).  History is read once (TMA) and written once per layer.
+// HL = H * ell stacked (head, link) rows.  History is read once (TMA) and written once per layer.
 //
-// Built for d = d_ff = 128 and H * ell = 128 (shared memory: 2 x 32 KB token stages + 160 KB of operands;
-// TMEM: 128 + 256 + 128 columns).
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 token rows: two threads per token (TMEM lane), each
+// owning 64 of the 128 columns of every step (a warp may only touch the TMEM lane quarter warp_id % 4, so the two
+// halves of a row sit in warps w and w + 4).  The steps of consecutive tiles are software-pipelined so that the
+// tensor pipe works on one tile while the token warps work on the other:
+//   token warps, tile g :  store S'(g-1) | statistics of tile g+1 | SiLU(g) | softmax(g+1)
+//   MMA issuer,  tile g :  [gate|up](g)  | scores(g+1)            | S'(g)
+// TMEM: two 128-column buffers that hold a tile's scores and later its S' (alternating by tile), 256 columns
+// [gate | up].  Shared memory: one token stage (32 KB), K2, [G2 | U2], W_o (128 KB), two P/U buffers (64 KB).
+// Each thread takes the LayerNorm statistics of its own token row from the staged tile.
+//
+// With `out_ln` the rows are written already LayerNorm-ed (the next layer applies LayerNorm to every row it reads and
+// nothing else reads them, Eq. 8), so that the next layer's kernels run with LN = false.
+//
+// Built for d = d_ff = 128 and H * ell = 128.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
 
-constexpr int HU_D = 128, HU_F = 128, HU_HL = 128, HU_TILE = 128, HU_THREADS = 192;
+constexpr int HU_D = 128, HU_F = 128, HU_HL = 128, HU_TILE = 128;
+constexpr int HU_ROW_WARPS = 8, HU_THREADS = 64 + 32 * HU_ROW_WARPS;
 constexpr uint32_t HU_SUB = 128 * 128;                 // bytes of one [128 rows x 64 bf16] swizzled sub-tile
-constexpr uint32_t HU_X_STAGE = 2 * HU_SUB;            // token tile: 2 K-blocks
-constexpr uint32_t HU_OFF_X = 0;                       // 2 stages
-constexpr uint32_t HU_OFF_K2 = 2 * HU_X_STAGE;         // [HL x d]      2 K-blocks x 16 KB
+constexpr uint32_t HU_OFF_X = 0;                       // token tile: 2 K-blocks
+constexpr uint32_t HU_OFF_K2 = 2 * HU_SUB;             // [HL x d]      2 K-blocks x 16 KB
 constexpr uint32_t HU_OFF_GU = HU_OFF_K2 + 2 * HU_SUB; // [2f x HL]     2 K-blocks x 32 KB (gate rows, then up rows)
 constexpr uint32_t HU_OFF_WO = HU_OFF_GU + 4 * HU_SUB; // [d x f]       2 K-blocks x 16 KB
-constexpr uint32_t HU_OFF_PU = HU_OFF_WO + 2 * HU_SUB; // P, then U     2 K-blocks x 16 KB
-constexpr uint32_t HU_OFF_BAR = HU_OFF_PU + 2 * HU_SUB;
-constexpr uint32_t HU_OFF_CK = HU_OFF_BAR + 128;       // 4 per-warp copies of the [HL] key row sums (fp32)
-constexpr uint32_t HU_SMEM = HU_OFF_CK + 4 * HU_HL * 4; // 231,680 B of the 232,448 B an SM offers one CTA
+constexpr uint32_t HU_OFF_PU = HU_OFF_WO + 2 * HU_SUB; // 2 buffers (P, then U, of alternating tiles), 2 K-blocks each
+constexpr uint32_t HU_OFF_EXCH = HU_OFF_PU + 4 * HU_SUB;    // pair exchange: [2 halves][128] sums, then the same of squares
+constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 4 * 128 * 4;   // the current user's HL key row sums (fp32)
+constexpr uint32_t HU_OFF_BAR = HU_OFF_CK + HU_HL * 4;
+constexpr uint32_t HU_SMEM = HU_OFF_BAR + 256;              // 232,192 B of the 232,448 B one CTA may have
+static_assert(HU_SMEM <= 232448, "shared memory budget of one CTA");
+constexpr float HU_LOG2E = 1.4426950408889634f;
 
 struct HistUpdateParams {
   __nv_bfloat16* out;            // [total x d]
   const float* cK;               // [users x HL] row sums of K2
   const int32_t* off;            // [B+1]
   const int32_t* tile_start;     // [B+1] prefix of per-user tile counts (tile = 128 tokens)
-  int B, ell, shared, ln;
+  int B, ell, shared, out_ln;
   float ln_eps;
   int* err;
 };
@@ -60,8 +74,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ float tanh_approx(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Rendezvous of `count` warps on an mbarrier with a bounded wait; shared-memory writes made by any lane before the
+// call are visible to every participant after it.
+__device__ __forceinline__ bool hu_group_sync(uint64_t* bar, uint32_t& uses, int lane, int* err, int where) {
+  __syncwarp();
+  if (lane == 0) tc::mbar_arrive(bar);
+  const bool ok = tc::mbar_wait(bar, uses & 1u, err, where);
+  ++uses;
+  return ok;
+}
 
-template <int ELL>
+template <int ELL, bool LN>
 __global__ void __launch_bounds__(HU_THREADS, 1)
 k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmK2,
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
@@ -73,29 +101,34 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     return;
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HU_OFF_BAR);
-  uint64_t* x_full = bars;          // [2]  TMA -> MMA, epilogue
-  uint64_t* x_empty = bars + 2;     // [2]  MMA commit (1) + epilogue warps (4)
-  uint64_t* uops_full = bars + 4;   //      per user segment: K2, G2, U2 landed
-  uint64_t* uops_empty = bars + 5;  //      per user segment: last MMA reading them done
+  uint64_t* x_full = bars;           // token tile landed
+  uint64_t* x_empty = bars + 1;      // scores MMA done (1) + statistics taken by the 8 row warps
+  uint64_t* k2_full = bars + 2;      // per user segment
+  uint64_t* k2_empty = bars + 3;
+  uint64_t* ops_full = bars + 4;     // per user segment: G2, U2
+  uint64_t* ops_empty = bars + 5;
   uint64_t* wo_full = bars + 6;
-  uint64_t* s2_full = bars + 7;     // per tile, MMA1 done
-  uint64_t* p_ready = bars + 8;     // per tile, P in smem (4 warps)
-  uint64_t* gu_full = bars + 9;     // per tile, MMA2 done
-  uint64_t* u_ready = bars + 10;    // per tile, U in smem (4 warps)
-  uint64_t* sp_full = bars + 11;    // per tile, MMA3 done
-  uint64_t* sp_free = bars + 12;    // per tile, S' read out of TMEM (4 warps)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 13);
+  uint64_t* s2_full = bars + 7;      // per tile: scores in TMEM
+  uint64_t* p_ready = bars + 8;      // per tile: P in smem (8 warps)
+  uint64_t* gu_full = bars + 9;      // per tile: [gate | up] in TMEM
+  uint64_t* u_ready = bars + 10;     // per tile: U in smem (8 warps)
+  uint64_t* sp_full = bars + 11;     // per tile: S' in TMEM
+  uint64_t* sp_free = bars + 12;     // per tile: S' read out (8 warps)
+  uint64_t* pair_bar = bars + 13;    // [4] rendezvous of the two warps sharing a TMEM lane quarter
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tiles = p.tile_start[p.B];
-  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles) / gridDim.x);
-  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles) / gridDim.x);
+  const int n_tiles_all = p.tile_start[p.B];
+  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
+  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
+  const int n = t_end - t_begin;                            // tiles of this CTA, g = 0..n-1
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < 2; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 5); }
-    mbar_init(uops_full, 1); mbar_init(uops_empty, 1); mbar_init(wo_full, 1);
-    mbar_init(s2_full, 1); mbar_init(p_ready, 4); mbar_init(gu_full, 1); mbar_init(u_ready, 4);
-    mbar_init(sp_full, 1); mbar_init(sp_free, 4);
+    mbar_init(x_full, 1); mbar_init(x_empty, 1 + HU_ROW_WARPS);
+    mbar_init(k2_full, 1); mbar_init(k2_empty, 1); mbar_init(ops_full, 1); mbar_init(ops_empty, 1); mbar_init(wo_full, 1);
+    mbar_init(s2_full, 1); mbar_init(p_ready, HU_ROW_WARPS); mbar_init(gu_full, 1); mbar_init(u_ready, HU_ROW_WARPS);
+    mbar_init(sp_full, 1); mbar_init(sp_free, HU_ROW_WARPS);
+    for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
@@ -104,238 +137,321 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_S2 = 0, COL_GU = 128, COL_SP = 384;
+  constexpr uint32_t COL_SS = 0, COL_GU = 256;      // scores / S' buffer of tile g: COL_SS + (g & 1) * 128
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0 && t_begin < t_end) {
+    if (lane == 0 && n > 0) {
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
       mbar_arrive_expect_tx(wo_full, 2 * HU_SUB);
       for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + HU_OFF_WO + kb * HU_SUB, &tmWo, kb * 64, 0, wo_full, pol_keep);
-      int cur_user = -1, seg = 0, it = 0;
+      int cur_user = -1, seg = 0, g = 0;
       bool ok = true;
       TileUser tu;
-      for (int t = t_begin; t < t_end && ok; ++t, ++it) {
+      for (; g < n && ok; ++g) {
+        const int t = t_begin + g;
         const int b = tu.of(p.tile_start, p.B, t);
-        if (b != cur_user) {
-          if (seg > 0 && !mbar_wait(uops_empty, (uint32_t)(seg - 1) & 1u, p.err, 11)) { ok = false; break; }
+        if (b != cur_user && (seg == 0 || !p.shared)) {
           const int urow = p.shared ? 0 : b;
-          mbar_arrive_expect_tx(uops_full, 6 * HU_SUB);
+          if (seg > 0 && !mbar_wait(k2_empty, (uint32_t)(seg - 1) & 1u, p.err, 11)) { ok = false; break; }
+          mbar_arrive_expect_tx(k2_full, 2 * HU_SUB);
+          for (int kb = 0; kb < 2; ++kb)
+            tma_load_2d_hint(smem + HU_OFF_K2 + kb * HU_SUB, &tmK2, kb * 64, urow * HU_HL, k2_full, pol_keep);
+          if (seg > 0 && !mbar_wait(ops_empty, (uint32_t)(seg - 1) & 1u, p.err, 13)) { ok = false; break; }
+          mbar_arrive_expect_tx(ops_full, 4 * HU_SUB);
           for (int kb = 0; kb < 2; ++kb) {
-            tma_load_2d_hint(smem + HU_OFF_K2 + kb * HU_SUB, &tmK2, kb * 64, urow * HU_HL, uops_full, pol_keep);
-            tma_load_2d_hint(smem + HU_OFF_GU + kb * 2 * HU_SUB, &tmG, kb * 64, urow * HU_F, uops_full, pol_keep);
-            tma_load_2d_hint(smem + HU_OFF_GU + kb * 2 * HU_SUB + HU_SUB, &tmU, kb * 64, urow * HU_F, uops_full, pol_keep);
+            tma_load_2d_hint(smem + HU_OFF_GU + kb * 2 * HU_SUB, &tmG, kb * 64, urow * HU_F, ops_full, pol_keep);
+            tma_load_2d_hint(smem + HU_OFF_GU + kb * 2 * HU_SUB + HU_SUB, &tmU, kb * 64, urow * HU_F, ops_full, pol_keep);
           }
-          cur_user = b;
           ++seg;
         }
-        const int s = it & 1;
-        if (!mbar_wait(&x_empty[s], ((uint32_t)(it >> 1) & 1u) ^ 1u, p.err, 12)) { ok = false; break; }
+        cur_user = b;
+        if (g > 0 && !mbar_wait(x_empty, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
         const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
-        mbar_arrive_expect_tx(&x_full[s], HU_X_STAGE);
-        for (int kb = 0; kb < 2; ++kb)
-          tma_load_2d_hint(smem + HU_OFF_X + s * HU_X_STAGE + kb * HU_SUB, &tmX, kb * 64, row0, &x_full[s], pol_stream);
+        mbar_arrive_expect_tx(x_full, 2 * HU_SUB);
+        for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + HU_OFF_X + kb * HU_SUB, &tmX, kb * 64, row0, x_full, pol_stream);
       }
       if (!ok || *(volatile int*)p.err != 0) {
-        for (int j = 0; j < it && j < 2; ++j) mbar_wait_quiet(&x_full[(it - 1 - j) & 1], (uint32_t)((it - 1 - j) >> 1) & 1u);
-        if (seg > 0) mbar_wait_quiet(uops_full, (uint32_t)(seg - 1) & 1u);
+        // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
+        if (g > 0) mbar_wait_quiet(x_full, (uint32_t)(g - 1) & 1u);
+        if (seg > 0) { mbar_wait_quiet(k2_full, (uint32_t)(seg - 1) & 1u); mbar_wait_quiet(ops_full, (uint32_t)(seg - 1) & 1u); }
         mbar_wait_quiet(wo_full, 0);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && t_begin < t_end) {
+    if (lane == 0 && n > 0) {
       constexpr uint32_t idesc_128 = make_idesc_bf16(128, 128);
       constexpr uint32_t idesc_256 = make_idesc_bf16(128, 256);
       const uint32_t sbase = smem_u32(smem);
-      int cur_user = -1, seg = 0, it = 0;
-      bool ok = mbar_wait(wo_full, 0, p.err, 21);
       TileUser tu;
-      for (int t = t_begin; t < t_end && ok; ++t, ++it) {
-        const int b = tu.of(p.tile_start, p.B, t);
-        const uint32_t tp = (uint32_t)it & 1u;
-        if (b != cur_user) {
-          if (!mbar_wait(uops_full, (uint32_t)seg & 1u, p.err, 22)) break;
-          cur_user = b;
-          ++seg;
+      int user_of_scores = -1, user_of_mix = -1, seg_k = 0, seg_o = 0;
+      // does tile g close its user's run of tiles inside this CTA (so that the user's operands may be replaced)?
+      auto last_of_user = [&](int g) {
+        if (p.shared) return false;
+        const int t = t_begin + g;
+        tu.of(p.tile_start, p.B, t);
+        return g + 1 < n && t + 1 >= tu.hi;
+      };
+      // 1. scores(g) = X . K2^T
+      auto issue_scores = [&](int g) -> bool {
+        const int b = tu.of(p.tile_start, p.B, t_begin + g);
+        if (b != user_of_scores && (seg_k == 0 || !p.shared)) {
+          if (!mbar_wait(k2_full, (uint32_t)seg_k & 1u, p.err, 22)) return false;
+          ++seg_k;
         }
-        const int s = it & 1;
-        if (!mbar_wait(&x_full[s], (uint32_t)(it >> 1) & 1u, p.err, 23)) break;
+        user_of_scores = b;
+        if (g >= 2 && !mbar_wait(sp_free, (uint32_t)(g - 2) & 1u, p.err, 26)) return false;   // S'(g-2) shared the buffer
+        if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 23)) return false;
         tc_fence_after();
-        // 1. scores = X . K2^T
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (uint32_t)(kk >> 2) * HU_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_S2, make_sdesc_k_sw128(sbase + HU_OFF_X + s * HU_X_STAGE + o),
+          mma_bf16_ss(tmem_base + COL_SS + (uint32_t)(g & 1) * 128, make_sdesc_k_sw128(sbase + HU_OFF_X + o),
                       make_sdesc_k_sw128(sbase + HU_OFF_K2 + o), idesc_128, kk != 0);
         }
-        mma_commit(&x_empty[s]);
+        mma_commit(x_empty);
         mma_commit(s2_full);
-        // 3. [gate | up] = P . [G2 | U2]
+        if (last_of_user(g)) mma_commit(k2_empty);
+        return true;
+      };
+      bool ok = mbar_wait(wo_full, 0, p.err, 21);
+      if (ok) ok = issue_scores(0);
+      for (int g = 0; g < n && ok; ++g) {
+        const uint32_t tp = (uint32_t)g & 1u;
+        const uint32_t pu = sbase + HU_OFF_PU + (uint32_t)(g & 1) * 2 * HU_SUB;
+        // 3. [gate | up](g) = P(g) . [G2 | U2]
+        const int b = tu.of(p.tile_start, p.B, t_begin + g);
+        if (b != user_of_mix && (seg_o == 0 || !p.shared)) {
+          if (!mbar_wait(ops_full, (uint32_t)seg_o & 1u, p.err, 27)) break;
+          ++seg_o;
+        }
+        user_of_mix = b;
         if (!mbar_wait(p_ready, tp, p.err, 24)) break;
         tc_fence_after();
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t oa = (uint32_t)(kk >> 2) * HU_SUB + (uint32_t)(kk & 3) * 32;
           const uint32_t ob = (uint32_t)(kk >> 2) * 2 * HU_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_GU, make_sdesc_k_sw128(sbase + HU_OFF_PU + oa),
-                      make_sdesc_k_sw128(sbase + HU_OFF_GU + ob), idesc_256, kk != 0);
+          mma_bf16_ss(tmem_base + COL_GU, make_sdesc_k_sw128(pu + oa), make_sdesc_k_sw128(sbase + HU_OFF_GU + ob), idesc_256,
+                      kk != 0);
         }
         mma_commit(gu_full);
-        // the user's operands are free once the last tile of the segment has issued its MMAs on them
-        const bool last_of_user = (t + 1 == t_end) || (t + 1 >= tu.hi);
-        if (last_of_user) mma_commit(uops_empty);
-        // 5. S' = U . W_o
+        if (last_of_user(g)) mma_commit(ops_empty);
+        // 1'. scores of the next tile, while the row warps turn [gate | up](g) into U(g)
+        if (g + 1 < n && !issue_scores(g + 1)) break;
+        // 5. S'(g) = U(g) . W_o, into the buffer that held scores(g)
         if (!mbar_wait(u_ready, tp, p.err, 25)) break;
-        if (it > 0 && !mbar_wait(sp_free, (uint32_t)(it - 1) & 1u, p.err, 26)) break;
         tc_fence_after();
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (uint32_t)(kk >> 2) * HU_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_SP, make_sdesc_k_sw128(sbase + HU_OFF_PU + o),
+          mma_bf16_ss(tmem_base + COL_SS + (uint32_t)(g & 1) * 128, make_sdesc_k_sw128(pu + o),
                       make_sdesc_k_sw128(sbase + HU_OFF_WO + o), idesc_128, kk != 0);
         }
         mma_commit(sp_full);
       }
     }
-  } else {
-    // ------------------------------------------------------------------ token-row warps (2..5)
-    const int q = warp & 3;
-    const uint32_t r = (uint32_t)(q * 32 + lane);           // token row of the tile == TMEM lane
+  } else if (n > 0) {
+    // ------------------------------------------------------------------ token-row warps (2..9)
+    const int rw = warp - 2;                                 // 0..7
+    const int q = warp & 3;                                  // TMEM lane quarter of this warp
+    const int half = rw >> 2;                                // which 64 columns of every step
+    const uint32_t r = (uint32_t)(q * 32 + lane);            // token row of the tile == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    uint8_t* pu = smem + HU_OFF_PU;
-    float* ck_s = reinterpret_cast<float*>(smem + HU_OFF_CK) + (warp - 2) * HU_HL;   // this warp's own copy
-    int cur_user = -1, it = 0;
-    constexpr int H = HU_HL / ELL;
+    float* exch = reinterpret_cast<float*>(smem + HU_OFF_EXCH);                 // [2 slots][2 halves][128]
+    float* ck_s = reinterpret_cast<float*>(smem + HU_OFF_CK) + half * 64;      // key row sums of this thread's 64 columns
+    uint32_t pair_uses = 0;
+    int ck_user = -1;
+    bool ok = true;
     TileUser tu;
-    for (int t = t_begin; t < t_end; ++t, ++it) {
-      const int b = tu.of(p.tile_start, p.B, t);
-      const uint32_t tp = (uint32_t)it & 1u;
-      const int s = it & 1;
-      if (b != cur_user) {
-        __syncwarp();                                         // every lane is done with the previous user's sums
-        for (int i = lane; i < HU_HL; i += 32) ck_s[i] = p.cK[(int64_t)(p.shared ? 0 : b) * HU_HL + i];
-        __syncwarp();
-        cur_user = b;
-      }
-      const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
-      const bool valid = row0 + (int)r < p.off[b + 1];
-      // LayerNorm statistics of this thread's token from the staged tile (two passes, rotated chunk order)
-      if (!mbar_wait(&x_full[s], (uint32_t)(it >> 1) & 1u, p.err, 31)) break;
-      float mu = 0.f, rstd = 1.f;
-      if (p.ln) {
-        const uint8_t* xs = smem + HU_OFF_X + s * HU_X_STAGE + r * 128u;
+    float sA = HU_LOG2E, sB = 0.f;                           // this row's rstd * log2e and -mu * rstd * log2e
+
+    // LayerNorm statistics of this thread's token row of tile g, straight from the staged tile (both threads of a
+    // row compute them: cheaper than an exchange); then the stage is released
+    auto take_stats = [&](int g) -> bool {
+      if (LN) {
+        if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 31)) return false;
+        const uint8_t* xs = smem + HU_OFF_X + r * 128u;
+        uint4 u[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) u[c] = *reinterpret_cast<const uint4*>(xs + (c >> 3) * HU_SUB + (((c + (int)r) & 7) << 4));
         float sum = 0.f;
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
-          const int cc = (c + (int)r) & 7;
-          const uint4 u = *reinterpret_cast<const uint4*>(xs + (c >> 3) * HU_SUB + cc * 16);
-          const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+          const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) sum += __uint_as_float(w[j] << 16) + __uint_as_float(w[j] & 0xffff0000u);
         }
-        mu = sum * (1.0f / HU_D);
-        float var = 0.f;
+        const float mu = sum * (1.0f / HU_D);
+        float var0 = 0.f, var1 = 0.f;
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
-          const int cc = (c + (int)r) & 7;
-          const uint4 u = *reinterpret_cast<const uint4*>(xs + (c >> 3) * HU_SUB + cc * 16);
-          const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+          const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float a = __uint_as_float(w[j] << 16) - mu, bb = __uint_as_float(w[j] & 0xffff0000u) - mu;
-            var = fmaf(a, a, var);
-            var = fmaf(bb, bb, var);
+            var0 = fmaf(a, a, var0);
+            var1 = fmaf(bb, bb, var1);
           }
         }
-        rstd = rsqrtf(var * (1.0f / HU_D) + p.ln_eps);
+        const float rstd = rsqrtf((var0 + var1) * (1.0f / HU_D) + p.ln_eps);
+        sA = rstd * HU_LOG2E;
+        sB = -mu * sA;
+        __syncwarp();
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&x_empty[s]);
+      if (lane == 0) mbar_arrive(x_empty);                   // this warp is done with the staged tile
+      return true;
+    };
 
-      // 2. per-head softmax over the links, P -> smem (A operand of the next MMA, K-major, 128B swizzle)
-      if (!mbar_wait(s2_full, tp, p.err, 32)) break;
+    // 2. per-head softmax over the links of this thread's heads (64 score columns), P -> smem
+    auto softmax = [&](int g) -> bool {
+      const int b = tu.of(p.tile_start, p.B, t_begin + g);
+      if (!mbar_wait(s2_full, (uint32_t)g & 1u, p.err, 32)) return false;
       tc_fence_after();
+      if (LN && b != ck_user && (ck_user < 0 || !p.shared)) {
+        // scores(g) exist, so every warp has finished the softmax of tile g-1 (its P was needed first): nobody still
+        // reads the previous user's sums.  The four warps of a half write identical values.
+        for (int i = lane; i < 64; i += 32) ck_s[i] = p.cK[(int64_t)(p.shared ? 0 : b) * HU_HL + half * 64 + i];
+        __syncwarp();
+      }
+      ck_user = b;
+      float v[64];
+      {
+        float v0[32], v1[32];
+        const uint32_t ta = lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + half * 64;
+        tmem_ld_32x32(ta, v0);
+        tmem_ld_32x32(ta + 32, v1);
+        tmem_wait_ld();
 #pragma unroll
-      for (int h = 0; h < H; ++h) {
-        float sc[ELL];
+        for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
+      }
+      uint8_t* pu = smem + HU_OFF_PU + (g & 1) * 2 * HU_SUB + half * HU_SUB;   // K-block `half` holds columns 64*half..
 #pragma unroll
-        for (int c = 0; c < ELL; c += 16) {
-          float v[16];
-          tmem_ld_32x16(lane_addr + COL_S2 + h * ELL + c, v);
-          tmem_wait_ld();
+      for (int h = 0; h < 64 / ELL; ++h) {
+        float mx = -INFINITY;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) sc[c + j] = (v[j] - mu * ck_s[h * ELL + c + j]) * rstd;
+        for (int j = 0; j < ELL; ++j) {
+          const int c = h * ELL + j;
+          v[c] = LN ? fmaf(v[c], sA, ck_s[c] * sB) : v[c] * HU_LOG2E;
+          mx = fmaxf(mx, v[c]);
         }
-        float mx = sc[0];
+        float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int j = 1; j < ELL; ++j) mx = fmaxf(mx, sc[j]);
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < ELL; ++j) { sc[j] = __expf(sc[j] - mx); sum += sc[j]; }
-        const float inv = 1.f / sum;
+        for (int j = 0; j < ELL; j += 2) {
+          v[h * ELL + j] = exp2f(v[h * ELL + j] - mx);
+          v[h * ELL + j + 1] = exp2f(v[h * ELL + j + 1] - mx);
+          s0 += v[h * ELL + j];
+          s1 += v[h * ELL + j + 1];
+        }
+        const float inv = 1.f / (s0 + s1);
 #pragma unroll
         for (int c8 = 0; c8 < ELL / 8; ++c8) {
-          const int k = h * ELL + c8 * 8;                    // first of 8 consecutive contraction indices
+          const int c = h * ELL + c8 * 8;                    // first of 8 consecutive contraction indices
           uint4 o;
-          o.x = pack_bf16(sc[c8 * 8 + 0] * inv, sc[c8 * 8 + 1] * inv);
-          o.y = pack_bf16(sc[c8 * 8 + 2] * inv, sc[c8 * 8 + 3] * inv);
-          o.z = pack_bf16(sc[c8 * 8 + 4] * inv, sc[c8 * 8 + 5] * inv);
-          o.w = pack_bf16(sc[c8 * 8 + 6] * inv, sc[c8 * 8 + 7] * inv);
-          *reinterpret_cast<uint4*>(pu + (k >> 6) * HU_SUB + sw128_chunk(r, (uint32_t)(k & 63) >> 3)) = o;
+          o.x = pack_bf16(v[c + 0] * inv, v[c + 1] * inv);
+          o.y = pack_bf16(v[c + 2] * inv, v[c + 3] * inv);
+          o.z = pack_bf16(v[c + 4] * inv, v[c + 5] * inv);
+          o.w = pack_bf16(v[c + 6] * inv, v[c + 7] * inv);
+          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, (uint32_t)c >> 3)) = o;
         }
       }
       tc_fence_before();
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(p_ready);
+      return true;
+    };
 
-      // 4. U = SiLU(gate) * up -> smem (over P, which the second MMA has finished reading)
-      if (!mbar_wait(gu_full, tp, p.err, 33)) break;
+    // 4. U = SiLU(gate) * up for this thread's 64 hidden columns -> smem (over P(g), which [gate|up](g) has read)
+    auto silu_mul = [&](int g) -> bool {
+      if (!mbar_wait(gu_full, (uint32_t)g & 1u, p.err, 33)) return false;
       tc_fence_after();
+      uint8_t* pu = smem + HU_OFF_PU + (g & 1) * 2 * HU_SUB + half * HU_SUB;
 #pragma unroll
-      for (int c = 0; c < HU_F; c += 16) {
-        float g[16], u[16];
-        tmem_ld_32x16(lane_addr + COL_GU + c, g);
-        tmem_ld_32x16(lane_addr + COL_GU + HU_F + c, u);
+      for (int c = 0; c < 64; c += 32) {
+        float gt[32], up[32];
+        tmem_ld_32x32(lane_addr + COL_GU + half * 64 + c, gt);
+        tmem_ld_32x32(lane_addr + COL_GU + HU_F + half * 64 + c, up);
         tmem_wait_ld();
-        float y[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) y[j] = silu_f(g[j]) * u[j];
+        for (int c8 = 0; c8 < 4; ++c8) {
+          float y[8];
 #pragma unroll
-        for (int c8 = 0; c8 < 2; ++c8) {
-          const int k = c + c8 * 8;
+          for (int j = 0; j < 8; ++j) {
+            const float x = gt[c8 * 8 + j];
+            const float hx = 0.5f * x;
+            y[j] = fmaf(hx, tanh_approx(hx), hx) * up[c8 * 8 + j];    // x * sigmoid(x) = x/2 * (1 + tanh(x/2))
+          }
           uint4 o;
-          o.x = pack_bf16(y[c8 * 8 + 0], y[c8 * 8 + 1]);
-          o.y = pack_bf16(y[c8 * 8 + 2], y[c8 * 8 + 3]);
-          o.z = pack_bf16(y[c8 * 8 + 4], y[c8 * 8 + 5]);
-          o.w = pack_bf16(y[c8 * 8 + 6], y[c8 * 8 + 7]);
-          *reinterpret_cast<uint4*>(pu + (k >> 6) * HU_SUB + sw128_chunk(r, (uint32_t)(k & 63) >> 3)) = o;
+          o.x = pack_bf16(y[0], y[1]); o.y = pack_bf16(y[2], y[3]); o.z = pack_bf16(y[4], y[5]); o.w = pack_bf16(y[6], y[7]);
+          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, (uint32_t)(c >> 3) + c8)) = o;
         }
       }
       tc_fence_before();
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(u_ready);
+      return true;
+    };
 
-      // 6. S' row -> bf16 -> global
-      if (!mbar_wait(sp_full, tp, p.err, 34)) break;
+    // 6. this thread's 64 columns of its S' row -> (LayerNorm) -> bf16 -> global
+    auto store_rows = [&](int g) -> bool {
+      const int t = t_begin + g;
+      const int b = tu.of(p.tile_start, p.B, t);
+      const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
+      const bool valid = row0 + (int)r < p.off[b + 1];
+      if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 34)) return false;
       tc_fence_after();
-      uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * HU_D);
-#pragma unroll
-      for (int c = 0; c < HU_D; c += 16) {
-        float v[16];
-        tmem_ld_32x16(lane_addr + COL_SP + c, v);
+      float v[64];
+      {
+        float v0[32], v1[32];
+        const uint32_t ta = lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + half * 64;
+        tmem_ld_32x32(ta, v0);
+        tmem_ld_32x32(ta + 32, v1);
         tmem_wait_ld();
-        if (valid) {
-          uint4 o0, o1;
-          o0.x = pack_bf16(v[0], v[1]); o0.y = pack_bf16(v[2], v[3]); o0.z = pack_bf16(v[4], v[5]); o0.w = pack_bf16(v[6], v[7]);
-          o1.x = pack_bf16(v[8], v[9]); o1.y = pack_bf16(v[10], v[11]); o1.z = pack_bf16(v[12], v[13]); o1.w = pack_bf16(v[14], v[15]);
-          dst[c / 8] = o0;
-          dst[c / 8 + 1] = o1;
-        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(sp_free);
+      if (p.out_ln) {
+        float s = 0.f;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) s += v[j];
+        // separate slots for the two exchanges: each is rewritten only after a later rendezvous of the same pair
+        exch[half * 128 + r] = s;
+        if (!hu_group_sync(&pair_bar[q], pair_uses, lane, p.err, 37)) return false;
+        const float mu = (s + exch[(half ^ 1) * 128 + r]) * (1.0f / HU_D);
+        float var = 0.f;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
+        exch[256 + half * 128 + r] = var;
+        if (!hu_group_sync(&pair_bar[q], pair_uses, lane, p.err, 39)) return false;
+        const float rstd = rsqrtf((var + exch[256 + (half ^ 1) * 128 + r]) * (1.0f / HU_D) + p.ln_eps);
+#pragma unroll
+        for (int j = 0; j < 64; ++j) v[j] *= rstd;
+      }
+      if (valid) {
+        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * HU_D + half * 64);
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          uint4 o;
+          o.x = pack_bf16(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = pack_bf16(v[c8 * 8 + 2], v[c8 * 8 + 3]);
+          o.z = pack_bf16(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = pack_bf16(v[c8 * 8 + 6], v[c8 * 8 + 7]);
+          dst[c8] = o;
+        }
+      }
+      return true;
+    };
+
+    ok = take_stats(0) && softmax(0);
+    for (int g = 0; g < n && ok; ++g) {
+      if (g > 0 && !store_rows(g - 1)) { ok = false; break; }
+      // statistics of the next tile as soon as it has landed, so that its stage can be refilled a whole tile early
+      if (g + 1 < n && !take_stats(g + 1)) { ok = false; break; }
+      if (!silu_mul(g)) { ok = false; break; }
+      if (g + 1 < n && !softmax(g + 1)) { ok = false; break; }
     }
+    if (ok) store_rows(n - 1);
   }
 
   tc_fence_before();
@@ -363,12 +479,17 @@ static lime_status launch_hu(const HistUpdateArgs& a, cudaStream_t st) {
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   HistUpdateParams p;
   p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.ell = ELL;
-  p.shared = a.shared; p.ln = a.ln; p.ln_eps = a.ln_eps; p.err = a.err;
+  p.shared = a.shared; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
   int grid = a.n_tile_upper < kSMs ? a.n_tile_upper : kSMs;
   if (grid < 1) return LIME_OK;
-  LIME_CUDA(cudaFuncSetAttribute(k_hist_update_tc<ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)HU_SMEM));
   ProfScope _p("k_hist_update_tc", st);
-  k_hist_update_tc<ELL><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  if (a.ln) {
+    LIME_CUDA(cudaFuncSetAttribute(k_hist_update_tc<ELL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)HU_SMEM));
+    k_hist_update_tc<ELL, true><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  } else {
+    LIME_CUDA(cudaFuncSetAttribute(k_hist_update_tc<ELL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)HU_SMEM));
+    k_hist_update_tc<ELL, false><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  }
   LIME_LAUNCH_CHECK("k_hist_update_tc");
   return LIME_OK;
 }

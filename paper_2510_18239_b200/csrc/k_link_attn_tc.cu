@@ -9,11 +9,17 @@
 //                         s_ij = rstd_j * (raw_ij - mu_j * rowsum(Q2)_i)
 //   acc    [HL x d]    += P' [HL x 128] . X_tile            P'_ij = p_ij * rstd_j;  the mean term sum_j P'_ij mu_j is
 //                                                           a per-row scalar subtracted from every column at the end
-//   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (chunks merged in k_link_prep.cu, W_V folded into the GEMM after)
-// HL = H * ell stacked (head, link) rows = 128 TMEM lanes; thread i of the softmax warps owns row i: an online
-// softmax whose reference maximum is only raised when the true maximum exceeds it by more than 8 (then the
-// accumulator row is rescaled in TMEM), so most tiles need no correction pass.
-// One CTA per (user, chunk of the history); warp 0 TMA producer, warp 1 MMA issuer, warps 2-5 softmax.
+//   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (W_V is folded into the GEMM that follows)
+// HL = H * ell stacked (head, link) rows = 128 TMEM lanes.  Online softmax in the log2 domain whose reference
+// maximum is only raised when the true maximum exceeds it by more than 8 (then the accumulator row is rescaled in
+// TMEM), so most tiles need no correction pass.
+//
+// Persistent CTAs walk (user, chunk-of-history) items.  Warp roles: warp 0 TMA producer (runs ahead across items),
+// warp 1 MMA issuer, warps 2-9 softmax: two threads per (head, link) row, each owning 64 of the tile's 128 token
+// columns (a warp may only touch the TMEM lane quarter warp_id % 4, so the two halves of a row sit in warps w and
+// w + 4 and exchange their row maximum through shared memory).  A user whose history is a single chunk is
+// normalised and written directly; longer histories leave (max, sum, accumulator) partials per chunk that
+// k_link_attn_merge_norm combines.
 //
 // Built for d = 128 and H * ell = 128.
 #include "lime_common.cuh"
@@ -21,24 +27,28 @@
 
 namespace lime {
 
-constexpr int LA_D = 128, LA_HL = 128, LA_TILE = 128, LA_THREADS = 192, LA_XSTAGES = 3;
+constexpr int LA_D = 128, LA_HL = 128, LA_TILE = 128, LA_XSTAGES = 3;
+constexpr int LA_SOFTMAX_WARPS = 8, LA_THREADS = 64 + 32 * LA_SOFTMAX_WARPS;
 constexpr uint32_t LA_SUB = 128 * 128;
 constexpr uint32_t LA_X_STAGE = 2 * LA_SUB;
 constexpr uint32_t LA_OFF_X = 0;
 constexpr uint32_t LA_OFF_Q2 = LA_XSTAGES * LA_X_STAGE;
 constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_SUB;        // 2 buffers of [HL x 128 tokens]
-constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 4 * LA_SUB;     // per X stage: mu[128], rstd[128]
-constexpr uint32_t LA_OFF_BAR = LA_OFF_STATS + LA_XSTAGES * 2 * 128 * 4;
+constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 4 * LA_SUB;     // per X stage: float4 {rstd*log2e, -mu*rstd*log2e, rstd, mu} x 128
+constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 16;   // 2 x 2 x 128 maxima, 2 x 128 sums, 2 x 128 mean terms
+constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 8 * 128 * 4;
 constexpr uint32_t LA_SMEM = LA_OFF_BAR + 256;
-constexpr float LA_RESCALE_THRESHOLD = 8.0f;
+constexpr float LA_RESCALE_THRESHOLD = 8.0f;                 // in log2 units
+constexpr float LA_LOG2E = 1.4426950408889634f;
 
 struct LinkAttnParams {
   const float* cQ;                // [users x HL]
   const int32_t* off;
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
-  int B, chunk, shared, ln;
+  int B, chunk, shared, ell, H;
   float ln_eps;
   float *part_m, *part_s, *part_acc;   // [items x HL], [items x HL], [items x HL x d]
+  __nv_bfloat16* Ohat;                 // [B*ell x H*d]: final rows of single-chunk users
   int* err;
 };
 
@@ -47,12 +57,22 @@ __device__ __forceinline__ uint32_t la_pack(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+// Rendezvous of `count` warps on an mbarrier (every wait in this kernel is bounded, so no bar.sync): shared-memory
+// writes made by any lane before the call are visible to every participant after it.
+__device__ __forceinline__ bool la_group_sync(uint64_t* bar, uint32_t& uses, int lane, int* err, int where) {
+  __syncwarp();
+  if (lane == 0) tc::mbar_arrive(bar);
+  const bool ok = tc::mbar_wait(bar, uses & 1u, err, where);
+  ++uses;
+  return ok;
+}
 
+template <bool LN>
 __global__ void __launch_bounds__(LA_THREADS, 1)
 k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttnParams p) {
   using namespace tc;
-  const int item = blockIdx.x;
-  if (item >= p.chunk_start[p.B]) return;
+  const int n_items = p.chunk_start[p.B];
+  if ((int)blockIdx.x >= n_items) return;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {
     if (threadIdx.x == 0) atomicCAS(p.err, 0, 91);
@@ -61,23 +81,25 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LA_OFF_BAR);
   uint64_t* x_full = bars;             // [3]
   uint64_t* x_empty = bars + 3;        // [3]  second MMA of the tile done
-  uint64_t* stats_ready = bars + 6;    // [3]  128 arrivals
-  uint64_t* q_full = bars + 9;
-  uint64_t* s_full = bars + 10;        // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 12;       // [2]  P' in smem (4 warps)
-  uint64_t* p_free = bars + 14;        // [2]  second MMA done reading P' (and accumulator up to date)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+  uint64_t* q_full = bars + 6;         //      folded queries of the item's user landed
+  uint64_t* q_empty = bars + 7;        //      every score MMA of the item has read them
+  uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
+  uint64_t* p_ready = bars + 10;       // [2]  P' in smem (8 warps)
+  uint64_t* p_free = bars + 12;        // [2]  second MMA done reading P' (and accumulator up to date)
+  uint64_t* o_free = bars + 14;        //      accumulator of the item read out (8 warps)
+  uint64_t* stats_bar = bars + 15;     //      rendezvous of the 8 softmax warps (token statistics written)
+  uint64_t* pair_bar = bars + 16;      // [4]  rendezvous of the two warps that share a TMEM lane quarter
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = upper_user(p.chunk_start, p.B, item);
-  const int tok0 = p.off[b] + (item - p.chunk_start[b]) * p.chunk;
-  const int tok1 = min(p.off[b + 1], tok0 + p.chunk);
-  const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); mbar_init(&stats_ready[s], 128); }
-    mbar_init(q_full, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 4); mbar_init(&p_free[i], 1); }
+    for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
+    mbar_init(q_full, 1); mbar_init(q_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], LA_SOFTMAX_WARPS); mbar_init(&p_free[i], 1); }
+    mbar_init(o_free, LA_SOFTMAX_WARPS);
+    mbar_init(stats_bar, LA_SOFTMAX_WARPS);
+    for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
@@ -88,27 +110,46 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   const uint32_t tmem_base = *tmem_slot;
   constexpr uint32_t COL_S = 0, COL_O = 256;      // scores: 2 x 128 columns; accumulator: d columns
 
+  // item -> (user, token range); identical in every role
+  auto item_range = [&](int item, int& b, int& tok0, int& tok1) {
+    b = upper_user(p.chunk_start, p.B, item);
+    tok0 = p.off[b] + (item - p.chunk_start[b]) * p.chunk;
+    tok1 = min(p.off[b + 1], tok0 + p.chunk);
+  };
+
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
-      mbar_arrive_expect_tx(q_full, 2 * LA_SUB);
-      for (int kb = 0; kb < 2; ++kb)
-        tma_load_2d_hint(smem + LA_OFF_Q2 + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * LA_HL, q_full, pol_keep);
       bool ok = true;
-      int t = 0;
-      for (; t < n_tiles; ++t) {
-        const int s = t % LA_XSTAGES;
-        if (!mbar_wait(&x_empty[s], ((uint32_t)(t / LA_XSTAGES) & 1u) ^ 1u, p.err, 41)) { ok = false; break; }
-        mbar_arrive_expect_tx(&x_full[s], LA_X_STAGE);
-        for (int kb = 0; kb < 2; ++kb)
-          tma_load_2d_hint(smem + LA_OFF_X + s * LA_X_STAGE + kb * LA_SUB, &tmX, kb * 64, tok0 + t * LA_TILE, &x_full[s],
-                           pol_stream);
+      int g = 0, qn = 0, prev_user = -1;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        int b, tok0, tok1;
+        item_range(item, b, tok0, tok1);
+        const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
+        prev_user = b;
+        if (load_q) {
+          if (qn > 0 && !mbar_wait(q_empty, (uint32_t)(qn - 1) & 1u, p.err, 42)) { ok = false; break; }
+          mbar_arrive_expect_tx(q_full, 2 * LA_SUB);
+          for (int kb = 0; kb < 2; ++kb)
+            tma_load_2d_hint(smem + LA_OFF_Q2 + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * LA_HL, q_full, pol_keep);
+          ++qn;
+        }
+        const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
+        for (int t = 0; t < n_tiles; ++t, ++g) {
+          const int s = g % LA_XSTAGES;
+          if (!mbar_wait(&x_empty[s], ((uint32_t)(g / LA_XSTAGES) & 1u) ^ 1u, p.err, 41)) { ok = false; break; }
+          mbar_arrive_expect_tx(&x_full[s], LA_X_STAGE);
+          for (int kb = 0; kb < 2; ++kb)
+            tma_load_2d_hint(smem + LA_OFF_X + s * LA_X_STAGE + kb * LA_SUB, &tmX, kb * 64, tok0 + t * LA_TILE, &x_full[s],
+                             pol_stream);
+        }
       }
       if (!ok || *(volatile int*)p.err != 0) {
-        for (int j = 0; j < t && j < LA_XSTAGES; ++j)
-          mbar_wait_quiet(&x_full[(t - 1 - j) % LA_XSTAGES], (uint32_t)((t - 1 - j) / LA_XSTAGES) & 1u);
-        mbar_wait_quiet(q_full, 0);
+        // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
+        for (int j = 0; j < g && j < LA_XSTAGES; ++j)
+          mbar_wait_quiet(&x_full[(g - 1 - j) % LA_XSTAGES], (uint32_t)((g - 1 - j) / LA_XSTAGES) & 1u);
+        if (qn > 0) mbar_wait_quiet(q_full, (uint32_t)(qn - 1) & 1u);
       }
     }
   } else if (warp == 1) {
@@ -117,72 +158,102 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128);                 // Q2 . X^T  : both K-major
       constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);    // P' . X    : B is MN-major
       const uint32_t sbase = smem_u32(smem);
-      auto issue_scores = [&](int t) -> bool {
-        const int s = t % LA_XSTAGES;
-        if (!mbar_wait(&x_full[s], (uint32_t)(t / LA_XSTAGES) & 1u, p.err, 51)) return false;
+      auto issue_scores = [&](int g) -> bool {
+        const int s = g % LA_XSTAGES;
+        if (!mbar_wait(&x_full[s], (uint32_t)(g / LA_XSTAGES) & 1u, p.err, 51)) return false;
         tc_fence_after();
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(t & 1) * 128, make_sdesc_k_sw128(sbase + LA_OFF_Q2 + o),
+          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * 128, make_sdesc_k_sw128(sbase + LA_OFF_Q2 + o),
                       make_sdesc_k_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + o), idesc_s, kk != 0);
         }
-        mma_commit(&s_full[t & 1]);
+        mma_commit(&s_full[g & 1]);
         return true;
       };
-      bool ok = mbar_wait(q_full, 0, p.err, 50);
-      if (ok && n_tiles > 0) ok = issue_scores(0);
-      for (int t = 0; t < n_tiles && ok; ++t) {
-        // the next tile's scores overlap this tile's softmax (its score buffer was released by p_ready(t-1))
-        if (t + 1 < n_tiles && !issue_scores(t + 1)) { ok = false; break; }
-        const int s = t % LA_XSTAGES, pb = t & 1;
-        if (!mbar_wait(&p_ready[pb], (uint32_t)(t >> 1) & 1u, p.err, 52)) { ok = false; break; }
-        tc_fence_after();
-        for (int kk = 0; kk < 8; ++kk) {      // contraction over the tile's 128 tokens, 16 per instruction
-          const uint32_t oa = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + pb * 2 * LA_SUB + oa),
-                      make_sdesc_mn_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + (uint32_t)kk * 2048, LA_SUB), idesc_o,
-                      (t | kk) != 0);
+      bool ok = true;
+      int g = 0, qn = 0, k = 0, prev_user = -1;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
+        int b, tok0, tok1;
+        item_range(item, b, tok0, tok1);
+        const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
+        prev_user = b;
+        if (load_q) {
+          if (!mbar_wait(q_full, (uint32_t)qn & 1u, p.err, 50)) { ok = false; break; }
+          ++qn;
         }
-        mma_commit(&x_empty[s]);
-        mma_commit(&p_free[pb]);
+        // will the producer replace the queries after this item?
+        bool next_reloads = false;
+        if (!p.shared && item + (int)gridDim.x < n_items) next_reloads = upper_user(p.chunk_start, p.B, item + gridDim.x) != b;
+        const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
+        if (!issue_scores(g)) { ok = false; break; }
+        if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
+        for (int t = 0; t < n_tiles; ++t, ++g) {
+          // the next tile's scores overlap this tile's softmax (its score buffer was released by p_ready(g-1))
+          if (t + 1 < n_tiles) {
+            if (!issue_scores(g + 1)) { ok = false; break; }
+            if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
+          }
+          const int s = g % LA_XSTAGES, pb = g & 1;
+          if (!mbar_wait(&p_ready[pb], (uint32_t)(g >> 1) & 1u, p.err, 52)) { ok = false; break; }
+          // the first tile of an item overwrites the accumulator: the previous item must have been read out
+          if (t == 0 && k > 0 && !mbar_wait(o_free, (uint32_t)(k - 1) & 1u, p.err, 53)) { ok = false; break; }
+          tc_fence_after();
+          for (int kk = 0; kk < 8; ++kk) {      // contraction over the tile's 128 tokens, 16 per instruction
+            const uint32_t oa = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
+            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + pb * 2 * LA_SUB + oa),
+                        make_sdesc_mn_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + (uint32_t)kk * 2048, LA_SUB), idesc_o,
+                        (t | kk) != 0);
+          }
+          mma_commit(&x_empty[s]);
+          mma_commit(&p_free[pb]);
+        }
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax warps (2..5): thread i owns row i
-    const int q = warp & 3;
-    const uint32_t r = (uint32_t)(q * 32 + lane);
+    // ------------------------------------------------------------------ softmax warps (2..9)
+    const int sw = warp - 2;                                   // 0..7
+    const int q = warp & 3;                                    // TMEM lane quarter of this warp
+    const int half = sw >> 2;                                  // which 64 token columns of the tile
+    const uint32_t r = (uint32_t)(q * 32 + lane);              // (head, link) row == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    const float cq = p.cQ[(int64_t)(p.shared ? 0 : b) * LA_HL + r];
-    float m_ref = -INFINITY, l_sum = 0.f, mean_corr = 0.f;
+    float4* stats = reinterpret_cast<float4*>(smem + LA_OFF_STATS);
+    float* exch_max = reinterpret_cast<float*>(smem + LA_OFF_EXCH);          // [2 tile parities][2 halves][128]
+    float* exch_sum = exch_max + 4 * 128;                                    // [2][128]
+    float* exch_mean = exch_sum + 2 * 128;                                   // [2][128]
     bool ok = true;
-    for (int t = 0; t < n_tiles && ok; ++t) {
-      const int s = t % LA_XSTAGES, pb = t & 1;
-      const uint32_t xph = (uint32_t)(t / LA_XSTAGES) & 1u;
-      float* mu_s = reinterpret_cast<float*>(smem + LA_OFF_STATS) + s * 256;
-      float* rstd_s = mu_s + 128;
-      const int nvalid = min(LA_TILE, tok1 - tok0 - t * LA_TILE);
-      // LayerNorm statistics of token r of this tile (each thread one token), shared through smem
-      if (!mbar_wait(&x_full[s], xph, p.err, 61)) { ok = false; break; }
-      {
-        float mu = 0.f, rstd = 1.f;
-        if (p.ln) {
-          const uint8_t* xs = smem + LA_OFF_X + s * LA_X_STAGE + r * 128u;
+    int g = 0, k = 0;
+    uint32_t stats_uses = 0, pair_uses = 0;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
+      int b, tok0, tok1;
+      item_range(item, b, tok0, tok1);
+      const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
+      const float cq = LN ? p.cQ[(int64_t)(p.shared ? 0 : b) * LA_HL + r] : 0.f;
+      float m_ref = -INFINITY, l_sum = 0.f, mean_corr = 0.f;
+      for (int t = 0; t < n_tiles && ok; ++t, ++g) {
+        const int s = g % LA_XSTAGES, pb = g & 1;
+        const int nvalid = min(LA_TILE, tok1 - tok0 - t * LA_TILE);
+        const float4* st = stats + s * 128;
+        if (LN) {
+          // LayerNorm statistics of the tile's tokens: two lanes per token, 64 features each, held in registers
+          if (!mbar_wait(&x_full[s], (uint32_t)(g / LA_XSTAGES) & 1u, p.err, 61)) { ok = false; break; }
+          const int tok = 16 * sw + (lane >> 1), hf = lane & 1;
+          const uint8_t* xs = smem + LA_OFF_X + s * LA_X_STAGE + hf * LA_SUB + tok * 128;
+          uint4 u[8];
+#pragma unroll
+          for (int c = 0; c < 8; ++c) u[c] = *reinterpret_cast<const uint4*>(xs + (((c + tok + 4 * hf) & 7) << 4));
           float sum = 0.f;
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const int cc = (c + (int)r) & 7;
-            const uint4 u = *reinterpret_cast<const uint4*>(xs + (c >> 3) * LA_SUB + cc * 16);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+          for (int c = 0; c < 8; ++c) {
+            const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) sum += __uint_as_float(w[j] << 16) + __uint_as_float(w[j] & 0xffff0000u);
           }
-          mu = sum * (1.0f / LA_D);
+          sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+          const float mu = sum * (1.0f / LA_D);
           float var = 0.f;
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const int cc = (c + (int)r) & 7;
-            const uint4 u = *reinterpret_cast<const uint4*>(xs + (c >> 3) * LA_SUB + cc * 16);
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+          for (int c = 0; c < 8; ++c) {
+            const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const float a = __uint_as_float(w[j] << 16) - mu, bb = __uint_as_float(w[j] & 0xffff0000u) - mu;
@@ -190,106 +261,140 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
               var = fmaf(bb, bb, var);
             }
           }
-          rstd = rsqrtf(var * (1.0f / LA_D) + p.ln_eps);
+          var += __shfl_xor_sync(0xffffffffu, var, 1);
+          const float rstd = rsqrtf(var * (1.0f / LA_D) + p.ln_eps);
+          if (hf == 0) stats[s * 128 + tok] = make_float4(rstd * LA_LOG2E, -mu * rstd * LA_LOG2E, rstd, mu);
+          if (!la_group_sync(stats_bar, stats_uses, lane, p.err, 62)) { ok = false; break; }
         }
-        mu_s[r] = mu;
-        rstd_s[r] = rstd;
-        mbar_arrive(&stats_ready[s]);
-      }
-      if (!mbar_wait(&stats_ready[s], xph, p.err, 62)) { ok = false; break; }
-      if (!mbar_wait(&s_full[pb], (uint32_t)(t >> 1) & 1u, p.err, 63)) { ok = false; break; }
-      tc_fence_after();
-
-      // pass 1: row maximum of the tile's valid scores
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < LA_TILE; c += 16) {
-        float v[16];
-        tmem_ld_32x16(lane_addr + COL_S + pb * 128 + c, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float sc = (v[j] - cq * mu_s[c + j]) * rstd_s[c + j];
-          if (c + j < nvalid) mx = fmaxf(mx, sc);
-        }
-      }
-      // raise the reference maximum only when it is exceeded by more than the threshold (or unset)
-      const bool need = mx > m_ref + LA_RESCALE_THRESHOLD;
-      const float m_new = need ? mx : m_ref;
-      const float factor = (need && m_ref != -INFINITY) ? __expf(m_ref - m_new) : 1.0f;
-      if (__any_sync(0xffffffffu, need && t > 0)) {
-        // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this row
-        if (!mbar_wait(&p_free[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u, p.err, 64)) { ok = false; break; }
+        if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
         tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < LA_D; c += 16) {
-          float v[16];
-          tmem_ld_32x16(lane_addr + COL_O + c, v);
+
+        // pass 1: this thread's 64 scores (log2 domain) into registers, and their maximum
+        float v[64];
+        {
+          float v0[32], v1[32];
+          tmem_ld_32x32(lane_addr + COL_S + pb * 128 + half * 64, v0);
+          tmem_ld_32x32(lane_addr + COL_S + pb * 128 + half * 64 + 32, v1);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] *= factor;
-          tmem_st_32x16(lane_addr + COL_O + c, v);
+          for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
         }
-        tmem_wait_st();
-      }
-      l_sum *= factor;
-      mean_corr *= factor;
-      m_ref = m_new;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          if (LN) {
+            const float4 c4 = st[half * 64 + j];
+            v[j] = fmaf(v[j], c4.x, cq * c4.y);
+          } else {
+            v[j] *= LA_LOG2E;
+          }
+          if (half * 64 + j < nvalid) mx = fmaxf(mx, v[j]);
+        }
+        exch_max[(pb * 2 + half) * 128 + r] = mx;
+        if (!la_group_sync(&pair_bar[q], pair_uses, lane, p.err, 67)) { ok = false; break; }
+        mx = fmaxf(mx, exch_max[(pb * 2 + (half ^ 1)) * 128 + r]);
 
-      // the P' buffer of two tiles ago must have been consumed
-      if (t >= 2 && !mbar_wait(&p_free[pb], (uint32_t)((t - 2) >> 1) & 1u, p.err, 65)) { ok = false; break; }
-      // pass 2: p = exp(s - m_ref); P' = p * rstd -> smem (A operand, K-major over the tile's tokens)
-      uint8_t* pbuf = smem + LA_OFF_P + pb * 2 * LA_SUB;
+        // raise the reference maximum only when it is exceeded by more than the threshold (or unset)
+        const bool need = mx > m_ref + LA_RESCALE_THRESHOLD;
+        const float m_new = need ? mx : m_ref;
+        const float factor = (need && m_ref != -INFINITY) ? exp2f(m_ref - m_new) : 1.0f;
+        if (__any_sync(0xffffffffu, need && t > 0)) {
+          // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this half-row
+          if (!mbar_wait(&p_free[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, p.err, 64)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-      for (int c = 0; c < LA_TILE; c += 16) {
-        float v[16];
-        tmem_ld_32x16(lane_addr + COL_S + pb * 128 + c, v);
-        tmem_wait_ld();
-        float pp[16];
+          for (int c = 0; c < 64; c += 16) {
+            float a[16];
+            tmem_ld_32x16(lane_addr + COL_O + half * 64 + c, a);
+            tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float rs = rstd_s[c + j], mj = mu_s[c + j];
-          const float sc = (v[j] - cq * mj) * rs;
-          const float e = (c + j < nvalid) ? __expf(sc - m_ref) : 0.f;
-          l_sum += e;
-          // what the MMA will see is the bf16-rounded P'; use the same rounded value for the mean term
-          const float pr = __bfloat162float(__float2bfloat16_rn(e * rs));
-          mean_corr = fmaf(pr, mj, mean_corr);
-          pp[j] = pr;
+            for (int j = 0; j < 16; ++j) a[j] *= factor;
+            tmem_st_32x16(lane_addr + COL_O + half * 64 + c, a);
+          }
+          tmem_wait_st();
         }
+        l_sum *= factor;
+        mean_corr *= factor;
+        m_ref = m_new;
+
+        // the P' buffer of two tiles ago must have been consumed
+        if (g >= 2 && !mbar_wait(&p_free[pb], (uint32_t)((g - 2) >> 1) & 1u, p.err, 65)) { ok = false; break; }
+        // pass 2: p = 2^(s - m_ref); P' = p * rstd -> smem (A operand, K-major over the tile's tokens)
+        uint8_t* pbuf = smem + LA_OFF_P + pb * 2 * LA_SUB + half * LA_SUB;
 #pragma unroll
-        for (int c8 = 0; c8 < 2; ++c8) {
-          const int k = c + c8 * 8;
+        for (int c8 = 0; c8 < 8; ++c8) {
+          float pp[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int col = c8 * 8 + j;
+            const float e = (half * 64 + col < nvalid) ? exp2f(v[col] - m_ref) : 0.f;
+            l_sum += e;
+            if (LN) {
+              const float4 c4 = st[half * 64 + col];
+              // what the MMA will see is the bf16-rounded P'; use the same rounded value for the mean term
+              const float pr = __bfloat162float(__float2bfloat16_rn(e * c4.z));
+              mean_corr = fmaf(pr, c4.w, mean_corr);
+              pp[j] = pr;
+            } else {
+              pp[j] = e;
+            }
+          }
           uint4 o;
-          o.x = la_pack(pp[c8 * 8 + 0], pp[c8 * 8 + 1]);
-          o.y = la_pack(pp[c8 * 8 + 2], pp[c8 * 8 + 3]);
-          o.z = la_pack(pp[c8 * 8 + 4], pp[c8 * 8 + 5]);
-          o.w = la_pack(pp[c8 * 8 + 6], pp[c8 * 8 + 7]);
-          *reinterpret_cast<uint4*>(pbuf + (k >> 6) * LA_SUB + la_chunk_addr(r, (uint32_t)(k & 63) >> 3)) = o;
+          o.x = la_pack(pp[0], pp[1]); o.y = la_pack(pp[2], pp[3]); o.z = la_pack(pp[4], pp[5]); o.w = la_pack(pp[6], pp[7]);
+          *reinterpret_cast<uint4*>(pbuf + la_chunk_addr(r, (uint32_t)c8)) = o;
         }
+        tc_fence_before();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_ready[pb]);
+      }
+      if (!ok) break;
+      // item result: wait for the last second MMA, combine the two halves' sums, read the accumulator half-row
+      const int gl = g - 1;
+      if (!mbar_wait(&p_free[gl & 1], (uint32_t)(gl >> 1) & 1u, p.err, 66)) { ok = false; break; }
+      tc_fence_after();
+      exch_sum[half * 128 + r] = l_sum;
+      exch_mean[half * 128 + r] = mean_corr;
+      if (!la_group_sync(&pair_bar[q], pair_uses, lane, p.err, 68)) { ok = false; break; }
+      const float l_tot = l_sum + exch_sum[(half ^ 1) * 128 + r];
+      const float c_tot = mean_corr + exch_mean[(half ^ 1) * 128 + r];
+      float a[64];
+      {
+        float a0[32], a1[32];
+        tmem_ld_32x32(lane_addr + COL_O + half * 64, a0);
+        tmem_ld_32x32(lane_addr + COL_O + half * 64 + 32, a1);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) { a[j] = a0[j]; a[32 + j] = a1[j]; }
       }
       tc_fence_before();
-      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&p_ready[pb]);
-    }
-    // chunk result: (m_ref, sum, accumulator row minus the mean term) -> scratch, merged per user afterwards
-    if (ok && n_tiles > 0) ok = mbar_wait(&p_free[(n_tiles - 1) & 1], (uint32_t)((n_tiles - 1) >> 1) & 1u, p.err, 66);
-    if (ok) {
-      tc_fence_after();
-      float* dst = p.part_acc + ((int64_t)item * LA_HL + r) * LA_D;
+      if (lane == 0) mbar_arrive(o_free);
+      const bool single = p.chunk_start[b + 1] - p.chunk_start[b] == 1;
+      if (single) {
+        // the whole history of this user was one chunk: normalise and write the attention rows directly
+        const float inv = 1.0f / l_tot;
+        const int h = (int)r / p.ell, l = (int)r % p.ell;
+        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + ((int64_t)b * p.ell + l) * (p.H * LA_D) + h * LA_D + half * 64);
 #pragma unroll
-      for (int c = 0; c < LA_D; c += 16) {
-        float v[16];
-        tmem_ld_32x16(lane_addr + COL_O + c, v);
-        tmem_wait_ld();
+        for (int c8 = 0; c8 < 8; ++c8) {
+          uint4 o;
+          o.x = la_pack((a[c8 * 8 + 0] - c_tot) * inv, (a[c8 * 8 + 1] - c_tot) * inv);
+          o.y = la_pack((a[c8 * 8 + 2] - c_tot) * inv, (a[c8 * 8 + 3] - c_tot) * inv);
+          o.z = la_pack((a[c8 * 8 + 4] - c_tot) * inv, (a[c8 * 8 + 5] - c_tot) * inv);
+          o.w = la_pack((a[c8 * 8 + 6] - c_tot) * inv, (a[c8 * 8 + 7] - c_tot) * inv);
+          dst[c8] = o;
+        }
+      } else {
+        float4* dst = reinterpret_cast<float4*>(p.part_acc + ((int64_t)item * LA_HL + r) * LA_D + half * 64);
 #pragma unroll
-        for (int j = 0; j < 16; j += 4)
-          *reinterpret_cast<float4*>(dst + c + j) =
-              make_float4(v[j] - mean_corr, v[j + 1] - mean_corr, v[j + 2] - mean_corr, v[j + 3] - mean_corr);
+        for (int j = 0; j < 64; j += 4)
+          dst[j / 4] = make_float4(a[j] - c_tot, a[j + 1] - c_tot, a[j + 2] - c_tot, a[j + 3] - c_tot);
+        if (half == 0) {
+          p.part_m[(int64_t)item * LA_HL + r] = m_ref;        // log2 domain
+          p.part_s[(int64_t)item * LA_HL + r] = l_tot;
+        }
       }
-      p.part_m[(int64_t)item * LA_HL + r] = m_ref;
-      p.part_s[(int64_t)item * LA_HL + r] = l_sum;
     }
   }
 
@@ -314,13 +419,18 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   LinkAttnParams p;
   p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
-  p.ln = a.ln; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc; p.err = a.err;
-  LIME_CUDA(cudaFuncSetAttribute(k_link_attn_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LA_SMEM));
-  {
-    ProfScope _p("k_link_attn_tc", st);
-    k_link_attn_tc<<<a.n_chunk_upper, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
-    LIME_LAUNCH_CHECK("k_link_attn_tc");
+  p.ell = a.ell; p.H = a.H; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
+  p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
+  const int grid = a.n_chunk_upper < kSMs ? a.n_chunk_upper : kSMs;
+  ProfScope _p("k_link_attn_tc", st);
+  if (a.ln) {
+    LIME_CUDA(cudaFuncSetAttribute(k_link_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LA_SMEM));
+    k_link_attn_tc<true><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
+  } else {
+    LIME_CUDA(cudaFuncSetAttribute(k_link_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LA_SMEM));
+    k_link_attn_tc<false><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
   }
+  LIME_LAUNCH_CHECK("k_link_attn_tc");
   return LIME_OK;
 }
 

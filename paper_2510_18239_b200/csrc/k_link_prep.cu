@@ -86,15 +86,17 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
   return LIME_OK;
 }
 
-// Combine the chunks of a user with log-sum-exp weights and normalise:
-//   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = exp(m_c - max_c m_c)
-// grid (B * H * ell), block d threads.  A user without history gets zeros.
+// Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
+//   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
+// grid (B * H * ell), block d threads.  A user without history gets zeros; a user with a single chunk was
+// already written by the attention kernel.
 __global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H,
                                        const float* __restrict__ part_m, const float* __restrict__ part_s,
                                        const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
   const int HL = H * ell;
   const int u = blockIdx.x / HL, row = blockIdx.x % HL, h = row / ell, l = row % ell;
   const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
+  if (c1 - c0 == 1) return;
   const int i = threadIdx.x;
   float out = 0.f;
   if (c1 > c0) {
@@ -102,7 +104,7 @@ __global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, 
     for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
     float S = 0.f, O = 0.f;
     for (int c = c0; c < c1; ++c) {
-      const float w = __expf(part_m[(int64_t)c * HL + row] - M);
+      const float w = exp2f(part_m[(int64_t)c * HL + row] - M);
       S = fmaf(part_s[(int64_t)c * HL + row], w, S);
       O = fmaf(part_acc[((int64_t)c * HL + row) * d + i], w, O);
     }

@@ -103,11 +103,14 @@ static bool layer_on_tensor_cores(const Ctx* c, int layer) {
 }
 
 // One XOR layer, tensor-core path: three link-row GEMMs around the two streaming attention kernels.
+// `in_prenorm`: hist_in holds LayerNorm-ed rows already (written by the previous layer with `out_ln`); `out_ln`:
+// write LayerNorm(S') to hist_out.  Both are internal to lime_encode_user; the public layer call passes 0, 0.
 static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B, int64_t total,
                                 const float* links_in, int links_shared, void* hist_out, float* links_out,
-                                const Workspace& w, cudaStream_t st) {
+                                const Workspace& w, int in_prenorm, int out_ln, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
+  const int hist_ln = (g.ln && !in_prenorm) ? 1 : 0;
   const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
   const int64_t BL = (int64_t)B * g.ell;
   // LN(T) -> bf16, then one GEMM gives every folded link-side operand of both attention directions
@@ -121,7 +124,7 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
   LinkAttnArgs la{};
   la.hist = hist_in; la.total = total; la.Q2 = w.Q2; la.cQ = w.cQ; la.off = off; la.chunk_start = w.chunk_start; la.B = B;
   la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = links_shared;
-  la.ln = g.ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.err = c->dev_err;
+  la.ln = hist_ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat; la.err = c->dev_err;
   if ((s = launch_link_attn_tc(la, st)) != LIME_OK) return s;
   if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
     return s;
@@ -137,8 +140,8 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
     HistUpdateArgs hu{};
     hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
     hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
-    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = g.ln; hu.ln_eps = c->ln_eps;
-    hu.err = c->dev_err;
+    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
+    hu.out_ln = out_ln; hu.err = c->dev_err;
     if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
   }
   return LIME_OK;
@@ -147,7 +150,8 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
 // One XOR layer on a carved workspace (see lime_xor_layer in lime.h for the contract).
 static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B,
                                   int64_t total, const float* links_in, int links_shared, void* hist_out,
-                                  float* links_out, const Workspace& w, bool schedules_ready, cudaStream_t st) {
+                                  float* links_out, const Workspace& w, bool schedules_ready, int in_prenorm, int out_ln,
+                                  cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
   if (!schedules_ready) {
@@ -155,7 +159,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
     if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
   }
   if (layer_on_tensor_cores(c, layer))
-    return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, st);
+    return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, in_prenorm, out_ln, st);
 
   // ---- generic path on CUDA cores (fp32 storage, other shapes, SiLU attention, no GatedMLP) ----
   const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
@@ -429,7 +433,7 @@ lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hist_in, co
   const size_t pad = base - static_cast<char*>(ws);
   Workspace w = carve(c, base, B, total_tokens);
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
-  return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false,
+  return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false, 0, 0,
                         static_cast<cudaStream_t>(stream));
 }
 
@@ -457,7 +461,11 @@ lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off
     const bool last = j == g.n_layers - 1;
     const float* lin = j == 0 ? (link_ctx ? link_ctx : c->links32) : w.T;
     const int shared = (j == 0 && !link_ctx) ? 1 : 0;
-    s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true, st);
+    // tensor-core path: between layers the history is kept LayerNorm-ed (every consumer normalises it first, Eq. 1
+    // with App. C's LayerNorm), so only the first layer pays for the statistics
+    const int keep_norm = (g.ln && layer_on_tensor_cores(c, j)) ? 1 : 0;
+    s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true,
+                       j > 0 ? keep_norm : 0, last ? 0 : keep_norm, st);
     if (s != LIME_OK) return s;
     if ((s = launch_axpy(w.T, w.LP, BLd, j == 0, st)) != LIME_OK) return s;   // L^P = sum_j T^j  (Eq. 8)
   }

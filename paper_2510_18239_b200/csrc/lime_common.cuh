@@ -188,6 +188,7 @@ struct LinkAttnArgs {
   const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
   int ell, d, H, shared, ln; float ln_eps;
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
+  void* Ohat;                               // [B*ell x H*d] bf16: rows of users whose history is one chunk
   int* err;
 };
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi);
@@ -197,7 +198,8 @@ struct HistUpdateArgs {
   const void* hist_in; void* hist_out; int64_t total;
   const void *K2, *G2t, *U2t; const float* cK; const void* WoT;   // WoT [d x f] bf16 (W_o transposed)
   const int32_t* off; const int32_t* tile_start; int B, n_tile_upper;
-  int ell, shared, ln; float ln_eps;
+  int ell, shared, ln; float ln_eps;    // ln: apply LayerNorm to the rows read (0 when they were stored normalised)
+  int out_ln;                           // 1: store LayerNorm(S') instead of S'
   int* err;
 };
 bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
