@@ -3,46 +3,49 @@
 //   S'[t,:] = GatedMLP( O[S]_t ),   O[S]_t = concat_h softmax_l( Q[S]_{t,h} K[T]_{l,h}^T * scale ) V[T]_{l,h}     (Eq. 7, Eq. 5)
 //
 // fused per 128-token tile into three chained tensor-core contractions whose operands never leave the SM:
-//   1. scores  [128 x HL]  = X_tile [128 x d] . K2^T               (K2 = folded link keys, see k_link_prep.cu)
-//      LayerNorm is applied afterwards as s = rstd_t * (raw - mu_t * rowsum(K2)), exact for the bf16 operands
+//   1. scores  [128 x HL]  = X_tile [128 x d] . K2^T               (K2 = folded link keys, see k_link_prep.cu; the fold
+//      carries scale * log2(e)).  LayerNorm is applied afterwards as s = rstd_t * (raw - mu_t * rowsum(K2)), exact
+//      for the bf16 operands
 //   2. per-head softmax over the ell links of each token (registers only) -> P (bf16, smem)
 //   3. [gate | up] [128 x 2f] = P [128 x HL] . [G2 | U2]           (value mix and first GatedMLP layer folded)
 //   4. U = SiLU(gate) * up (bf16, smem)       5. S' = U [128 x f] . W_o [f x d]  -> bf16 rows to global
 // HL = H * ell stacked (head, link) rows.  History is read once (TMA) and written once per layer.
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 token rows: two threads per token (TMEM lane), each
-// owning 64 of the 128 columns of every step (a warp may only touch the TMEM lane quarter warp_id % 4, so the two
-// halves of a row sit in warps w and w + 4).  The steps of consecutive tiles are software-pipelined so that the
-// tensor pipe works on one tile while the token warps work on the other:
-//   token warps, tile g :  store S'(g-1) | statistics of tile g+1 | SiLU(g) | softmax(g+1)
-//   MMA issuer,  tile g :  [gate|up](g)  | scores(g+1)            | S'(g)
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 token rows: four threads per token (TMEM lane), each
+// owning 32 of the 128 columns of every step - one head of the softmax when ell = 32 (a warp may only touch the TMEM
+// lane quarter warp_id % 4, so the four parts of a row sit in warps w, w + 4, w + 8, w + 12).  Four warps per
+// scheduler keep the issue slots busy while TMEM loads and transcendentals are in flight.  The steps of consecutive
+// tiles are software-pipelined so that the tensor pipe works on one tile while the token warps work on the other:
+//   token warps, tile g :  SiLU(g) | statistics of tile g+1 | softmax(g+1) | store S'(g)
+//   MMA issuer,  tile g :  [gate|up](g) , scores(g+1) | S'(g)             | [gate|up](g+1) ...
 // TMEM: two 128-column buffers that hold a tile's scores and later its S' (alternating by tile), 256 columns
-// [gate | up].  Shared memory: one token stage (32 KB), K2, [G2 | U2], W_o (128 KB), two P/U buffers (64 KB).
-// Each thread takes the LayerNorm statistics of its own token row from the staged tile.
+// [gate | up].  Shared memory: one token stage (32 KB), K2, [G2 | U2], W_o (128 KB), one P/U buffer (32 KB).
 //
 // With `out_ln` the rows are written already LayerNorm-ed (the next layer applies LayerNorm to every row it reads and
 // nothing else reads them, Eq. 8), so that the next layer's kernels run with LN = false.
 //
-// Built for d = d_ff = 128 and H * ell = 128.
+// Built for d = d_ff = 128, H * ell = 128 and ell in {16, 32}.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
 
 constexpr int HU_D = 128, HU_F = 128, HU_HL = 128, HU_TILE = 128;
-constexpr int HU_ROW_WARPS = 8, HU_THREADS = 64 + 32 * HU_ROW_WARPS;
+constexpr int HU_PARTS = 4;                            // threads per token row
+constexpr int HU_COLS = 128 / HU_PARTS;                // columns per thread in every step
+constexpr int HU_ROW_WARPS = 4 * HU_PARTS, HU_THREADS = 64 + 32 * HU_ROW_WARPS;
 constexpr uint32_t HU_SUB = 128 * 128;                 // bytes of one [128 rows x 64 bf16] swizzled sub-tile
 constexpr uint32_t HU_OFF_X = 0;                       // token tile: 2 K-blocks
 constexpr uint32_t HU_OFF_K2 = 2 * HU_SUB;             // [HL x d]      2 K-blocks x 16 KB
 constexpr uint32_t HU_OFF_GU = HU_OFF_K2 + 2 * HU_SUB; // [2f x HL]     2 K-blocks x 32 KB (gate rows, then up rows)
 constexpr uint32_t HU_OFF_WO = HU_OFF_GU + 4 * HU_SUB; // [d x f]       2 K-blocks x 16 KB
-constexpr uint32_t HU_OFF_PU = HU_OFF_WO + 2 * HU_SUB; // 2 buffers (P, then U, of alternating tiles), 2 K-blocks each
-constexpr uint32_t HU_OFF_EXCH = HU_OFF_PU + 4 * HU_SUB;    // pair exchange: [2 halves][128] sums, then the same of squares
-constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 4 * 128 * 4;   // the current user's HL key row sums (fp32)
+constexpr uint32_t HU_OFF_PU = HU_OFF_WO + 2 * HU_SUB; // P, then U, of the current tile: 2 K-blocks
+constexpr uint32_t HU_OFF_STATS = HU_OFF_PU + 2 * HU_SUB;   // 2 (tile parity) x 128 float2 {rstd, mu}
+constexpr uint32_t HU_OFF_EXCH = HU_OFF_STATS + 2 * 128 * 8;   // row exchange: [PARTS][128] sums, then the same of squares
+constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 2 * HU_PARTS * 128 * 4;   // the current user's HL key row sums (fp32)
 constexpr uint32_t HU_OFF_BAR = HU_OFF_CK + HU_HL * 4;
-constexpr uint32_t HU_SMEM = HU_OFF_BAR + 256;              // 232,192 B of the 232,448 B one CTA may have
+constexpr uint32_t HU_SMEM = HU_OFF_BAR + 256;
 static_assert(HU_SMEM <= 232448, "shared memory budget of one CTA");
-constexpr float HU_LOG2E = 1.4426950408889634f;
 
 struct HistUpdateParams {
   __nv_bfloat16* out;            // [total x d]
@@ -79,7 +82,12 @@ __device__ __forceinline__ float tanh_approx(float x) {
   asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// Rendezvous of `count` warps on an mbarrier with a bounded wait; shared-memory writes made by any lane before the
+__device__ __forceinline__ float hu_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Rendezvous of the warps that arrive on `bar`, with a bounded wait; shared-memory writes made by any lane before the
 // call are visible to every participant after it.
 __device__ __forceinline__ bool hu_group_sync(uint64_t* bar, uint32_t& uses, int lane, int* err, int where) {
   __syncwarp();
@@ -95,6 +103,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmG, const __grid_constant__ CUtensorMap tmU,
                  const __grid_constant__ CUtensorMap tmWo, const HistUpdateParams p) {
   using namespace tc;
+  static_assert(HU_COLS % ELL == 0, "a thread owns whole heads");
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {                       // swizzled tiles need a 1024-byte aligned base
     if (threadIdx.x == 0) atomicCAS(p.err, 0, 90);
@@ -102,20 +111,21 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HU_OFF_BAR);
   uint64_t* x_full = bars;           // token tile landed
-  uint64_t* x_empty = bars + 1;      // scores MMA done (1) + statistics taken by the 8 row warps
+  uint64_t* x_empty = bars + 1;      // scores MMA done (1) + statistics taken by the row warps
   uint64_t* k2_full = bars + 2;      // per user segment
   uint64_t* k2_empty = bars + 3;
   uint64_t* ops_full = bars + 4;     // per user segment: G2, U2
   uint64_t* ops_empty = bars + 5;
   uint64_t* wo_full = bars + 6;
   uint64_t* s2_full = bars + 7;      // per tile: scores in TMEM
-  uint64_t* p_ready = bars + 8;      // per tile: P in smem (8 warps)
+  uint64_t* p_ready = bars + 8;      // per tile: P in smem (all row warps)
   uint64_t* gu_full = bars + 9;      // per tile: [gate | up] in TMEM
-  uint64_t* u_ready = bars + 10;     // per tile: U in smem (8 warps)
-  uint64_t* sp_full = bars + 11;     // per tile: S' in TMEM
-  uint64_t* sp_free = bars + 12;     // per tile: S' read out (8 warps)
-  uint64_t* pair_bar = bars + 13;    // [4] rendezvous of the two warps sharing a TMEM lane quarter
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 17);
+  uint64_t* u_ready = bars + 10;     // per tile: U in smem (all row warps)
+  uint64_t* sp_full = bars + 11;     // per tile: S' in TMEM (and U read)
+  uint64_t* sp_free = bars + 12;     // per tile: S' read out (all row warps)
+  uint64_t* stats_bar = bars + 13;   // rendezvous of the row warps (token statistics written)
+  uint64_t* row_bar = bars + 14;     // [4] rendezvous of the warps sharing a TMEM lane quarter
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_all = p.tile_start[p.B];
@@ -127,8 +137,8 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     mbar_init(x_full, 1); mbar_init(x_empty, 1 + HU_ROW_WARPS);
     mbar_init(k2_full, 1); mbar_init(k2_empty, 1); mbar_init(ops_full, 1); mbar_init(ops_empty, 1); mbar_init(wo_full, 1);
     mbar_init(s2_full, 1); mbar_init(p_ready, HU_ROW_WARPS); mbar_init(gu_full, 1); mbar_init(u_ready, HU_ROW_WARPS);
-    mbar_init(sp_full, 1); mbar_init(sp_free, HU_ROW_WARPS);
-    for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
+    mbar_init(sp_full, 1); mbar_init(sp_free, HU_ROW_WARPS); mbar_init(stats_bar, HU_ROW_WARPS);
+    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], HU_PARTS);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
@@ -184,6 +194,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       constexpr uint32_t idesc_128 = make_idesc_bf16(128, 128);
       constexpr uint32_t idesc_256 = make_idesc_bf16(128, 256);
       const uint32_t sbase = smem_u32(smem);
+      const uint32_t pu = sbase + HU_OFF_PU;
       TileUser tu;
       int user_of_scores = -1, user_of_mix = -1, seg_k = 0, seg_o = 0;
       // does tile g close its user's run of tiles inside this CTA (so that the user's operands may be replaced)?
@@ -218,7 +229,6 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       if (ok) ok = issue_scores(0);
       for (int g = 0; g < n && ok; ++g) {
         const uint32_t tp = (uint32_t)g & 1u;
-        const uint32_t pu = sbase + HU_OFF_PU + (uint32_t)(g & 1) * 2 * HU_SUB;
         // 3. [gate | up](g) = P(g) . [G2 | U2]
         const int b = tu.of(p.tile_start, p.B, t_begin + g);
         if (b != user_of_mix && (seg_o == 0 || !p.shared)) {
@@ -250,98 +260,107 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       }
     }
   } else if (n > 0) {
-    // ------------------------------------------------------------------ token-row warps (2..9)
-    const int rw = warp - 2;                                 // 0..7
+    // ------------------------------------------------------------------ token-row warps (2..17)
+    const int rw = warp - 2;                                 // 0..15
     const int q = warp & 3;                                  // TMEM lane quarter of this warp
-    const int half = rw >> 2;                                // which 64 columns of every step
+    const int part = rw >> 2;                                // which 32 columns of every step
+    const int col0 = part * HU_COLS;
     const uint32_t r = (uint32_t)(q * 32 + lane);            // token row of the tile == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    float* exch = reinterpret_cast<float*>(smem + HU_OFF_EXCH);                 // [2 slots][2 halves][128]
-    float* ck_s = reinterpret_cast<float*>(smem + HU_OFF_CK) + half * 64;      // key row sums of this thread's 64 columns
-    uint32_t pair_uses = 0;
+    float2* stats = reinterpret_cast<float2*>(smem + HU_OFF_STATS);
+    float* exch = reinterpret_cast<float*>(smem + HU_OFF_EXCH);                 // [2 slots][PARTS][128]
+    const float* ck_s = reinterpret_cast<const float*>(smem + HU_OFF_CK) + col0;   // key row sums of this thread's columns
+    // K index = column, so this thread's columns live in K-block col0 / 64, chunks (col0 % 64) / 8 ..
+    uint8_t* pu = smem + HU_OFF_PU + (col0 >> 6) * HU_SUB;
+    const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
+    uint32_t stats_uses = 0, row_uses = 0;
     int ck_user = -1;
     bool ok = true;
     TileUser tu;
-    float sA = HU_LOG2E, sB = 0.f;                           // this row's rstd * log2e and -mu * rstd * log2e
+    float rstd_r = 1.f, mu_r = 0.f;                          // LayerNorm constants of this thread's token row
 
-    // LayerNorm statistics of this thread's token row of tile g, straight from the staged tile (both threads of a
-    // row compute them: cheaper than an exchange); then the stage is released
+    // LayerNorm statistics of tile g: four lanes per token, 32 features each; then this thread's own row constants.
+    // Two slots by tile parity: a warp past the rendezvous of tile g+1 knows every warp has read tile g's.
     auto take_stats = [&](int g) -> bool {
       if (LN) {
         if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 31)) return false;
-        const uint8_t* xs = smem + HU_OFF_X + r * 128u;
-        uint4 u[16];
+        const int tok = 8 * rw + (lane >> 2), p4 = lane & 3;
+        const uint8_t* xs = smem + HU_OFF_X + (p4 >> 1) * HU_SUB + tok * 128;
+        uint4 u[4];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) u[c] = *reinterpret_cast<const uint4*>(xs + (c >> 3) * HU_SUB + (((c + (int)r) & 7) << 4));
+        for (int c = 0; c < 4; ++c) {
+          const int ch = (p4 & 1) * 4 + ((c + (p4 >> 1)) & 3);
+          u[c] = *reinterpret_cast<const uint4*>(xs + ((ch ^ (tok & 7)) << 4));
+        }
         float sum = 0.f;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < 4; ++c) {
           const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) sum += __uint_as_float(w[j] << 16) + __uint_as_float(w[j] & 0xffff0000u);
         }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
         const float mu = sum * (1.0f / HU_D);
-        float var0 = 0.f, var1 = 0.f;
+        float var = 0.f;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < 4; ++c) {
           const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float a = __uint_as_float(w[j] << 16) - mu, bb = __uint_as_float(w[j] & 0xffff0000u) - mu;
-            var0 = fmaf(a, a, var0);
-            var1 = fmaf(bb, bb, var1);
+            var = fmaf(a, a, var);
+            var = fmaf(bb, bb, var);
           }
         }
-        const float rstd = rsqrtf((var0 + var1) * (1.0f / HU_D) + p.ln_eps);
-        sA = rstd * HU_LOG2E;
-        sB = -mu * sA;
+        var += __shfl_xor_sync(0xffffffffu, var, 1);
+        var += __shfl_xor_sync(0xffffffffu, var, 2);
+        if (p4 == 0) stats[(g & 1) * 128 + tok] = make_float2(rsqrtf(var * (1.0f / HU_D) + p.ln_eps), mu);
         __syncwarp();
+        if (lane == 0) mbar_arrive(x_empty);                 // this warp is done with the staged tile
+        if (!hu_group_sync(stats_bar, stats_uses, lane, p.err, 35)) return false;
+        const float2 st = stats[(g & 1) * 128 + r];
+        rstd_r = st.x; mu_r = st.y;
+      } else {
+        if (lane == 0) mbar_arrive(x_empty);
       }
-      if (lane == 0) mbar_arrive(x_empty);                   // this warp is done with the staged tile
       return true;
     };
 
-    // 2. per-head softmax over the links of this thread's heads (64 score columns), P -> smem
+    // 2. per-head softmax over the links of this thread's heads (32 score columns), P -> smem
     auto softmax = [&](int g) -> bool {
       const int b = tu.of(p.tile_start, p.B, t_begin + g);
       if (!mbar_wait(s2_full, (uint32_t)g & 1u, p.err, 32)) return false;
       tc_fence_after();
       if (LN && b != ck_user && (ck_user < 0 || !p.shared)) {
         // scores(g) exist, so every warp has finished the softmax of tile g-1 (its P was needed first): nobody still
-        // reads the previous user's sums.  The four warps of a half write identical values.
-        for (int i = lane; i < 64; i += 32) ck_s[i] = p.cK[(int64_t)(p.shared ? 0 : b) * HU_HL + half * 64 + i];
+        // reads the previous user's sums.  Every warp of a part writes the same values.
+        float* ckw = reinterpret_cast<float*>(smem + HU_OFF_CK) + col0;
+        ckw[lane] = p.cK[(int64_t)(p.shared ? 0 : b) * HU_HL + col0 + lane];
         __syncwarp();
       }
       ck_user = b;
-      float v[64];
-      {
-        float v0[32], v1[32];
-        const uint32_t ta = lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + half * 64;
-        tmem_ld_32x32(ta, v0);
-        tmem_ld_32x32(ta + 32, v1);
-        tmem_wait_ld();
+      float v[HU_COLS];
+      tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
+      tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
-      }
-      uint8_t* pu = smem + HU_OFF_PU + (g & 1) * 2 * HU_SUB + half * HU_SUB;   // K-block `half` holds columns 64*half..
-#pragma unroll
-      for (int h = 0; h < 64 / ELL; ++h) {
+      for (int h = 0; h < HU_COLS / ELL; ++h) {
         float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < ELL; ++j) {
           const int c = h * ELL + j;
-          v[c] = LN ? fmaf(v[c], sA, ck_s[c] * sB) : v[c] * HU_LOG2E;
+          if (LN) v[c] = (v[c] - mu_r * ck_s[c]) * rstd_r;
           mx = fmaxf(mx, v[c]);
         }
         float s0 = 0.f, s1 = 0.f;
 #pragma unroll
         for (int j = 0; j < ELL; j += 2) {
-          v[h * ELL + j] = exp2f(v[h * ELL + j] - mx);
-          v[h * ELL + j + 1] = exp2f(v[h * ELL + j + 1] - mx);
+          v[h * ELL + j] = hu_ex2(v[h * ELL + j] - mx);
+          v[h * ELL + j + 1] = hu_ex2(v[h * ELL + j + 1] - mx);
           s0 += v[h * ELL + j];
           s1 += v[h * ELL + j + 1];
         }
-        const float inv = 1.f / (s0 + s1);
+        const float inv = __fdividef(1.f, s0 + s1);
 #pragma unroll
         for (int c8 = 0; c8 < ELL / 8; ++c8) {
           const int c = h * ELL + c8 * 8;                    // first of 8 consecutive contraction indices
@@ -350,7 +369,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           o.y = pack_bf16(v[c + 2] * inv, v[c + 3] * inv);
           o.z = pack_bf16(v[c + 4] * inv, v[c + 5] * inv);
           o.w = pack_bf16(v[c + 6] * inv, v[c + 7] * inv);
-          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, (uint32_t)c >> 3)) = o;
+          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, chunk0 + ((uint32_t)c >> 3))) = o;
         }
       }
       tc_fence_before();
@@ -360,30 +379,25 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       return true;
     };
 
-    // 4. U = SiLU(gate) * up for this thread's 64 hidden columns -> smem (over P(g), which [gate|up](g) has read)
+    // 4. U = SiLU(gate) * up for this thread's 32 hidden columns -> smem (over P(g), which [gate|up](g) has read)
     auto silu_mul = [&](int g) -> bool {
       if (!mbar_wait(gu_full, (uint32_t)g & 1u, p.err, 33)) return false;
       tc_fence_after();
-      uint8_t* pu = smem + HU_OFF_PU + (g & 1) * 2 * HU_SUB + half * HU_SUB;
+      float gt[HU_COLS], up[HU_COLS];
+      tmem_ld_32x32(lane_addr + COL_GU + col0, gt);
+      tmem_ld_32x32(lane_addr + COL_GU + HU_F + col0, up);
+      tmem_wait_ld();
 #pragma unroll
-      for (int c = 0; c < 64; c += 32) {
-        float gt[32], up[32];
-        tmem_ld_32x32(lane_addr + COL_GU + half * 64 + c, gt);
-        tmem_ld_32x32(lane_addr + COL_GU + HU_F + half * 64 + c, up);
-        tmem_wait_ld();
+      for (int c8 = 0; c8 < HU_COLS / 8; ++c8) {
+        float y[8];
 #pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
-          float y[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float x = gt[c8 * 8 + j];
-            const float hx = 0.5f * x;
-            y[j] = fmaf(hx, tanh_approx(hx), hx) * up[c8 * 8 + j];    // x * sigmoid(x) = x/2 * (1 + tanh(x/2))
-          }
-          uint4 o;
-          o.x = pack_bf16(y[0], y[1]); o.y = pack_bf16(y[2], y[3]); o.z = pack_bf16(y[4], y[5]); o.w = pack_bf16(y[6], y[7]);
-          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, (uint32_t)(c >> 3) + c8)) = o;
+        for (int j = 0; j < 8; ++j) {
+          const float hx = 0.5f * gt[c8 * 8 + j];
+          y[j] = fmaf(hx, tanh_approx(hx), hx) * up[c8 * 8 + j];    // x * sigmoid(x) = x/2 * (1 + tanh(x/2))
         }
+        uint4 o;
+        o.x = pack_bf16(y[0], y[1]); o.y = pack_bf16(y[2], y[3]); o.z = pack_bf16(y[4], y[5]); o.w = pack_bf16(y[6], y[7]);
+        *reinterpret_cast<uint4*>(pu + sw128_chunk(r, chunk0 + (uint32_t)c8)) = o;
       }
       tc_fence_before();
       fence_proxy_async_smem();
@@ -392,48 +406,45 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       return true;
     };
 
-    // 6. this thread's 64 columns of its S' row -> (LayerNorm) -> bf16 -> global
+    // 6. this thread's 32 columns of its S' row -> (LayerNorm) -> bf16 -> global.  The caller has waited for sp_full(g).
     auto store_rows = [&](int g) -> bool {
       const int t = t_begin + g;
       const int b = tu.of(p.tile_start, p.B, t);
       const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
       const bool valid = row0 + (int)r < p.off[b + 1];
-      if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 34)) return false;
-      tc_fence_after();
-      float v[64];
-      {
-        float v0[32], v1[32];
-        const uint32_t ta = lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + half * 64;
-        tmem_ld_32x32(ta, v0);
-        tmem_ld_32x32(ta + 32, v1);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
-      }
+      float v[HU_COLS];
+      tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
+      tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(sp_free);
       if (p.out_ln) {
+        // separate slots for the two exchanges: each is rewritten only after a later rendezvous of the same row group
         float s = 0.f;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) s += v[j];
-        // separate slots for the two exchanges: each is rewritten only after a later rendezvous of the same pair
-        exch[half * 128 + r] = s;
-        if (!hu_group_sync(&pair_bar[q], pair_uses, lane, p.err, 37)) return false;
-        const float mu = (s + exch[(half ^ 1) * 128 + r]) * (1.0f / HU_D);
+        for (int j = 0; j < HU_COLS; ++j) s += v[j];
+        exch[part * 128 + r] = s;
+        if (!hu_group_sync(&row_bar[q], row_uses, lane, p.err, 37)) return false;
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < HU_PARTS; ++i) tot += exch[i * 128 + r];
+        const float mu = tot * (1.0f / HU_D);
         float var = 0.f;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
-        exch[256 + half * 128 + r] = var;
-        if (!hu_group_sync(&pair_bar[q], pair_uses, lane, p.err, 39)) return false;
-        const float rstd = rsqrtf((var + exch[256 + (half ^ 1) * 128 + r]) * (1.0f / HU_D) + p.ln_eps);
+        for (int j = 0; j < HU_COLS; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
+        exch[(HU_PARTS + part) * 128 + r] = var;
+        if (!hu_group_sync(&row_bar[q], row_uses, lane, p.err, 39)) return false;
+        float vt = 0.f;
 #pragma unroll
-        for (int j = 0; j < 64; ++j) v[j] *= rstd;
+        for (int i = 0; i < HU_PARTS; ++i) vt += exch[(HU_PARTS + i) * 128 + r];
+        const float rstd = rsqrtf(vt * (1.0f / HU_D) + p.ln_eps);
+#pragma unroll
+        for (int j = 0; j < HU_COLS; ++j) v[j] *= rstd;
       }
       if (valid) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * HU_D + half * 64);
+        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * HU_D + col0);
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
+        for (int c8 = 0; c8 < HU_COLS / 8; ++c8) {
           uint4 o;
           o.x = pack_bf16(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = pack_bf16(v[c8 * 8 + 2], v[c8 * 8 + 3]);
           o.z = pack_bf16(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = pack_bf16(v[c8 * 8 + 6], v[c8 * 8 + 7]);
@@ -445,13 +456,15 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
     ok = take_stats(0) && softmax(0);
     for (int g = 0; g < n && ok; ++g) {
-      if (g > 0 && !store_rows(g - 1)) { ok = false; break; }
-      // statistics of the next tile as soon as it has landed, so that its stage can be refilled a whole tile early
+      if (!silu_mul(g)) { ok = false; break; }                                   // [gate|up](g) ran under store(g-1)
+      // statistics of the next tile while S'(g) is formed, so that its stage can be refilled a whole tile early
       if (g + 1 < n && !take_stats(g + 1)) { ok = false; break; }
-      if (!silu_mul(g)) { ok = false; break; }
+      // P(g+1) overwrites U(g): wait until S'(g) has consumed it
+      if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 34)) { ok = false; break; }
+      tc_fence_after();
       if (g + 1 < n && !softmax(g + 1)) { ok = false; break; }
+      if (!store_rows(g)) { ok = false; break; }                                 // runs under [gate|up](g+1)
     }
-    if (ok) store_rows(n - 1);
   }
 
   tc_fence_before();
@@ -463,7 +476,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 }
 
 bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp) {
-  return dtype == LIME_BF16 && d == HU_D && f == HU_F && H * ell == HU_HL && (ell == 16 || ell == 32 || ell == 64) &&
+  return dtype == LIME_BF16 && d == HU_D && f == HU_F && H * ell == HU_HL && (ell == 16 || ell == 32) &&
          phi == LIME_PHI_SOFTMAX && gated_mlp != 0;
 }
 
@@ -482,14 +495,13 @@ static lime_status launch_hu(const HistUpdateArgs& a, cudaStream_t st) {
   p.shared = a.shared; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
   int grid = a.n_tile_upper < kSMs ? a.n_tile_upper : kSMs;
   if (grid < 1) return LIME_OK;
+  static bool smem_ln[kMaxDeviceOrdinals] = {}, smem_plain[kMaxDeviceOrdinals] = {};
+  lime_status es = a.ln ? ensure_dynamic_smem((const void*)k_hist_update_tc<ELL, true>, (int)HU_SMEM, smem_ln)
+                        : ensure_dynamic_smem((const void*)k_hist_update_tc<ELL, false>, (int)HU_SMEM, smem_plain);
+  if (es != LIME_OK) return es;
   ProfScope _p("k_hist_update_tc", st);
-  if (a.ln) {
-    LIME_CUDA(cudaFuncSetAttribute(k_hist_update_tc<ELL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)HU_SMEM));
-    k_hist_update_tc<ELL, true><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
-  } else {
-    LIME_CUDA(cudaFuncSetAttribute(k_hist_update_tc<ELL, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)HU_SMEM));
-    k_hist_update_tc<ELL, false><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
-  }
+  if (a.ln) k_hist_update_tc<ELL, true><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  else k_hist_update_tc<ELL, false><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
   LIME_LAUNCH_CHECK("k_hist_update_tc");
   return LIME_OK;
 }
@@ -499,7 +511,6 @@ lime_status launch_hist_update_tc(const HistUpdateArgs& a, cudaStream_t st) {
   switch (a.ell) {
     case 16: return launch_hu<16>(a, st);
     case 32: return launch_hu<32>(a, st);
-    case 64: return launch_hu<64>(a, st);
   }
   return LIME_UNSUPPORTED_SHAPE;
 }

@@ -2,22 +2,24 @@
 //
 //   O[T]_h = softmax_j( Q[T]_h K[S]_h^T * scale ) V[S]_h,  K[S] = LN(S) W_K,  V[S] = LN(S) W_V          (Eq. 3 / Eq. 7)
 //
-// With W_K folded into the link queries (Q2, see k_link_prep.cu) and W_V applied after the attention, both
-// contractions run against the *stored* history rows X, which are streamed exactly once (TMA) and used both as
-// keys and as values - K[S] and V[S] are never materialised:
+// With W_K folded into the link queries (Q2, see k_link_prep.cu; the fold also carries scale * log2(e), so scores
+// arrive in the log2 domain) and W_V applied after the attention, both contractions run against the *stored*
+// history rows X, which are streamed exactly once (TMA) and used both as keys and as values - K[S] and V[S] are
+// never materialised:
 //   scores [HL x 128]   = Q2 [HL x d] . X_tile^T            LayerNorm folded in afterwards:
 //                         s_ij = rstd_j * (raw_ij - mu_j * rowsum(Q2)_i)
 //   acc    [HL x d]    += P' [HL x 128] . X_tile            P'_ij = p_ij * rstd_j;  the mean term sum_j P'_ij mu_j is
 //                                                           a per-row scalar subtracted from every column at the end
 //   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (W_V is folded into the GEMM that follows)
-// HL = H * ell stacked (head, link) rows = 128 TMEM lanes.  Online softmax in the log2 domain whose reference
-// maximum is only raised when the true maximum exceeds it by more than 8 (then the accumulator row is rescaled in
-// TMEM), so most tiles need no correction pass.
+// HL = H * ell stacked (head, link) rows = 128 TMEM lanes.  Online softmax whose reference maximum is only raised
+// when the true maximum exceeds it by more than 8 (then the accumulator row is rescaled in TMEM), so most tiles need
+// no correction pass.  With LN = false the rows of X are LayerNorm-ed already and the corrections vanish.
 //
 // Persistent CTAs walk (user, chunk-of-history) items.  Warp roles: warp 0 TMA producer (runs ahead across items),
-// warp 1 MMA issuer, warps 2-9 softmax: two threads per (head, link) row, each owning 64 of the tile's 128 token
-// columns (a warp may only touch the TMEM lane quarter warp_id % 4, so the two halves of a row sit in warps w and
-// w + 4 and exchange their row maximum through shared memory).  A user whose history is a single chunk is
+// warp 1 MMA issuer, warps 2-17 softmax: four threads per (head, link) row, each owning 32 of the tile's 128 token
+// columns (a warp may only touch the TMEM lane quarter warp_id % 4, so the four parts of a row sit in warps w,
+// w + 4, w + 8, w + 12 and exchange their row maximum through shared memory).  Four warps per scheduler keep the
+// issue slots busy while TMEM loads and exponentials are in flight.  A user whose history is a single chunk is
 // normalised and written directly; longer histories leave (max, sum, accumulator) partials per chunk that
 // k_link_attn_merge_norm combines.
 //
@@ -28,18 +30,20 @@
 namespace lime {
 
 constexpr int LA_D = 128, LA_HL = 128, LA_TILE = 128, LA_XSTAGES = 3;
-constexpr int LA_SOFTMAX_WARPS = 8, LA_THREADS = 64 + 32 * LA_SOFTMAX_WARPS;
+constexpr int LA_PARTS = 4;                                   // threads per row
+constexpr int LA_COLS = LA_TILE / LA_PARTS;                   // token columns per thread
+constexpr int LA_SOFTMAX_WARPS = 4 * LA_PARTS, LA_THREADS = 64 + 32 * LA_SOFTMAX_WARPS;
 constexpr uint32_t LA_SUB = 128 * 128;
 constexpr uint32_t LA_X_STAGE = 2 * LA_SUB;
 constexpr uint32_t LA_OFF_X = 0;
 constexpr uint32_t LA_OFF_Q2 = LA_XSTAGES * LA_X_STAGE;
 constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_SUB;        // 2 buffers of [HL x 128 tokens]
-constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 4 * LA_SUB;     // per X stage: float4 {rstd*log2e, -mu*rstd*log2e, rstd, mu} x 128
-constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 16;   // 2 x 2 x 128 maxima, 2 x 128 sums, 2 x 128 mean terms
-constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 8 * 128 * 4;
+constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 4 * LA_SUB;     // per X stage: float2 {rstd, mu} x 128 tokens
+constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 8;   // [2 tile parities][PARTS][128] maxima, then
+                                                                        // [PARTS][128] sums and [PARTS][128] mean terms
+constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 4 * LA_PARTS * 128 * 4;
 constexpr uint32_t LA_SMEM = LA_OFF_BAR + 256;
 constexpr float LA_RESCALE_THRESHOLD = 8.0f;                 // in log2 units
-constexpr float LA_LOG2E = 1.4426950408889634f;
 
 struct LinkAttnParams {
   const float* cQ;                // [users x HL]
@@ -57,7 +61,12 @@ __device__ __forceinline__ uint32_t la_pack(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-// Rendezvous of `count` warps on an mbarrier (every wait in this kernel is bounded, so no bar.sync): shared-memory
+__device__ __forceinline__ float la_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// Rendezvous of the warps that arrive on `bar` (every wait in this kernel is bounded, so no bar.sync): shared-memory
 // writes made by any lane before the call are visible to every participant after it.
 __device__ __forceinline__ bool la_group_sync(uint64_t* bar, uint32_t& uses, int lane, int* err, int where) {
   __syncwarp();
@@ -65,6 +74,57 @@ __device__ __forceinline__ bool la_group_sync(uint64_t* bar, uint32_t& uses, int
   const bool ok = tc::mbar_wait(bar, uses & 1u, err, where);
   ++uses;
   return ok;
+}
+
+// Pass 1 over this thread's LA_COLS scores: LayerNorm correction (LN) and the maximum over the valid columns.
+template <bool LN, bool MASK>
+__device__ __forceinline__ float la_pass1(float (&v)[LA_COLS], const float2* __restrict__ st, float cq, int col0, int nvalid) {
+  float mx = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < LA_COLS; ++j) {
+    if (LN) {
+      const float2 c2 = st[col0 + j];
+      v[j] = (v[j] - cq * c2.y) * c2.x;
+    }
+    if (!MASK || col0 + j < nvalid) mx = fmaxf(mx, v[j]);
+  }
+  return mx;
+}
+
+// Pass 2: p = 2^(s - m_ref), P' = p * rstd as bf16 into the A-operand buffer (K-major over the tile's tokens,
+// 128-byte swizzle); returns the sums of p and of P' * mu through l_sum / mean_corr.
+template <bool LN, bool MASK>
+__device__ __forceinline__ void la_pass2(const float (&v)[LA_COLS], const float2* __restrict__ st, float m_ref, int col0, int nvalid,
+                                         uint8_t* prow_base, uint32_t r, uint32_t chunk0, float& l_sum, float& mean_corr) {
+  float ls0 = 0.f, ls1 = 0.f, mc0 = 0.f, mc1 = 0.f;
+#pragma unroll
+  for (int c8 = 0; c8 < LA_COLS / 8; ++c8) {
+    uint32_t packed[4];
+#pragma unroll
+    for (int j2 = 0; j2 < 4; ++j2) {
+      const int j = c8 * 8 + 2 * j2;
+      float e0 = la_ex2(v[j] - m_ref), e1 = la_ex2(v[j + 1] - m_ref);
+      if (MASK) {
+        if (col0 + j >= nvalid) e0 = 0.f;
+        if (col0 + j + 1 >= nvalid) e1 = 0.f;
+      }
+      ls0 += e0;
+      ls1 += e1;
+      if (LN) {
+        const float2 a = st[col0 + j], b = st[col0 + j + 1];
+        // what the MMA will see is the bf16-rounded P'; use the same rounded values for the mean term
+        const uint32_t pk = la_pack(e0 * a.x, e1 * b.x);
+        mc0 = fmaf(__uint_as_float(pk << 16), a.y, mc0);
+        mc1 = fmaf(__uint_as_float(pk & 0xffff0000u), b.y, mc1);
+        packed[j2] = pk;
+      } else {
+        packed[j2] = la_pack(e0, e1);
+      }
+    }
+    *reinterpret_cast<uint4*>(prow_base + la_chunk_addr(r, chunk0 + (uint32_t)c8)) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+  }
+  l_sum += ls0 + ls1;
+  mean_corr += mc0 + mc1;
 }
 
 template <bool LN>
@@ -84,11 +144,11 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   uint64_t* q_full = bars + 6;         //      folded queries of the item's user landed
   uint64_t* q_empty = bars + 7;        //      every score MMA of the item has read them
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       // [2]  P' in smem (8 warps)
+  uint64_t* p_ready = bars + 10;       // [2]  P' in smem (all softmax warps)
   uint64_t* p_free = bars + 12;        // [2]  second MMA done reading P' (and accumulator up to date)
-  uint64_t* o_free = bars + 14;        //      accumulator of the item read out (8 warps)
-  uint64_t* stats_bar = bars + 15;     //      rendezvous of the 8 softmax warps (token statistics written)
-  uint64_t* pair_bar = bars + 16;      // [4]  rendezvous of the two warps that share a TMEM lane quarter
+  uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
+  uint64_t* stats_bar = bars + 15;     //      rendezvous of the softmax warps (token statistics written)
+  uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the warps that share a TMEM lane quarter
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -99,7 +159,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], LA_SOFTMAX_WARPS); mbar_init(&p_free[i], 1); }
     mbar_init(o_free, LA_SOFTMAX_WARPS);
     mbar_init(stats_bar, LA_SOFTMAX_WARPS);
-    for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
+    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LA_PARTS);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
@@ -210,19 +270,20 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax warps (2..9)
-    const int sw = warp - 2;                                   // 0..7
+    // ------------------------------------------------------------------ softmax warps (2..17)
+    const int sw = warp - 2;                                   // 0..15
     const int q = warp & 3;                                    // TMEM lane quarter of this warp
-    const int half = sw >> 2;                                  // which 64 token columns of the tile
+    const int part = sw >> 2;                                  // which LA_COLS token columns of the tile
+    const int col0 = part * LA_COLS;
     const uint32_t r = (uint32_t)(q * 32 + lane);              // (head, link) row == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    float4* stats = reinterpret_cast<float4*>(smem + LA_OFF_STATS);
-    float* exch_max = reinterpret_cast<float*>(smem + LA_OFF_EXCH);          // [2 tile parities][2 halves][128]
-    float* exch_sum = exch_max + 4 * 128;                                    // [2][128]
-    float* exch_mean = exch_sum + 2 * 128;                                   // [2][128]
+    float2* stats = reinterpret_cast<float2*>(smem + LA_OFF_STATS);
+    float* exch_max = reinterpret_cast<float*>(smem + LA_OFF_EXCH);          // [2 tile parities][PARTS][128]
+    float* exch_sum = exch_max + 2 * LA_PARTS * 128;                         // [PARTS][128]
+    float* exch_mean = exch_sum + LA_PARTS * 128;                            // [PARTS][128]
     bool ok = true;
     int g = 0, k = 0;
-    uint32_t stats_uses = 0, pair_uses = 0;
+    uint32_t stats_uses = 0, row_uses = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
       int b, tok0, tok1;
       item_range(item, b, tok0, tok1);
@@ -232,27 +293,31 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         const int s = g % LA_XSTAGES, pb = g & 1;
         const int nvalid = min(LA_TILE, tok1 - tok0 - t * LA_TILE);
-        const float4* st = stats + s * 128;
+        const float2* st = stats + s * 128;
         if (LN) {
-          // LayerNorm statistics of the tile's tokens: two lanes per token, 64 features each, held in registers
+          // LayerNorm statistics of the tile's tokens: four lanes per token, 32 features each, held in registers
           if (!mbar_wait(&x_full[s], (uint32_t)(g / LA_XSTAGES) & 1u, p.err, 61)) { ok = false; break; }
-          const int tok = 16 * sw + (lane >> 1), hf = lane & 1;
-          const uint8_t* xs = smem + LA_OFF_X + s * LA_X_STAGE + hf * LA_SUB + tok * 128;
-          uint4 u[8];
+          const int tok = 8 * sw + (lane >> 2), p4 = lane & 3;
+          const uint8_t* xs = smem + LA_OFF_X + s * LA_X_STAGE + (p4 >> 1) * LA_SUB + tok * 128;
+          uint4 u[4];
 #pragma unroll
-          for (int c = 0; c < 8; ++c) u[c] = *reinterpret_cast<const uint4*>(xs + (((c + tok + 4 * hf) & 7) << 4));
+          for (int c = 0; c < 4; ++c) {
+            const int ch = (p4 & 1) * 4 + ((c + (p4 >> 1)) & 3);             // this lane's 4 chunks, rotated start
+            u[c] = *reinterpret_cast<const uint4*>(xs + ((ch ^ (tok & 7)) << 4));
+          }
           float sum = 0.f;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
+          for (int c = 0; c < 4; ++c) {
             const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) sum += __uint_as_float(w[j] << 16) + __uint_as_float(w[j] & 0xffff0000u);
           }
           sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+          sum += __shfl_xor_sync(0xffffffffu, sum, 2);
           const float mu = sum * (1.0f / LA_D);
           float var = 0.f;
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
+          for (int c = 0; c < 4; ++c) {
             const uint32_t w[4] = {u[c].x, u[c].y, u[c].z, u[c].w};
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -262,55 +327,37 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             }
           }
           var += __shfl_xor_sync(0xffffffffu, var, 1);
-          const float rstd = rsqrtf(var * (1.0f / LA_D) + p.ln_eps);
-          if (hf == 0) stats[s * 128 + tok] = make_float4(rstd * LA_LOG2E, -mu * rstd * LA_LOG2E, rstd, mu);
+          var += __shfl_xor_sync(0xffffffffu, var, 2);
+          if (p4 == 0) stats[s * 128 + tok] = make_float2(rsqrtf(var * (1.0f / LA_D) + p.ln_eps), mu);
           if (!la_group_sync(stats_bar, stats_uses, lane, p.err, 62)) { ok = false; break; }
         }
         if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
         tc_fence_after();
 
-        // pass 1: this thread's 64 scores (log2 domain) into registers, and their maximum
-        float v[64];
-        {
-          float v0[32], v1[32];
-          tmem_ld_32x32(lane_addr + COL_S + pb * 128 + half * 64, v0);
-          tmem_ld_32x32(lane_addr + COL_S + pb * 128 + half * 64 + 32, v1);
-          tmem_wait_ld();
+        // pass 1: this thread's scores (log2 domain) into registers, and their maximum
+        float v[LA_COLS];
+        tmem_ld_32x32(lane_addr + COL_S + pb * 128 + col0, v);
+        tmem_wait_ld();
+        float mx = nvalid == LA_TILE ? la_pass1<LN, false>(v, st, cq, col0, nvalid) : la_pass1<LN, true>(v, st, cq, col0, nvalid);
+        exch_max[(pb * LA_PARTS + part) * 128 + r] = mx;
+        if (!la_group_sync(&row_bar[q], row_uses, lane, p.err, 67)) { ok = false; break; }
 #pragma unroll
-          for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
-        }
-        float mx = -INFINITY;
-#pragma unroll
-        for (int j = 0; j < 64; ++j) {
-          if (LN) {
-            const float4 c4 = st[half * 64 + j];
-            v[j] = fmaf(v[j], c4.x, cq * c4.y);
-          } else {
-            v[j] *= LA_LOG2E;
-          }
-          if (half * 64 + j < nvalid) mx = fmaxf(mx, v[j]);
-        }
-        exch_max[(pb * 2 + half) * 128 + r] = mx;
-        if (!la_group_sync(&pair_bar[q], pair_uses, lane, p.err, 67)) { ok = false; break; }
-        mx = fmaxf(mx, exch_max[(pb * 2 + (half ^ 1)) * 128 + r]);
+        for (int i = 1; i < LA_PARTS; ++i) mx = fmaxf(mx, exch_max[(pb * LA_PARTS + ((part + i) & (LA_PARTS - 1))) * 128 + r]);
 
         // raise the reference maximum only when it is exceeded by more than the threshold (or unset)
         const bool need = mx > m_ref + LA_RESCALE_THRESHOLD;
         const float m_new = need ? mx : m_ref;
-        const float factor = (need && m_ref != -INFINITY) ? exp2f(m_ref - m_new) : 1.0f;
+        const float factor = (need && m_ref != -INFINITY) ? la_ex2(m_ref - m_new) : 1.0f;
         if (__any_sync(0xffffffffu, need && t > 0)) {
-          // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this half-row
+          // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this part of the row
           if (!mbar_wait(&p_free[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, p.err, 64)) { ok = false; break; }
           tc_fence_after();
+          float a[LA_COLS];
+          tmem_ld_32x32(lane_addr + COL_O + col0, a);
+          tmem_wait_ld();
 #pragma unroll
-          for (int c = 0; c < 64; c += 16) {
-            float a[16];
-            tmem_ld_32x16(lane_addr + COL_O + half * 64 + c, a);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 16; ++j) a[j] *= factor;
-            tmem_st_32x16(lane_addr + COL_O + half * 64 + c, a);
-          }
+          for (int j = 0; j < LA_COLS; ++j) a[j] *= factor;
+          tmem_st_32x32(lane_addr + COL_O + col0, a);
           tmem_wait_st();
         }
         l_sum *= factor;
@@ -319,54 +366,30 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
         // the P' buffer of two tiles ago must have been consumed
         if (g >= 2 && !mbar_wait(&p_free[pb], (uint32_t)((g - 2) >> 1) & 1u, p.err, 65)) { ok = false; break; }
-        // pass 2: p = 2^(s - m_ref); P' = p * rstd -> smem (A operand, K-major over the tile's tokens)
-        uint8_t* pbuf = smem + LA_OFF_P + pb * 2 * LA_SUB + half * LA_SUB;
-#pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
-          float pp[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const int col = c8 * 8 + j;
-            const float e = (half * 64 + col < nvalid) ? exp2f(v[col] - m_ref) : 0.f;
-            l_sum += e;
-            if (LN) {
-              const float4 c4 = st[half * 64 + col];
-              // what the MMA will see is the bf16-rounded P'; use the same rounded value for the mean term
-              const float pr = __bfloat162float(__float2bfloat16_rn(e * c4.z));
-              mean_corr = fmaf(pr, c4.w, mean_corr);
-              pp[j] = pr;
-            } else {
-              pp[j] = e;
-            }
-          }
-          uint4 o;
-          o.x = la_pack(pp[0], pp[1]); o.y = la_pack(pp[2], pp[3]); o.z = la_pack(pp[4], pp[5]); o.w = la_pack(pp[6], pp[7]);
-          *reinterpret_cast<uint4*>(pbuf + la_chunk_addr(r, (uint32_t)c8)) = o;
-        }
+        // pass 2: P' -> smem; K index = token column, so columns col0.. live in K-block col0 / 64, chunk (col0 % 64) / 8..
+        uint8_t* pbuf = smem + LA_OFF_P + pb * 2 * LA_SUB + (col0 >> 6) * LA_SUB;
+        const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
+        if (nvalid == LA_TILE) la_pass2<LN, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
+        else la_pass2<LN, true>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(&p_ready[pb]);
       }
       if (!ok) break;
-      // item result: wait for the last second MMA, combine the two halves' sums, read the accumulator half-row
+      // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
       const int gl = g - 1;
       if (!mbar_wait(&p_free[gl & 1], (uint32_t)(gl >> 1) & 1u, p.err, 66)) { ok = false; break; }
       tc_fence_after();
-      exch_sum[half * 128 + r] = l_sum;
-      exch_mean[half * 128 + r] = mean_corr;
-      if (!la_group_sync(&pair_bar[q], pair_uses, lane, p.err, 68)) { ok = false; break; }
-      const float l_tot = l_sum + exch_sum[(half ^ 1) * 128 + r];
-      const float c_tot = mean_corr + exch_mean[(half ^ 1) * 128 + r];
-      float a[64];
-      {
-        float a0[32], a1[32];
-        tmem_ld_32x32(lane_addr + COL_O + half * 64, a0);
-        tmem_ld_32x32(lane_addr + COL_O + half * 64 + 32, a1);
-        tmem_wait_ld();
+      exch_sum[part * 128 + r] = l_sum;
+      exch_mean[part * 128 + r] = mean_corr;
+      if (!la_group_sync(&row_bar[q], row_uses, lane, p.err, 68)) { ok = false; break; }
+      float l_tot = 0.f, c_tot = 0.f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) { a[j] = a0[j]; a[32 + j] = a1[j]; }
-      }
+      for (int i = 0; i < LA_PARTS; ++i) { l_tot += exch_sum[i * 128 + r]; c_tot += exch_mean[i * 128 + r]; }
+      float a[LA_COLS];
+      tmem_ld_32x32(lane_addr + COL_O + col0, a);
+      tmem_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
@@ -375,9 +398,9 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // the whole history of this user was one chunk: normalise and write the attention rows directly
         const float inv = 1.0f / l_tot;
         const int h = (int)r / p.ell, l = (int)r % p.ell;
-        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + ((int64_t)b * p.ell + l) * (p.H * LA_D) + h * LA_D + half * 64);
+        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + ((int64_t)b * p.ell + l) * (p.H * LA_D) + h * LA_D + col0);
 #pragma unroll
-        for (int c8 = 0; c8 < 8; ++c8) {
+        for (int c8 = 0; c8 < LA_COLS / 8; ++c8) {
           uint4 o;
           o.x = la_pack((a[c8 * 8 + 0] - c_tot) * inv, (a[c8 * 8 + 1] - c_tot) * inv);
           o.y = la_pack((a[c8 * 8 + 2] - c_tot) * inv, (a[c8 * 8 + 3] - c_tot) * inv);
@@ -386,11 +409,11 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           dst[c8] = o;
         }
       } else {
-        float4* dst = reinterpret_cast<float4*>(p.part_acc + ((int64_t)item * LA_HL + r) * LA_D + half * 64);
+        float4* dst = reinterpret_cast<float4*>(p.part_acc + ((int64_t)item * LA_HL + r) * LA_D + col0);
 #pragma unroll
-        for (int j = 0; j < 64; j += 4)
+        for (int j = 0; j < LA_COLS; j += 4)
           dst[j / 4] = make_float4(a[j] - c_tot, a[j + 1] - c_tot, a[j + 2] - c_tot, a[j + 3] - c_tot);
-        if (half == 0) {
+        if (part == 0) {
           p.part_m[(int64_t)item * LA_HL + r] = m_ref;        // log2 domain
           p.part_s[(int64_t)item * LA_HL + r] = l_tot;
         }
@@ -422,14 +445,13 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
   p.ell = a.ell; p.H = a.H; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
   const int grid = a.n_chunk_upper < kSMs ? a.n_chunk_upper : kSMs;
+  static bool smem_ln[kMaxDeviceOrdinals] = {}, smem_plain[kMaxDeviceOrdinals] = {};
+  lime_status es = a.ln ? ensure_dynamic_smem((const void*)k_link_attn_tc<true>, (int)LA_SMEM, smem_ln)
+                        : ensure_dynamic_smem((const void*)k_link_attn_tc<false>, (int)LA_SMEM, smem_plain);
+  if (es != LIME_OK) return es;
   ProfScope _p("k_link_attn_tc", st);
-  if (a.ln) {
-    LIME_CUDA(cudaFuncSetAttribute(k_link_attn_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LA_SMEM));
-    k_link_attn_tc<true><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
-  } else {
-    LIME_CUDA(cudaFuncSetAttribute(k_link_attn_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)LA_SMEM));
-    k_link_attn_tc<false><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
-  }
+  if (a.ln) k_link_attn_tc<true><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
+  else k_link_attn_tc<false><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
   LIME_LAUNCH_CHECK("k_link_attn_tc");
   return LIME_OK;
 }

@@ -8,7 +8,8 @@
 //   history <- links scores  Q[S]_h K[T]_h^T = LN(S) . K2_(h,l)^T    K2_(h,l) = That_l (scale W_{K,h} W_{Q,h}^T)
 //   GatedMLP input           O[S] W_g = P . G2,  O[S] W_u = P . U2   G2_(h,l) = That_l (W_{V,h} W_g[h rows, :])
 //   link rows                O[T] W_g = sum_h Ohat_(h,l) (W_{V,h} W_g[h rows, :])        (same folded matrices)
-// The bracketed products depend on the weights only and are formed once, here, at lime_set_weights time.
+// The bracketed products depend on the weights only and are formed once, here, at lime_set_weights time; `scale`
+// is the softmax scale times log2(e), so that the streaming kernels exponentiate with ex2 directly.
 #include "lime_common.cuh"
 
 namespace lime {
@@ -88,36 +89,39 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
 
 // Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
 //   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
-// grid (B * H * ell), block d threads.  A user without history gets zeros; a user with a single chunk was
-// already written by the attention kernel.
+// One block of d threads per user walks the user's H * ell rows.  A user without history gets zeros; a user with a
+// single chunk was already written by the attention kernel (its block returns at once).
 __global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H,
                                        const float* __restrict__ part_m, const float* __restrict__ part_s,
                                        const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
   const int HL = H * ell;
-  const int u = blockIdx.x / HL, row = blockIdx.x % HL, h = row / ell, l = row % ell;
+  const int u = blockIdx.x;
   const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
   if (c1 - c0 == 1) return;
   const int i = threadIdx.x;
-  float out = 0.f;
-  if (c1 > c0) {
-    float M = -INFINITY;
-    for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
-    float S = 0.f, O = 0.f;
-    for (int c = c0; c < c1; ++c) {
-      const float w = exp2f(part_m[(int64_t)c * HL + row] - M);
-      S = fmaf(part_s[(int64_t)c * HL + row], w, S);
-      O = fmaf(part_acc[((int64_t)c * HL + row) * d + i], w, O);
+  for (int row = 0; row < HL; ++row) {
+    const int h = row / ell, l = row % ell;
+    float out = 0.f;
+    if (c1 > c0) {
+      float M = -INFINITY;
+      for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
+      float S = 0.f, O = 0.f;
+      for (int c = c0; c < c1; ++c) {
+        const float w = exp2f(part_m[(int64_t)c * HL + row] - M);
+        S = fmaf(part_s[(int64_t)c * HL + row], w, S);
+        O = fmaf(part_acc[((int64_t)c * HL + row) * d + i], w, O);
+      }
+      out = O / S;
     }
-    out = O / S;
+    Ohat[((int64_t)u * ell + l) * (H * d) + h * d + i] = __float2bfloat16_rn(out);
   }
-  Ohat[((int64_t)u * ell + l) * (H * d) + h * d + i] = __float2bfloat16_rn(out);
 }
 
 lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
                                         const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
   if (B == 0) return LIME_OK;
   ProfScope _p("k_link_attn_merge_norm", st);
-  k_link_attn_merge_norm<<<B * H * ell, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  k_link_attn_merge_norm<<<B, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }

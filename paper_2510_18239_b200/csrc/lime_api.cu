@@ -375,7 +375,8 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
       if (!c->WprepT[j]) LIME_CUDA(cudaMalloc(&c->WprepT[j], (size_t)4 * g.H * 128 * g.d * 2));
       if (!c->WpostT[j]) LIME_CUDA(cudaMalloc(&c->WpostT[j], (size_t)2 * c->d_ff * g.H * g.d * 2));
       if ((s = launch_transpose_bf16(w->Wo[j], c->d_ff, g.d, c->WoT[j], st)) != LIME_OK) return s;
-      if ((s = launch_fold_weights(w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], g.d, g.H, c->d_ff, c->attn_scale,
+      if ((s = launch_fold_weights(w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], g.d, g.H, c->d_ff,
+                                   c->attn_scale * 1.4426950408889634f /* scores leave the fold in the log2 domain */,
                                    c->WprepT[j], c->WpostT[j], st)) != LIME_OK)
         return s;
     }

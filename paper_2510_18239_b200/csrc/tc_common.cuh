@@ -166,6 +166,24 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const float (&v)[1
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+        "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+        "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+        "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])),
+        "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])), "r"(__float_as_uint(v[16])),
+        "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])),
+        "r"(__float_as_uint(v[23])), "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])),
+        "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])), "r"(__float_as_uint(v[28])),
+        "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+
 // ----------------------------------------------------------------------------- tcgen05.mma (bf16 x bf16 -> fp32)
 // Instruction descriptor, kind::f16: D fp32, A and B bf16, both operands K-major unless flagged, M x N tile.
 __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, bool a_mn_major = false, bool b_mn_major = false) {
@@ -226,6 +244,10 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 // 128-byte swizzle.  Returns false if the driver entry point is unavailable or the encode fails.
 bool make_tmap_bf16_sw128(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
                           uint32_t box_rows);
+// Kernels that need more than 48 KB of dynamic shared memory must have the limit raised once per device; `done` is
+// the caller's per-kernel record (one flag per device ordinal).
+constexpr int kMaxDeviceOrdinals = 64;
+lime_status ensure_dynamic_smem(const void* kernel, int bytes, bool (&done)[kMaxDeviceOrdinals]);
 // Row-major bf16 matrix [rows x cols], cols <= 256, box [box_rows x cols] (whole rows), no swizzle.
 bool make_tmap_bf16_plain(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
                           uint32_t box_rows);

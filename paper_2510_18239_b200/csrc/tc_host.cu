@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
@@ -37,6 +38,17 @@ bool make_tmap_bf16_sw128(CUtensorMap* out, const void* base, uint64_t rows, uin
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+lime_status ensure_dynamic_smem(const void* kernel, int bytes, bool (&done)[kMaxDeviceOrdinals]) {
+  int dev = 0;
+  LIME_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDeviceOrdinals) return LIME_INVALID_ARG;
+  if (!done[dev]) {
+    LIME_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done[dev] = true;
+  }
+  return LIME_OK;
 }
 
 // Same matrix, box [box_rows x cols] covering whole rows, no swizzle (rows land back to back in shared memory).
