@@ -1,13 +1,11 @@
-// Link-row algebra of the XOR layers as tcgen05 GEMMs (bf16 in, fp32 accumulate in TMEM).
+// Link-side preparation GEMM of the XOR layers on tcgen05 (bf16 in, fp32 accumulate in TMEM).
 //
-// The B*ell link rows of a layer go through three dense contractions per layer (weights folded once at set-up,
-// see k_link_prep.cu):
 //   PREP   LN(T) [rows x d] . Wprep [d x 4*H*128]  -> folded queries Q2, folded keys K2 (+ their row sums) and the
-//          folded gate / up operands G2t, U2t that the streaming kernels contract against the history (Eq. 7)
-//   GLU    Ohat [rows x H*d] . [Mvg | Mvu] [H*d x 2f] -> SiLU(gate) * up      (value projection + GatedMLP input, Eq. 5)
-//   F32    U [rows x f] . W_o [f x d]               -> link rows of the layer's output, fp32  (Eq. 8 terms)
-// One CTA per 128-row x N_TILE output tile: warp 0 streams K blocks of A and B with TMA through a stage ring,
-// warp 1 issues the MMAs, warps 2-5 (one thread per output row = TMEM lane) run the epilogue.
+//          folded gate / up operands G2t, U2t that the streaming kernels contract against the history (Eq. 7);
+//          weights folded once at set-up, see k_link_prep.cu
+// One CTA per 128-row x 128-column output tile: warp 0 streams K blocks of A and B with TMA through a stage ring,
+// warp 1 issues the MMAs, warps 2-5 (one thread per output row = TMEM lane) run the epilogue.  The GatedMLP on the
+// link rows lives in k_link_mlp_tc.cu.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
@@ -16,7 +14,7 @@ namespace lime {
 constexpr int GM_THREADS = 192, GM_MAX_STAGES = 6;
 constexpr uint32_t GM_SUB = 128 * 128;    // [128 rows x 64 bf16]
 
-enum { GM_EPI_PREP = 0, GM_EPI_GLU = 1, GM_EPI_F32 = 2 };
+enum { GM_EPI_PREP = 0 };
 
 struct GemmParams {
   int64_t M;            // valid rows of A / C
@@ -26,9 +24,6 @@ struct GemmParams {
   int ell, H, shared_rows;          // rows are (user, link): user = row / ell
   __nv_bfloat16 *Q2, *K2, *G2t, *U2t;
   float *cQ, *cK;
-  // GLU: out bf16 [M x 128]; F32: out fp32 [M x n_total]
-  void* out;
-  int n_total;
   int* err;
 };
 
@@ -82,7 +77,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         mbar_arrive_expect_tx(&full[s], STAGE);
         tma_load_2d_hint(st, &tmA, kb * 64, m0, &full[s], pol);
         tma_load_2d_hint(st + GM_SUB, &tmB, kb * 64, nt * NT, &full[s], pol);
-        if (NT == 256) tma_load_2d_hint(st + GM_SUB + GM_SUB, &tmB, kb * 64, nt * NT + 128, &full[s], pol);
       }
       if (!ok || *(volatile int*)p.err != 0)
         for (int j = 0; j < kb && j < S; ++j) mbar_wait_quiet(&full[(kb - 1 - j) % S], (uint32_t)((kb - 1 - j) / S) & 1u);
@@ -151,37 +145,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
           }
         }
-      } else if (EPI == GM_EPI_GLU) {
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + row * 128;
-#pragma unroll
-        for (int c = 0; c < 128; c += 16) {
-          float g[16], u[16];
-          tmem_ld_32x16(lane_addr + c, g);
-          tmem_ld_32x16(lane_addr + 128 + c, u);
-          tmem_wait_ld();
-          float y[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) y[j] = silu_f(g[j]) * u[j];
-          if (valid) {
-            uint4 o0, o1;
-            o0.x = gm_pack(y[0], y[1]); o0.y = gm_pack(y[2], y[3]); o0.z = gm_pack(y[4], y[5]); o0.w = gm_pack(y[6], y[7]);
-            o1.x = gm_pack(y[8], y[9]); o1.y = gm_pack(y[10], y[11]); o1.z = gm_pack(y[12], y[13]); o1.w = gm_pack(y[14], y[15]);
-            *reinterpret_cast<uint4*>(dst + c) = o0;
-            *reinterpret_cast<uint4*>(dst + c + 8) = o1;
-          }
-        }
-      } else {
-        float* dst = reinterpret_cast<float*>(p.out) + row * p.n_total + (int64_t)nt * NT;
-#pragma unroll
-        for (int c = 0; c < NT; c += 16) {
-          float v[16];
-          tmem_ld_32x16(lane_addr + c, v);
-          tmem_wait_ld();
-          if (valid) {
-#pragma unroll
-            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4*>(dst + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-          }
-        }
       }
     }
   }
@@ -221,18 +184,6 @@ lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st) {
   // segments: Q2 | K2 | G2 | U2, H n-tiles each; the last layer needs only the queries
   const int n_tiles = (a.need_hist ? 4 : 1) * a.H;
   return launch_gemm<GM_EPI_PREP, 128>(a.A, a.M, 128, a.Bt, 4 * a.H * 128, n_tiles, p, "k_gemm_tc_prep", st);
-}
-
-lime_status launch_gemm_glu(const LinkGemmArgs& a, cudaStream_t st) {
-  GemmParams p{};
-  p.out = a.out; p.err = a.err;
-  return launch_gemm<GM_EPI_GLU, 256>(a.A, a.M, a.K, a.Bt, 256, 1, p, "k_gemm_tc_glu", st);
-}
-
-lime_status launch_gemm_f32(const LinkGemmArgs& a, cudaStream_t st) {
-  GemmParams p{};
-  p.out = a.out; p.n_total = 128; p.err = a.err;
-  return launch_gemm<GM_EPI_F32, 128>(a.A, a.M, a.K, a.Bt, 128, 1, p, "k_gemm_tc_f32", st);
 }
 
 }  // namespace lime

@@ -411,7 +411,6 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       const int t = t_begin + g;
       const int b = tu.of(p.tile_start, p.B, t);
       const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
-      const bool valid = row0 + (int)r < p.off[b + 1];
       float v[HU_COLS];
       tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
       tmem_wait_ld();
@@ -441,16 +440,32 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < HU_COLS; ++j) v[j] *= rstd;
       }
-      if (valid) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * HU_D + col0);
+      // bf16 row part = 4 chunks of 16 bytes.  A 4 x 4 transpose of chunks inside each group of four lanes (two
+      // butterfly steps of warp shuffles) leaves lane 4j+i with chunk i of rows 4j..4j+3, so that every store
+      // instruction writes whole 64-byte row parts (full sectors) instead of 32 scattered 16-byte pieces.
+      uint4 tch[4];
 #pragma unroll
-        for (int c8 = 0; c8 < HU_COLS / 8; ++c8) {
-          uint4 o;
-          o.x = pack_bf16(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = pack_bf16(v[c8 * 8 + 2], v[c8 * 8 + 3]);
-          o.z = pack_bf16(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = pack_bf16(v[c8 * 8 + 6], v[c8 * 8 + 7]);
-          dst[c8] = o;
-        }
+      for (int c8 = 0; c8 < 4; ++c8) {
+        tch[c8].x = pack_bf16(v[c8 * 8 + 0], v[c8 * 8 + 1]); tch[c8].y = pack_bf16(v[c8 * 8 + 2], v[c8 * 8 + 3]);
+        tch[c8].z = pack_bf16(v[c8 * 8 + 4], v[c8 * 8 + 5]); tch[c8].w = pack_bf16(v[c8 * 8 + 6], v[c8 * 8 + 7]);
       }
+      auto xchg = [&](uint4& keep_lo, uint4& keep_hi, bool upper, int dist) {
+        // lanes with `upper` clear give away keep_hi and receive into it; lanes with it set give away keep_lo
+        uint4 send = upper ? keep_lo : keep_hi, recv;
+        recv.x = __shfl_xor_sync(0xffffffffu, send.x, dist); recv.y = __shfl_xor_sync(0xffffffffu, send.y, dist);
+        recv.z = __shfl_xor_sync(0xffffffffu, send.z, dist); recv.w = __shfl_xor_sync(0xffffffffu, send.w, dist);
+        if (upper) keep_lo = recv; else keep_hi = recv;
+      };
+      xchg(tch[0], tch[1], (lane & 1) != 0, 1);
+      xchg(tch[2], tch[3], (lane & 1) != 0, 1);
+      xchg(tch[0], tch[2], (lane & 2) != 0, 2);
+      xchg(tch[1], tch[3], (lane & 2) != 0, 2);
+      const int rbase = row0 + q * 32 + (lane & ~3);          // first of the four rows this lane group holds
+      const int row_end = p.off[b + 1];
+#pragma unroll
+      for (int m = 0; m < 4; ++m)
+        if (rbase + m < row_end)
+          *reinterpret_cast<uint4*>(p.out + (int64_t)(rbase + m) * HU_D + col0 + (lane & 3) * 8) = tch[m];
       return true;
     };
 

@@ -1,0 +1,290 @@
+// GatedMLP on the link rows of one XOR layer, fused with everything that consumes its result (bf16 operands, fp32
+// accumulation in TMEM):
+//
+//   T^j = GatedMLP(O[T]) = ( SiLU(O[T] W_g) * (O[T] W_u) ) W_o                                   (Eq. 5 on link rows, Eq. 8)
+//
+// The attention kernel leaves Ohat [rows x H*d]: per (user, link) row the H un-projected head outputs side by side;
+// W_V is folded into the gate / up weights (k_link_prep.cu), so
+//   1. [gate | up] [128 x 2f] = Ohat_tile [128 x H*d] . [Mvg | Mvu]     streamed over K = H*d through a TMA stage ring
+//   2. U = SiLU(gate) * up -> bf16 -> shared memory (A operand of the next contraction)
+//   3. T^j = U [128 x f] . W_o [f x d]
+// and the epilogue of step 3, one thread pair per row, writes what the rest of the layer stack needs:
+//   - T^j as fp32 (only when the caller asks for the layer's link rows)
+//   - L^P (+)= T^j, the running sum of Eq. 8
+//   - LN(T^j) as bf16, the A operand of the next layer's link-side GEMM (LayerNorm before the projections, App. C)
+//   - on the last layer, the link states bf16(L^P) of Eq. 4 when no candidate-side value projection follows
+// One CTA per 128 rows.  Warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 epilogue (two threads per row, 64 columns
+// each; a warp may only touch the TMEM lane quarter warp_id % 4).
+//
+// Built for d = d_ff = 128.
+#include "lime_common.cuh"
+#include "tc_common.cuh"
+
+namespace lime {
+
+constexpr int LM_THREADS = 64 + 256, LM_STAGES = 3;
+constexpr uint32_t LM_SUB = 128 * 128;                       // [128 rows x 64 bf16]
+constexpr uint32_t LM_STAGE = 3 * LM_SUB;                    // A tile + 256 rows of B
+constexpr uint32_t LM_OFF_WO = LM_STAGES * LM_STAGE;         // [d x f] 2 K-blocks
+constexpr uint32_t LM_OFF_U = LM_OFF_WO + 2 * LM_SUB;        // U [128 x f] 2 K-blocks
+constexpr uint32_t LM_OFF_EXCH = LM_OFF_U + 2 * LM_SUB;      // [2 slots][2 halves][128] floats
+constexpr uint32_t LM_OFF_BAR = LM_OFF_EXCH + 4 * 128 * 4;
+constexpr uint32_t LM_SMEM = LM_OFF_BAR + 256;
+
+struct LinkMlpParams {
+  int64_t M;                    // rows (users x links)
+  int kblocks;                  // H*d / 64
+  float* T_out;                 // nullable: fp32 [M x d]
+  float* LP;                    // nullable: fp32 [M x d] running sum
+  int lp_accumulate;            // 0: LP = T, 1: LP += T
+  __nv_bfloat16* That_next;     // nullable: bf16 [M x d] = LN(T) (or T when ln == 0)
+  __nv_bfloat16* link_states;   // nullable: bf16 [M x d] = LP after this layer
+  int ln;
+  float ln_eps;
+  int* err;
+};
+
+__device__ __forceinline__ uint32_t lm_pack(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float lm_tanh(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t lm_chunk(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
+
+__global__ void __launch_bounds__(LM_THREADS, 1)
+k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const __grid_constant__ CUtensorMap tmWo, const LinkMlpParams p) {
+  using namespace tc;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (threadIdx.x == 0) atomicCAS(p.err, 0, 93);
+    return;
+  }
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LM_OFF_BAR);
+  uint64_t* full = bars;                 // [LM_STAGES]
+  uint64_t* empty = bars + LM_STAGES;    // [LM_STAGES]
+  uint64_t* wo_full = bars + 2 * LM_STAGES;
+  uint64_t* gu_full = wo_full + 1;
+  uint64_t* u_ready = wo_full + 2;       // 8 warps
+  uint64_t* out_full = wo_full + 3;
+  uint64_t* pair_bar = wo_full + 4;      // [4], 2 warps each
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wo_full + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.x * 128;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < LM_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(wo_full, 1); mbar_init(gu_full, 1); mbar_init(u_ready, 8); mbar_init(out_full, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
+    fence_barrier_init();
+    prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmWo);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  constexpr uint32_t COL_GU = 0, COL_OUT = 256;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol = policy_evict_last();
+      mbar_arrive_expect_tx(wo_full, 2 * LM_SUB);
+      for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + LM_OFF_WO + kb * LM_SUB, &tmWo, kb * 64, 0, wo_full, pol);
+      bool ok = true;
+      int kb = 0;
+      for (; kb < p.kblocks; ++kb) {
+        const int s = kb % LM_STAGES;
+        if (!mbar_wait(&empty[s], ((uint32_t)(kb / LM_STAGES) & 1u) ^ 1u, p.err, 71)) { ok = false; break; }
+        uint8_t* st = smem + (size_t)s * LM_STAGE;
+        mbar_arrive_expect_tx(&full[s], LM_STAGE);
+        tma_load_2d_hint(st, &tmA, kb * 64, m0, &full[s], pol);
+        tma_load_2d_hint(st + LM_SUB, &tmB, kb * 64, 0, &full[s], pol);
+        tma_load_2d_hint(st + 2 * LM_SUB, &tmB, kb * 64, 128, &full[s], pol);
+      }
+      if (!ok || *(volatile int*)p.err != 0) {
+        for (int j = 0; j < kb && j < LM_STAGES; ++j)
+          mbar_wait_quiet(&full[(kb - 1 - j) % LM_STAGES], (uint32_t)((kb - 1 - j) / LM_STAGES) & 1u);
+        mbar_wait_quiet(wo_full, 0);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_256 = make_idesc_bf16(128, 256);
+      constexpr uint32_t idesc_128 = make_idesc_bf16(128, 128);
+      const uint32_t sbase = smem_u32(smem);
+      bool ok = true;
+      for (int kb = 0; kb < p.kblocks && ok; ++kb) {
+        const int s = kb % LM_STAGES;
+        if (!mbar_wait(&full[s], (uint32_t)(kb / LM_STAGES) & 1u, p.err, 72)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_bf16_ss(tmem_base + COL_GU, make_sdesc_k_sw128(sbase + s * LM_STAGE + k * 32),
+                      make_sdesc_k_sw128(sbase + s * LM_STAGE + LM_SUB + k * 32), idesc_256, (kb | k) != 0);
+        mma_commit(&empty[s]);
+      }
+      if (ok) {
+        mma_commit(gu_full);
+        ok = mbar_wait(wo_full, 0, p.err, 74) && mbar_wait(u_ready, 0, p.err, 75);
+      }
+      if (ok) {
+        tc_fence_after();
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t o = (uint32_t)(kk >> 2) * LM_SUB + (uint32_t)(kk & 3) * 32;
+          mma_bf16_ss(tmem_base + COL_OUT, make_sdesc_k_sw128(sbase + LM_OFF_U + o), make_sdesc_k_sw128(sbase + LM_OFF_WO + o),
+                      idesc_128, kk != 0);
+        }
+        mma_commit(out_full);
+      }
+    }
+  } else {
+    const int ew = warp - 2;                                   // 0..7
+    const int q = warp & 3;
+    const int half = ew >> 2;
+    const uint32_t r = (uint32_t)(q * 32 + lane);
+    const int64_t row = (int64_t)m0 + r;
+    const bool valid = row < p.M;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+    float* exch = reinterpret_cast<float*>(smem + LM_OFF_EXCH);
+    if (mbar_wait(gu_full, 0, p.err, 73)) {
+      tc_fence_after();
+      // 2. U = SiLU(gate) * up for this thread's 64 hidden columns (K-block `half` of the A operand)
+      uint8_t* ub = smem + LM_OFF_U + half * LM_SUB;
+#pragma unroll
+      for (int c = 0; c < 64; c += 32) {
+        float gt[32], up[32];
+        tmem_ld_32x32(lane_addr + COL_GU + half * 64 + c, gt);
+        tmem_ld_32x32(lane_addr + COL_GU + 128 + half * 64 + c, up);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c8 = 0; c8 < 4; ++c8) {
+          float y[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const float hx = 0.5f * gt[c8 * 8 + j];
+            y[j] = fmaf(hx, lm_tanh(hx), hx) * up[c8 * 8 + j];
+          }
+          uint4 o;
+          o.x = lm_pack(y[0], y[1]); o.y = lm_pack(y[2], y[3]); o.z = lm_pack(y[4], y[5]); o.w = lm_pack(y[6], y[7]);
+          *reinterpret_cast<uint4*>(ub + lm_chunk(r, (uint32_t)(c >> 3) + c8)) = o;
+        }
+      }
+      tc_fence_before();
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(u_ready);
+
+      // 3'. epilogue of T = U . W_o: this thread's 64 columns of its row
+      if (mbar_wait(out_full, 0, p.err, 76)) {
+        tc_fence_after();
+        float v[64];
+        {
+          float v0[32], v1[32];
+          tmem_ld_32x32(lane_addr + COL_OUT + half * 64, v0);
+          tmem_ld_32x32(lane_addr + COL_OUT + half * 64 + 32, v1);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
+        }
+        const int64_t o64 = row * 128 + half * 64;
+        if (valid && p.T_out) {
+#pragma unroll
+          for (int j = 0; j < 64; j += 4) *reinterpret_cast<float4*>(p.T_out + o64 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+        if (valid && p.LP) {
+          // running sum of Eq. 8; on the last layer it also leaves as the link states
+#pragma unroll
+          for (int j = 0; j < 64; j += 8) {
+            float s[8];
+            if (p.lp_accumulate) {
+              const float4 a = *reinterpret_cast<const float4*>(p.LP + o64 + j), b = *reinterpret_cast<const float4*>(p.LP + o64 + j + 4);
+              s[0] = a.x + v[j]; s[1] = a.y + v[j + 1]; s[2] = a.z + v[j + 2]; s[3] = a.w + v[j + 3];
+              s[4] = b.x + v[j + 4]; s[5] = b.y + v[j + 5]; s[6] = b.z + v[j + 6]; s[7] = b.w + v[j + 7];
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) s[i] = v[j + i];
+            }
+            *reinterpret_cast<float4*>(p.LP + o64 + j) = make_float4(s[0], s[1], s[2], s[3]);
+            *reinterpret_cast<float4*>(p.LP + o64 + j + 4) = make_float4(s[4], s[5], s[6], s[7]);
+            if (p.link_states) {
+              uint4 o;
+              o.x = lm_pack(s[0], s[1]); o.y = lm_pack(s[2], s[3]); o.z = lm_pack(s[4], s[5]); o.w = lm_pack(s[6], s[7]);
+              *reinterpret_cast<uint4*>(p.link_states + o64 + j) = o;
+            }
+          }
+        }
+        if (p.That_next) {
+          // LN(T) for the next layer's link-side GEMM: the two halves of a row exchange their partial sums
+          bool ok = true;
+          if (p.ln) {
+            uint32_t uses = 0;
+            auto pair_sync = [&](int where) {
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&pair_bar[q]);
+              const bool w = mbar_wait(&pair_bar[q], uses & 1u, p.err, where);
+              ++uses;
+              return w;
+            };
+            float s = 0.f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) s += v[j];
+            exch[half * 128 + r] = s;
+            ok = pair_sync(77);
+            const float mu = (s + exch[(half ^ 1) * 128 + r]) * (1.0f / 128);
+            float var = 0.f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
+            exch[256 + half * 128 + r] = var;
+            ok = ok && pair_sync(78);
+            const float rstd = rsqrtf((var + exch[256 + (half ^ 1) * 128 + r]) * (1.0f / 128) + p.ln_eps);
+#pragma unroll
+            for (int j = 0; j < 64; ++j) v[j] *= rstd;
+          }
+          if (ok && valid) {
+#pragma unroll
+            for (int j = 0; j < 64; j += 8) {
+              uint4 o;
+              o.x = lm_pack(v[j], v[j + 1]); o.y = lm_pack(v[j + 2], v[j + 3]); o.z = lm_pack(v[j + 4], v[j + 5]); o.w = lm_pack(v[j + 6], v[j + 7]);
+              *reinterpret_cast<uint4*>(p.That_next + o64 + j) = o;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+lime_status launch_link_mlp_tc(const LinkMlpArgs& a, cudaStream_t st) {
+  if (a.M == 0) return LIME_OK;
+  CUtensorMap tmA, tmB, tmWo;
+  if (!make_tmap_bf16_sw128(&tmA, a.Ohat, (uint64_t)a.M, (uint64_t)a.K, (uint64_t)a.K, 128) ||
+      !make_tmap_bf16_sw128(&tmB, a.WpostT, 256, (uint64_t)a.K, (uint64_t)a.K, 128) ||
+      !make_tmap_bf16_sw128(&tmWo, a.WoT, 128, 128, 128, 128))
+    return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+  LinkMlpParams p;
+  p.M = a.M; p.kblocks = a.K / 64; p.T_out = a.T_out; p.LP = a.LP; p.lp_accumulate = a.lp_accumulate;
+  p.That_next = (__nv_bfloat16*)a.That_next; p.link_states = (__nv_bfloat16*)a.link_states; p.ln = a.ln; p.ln_eps = a.ln_eps;
+  p.err = a.err;
+  static bool smem_set[kMaxDeviceOrdinals] = {};
+  lime_status es = ensure_dynamic_smem((const void*)k_link_mlp_tc, (int)LM_SMEM, smem_set);
+  if (es != LIME_OK) return es;
+  ProfScope _p("k_link_mlp_tc", st);
+  k_link_mlp_tc<<<(unsigned)((a.M + 127) / 128), LM_THREADS, LM_SMEM, st>>>(tmA, tmB, tmWo, p);
+  LIME_LAUNCH_CHECK("k_link_mlp_tc");
+  return LIME_OK;
+}
+
+}  // namespace lime

@@ -103,46 +103,99 @@ static bool layer_on_tensor_cores(const Ctx* c, int layer) {
 }
 
 // One XOR layer, tensor-core path: three link-row GEMMs around the two streaming attention kernels.
-// `in_prenorm`: hist_in holds LayerNorm-ed rows already (written by the previous layer with `out_ln`); `out_ln`:
-// write LayerNorm(S') to hist_out.  Both are internal to lime_encode_user; the public layer call passes 0, 0.
-static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B, int64_t total,
-                                const float* links_in, int links_shared, void* hist_out, float* links_out,
-                                const Workspace& w, int in_prenorm, int out_ln, cudaStream_t st) {
+// Link-side operands of one layer's two attention directions (folded through the weights, k_link_prep.cu).
+struct LinkOperands {
+  const void *Q2, *K2, *G2t, *U2t;
+  const float *cQ, *cK;
+  int shared;                 // one set for every user (T^0 = L) or one per user
+};
+
+// LN(links_in) -> bf16 -> PREP GEMM: the operands of `layer` for `rows` link rows, written to the given buffers.
+static lime_status make_link_operands(Ctx* c, int layer, const void* That, int64_t rows, int need_hist, void* Q2, void* K2,
+                                      void* G2t, void* U2t, float* cQ, float* cK, cudaStream_t st) {
+  const lime_config& g = c->cfg;
+  LinkGemmArgs gp{};
+  gp.A = That; gp.M = rows; gp.K = g.d; gp.Bt = c->WprepT[layer]; gp.ell = g.ell; gp.H = g.H;
+  gp.need_hist = need_hist; gp.Q2 = Q2; gp.K2 = K2; gp.G2t = G2t; gp.U2t = U2t; gp.cQ = cQ; gp.cK = cK;
+  gp.err = c->dev_err;
+  return launch_gemm_prep(gp, st);
+}
+
+// The streaming part of one XOR layer on tensor cores: links<-history attention, GatedMLP on the link rows with its
+// fused consumers (`mlp` carries the outputs wanted), and the history update.  `hist_ln`: apply LayerNorm to the rows
+// read (0 when they were stored normalised by the previous layer); `out_ln`: store LayerNorm(S').
+static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B, int64_t total,
+                                 const LinkOperands& ops, void* hist_out, int hist_ln, int out_ln, LinkMlpArgs mlp,
+                                 const Workspace& w, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
-  const int hist_ln = (g.ln && !in_prenorm) ? 1 : 0;
-  const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
-  const int64_t BL = (int64_t)B * g.ell;
-  // LN(T) -> bf16, then one GEMM gives every folded link-side operand of both attention directions
-  if ((s = launch_ln_rows_bf16(links_in, link_rows, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
-  LinkGemmArgs gp{};
-  gp.A = w.That; gp.M = link_rows; gp.K = g.d; gp.Bt = c->WprepT[layer]; gp.ell = g.ell; gp.H = g.H;
-  gp.need_hist = hist_out != nullptr; gp.Q2 = w.Q2; gp.K2 = w.K2; gp.G2t = w.G2t; gp.U2t = w.U2t; gp.cQ = w.cQ; gp.cK = w.cK;
-  gp.err = c->dev_err;
-  if ((s = launch_gemm_prep(gp, st)) != LIME_OK) return s;
   // O[T]: links attend over the stored history (keys = values = history rows), chunks merged and normalised
   LinkAttnArgs la{};
-  la.hist = hist_in; la.total = total; la.Q2 = w.Q2; la.cQ = w.cQ; la.off = off; la.chunk_start = w.chunk_start; la.B = B;
-  la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = links_shared;
-  la.ln = hist_ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat; la.err = c->dev_err;
+  la.hist = hist_in; la.total = total; la.Q2 = ops.Q2; la.cQ = ops.cQ; la.off = off; la.chunk_start = w.chunk_start; la.B = B;
+  la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = ops.shared;
+  la.ln = hist_ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
+  la.err = c->dev_err;
   if ((s = launch_link_attn_tc(la, st)) != LIME_OK) return s;
   if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
     return s;
-  // links_out = GatedMLP(O[T]) with W_V folded into the gate / up weights
-  LinkGemmArgs gg{};
-  gg.A = w.Ohat; gg.M = BL; gg.K = g.H * g.d; gg.Bt = c->WpostT[layer]; gg.out = w.UTb; gg.err = c->dev_err;
-  if ((s = launch_gemm_glu(gg, st)) != LIME_OK) return s;
-  LinkGemmArgs go{};
-  go.A = w.UTb; go.M = BL; go.K = c->d_ff; go.Bt = c->WoT[layer]; go.out = links_out; go.err = c->dev_err;
-  if ((s = launch_gemm_f32(go, st)) != LIME_OK) return s;
+  // T^j = GatedMLP(O[T]) with W_V folded into the gate / up weights, and what the next step needs from it
+  mlp.Ohat = w.Ohat; mlp.M = (int64_t)B * g.ell; mlp.K = g.H * g.d; mlp.WpostT = c->WpostT[layer]; mlp.WoT = c->WoT[layer];
+  mlp.ln = g.ln; mlp.ln_eps = c->ln_eps; mlp.err = c->dev_err;
+  if ((s = launch_link_mlp_tc(mlp, st)) != LIME_OK) return s;
   if (hist_out) {
     // history attends back over the links; scores, per-head softmax, value mix and GatedMLP in one fused kernel
     HistUpdateArgs hu{};
-    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = w.K2; hu.G2t = w.G2t; hu.U2t = w.U2t;
-    hu.cK = w.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
-    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = links_shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
+    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = ops.K2; hu.G2t = ops.G2t; hu.U2t = ops.U2t;
+    hu.cK = ops.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
+    hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = ops.shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
     hu.out_ln = out_ln; hu.err = c->dev_err;
     if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
+  }
+  return LIME_OK;
+}
+
+// One XOR layer, tensor-core path, for the public layer call: link rows in and out as fp32.
+static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B, int64_t total,
+                                const float* links_in, int links_shared, void* hist_out, float* links_out,
+                                const Workspace& w, cudaStream_t st) {
+  const lime_config& g = c->cfg;
+  lime_status s;
+  const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
+  if ((s = launch_ln_rows_bf16(links_in, link_rows, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
+  if ((s = make_link_operands(c, layer, w.That, link_rows, hist_out != nullptr, w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, st)) != LIME_OK)
+    return s;
+  LinkOperands ops{w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, links_shared};
+  LinkMlpArgs mlp{};
+  mlp.T_out = links_out;
+  return tc_layer_core(c, layer, hist_in, off, B, total, ops, hist_out, g.ln, 0, mlp, w, st);
+}
+
+// lime_encode_user on the tensor-core path: per layer one link-side GEMM (none on the first layer when the links are
+// the shared L: its operands are weights-only and were formed at lime_set_weights), then the streaming kernels.
+// Between layers the history is kept LayerNorm-ed (every consumer normalises it first, Eq. 1 with App. C's LayerNorm),
+// so only the first layer pays for the statistics.
+static lime_status encode_user_tc(Ctx* c, const void* hist, const int32_t* off, int32_t B, int64_t total,
+                                  const float* link_ctx, void* link_states, const Workspace& w, cudaStream_t st) {
+  const lime_config& g = c->cfg;
+  lime_status s;
+  const int64_t BL = (int64_t)B * g.ell;
+  for (int j = 0; j < g.n_layers; ++j) {
+    const bool last = j == g.n_layers - 1;
+    LinkOperands ops;
+    if (j == 0 && !link_ctx) {
+      ops = LinkOperands{c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_cQ, c->sh_cK, 1};
+    } else {
+      if (j == 0 && (s = launch_ln_rows_bf16(link_ctx, BL, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
+      if ((s = make_link_operands(c, j, w.That, BL, !last, w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, st)) != LIME_OK) return s;
+      ops = LinkOperands{w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, 0};
+    }
+    LinkMlpArgs mlp{};
+    mlp.LP = w.LP; mlp.lp_accumulate = j > 0;                                   // L^P = sum_j T^j  (Eq. 8)
+    mlp.That_next = last ? nullptr : w.That;
+    mlp.link_states = (last && !c->w.cand_Wv) ? link_states : nullptr;
+    s = tc_layer_core(c, j, j == 0 ? hist : w.S, off, B, total, ops, last ? nullptr : w.S, (g.ln && j == 0) ? 1 : 0,
+                      (g.ln && !last) ? 1 : 0, mlp, w, st);
+    if (s != LIME_OK) return s;
   }
   return LIME_OK;
 }
@@ -150,16 +203,14 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
 // One XOR layer on a carved workspace (see lime_xor_layer in lime.h for the contract).
 static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B,
                                   int64_t total, const float* links_in, int links_shared, void* hist_out,
-                                  float* links_out, const Workspace& w, bool schedules_ready, int in_prenorm, int out_ln,
-                                  cudaStream_t st) {
+                                  float* links_out, const Workspace& w, bool schedules_ready, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
   if (!schedules_ready) {
-    if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
-    if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
+    if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, st)) != LIME_OK) return s;
   }
   if (layer_on_tensor_cores(c, layer))
-    return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, in_prenorm, out_ln, st);
+    return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, st);
 
   // ---- generic path on CUDA cores (fp32 storage, other shapes, SiLU attention, no GatedMLP) ----
   const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
@@ -317,6 +368,7 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = nullptr;
+  c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff_hl, 2 * (size_t)2 * g.ell * g.d);
@@ -343,6 +395,8 @@ lime_status lime_destroy(lime_ctx* ctx) {
   cudaFree(c->links32);
   cudaFree(c->dev_err);
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); }
+  cudaFree(c->sh_That); cudaFree(c->sh_Q2); cudaFree(c->sh_K2); cudaFree(c->sh_G2t); cudaFree(c->sh_U2t); cudaFree(c->sh_cQ);
+  cudaFree(c->sh_cK);
   delete c;
   return LIME_OK;
 }
@@ -380,6 +434,21 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
                                    c->WprepT[j], c->WpostT[j], st)) != LIME_OK)
         return s;
     }
+    // first-layer operands for the shared links T^0 = L: LN(L) through the PREP GEMM, once
+    const size_t HL = (size_t)g.H * g.ell;
+    if (!c->sh_That) {
+      LIME_CUDA(cudaMalloc(&c->sh_That, (size_t)g.ell * g.d * 2));
+      LIME_CUDA(cudaMalloc(&c->sh_Q2, HL * g.d * 2));
+      LIME_CUDA(cudaMalloc(&c->sh_K2, HL * g.d * 2));
+      LIME_CUDA(cudaMalloc(&c->sh_G2t, (size_t)c->d_ff * HL * 2));
+      LIME_CUDA(cudaMalloc(&c->sh_U2t, (size_t)c->d_ff * HL * 2));
+      LIME_CUDA(cudaMalloc(&c->sh_cQ, HL * 4));
+      LIME_CUDA(cudaMalloc(&c->sh_cK, HL * 4));
+    }
+    if ((s = launch_ln_rows_bf16(c->links32, g.ell, g.d, g.ln, c->ln_eps, c->sh_That, st)) != LIME_OK) return s;
+    if ((s = make_link_operands(c, 0, c->sh_That, g.ell, g.n_layers > 1, c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_cQ,
+                                c->sh_cK, st)) != LIME_OK)
+      return s;
   }
   c->have_weights = true;
   return LIME_OK;
@@ -434,7 +503,7 @@ lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hist_in, co
   const size_t pad = base - static_cast<char*>(ws);
   Workspace w = carve(c, base, B, total_tokens);
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
-  return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false, 0, 0,
+  return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false,
                         static_cast<cudaStream_t>(stream));
 }
 
@@ -455,20 +524,20 @@ lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   lime_status s;
-  if ((s = launch_tile_schedule(off, B, w.chunk, w.chunk_start, st)) != LIME_OK) return s;
-  if ((s = launch_tile_schedule(off, B, kHistTile, w.tile_start, st)) != LIME_OK) return s;
+  if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, st)) != LIME_OK) return s;
   const int64_t BLd = (int64_t)B * g.ell * g.d;
-  for (int j = 0; j < g.n_layers; ++j) {
-    const bool last = j == g.n_layers - 1;
-    const float* lin = j == 0 ? (link_ctx ? link_ctx : c->links32) : w.T;
-    const int shared = (j == 0 && !link_ctx) ? 1 : 0;
-    // tensor-core path: between layers the history is kept LayerNorm-ed (every consumer normalises it first, Eq. 1
-    // with App. C's LayerNorm), so only the first layer pays for the statistics
-    const int keep_norm = (g.ln && layer_on_tensor_cores(c, j)) ? 1 : 0;
-    s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true,
-                       j > 0 ? keep_norm : 0, last ? 0 : keep_norm, st);
-    if (s != LIME_OK) return s;
-    if ((s = launch_axpy(w.T, w.LP, BLd, j == 0, st)) != LIME_OK) return s;   // L^P = sum_j T^j  (Eq. 8)
+  if (layer_on_tensor_cores(c, 0)) {
+    if ((s = encode_user_tc(c, hist, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;
+    if (!c->w.cand_Wv) return LIME_OK;        // the last layer's kernel wrote the link states
+  } else {
+    for (int j = 0; j < g.n_layers; ++j) {
+      const bool last = j == g.n_layers - 1;
+      const float* lin = j == 0 ? (link_ctx ? link_ctx : c->links32) : w.T;
+      const int shared = (j == 0 && !link_ctx) ? 1 : 0;
+      s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true, st);
+      if (s != LIME_OK) return s;
+      if ((s = launch_axpy(w.T, w.LP, BLd, j == 0, st)) != LIME_OK) return s;   // L^P = sum_j T^j  (Eq. 8)
+    }
   }
   // link states = L^P W_V^c (Eq. 4's values), stored as the run's dtype
   const float* src = w.LP;

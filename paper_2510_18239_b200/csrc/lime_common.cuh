@@ -56,6 +56,9 @@ struct Ctx {
   void* WoT[LIME_MAX_LAYERS];    // tensor-core path, per layer (NULL otherwise): W_o transposed [d x d_ff] bf16,
   void* WprepT[LIME_MAX_LAYERS]; //   folded PREP operand [4*H*128 x d], folded link-row GLU operand [2*d_ff x H*d]
   void* WpostT[LIME_MAX_LAYERS];
+  // link-side operands of the first layer for the shared links T^0 = L (weights only, formed at lime_set_weights)
+  void *sh_That, *sh_Q2, *sh_K2, *sh_G2t, *sh_U2t;
+  float *sh_cQ, *sh_cK;
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
   int d_ff, d_h;
@@ -94,6 +97,9 @@ lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const 
 
 // tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B  (work list of per-user token tiles)
 lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st);
+// chunk_start (tile = chunk) and tile_start (tile = tile) in one launch
+lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
+                                   cudaStream_t st);
 
 // Y[r, n] (+)= epilogue( LN?(X[r, :]) . W[:, n] ) for up to three weight matrices sharing X.
 struct LinearArgs {
@@ -179,8 +185,19 @@ struct LinkGemmArgs {
   int* err;
 };
 lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st);
-lime_status launch_gemm_glu(const LinkGemmArgs& a, cudaStream_t st);
-lime_status launch_gemm_f32(const LinkGemmArgs& a, cudaStream_t st);
+
+// GatedMLP on link rows fused with its consumers (k_link_mlp_tc.cu); d = d_ff = 128
+struct LinkMlpArgs {
+  const void* Ohat; int64_t M; int K;          // attention rows [M x K = H*d] bf16
+  const void* WpostT; const void* WoT;         // folded [2f x H*d] and transposed [d x f] weights, bf16
+  float* T_out;                                // nullable: the layer's link rows, fp32 [M x d]
+  float* LP; int lp_accumulate;                // nullable running sum of Eq. 8 (0: assign, 1: add)
+  void* That_next;                             // nullable: bf16 LN(T) for the next layer's link-side GEMM
+  void* link_states;                           // nullable: bf16 copy of LP after this layer
+  int ln; float ln_eps;
+  int* err;
+};
+lime_status launch_link_mlp_tc(const LinkMlpArgs& a, cudaStream_t st);
 
 struct LinkAttnArgs {
   const void* hist; int64_t total;          // [total x d] bf16
