@@ -227,6 +227,10 @@ def workload_config(wl):
             "l2": f"{ROTATE} rotating input sets per step slot (candidate streams total > 126 MB L2)"}
 
 
+def launch_mode(args):
+    return "host launches" if args.no_graph else f"one CUDA graph per input set ({ROTATE}), replayed"
+
+
 # ----------------------------------------------------------------------------- the CUDA arm
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels captured with ncu, keyed by
 # kernel and workload, with the hash of the kernel's source at capture time: once the source changes the figure
@@ -253,7 +257,7 @@ def ncu_traffic(kernel, wl):
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
-    from paper_2510_18239_b200 import binding as Bd
+    from paper_2510_18239_b200 import binding as Bd, shard
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -323,9 +327,31 @@ def run_ours(args, wl):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    for i in range(args.warmup):
+    for i in range(max(args.warmup, ROTATE)):
         step(i)
     barrier()
+
+    # One CUDA graph per rotating input set: the step's launches are recorded once and replayed, so the timed region
+    # holds the library's kernels back to back instead of the host's launch calls.
+    def capture(fn):
+        graphs = []
+        for r in range(ROTATE):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn(r)
+            graphs.append(g)
+        return graphs
+
+    direct_step = step
+    if not args.no_graph:
+        step_graphs = capture(direct_step)
+
+        def step(i):                                   # noqa: F811
+            step_graphs[i % ROTATE].replay()
+
+        for i in range(ROTATE):
+            step(i)
+        barrier()
 
     # ---- timed region: exactly `steps` steps, device-timed, nothing but the library's launches in between
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
@@ -341,11 +367,10 @@ def run_ours(args, wl):
     clocks = sampler.stop() if rank == 0 else None
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = world * wl.B * wl.C * args.steps / (total_ms * 1e-3)
+    # every rank serves its own batch of B users (users are independent: no collective on the data path); the job's
+    # throughput is all ranks' candidates over the slowest rank's device time
+    total_ms = shard.max_over_ranks(total_ms, dev)
+    value = shard.sum_over_ranks(wl.B * wl.C * args.steps, dev) / (total_ms * 1e-3)
 
     # ---- the same steps again with every launch of the library bracketed by CUDA events on its stream: per-kernel
     #      launch durations and the launch count of one step (the brackets add gaps, so this pass is not `value`)
@@ -353,7 +378,7 @@ def run_ours(args, wl):
     cap = 64 * prof_steps + 64
     Bd.lime_profile_start(cap)
     for i in range(prof_steps):
-        step(i)
+        direct_step(i)
     torch.cuda.synchronize()
     records, launches = Bd.lime_profile_stop(cap)
     launches_per_step = launches / prof_steps
@@ -401,24 +426,32 @@ def run_ours(args, wl):
         h_logits.copy_(logits, non_blocking=True)
         return 4 * (wl.B + n + wl.B * wl.C), 4 * wl.B * wl.C
 
-    for i in range(3):
+    for i in range(ROTATE):
         e2e_step(i)
     barrier()
+    e2e_bytes = [e2e_step(i) for i in range(ROTATE)]
+    barrier()
+    if not args.no_graph:
+        e2e_graphs = capture(e2e_step)
+        for i in range(ROTATE):
+            e2e_graphs[i].replay()
+        barrier()
     h2d = d2h = 0
     e0.record()
     for i in range(args.steps):
-        a, b = e2e_step(i)
+        if args.no_graph:
+            e2e_step(i)
+        else:
+            e2e_graphs[i % ROTATE].replay()
+        a, b = e2e_bytes[i % ROTATE]
         h2d += a
         d2h += b
     e1.record()
     torch.cuda.synchronize()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * wl.B * wl.C * args.steps / (e2e_ms * 1e-3)
+    e2e_ms = shard.max_over_ranks(e2e_ms, dev)
+    e2e_value = shard.sum_over_ranks(wl.B * wl.C * args.steps, dev) / (e2e_ms * 1e-3)
     Bd.lime_device_status(ctx)          # raises if any bounded in-kernel wait gave up during the run
 
     if rank == 0:
@@ -471,7 +504,7 @@ def run_ours(args, wl):
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "p50_batch_latency_ms": step_ms[len(step_ms) // 2],
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == synth.BF16 else "f32",
-                "data": "synthetic", "config": workload_config(wl), "clocks": clocks,
+                "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args)), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roofline, "scoring_roofline": scoring,
@@ -496,6 +529,8 @@ def main():
     ap.add_argument("--B", type=int, default=0)
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default="", choices=["", "C", "N"], help="one line per point of the candidate / history sweep")
+    ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying CUDA graphs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = synth.named_workloads()[args.workload]
@@ -507,6 +542,16 @@ def main():
         wl = wl.replace(B=args.B)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.sweep == "C":
+        # latency vs number of candidates (App. F, table a): one JSON line per C, model and batch of `candidate_sweep`
+        base = synth.named_workloads()["candidate_sweep"]
+        for C in synth.CANDIDATE_SWEEP_C:
+            run_ours(args, base.replace(C=C, B=args.B or base.B))
+    elif args.sweep == "N":
+        # latency vs history length (App. F, table b): one JSON line per N, model and batch of `long_history`
+        base = synth.named_workloads()["long_history"]
+        for N in synth.LONG_HISTORY_N:
+            run_ours(args, base.replace(n_min=N, n_max=N, B=args.B or base.B))
     else:
         run_ours(args, wl)
 

@@ -4,4 +4,4 @@
 library (built in-tree by `build`).  Importing the package does not load the CUDA library;
 the first call through `binding` does, and raises if it is missing.
 """
-__all__ = ["synth", "binding", "build"]
+__all__ = ["synth", "binding", "build", "shard"]

@@ -89,8 +89,9 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
 
 // Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
 //   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
-// One block of d threads per user walks the user's H * ell rows.  A user without history gets zeros; a user with a
-// single chunk was already written by the attention kernel (its block returns at once).
+// grid (B, H * ell / MERGE_ROWS): a block of d threads walks MERGE_ROWS rows of one user.  A user without history gets
+// zeros; a user with a single chunk was already written by the attention kernel (its blocks return at once).
+constexpr int MERGE_ROWS = 8;
 __global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H,
                                        const float* __restrict__ part_m, const float* __restrict__ part_s,
                                        const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
@@ -99,7 +100,8 @@ __global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, 
   const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
   if (c1 - c0 == 1) return;
   const int i = threadIdx.x;
-  for (int row = 0; row < HL; ++row) {
+  const int row_end = min(HL, ((int)blockIdx.y + 1) * MERGE_ROWS);
+  for (int row = blockIdx.y * MERGE_ROWS; row < row_end; ++row) {
     const int h = row / ell, l = row % ell;
     float out = 0.f;
     if (c1 > c0) {
@@ -121,7 +123,8 @@ lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int e
                                         const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
   if (B == 0) return LIME_OK;
   ProfScope _p("k_link_attn_merge_norm", st);
-  k_link_attn_merge_norm<<<B, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  const dim3 grid((unsigned)B, (unsigned)((H * ell + MERGE_ROWS - 1) / MERGE_ROWS));
+  k_link_attn_merge_norm<<<grid, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }
