@@ -11,7 +11,8 @@
 //   acc    [HL x d]    += P' [HL x 128] . X_tile            P'_ij = p_ij * rstd_j;  the mean term sum_j P'_ij mu_j is
 //                                                           a per-row scalar subtracted from every column at the end
 //   O[T]_{l,h} = (acc_(h,l) / sum) . W_V[:, head h]         (W_V is folded into the GEMM that follows)
-// HL = H * ell stacked (head, link) rows = 128 TMEM lanes.  Online softmax whose reference maximum is only raised
+// The H * ell stacked (head, link) rows are processed in blocks of 128 = the TMEM lanes (one block per work item; a
+// second block of the same tokens finds them in L2).  Online softmax whose reference maximum is only raised
 // when the true maximum exceeds it by more than 8 (then the accumulator row is rescaled in TMEM), so most tiles need
 // no correction pass.  With LN = false the rows of X are LayerNorm-ed already and the corrections vanish.
 //
@@ -23,7 +24,7 @@
 // normalised and written directly; longer histories leave (max, sum, accumulator) partials per chunk that
 // k_link_attn_merge_norm combines.
 //
-// Built for d = 128 and H * ell = 128.
+// Built for d = 128 and H * ell a multiple of 128.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
@@ -50,6 +51,7 @@ struct LinkAttnParams {
   const int32_t* off;
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
   int B, chunk, shared, ell, H;
+  int HL, RB;                     // stacked (head, link) rows in all, and 128-row blocks of them (one per work item)
   float ln_eps;
   float *part_m, *part_s, *part_acc;   // [items x HL], [items x HL], [items x HL x d]
   __nv_bfloat16* Ohat;                 // [B*ell x H*d]: final rows of single-chunk users
@@ -131,8 +133,8 @@ template <bool LN>
 __global__ void __launch_bounds__(LA_THREADS, 1)
 k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttnParams p) {
   using namespace tc;
-  const int n_items = p.chunk_start[p.B];
-  if ((int)blockIdx.x >= n_items) return;
+  const int n_items = p.chunk_start[p.B] * p.RB;          // work items: (user, chunk) x row block; gridDim % RB == 0, so
+  if ((int)blockIdx.x >= n_items) return;                  // a CTA keeps one row block for its whole life
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {
     if (threadIdx.x == 0) atomicCAS(p.err, 0, 91);
@@ -171,7 +173,9 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   constexpr uint32_t COL_S = 0, COL_O = 256;      // scores: 2 x 128 columns; accumulator: d columns
 
   // item -> (user, token range); identical in every role
-  auto item_range = [&](int item, int& b, int& tok0, int& tok1) {
+  const int rb = (int)blockIdx.x % p.RB;
+  auto item_range = [&](int wi, int& b, int& tok0, int& tok1) {
+    const int item = wi / p.RB;
     b = upper_user(p.chunk_start, p.B, item);
     tok0 = p.off[b] + (item - p.chunk_start[b]) * p.chunk;
     tok1 = min(p.off[b + 1], tok0 + p.chunk);
@@ -192,7 +196,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           if (qn > 0 && !mbar_wait(q_empty, (uint32_t)(qn - 1) & 1u, p.err, 42)) { ok = false; break; }
           mbar_arrive_expect_tx(q_full, 2 * LA_SUB);
           for (int kb = 0; kb < 2; ++kb)
-            tma_load_2d_hint(smem + LA_OFF_Q2 + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * LA_HL, q_full, pol_keep);
+            tma_load_2d_hint(smem + LA_OFF_Q2 + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128, q_full, pol_keep);
           ++qn;
         }
         const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
@@ -243,7 +247,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
         // will the producer replace the queries after this item?
         bool next_reloads = false;
-        if (!p.shared && item + (int)gridDim.x < n_items) next_reloads = upper_user(p.chunk_start, p.B, item + gridDim.x) != b;
+        if (!p.shared && item + (int)gridDim.x < n_items)
+          next_reloads = upper_user(p.chunk_start, p.B, (item + (int)gridDim.x) / p.RB) != b;
         const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
         if (!issue_scores(g)) { ok = false; break; }
         if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
@@ -288,7 +293,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       int b, tok0, tok1;
       item_range(item, b, tok0, tok1);
       const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
-      const float cq = LN ? p.cQ[(int64_t)(p.shared ? 0 : b) * LA_HL + r] : 0.f;
+      const float cq = LN ? p.cQ[(int64_t)(p.shared ? 0 : b) * p.HL + rb * 128 + r] : 0.f;
       float m_ref = -INFINITY, l_sum = 0.f, mean_corr = 0.f;
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         const int s = g % LA_XSTAGES, pb = g & 1;
@@ -394,10 +399,12 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
       const bool single = p.chunk_start[b + 1] - p.chunk_start[b] == 1;
+      const int R = rb * 128 + (int)r;                          // row among all H * ell
+      const int64_t prow = (int64_t)(item / p.RB) * p.HL + R;   // row of the per-chunk partials
       if (single) {
         // the whole history of this user was one chunk: normalise and write the attention rows directly
         const float inv = 1.0f / l_tot;
-        const int h = (int)r / p.ell, l = (int)r % p.ell;
+        const int h = R / p.ell, l = R % p.ell;
         uint4* dst = reinterpret_cast<uint4*>(p.Ohat + ((int64_t)b * p.ell + l) * (p.H * LA_D) + h * LA_D + col0);
 #pragma unroll
         for (int c8 = 0; c8 < LA_COLS / 8; ++c8) {
@@ -409,13 +416,13 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           dst[c8] = o;
         }
       } else {
-        float4* dst = reinterpret_cast<float4*>(p.part_acc + ((int64_t)item * LA_HL + r) * LA_D + col0);
+        float4* dst = reinterpret_cast<float4*>(p.part_acc + prow * LA_D + col0);
 #pragma unroll
         for (int j = 0; j < LA_COLS; j += 4)
           dst[j / 4] = make_float4(a[j] - c_tot, a[j + 1] - c_tot, a[j + 2] - c_tot, a[j + 3] - c_tot);
         if (part == 0) {
-          p.part_m[(int64_t)item * LA_HL + r] = m_ref;        // log2 domain
-          p.part_s[(int64_t)item * LA_HL + r] = l_tot;
+          p.part_m[prow] = m_ref;        // log2 domain
+          p.part_s[prow] = l_tot;
         }
       }
     }
@@ -430,7 +437,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 }
 
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi) {
-  return dtype == LIME_BF16 && d == LA_D && H * ell == LA_HL && phi == LIME_PHI_SOFTMAX;
+  return dtype == LIME_BF16 && d == LA_D && (H * ell) % 128 == 0 && H * ell <= 512 && phi == LIME_PHI_SOFTMAX;
 }
 
 lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
@@ -438,13 +445,14 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
   CUtensorMap tmX, tmQ2;
   const uint64_t users = a.shared ? 1 : (uint64_t)a.B;
   if (!make_tmap_bf16_sw128(&tmX, a.hist, (uint64_t)a.total, LA_D, LA_D, LA_TILE) ||
-      !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * LA_HL, LA_D, LA_D, 128))
+      !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), LA_D, LA_D, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   LinkAttnParams p;
   p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
-  p.ell = a.ell; p.H = a.H; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
+  p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
-  const int grid = a.n_chunk_upper < kSMs ? a.n_chunk_upper : kSMs;
+  int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;
+  grid -= grid % p.RB;                              // a CTA's work items then all share its row block
   static bool smem_ln[kMaxDeviceOrdinals] = {}, smem_plain[kMaxDeviceOrdinals] = {};
   lime_status es = a.ln ? ensure_dynamic_smem((const void*)k_link_attn_tc<true>, (int)LA_SMEM, smem_ln)
                         : ensure_dynamic_smem((const void*)k_link_attn_tc<false>, (int)LA_SMEM, smem_plain);

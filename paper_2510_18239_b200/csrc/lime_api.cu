@@ -99,7 +99,8 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
 static bool layer_on_tensor_cores(const Ctx* c, int layer) {
   const lime_config& g = c->cfg;
   return c->WoT[layer] && c->WprepT[layer] && c->WpostT[layer] && link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi) &&
-         hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
+         (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) ||
+          hist_update2_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp));
 }
 
 // One XOR layer, tensor-core path: three link-row GEMMs around the two streaming attention kernels.
@@ -149,7 +150,9 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
     hu.cK = ops.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
     hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = ops.shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
     hu.out_ln = out_ln; hu.err = c->dev_err;
-    if ((s = launch_hist_update_tc(hu, st)) != LIME_OK) return s;
+    if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) s = launch_hist_update_tc(hu, st);
+    else s = launch_hist_update2_tc(hu, g.H, st);
+    if (s != LIME_OK) return s;
   }
   return LIME_OK;
 }
@@ -422,7 +425,8 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
     return s;
   // tensor-core path: per layer, W_o as a K-major B operand ([d x d_ff], contraction index contiguous) and the
   // weight-only products that fold the history-side projections into the link rows
-  if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) &&
+  if ((hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) ||
+       hist_update2_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) &&
       link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi)) {
     for (int j = 0; j < g.n_layers; ++j) {
       if (!c->WoT[j]) LIME_CUDA(cudaMalloc(&c->WoT[j], (size_t)g.d * c->d_ff * 2));

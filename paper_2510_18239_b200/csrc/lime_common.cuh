@@ -221,5 +221,8 @@ struct HistUpdateArgs {
 };
 bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
 lime_status launch_hist_update_tc(const HistUpdateArgs& a, cudaStream_t st);
+// same step for H * ell in {256, 384, 512} (link-side operands streamed per tile, k_hist_update2_tc.cu)
+bool hist_update2_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
+lime_status launch_hist_update2_tc(const HistUpdateArgs& a, int H, cudaStream_t st);
 
 }  // namespace lime

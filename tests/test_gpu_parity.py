@@ -219,12 +219,13 @@ def test_xor_layer_history_lengths(N, dtype):
         assert torch.count_nonzero(links_out).item() == 0
 
 
-@pytest.mark.parametrize("ell,H", [(32, 4), (16, 8), (64, 2)])
+@pytest.mark.parametrize("ell,H", [(32, 4), (16, 8), (64, 2), (64, 4), (32, 8), (64, 8)])
 @pytest.mark.parametrize("lengths", [[1], [127, 128, 129], [0, 300, 5, 0, 1000], [256] * 40])
 @pytest.mark.parametrize("shared_links", [True, False])
 def test_xor_layer_tensor_core_path(ell, H, lengths, shared_links):
-    """One XOR layer at the shapes the fused tensor-core kernels serve (bf16, d = 128, H * ell = 128), ragged
-    histories around the 128-token tile, shared and per-user link rows."""
+    """One XOR layer at the shapes the fused tensor-core kernels serve (bf16, d = 128, H * ell = 128 with all operands
+    resident, 256 and 512 with the link-side operands streamed; (64, 2) falls to the generic path), ragged histories
+    around the 128-token tile, shared and per-user link rows."""
     Bd = _lib()
     B = len(lengths)
     wl = small(synth.BF16, B=B, n_min=0, n_max=1, d=128, H=H, ell=ell, n_layers=1, V=3000, table_std=0.05)
