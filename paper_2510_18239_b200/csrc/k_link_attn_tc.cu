@@ -30,7 +30,7 @@
 
 namespace lime {
 
-constexpr int LA_D = 128, LA_HL = 128, LA_TILE = 128, LA_XSTAGES = 3;
+constexpr int LA_D = 128, LA_TILE = 128, LA_XSTAGES = 4;
 constexpr int LA_PARTS = 4;                                   // threads per row
 constexpr int LA_COLS = LA_TILE / LA_PARTS;                   // token columns per thread
 constexpr int LA_SOFTMAX_WARPS = 4 * LA_PARTS, LA_THREADS = 64 + 32 * LA_SOFTMAX_WARPS;
@@ -38,8 +38,8 @@ constexpr uint32_t LA_SUB = 128 * 128;
 constexpr uint32_t LA_X_STAGE = 2 * LA_SUB;
 constexpr uint32_t LA_OFF_X = 0;
 constexpr uint32_t LA_OFF_Q2 = LA_XSTAGES * LA_X_STAGE;
-constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_SUB;        // 2 buffers of [HL x 128 tokens]
-constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 4 * LA_SUB;     // per X stage: float2 {rstd, mu} x 128 tokens
+constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_SUB;        // P' [128 rows x 128 tokens]; a fourth token stage buys more than a second P'
+constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 2 * LA_SUB;     // per X stage: float2 {rstd, mu} x 128 tokens
 constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 8;   // [2 tile parities][PARTS][128] maxima, then
                                                                         // [PARTS][128] sums and [PARTS][128] mean terms
 constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 4 * LA_PARTS * 128 * 4;
@@ -141,13 +141,13 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     return;
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LA_OFF_BAR);
-  uint64_t* x_full = bars;             // [3]
-  uint64_t* x_empty = bars + 3;        // [3]  second MMA of the tile done
-  uint64_t* q_full = bars + 6;         //      folded queries of the item's user landed
-  uint64_t* q_empty = bars + 7;        //      every score MMA of the item has read them
+  uint64_t* x_full = bars;             // [4]
+  uint64_t* x_empty = bars + 4;        // [4]  second MMA of the tile done
+  uint64_t* q_full = bars + 22;         //      folded queries of the item's user landed
+  uint64_t* q_empty = bars + 23;       //      every score MMA of the item has read them
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       // [2]  P' in smem (all softmax warps)
-  uint64_t* p_free = bars + 12;        // [2]  second MMA done reading P' (and accumulator up to date)
+  uint64_t* p_ready = bars + 10;       //      per tile: P' in smem (all softmax warps)
+  uint64_t* p_free = bars + 12;        //      per tile: second MMA done reading P' (and accumulator up to date)
   uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
   uint64_t* stats_bar = bars + 15;     //      rendezvous of the softmax warps (token statistics written)
   uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the warps that share a TMEM lane quarter
@@ -158,7 +158,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   if (threadIdx.x == 0) {
     for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], LA_SOFTMAX_WARPS); mbar_init(&p_free[i], 1); }
+    for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
+    mbar_init(p_ready, LA_SOFTMAX_WARPS); mbar_init(p_free, 1);
     mbar_init(o_free, LA_SOFTMAX_WARPS);
     mbar_init(stats_bar, LA_SOFTMAX_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LA_PARTS);
@@ -253,24 +254,24 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         if (!issue_scores(g)) { ok = false; break; }
         if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
         for (int t = 0; t < n_tiles; ++t, ++g) {
-          // the next tile's scores overlap this tile's softmax (its score buffer was released by p_ready(g-1))
+          // the next tile's scores overlap this tile's softmax (its score buffer was read before p_ready(g-1))
           if (t + 1 < n_tiles) {
             if (!issue_scores(g + 1)) { ok = false; break; }
             if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
           }
-          const int s = g % LA_XSTAGES, pb = g & 1;
-          if (!mbar_wait(&p_ready[pb], (uint32_t)(g >> 1) & 1u, p.err, 52)) { ok = false; break; }
+          const int s = g % LA_XSTAGES;
+          if (!mbar_wait(p_ready, (uint32_t)g & 1u, p.err, 52)) { ok = false; break; }
           // the first tile of an item overwrites the accumulator: the previous item must have been read out
           if (t == 0 && k > 0 && !mbar_wait(o_free, (uint32_t)(k - 1) & 1u, p.err, 53)) { ok = false; break; }
           tc_fence_after();
           for (int kk = 0; kk < 8; ++kk) {      // contraction over the tile's 128 tokens, 16 per instruction
             const uint32_t oa = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
-            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + pb * 2 * LA_SUB + oa),
+            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + oa),
                         make_sdesc_mn_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + (uint32_t)kk * 2048, LA_SUB), idesc_o,
                         (t | kk) != 0);
           }
           mma_commit(&x_empty[s]);
-          mma_commit(&p_free[pb]);
+          mma_commit(p_free);
         }
       }
     }
@@ -355,7 +356,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         const float factor = (need && m_ref != -INFINITY) ? la_ex2(m_ref - m_new) : 1.0f;
         if (__any_sync(0xffffffffu, need && t > 0)) {
           // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this part of the row
-          if (!mbar_wait(&p_free[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, p.err, 64)) { ok = false; break; }
+          if (!mbar_wait(p_free, (uint32_t)(g - 1) & 1u, p.err, 64)) { ok = false; break; }
           tc_fence_after();
           float a[LA_COLS];
           tmem_ld_32x32(lane_addr + COL_O + col0, a);
@@ -369,22 +370,22 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         mean_corr *= factor;
         m_ref = m_new;
 
-        // the P' buffer of two tiles ago must have been consumed
-        if (g >= 2 && !mbar_wait(&p_free[pb], (uint32_t)((g - 2) >> 1) & 1u, p.err, 65)) { ok = false; break; }
+        // the previous tile's P' must have been consumed
+        if (g >= 1 && !mbar_wait(p_free, (uint32_t)(g - 1) & 1u, p.err, 65)) { ok = false; break; }
         // pass 2: P' -> smem; K index = token column, so columns col0.. live in K-block col0 / 64, chunk (col0 % 64) / 8..
-        uint8_t* pbuf = smem + LA_OFF_P + pb * 2 * LA_SUB + (col0 >> 6) * LA_SUB;
+        uint8_t* pbuf = smem + LA_OFF_P + (col0 >> 6) * LA_SUB;
         const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
         if (nvalid == LA_TILE) la_pass2<LN, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
         else la_pass2<LN, true>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_ready[pb]);
+        if (lane == 0) mbar_arrive(p_ready);
       }
       if (!ok) break;
       // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
       const int gl = g - 1;
-      if (!mbar_wait(&p_free[gl & 1], (uint32_t)(gl >> 1) & 1u, p.err, 66)) { ok = false; break; }
+      if (!mbar_wait(p_free, (uint32_t)gl & 1u, p.err, 66)) { ok = false; break; }
       tc_fence_after();
       exch_sum[part * 128 + r] = l_sum;
       exch_mean[part * 128 + r] = mean_corr;

@@ -38,11 +38,12 @@ static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t
 static inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 static inline int elem_size(int dtype) { return dtype == LIME_F32 ? 4 : 2; }
 
-// Tokens per work item of the link<-history attention: a power of two in [64, 1024] giving a few items per SM.
+// Tokens per work item of the link<-history attention: a power of two in [64, 2048] giving a few items per SM
+// (every chunk of a multi-chunk history costs a set of fp32 partials, so long histories take long chunks).
 static int pick_chunk(int64_t total_tokens) {
   int64_t target = total_tokens / (4 * kSMs);
   int c = 64;
-  while (c < 1024 && c < target) c <<= 1;
+  while (c < 2048 && c < target) c <<= 1;
   return c;
 }
 constexpr int kHistTile = 128;  // tokens per block of the history<-links attention
