@@ -38,11 +38,12 @@ static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t
 static inline size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 static inline int elem_size(int dtype) { return dtype == LIME_F32 ? 4 : 2; }
 
-// Tokens per work item of the link<-history attention: a power of two in [64, 2048] giving a few items per SM
-// (every chunk of a multi-chunk history costs a set of fp32 partials, so long histories take long chunks).
-static int pick_chunk(int64_t total_tokens) {
-  int64_t target = total_tokens / (4 * kSMs);
-  int c = 64;
+// Tokens per work item of the link<-history attention: a power of two in [lo, 2048] giving about three work items per
+// SM (`row_blocks` items per chunk).  Every chunk of a multi-chunk history costs a set of fp32 partials and a pipeline
+// refill, so long histories take long chunks.
+static int pick_chunk(int64_t total_tokens, int row_blocks, int lo) {
+  const int64_t target = total_tokens * row_blocks / (3 * kSMs);
+  int c = lo;
   while (c < 2048 && c < target) c <<= 1;
   return c;
 }
@@ -77,9 +78,9 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.AT = (float*)take(ld); w.UT = (float*)take(lf); w.LP = (float*)take(ld); w.LS32 = (float*)take(ld);
   w.chunk_start = (int32_t*)take((size_t)(B + 1) * 4);
   w.tile_start = (int32_t*)take((size_t)(B + 1) * 4);
-  w.chunk = pick_chunk(total);
   const bool tc_link = link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi);
-  if (tc_link && w.chunk < 512) w.chunk = 512;   // one CTA per chunk: amortise its set-up over >= 4 token tiles
+  // tensor-core path: at least 4 token tiles per work item, one item per 128-row block of H * ell
+  w.chunk = tc_link ? pick_chunk(total, (g.H * g.ell + 127) / 128, 512) : pick_chunk(total, 1, 64);
   w.n_chunk_upper = (int)((total + w.chunk - 1) / w.chunk + B);
   w.n_tile_upper = (int)((total + kHistTile - 1) / kHistTile + B);
   const size_t rows = (size_t)w.n_chunk_upper * g.H * g.ell;
