@@ -241,7 +241,7 @@ NCU_TRAFFIC = {
     # profiles/k_score_tc_bf16_baseline.md: 169.9 MB read + 4.0-4.5 MB written per launch
     ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
     # profiles/xor_layer_kernels_bf16_baseline.md: 33.7 MB (layer 1) and 42.0 MB (layer 2) read; average per launch
-    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.8e6, "source": "k_link_attn_tc.cu", "sha": "5816f4a99dd58671"},
+    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.8e6, "source": "k_link_attn_tc.cu", "sha": "e56b781284e88a10"},
     ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.4e6, "source": "k_hist_update_tc.cu", "sha": "24cb0f708e8e5b84"},
 }
 
