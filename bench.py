@@ -418,9 +418,6 @@ def run_ours(args, wl):
     d_cid = [torch.empty(wl.B * wl.C, dtype=torch.int32, device=dev) for _ in range(SLOTS)]
     d_logits = [torch.empty(wl.B * wl.C, dtype=torch.float32, device=dev) for _ in range(SLOTS)]
     h_logits = [torch.empty(wl.B * wl.C, dtype=torch.float32).pin_memory() for _ in range(SLOTS)]
-    Tbuf = torch.empty((wl.B * wl.C, wl.d), dtype=lime.tdtype, device=dev)
-    Wbuf = torch.empty((wl.B * wl.C, wl.ell), dtype=lime.tdtype, device=dev)
-    lime_w = Bd.Lime(wl.ell, 1, 1, 1, dtype=dt, gated_mlp=False)       # row gather of the [V x ell] weight cache
     assert ROTATE % SLOTS == 0
 
     def e2e_copy_in(i):
@@ -437,9 +434,8 @@ def run_ours(args, wl):
         Bd.lime_lengths_to_offsets(ctx, d_len[k], off)
         Bd.lime_gather_history(ctx, table, d_hid[k][:n], h)
         Bd.lime_encode_user(ctx, h, off, wl.B, None, ls, ws)
-        Bd.lime_gather_history(ctx, table, d_cid[k], Tbuf)
-        Bd.lime_gather_history(lime_w.ctx, w_corpus, d_cid[k], Wbuf)
-        Bd.lime_score_candidates(ctx, ls, wl.B, Wbuf, Tbuf, None, wl.C, wl.B * wl.C, None, d_logits[k])
+        # candidates are scored straight from the corpus caches by id (no gather of their rows)
+        Bd.lime_score_candidates(ctx, ls, wl.B, w_corpus, table, None, wl.C, wl.B * wl.C, d_cid[k], d_logits[k])
 
     def e2e_copy_out(i):
         k = i % SLOTS
@@ -486,6 +482,15 @@ def run_ours(args, wl):
         for i in range(ROTATE):
             e2e_step(i)
         barrier()
+    # the by-id scorer alone, back to back (random rows of the 256 MB+ table: no reuse between launches)
+    torch.cuda.synchronize()
+    eg0, eg1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    eg0.record()
+    for i in range(50):
+        Bd.lime_score_candidates(ctx, ls, wl.B, w_corpus, table, None, wl.C, wl.B * wl.C, d_cid[i % SLOTS], d_logits[i % SLOTS])
+    eg1.record()
+    torch.cuda.synchronize()
+    score_by_id_ms = eg0.elapsed_time(eg1) / 50
     h2d = d2h = 0
     e0.record(s_in)
     t_issue = time.perf_counter()
@@ -555,8 +560,9 @@ def run_ours(args, wl):
                 "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args)), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps, "host_issue_ms_per_step": 1e3 * t_issue / args.steps,
-                        "how": "pinned host ids -> H2D | offsets, gathers (history and candidate rows from the resident caches), "
-                               "encode, score | logits D2H; three streams, two request slots"},
+                        "score_by_id_alone_ms": score_by_id_ms,
+                        "how": "pinned host ids -> H2D | offsets, history gather, encode, scoring by candidate id from the resident "
+                               "corpus caches | logits D2H; three streams, two request slots"},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roofline, "scoring_roofline": scoring,
                 "kernels": kernels[:14],
                 "precompute": {"ms": pre_ms, "candidates": wl.B * wl.C, "candidates_per_s": wl.B * wl.C / (pre_ms * 1e-3),

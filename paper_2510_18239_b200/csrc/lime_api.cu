@@ -570,6 +570,7 @@ lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_
   a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->cfg.ell; a.d = c->cfg.d;
   a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
   if (score_tc_supported(a)) return launch_score_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
+  if (score_gather_tc_supported(a)) return launch_score_gather_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   return launch_score_simt(a, static_cast<cudaStream_t>(stream));
 }
 

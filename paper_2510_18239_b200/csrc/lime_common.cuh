@@ -168,6 +168,9 @@ lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);
 // bf16 streaming scorer on tcgen05 tensor cores (fixed C per user, dense rows, ell in {16,32,64,128}, d % 64 == 0)
 bool score_tc_supported(const ScoreArgs& a);
 lime_status launch_score_tc(const ScoreArgs& a, int* err, cudaStream_t st);
+// the same with rows taken from corpus-level caches by cand_ids (fixed C per user), k_score_gather_tc.cu
+bool score_gather_tc_supported(const ScoreArgs& a);
+lime_status launch_score_gather_tc(const ScoreArgs& a, int* err, cudaStream_t st);
 
 // ---- tensor-core XOR layer (bf16, d = d_ff = 128, H * ell = 128) ----------------------------------------------
 lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,

@@ -160,6 +160,27 @@ def test_score_ragged_offsets_ids_and_empty_users():
     assert np.abs(Hh.to_f64(logits) - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
 
 
+@pytest.mark.parametrize("B,C,ell,d,corpus", [(3, 2048, 32, 128, 5000), (2, 129, 64, 256, 300), (160, 130, 16, 64, 1000),
+                                              (1, 1, 32, 128, 7), (150, 1000, 32, 128, 100000), (5, 300, 128, 64, 999)])
+def test_score_from_corpus_caches_by_ids(B, C, ell, d, corpus):
+    """Fixed C per user with candidate ids into corpus-level caches (item embeddings and cached weights): the bf16
+    scorer that gathers rows itself, against the oracle on the gathered rows; many tiles per CTA in the larger cases."""
+    Bd = _lib()
+    dtype = synth.BF16
+    lime = Bd.Lime(d, max(1, d // 128), ell, 1, dtype=Bd.LIME_BF16, gated_mlp=False)
+    LS = synth.normal_storage(8, "ls", (B, ell, d), 1.0, dtype)
+    Tc = synth.normal_storage(8, "t", (corpus, d), 1.0, dtype)
+    Wc = synth.to_storage(O.softmax_rows(np.random.default_rng(8).normal(size=(corpus, ell))), dtype)
+    ids = synth.uniform_ids(8, "ids", B * C, corpus)
+    logits = lime.score_candidates(Bd.to_device(LS, dtype), Bd.to_device(Wc, dtype), Bd.to_device(Tc, dtype), C=C,
+                                   cand_ids=torch.from_numpy(ids).cuda(), total_cands=B * C)
+    assert Bd.lime_device_status(lime.ctx) == 0
+    W64, T64, LS64 = (synth.storage_to_f64(x, dtype) for x in (Wc, Tc, LS))
+    want = np.concatenate([O.score_candidates(W64[ids[b * C:(b + 1) * C]], LS64[b], T64[ids[b * C:(b + 1) * C]]) for b in range(B)])
+    err = np.abs(Hh.to_f64(logits) - want).max()
+    assert err <= 1e-4 * max(1.0, np.abs(want).max()), err
+
+
 # ----------------------------------------------------------------------------- XOR layer and encode
 def _oracle_batch(wl, inp, phi=O.SOFTMAX, ln=True, gated_mlp=True, cand_np=None):
     cfg = Hh.oracle_config(wl, phi=phi, ln=ln, gated_mlp=gated_mlp)
