@@ -86,13 +86,38 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
     for (int s = 0; s < SG_MAX_STAGES; ++s) stage_user[s] = -1;
     const uint64_t pol_keep = policy_evict_last(), pol_stream = policy_evict_first();
     const int n_jobs = 32 * (KB + 1);              // per tile: 32 row quads x (KB embedding blocks + the weight rows)
+    // Thread (warp w, lane g) issues the copies of row quad g (rows 4g..4g+3 of the tile) for K blocks w, w+4, ... and,
+    // as job KB, the weight rows.  Its four ids are read two tiles ahead of their use, so the round trip of that read
+    // is off the path that refills a freed stage.
+    auto read_ids = [&](int t, int (&id)[4]) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) id[i] = 0;
+      if (t >= t_end) return;
+      const int b = t / p.tiles_per_user;
+      const int c = (t % p.tiles_per_user) * SG_TILE + 4 * lane;
+      const int32_t* src = p.ids + (int64_t)b * p.C + c;
+      // rows past the user's last candidate fetch row 0 (a stage's byte count stays fixed; their logits are never written)
+      if (c + 3 < p.C && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+        const int4 v = __ldg(reinterpret_cast<const int4*>(src));
+        id[0] = v.x; id[1] = v.y; id[2] = v.z; id[3] = v.w;
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (c + i < p.C) id[i] = __ldg(src + i);
+      }
+    };
+    int id_now[4], id_next[4], id_after[4];
+    read_ids(t_begin, id_next);
+    read_ids(t_begin + 1, id_after);
     int it = 0;
     bool ok = true;
     for (int t = t_begin; t < t_end; ++t, ++it) {
       const int s = it % S;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { id_now[i] = id_next[i]; id_next[i] = id_after[i]; }
+      read_ids(t + 2, id_after);
       if (!mbar_wait(&empty[s], ((uint32_t)(it / S) & 1u) ^ 1u, p.err, 101)) { ok = false; break; }
       const int b = t / p.tiles_per_user;
-      const int c0 = (t % p.tiles_per_user) * SG_TILE;
       uint8_t* st = smem + (size_t)s * stage_bytes;
       // every thread announces its own bytes before it issues its copies, so the phase cannot complete early
       bool load_ls = false;
@@ -108,20 +133,13 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
         for (int kb = 0; kb < KB; ++kb)
           tma_load_2d_hint(st + t_bytes + (size_t)kb * ELL * 128, &tmLS, kb * 64, b * ELL, &full[s], pol_keep);
       for (int j = (int)r; j < n_jobs; j += 128) {
-        const int g = j & 31, what = j >> 5;       // rows 4g..4g+3 of the tile; what < KB: embedding K block, else weights
-        int id[4];
-        // rows past the user's last candidate fetch row 0 (a stage's byte count stays fixed; their logits are never written)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int c = c0 + 4 * g + i;
-          id[i] = c < p.C ? __ldg(p.ids + (int64_t)b * p.C + c) : 0;
-        }
+        const int what = j >> 5;                   // what < KB: K block of the embedding rows, else the weight rows
         if (what < KB)
-          tma_gather4_2d_hint(st + (size_t)what * SG_TILE * 128 + (size_t)g * 512, &tmT, what * 64, id[0], id[1], id[2],
-                              id[3], &full[s], pol_stream);
+          tma_gather4_2d_hint(st + (size_t)what * SG_TILE * 128 + (size_t)lane * 512, &tmT, what * 64, id_now[0],
+                              id_now[1], id_now[2], id_now[3], &full[s], pol_stream);
         else
-          tma_gather4_2d_hint(st + t_bytes + ls_bytes + (size_t)g * (4 * ELL * 2), &tmW, 0, id[0], id[1], id[2], id[3],
-                              &full[s], pol_stream);
+          tma_gather4_2d_hint(st + t_bytes + ls_bytes + (size_t)lane * (4 * ELL * 2), &tmW, 0, id_now[0], id_now[1],
+                              id_now[2], id_now[3], &full[s], pol_stream);
       }
     }
     if (r == 0 && (!ok || *(volatile int*)p.err != 0)) {
