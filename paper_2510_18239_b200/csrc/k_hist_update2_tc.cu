@@ -31,7 +31,9 @@ constexpr uint32_t H2_OFF_STATS = H2_OFF_PU + 2 * H2_SUB;    // 2 (tile parity) 
 constexpr uint32_t H2_OFF_EXCH = H2_OFF_STATS + 2 * 128 * 8; // pair exchange: [2 slots][2 halves][128]
 constexpr uint32_t H2_OFF_CK = H2_OFF_EXCH + 4 * 128 * 4;    // the current user's HL key row sums (up to 512 floats)
 constexpr uint32_t H2_OFF_BAR = H2_OFF_CK + 512 * 4;
-constexpr uint32_t H2_SMEM = H2_OFF_BAR + 256;
+constexpr int H2_IDX_CAP = 1025;                            // users + 1 whose offsets are staged in shared memory (the
+constexpr uint32_t H2_OFF_IDX = H2_OFF_BAR + 256;           // search for a tile's user is a chain of dependent reads:
+constexpr uint32_t H2_SMEM = H2_OFF_IDX + 2 * H2_IDX_CAP * 4 + 8;   // microseconds from global memory)
 static_assert(H2_SMEM <= 232448, "shared memory budget of one CTA");
 
 struct HistUpdate2Params {
@@ -70,7 +72,10 @@ struct H2TileUser {
   int b = -1, lo = 0, hi = 0;
   __device__ __forceinline__ int of(const int32_t* __restrict__ tile_start, int B, int t) {
     if (t < lo || t >= hi) {
-      b = upper_user(tile_start, B, t);
+      // the user is a neighbour of the cached one: step through tile_start (staged in shared memory), no search
+      if (b < 0) b = upper_user(tile_start, B, t);
+      else if (t >= hi) { do { ++b; } while (tile_start[b + 1] <= t); }
+      else { do { --b; } while (tile_start[b] > t); }
       lo = tile_start[b];
       hi = tile_start[b + 1];
     }
@@ -126,6 +131,14 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  const int32_t* tile_start = p.tile_start;
+  const int32_t* off = p.off;
+  if (p.B + 1 <= H2_IDX_CAP) {
+    int32_t* idx = reinterpret_cast<int32_t*>(smem + H2_OFF_IDX);
+    for (int i = threadIdx.x; i <= p.B; i += H2_THREADS) { idx[i] = p.tile_start[i]; idx[H2_IDX_CAP + i] = p.off[i]; }
+    tile_start = idx;
+    off = idx + H2_IDX_CAP;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -143,10 +156,10 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       H2TileUser tu;
       for (; g < n && ok; ++g) {
         const int t = t_begin + g;
-        const int b = tu.of(p.tile_start, p.B, t);
+        const int b = tu.of(tile_start, p.B, t);
         const int urow = p.shared ? 0 : b;
         if (g > 0 && !mbar_wait(x_empty, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
-        const int row0 = p.off[b] + (t - tu.lo) * H2_TILE;
+        const int row0 = off[b] + (t - tu.lo) * H2_TILE;
         mbar_arrive_expect_tx(x_full, 2 * H2_SUB);
         for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + H2_OFF_X + kb * H2_SUB, &tmX, kb * 64, row0, x_full, pol_stream);
         for (int c = 0; c < NG; ++c, ++q) {
@@ -236,9 +249,9 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     H2TileUser tu;
     for (int g = 0; g < n && ok; ++g) {
       const int t = t_begin + g;
-      const int b = tu.of(p.tile_start, p.B, t);
-      const int row0 = p.off[b] + (t - tu.lo) * H2_TILE;
-      const bool valid = row0 + (int)r < p.off[b + 1];
+      const int b = tu.of(tile_start, p.B, t);
+      const int row0 = off[b] + (t - tu.lo) * H2_TILE;
+      const bool valid = row0 + (int)r < off[b + 1];
       // ---- LayerNorm statistics of the tile (two lanes per token, 64 features each), then this row's constants
       float rstd_r = 1.f, mu_r = 0.f;
       if (LN) {

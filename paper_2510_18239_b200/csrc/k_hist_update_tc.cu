@@ -44,7 +44,9 @@ constexpr uint32_t HU_OFF_STATS = HU_OFF_PU + 2 * HU_SUB;   // 2 (tile parity) x
 constexpr uint32_t HU_OFF_EXCH = HU_OFF_STATS + 2 * 128 * 8;   // row exchange: [PARTS][128] sums, then the same of squares
 constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 2 * HU_PARTS * 128 * 4;   // the current user's HL key row sums (fp32)
 constexpr uint32_t HU_OFF_BAR = HU_OFF_CK + HU_HL * 4;
-constexpr uint32_t HU_SMEM = HU_OFF_BAR + 256;
+constexpr int HU_IDX_CAP = 1025;                            // users + 1 whose offsets are staged in shared memory (the
+constexpr uint32_t HU_OFF_IDX = HU_OFF_BAR + 256;           // search for a tile's user is a chain of dependent reads:
+constexpr uint32_t HU_SMEM = HU_OFF_IDX + 2 * HU_IDX_CAP * 4 + 8;   // microseconds from global memory)
 static_assert(HU_SMEM <= 232448, "shared memory budget of one CTA");
 
 struct HistUpdateParams {
@@ -60,12 +62,15 @@ struct HistUpdateParams {
 // address of 16-byte chunk `c` (0..7) of row r inside a 128B-swizzled [rows x 64 bf16] sub-tile
 __device__ __forceinline__ uint32_t sw128_chunk(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
 
-// user of tile t, cached: the tile ranges of consecutive tiles are the same user most of the time
+// user of tile t, cached: consecutive tiles are the same user most of the time, and when they are not the user is a
+// neighbour of the cached one, found by stepping through tile_start (staged in shared memory) instead of a search
 struct TileUser {
   int b = -1, lo = 0, hi = 0;
   __device__ __forceinline__ int of(const int32_t* __restrict__ tile_start, int B, int t) {
     if (t < lo || t >= hi) {
-      b = upper_user(tile_start, B, t);
+      if (b < 0) b = upper_user(tile_start, B, t);
+      else if (t >= hi) { do { ++b; } while (tile_start[b + 1] <= t); }
+      else { do { --b; } while (tile_start[b] > t); }
       lo = tile_start[b];
       hi = tile_start[b + 1];
     }
@@ -143,6 +148,14 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  const int32_t* tile_start = p.tile_start;
+  const int32_t* off = p.off;
+  if (p.B + 1 <= HU_IDX_CAP) {
+    int32_t* idx = reinterpret_cast<int32_t*>(smem + HU_OFF_IDX);
+    for (int i = threadIdx.x; i <= p.B; i += HU_THREADS) { idx[i] = p.tile_start[i]; idx[HU_IDX_CAP + i] = p.off[i]; }
+    tile_start = idx;
+    off = idx + HU_IDX_CAP;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -160,7 +173,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       TileUser tu;
       for (; g < n && ok; ++g) {
         const int t = t_begin + g;
-        const int b = tu.of(p.tile_start, p.B, t);
+        const int b = tu.of(tile_start, p.B, t);
         if (b != cur_user && (seg == 0 || !p.shared)) {
           const int urow = p.shared ? 0 : b;
           if (seg > 0 && !mbar_wait(k2_empty, (uint32_t)(seg - 1) & 1u, p.err, 11)) { ok = false; break; }
@@ -177,7 +190,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
         cur_user = b;
         if (g > 0 && !mbar_wait(x_empty, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
-        const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
+        const int row0 = off[b] + (t - tu.lo) * HU_TILE;
         mbar_arrive_expect_tx(x_full, 2 * HU_SUB);
         for (int kb = 0; kb < 2; ++kb) tma_load_2d_hint(smem + HU_OFF_X + kb * HU_SUB, &tmX, kb * 64, row0, x_full, pol_stream);
       }
@@ -201,12 +214,12 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       auto last_of_user = [&](int g) {
         if (p.shared) return false;
         const int t = t_begin + g;
-        tu.of(p.tile_start, p.B, t);
+        tu.of(tile_start, p.B, t);
         return g + 1 < n && t + 1 >= tu.hi;
       };
       // 1. scores(g) = X . K2^T
       auto issue_scores = [&](int g) -> bool {
-        const int b = tu.of(p.tile_start, p.B, t_begin + g);
+        const int b = tu.of(tile_start, p.B, t_begin + g);
         if (b != user_of_scores && (seg_k == 0 || !p.shared)) {
           if (!mbar_wait(k2_full, (uint32_t)seg_k & 1u, p.err, 22)) return false;
           ++seg_k;
@@ -230,7 +243,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       for (int g = 0; g < n && ok; ++g) {
         const uint32_t tp = (uint32_t)g & 1u;
         // 3. [gate | up](g) = P(g) . [G2 | U2]
-        const int b = tu.of(p.tile_start, p.B, t_begin + g);
+        const int b = tu.of(tile_start, p.B, t_begin + g);
         if (b != user_of_mix && (seg_o == 0 || !p.shared)) {
           if (!mbar_wait(ops_full, (uint32_t)seg_o & 1u, p.err, 27)) break;
           ++seg_o;
@@ -329,7 +342,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
     // 2. per-head softmax over the links of this thread's heads (32 score columns), P -> smem
     auto softmax = [&](int g) -> bool {
-      const int b = tu.of(p.tile_start, p.B, t_begin + g);
+      const int b = tu.of(tile_start, p.B, t_begin + g);
       if (!mbar_wait(s2_full, (uint32_t)g & 1u, p.err, 32)) return false;
       tc_fence_after();
       if (LN && b != ck_user && (ck_user < 0 || !p.shared)) {
@@ -409,8 +422,8 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     // 6. this thread's 32 columns of its S' row -> (LayerNorm) -> bf16 -> global.  The caller has waited for sp_full(g).
     auto store_rows = [&](int g) -> bool {
       const int t = t_begin + g;
-      const int b = tu.of(p.tile_start, p.B, t);
-      const int row0 = p.off[b] + (t - tu.lo) * HU_TILE;
+      const int b = tu.of(tile_start, p.B, t);
+      const int row0 = off[b] + (t - tu.lo) * HU_TILE;
       float v[HU_COLS];
       tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
       tmem_wait_ld();
@@ -461,7 +474,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       xchg(tch[0], tch[2], (lane & 2) != 0, 2);
       xchg(tch[1], tch[3], (lane & 2) != 0, 2);
       const int rbase = row0 + q * 32 + (lane & ~3);          // first of the four rows this lane group holds
-      const int row_end = p.off[b + 1];
+      const int row_end = off[b + 1];
 #pragma unroll
       for (int m = 0; m < 4; ++m)
         if (rbase + m < row_end)

@@ -30,7 +30,7 @@
 
 namespace lime {
 
-constexpr int LA_D = 128, LA_TILE = 128, LA_XSTAGES = 4;
+constexpr int LA_D = 128, LA_TILE = 128, LA_XSTAGES = 3;
 constexpr int LA_PARTS = 4;                                   // threads per row
 constexpr int LA_COLS = LA_TILE / LA_PARTS;                   // token columns per thread
 constexpr int LA_SOFTMAX_WARPS = 4 * LA_PARTS, LA_THREADS = 64 + 32 * LA_SOFTMAX_WARPS;
@@ -38,18 +38,24 @@ constexpr uint32_t LA_SUB = 128 * 128;
 constexpr uint32_t LA_X_STAGE = 2 * LA_SUB;
 constexpr uint32_t LA_OFF_X = 0;
 constexpr uint32_t LA_OFF_Q2 = LA_XSTAGES * LA_X_STAGE;
-constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_SUB;        // P' [128 rows x 128 tokens]; a fourth token stage buys more than a second P'
+constexpr uint32_t LA_Q2_BUF = 2 * LA_SUB;                    // folded queries of one user's row block; two buffers, so the
+                                                             // producer fetches the next user's while this one is in use
+constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_Q2_BUF;     // P' [128 rows x 128 tokens]
 constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 2 * LA_SUB;     // per X stage: float2 {rstd, mu} x 128 tokens
 constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 8;   // [2 tile parities][PARTS][128] maxima, then
                                                                         // [PARTS][128] sums and [PARTS][128] mean terms
 constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 4 * LA_PARTS * 128 * 4;
-constexpr uint32_t LA_SMEM = LA_OFF_BAR + 256;
+constexpr int LA_IDX_CAP = 1025;                             // users + 1 whose offsets are staged in shared memory
+constexpr uint32_t LA_OFF_IDX = LA_OFF_BAR + 256;            // chunk_start[0..B], off[0..B] (a search over them per work item
+                                                             // costs a chain of dependent reads: microseconds from global memory)
+constexpr uint32_t LA_SMEM = LA_OFF_IDX + 2 * LA_IDX_CAP * 4 + 8;
 constexpr float LA_RESCALE_THRESHOLD = 8.0f;                 // in log2 units
 
 struct LinkAttnParams {
   const float* cQ;                // [users x HL]
   const int32_t* off;
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
+  const int32_t* chunk_user;      // [chunk items] user of each (user, chunk) item
   int B, chunk, shared, ell, H;
   int HL, RB;                     // stacked (head, link) rows in all, and 128-row blocks of them (one per work item)
   float ln_eps;
@@ -129,6 +135,25 @@ __device__ __forceinline__ void la_pass2(const float (&v)[LA_COLS], const float2
   mean_corr += mc0 + mc1;
 }
 
+// Walk over this CTA's work items.  The user of an item comes from the chunk_user table, read two items ahead, and the
+// token range from the offset tables staged in shared memory: the code between two items is executed once per item by
+// every role, so it is kept to a few instructions with no dependent chain of global reads.
+struct ItemWalk {
+  int ci, stride, n_ci;     // (user, chunk) index of the current item, its step, and the number of such items
+  int b0, b1, b2;           // users of the current item, the next, and the one after (-1: none)
+  __device__ __forceinline__ void init(const int32_t* __restrict__ chunk_user, int first, int step, int n) {
+    ci = first; stride = step; n_ci = n;
+    b0 = ci < n ? __ldg(chunk_user + ci) : -1;
+    b1 = ci + step < n ? __ldg(chunk_user + ci + step) : -1;
+    b2 = -1;
+  }
+  __device__ __forceinline__ bool valid() const { return ci < n_ci; }
+  __device__ __forceinline__ void prefetch(const int32_t* __restrict__ chunk_user) {
+    b2 = ci + 2 * stride < n_ci ? __ldg(chunk_user + ci + 2 * stride) : -1;
+  }
+  __device__ __forceinline__ void advance() { ci += stride; b0 = b1; b1 = b2; }
+};
+
 template <bool LN>
 __global__ void __launch_bounds__(LA_THREADS, 1)
 k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttnParams p) {
@@ -141,10 +166,10 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     return;
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LA_OFF_BAR);
-  uint64_t* x_full = bars;             // [4]
-  uint64_t* x_empty = bars + 4;        // [4]  second MMA of the tile done
-  uint64_t* q_full = bars + 22;         //      folded queries of the item's user landed
-  uint64_t* q_empty = bars + 23;       //      every score MMA of the item has read them
+  uint64_t* x_full = bars;             // [LA_XSTAGES]
+  uint64_t* x_empty = bars + 4;        // [LA_XSTAGES]  second MMA of the tile done
+  uint64_t* q_full = bars + 22;        // [2]  folded queries of a user landed in buffer i
+  uint64_t* q_empty = bars + 24;       // [2]  every score MMA that reads buffer i has run
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
   uint64_t* p_ready = bars + 10;       //      per tile: P' in smem (all softmax warps)
   uint64_t* p_free = bars + 12;        //      per tile: second MMA done reading P' (and accumulator up to date)
@@ -157,7 +182,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
-    mbar_init(q_full, 1); mbar_init(q_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
     mbar_init(p_ready, LA_SOFTMAX_WARPS); mbar_init(p_free, 1);
     mbar_init(o_free, LA_SOFTMAX_WARPS);
@@ -167,19 +192,26 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  const int32_t* chunk_start = p.chunk_start;
+  const int32_t* off = p.off;
+  if (p.B + 1 <= LA_IDX_CAP) {
+    int32_t* idx = reinterpret_cast<int32_t*>(smem + LA_OFF_IDX);
+    for (int i = threadIdx.x; i <= p.B; i += LA_THREADS) { idx[i] = p.chunk_start[i]; idx[LA_IDX_CAP + i] = p.off[i]; }
+    chunk_start = idx;
+    off = idx + LA_IDX_CAP;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   constexpr uint32_t COL_S = 0, COL_O = 256;      // scores: 2 x 128 columns; accumulator: d columns
 
-  // item -> (user, token range); identical in every role
+  // item -> token range; identical in every role
   const int rb = (int)blockIdx.x % p.RB;
-  auto item_range = [&](int wi, int& b, int& tok0, int& tok1) {
-    const int item = wi / p.RB;
-    b = upper_user(p.chunk_start, p.B, item);
-    tok0 = p.off[b] + (item - p.chunk_start[b]) * p.chunk;
-    tok1 = min(p.off[b + 1], tok0 + p.chunk);
+  const int ci_first = (int)blockIdx.x / p.RB, ci_step = (int)gridDim.x / p.RB, n_ci = n_items / p.RB;
+  auto item_range = [&](int ci, int b, int& tok0, int& tok1) {
+    tok0 = off[b] + (ci - chunk_start[b]) * p.chunk;
+    tok1 = min(off[b + 1], tok0 + p.chunk);
   };
 
   if (warp == 0) {
@@ -188,16 +220,21 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
       bool ok = true;
       int g = 0, qn = 0, prev_user = -1;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        int b, tok0, tok1;
-        item_range(item, b, tok0, tok1);
+      ItemWalk w;
+      for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance()) {
+        w.prefetch(p.chunk_user);
+        const int b = w.b0;
+        int tok0, tok1;
+        item_range(w.ci, b, tok0, tok1);
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
-          if (qn > 0 && !mbar_wait(q_empty, (uint32_t)(qn - 1) & 1u, p.err, 42)) { ok = false; break; }
-          mbar_arrive_expect_tx(q_full, 2 * LA_SUB);
+          const int qb = qn & 1;
+          if (!mbar_wait(&q_empty[qb], ((uint32_t)(qn >> 1) & 1u) ^ 1u, p.err, 42)) { ok = false; break; }
+          mbar_arrive_expect_tx(&q_full[qb], LA_Q2_BUF);
           for (int kb = 0; kb < 2; ++kb)
-            tma_load_2d_hint(smem + LA_OFF_Q2 + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128, q_full, pol_keep);
+            tma_load_2d_hint(smem + LA_OFF_Q2 + qb * LA_Q2_BUF + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128,
+                             &q_full[qb], pol_keep);
           ++qn;
         }
         const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
@@ -214,7 +251,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
         for (int j = 0; j < g && j < LA_XSTAGES; ++j)
           mbar_wait_quiet(&x_full[(g - 1 - j) % LA_XSTAGES], (uint32_t)((g - 1 - j) / LA_XSTAGES) & 1u);
-        if (qn > 0) mbar_wait_quiet(q_full, (uint32_t)(qn - 1) & 1u);
+        for (int j = 0; j < qn && j < 2; ++j) mbar_wait_quiet(&q_full[(qn - 1 - j) & 1], (uint32_t)((qn - 1 - j) >> 1) & 1u);
       }
     }
   } else if (warp == 1) {
@@ -223,13 +260,14 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128);                 // Q2 . X^T  : both K-major
       constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);    // P' . X    : B is MN-major
       const uint32_t sbase = smem_u32(smem);
+      uint32_t q2_off = LA_OFF_Q2;                 // buffer of the current user's folded queries
       auto issue_scores = [&](int g) -> bool {
         const int s = g % LA_XSTAGES;
         if (!mbar_wait(&x_full[s], (uint32_t)(g / LA_XSTAGES) & 1u, p.err, 51)) return false;
         tc_fence_after();
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * 128, make_sdesc_k_sw128(sbase + LA_OFF_Q2 + o),
+          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * 128, make_sdesc_k_sw128(sbase + q2_off + o),
                       make_sdesc_k_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + o), idesc_s, kk != 0);
         }
         mma_commit(&s_full[g & 1]);
@@ -237,27 +275,29 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       };
       bool ok = true;
       int g = 0, qn = 0, k = 0, prev_user = -1;
-      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
-        int b, tok0, tok1;
-        item_range(item, b, tok0, tok1);
+      ItemWalk w;
+      for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance(), ++k) {
+        w.prefetch(p.chunk_user);
+        const int b = w.b0;
+        int tok0, tok1;
+        item_range(w.ci, b, tok0, tok1);
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
-          if (!mbar_wait(q_full, (uint32_t)qn & 1u, p.err, 50)) { ok = false; break; }
+          if (!mbar_wait(&q_full[qn & 1], (uint32_t)(qn >> 1) & 1u, p.err, 50)) { ok = false; break; }
+          q2_off = LA_OFF_Q2 + (uint32_t)(qn & 1) * LA_Q2_BUF;
           ++qn;
         }
         // will the producer replace the queries after this item?
-        bool next_reloads = false;
-        if (!p.shared && item + (int)gridDim.x < n_items)
-          next_reloads = upper_user(p.chunk_start, p.B, (item + (int)gridDim.x) / p.RB) != b;
+        const bool next_reloads = !p.shared && w.b1 >= 0 && w.b1 != b;
         const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
         if (!issue_scores(g)) { ok = false; break; }
-        if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
+        if (n_tiles == 1 && next_reloads) mma_commit(&q_empty[(qn - 1) & 1]);
         for (int t = 0; t < n_tiles; ++t, ++g) {
           // the next tile's scores overlap this tile's softmax (its score buffer was read before p_ready(g-1))
           if (t + 1 < n_tiles) {
             if (!issue_scores(g + 1)) { ok = false; break; }
-            if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
+            if (t + 2 == n_tiles && next_reloads) mma_commit(&q_empty[(qn - 1) & 1]);
           }
           const int s = g % LA_XSTAGES;
           if (!mbar_wait(p_ready, (uint32_t)g & 1u, p.err, 52)) { ok = false; break; }
@@ -287,12 +327,18 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     float* exch_max = reinterpret_cast<float*>(smem + LA_OFF_EXCH);          // [2 tile parities][PARTS][128]
     float* exch_sum = exch_max + 2 * LA_PARTS * 128;                         // [PARTS][128]
     float* exch_mean = exch_sum + LA_PARTS * 128;                            // [PARTS][128]
+    // where this thread's part of its (head, link) row goes: fixed for the life of the CTA
+    const int R = rb * 128 + (int)r;                            // row among all H * ell
+    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * LA_D) + (R / p.ell) * LA_D + col0;
     bool ok = true;
     int g = 0, k = 0;
     uint32_t stats_uses = 0, row_uses = 0;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++k) {
-      int b, tok0, tok1;
-      item_range(item, b, tok0, tok1);
+    ItemWalk w;
+    for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance(), ++k) {
+      w.prefetch(p.chunk_user);
+      const int b = w.b0;
+      int tok0, tok1;
+      item_range(w.ci, b, tok0, tok1);
       const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
       const float cq = LN ? p.cQ[(int64_t)(p.shared ? 0 : b) * p.HL + rb * 128 + r] : 0.f;
       float m_ref = -INFINITY, l_sum = 0.f, mean_corr = 0.f;
@@ -399,14 +445,12 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
-      const bool single = p.chunk_start[b + 1] - p.chunk_start[b] == 1;
-      const int R = rb * 128 + (int)r;                          // row among all H * ell
-      const int64_t prow = (int64_t)(item / p.RB) * p.HL + R;   // row of the per-chunk partials
+      const bool single = chunk_start[b + 1] - chunk_start[b] == 1;
+      const int64_t prow = (int64_t)w.ci * p.HL + R;            // row of the per-chunk partials
       if (single) {
         // the whole history of this user was one chunk: normalise and write the attention rows directly
         const float inv = 1.0f / l_tot;
-        const int h = R / p.ell, l = R % p.ell;
-        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + ((int64_t)b * p.ell + l) * (p.H * LA_D) + h * LA_D + col0);
+        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + (int64_t)b * p.ell * (p.H * LA_D) + ohat_off);
 #pragma unroll
         for (int c8 = 0; c8 < LA_COLS / 8; ++c8) {
           uint4 o;
@@ -449,7 +493,7 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
       !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), LA_D, LA_D, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   LinkAttnParams p;
-  p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
+  p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
   int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;

@@ -59,7 +59,7 @@ k_tile_schedule(const int32_t* __restrict__ off, int B, int tile, int32_t* __res
 // both work lists of the XOR layers in one launch: chunks of the links<-history attention, tiles of the history update
 __global__ void __launch_bounds__(1024)
 k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __restrict__ chunk_start, int tile,
-                  int32_t* __restrict__ tile_start) {
+                  int32_t* __restrict__ tile_start, int32_t* __restrict__ chunk_user) {
   block_exclusive_scan(B, chunk_start, [&](int i) {
     int n = off[i + 1] - off[i];
     return n > 0 ? (n + chunk - 1) / chunk : 0;
@@ -69,12 +69,18 @@ k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __
     int n = off[i + 1] - off[i];
     return n > 0 ? (n + tile - 1) / tile : 0;
   });
+  // inverse map (chunk item -> user): the attention kernel strides through the items, and one read of this table
+  // replaces a search over chunk_start per item
+  __syncthreads();
+  if (chunk_user != nullptr)
+    for (int b = threadIdx.x; b < B; b += blockDim.x)
+      for (int i = chunk_start[b]; i < chunk_start[b + 1]; ++i) chunk_user[i] = b;
 }
 
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
-                                   cudaStream_t st) {
+                                   int32_t* chunk_user, cudaStream_t st) {
   ProfScope _p("k_layer_schedules", st);
-  k_layer_schedules<<<1, 1024, 0, st>>>(off, B, chunk, chunk_start, tile, tile_start);
+  k_layer_schedules<<<1, 1024, 0, st>>>(off, B, chunk, chunk_start, tile, tile_start, chunk_user);
   LIME_LAUNCH_CHECK("k_layer_schedules");
   return LIME_OK;
 }

@@ -97,9 +97,10 @@ lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const 
 
 // tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B  (work list of per-user token tiles)
 lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st);
-// chunk_start (tile = chunk) and tile_start (tile = tile) in one launch
+// chunk_start (tile = chunk) and tile_start (tile = tile) in one launch; chunk_user[item] = user of the chunk item
+// (may be NULL)
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
-                                   cudaStream_t st);
+                                   int32_t* chunk_user, cudaStream_t st);
 
 // Y[r, n] (+)= epilogue( LN?(X[r, :]) . W[:, n] ) for up to three weight matrices sharing X.
 struct LinearArgs {
@@ -206,6 +207,7 @@ struct LinkAttnArgs {
   const void* hist; int64_t total;          // [total x d] bf16
   const void* Q2; const float* cQ;          // folded link queries [users x H*ell x d] bf16 and their row sums
   const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
+  const int32_t* chunk_user;                // [items] user of each (user, chunk) work item
   int ell, d, H, shared, ln; float ln_eps;
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
   void* Ohat;                               // [B*ell x H*d] bf16: rows of users whose history is one chunk
