@@ -329,7 +329,11 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     float* exch_mean = exch_sum + LA_PARTS * 128;                            // [PARTS][128]
     // where this thread's part of its (head, link) row goes: fixed for the life of the CTA
     const int R = rb * 128 + (int)r;                            // row among all H * ell
-    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * LA_D) + (R / p.ell) * LA_D + col0;
+    // final rows are stored after a 4 x 4 transpose of 16-byte chunks inside each group of four lanes: lane 4j+i then
+    // holds chunk i of rows 4j..4j+3, so every store instruction writes whole 64-byte row parts.  Four consecutive
+    // rows share a head (ell is a multiple of 4), so they are H * d elements apart.
+    const int R4 = rb * 128 + q * 32 + (lane & ~3);
+    const int64_t ohat_off = (int64_t)(R4 % p.ell) * (p.H * LA_D) + (R4 / p.ell) * LA_D + col0 + (lane & 3) * 8;
     bool ok = true;
     int g = 0, k = 0;
     uint32_t stats_uses = 0, row_uses = 0;
@@ -450,16 +454,29 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       if (single) {
         // the whole history of this user was one chunk: normalise and write the attention rows directly
         const float inv = 1.0f / l_tot;
-        uint4* dst = reinterpret_cast<uint4*>(p.Ohat + (int64_t)b * p.ell * (p.H * LA_D) + ohat_off);
+        static_assert(LA_COLS == 32, "the chunk transpose below moves four 16-byte chunks per thread");
+        uint4 tch[4];
 #pragma unroll
-        for (int c8 = 0; c8 < LA_COLS / 8; ++c8) {
-          uint4 o;
-          o.x = la_pack((a[c8 * 8 + 0] - c_tot) * inv, (a[c8 * 8 + 1] - c_tot) * inv);
-          o.y = la_pack((a[c8 * 8 + 2] - c_tot) * inv, (a[c8 * 8 + 3] - c_tot) * inv);
-          o.z = la_pack((a[c8 * 8 + 4] - c_tot) * inv, (a[c8 * 8 + 5] - c_tot) * inv);
-          o.w = la_pack((a[c8 * 8 + 6] - c_tot) * inv, (a[c8 * 8 + 7] - c_tot) * inv);
-          dst[c8] = o;
+        for (int c8 = 0; c8 < 4; ++c8) {
+          tch[c8].x = la_pack((a[c8 * 8 + 0] - c_tot) * inv, (a[c8 * 8 + 1] - c_tot) * inv);
+          tch[c8].y = la_pack((a[c8 * 8 + 2] - c_tot) * inv, (a[c8 * 8 + 3] - c_tot) * inv);
+          tch[c8].z = la_pack((a[c8 * 8 + 4] - c_tot) * inv, (a[c8 * 8 + 5] - c_tot) * inv);
+          tch[c8].w = la_pack((a[c8 * 8 + 6] - c_tot) * inv, (a[c8 * 8 + 7] - c_tot) * inv);
         }
+        auto xchg = [&](uint4& keep_lo, uint4& keep_hi, bool upper, int dist) {
+          // lanes with `upper` clear give away keep_hi and receive into it; lanes with it set give away keep_lo
+          uint4 send = upper ? keep_lo : keep_hi, recv;
+          recv.x = __shfl_xor_sync(0xffffffffu, send.x, dist); recv.y = __shfl_xor_sync(0xffffffffu, send.y, dist);
+          recv.z = __shfl_xor_sync(0xffffffffu, send.z, dist); recv.w = __shfl_xor_sync(0xffffffffu, send.w, dist);
+          if (upper) keep_lo = recv; else keep_hi = recv;
+        };
+        xchg(tch[0], tch[1], (lane & 1) != 0, 1);
+        xchg(tch[2], tch[3], (lane & 1) != 0, 1);
+        xchg(tch[0], tch[2], (lane & 2) != 0, 2);
+        xchg(tch[1], tch[3], (lane & 2) != 0, 2);
+        __nv_bfloat16* dst = p.Ohat + (int64_t)b * p.ell * (p.H * LA_D) + ohat_off;
+#pragma unroll
+        for (int m = 0; m < 4; ++m) *reinterpret_cast<uint4*>(dst + (int64_t)m * (p.H * LA_D)) = tch[m];
       } else {
         float4* dst = reinterpret_cast<float4*>(p.part_acc + prow * LA_D + col0);
 #pragma unroll

@@ -427,6 +427,18 @@ def test_config4_long_history_sampled():
     _sampled_parity(wl, seed=0, users=[0, 7])
 
 
+def test_config3_candidate_sweep_largest_C_sampled():
+    # the last point of the candidate sweep (App. F): 32768 candidates per user, in the launch shape the bench times
+    wl = synth.named_workloads()["candidate_sweep"].replace(C=32768)
+    _sampled_parity(wl, seed=1, users=[0, 31, 63], n_cand=48)
+
+
+def test_config4_long_history_longest_N_sampled():
+    # the last point of the history sweep: 32768 tokens per user, 32 users (many chunks per user, merged partials)
+    wl = synth.named_workloads()["long_history"].replace(n_min=32768, n_max=32768)
+    _sampled_parity(wl, seed=1, users=[0, 31], n_cand=48)
+
+
 def test_config5_production_ragged_sampled():
     wl = synth.named_workloads()["production_ragged"].replace(B=32, V=200_000, C=512)
     inp_len = synth.history_lengths(0, wl.B, wl.n_min, wl.n_max)
