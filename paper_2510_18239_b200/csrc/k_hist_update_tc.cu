@@ -41,8 +41,8 @@ constexpr uint32_t HU_OFF_GU = HU_OFF_K2 + 2 * HU_SUB; // [2f x HL]     2 K-bloc
 constexpr uint32_t HU_OFF_WO = HU_OFF_GU + 4 * HU_SUB; // [d x f]       2 K-blocks x 16 KB
 constexpr uint32_t HU_OFF_PU = HU_OFF_WO + 2 * HU_SUB; // P, then U, of the current tile: 2 K-blocks
 constexpr uint32_t HU_OFF_STATS = HU_OFF_PU + 2 * HU_SUB;   // 2 (tile parity) x 128 float2 {rstd, mu}
-constexpr uint32_t HU_OFF_EXCH = HU_OFF_STATS + 2 * 128 * 8;   // row exchange: [PARTS][128] sums, then the same of squares
-constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 2 * HU_PARTS * 128 * 4;   // the current user's HL key row sums (fp32)
+constexpr uint32_t HU_OFF_EXCH = HU_OFF_STATS + 2 * 128 * 8;   // row exchange: [2 tile parities][PARTS][128] float2 {mean, M2}
+constexpr uint32_t HU_OFF_CK = HU_OFF_EXCH + 2 * HU_PARTS * 128 * 8;   // the current user's HL key row sums (fp32)
 constexpr uint32_t HU_OFF_BAR = HU_OFF_CK + HU_HL * 4;
 constexpr int HU_IDX_CAP = 1025;                            // users + 1 whose offsets are staged in shared memory (the
 constexpr uint32_t HU_OFF_IDX = HU_OFF_BAR + 256;           // search for a tile's user is a chain of dependent reads:
@@ -52,6 +52,7 @@ static_assert(HU_SMEM <= 232448, "shared memory budget of one CTA");
 struct HistUpdateParams {
   __nv_bfloat16* out;            // [total x d]
   const float* cK;               // [users x HL] row sums of K2
+  const float2* stats_in;        // nullable (LN): {rstd, mean} of every history row, computed by the attention kernel
   const int32_t* off;            // [B+1]
   const int32_t* tile_start;     // [B+1] prefix of per-user tile counts (tile = 128 tokens)
   int B, ell, shared, out_ln;
@@ -75,6 +76,19 @@ struct TileUser {
       hi = tile_start[b + 1];
     }
     return b;
+  }
+};
+// the same walk for code that needs the token rows of a tile: the user's row range is cached with the tile range
+struct TileRows {
+  TileUser tu;
+  int row_lo = 0, row_hi = 0;
+  // first token row of tile t; row_hi is the end of its user's rows
+  __device__ __forceinline__ int first_row(const int32_t* __restrict__ tile_start, const int32_t* __restrict__ off, int B,
+                                           int t, int tile) {
+    const int before = tu.b;
+    const int b = tu.of(tile_start, B, t);
+    if (b != before) { row_lo = off[b]; row_hi = off[b + 1]; }
+    return row_lo + (t - tu.lo) * tile;
   }
 };
 
@@ -281,7 +295,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const uint32_t r = (uint32_t)(q * 32 + lane);            // token row of the tile == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     float2* stats = reinterpret_cast<float2*>(smem + HU_OFF_STATS);
-    float* exch = reinterpret_cast<float*>(smem + HU_OFF_EXCH);                 // [2 slots][PARTS][128]
+    float* exch = reinterpret_cast<float*>(smem + HU_OFF_EXCH);                 // [2 tile parities][PARTS][128] float2
     const float* ck_s = reinterpret_cast<const float*>(smem + HU_OFF_CK) + col0;   // key row sums of this thread's columns
     // K index = column, so this thread's columns live in K-block col0 / 64, chunks (col0 % 64) / 8 ..
     uint8_t* pu = smem + HU_OFF_PU + (col0 >> 6) * HU_SUB;
@@ -289,12 +303,24 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     uint32_t stats_uses = 0, row_uses = 0;
     int ck_user = -1;
     bool ok = true;
-    TileUser tu;
     float rstd_r = 1.f, mu_r = 0.f;                          // LayerNorm constants of this thread's token row
 
     // LayerNorm statistics of tile g: four lanes per token, 32 features each; then this thread's own row constants.
     // Two slots by tile parity: a warp past the rendezvous of tile g+1 knows every warp has read tile g's.
+    // With statistics handed over by the attention kernel, a thread needs only those of its own row: one 8-byte read,
+    // issued a tile ahead (fetch_stats) and taken here.
+    TileRows tr_next, tr_out;       // walkers over the tile being prepared (g + 1) and the tile being stored (g)
+    float2 st_ahead = make_float2(1.f, 0.f);
+    auto fetch_stats = [&](int g) {
+      const int row = tr_next.first_row(tile_start, off, p.B, t_begin + g, HU_TILE) + (int)r;
+      st_ahead = row < tr_next.row_hi ? __ldg(p.stats_in + row) : make_float2(1.f, 0.f);
+    };
     auto take_stats = [&](int g) -> bool {
+      if (LN && p.stats_in != nullptr) {
+        rstd_r = st_ahead.x; mu_r = st_ahead.y;
+        if (lane == 0) mbar_arrive(x_empty);
+        return true;
+      }
       if (LN) {
         if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 31)) return false;
         const int tok = 8 * rw + (lane >> 2), p4 = lane & 3;
@@ -342,7 +368,9 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
     // 2. per-head softmax over the links of this thread's heads (32 score columns), P -> smem
     auto softmax = [&](int g) -> bool {
-      const int b = tu.of(tile_start, p.B, t_begin + g);
+      float v[HU_COLS];
+      tr_next.first_row(tile_start, off, p.B, t_begin + g, HU_TILE);
+      const int b = tr_next.tu.b;
       if (!mbar_wait(s2_full, (uint32_t)g & 1u, p.err, 32)) return false;
       tc_fence_after();
       if (LN && b != ck_user && (ck_user < 0 || !p.shared)) {
@@ -353,7 +381,6 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         __syncwarp();
       }
       ck_user = b;
-      float v[HU_COLS];
       tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
       tmem_wait_ld();
 #pragma unroll
@@ -375,15 +402,17 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         }
         const float inv = __fdividef(1.f, s0 + s1);
 #pragma unroll
-        for (int c8 = 0; c8 < ELL / 8; ++c8) {
-          const int c = h * ELL + c8 * 8;                    // first of 8 consecutive contraction indices
-          uint4 o;
-          o.x = pack_bf16(v[c + 0] * inv, v[c + 1] * inv);
-          o.y = pack_bf16(v[c + 2] * inv, v[c + 3] * inv);
-          o.z = pack_bf16(v[c + 4] * inv, v[c + 5] * inv);
-          o.w = pack_bf16(v[c + 6] * inv, v[c + 7] * inv);
-          *reinterpret_cast<uint4*>(pu + sw128_chunk(r, chunk0 + ((uint32_t)c >> 3))) = o;
-        }
+        for (int j = 0; j < ELL; ++j) v[h * ELL + j] *= inv;
+      }
+#pragma unroll
+      for (int c8 = 0; c8 < HU_COLS / 8; ++c8) {
+        const int c = c8 * 8;                                // first of 8 consecutive contraction indices
+        uint4 o;
+        o.x = pack_bf16(v[c + 0], v[c + 1]);
+        o.y = pack_bf16(v[c + 2], v[c + 3]);
+        o.z = pack_bf16(v[c + 4], v[c + 5]);
+        o.w = pack_bf16(v[c + 6], v[c + 7]);
+        *reinterpret_cast<uint4*>(pu + sw128_chunk(r, chunk0 + (uint32_t)c8)) = o;
       }
       tc_fence_before();
       fence_proxy_async_smem();
@@ -421,9 +450,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
     // 6. this thread's 32 columns of its S' row -> (LayerNorm) -> bf16 -> global.  The caller has waited for sp_full(g).
     auto store_rows = [&](int g) -> bool {
-      const int t = t_begin + g;
-      const int b = tu.of(tile_start, p.B, t);
-      const int row0 = off[b] + (t - tu.lo) * HU_TILE;
+      const int row0 = tr_out.first_row(tile_start, off, p.B, t_begin + g, HU_TILE);
       float v[HU_COLS];
       tmem_ld_32x32(lane_addr + COL_SS + (uint32_t)(g & 1) * 128 + col0, v);
       tmem_wait_ld();
@@ -431,27 +458,30 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       __syncwarp();
       if (lane == 0) mbar_arrive(sp_free);
       if (p.out_ln) {
-        // separate slots for the two exchanges: each is rewritten only after a later rendezvous of the same row group
+        // one exchange per row: every part sends the mean of its columns and their squared deviations from it, and
+        // the four pairs are combined exactly (sum of the parts' deviations + the spread of the parts' means).  Two
+        // slots by tile parity: a slot is rewritten only after a later rendezvous of the same row group.
         float s = 0.f;
 #pragma unroll
         for (int j = 0; j < HU_COLS; ++j) s += v[j];
-        exch[part * 128 + r] = s;
+        const float m_part = s * (1.0f / HU_COLS);
+        float m2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < HU_COLS; ++j) { const float dv = v[j] - m_part; m2 = fmaf(dv, dv, m2); }
+        float2* ex2 = reinterpret_cast<float2*>(exch) + (g & 1) * HU_PARTS * 128;
+        ex2[part * 128 + r] = make_float2(m_part, m2);
         if (!hu_group_sync(&row_bar[q], row_uses, lane, p.err, 37)) return false;
-        float tot = 0.f;
+        float2 pm[HU_PARTS];
+        float mu = 0.f;
 #pragma unroll
-        for (int i = 0; i < HU_PARTS; ++i) tot += exch[i * 128 + r];
-        const float mu = tot * (1.0f / HU_D);
-        float var = 0.f;
-#pragma unroll
-        for (int j = 0; j < HU_COLS; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
-        exch[(HU_PARTS + part) * 128 + r] = var;
-        if (!hu_group_sync(&row_bar[q], row_uses, lane, p.err, 39)) return false;
+        for (int i = 0; i < HU_PARTS; ++i) { pm[i] = ex2[i * 128 + r]; mu += pm[i].x; }
+        mu *= (1.0f / HU_PARTS);
         float vt = 0.f;
 #pragma unroll
-        for (int i = 0; i < HU_PARTS; ++i) vt += exch[(HU_PARTS + i) * 128 + r];
+        for (int i = 0; i < HU_PARTS; ++i) { const float dm = pm[i].x - mu; vt += pm[i].y + (float)HU_COLS * dm * dm; }
         const float rstd = rsqrtf(vt * (1.0f / HU_D) + p.ln_eps);
 #pragma unroll
-        for (int j = 0; j < HU_COLS; ++j) v[j] *= rstd;
+        for (int j = 0; j < HU_COLS; ++j) v[j] = (v[j] - mu) * rstd;
       }
       // bf16 row part = 4 chunks of 16 bytes.  A 4 x 4 transpose of chunks inside each group of four lanes (two
       // butterfly steps of warp shuffles) leaves lane 4j+i with chunk i of rows 4j..4j+3, so that every store
@@ -474,7 +504,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       xchg(tch[0], tch[2], (lane & 2) != 0, 2);
       xchg(tch[1], tch[3], (lane & 2) != 0, 2);
       const int rbase = row0 + q * 32 + (lane & ~3);          // first of the four rows this lane group holds
-      const int row_end = off[b + 1];
+      const int row_end = tr_out.row_hi;
 #pragma unroll
       for (int m = 0; m < 4; ++m)
         if (rbase + m < row_end)
@@ -482,8 +512,10 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       return true;
     };
 
+    if (LN && p.stats_in != nullptr) fetch_stats(0);
     ok = take_stats(0) && softmax(0);
     for (int g = 0; g < n && ok; ++g) {
+      if (LN && p.stats_in != nullptr && g + 1 < n) fetch_stats(g + 1);
       if (!silu_mul(g)) { ok = false; break; }                                   // [gate|up](g) ran under store(g-1)
       // statistics of the next tile while S'(g) is formed, so that its stage can be refilled a whole tile early
       if (g + 1 < n && !take_stats(g + 1)) { ok = false; break; }
@@ -519,7 +551,7 @@ static lime_status launch_hu(const HistUpdateArgs& a, cudaStream_t st) {
       !make_tmap_bf16_sw128(&tmWo, a.WoT, HU_D, HU_F, HU_F, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   HistUpdateParams p;
-  p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.ell = ELL;
+  p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.stats_in = a.ln ? a.stats_in : nullptr; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.ell = ELL;
   p.shared = a.shared; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
   int grid = a.n_tile_upper < kSMs ? a.n_tile_upper : kSMs;
   if (grid < 1) return LIME_OK;

@@ -61,6 +61,7 @@ struct LinkAttnParams {
   float ln_eps;
   float *part_m, *part_s, *part_acc;   // [items x HL], [items x HL], [items x HL x d]
   __nv_bfloat16* Ohat;                 // [B*ell x H*d]: final rows of single-chunk users
+  float2* stats_out;                   // nullable: {rstd, mean} per history row (written by the CTAs of row block 0)
   int* err;
 };
 
@@ -384,7 +385,11 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           }
           var += __shfl_xor_sync(0xffffffffu, var, 1);
           var += __shfl_xor_sync(0xffffffffu, var, 2);
-          if (p4 == 0) stats[s * 128 + tok] = make_float2(rsqrtf(var * (1.0f / LA_D) + p.ln_eps), mu);
+          if (p4 == 0) {
+            const float2 rm = make_float2(rsqrtf(var * (1.0f / LA_D) + p.ln_eps), mu);
+            stats[s * 128 + tok] = rm;
+            if (p.stats_out != nullptr && rb == 0 && tok < nvalid) p.stats_out[tok0 + t * LA_TILE + tok] = rm;
+          }
           if (!la_group_sync(stats_bar, stats_uses, lane, p.err, 62)) { ok = false; break; }
         }
         if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
@@ -512,7 +517,7 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
   LinkAttnParams p;
   p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
-  p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
+  p.Ohat = (__nv_bfloat16*)a.Ohat; p.stats_out = a.ln ? a.stats_out : nullptr; p.err = a.err;
   int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;
   grid -= grid % p.RB;                              // a CTA's work items then all share its row block
   static bool smem_ln[kMaxDeviceOrdinals] = {}, smem_plain[kMaxDeviceOrdinals] = {};

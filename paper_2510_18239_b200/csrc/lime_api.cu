@@ -59,6 +59,7 @@ struct Workspace {
   // tensor-core path: folded link-side operands (bf16) and their row sums
   void *Q2, *K2, *G2t, *U2t;
   float *cQ, *cK;
+  float2* row_stats;   // LayerNorm {rstd, mean} of the history rows of the layer being processed
   void *That, *Ohat, *UTb;   // LN(T) [B*ell x d], merged attention rows [B*ell x H*d], GLU output [B*ell x d_ff] (bf16)
   int chunk, n_chunk_upper, n_tile_upper;
   size_t bytes;
@@ -92,6 +93,7 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.Q2 = take((size_t)B * HL * g.d * 2); w.K2 = take((size_t)B * HL * g.d * 2);
   w.G2t = take((size_t)B * c->d_ff * HL * 2); w.U2t = take((size_t)B * c->d_ff * HL * 2);
   w.cQ = (float*)take((size_t)B * HL * 4); w.cK = (float*)take((size_t)B * HL * 4);
+  w.row_stats = (float2*)take((size_t)total * 8);
   w.That = take((size_t)B * g.ell * g.d * 2); w.Ohat = take((size_t)B * g.ell * g.H * g.d * 2);
   w.UTb = take((size_t)B * g.ell * c->d_ff * 2);
   w.bytes = o;
@@ -139,6 +141,10 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
   la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = ops.shared;
   la.ln = hist_ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
   la.err = c->dev_err;
+  // the attention kernel forms the LayerNorm statistics of every history row anyway; the history update reuses them
+  const bool one_block_update = hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
+  const bool pass_stats = hist_ln && hist_out && one_block_update && total > 0;
+  la.stats_out = pass_stats ? w.row_stats : nullptr;
   if ((s = launch_link_attn_tc(la, st)) != LIME_OK) return s;
   if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
     return s;
@@ -153,7 +159,8 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
     hu.cK = ops.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
     hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = ops.shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
     hu.out_ln = out_ln; hu.err = c->dev_err;
-    if (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) s = launch_hist_update_tc(hu, st);
+    hu.stats_in = pass_stats ? w.row_stats : nullptr;
+    if (one_block_update) s = launch_hist_update_tc(hu, st);
     else s = launch_hist_update2_tc(hu, g.H, st);
     if (s != LIME_OK) return s;
   }

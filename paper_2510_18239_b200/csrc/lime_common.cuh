@@ -211,6 +211,7 @@ struct LinkAttnArgs {
   int ell, d, H, shared, ln; float ln_eps;
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
   void* Ohat;                               // [B*ell x H*d] bf16: rows of users whose history is one chunk
+  float2* stats_out;                        // nullable, ln only: {rstd, mean} of every history row, for the history update
   int* err;
 };
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi);
@@ -222,6 +223,7 @@ struct HistUpdateArgs {
   const int32_t* off; const int32_t* tile_start; int B, n_tile_upper;
   int ell, shared, ln; float ln_eps;    // ln: apply LayerNorm to the rows read (0 when they were stored normalised)
   int out_ln;                           // 1: store LayerNorm(S') instead of S'
+  const float2* stats_in;               // nullable, ln only: {rstd, mean} of every row read, as left by the attention kernel
   int* err;
 };
 bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
