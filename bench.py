@@ -58,6 +58,8 @@ def kernel_models(wl: synth.Workload, total_tokens: int):
     down = 2.0 * d * f * (BL * n + N * (n - 1))
     return {
         "k_score": dict(bytes=BC * (es * ell + es * d + 4.0)),
+        # by id from the corpus caches: the same rows, fetched one by one, + the 4-byte id
+        "k_score_gather_tc": dict(bytes=BC * (es * ell + es * d + 8.0)),
         "k_gather": dict(bytes=N * (4.0 + 2 * es * d)),
         "k_precompute": dict(bytes=BC * es * (d + ell)),
         # fused tensor-core layer kernels: history rows read once per direction, written once by the update
@@ -240,9 +242,11 @@ def launch_mode(args):
 NCU_TRAFFIC = {
     # profiles/k_score_tc_bf16_baseline.md: 169.9 MB read + 4.0-4.5 MB written per launch
     ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
-    # profiles/xor_layer_kernels_bf16_baseline.md: 33.7 MB (layer 1) and 42.0 MB (layer 2) read; average per launch
-    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.8e6, "source": "k_link_attn_tc.cu", "sha": "e56b781284e88a10"},
-    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.4e6, "source": "k_hist_update_tc.cu", "sha": "24cb0f708e8e5b84"},
+    # profiles/xor_layer_kernels_bf16_baseline.md: 33.9 MB (layer 1) and 42.2 MB (layer 2) read + written; average per launch
+    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 38.1e6, "source": "k_link_attn_tc.cu", "sha": "bbd1c1f1fbb6c856"},
+    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 35.6e6, "source": "k_hist_update_tc.cu", "sha": "5d823b7efc1ff4d8"},
+    # profiles/k_score_gather_tc_bf16_baseline.md: 170.0 MB read + 3.9 MB written per launch
+    ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 173.9e6, "source": "k_score_gather_tc.cu", "sha": "4daad32675f4aff5"},
 }
 
 
@@ -561,6 +565,9 @@ def run_ours(args, wl):
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps, "host_issue_ms_per_step": 1e3 * t_issue / args.steps,
                         "score_by_id_alone_ms": score_by_id_ms,
+                        "score_by_id_roofline": dict(kernel="k_score_gather_tc", **roofline_entry(models["k_score_gather_tc"], score_by_id_ms, pk),
+                                                     traffic=ncu_traffic("k_score_gather_tc", wl),
+                                                     note="random 128-byte pieces; the copy peak is for contiguous streams"),
                         "how": "pinned host ids -> H2D | offsets, history gather, encode, scoring by candidate id from the resident "
                                "corpus caches | logits D2H; three streams, two request slots"},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roofline, "scoring_roofline": scoring,
