@@ -282,6 +282,44 @@ def test_xor_layer_tensor_core_path(ell, H, lengths, shared_links):
             assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
 
 
+@pytest.mark.parametrize("ell,H", [(32, 4), (64, 4)])
+def test_xor_layer_tensor_core_path_many_users(ell, H):
+    """More users than the kernels stage offsets for in shared memory (1024): the work lists are then read from global
+    memory.  Short ragged histories (some empty, some longer than a tile), sampled users checked against the oracle."""
+    Bd = _lib()
+    B = 1100
+    r = np.random.default_rng(5)
+    lengths = r.integers(0, 200, size=B).astype(np.int32)
+    lengths[[0, 7, 500, 1099]] = [130, 0, 257, 129]
+    wl = small(synth.BF16, B=B, n_min=0, n_max=1, d=128, H=H, ell=ell, n_layers=1, V=3000, table_std=0.05)
+    inp = synth.make_inputs(wl, seed=ell)
+    inp["lengths"] = lengths
+    total = int(lengths.sum())
+    inp["hist_ids"] = synth.zipf_ids(4, "h", total, wl.V, 1.1)
+    dev = Hh.DeviceBatch(wl, inp)
+    L = dev.lime
+    off = L.lengths_to_offsets(dev.lengths)
+    hist = L.gather_history(dev.table, dev.hist_ids)
+    links32 = dev.links.float().contiguous()
+    hist_out = torch.zeros_like(hist)
+    links_out = torch.empty((B, ell, wl.d), dtype=torch.float32, device="cuda")
+    Bd.lime_xor_layer(L.ctx, 0, hist, off, B, links32, True, hist_out, links_out, L.workspace(B, total))
+    assert Bd.lime_device_status(L.ctx) == 0
+    cfg = Hh.oracle_config(wl)
+    lw = Hh.oracle_layers(inp, wl)[0]
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    offh = O.lengths_to_offsets(lengths)
+    assert np.array_equal(off.cpu().numpy(), offh)
+    for b in [0, 1, 7, 8, 499, 500, 501, 1023, 1024, 1025, 1098, 1099]:
+        E = O.gather_history(table64, inp["hist_ids"][offh[b]:offh[b + 1]])
+        S_next, T_next = O.xor_layer(E, links64, lw, cfg)
+        assert np.abs(Hh.to_f64(links_out[b]) - T_next).max() <= 4e-2 * max(1.0, np.abs(T_next).max()), b
+        if lengths[b]:
+            got = Hh.to_f64(hist_out[offh[b]:offh[b + 1]])
+            assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
+
+
 @pytest.mark.parametrize("ln", [True, False])
 def test_link_attention_running_max_is_raised_mid_history(ln):
     """History whose later tiles score far higher than the first one for half of the link rows (the second 128 tokens
