@@ -327,8 +327,9 @@ def run_ours(args, wl):
         s = sets[i % ROTATE]
         h = hist[: s["total"]]
         Bd.lime_lengths_to_offsets(ctx, s["lengths"], off)
-        Bd.lime_gather_history(ctx, table, s["hist_ids"], h)
-        Bd.lime_encode_user(ctx, h, off, wl.B, None, ls, ws)
+        # the lookup applies the first layer's LayerNorm on the way (every layer reads the history through it only)
+        Bd.lime_gather_history_normalized(ctx, table, s["hist_ids"], h)
+        Bd.lime_encode_user_normalized(ctx, h, off, wl.B, None, ls, ws)
         Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
 
     def barrier():
@@ -436,8 +437,8 @@ def run_ours(args, wl):
         k, n = i % SLOTS, host_sets[i % ROTATE]["total"]
         h = hist[:n]
         Bd.lime_lengths_to_offsets(ctx, d_len[k], off)
-        Bd.lime_gather_history(ctx, table, d_hid[k][:n], h)
-        Bd.lime_encode_user(ctx, h, off, wl.B, None, ls, ws)
+        Bd.lime_gather_history_normalized(ctx, table, d_hid[k][:n], h)
+        Bd.lime_encode_user_normalized(ctx, h, off, wl.B, None, ls, ws)
         # candidates are scored straight from the corpus caches by id (no gather of their rows)
         Bd.lime_score_candidates(ctx, ls, wl.B, w_corpus, table, None, wl.C, wl.B * wl.C, d_cid[k], d_logits[k])
 

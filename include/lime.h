@@ -117,6 +117,15 @@ LIME_API lime_status lime_lengths_to_offsets(lime_ctx* ctx, const int32_t* len, 
 LIME_API lime_status lime_gather_history(lime_ctx* ctx, const void* table, int64_t V, const int32_t* ids,
                                 int64_t total_tokens, void* out, int32_t* dev_flag, void* stream);
 
+/* The same lookup with the LayerNorm of the first XOR layer applied on the way:
+ *   out[t,:] = LN(table[ids[t],:])   (non-affine, eps of the config, rounded to config.dtype).
+ * The XOR layers read the history only through the LayerNorm that precedes their Q/K/V projections (App. C, Eq. 1 /
+ * Eq. 7), so nothing downstream needs the raw rows; normalising them here, while a row sits in registers, spares both
+ * attention directions of the first layer the per-token statistics.  Pass the result to lime_encode_user_normalized.
+ * Same arguments, layouts and treatment of bad ids as lime_gather_history; with config.ln = 0 it is that call. */
+LIME_API lime_status lime_gather_history_normalized(lime_ctx* ctx, const void* table, int64_t V, const int32_t* ids,
+                                           int64_t total_tokens, void* out, int32_t* dev_flag, void* stream);
+
 /* Offline item-side stage (Eq. 4, Sec. 3.3 "pre-computed and cached"): out_w[c,:] = softmax over the ell
  * links of (T_c W_Q^c)(L W_K^c)^T * cand_scale.  cand_emb [M x d], out_w [M x ell] stored as config.dtype. */
 LIME_API lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb, int64_t M, void* out_w,
@@ -140,6 +149,14 @@ LIME_API lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hi
 LIME_API lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off, int32_t B,
                              int64_t total_tokens, const float* link_ctx, void* link_states, void* ws,
                              size_t ws_bytes, void* stream);
+
+/* lime_encode_user for history rows that are LayerNorm-ed already (as lime_gather_history_normalized leaves them):
+ * the first layer then skips its LayerNorm of the history.  Same arguments, ownership and errors.  The result equals
+ * lime_encode_user on the raw rows up to the rounding of the normalised rows to config.dtype.  With config.ln = 0 the
+ * two calls are the same. */
+LIME_API lime_status lime_encode_user_normalized(lime_ctx* ctx, const void* hist_normalized, const int32_t* off, int32_t B,
+                                        int64_t total_tokens, const float* link_ctx, void* link_states, void* ws,
+                                        size_t ws_bytes, void* stream);
 
 /* Per-candidate stage (Eq. 4 and Sec. 3.3 "lightweight user-item interaction"):
  *   logits[i] = < sum_l cand_w[i,l] * link_states[b(i),l,:] , cand_emb[i,:] >   for every candidate slot i.

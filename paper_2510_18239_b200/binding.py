@@ -45,7 +45,8 @@ class lime_weights(ctypes.Structure):
 
 
 EXPORTS = ("lime_create", "lime_destroy", "lime_set_weights", "lime_workspace_bytes", "lime_lengths_to_offsets",
-           "lime_gather_history", "lime_precompute_candidate_links", "lime_xor_layer", "lime_encode_user",
+           "lime_gather_history", "lime_gather_history_normalized", "lime_precompute_candidate_links", "lime_xor_layer",
+           "lime_encode_user", "lime_encode_user_normalized",
            "lime_score_candidates", "lime_precompute_candidate_links_noalloc", "lime_device_status", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
            "lime_version")
 
@@ -70,9 +71,11 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_workspace_bytes.restype = sz
     lib.lime_lengths_to_offsets.argtypes = [vp, vp, i32, vp, vp]
     lib.lime_gather_history.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp]
+    lib.lime_gather_history_normalized.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp]
     lib.lime_precompute_candidate_links.argtypes = [vp, vp, i64, vp, vp]
     lib.lime_xor_layer.argtypes = [vp, i32, vp, vp, i32, i64, vp, i32, vp, vp, vp, sz, vp]
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
+    lib.lime_encode_user_normalized.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, vp, vp]
     lib.lime_precompute_candidate_links_noalloc.argtypes = [i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, i64, vp, vp]
     lib.lime_device_status.argtypes = [vp, ctypes.POINTER(i32)]
@@ -142,6 +145,12 @@ def lime_gather_history(ctx: int, table: torch.Tensor, ids: torch.Tensor, out: t
                                               _ptr(dev_flag), _stream()), "lime_gather_history")
 
 
+def lime_gather_history_normalized(ctx: int, table: torch.Tensor, ids: torch.Tensor, out: torch.Tensor,
+                                   dev_flag: Optional[torch.Tensor] = None) -> None:
+    _check(load_library().lime_gather_history_normalized(ctx, _ptr(table), table.shape[0], _ptr(ids), ids.numel(), _ptr(out),
+                                                         _ptr(dev_flag), _stream()), "lime_gather_history_normalized")
+
+
 def lime_precompute_candidate_links(ctx: int, cand_emb: torch.Tensor, out_w: torch.Tensor) -> None:
     _check(load_library().lime_precompute_candidate_links(ctx, _ptr(cand_emb), cand_emb.shape[0], _ptr(out_w), _stream()),
            "lime_precompute_candidate_links")
@@ -160,6 +169,14 @@ def lime_encode_user(ctx: int, hist: torch.Tensor, off: torch.Tensor, B: int, li
     _check(load_library().lime_encode_user(ctx, _ptr(hist), _ptr(off), B, hist.shape[0], _ptr(link_ctx),
                                            _ptr(link_states), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "lime_encode_user")
+
+
+def lime_encode_user_normalized(ctx: int, hist_normalized: torch.Tensor, off: torch.Tensor, B: int,
+                                link_ctx: Optional[torch.Tensor], link_states: torch.Tensor, ws: torch.Tensor) -> None:
+    _check(load_library().lime_encode_user_normalized(ctx, _ptr(hist_normalized), _ptr(off), B, hist_normalized.shape[0],
+                                                      _ptr(link_ctx), _ptr(link_states), _ptr(ws),
+                                                      ws.numel() * ws.element_size(), _stream()),
+           "lime_encode_user_normalized")
 
 
 def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: torch.Tensor, cand_emb: torch.Tensor,
@@ -276,6 +293,19 @@ class Lime:
         out = torch.empty((ids.numel(), self.cfg.d), dtype=self.tdtype, device=ids.device)
         lime_gather_history(self.ctx, table, ids, out, flag)
         return out
+
+    def gather_history_normalized(self, table: torch.Tensor, ids: torch.Tensor,
+                                  flag: Optional[torch.Tensor] = None) -> torch.Tensor:
+        out = torch.empty((ids.numel(), self.cfg.d), dtype=self.tdtype, device=ids.device)
+        lime_gather_history_normalized(self.ctx, table, ids, out, flag)
+        return out
+
+    def encode_user_normalized(self, hist_normalized: torch.Tensor, off: torch.Tensor,
+                               link_ctx: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B = off.numel() - 1
+        ls = torch.empty((B, self.cfg.ell, self.cfg.d), dtype=self.tdtype, device=hist_normalized.device)
+        lime_encode_user_normalized(self.ctx, hist_normalized, off, B, link_ctx, ls, self.workspace(B, hist_normalized.shape[0]))
+        return ls
 
     def precompute_candidate_links(self, cand_emb: torch.Tensor) -> torch.Tensor:
         out = torch.empty((cand_emb.shape[0], self.cfg.ell), dtype=self.tdtype, device=cand_emb.device)

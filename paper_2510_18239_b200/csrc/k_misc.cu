@@ -124,6 +124,126 @@ k_gather(const uint4* __restrict__ table, int64_t V, int row_vec, const int32_t*
   }
 }
 
+// out[t, :] = LayerNorm(table[ids[t], :]) (non-affine), in the storage type.  Same row-per-LANES mapping; a lane keeps
+// its WORDS 16-byte words of the row in registers, the lanes of a row reduce the sum and then the squared
+// deviations with shuffles (two passes: exact mean first), and the normalised row is written once.  The loop runs
+// per warp-wide group of rows so that every lane takes part in the shuffles.
+template <typename T, int LANES, int WORDS>
+__global__ void __launch_bounds__(256)
+k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, float eps, const int32_t* __restrict__ ids,
+            int64_t total, uint4* __restrict__ out, int32_t* __restrict__ dev_flag) {
+  constexpr int PER = 16 / (int)sizeof(T);                 // elements per 16-byte word
+  constexpr int ROWS = 1;   // rows per lane group and pass (more in flight measured slower: the grid already covers the latency)
+  const int rows_per_block = blockDim.x / LANES;
+  const int sub = threadIdx.x % LANES;
+  const int64_t stride = (int64_t)gridDim.x * rows_per_block * ROWS;
+  for (int64_t base = (int64_t)blockIdx.x * rows_per_block * ROWS; base < total; base += stride) {
+    int64_t t[ROWS];
+    bool live[ROWS], ok[ROWS];
+    int32_t id[ROWS];
+#pragma unroll
+    for (int k = 0; k < ROWS; ++k) {
+      t[k] = base + (int64_t)k * rows_per_block + threadIdx.x / LANES;
+      live[k] = t[k] < total;
+      id[k] = live[k] ? __ldg(ids + t[k]) : 0;
+      ok[k] = live[k] && id[k] >= 0 && (int64_t)id[k] < V;
+    }
+    uint4 w[ROWS][WORDS];
+#pragma unroll
+    for (int k = 0; k < ROWS; ++k)
+#pragma unroll
+      for (int i = 0; i < WORDS; ++i) {
+        const int v = sub + i * LANES;
+        w[k][i] = (ok[k] && v < row_vec) ? __ldg(table + (int64_t)id[k] * row_vec + v) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+    for (int k = 0; k < ROWS; ++k) {
+      float x[WORDS][PER];
+      float sum = 0.f;
+#pragma unroll
+      for (int i = 0; i < WORDS; ++i) {
+        const T* e = reinterpret_cast<const T*>(&w[k][i]);
+#pragma unroll
+        for (int j = 0; j < PER; ++j) { x[i][j] = Store<T>::ld(e + j); sum += x[i][j]; }
+      }
+#pragma unroll
+      for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      const float mu = sum / (float)d;
+      float var = 0.f;
+#pragma unroll
+      for (int i = 0; i < WORDS; ++i) {
+        if (sub + i * LANES < row_vec) {
+#pragma unroll
+          for (int j = 0; j < PER; ++j) { const float c = x[i][j] - mu; var = fmaf(c, c, var); }
+        }
+      }
+#pragma unroll
+      for (int o = LANES / 2; o > 0; o >>= 1) var += __shfl_xor_sync(0xffffffffu, var, o);
+      const float rstd = rsqrtf(var / (float)d + eps);
+      if (live[k]) {
+#pragma unroll
+        for (int i = 0; i < WORDS; ++i) {
+          const int v = sub + i * LANES;
+          if (v < row_vec) {
+            uint4 o4 = make_uint4(0, 0, 0, 0);              // an id outside [0, V) gives a zero row, as in k_gather
+            if (ok[k]) {
+              T* e = reinterpret_cast<T*>(&o4);
+#pragma unroll
+              for (int j = 0; j < PER; ++j) Store<T>::st(e + j, (x[i][j] - mu) * rstd);
+            }
+            out[t[k] * row_vec + v] = o4;
+          }
+        }
+        if (!ok[k] && sub == 0 && dev_flag != nullptr) atomicMin(dev_flag, (int32_t)min(t[k], (int64_t)INT32_MAX));
+      }
+    }
+  }
+}
+
+template <typename T, int WORDS>
+static void launch_gather_ln_w(int lanes, int blocks, const uint4* tb, int64_t V, int row_vec, int d, float eps,
+                               const int32_t* ids, int64_t total, uint4* o, int32_t* dev_flag, cudaStream_t st) {
+  switch (lanes) {
+    case 32: k_gather_ln<T, 32, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    case 16: k_gather_ln<T, 16, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    case 8:  k_gather_ln<T, 8, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    default: k_gather_ln<T, 4, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+  }
+}
+template <typename T>
+static lime_status launch_gather_ln_t(int lanes, int words, int blocks, const uint4* tb, int64_t V, int row_vec, int d, float eps,
+                                      const int32_t* ids, int64_t total, uint4* o, int32_t* dev_flag, cudaStream_t st) {
+  if (words <= 1) launch_gather_ln_w<T, 1>(lanes, blocks, tb, V, row_vec, d, eps, ids, total, o, dev_flag, st);
+  else if (words <= 2) launch_gather_ln_w<T, 2>(lanes, blocks, tb, V, row_vec, d, eps, ids, total, o, dev_flag, st);
+  else if (words <= 4) launch_gather_ln_w<T, 4>(lanes, blocks, tb, V, row_vec, d, eps, ids, total, o, dev_flag, st);
+  else if (words <= 8) launch_gather_ln_w<T, 8>(lanes, blocks, tb, V, row_vec, d, eps, ids, total, o, dev_flag, st);
+  else return LIME_UNSUPPORTED_SHAPE;                                  // d <= 1024 keeps a row within 32 lanes x 8 words
+  return LIME_OK;
+}
+
+lime_status launch_gather_ln(int dtype, const void* table, int64_t V, int d, float eps, const int32_t* ids, int64_t total,
+                             void* out, int32_t* dev_flag, cudaStream_t st) {
+  if (total == 0) return LIME_OK;
+  const int es = dtype == LIME_F32 ? 4 : 2;
+  const int row_vec = d * es / 16;
+  // two words per lane where the row allows: half the shuffle steps and two independent loads per thread
+  int lanes = row_vec >= 64 ? 32 : (row_vec >= 32 ? 16 : (row_vec >= 16 ? 8 : 4));
+  const int words = (row_vec + lanes - 1) / lanes;
+  const int rows_per_block = 256 / lanes;
+  int64_t blocks = (total + rows_per_block - 1) / rows_per_block;
+  const int64_t cap = (int64_t)kSMs * 16;
+  if (blocks > cap) blocks = cap;
+  ProfScope _p("k_gather_ln", st);
+  const lime_status s =
+      dtype == LIME_F32
+          ? launch_gather_ln_t<float>(lanes, words, (int)blocks, (const uint4*)table, V, row_vec, d, eps, ids, total, (uint4*)out, dev_flag, st)
+          : launch_gather_ln_t<__nv_bfloat16>(lanes, words, (int)blocks, (const uint4*)table, V, row_vec, d, eps, ids, total, (uint4*)out,
+                                              dev_flag, st);
+  if (s != LIME_OK) return s;
+  LIME_LAUNCH_CHECK("k_gather_ln");
+  return LIME_OK;
+}
+
 lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const int32_t* ids, int64_t total,
                           void* out, int32_t* dev_flag, cudaStream_t st) {
   if (total == 0) return LIME_OK;

@@ -187,7 +187,7 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
 // the shared L: its operands are weights-only and were formed at lime_set_weights), then the streaming kernels.
 // Between layers the history is kept LayerNorm-ed (every consumer normalises it first, Eq. 1 with App. C's LayerNorm),
 // so only the first layer pays for the statistics.
-static lime_status encode_user_tc(Ctx* c, const void* hist, const int32_t* off, int32_t B, int64_t total,
+static lime_status encode_user_tc(Ctx* c, const void* hist, bool hist_normalized, const int32_t* off, int32_t B, int64_t total,
                                   const float* link_ctx, void* link_states, const Workspace& w, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
@@ -206,7 +206,7 @@ static lime_status encode_user_tc(Ctx* c, const void* hist, const int32_t* off, 
     mlp.LP = w.LP; mlp.lp_accumulate = j > 0;                                   // L^P = sum_j T^j  (Eq. 8)
     mlp.That_next = last ? nullptr : w.That;
     mlp.link_states = (last && !c->w.cand_Wv) ? link_states : nullptr;
-    s = tc_layer_core(c, j, j == 0 ? hist : w.S, off, B, total, ops, last ? nullptr : w.S, (g.ln && j == 0) ? 1 : 0,
+    s = tc_layer_core(c, j, j == 0 ? hist : w.S, off, B, total, ops, last ? nullptr : w.S, (g.ln && j == 0 && !hist_normalized) ? 1 : 0,
                       (g.ln && !last) ? 1 : 0, mlp, w, st);
     if (s != LIME_OK) return s;
   }
@@ -216,7 +216,9 @@ static lime_status encode_user_tc(Ctx* c, const void* hist, const int32_t* off, 
 // One XOR layer on a carved workspace (see lime_xor_layer in lime.h for the contract).
 static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const int32_t* off, int32_t B,
                                   int64_t total, const float* links_in, int links_shared, void* hist_out,
-                                  float* links_out, const Workspace& w, bool schedules_ready, cudaStream_t st) {
+                                  float* links_out, const Workspace& w, bool schedules_ready, int hist_ln, cudaStream_t st) {
+  // hist_ln: LayerNorm the history rows read (config.ln, except on the first layer of an encode whose rows arrive
+  // normalised).  The tensor-core branch is only taken by the single-layer call, whose input is never normalised.
   const lime_config& g = c->cfg;
   lime_status s;
   if (!schedules_ready) {
@@ -241,7 +243,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   lh.X = hist_in; lh.x_dtype = g.dtype; lh.M = total; lh.K = g.d; lh.N = g.d; lh.w_dtype = g.dtype; lh.y_dtype = g.dtype;
   lh.W[0] = c->w.Wk[layer]; lh.W[1] = c->w.Wv[layer]; lh.W[2] = c->w.Wq[layer];
   lh.Y[0] = w.K; lh.Y[1] = w.V; lh.Y[2] = w.Q; lh.n_out = hist_out ? 3 : 2;
-  lh.ln = g.ln; lh.ln_eps = c->ln_eps;
+  lh.ln = hist_ln; lh.ln_eps = c->ln_eps;
   if ((s = launch_linear_simt(lh, st)) != LIME_OK) return s;
 
   // O[T] = phi(Q[T] K[S]^T) V[S]
@@ -489,6 +491,18 @@ lime_status lime_gather_history(lime_ctx* ctx, const void* table, int64_t V, con
                        static_cast<cudaStream_t>(stream));
 }
 
+lime_status lime_gather_history_normalized(lime_ctx* ctx, const void* table, int64_t V, const int32_t* ids,
+                                           int64_t total_tokens, void* out, int32_t* dev_flag, void* stream) {
+  if (!ctx || total_tokens < 0 || V < 0) return LIME_INVALID_ARG;
+  if (total_tokens == 0) return LIME_OK;
+  if (!table || !ids || !out || !aligned16(table) || !aligned16(out)) return LIME_INVALID_ARG;
+  const Ctx* c = reinterpret_cast<const Ctx*>(ctx);
+  if (!c->cfg.ln)
+    return launch_gather(c->cfg.dtype, table, V, c->cfg.d, ids, total_tokens, out, dev_flag, static_cast<cudaStream_t>(stream));
+  return launch_gather_ln(c->cfg.dtype, table, V, c->cfg.d, c->ln_eps, ids, total_tokens, out, dev_flag,
+                          static_cast<cudaStream_t>(stream));
+}
+
 lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb, int64_t M, void* out_w, void* stream) {
   if (!ctx || M < 0) return LIME_INVALID_ARG;
   Ctx* c = reinterpret_cast<Ctx*>(ctx);
@@ -518,11 +532,12 @@ lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hist_in, co
   Workspace w = carve(c, base, B, total_tokens);
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
   return xor_layer_impl(c, layer, hist_in, off, B, total_tokens, links_in, links_shared, hist_out, links_out, w, false,
-                        static_cast<cudaStream_t>(stream));
+                        c->cfg.ln, static_cast<cudaStream_t>(stream));
 }
 
-lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off, int32_t B, int64_t total_tokens,
-                             const float* link_ctx, void* link_states, void* ws, size_t ws_bytes, void* stream) {
+static lime_status encode_user_impl(lime_ctx* ctx, const void* hist, bool hist_normalized, const int32_t* off, int32_t B,
+                                    int64_t total_tokens, const float* link_ctx, void* link_states, void* ws, size_t ws_bytes,
+                                    void* stream) {
   if (!ctx || B < 0 || total_tokens < 0 || total_tokens > 0x7fffffffLL) return LIME_INVALID_ARG;
   Ctx* c = reinterpret_cast<Ctx*>(ctx);
   if (!c->have_weights) return LIME_NOT_READY;
@@ -541,14 +556,15 @@ lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off
   if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, st)) != LIME_OK) return s;
   const int64_t BLd = (int64_t)B * g.ell * g.d;
   if (layer_on_tensor_cores(c, 0)) {
-    if ((s = encode_user_tc(c, hist, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;
+    if ((s = encode_user_tc(c, hist, hist_normalized, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;
     if (!c->w.cand_Wv) return LIME_OK;        // the last layer's kernel wrote the link states
   } else {
     for (int j = 0; j < g.n_layers; ++j) {
       const bool last = j == g.n_layers - 1;
       const float* lin = j == 0 ? (link_ctx ? link_ctx : c->links32) : w.T;
       const int shared = (j == 0 && !link_ctx) ? 1 : 0;
-      s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true, st);
+      s = xor_layer_impl(c, j, j == 0 ? hist : w.S, off, B, total_tokens, lin, shared, last ? nullptr : w.S, w.T, w, true,
+                         (g.ln && !(j == 0 && hist_normalized)) ? 1 : 0, st);
       if (s != LIME_OK) return s;
       if ((s = launch_axpy(w.T, w.LP, BLd, j == 0, st)) != LIME_OK) return s;   // L^P = sum_j T^j  (Eq. 8)
     }
@@ -563,6 +579,17 @@ lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off
     src = w.LS32;
   }
   return launch_cast_rows(src, BLd, link_states, g.dtype, st);
+}
+
+lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off, int32_t B, int64_t total_tokens,
+                             const float* link_ctx, void* link_states, void* ws, size_t ws_bytes, void* stream) {
+  return encode_user_impl(ctx, hist, false, off, B, total_tokens, link_ctx, link_states, ws, ws_bytes, stream);
+}
+
+lime_status lime_encode_user_normalized(lime_ctx* ctx, const void* hist_normalized, const int32_t* off, int32_t B,
+                                        int64_t total_tokens, const float* link_ctx, void* link_states, void* ws,
+                                        size_t ws_bytes, void* stream) {
+  return encode_user_impl(ctx, hist_normalized, true, off, B, total_tokens, link_ctx, link_states, ws, ws_bytes, stream);
 }
 
 lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,

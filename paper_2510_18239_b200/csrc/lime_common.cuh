@@ -94,6 +94,9 @@ lime_status launch_offsets(const int32_t* len, int B, int32_t* off, cudaStream_t
 
 lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const int32_t* ids, int64_t total,
                           void* out, int32_t* dev_flag, cudaStream_t st);
+// the same lookup with the non-affine LayerNorm of the row applied before it is stored
+lime_status launch_gather_ln(int dtype, const void* table, int64_t V, int d, float eps, const int32_t* ids, int64_t total,
+                             void* out, int32_t* dev_flag, cudaStream_t st);
 
 // tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B  (work list of per-user token tiles)
 lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st);

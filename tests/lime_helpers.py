@@ -61,12 +61,17 @@ class DeviceBatch:
         self.hist_ids = torch.from_numpy(inp["hist_ids"]).cuda()
         self.cand_ids = torch.from_numpy(inp["cand_ids"]).cuda() if "cand_ids" in inp else None
 
-    def run(self):
-        """offsets -> gather -> encode -> (candidate gather, precompute) -> score. Returns dict of tensors."""
+    def run(self, normalized=False):
+        """offsets -> gather -> encode -> (candidate gather, precompute) -> score. Returns dict of tensors.
+        normalized: take the history through the fused lookup + LayerNorm and the encode entry that expects it."""
         L = self.lime
         off = L.lengths_to_offsets(self.lengths)
-        hist = L.gather_history(self.table, self.hist_ids)
-        ls = L.encode_user(hist, off)
+        if normalized:
+            hist = L.gather_history_normalized(self.table, self.hist_ids)
+            ls = L.encode_user_normalized(hist, off)
+        else:
+            hist = L.gather_history(self.table, self.hist_ids)
+            ls = L.encode_user(hist, off)
         cand = L.gather_history(self.table, self.cand_ids)
         W = L.precompute_candidate_links(cand)
         logits = L.score_candidates(ls, W, cand, C=self.wl.C)

@@ -68,6 +68,33 @@ def test_gather_bit_exact_and_bad_ids(dtype, d):
 
 
 # ----------------------------------------------------------------------------- candidate side
+@pytest.mark.parametrize("dtype,d", [(synth.F32, 8), (synth.F32, 64), (synth.F32, 1024), (synth.BF16, 8), (synth.BF16, 40),
+                                     (synth.BF16, 128), (synth.BF16, 256), (synth.BF16, 1024)])
+def test_gather_normalized_is_layer_norm_of_the_rows(dtype, d):
+    """Lookup fused with the non-affine LayerNorm (App. C): every row equals the oracle's LayerNorm of the table row
+    to the rounding of the storage type; ids outside the table give zero rows and the smallest bad position."""
+    Bd = _lib()
+    V, n = 777, 5000
+    r = np.random.default_rng(d)
+    table = synth.to_storage(r.normal(size=(V, d)) * r.uniform(0.01, 3.0, size=(V, 1)) + r.normal(size=(V, 1)), dtype)
+    ids = r.integers(0, V, size=n).astype(np.int32)
+    ids[[17, 4000]] = [V, -1]
+    H = max(1, d // 128)
+    L = Bd.Lime(d, H, 4, 1, dtype=Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16)
+    flag = torch.full((1,), 2 ** 31 - 1, dtype=torch.int32, device="cuda")
+    got = Hh.to_f64(L.gather_history_normalized(Bd.to_device(table, dtype), torch.from_numpy(ids).cuda(), flag))
+    assert int(flag.item()) == 17
+    want = O.layer_norm(synth.storage_to_f64(table, dtype)[np.clip(ids, 0, V - 1)])
+    want[[17, 4000]] = 0.0
+    tol = 1e-5 if dtype == synth.F32 else 2.0 ** -8
+    assert np.abs(got - want).max() <= tol * max(1.0, np.abs(want).max())
+    # with LayerNorm switched off in the configuration the call is the plain lookup
+    L0 = Bd.Lime(d, H, 4, 1, dtype=Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16, ln=False)
+    ok = np.clip(ids, 0, V - 1)
+    raw = Hh.to_f64(L0.gather_history_normalized(Bd.to_device(table, dtype), torch.from_numpy(ok).cuda()))
+    assert np.array_equal(raw, synth.storage_to_f64(table, dtype)[ok])
+
+
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 @pytest.mark.parametrize("ell,d,M", [(1, 8, 5), (8, 64, 300), (32, 128, 1000), (64, 256, 257), (33, 40, 64)])
 @pytest.mark.parametrize("proj", [False, True])
@@ -427,9 +454,9 @@ def test_config1_tiny_fp32_full_parity():
     assert np.abs(got - want_logits).max() <= 1e-3 * want_logits.std()     # fp32 path is far inside 1e-4
 
 
-def _sampled_parity(wl, seed, users, n_cand=64):
+def _sampled_parity(wl, seed, users, n_cand=64, normalized=False):
     inp = synth.make_inputs(wl, seed=seed)
-    out = Hh.DeviceBatch(wl, inp).run()
+    out = Hh.DeviceBatch(wl, inp).run(normalized=normalized)
     torch.cuda.synchronize()
     cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
     table64 = synth.storage_to_f64(inp["table"], wl.dtype)
@@ -439,8 +466,14 @@ def _sampled_parity(wl, seed, users, n_cand=64):
     # gathered rows: bit exact on a sample of tokens
     r = np.random.default_rng(seed)
     tok = r.integers(0, off[-1], size=512)
-    got_rows = out["hist"][torch.from_numpy(tok).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
-    assert np.array_equal(got_rows, inp["table"][inp["hist_ids"][tok]])
+    if normalized:
+        # rows after the fused lookup + LayerNorm: the oracle's LayerNorm of the same table rows, to bf16 rounding
+        got_rows = Hh.to_f64(out["hist"][torch.from_numpy(tok).cuda()])
+        want_rows = O.layer_norm(table64[inp["hist_ids"][tok]])
+        assert np.abs(got_rows - want_rows).max() <= 2.0 ** -8 * max(1.0, np.abs(want_rows).max())
+    else:
+        got_rows = out["hist"][torch.from_numpy(tok).cuda()].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert np.array_equal(got_rows, inp["table"][inp["hist_ids"][tok]])
     got_all, want_all = [], []
     for b in users:
         rows = np.sort(r.choice(wl.C, size=min(n_cand, wl.C), replace=False))
@@ -453,6 +486,37 @@ def _sampled_parity(wl, seed, users, n_cand=64):
 def test_config2_bf16_baseline_sampled():
     wl = synth.named_workloads()["bf16_baseline"]
     _sampled_parity(wl, seed=0, users=[0, 1, 100, 255])
+
+
+def test_config2_bf16_baseline_normalized_lookup_sampled():
+    # the launch sequence bench.py times: lookup fused with the first layer's LayerNorm, encode on normalised rows
+    wl = synth.named_workloads()["bf16_baseline"]
+    _sampled_parity(wl, seed=2, users=[0, 3, 128, 255], normalized=True)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny_fp32", {}), ("long_history", dict(n_min=700, n_max=1500, B=6)),
+                                     ("production_ragged", dict(B=8, V=50_000, C=256, n_min=100, n_max=700))])
+def test_normalized_lookup_on_other_paths(name, kw):
+    # fp32 storage and d = 256 run the generic path, which normalises again (a fixed point up to rounding);
+    # H * ell = 256 runs the streamed-operand kernels without their LayerNorm
+    wl = synth.named_workloads()[name].replace(**kw) if kw else synth.named_workloads()[name]
+    _sampled_parity_any_dtype(wl, normalized=True)
+
+
+def _sampled_parity_any_dtype(wl, normalized):
+    inp = synth.make_inputs(wl, seed=4)
+    out = Hh.DeviceBatch(wl, inp).run(normalized=normalized)
+    torch.cuda.synchronize()
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(inp["lengths"])
+    got_all, want_all = [], []
+    for b in sorted({0, wl.B - 1}):
+        lg, _, _ = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg)
+        got_all.append(Hh.to_f64(out["logits"][b * wl.C:(b + 1) * wl.C]))
+        want_all.append(lg)
+    _check_logits(np.concatenate(got_all), np.concatenate(want_all), wl.dtype)
 
 
 def test_config3_candidate_sweep_sampled():
