@@ -38,10 +38,13 @@ constexpr uint32_t LA_SUB = 128 * 128;
 constexpr uint32_t LA_X_STAGE = 2 * LA_SUB;
 constexpr uint32_t LA_OFF_X = 0;
 constexpr uint32_t LA_OFF_Q2 = LA_XSTAGES * LA_X_STAGE;
-constexpr uint32_t LA_Q2_BUF = 2 * LA_SUB;                    // folded queries of one user's row block; two buffers, so the
-                                                             // producer fetches the next user's while this one is in use
-constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + 2 * LA_Q2_BUF;     // P' [128 rows x 128 tokens]
-constexpr uint32_t LA_OFF_STATS = LA_OFF_P + 2 * LA_SUB;     // per X stage: float2 {rstd, mu} x 128 tokens
+constexpr uint32_t LA_Q2_BUF = 2 * LA_SUB;                    // folded queries of one user's row block
+constexpr int LA_Q2_BUFS = 1;                                // buffers of them (a user's queries are replaced after its last
+                                                             // score MMA, a tile before the item ends)
+constexpr int LA_PBUFS = 2;                                  // buffers of P': the second MMA of a tile runs while the
+constexpr uint32_t LA_P_BUF = 2 * LA_SUB;                    // softmax warps already write the next tile's P'
+constexpr uint32_t LA_OFF_P = LA_OFF_Q2 + LA_Q2_BUFS * LA_Q2_BUF;   // P' [128 rows x 128 tokens] x LA_PBUFS
+constexpr uint32_t LA_OFF_STATS = LA_OFF_P + LA_PBUFS * LA_P_BUF;   // per X stage: float2 {rstd, mu} x 128 tokens
 constexpr uint32_t LA_OFF_EXCH = LA_OFF_STATS + LA_XSTAGES * 128 * 8;   // [2 tile parities][PARTS][128] maxima, then
                                                                         // [PARTS][128] sums and [PARTS][128] mean terms
 constexpr uint32_t LA_OFF_BAR = LA_OFF_EXCH + 4 * LA_PARTS * 128 * 4;
@@ -173,7 +176,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   uint64_t* q_empty = bars + 24;       // [2]  every score MMA that reads buffer i has run
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
   uint64_t* p_ready = bars + 10;       //      per tile: P' in smem (all softmax warps)
-  uint64_t* p_free = bars + 12;        //      per tile: second MMA done reading P' (and accumulator up to date)
+  uint64_t* p_free = bars + 12;        // [2]  per tile and P' buffer: second MMA done reading P' (and accumulator up to date)
   uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
   uint64_t* stats_bar = bars + 15;     //      rendezvous of the softmax warps (token statistics written)
   uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the warps that share a TMEM lane quarter
@@ -185,7 +188,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
-    mbar_init(p_ready, LA_SOFTMAX_WARPS); mbar_init(p_free, 1);
+    mbar_init(p_ready, LA_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
     mbar_init(o_free, LA_SOFTMAX_WARPS);
     mbar_init(stats_bar, LA_SOFTMAX_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LA_PARTS);
@@ -230,8 +233,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
-          const int qb = qn & 1;
-          if (!mbar_wait(&q_empty[qb], ((uint32_t)(qn >> 1) & 1u) ^ 1u, p.err, 42)) { ok = false; break; }
+          const int qb = qn % LA_Q2_BUFS;
+          if (!mbar_wait(&q_empty[qb], ((uint32_t)(qn / LA_Q2_BUFS) & 1u) ^ 1u, p.err, 42)) { ok = false; break; }
           mbar_arrive_expect_tx(&q_full[qb], LA_Q2_BUF);
           for (int kb = 0; kb < 2; ++kb)
             tma_load_2d_hint(smem + LA_OFF_Q2 + qb * LA_Q2_BUF + kb * LA_SUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128,
@@ -252,7 +255,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
         for (int j = 0; j < g && j < LA_XSTAGES; ++j)
           mbar_wait_quiet(&x_full[(g - 1 - j) % LA_XSTAGES], (uint32_t)((g - 1 - j) / LA_XSTAGES) & 1u);
-        for (int j = 0; j < qn && j < 2; ++j) mbar_wait_quiet(&q_full[(qn - 1 - j) & 1], (uint32_t)((qn - 1 - j) >> 1) & 1u);
+        for (int j = 0; j < qn && j < LA_Q2_BUFS; ++j)
+          mbar_wait_quiet(&q_full[(qn - 1 - j) % LA_Q2_BUFS], (uint32_t)((qn - 1 - j) / LA_Q2_BUFS) & 1u);
       }
     }
   } else if (warp == 1) {
@@ -285,20 +289,20 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
-          if (!mbar_wait(&q_full[qn & 1], (uint32_t)(qn >> 1) & 1u, p.err, 50)) { ok = false; break; }
-          q2_off = LA_OFF_Q2 + (uint32_t)(qn & 1) * LA_Q2_BUF;
+          if (!mbar_wait(&q_full[qn % LA_Q2_BUFS], (uint32_t)(qn / LA_Q2_BUFS) & 1u, p.err, 50)) { ok = false; break; }
+          q2_off = LA_OFF_Q2 + (uint32_t)(qn % LA_Q2_BUFS) * LA_Q2_BUF;
           ++qn;
         }
         // will the producer replace the queries after this item?
         const bool next_reloads = !p.shared && w.b1 >= 0 && w.b1 != b;
         const int n_tiles = (tok1 - tok0 + LA_TILE - 1) / LA_TILE;
         if (!issue_scores(g)) { ok = false; break; }
-        if (n_tiles == 1 && next_reloads) mma_commit(&q_empty[(qn - 1) & 1]);
+        if (n_tiles == 1 && next_reloads) mma_commit(&q_empty[(qn - 1) % LA_Q2_BUFS]);
         for (int t = 0; t < n_tiles; ++t, ++g) {
           // the next tile's scores overlap this tile's softmax (its score buffer was read before p_ready(g-1))
           if (t + 1 < n_tiles) {
             if (!issue_scores(g + 1)) { ok = false; break; }
-            if (t + 2 == n_tiles && next_reloads) mma_commit(&q_empty[(qn - 1) & 1]);
+            if (t + 2 == n_tiles && next_reloads) mma_commit(&q_empty[(qn - 1) % LA_Q2_BUFS]);
           }
           const int s = g % LA_XSTAGES;
           if (!mbar_wait(p_ready, (uint32_t)g & 1u, p.err, 52)) { ok = false; break; }
@@ -307,12 +311,12 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           tc_fence_after();
           for (int kk = 0; kk < 8; ++kk) {      // contraction over the tile's 128 tokens, 16 per instruction
             const uint32_t oa = (uint32_t)(kk >> 2) * LA_SUB + (uint32_t)(kk & 3) * 32;
-            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + oa),
+            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LA_OFF_P + (uint32_t)(g % LA_PBUFS) * LA_P_BUF + oa),
                         make_sdesc_mn_sw128(sbase + LA_OFF_X + s * LA_X_STAGE + (uint32_t)kk * 2048, LA_SUB), idesc_o,
                         (t | kk) != 0);
           }
           mma_commit(&x_empty[s]);
-          mma_commit(p_free);
+          mma_commit(&p_free[g % LA_PBUFS]);
         }
       }
     }
@@ -411,7 +415,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         const float factor = (need && m_ref != -INFINITY) ? la_ex2(m_ref - m_new) : 1.0f;
         if (__any_sync(0xffffffffu, need && t > 0)) {
           // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this part of the row
-          if (!mbar_wait(p_free, (uint32_t)(g - 1) & 1u, p.err, 64)) { ok = false; break; }
+          if (!mbar_wait(&p_free[(g - 1) % LA_PBUFS], (uint32_t)((g - 1) / LA_PBUFS) & 1u, p.err, 64)) { ok = false; break; }
           tc_fence_after();
           float a[LA_COLS];
           tmem_ld_32x32(lane_addr + COL_O + col0, a);
@@ -425,10 +429,10 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         mean_corr *= factor;
         m_ref = m_new;
 
-        // the previous tile's P' must have been consumed
-        if (g >= 1 && !mbar_wait(p_free, (uint32_t)(g - 1) & 1u, p.err, 65)) { ok = false; break; }
+        // the P' that last sat in this buffer must have been consumed
+        if (g >= LA_PBUFS && !mbar_wait(&p_free[g % LA_PBUFS], (uint32_t)((g - LA_PBUFS) / LA_PBUFS) & 1u, p.err, 65)) { ok = false; break; }
         // pass 2: P' -> smem; K index = token column, so columns col0.. live in K-block col0 / 64, chunk (col0 % 64) / 8..
-        uint8_t* pbuf = smem + LA_OFF_P + (col0 >> 6) * LA_SUB;
+        uint8_t* pbuf = smem + LA_OFF_P + (g % LA_PBUFS) * LA_P_BUF + (col0 >> 6) * LA_SUB;
         const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
         if (nvalid == LA_TILE) la_pass2<LN, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
         else la_pass2<LN, true>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
@@ -440,7 +444,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       if (!ok) break;
       // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
       const int gl = g - 1;
-      if (!mbar_wait(p_free, (uint32_t)gl & 1u, p.err, 66)) { ok = false; break; }
+      if (!mbar_wait(&p_free[gl % LA_PBUFS], (uint32_t)(gl / LA_PBUFS) & 1u, p.err, 66)) { ok = false; break; }
       tc_fence_after();
       exch_sum[part * 128 + r] = l_sum;
       exch_mean[part * 128 + r] = mean_corr;
