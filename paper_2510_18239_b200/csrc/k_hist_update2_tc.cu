@@ -28,8 +28,8 @@ constexpr uint32_t H2_OFF_GU = H2_OFF_K2 + 2 * H2_SUB;  // [G2 | U2]_c [2f x 128
 constexpr uint32_t H2_OFF_WO = H2_OFF_GU + 4 * H2_SUB;  // [d x f]: 2 K-blocks
 constexpr uint32_t H2_OFF_PU = H2_OFF_WO + 2 * H2_SUB;  // P_c, then U: 2 K-blocks
 constexpr uint32_t H2_OFF_STATS = H2_OFF_PU + 2 * H2_SUB;    // 2 (tile parity) x 128 float2 {rstd, mu}
-constexpr uint32_t H2_OFF_EXCH = H2_OFF_STATS + 2 * 128 * 8; // pair exchange: [2 slots][2 halves][128]
-constexpr uint32_t H2_OFF_CK = H2_OFF_EXCH + 4 * 128 * 4;    // the current user's HL key row sums (up to 512 floats)
+constexpr uint32_t H2_OFF_EXCH = H2_OFF_STATS + 2 * 128 * 8; // pair exchange: [2 tile parities][2 halves][128] float2 {mean, M2}
+constexpr uint32_t H2_OFF_CK = H2_OFF_EXCH + 4 * 128 * 8;    // the current user's HL key row sums (up to 512 floats)
 constexpr uint32_t H2_OFF_BAR = H2_OFF_CK + 512 * 4;
 constexpr int H2_IDX_CAP = 1025;                            // users + 1 whose offsets are staged in shared memory (the
 constexpr uint32_t H2_OFF_IDX = H2_OFF_BAR + 256;           // search for a tile's user is a chain of dependent reads:
@@ -103,7 +103,7 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   uint64_t* ops_full = bars + 4;     // per (tile, group): [G2 | U2]_c landed
   uint64_t* ops_empty = bars + 5;    // per (tile, group): mix MMA done (producer's view)
   uint64_t* wo_full = bars + 6;
-  uint64_t* s2_full = bars + 7;      // per (tile, group): scores in TMEM
+  uint64_t* s2_full = bars + 20;     // [2] per (tile, group), by parity of the group counter: scores in TMEM
   uint64_t* p_ready = bars + 8;      // per (tile, group): P_c in smem (8 warps)
   uint64_t* p_free = bars + 9;       // per (tile, group): mix MMA done (row warps' view)
   uint64_t* gu_full = bars + 10;     // per tile: [gate | up] complete
@@ -124,7 +124,7 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   if (threadIdx.x == 0) {
     mbar_init(x_full, 1); mbar_init(x_empty, 1 + H2_ROW_WARPS);
     mbar_init(k2_full, 1); mbar_init(k2_empty, 1); mbar_init(ops_full, 1); mbar_init(ops_empty, 1); mbar_init(wo_full, 1);
-    mbar_init(s2_full, 1); mbar_init(p_ready, H2_ROW_WARPS); mbar_init(p_free, 1); mbar_init(gu_full, 1);
+    mbar_init(&s2_full[0], 1); mbar_init(&s2_full[1], 1); mbar_init(p_ready, H2_ROW_WARPS); mbar_init(p_free, 1); mbar_init(gu_full, 1);
     mbar_init(u_ready, H2_ROW_WARPS); mbar_init(sp_full, 1); mbar_init(sp_free, H2_ROW_WARPS); mbar_init(stats_bar, H2_ROW_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
     fence_barrier_init();
@@ -143,7 +143,10 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_S2 = 0, COL_GU = 128, COL_SP = 384;
+  // Two 128-column buffers take the scores of the groups and S' in rotation: use u of this CTA (per tile NG score uses,
+  // then S') goes to buffer u & 1, so the scores of the next group are formed while the row warps still read this one's.
+  constexpr uint32_t COL_A = 0, COL_GU = 128, COL_B = 384;
+  auto col_of = [&](int u) -> uint32_t { return (u & 1) ? COL_B : COL_A; };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -192,20 +195,31 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       const uint32_t pu = sbase + H2_OFF_PU;
       bool ok = mbar_wait(wo_full, 0, p.err, 21);
       int q = 0;
+      // scores of group qq (tile-local use index u): X . K2_c^T
+      auto issue_scores = [&](int qq, int u, bool last_of_tile) -> bool {
+        if (!mbar_wait(k2_full, (uint32_t)qq & 1u, p.err, 22)) return false;
+        tc_fence_after();
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint32_t o = (uint32_t)(kk >> 2) * H2_SUB + (uint32_t)(kk & 3) * 32;
+          mma_bf16_ss(tmem_base + col_of(u), make_sdesc_k_sw128(sbase + H2_OFF_X + o), make_sdesc_k_sw128(sbase + H2_OFF_K2 + o),
+                      idesc_128, kk != 0);
+        }
+        mma_commit(&s2_full[qq & 1]);
+        mma_commit(k2_empty);
+        if (last_of_tile) mma_commit(x_empty);
+        return true;
+      };
       for (int g = 0; g < n && ok; ++g) {
         if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 23)) break;
+        const int u0 = g * (NG + 1);
+        // 1. scores of the first group (its buffer last held the scores of the previous tile's last group: consumed)
+        if (!issue_scores(q, u0, NG == 1)) { ok = false; break; }
         for (int c = 0; c < NG && ok; ++c, ++q) {
-          // 1. scores_c = X . K2_c^T   (the previous scores were consumed before P_{q-1} was announced)
-          if (!mbar_wait(k2_full, (uint32_t)q & 1u, p.err, 22)) { ok = false; break; }
-          tc_fence_after();
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t o = (uint32_t)(kk >> 2) * H2_SUB + (uint32_t)(kk & 3) * 32;
-            mma_bf16_ss(tmem_base + COL_S2, make_sdesc_k_sw128(sbase + H2_OFF_X + o), make_sdesc_k_sw128(sbase + H2_OFF_K2 + o),
-                        idesc_128, kk != 0);
+          if (c + 1 < NG) {
+            // 1'. scores of the next group, under this group's softmax; for c = 0 the buffer last held S' of the previous tile
+            if (c == 0 && g > 0 && !mbar_wait(sp_free, (uint32_t)(g - 1) & 1u, p.err, 26)) { ok = false; break; }
+            if (!issue_scores(q + 1, u0 + c + 1, c + 1 == NG - 1)) { ok = false; break; }
           }
-          mma_commit(s2_full);
-          mma_commit(k2_empty);
-          if (c == NG - 1) mma_commit(x_empty);
           // 3. [gate | up] (+)= P_c . [G2 | U2]_c
           if (!mbar_wait(ops_full, (uint32_t)q & 1u, p.err, 27)) { ok = false; break; }
           if (!mbar_wait(p_ready, (uint32_t)q & 1u, p.err, 24)) { ok = false; break; }
@@ -221,13 +235,14 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           if (c == NG - 1) mma_commit(gu_full);
         }
         if (!ok) break;
-        // 5. S'(g) = U(g) . W_o
+        // 5. S'(g) = U(g) . W_o, into the buffer after the last group's (with one group that one last held S'(g-1))
         if (!mbar_wait(u_ready, (uint32_t)g & 1u, p.err, 25)) break;
-        if (g > 0 && !mbar_wait(sp_free, (uint32_t)(g - 1) & 1u, p.err, 26)) break;
+        if (NG == 1 && g > 0 && !mbar_wait(sp_free, (uint32_t)(g - 1) & 1u, p.err, 26)) break;
         tc_fence_after();
         for (int kk = 0; kk < 8; ++kk) {
           const uint32_t o = (uint32_t)(kk >> 2) * H2_SUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_SP, make_sdesc_k_sw128(pu + o), make_sdesc_k_sw128(sbase + H2_OFF_WO + o), idesc_128, kk != 0);
+          mma_bf16_ss(tmem_base + col_of(u0 + NG), make_sdesc_k_sw128(pu + o), make_sdesc_k_sw128(sbase + H2_OFF_WO + o), idesc_128,
+                      kk != 0);
         }
         mma_commit(sp_full);
       }
@@ -301,20 +316,19 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       }
       // ---- per group: softmax over the links of this thread's heads, P_c -> smem
       for (int c = 0; c < NG && ok; ++c, ++q) {
-        if (!mbar_wait(s2_full, (uint32_t)q & 1u, p.err, 32)) { ok = false; break; }
+        if (!mbar_wait(&s2_full[q & 1], (uint32_t)(q >> 1) & 1u, p.err, 32)) { ok = false; break; }
         tc_fence_after();
         float v[64];
         {
           float v0[32], v1[32];
-          tmem_ld_32x32(lane_addr + COL_S2 + half * 64, v0);
-          tmem_ld_32x32(lane_addr + COL_S2 + half * 64 + 32, v1);
+          const uint32_t cs = col_of(g * (NG + 1) + c);
+          tmem_ld_32x32(lane_addr + cs + half * 64, v0);
+          tmem_ld_32x32(lane_addr + cs + half * 64 + 32, v1);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
         }
         const float* ck_s = ck_all + c * 128 + half * 64;
-        // P_{q-1} (or U of the previous tile) must have been consumed before the buffer is rewritten
-        if (c > 0 && !mbar_wait(p_free, (uint32_t)(q - 1) & 1u, p.err, 36)) { ok = false; break; }
 #pragma unroll
         for (int h = 0; h < 64 / ELL; ++h) {
           float mx = -INFINITY;
@@ -334,15 +348,20 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
           }
           const float inv = __fdividef(1.f, s0 + s1);
 #pragma unroll
-          for (int c8 = 0; c8 < ELL / 8; ++c8) {
-            const int cc = h * ELL + c8 * 8;
-            uint4 o;
-            o.x = h2_pack(v[cc + 0] * inv, v[cc + 1] * inv);
-            o.y = h2_pack(v[cc + 2] * inv, v[cc + 3] * inv);
-            o.z = h2_pack(v[cc + 4] * inv, v[cc + 5] * inv);
-            o.w = h2_pack(v[cc + 6] * inv, v[cc + 7] * inv);
-            *reinterpret_cast<uint4*>(pu + h2_chunk(r, (uint32_t)cc >> 3)) = o;
-          }
+          for (int j = 0; j < ELL; ++j) v[h * ELL + j] *= inv;
+        }
+        // P_{q-1} must have been consumed by its mix MMA before the buffer is rewritten; the probabilities above were
+        // formed while that MMA ran
+        if (c > 0 && !mbar_wait(p_free, (uint32_t)(q - 1) & 1u, p.err, 36)) { ok = false; break; }
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8) {
+          const int cc = c8 * 8;
+          uint4 o;
+          o.x = h2_pack(v[cc + 0], v[cc + 1]);
+          o.y = h2_pack(v[cc + 2], v[cc + 3]);
+          o.z = h2_pack(v[cc + 4], v[cc + 5]);
+          o.w = h2_pack(v[cc + 6], v[cc + 7]);
+          *reinterpret_cast<uint4*>(pu + h2_chunk(r, (uint32_t)c8)) = o;
         }
         tc_fence_before();
         fence_proxy_async_smem();
@@ -382,8 +401,9 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       float v[64];
       {
         float v0[32], v1[32];
-        tmem_ld_32x32(lane_addr + COL_SP + half * 64, v0);
-        tmem_ld_32x32(lane_addr + COL_SP + half * 64 + 32, v1);
+        const uint32_t cs = col_of(g * (NG + 1) + NG);
+        tmem_ld_32x32(lane_addr + cs + half * 64, v0);
+        tmem_ld_32x32(lane_addr + cs + half * 64 + 32, v1);
         tmem_wait_ld();
 #pragma unroll
         for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
@@ -392,20 +412,24 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(sp_free);
       if (p.out_ln) {
+        // one exchange per row: each half sends the mean of its 64 columns and their squared deviations from it; the
+        // two pairs combine exactly.  Slots alternate by tile parity (rewritten only after a later rendezvous).
         float s = 0.f;
 #pragma unroll
         for (int j = 0; j < 64; ++j) s += v[j];
-        exch[half * 128 + r] = s;
+        const float m_half = s * (1.0f / 64);
+        float m2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 64; ++j) { const float dv = v[j] - m_half; m2 = fmaf(dv, dv, m2); }
+        float2* ex2 = reinterpret_cast<float2*>(exch) + (g & 1) * 256;
+        ex2[half * 128 + r] = make_float2(m_half, m2);
         if (!h2_group_sync(&pair_bar[q4], pair_uses, lane, p.err, 37)) { ok = false; break; }
-        const float mu = (s + exch[(half ^ 1) * 128 + r]) * (1.0f / H2_D);
-        float var = 0.f;
+        const float2 other = ex2[(half ^ 1) * 128 + r];
+        const float mu = 0.5f * (m_half + other.x);
+        const float dm = m_half - mu;
+        const float rstd = rsqrtf((m2 + other.y + 128.0f * dm * dm) * (1.0f / H2_D) + p.ln_eps);
 #pragma unroll
-        for (int j = 0; j < 64; ++j) { v[j] -= mu; var = fmaf(v[j], v[j], var); }
-        exch[256 + half * 128 + r] = var;
-        if (!h2_group_sync(&pair_bar[q4], pair_uses, lane, p.err, 39)) { ok = false; break; }
-        const float rstd = rsqrtf((var + exch[256 + (half ^ 1) * 128 + r]) * (1.0f / H2_D) + p.ln_eps);
-#pragma unroll
-        for (int j = 0; j < 64; ++j) v[j] *= rstd;
+        for (int j = 0; j < 64; ++j) v[j] = (v[j] - mu) * rstd;
       }
       if (valid) {
         uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * H2_D + half * 64);
