@@ -89,33 +89,57 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
 
 // Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
 //   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
-// grid (B, H * ell / MERGE_ROWS): a block of d threads walks MERGE_ROWS rows of one user.  A user without history gets
-// zeros; a user with a single chunk was already written by the attention kernel (its blocks return at once).
+// grid (B, H * ell / MERGE_ROWS), 128 threads: each warp takes rows of the block's MERGE_ROWS, a lane four consecutive
+// columns at a time (128-bit reads of the partial accumulators, four chunks in flight).  d is a multiple of 8.  A user
+// without history gets zeros; a user with a single chunk was already written by the attention kernel (its blocks
+// return at once).
 constexpr int MERGE_ROWS = 8;
-__global__ void k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H,
-                                       const float* __restrict__ part_m, const float* __restrict__ part_s,
-                                       const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
+__global__ void __launch_bounds__(128)
+k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H, const float* __restrict__ part_m,
+                       const float* __restrict__ part_s, const float* __restrict__ part_acc,
+                       __nv_bfloat16* __restrict__ Ohat) {
   const int HL = H * ell;
   const int u = blockIdx.x;
   const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
   if (c1 - c0 == 1) return;
-  const int i = threadIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int row_end = min(HL, ((int)blockIdx.y + 1) * MERGE_ROWS);
-  for (int row = blockIdx.y * MERGE_ROWS; row < row_end; ++row) {
+  for (int row = blockIdx.y * MERGE_ROWS + warp; row < row_end; row += 4) {
     const int h = row / ell, l = row % ell;
-    float out = 0.f;
-    if (c1 > c0) {
-      float M = -INFINITY;
-      for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
-      float S = 0.f, O = 0.f;
-      for (int c = c0; c < c1; ++c) {
-        const float w = exp2f(part_m[(int64_t)c * HL + row] - M);
-        S = fmaf(part_s[(int64_t)c * HL + row], w, S);
-        O = fmaf(part_acc[((int64_t)c * HL + row) * d + i], w, O);
+    __nv_bfloat16* dst = Ohat + ((int64_t)u * ell + l) * (H * d) + h * d;
+    float M = -INFINITY;
+    for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
+    float S = 0.f;
+    for (int c = c0; c < c1; ++c) S = fmaf(part_s[(int64_t)c * HL + row], exp2f(part_m[(int64_t)c * HL + row] - M), S);
+    const float inv = c1 > c0 ? 1.0f / S : 0.f;
+    for (int i = lane * 4; i < d; i += 128) {
+      float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+      int c = c0;
+      for (; c + 4 <= c1; c += 4) {
+        float4 a[4];
+        float w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          a[k] = *reinterpret_cast<const float4*>(part_acc + ((int64_t)(c + k) * HL + row) * d + i);
+          w[k] = exp2f(part_m[(int64_t)(c + k) * HL + row] - M);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          O.x = fmaf(a[k].x, w[k], O.x); O.y = fmaf(a[k].y, w[k], O.y);
+          O.z = fmaf(a[k].z, w[k], O.z); O.w = fmaf(a[k].w, w[k], O.w);
+        }
       }
-      out = O / S;
+      for (; c < c1; ++c) {
+        const float4 a = *reinterpret_cast<const float4*>(part_acc + ((int64_t)c * HL + row) * d + i);
+        const float w = exp2f(part_m[(int64_t)c * HL + row] - M);
+        O.x = fmaf(a.x, w, O.x); O.y = fmaf(a.y, w, O.y); O.z = fmaf(a.z, w, O.z); O.w = fmaf(a.w, w, O.w);
+      }
+      __nv_bfloat162 lo = __floats2bfloat162_rn(O.x * inv, O.y * inv), hi = __floats2bfloat162_rn(O.z * inv, O.w * inv);
+      uint2 o;
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(dst + i) = o;
     }
-    Ohat[((int64_t)u * ell + l) * (H * d) + h * d + i] = __float2bfloat16_rn(out);
   }
 }
 
@@ -124,7 +148,7 @@ lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int e
   if (B == 0) return LIME_OK;
   ProfScope _p("k_link_attn_merge_norm", st);
   const dim3 grid((unsigned)B, (unsigned)((H * ell + MERGE_ROWS - 1) / MERGE_ROWS));
-  k_link_attn_merge_norm<<<grid, d, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  k_link_attn_merge_norm<<<grid, 128, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }
