@@ -160,11 +160,11 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample(wl, inp, users, budget_s=None):
+def oracle_sample(wl, inp, users, budget_s=None, phi="softmax"):
     """Time the fp64 oracle (as it stands) on `users` of the batch: gather + encode + precompute + score."""
     from oracle import lime_oracle as O
     from tests import lime_helpers as Hh
-    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    cfg, layers = Hh.oracle_config(wl, phi=O.SILU if phi == "silu" else O.SOFTMAX), Hh.oracle_layers(inp, wl)
     table64_rows = {}
     links64 = synth.storage_to_f64(inp["links"], wl.dtype)
     off = O.lengths_to_offsets(inp["lengths"])
@@ -205,14 +205,14 @@ def run_reference(args, wl):
     if rank != 0:
         return
     inp = synth.make_inputs(wl, seed=0)
-    _, t_user = oracle_sample(wl, inp, range(1))          # calibrates the per-step sample; also the first warm-up
+    _, t_user = oracle_sample(wl, inp, range(1), phi=args.phi)          # calibrates the per-step sample; also the first warm-up
     users_per_step = 2 if (wl.B >= 2 and 2 * t_user * args.steps < 120.0) else 1
     for _ in range(max(0, args.warmup - 1)):
-        oracle_sample(wl, inp, range(1))
+        oracle_sample(wl, inp, range(1), phi=args.phi)
     times = []
     for s in range(args.steps):
         users = [(s * users_per_step + u) % wl.B for u in range(users_per_step)]
-        _, dt = oracle_sample(wl, inp, users)
+        _, dt = oracle_sample(wl, inp, users, phi=args.phi)
         times.append(dt)
     total = sum(times)
     value = users_per_step * wl.C * args.steps / total
@@ -283,7 +283,8 @@ def run_ours(args, wl):
     # a fixed per-GPU batch (weak scaling, no collective on the data path)
     inp = synth.make_inputs(wl, seed=rank)
     dt = Bd.LIME_F32 if wl.dtype == synth.F32 else Bd.LIME_BF16
-    lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff)
+    lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff,
+                   phi=Bd.LIME_PHI_SILU if args.phi == "silu" else Bd.LIME_PHI_SOFTMAX)
     table = Bd.to_device(inp["table"], wl.dtype, dev)
     links = Bd.to_device(inp["links"], wl.dtype, dev)
     wts = {k: Bd.to_device(inp[k], wl.dtype, dev) for k in ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")}
@@ -555,14 +556,14 @@ def run_ours(args, wl):
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget)
+            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget, phi=args.phi)
             cpu = {"value": n_done * wl.C / dt_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                    "sample": f"first {n_done} users x {wl.C} candidates of the same workload, {dt_s:.1f} s "
                              "(gather+encode+precompute+score, fp64 numpy)"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "p50_batch_latency_ms": step_ms[len(step_ms) // 2],
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == synth.BF16 else "f32",
-                "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args)), "clocks": clocks,
+                "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args), phi=args.phi), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps, "host_issue_ms_per_step": 1e3 * t_issue / args.steps,
                         "score_by_id_alone_ms": score_by_id_ms,
@@ -594,6 +595,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", default="", choices=["", "C", "N"], help="one line per point of the candidate / history sweep")
+    ap.add_argument("--phi", default="softmax", choices=["softmax", "silu"],
+                    help="attention activation of the XOR layers: online softmax (default) or SiLU(s) / n (Algorithms 1-2)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying CUDA graphs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

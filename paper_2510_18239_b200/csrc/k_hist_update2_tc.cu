@@ -42,6 +42,7 @@ struct HistUpdate2Params {
   const int32_t* off;            // [B+1]
   const int32_t* tile_start;     // [B+1] prefix of per-user tile counts (tile = 128 tokens)
   int B, HL, NG, shared, out_ln; // NG = HL / 128 groups
+  int silu;                      // 1: P = SiLU(scores) / ell (Algorithm 2) instead of the per-head softmax
   float ln_eps;
   int* err;
 };
@@ -338,15 +339,23 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             if (LN) v[cc] = (v[cc] - mu_r * ck_s[cc]) * rstd_r;
             mx = fmaxf(mx, v[cc]);
           }
-          float s0 = 0.f, s1 = 0.f;
+          float inv;
+          if (p.silu) {
+            // SiLU(s) / ell: every history query attends to the ell links of the head (Algorithm 1)
 #pragma unroll
-          for (int j = 0; j < ELL; j += 2) {
-            v[h * ELL + j] = h2_ex2(v[h * ELL + j] - mx);
-            v[h * ELL + j + 1] = h2_ex2(v[h * ELL + j + 1] - mx);
-            s0 += v[h * ELL + j];
-            s1 += v[h * ELL + j + 1];
+            for (int j = 0; j < ELL; ++j) { const float hx = 0.5f * v[h * ELL + j]; v[h * ELL + j] = fmaf(hx, h2_tanh(hx), hx); }
+            inv = 1.0f / ELL;
+          } else {
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < ELL; j += 2) {
+              v[h * ELL + j] = h2_ex2(v[h * ELL + j] - mx);
+              v[h * ELL + j + 1] = h2_ex2(v[h * ELL + j + 1] - mx);
+              s0 += v[h * ELL + j];
+              s1 += v[h * ELL + j + 1];
+            }
+            inv = __fdividef(1.f, s0 + s1);
           }
-          const float inv = __fdividef(1.f, s0 + s1);
 #pragma unroll
           for (int j = 0; j < ELL; ++j) v[h * ELL + j] *= inv;
         }
@@ -455,7 +464,7 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 bool hist_update2_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp) {
   const int HL = H * ell;
   return dtype == LIME_BF16 && d == H2_D && f == H2_F && HL % 128 == 0 && HL >= 256 && HL <= 512 && (ell == 32 || ell == 64) &&
-         phi == LIME_PHI_SOFTMAX && gated_mlp != 0;
+         (phi == LIME_PHI_SOFTMAX || phi == LIME_PHI_SILU) && gated_mlp != 0;
 }
 
 template <int ELL>
@@ -470,7 +479,7 @@ static lime_status launch_hu2(const HistUpdateArgs& a, int HL, cudaStream_t st) 
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   HistUpdate2Params p;
   p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.HL = HL;
-  p.NG = HL / 128; p.shared = a.shared; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
+  p.NG = HL / 128; p.shared = a.shared; p.silu = a.silu; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
   int grid = a.n_tile_upper < kSMs ? a.n_tile_upper : kSMs;
   if (grid < 1) return LIME_OK;
   static bool smem_ln[kMaxDeviceOrdinals] = {}, smem_plain[kMaxDeviceOrdinals] = {};

@@ -56,6 +56,7 @@ struct HistUpdateParams {
   const int32_t* off;            // [B+1]
   const int32_t* tile_start;     // [B+1] prefix of per-user tile counts (tile = 128 tokens)
   int B, ell, shared, out_ln;
+  int silu;                      // 1: P = SiLU(scores) / ell (Algorithm 2) instead of the per-head softmax
   float ln_eps;
   int* err;
 };
@@ -392,15 +393,23 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           if (LN) v[c] = (v[c] - mu_r * ck_s[c]) * rstd_r;
           mx = fmaxf(mx, v[c]);
         }
-        float s0 = 0.f, s1 = 0.f;
+        float inv;
+        if (p.silu) {
+          // SiLU(s) / ell: every history query attends to the ell links of the head (Algorithm 1)
 #pragma unroll
-        for (int j = 0; j < ELL; j += 2) {
-          v[h * ELL + j] = hu_ex2(v[h * ELL + j] - mx);
-          v[h * ELL + j + 1] = hu_ex2(v[h * ELL + j + 1] - mx);
-          s0 += v[h * ELL + j];
-          s1 += v[h * ELL + j + 1];
+          for (int j = 0; j < ELL; ++j) { const float hx = 0.5f * v[h * ELL + j]; v[h * ELL + j] = fmaf(hx, tanh_approx(hx), hx); }
+          inv = 1.0f / ELL;
+        } else {
+          float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+          for (int j = 0; j < ELL; j += 2) {
+            v[h * ELL + j] = hu_ex2(v[h * ELL + j] - mx);
+            v[h * ELL + j + 1] = hu_ex2(v[h * ELL + j + 1] - mx);
+            s0 += v[h * ELL + j];
+            s1 += v[h * ELL + j + 1];
+          }
+          inv = __fdividef(1.f, s0 + s1);
         }
-        const float inv = __fdividef(1.f, s0 + s1);
 #pragma unroll
         for (int j = 0; j < ELL; ++j) v[h * ELL + j] *= inv;
       }
@@ -537,7 +546,7 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
 
 bool hist_update_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp) {
   return dtype == LIME_BF16 && d == HU_D && f == HU_F && H * ell == HU_HL && (ell == 16 || ell == 32) &&
-         phi == LIME_PHI_SOFTMAX && gated_mlp != 0;
+         (phi == LIME_PHI_SOFTMAX || phi == LIME_PHI_SILU) && gated_mlp != 0;
 }
 
 template <int ELL>
@@ -551,7 +560,7 @@ static lime_status launch_hu(const HistUpdateArgs& a, cudaStream_t st) {
       !make_tmap_bf16_sw128(&tmWo, a.WoT, HU_D, HU_F, HU_F, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   HistUpdateParams p;
-  p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.stats_in = a.ln ? a.stats_in : nullptr; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.ell = ELL;
+  p.out = (__nv_bfloat16*)a.hist_out; p.cK = a.cK; p.stats_in = a.ln ? a.stats_in : nullptr; p.off = a.off; p.tile_start = a.tile_start; p.B = a.B; p.silu = a.silu; p.ell = ELL;
   p.shared = a.shared; p.out_ln = a.out_ln; p.ln_eps = a.ln_eps; p.err = a.err;
   int grid = a.n_tile_upper < kSMs ? a.n_tile_upper : kSMs;
   if (grid < 1) return LIME_OK;

@@ -60,6 +60,7 @@ struct LinkAttnParams {
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
   const int32_t* chunk_user;      // [chunk items] user of each (user, chunk) item
   int B, chunk, shared, ell, H;
+  int silu;                       // attention activation: 0 softmax (online, log2 domain), 1 SiLU(s) / N(U) (Algorithm 2)
   int HL, RB;                     // stacked (head, link) rows in all, and 128-row blocks of them (one per work item)
   float ln_eps;
   float *part_m, *part_s, *part_acc;   // [items x HL], [items x HL], [items x HL x d]
@@ -72,6 +73,13 @@ __device__ __forceinline__ uint32_t la_chunk_addr(uint32_t r, uint32_t c) { retu
 __device__ __forceinline__ uint32_t la_pack(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+// SiLU(x) = x * sigmoid(x) = x/2 * (1 + tanh(x/2)): one SFU operation
+__device__ __forceinline__ float la_silu(float x) {
+  const float hx = 0.5f * x;
+  float th;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hx));
+  return fmaf(hx, th, hx);
 }
 __device__ __forceinline__ float la_ex2(float x) {
   float y;
@@ -103,9 +111,10 @@ __device__ __forceinline__ float la_pass1(float (&v)[LA_COLS], const float2* __r
   return mx;
 }
 
-// Pass 2: p = 2^(s - m_ref), P' = p * rstd as bf16 into the A-operand buffer (K-major over the tile's tokens,
-// 128-byte swizzle); returns the sums of p and of P' * mu through l_sum / mean_corr.
-template <bool LN, bool MASK>
+// Pass 2: p = 2^(s - m_ref) (softmax) or SiLU(s) (SILU: no reference maximum, no row sum), P' = p * rstd as bf16 into
+// the A-operand buffer (K-major over the tile's tokens, 128-byte swizzle); returns the sums of p and of P' * mu
+// through l_sum / mean_corr.
+template <bool LN, bool MASK, bool SILU>
 __device__ __forceinline__ void la_pass2(const float (&v)[LA_COLS], const float2* __restrict__ st, float m_ref, int col0, int nvalid,
                                          uint8_t* prow_base, uint32_t r, uint32_t chunk0, float& l_sum, float& mean_corr) {
   float ls0 = 0.f, ls1 = 0.f, mc0 = 0.f, mc1 = 0.f;
@@ -115,7 +124,7 @@ __device__ __forceinline__ void la_pass2(const float (&v)[LA_COLS], const float2
 #pragma unroll
     for (int j2 = 0; j2 < 4; ++j2) {
       const int j = c8 * 8 + 2 * j2;
-      float e0 = la_ex2(v[j] - m_ref), e1 = la_ex2(v[j + 1] - m_ref);
+      float e0 = SILU ? la_silu(v[j]) : la_ex2(v[j] - m_ref), e1 = SILU ? la_silu(v[j + 1]) : la_ex2(v[j + 1] - m_ref);
       if (MASK) {
         if (col0 + j >= nvalid) e0 = 0.f;
         if (col0 + j + 1 >= nvalid) e1 = 0.f;
@@ -404,6 +413,19 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         tmem_ld_32x32(lane_addr + COL_S + pb * 128 + col0, v);
         tmem_wait_ld();
         float mx = nvalid == LA_TILE ? la_pass1<LN, false>(v, st, cq, col0, nvalid) : la_pass1<LN, true>(v, st, cq, col0, nvalid);
+        if (p.silu) {
+          // SiLU(s) / N(U) needs neither a reference maximum nor row sums: one pass, no exchange between the row's threads
+          if (g >= LA_PBUFS && !mbar_wait(&p_free[g % LA_PBUFS], (uint32_t)((g - LA_PBUFS) / LA_PBUFS) & 1u, p.err, 65)) { ok = false; break; }
+          uint8_t* pbuf = smem + LA_OFF_P + (g % LA_PBUFS) * LA_P_BUF + (col0 >> 6) * LA_SUB;
+          const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
+          if (nvalid == LA_TILE) la_pass2<LN, false, true>(v, st, 0.f, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
+          else la_pass2<LN, true, true>(v, st, 0.f, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
+          tc_fence_before();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(p_ready);
+          continue;
+        }
         exch_max[(pb * LA_PARTS + part) * 128 + r] = mx;
         if (!la_group_sync(&row_bar[q], row_uses, lane, p.err, 67)) { ok = false; break; }
 #pragma unroll
@@ -434,8 +456,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         // pass 2: P' -> smem; K index = token column, so columns col0.. live in K-block col0 / 64, chunk (col0 % 64) / 8..
         uint8_t* pbuf = smem + LA_OFF_P + (g % LA_PBUFS) * LA_P_BUF + (col0 >> 6) * LA_SUB;
         const uint32_t chunk0 = (uint32_t)(col0 & 63) >> 3;
-        if (nvalid == LA_TILE) la_pass2<LN, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
-        else la_pass2<LN, true>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
+        if (nvalid == LA_TILE) la_pass2<LN, false, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
+        else la_pass2<LN, true, false>(v, st, m_ref, col0, nvalid, pbuf, r, chunk0, l_sum, mean_corr);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
@@ -452,6 +474,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       float l_tot = 0.f, c_tot = 0.f;
 #pragma unroll
       for (int i = 0; i < LA_PARTS; ++i) { l_tot += exch_sum[i * 128 + r]; c_tot += exch_mean[i * 128 + r]; }
+      // SiLU mode normalises by the number of keys (Algorithm 1): this chunk's tokens, summed over the chunks by the merge
+      if (p.silu) l_tot = (float)(tok1 - tok0);
       float a[LA_COLS];
       tmem_ld_32x32(lane_addr + COL_O + col0, a);
       tmem_wait_ld();
@@ -492,7 +516,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         for (int j = 0; j < LA_COLS; j += 4)
           dst[j / 4] = make_float4(a[j] - c_tot, a[j + 1] - c_tot, a[j + 2] - c_tot, a[j + 3] - c_tot);
         if (part == 0) {
-          p.part_m[prow] = m_ref;        // log2 domain
+          p.part_m[prow] = p.silu ? 0.f : m_ref;        // log2 domain; equal weights for the chunks in SiLU mode
           p.part_s[prow] = l_tot;
         }
       }
@@ -508,7 +532,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 }
 
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi) {
-  return dtype == LIME_BF16 && d == LA_D && (H * ell) % 128 == 0 && H * ell <= 512 && phi == LIME_PHI_SOFTMAX;
+  return dtype == LIME_BF16 && d == LA_D && (H * ell) % 128 == 0 && H * ell <= 512 &&
+         (phi == LIME_PHI_SOFTMAX || phi == LIME_PHI_SILU);
 }
 
 lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
@@ -519,7 +544,7 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
       !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), LA_D, LA_D, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   LinkAttnParams p;
-  p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
+  p.cQ = a.cQ; p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.silu = a.silu; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.ln_eps = a.ln_eps; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.stats_out = a.ln ? a.stats_out : nullptr; p.err = a.err;
   int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;

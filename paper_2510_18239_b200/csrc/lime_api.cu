@@ -139,7 +139,7 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
   LinkAttnArgs la{};
   la.hist = hist_in; la.total = total; la.Q2 = ops.Q2; la.cQ = ops.cQ; la.off = off; la.chunk_start = w.chunk_start; la.chunk_user = w.chunk_user; la.B = B;
   la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = ops.shared;
-  la.ln = hist_ln; la.ln_eps = c->ln_eps; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
+  la.ln = hist_ln; la.ln_eps = c->ln_eps; la.silu = g.phi == LIME_PHI_SILU; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
   la.err = c->dev_err;
   // the attention kernel forms the LayerNorm statistics of every history row anyway; the history update reuses them
   const bool one_block_update = hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
@@ -158,7 +158,7 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
     hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = ops.K2; hu.G2t = ops.G2t; hu.U2t = ops.U2t;
     hu.cK = ops.cK; hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B;
     hu.n_tile_upper = w.n_tile_upper; hu.ell = g.ell; hu.shared = ops.shared; hu.ln = hist_ln; hu.ln_eps = c->ln_eps;
-    hu.out_ln = out_ln; hu.err = c->dev_err;
+    hu.out_ln = out_ln; hu.silu = g.phi == LIME_PHI_SILU; hu.err = c->dev_err;
     hu.stats_in = pass_stats ? w.row_stats : nullptr;
     if (one_block_update) s = launch_hist_update_tc(hu, st);
     else s = launch_hist_update2_tc(hu, g.H, st);
@@ -446,7 +446,8 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
       if (!c->WpostT[j]) LIME_CUDA(cudaMalloc(&c->WpostT[j], (size_t)2 * c->d_ff * g.H * g.d * 2));
       if ((s = launch_transpose_bf16(w->Wo[j], c->d_ff, g.d, c->WoT[j], st)) != LIME_OK) return s;
       if ((s = launch_fold_weights(w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], g.d, g.H, c->d_ff,
-                                   c->attn_scale * 1.4426950408889634f /* scores leave the fold in the log2 domain */,
+                                   // softmax: scores leave the fold scaled and in the log2 domain; SiLU(s) takes the raw scores
+                                   g.phi == LIME_PHI_SILU ? 1.0f : c->attn_scale * 1.4426950408889634f,
                                    c->WprepT[j], c->WpostT[j], st)) != LIME_OK)
         return s;
     }

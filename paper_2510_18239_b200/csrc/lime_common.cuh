@@ -212,6 +212,7 @@ struct LinkAttnArgs {
   const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
   const int32_t* chunk_user;                // [items] user of each (user, chunk) work item
   int ell, d, H, shared, ln; float ln_eps;
+  int silu;                                 // 1: SiLU(s) / N(U) instead of softmax (Algorithm 2)
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
   void* Ohat;                               // [B*ell x H*d] bf16: rows of users whose history is one chunk
   float2* stats_out;                        // nullable, ln only: {rstd, mean} of every history row, for the history update
@@ -226,6 +227,7 @@ struct HistUpdateArgs {
   const int32_t* off; const int32_t* tile_start; int B, n_tile_upper;
   int ell, shared, ln; float ln_eps;    // ln: apply LayerNorm to the rows read (0 when they were stored normalised)
   int out_ln;                           // 1: store LayerNorm(S') instead of S'
+  int silu;                             // 1: SiLU(s) / ell instead of the per-head softmax (Algorithm 2)
   const float2* stats_in;               // nullable, ln only: {rstd, mean} of every row read, as left by the attention kernel
   int* err;
 };

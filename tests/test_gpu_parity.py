@@ -309,6 +309,72 @@ def test_xor_layer_tensor_core_path(ell, H, lengths, shared_links):
             assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
 
 
+@pytest.mark.parametrize("ell,H", [(32, 4), (16, 8), (64, 4), (32, 8)])
+@pytest.mark.parametrize("lengths", [[127, 128, 129], [0, 300, 5, 0, 1000, 2100]])
+@pytest.mark.parametrize("shared_links", [True, False])
+def test_xor_layer_tensor_core_path_silu(ell, H, lengths, shared_links):
+    """The SiLU form of the XOR attention (Algorithms 1-2: SiLU(s) divided by the size of the attended partition, the
+    paper's choice for stacked layers) on the shapes the tensor-core kernels serve; ragged histories, one of them long
+    enough to span several chunks so that the per-chunk partials are summed."""
+    Bd = _lib()
+    B = len(lengths)
+    wl = small(synth.BF16, B=B, n_min=0, n_max=1, d=128, H=H, ell=ell, n_layers=1, V=3000, table_std=0.05)
+    inp = synth.make_inputs(wl, seed=ell + B)
+    inp["lengths"] = np.asarray(lengths, dtype=np.int32)
+    total = int(sum(lengths))
+    inp["hist_ids"] = synth.zipf_ids(3, "h", total, wl.V, 1.1)
+    dev = Hh.DeviceBatch(wl, inp, phi=Bd.LIME_PHI_SILU)
+    L = dev.lime
+    off = L.lengths_to_offsets(dev.lengths)
+    hist = L.gather_history(dev.table, dev.hist_ids)
+    if shared_links:
+        links_np = synth.storage_to_f64(inp["links"], wl.dtype)[None].repeat(B, axis=0)
+        links32 = dev.links.float().contiguous()
+    else:
+        links_np = np.random.default_rng(9).normal(size=(B, ell, wl.d)).astype(np.float32).astype(np.float64)
+        links32 = torch.from_numpy(links_np.astype(np.float32)).cuda()
+    hist_out = torch.zeros_like(hist)
+    links_out = torch.empty((B, ell, wl.d), dtype=torch.float32, device="cuda")
+    Bd.lime_xor_layer(L.ctx, 0, hist, off, B, links32, shared_links, hist_out, links_out, L.workspace(B, total))
+    assert Bd.lime_device_status(L.ctx) == 0
+    cfg = Hh.oracle_config(wl, phi=O.SILU)
+    lw = Hh.oracle_layers(inp, wl)[0]
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    offh = O.lengths_to_offsets(lengths)
+    for b in range(B):
+        E = O.gather_history(table64, inp["hist_ids"][offh[b]:offh[b + 1]])
+        S_next, T_next = O.xor_layer(E, links_np[b], lw, cfg)
+        assert np.abs(Hh.to_f64(links_out[b]) - T_next).max() <= 4e-2 * max(1.0, np.abs(T_next).max()), b
+        # unscaled scores through SiLU are not bounded like softmax weights, so single elements err more; the mean
+        # error must still be a fraction of a per cent of the spread (a wrong divisor or a dropped chunk is not)
+        assert np.abs(Hh.to_f64(links_out[b]) - T_next).mean() <= 1e-2 * max(T_next.std(), 1e-6) + 1e-5, b
+        if lengths[b]:
+            got = Hh.to_f64(hist_out[offh[b]:offh[b + 1]])
+            assert np.abs(got - S_next).max() <= 4e-2 * max(1.0, np.abs(S_next).max()), (b, np.abs(got - S_next).max())
+            assert np.abs(got - S_next).mean() <= 1e-2 * max(S_next.std(), 1e-6) + 1e-5, (b, np.abs(got - S_next).mean())
+
+
+def test_config2_bf16_baseline_silu_sampled():
+    # the bench workload with the SiLU form of the attention, through the fused lookup + LayerNorm as bench.py runs it
+    wl = synth.named_workloads()["bf16_baseline"].replace(B=64)
+    inp = synth.make_inputs(wl, seed=3)
+    Bd = _lib()
+    out = Hh.DeviceBatch(wl, inp, phi=Bd.LIME_PHI_SILU).run(normalized=True)
+    torch.cuda.synchronize()
+    cfg, layers = Hh.oracle_config(wl, phi=O.SILU), Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(inp["lengths"])
+    r = np.random.default_rng(3)
+    got_all, want_all = [], []
+    for b in [0, 31, 63]:
+        rows = np.sort(r.choice(wl.C, size=64, replace=False))
+        lg, _, _ = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg, cand_rows=rows)
+        got_all.append(Hh.to_f64(out["logits"][b * wl.C:(b + 1) * wl.C])[rows])
+        want_all.append(lg)
+    _check_logits(np.concatenate(got_all), np.concatenate(want_all), wl.dtype)
+
+
 @pytest.mark.parametrize("ell,H", [(32, 4), (64, 4)])
 def test_xor_layer_tensor_core_path_many_users(ell, H):
     """More users than the kernels stage offsets for in shared memory (1024): the work lists are then read from global
