@@ -585,6 +585,52 @@ def _sampled_parity_any_dtype(wl, normalized):
     _check_logits(np.concatenate(got_all), np.concatenate(want_all), wl.dtype)
 
 
+@pytest.mark.parametrize("seed", list(range(11, 41)))
+def test_random_ragged_batches_on_the_tensor_core_path(seed):
+    """Randomly drawn batch shapes (users, ragged lengths around tile and chunk boundaries, empty histories, layers,
+    heads x links, softmax or SiLU): both call sequences (raw rows, rows normalised by the lookup) must agree with each
+    other, and sampled users with the oracle."""
+    Bd = _lib()
+    r = np.random.default_rng(seed)
+    ell, H = [(32, 4), (16, 8), (64, 4), (32, 8), (64, 8)][seed % 5]
+    B = int(r.integers(1, 200))
+    kinds = r.integers(0, 5, size=B)
+    lengths = np.where(kinds == 0, 0,
+              np.where(kinds == 1, r.integers(1, 128, size=B),
+              np.where(kinds == 2, 128 * r.integers(1, 6, size=B) + r.integers(-1, 2, size=B),
+              np.where(kinds == 3, 512 * r.integers(1, 4, size=B) + r.integers(-1, 2, size=B),
+                       r.integers(1, 3000, size=B))))).astype(np.int32)
+    n_layers = int(r.integers(1, 4))
+    silu = bool(seed % 2)
+    wl = small(synth.BF16, B=B, n_min=0, n_max=1, d=128, H=H, ell=ell, n_layers=n_layers, V=5000, C=96, table_std=0.05)
+    inp = synth.make_inputs(wl, seed=seed)
+    inp["lengths"] = lengths
+    inp["hist_ids"] = synth.zipf_ids(seed, "h", int(lengths.sum()), wl.V, 1.1)
+    phi = Bd.LIME_PHI_SILU if silu else Bd.LIME_PHI_SOFTMAX
+    raw = Hh.DeviceBatch(wl, inp, phi=phi).run()
+    nrm = Hh.DeviceBatch(wl, inp, phi=phi).run(normalized=True)
+    a, b = Hh.to_f64(raw["logits"]), Hh.to_f64(nrm["logits"])
+    assert np.isfinite(a).all() and np.isfinite(b).all()
+    spread = max(a.std(), 1e-6)
+    assert np.abs(a - b).max() <= 2 * TOL_BF16 * max(1.0, np.abs(a).max())
+    assert np.abs(a - b).mean() <= 2e-2 * spread + 1e-5
+    cfg = Hh.oracle_config(wl, phi=O.SILU if silu else O.SOFTMAX)
+    layers = Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], wl.dtype)
+    links64 = synth.storage_to_f64(inp["links"], wl.dtype)
+    off = O.lengths_to_offsets(lengths)
+    users = sorted({0, B - 1, int(np.argmax(lengths)), int(np.argmin(lengths))})
+    for out in (raw, nrm):
+        got_all, want_all = [], []
+        for u in users:
+            lg, _, _ = Hh.oracle_user(inp, wl, u, off, table64, links64, layers, cfg)
+            got_all.append(Hh.to_f64(out["logits"][u * wl.C:(u + 1) * wl.C]))
+            want_all.append(lg)
+        got, want = np.concatenate(got_all), np.concatenate(want_all)
+        assert np.abs(got - want).max() <= TOL_BF16 * max(1.0, np.abs(want).max())
+        assert np.abs(got - want).mean() <= 2e-2 * max(want.std(), 1e-6) + 1e-5
+
+
 def test_config3_candidate_sweep_sampled():
     wl = synth.named_workloads()["candidate_sweep"].replace(C=4096)
     _sampled_parity(wl, seed=0, users=[0, 63])
