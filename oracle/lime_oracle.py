@@ -81,6 +81,11 @@ class OracleConfig:
     def c_scale(self) -> float:
         return self.cand_scale if self.cand_scale is not None else float(self.d) ** -0.5
 
+    @property
+    def c_scale_heads(self) -> float:
+        """Scale of the per-head candidate->link scores (Eq. 1 applied to Eq. 4 head by head): 1/sqrt(d_h)."""
+        return self.cand_scale if self.cand_scale is not None else float(self.d_h) ** -0.5
+
 
 # --------------------------------------------------------------------------- #
 # ragged bookkeeping and the embedding lookup (Sec. 3, history of N(U) items per user)
@@ -276,16 +281,55 @@ def score_candidates(W: np.ndarray, LS: np.ndarray, T: np.ndarray) -> np.ndarray
     return out
 
 
+# Eq. 4 with Eq. 1 taken literally, MHA(T, L, L^P) head by head: every head h has its own weight row
+# softmax_l(<(T W_Q)_h, (L W_K)_h> / sqrt(d_h)) and mixes only its d_h columns of the link states.
+def precompute_candidate_links_heads(T: np.ndarray, L: np.ndarray, cfg: OracleConfig,
+                                     Wq_c: Optional[np.ndarray] = None, Wk_c: Optional[np.ndarray] = None) -> np.ndarray:
+    """User-independent weights [M x H x l]: row (c, h) is the softmax over the l links of head h's scores."""
+    Tq = T if Wq_c is None else T @ Wq_c
+    Lk = L if Wk_c is None else L @ Wk_c
+    M, ell, H, d_h = T.shape[0], L.shape[0], cfg.H, cfg.d_h
+    W = np.zeros((M, H, ell), dtype=np.float64)
+    for h in range(H):
+        sl = slice(h * d_h, (h + 1) * d_h)
+        W[:, h, :] = softmax_rows((Tq[:, sl] @ Lk[:, sl].T) * cfg.c_scale_heads)
+    return W
+
+
+def candidate_outputs_heads(W: np.ndarray, LS: np.ndarray, cfg: OracleConfig) -> np.ndarray:
+    """O[c, head h's columns] = sum_l W[c, h, l] LS[l, head h's columns]."""
+    H, d_h = cfg.H, cfg.d_h
+    O = np.zeros((W.shape[0], LS.shape[1]), dtype=np.float64)
+    for h in range(H):
+        sl = slice(h * d_h, (h + 1) * d_h)
+        O[:, sl] = W[:, h, :] @ LS[:, sl]
+    return O
+
+
+def score_candidates_heads(W: np.ndarray, LS: np.ndarray, T: np.ndarray, cfg: OracleConfig) -> np.ndarray:
+    """logit[c] = <O_c, T_c> with the per-head mix above."""
+    O = candidate_outputs_heads(W, LS, cfg)
+    out = np.empty(T.shape[0], dtype=np.float64)
+    for c in range(T.shape[0]):
+        out[c] = float(np.dot(O[c, :], T[c, :]))
+    return out
+
+
 # --------------------------------------------------------------------------- #
 # whole batch
 # --------------------------------------------------------------------------- #
 def run_user(E: np.ndarray, L: np.ndarray, layers, cfg: OracleConfig, T: np.ndarray,
              LC: Optional[np.ndarray] = None, W: Optional[np.ndarray] = None,
-             cand_w: Optional[Dict[str, np.ndarray]] = None):
-    """Encode one user and score that user's candidates. Returns (logits [C], link states [l x d], W [C x l])."""
+             cand_w: Optional[Dict[str, np.ndarray]] = None, cand_heads: bool = False):
+    """Encode one user and score that user's candidates. Returns (logits [C], link states [l x d], W [C x l]);
+    with cand_heads the candidate side runs head by head (W [C x H x l])."""
     cand_w = cand_w or {}
     LP, _ = encode_user(E, L if LC is None else LC, layers, cfg)
     LS = link_states(LP, cand_w.get("Wv_c"))
+    if cand_heads:
+        if W is None:
+            W = precompute_candidate_links_heads(T, L, cfg, cand_w.get("Wq_c"), cand_w.get("Wk_c"))
+        return score_candidates_heads(W, LS, T, cfg), LS, W
     if W is None:
         W = precompute_candidate_links(T, L, cfg, cand_w.get("Wq_c"), cand_w.get("Wk_c"))
     return score_candidates(W, LS, T), LS, W

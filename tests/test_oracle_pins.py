@@ -291,6 +291,51 @@ def test_scoring_invariants():
     assert np.allclose(base, bf, atol=1e-13)
 
 
+def test_per_head_candidate_side_is_multi_head_attention():
+    """Eq. 1 applied to Eq. 4 head by head: the decoupled form (weights cached per head, then the per-head mix and the
+    dot with the candidate) must equal torch's multi-head attention of the candidates over the links with the link
+    states as values, and scalar loops; H = 1 must be the single-row form."""
+    r = rng(41)
+    C, ell, d, H = 7, 5, 12, 3
+    T, L, LS = r.normal(size=(C, d)), r.normal(size=(ell, d)), r.normal(size=(ell, d))
+    Wq, Wk = r.normal(size=(d, d)), r.normal(size=(d, d))
+    cfg = core_cfg(d, H, ell)
+    W = O.precompute_candidate_links_heads(T, L, cfg, Wq, Wk)
+    assert W.shape == (C, H, ell) and np.allclose(W.sum(axis=2), 1.0, atol=1e-12)
+    out = O.candidate_outputs_heads(W, LS, cfg)
+    # library second opinion: scaled_dot_product_attention over the head-split tensors (scale 1/sqrt(d_h) by default)
+    tq = torch.from_numpy(T @ Wq).reshape(C, H, d // H).transpose(0, 1)
+    lk = torch.from_numpy(L @ Wk).reshape(ell, H, d // H).transpose(0, 1)
+    lv = torch.from_numpy(LS).reshape(ell, H, d // H).transpose(0, 1)
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, lk, lv).transpose(0, 1).reshape(C, d).numpy()
+    assert np.allclose(out, ref, atol=1e-12)
+    # scalar loops for one candidate and head
+    c, h, dh = 4, 2, d // H
+    tqn, lkn = T @ Wq, L @ Wk
+    sc = [sum(tqn[c, h * dh + k] * lkn[l, h * dh + k] for k in range(dh)) / math.sqrt(dh) for l in range(ell)]
+    z = sum(math.exp(v - max(sc)) for v in sc)
+    w = [math.exp(v - max(sc)) / z for v in sc]
+    assert np.allclose(W[c, h], w, atol=1e-12)
+    logits = O.score_candidates_heads(W, LS, T, cfg)
+    bf = [sum(W[cc, hh, l] * LS[l, hh * dh + k] * T[cc, hh * dh + k] for hh in range(H) for l in range(ell) for k in range(dh))
+          for cc in range(C)]
+    assert np.allclose(logits, bf, atol=1e-12)
+    # candidate permutation
+    p = r.permutation(C)
+    assert np.allclose(O.score_candidates_heads(W[p], LS, T[p], cfg), logits[p], atol=1e-14)
+    # one head: the single-row form (its default scale 1/sqrt(d) equals 1/sqrt(d_h) then)
+    cfg1 = core_cfg(d, 1, ell)
+    W1 = O.precompute_candidate_links_heads(T, L, cfg1, Wq, Wk)
+    assert np.allclose(W1[:, 0, :], O.precompute_candidate_links(T, L, cfg1, Wq, Wk), atol=1e-14)
+    assert np.allclose(O.score_candidates_heads(W1, LS, T, cfg1), O.score_candidates(W1[:, 0, :], LS, T), atol=1e-13)
+    # a head only sees its own columns: changing another head's columns of the links leaves its weights alone
+    L2 = L.copy()
+    L2[0, :dh] += 1.0
+    W2 = O.precompute_candidate_links_heads(T, L2, cfg, None, None)
+    W0 = O.precompute_candidate_links_heads(T, L, cfg, None, None)
+    assert np.allclose(W2[:, 1:, :], W0[:, 1:, :], atol=1e-14) and not np.allclose(W2[:, 0, :], W0[:, 0, :])
+
+
 def test_link_states_value_projection():
     r = rng(16)
     LP, Wv = r.normal(size=(3, 4)), r.normal(size=(4, 4))
