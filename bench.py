@@ -44,7 +44,7 @@ def peaks():
 
 
 # ----------------------------------------------------------------------------- algorithmic work per kernel and step
-def kernel_models(wl: synth.Workload, total_tokens: int):
+def kernel_models(wl: synth.Workload, total_tokens: int, cand_heads: int = 1):
     """name -> dict(bytes=, flops=) : algorithmic work of ALL launches of that kernel in one step.  Bytes are what
     the stage must move through HBM (inputs read once, outputs written once, scratch excluded); flops what it must
     compute (2 per multiply-add).  A kernel with both is bounded by whichever floor (bytes / HBM peak, flops /
@@ -57,11 +57,12 @@ def kernel_models(wl: synth.Workload, total_tokens: int):
     glu = 4.0 * d * f * (BL * n + N * (n - 1))
     down = 2.0 * d * f * (BL * n + N * (n - 1))
     return {
-        "k_score": dict(bytes=BC * (es * ell + es * d + 4.0)),
+        # cand_heads = H: one weight row per (candidate, head), i.e. H * ell weights per candidate
+        "k_score": dict(bytes=BC * (es * ell * cand_heads + es * d + 4.0)),
         # by id from the corpus caches: the same rows, fetched one by one, + the 4-byte id
-        "k_score_gather_tc": dict(bytes=BC * (es * ell + es * d + 8.0)),
+        "k_score_gather_tc": dict(bytes=BC * (es * ell * cand_heads + es * d + 8.0)),
         "k_gather": dict(bytes=N * (4.0 + 2 * es * d)),
-        "k_precompute": dict(bytes=BC * es * (d + ell)),
+        "k_precompute": dict(bytes=BC * es * (d + ell * cand_heads)),
         # fused tensor-core layer kernels: history rows read once per direction, written once by the update
         "k_link_attn_tc": dict(bytes=n * N * d * es, flops=n * 4.0 * HL * d * N, pipe="tensor"),
         "k_hist_update_tc": dict(bytes=(n - 1) * 2.0 * N * d * es, flops=(n - 1) * 2.0 * N * (HL * d + 2 * HL * f + f * d),
@@ -160,7 +161,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample(wl, inp, users, budget_s=None, phi="softmax"):
+def oracle_sample(wl, inp, users, budget_s=None, phi="softmax", cand_heads=False):
     """Time the fp64 oracle (as it stands) on `users` of the batch: gather + encode + precompute + score."""
     from oracle import lime_oracle as O
     from tests import lime_helpers as Hh
@@ -184,7 +185,7 @@ def oracle_sample(wl, inp, users, budget_s=None, phi="softmax"):
     tab = LazyTable()
     done, t0 = 0, time.perf_counter()
     for b in users:
-        Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg)
+        Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg, cand_heads=cand_heads)
         done += 1
         if budget_s is not None and time.perf_counter() - t0 > budget_s:
             break
@@ -205,14 +206,14 @@ def run_reference(args, wl):
     if rank != 0:
         return
     inp = synth.make_inputs(wl, seed=0)
-    _, t_user = oracle_sample(wl, inp, range(1), phi=args.phi)          # calibrates the per-step sample; also the first warm-up
+    _, t_user = oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads)          # calibrates the per-step sample; also the first warm-up
     users_per_step = 2 if (wl.B >= 2 and 2 * t_user * args.steps < 120.0) else 1
     for _ in range(max(0, args.warmup - 1)):
-        oracle_sample(wl, inp, range(1), phi=args.phi)
+        oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads)
     times = []
     for s in range(args.steps):
         users = [(s * users_per_step + u) % wl.B for u in range(users_per_step)]
-        _, dt = oracle_sample(wl, inp, users, phi=args.phi)
+        _, dt = oracle_sample(wl, inp, users, phi=args.phi, cand_heads=args.cand_heads)
         times.append(dt)
     total = sum(times)
     value = users_per_step * wl.C * args.steps / total
@@ -256,10 +257,10 @@ def source_hash(rel):
         return hashlib.sha256(f.read()).hexdigest()[:16]
 
 
-def ncu_traffic(kernel, wl):
+def ncu_traffic(kernel, wl, args=None):
     rec = NCU_TRAFFIC.get((kernel, wl.name, wl.B, wl.C))
-    if not rec:
-        return None
+    if not rec or (args is not None and (args.cand_heads or args.phi != "softmax")):
+        return None          # the captures were taken in the default mode
     try:
         return rec["bytes"] if source_hash(rec["source"]) == rec["sha"] else None
     except OSError:
@@ -284,7 +285,8 @@ def run_ours(args, wl):
     inp = synth.make_inputs(wl, seed=rank)
     dt = Bd.LIME_F32 if wl.dtype == synth.F32 else Bd.LIME_BF16
     lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff,
-                   phi=Bd.LIME_PHI_SILU if args.phi == "silu" else Bd.LIME_PHI_SOFTMAX)
+                   phi=Bd.LIME_PHI_SILU if args.phi == "silu" else Bd.LIME_PHI_SOFTMAX,
+                   cand_heads=wl.H if args.cand_heads else 0)
     table = Bd.to_device(inp["table"], wl.dtype, dev)
     links = Bd.to_device(inp["links"], wl.dtype, dev)
     wts = {k: Bd.to_device(inp[k], wl.dtype, dev) for k in ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")}
@@ -319,7 +321,7 @@ def run_ours(args, wl):
     max_total = max(s["total"] for s in sets)
     off = torch.empty(wl.B + 1, dtype=torch.int32, device=dev)
     hist = torch.empty((max_total, wl.d), dtype=lime.tdtype, device=dev)
-    ls = torch.empty((wl.B, wl.ell, wl.d), dtype=lime.tdtype, device=dev)
+    ls = torch.empty((wl.B, lime.ell_c, wl.d), dtype=lime.tdtype, device=dev)
     logits = torch.empty(wl.B * wl.C, dtype=torch.float32, device=dev)
     ws = lime.workspace(wl.B, max_total)
     ctx = lime.ctx
@@ -516,7 +518,7 @@ def run_ours(args, wl):
     if rank == 0:
         pk = peaks()
         avg_tokens = int(sum(s["total"] for s in sets) / ROTATE)
-        models = kernel_models(wl, avg_tokens)
+        models = kernel_models(wl, avg_tokens, wl.H if args.cand_heads else 1)
         agg = {}
         for name, ms in records:
             a = agg.setdefault(name, [0, 0.0])
@@ -535,7 +537,7 @@ def run_ours(args, wl):
         def roof(k, ms=None, how="CUDA events around each launch inside the step"):
             mdl = model_for(k["kernel"], models)
             r = dict(kernel=k["kernel"], **roofline_entry(mdl, ms if ms is not None else k["ms_per_step"], pk))
-            r["traffic"] = ncu_traffic(k["kernel"], wl)
+            r["traffic"] = ncu_traffic(k["kernel"], wl, args)
             r["peak_source"] = ("derived: 148 SM x 128 lanes x 2 x 1.965 GHz" if r["bound"] == "alu" else
                                 f"{pk['source']} ({'copy bandwidth' if r['bound'] == 'hbm' else 'sustained bf16 GEMM'})")
             r["timing"] = how
@@ -556,19 +558,19 @@ def run_ours(args, wl):
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget, phi=args.phi)
+            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget, phi=args.phi, cand_heads=args.cand_heads)
             cpu = {"value": n_done * wl.C / dt_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                    "sample": f"first {n_done} users x {wl.C} candidates of the same workload, {dt_s:.1f} s "
                              "(gather+encode+precompute+score, fp64 numpy)"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
                 "ms_per_step": total_ms / args.steps, "p50_batch_latency_ms": step_ms[len(step_ms) // 2],
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if wl.dtype == synth.BF16 else "f32",
-                "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args), phi=args.phi), "clocks": clocks,
+                "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args), phi=args.phi, cand_heads=bool(args.cand_heads)), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps, "host_issue_ms_per_step": 1e3 * t_issue / args.steps,
                         "score_by_id_alone_ms": score_by_id_ms,
                         "score_by_id_roofline": dict(kernel="k_score_gather_tc", **roofline_entry(models["k_score_gather_tc"], score_by_id_ms, pk),
-                                                     traffic=ncu_traffic("k_score_gather_tc", wl),
+                                                     traffic=ncu_traffic("k_score_gather_tc", wl, args),
                                                      note="random 128-byte pieces; the copy peak is for contiguous streams"),
                         "how": "pinned host ids -> H2D | offsets, history gather, encode, scoring by candidate id from the resident "
                                "corpus caches | logits D2H; three streams, two request slots"},
@@ -597,6 +599,8 @@ def main():
     ap.add_argument("--sweep", default="", choices=["", "C", "N"], help="one line per point of the candidate / history sweep")
     ap.add_argument("--phi", default="softmax", choices=["softmax", "silu"],
                     help="attention activation of the XOR layers: online softmax (default) or SiLU(s) / n (Algorithms 1-2)")
+    ap.add_argument("--cand-heads", action="store_true",
+                    help="candidate side head by head (Eq. 1 applied to Eq. 4): H * ell cached weights per candidate")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying CUDA graphs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

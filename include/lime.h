@@ -72,6 +72,11 @@ typedef struct lime_config {
   float attn_scale;     /* softmax scale of the XOR layers; 0 means 1/sqrt(d_h)                           */
   float cand_scale;     /* softmax scale of the candidate->link attention; 0 means 1/sqrt(d)              */
   float ln_eps;         /* 0 means 1e-5                                                                   */
+  int32_t cand_heads;   /* candidate side (Eq. 4): 0 or 1 = one weight row per candidate over the full width,
+                           scale 1/sqrt(d); H = Eq. 1 applied head by head: one weight row per (candidate, head),
+                           scale 1/sqrt(d_h), each head mixing its own d_h columns of the link states.  With H the
+                           cached weights have ell_c = H*ell columns (head-major) and a user's link states ell_c
+                           rows (row h*ell + l = link l on head h's columns, zero elsewhere); H*ell <= 256.       */
 } lime_config;
 
 /* Device pointers to the parameters theta, eta of Eq. 1 / Eq. 5 / Eq. 8, all stored as config.dtype. */
@@ -127,7 +132,8 @@ LIME_API lime_status lime_gather_history_normalized(lime_ctx* ctx, const void* t
                                            int64_t total_tokens, void* out, int32_t* dev_flag, void* stream);
 
 /* Offline item-side stage (Eq. 4, Sec. 3.3 "pre-computed and cached"): out_w[c,:] = softmax over the ell
- * links of (T_c W_Q^c)(L W_K^c)^T * cand_scale.  cand_emb [M x d], out_w [M x ell] stored as config.dtype. */
+ * links of (T_c W_Q^c)(L W_K^c)^T * cand_scale.  cand_emb [M x d], out_w [M x ell_c] stored as config.dtype
+ * (ell_c = ell, or H*ell with cand_heads = H: per head the softmax over that head's scores). */
 LIME_API lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb, int64_t M, void* out_w,
                                             void* stream);
 
@@ -143,7 +149,7 @@ LIME_API lime_status lime_xor_layer(lime_ctx* ctx, int32_t layer, const void* hi
                            float* links_out, void* ws, size_t ws_bytes, void* stream);
 
 /* Online user-side stage (Eq. 8): runs the n_layers stacked XOR layers on hist [total_tokens x d] and writes
- * the link states V~ = L^P W_V^c (Eq. 4's values) as config.dtype into link_states [B x ell x d].
+ * the link states V~ = L^P W_V^c (Eq. 4's values) as config.dtype into link_states [B x ell_c x d].
  * link_ctx: optional per-user contextualised links L^C (Eq. 2) as fp32 [B x ell x d]; NULL uses the shared L.
  * hist is not modified. */
 LIME_API lime_status lime_encode_user(lime_ctx* ctx, const void* hist, const int32_t* off, int32_t B,
@@ -160,12 +166,12 @@ LIME_API lime_status lime_encode_user_normalized(lime_ctx* ctx, const void* hist
 
 /* Per-candidate stage (Eq. 4 and Sec. 3.3 "lightweight user-item interaction"):
  *   logits[i] = < sum_l cand_w[i,l] * link_states[b(i),l,:] , cand_emb[i,:] >   for every candidate slot i.
- * Candidates are per user: user b owns slots cand_off[b] .. cand_off[b+1]-1 of cand_w [total_cands x ell],
+ * Candidates are per user: user b owns slots cand_off[b] .. cand_off[b+1]-1 of cand_w [total_cands x ell_c],
  * cand_emb [total_cands x d] and logits [total_cands]; cand_off is a DEVICE int32 array [B+1], non-decreasing,
  * cand_off[0] = 0, cand_off[B] = total_cands.  With cand_off = NULL every user owns C slots (slot b*C + c) and
  * total_cands must equal B*C.  cand_ids (device int32 [total_cands], nullable): when given, cand_w and
  * cand_emb are corpus-level caches (Sec. 3.3 "QK cache") and row cand_ids[i] is read for slot i; ids are
- * not range-checked.  link_states [B x ell x d] as written by lime_encode_user. */
+ * not range-checked.  link_states [B x ell_c x d] as written by lime_encode_user. */
 LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
                                   const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
                                   const int32_t* cand_ids, float* logits, void* stream);

@@ -32,7 +32,7 @@ class lime_config(ctypes.Structure):
     _fields_ = [("d", ctypes.c_int32), ("H", ctypes.c_int32), ("ell", ctypes.c_int32), ("n_layers", ctypes.c_int32),
                 ("d_ff", ctypes.c_int32), ("dtype", ctypes.c_int32), ("phi", ctypes.c_int32), ("ln", ctypes.c_int32),
                 ("gated_mlp", ctypes.c_int32), ("attn_scale", ctypes.c_float), ("cand_scale", ctypes.c_float),
-                ("ln_eps", ctypes.c_float)]
+                ("ln_eps", ctypes.c_float), ("cand_heads", ctypes.c_int32)]
 
 
 _PtrArr = ctypes.c_void_p * LIME_MAX_LAYERS
@@ -241,8 +241,10 @@ class Lime:
 
     def __init__(self, d: int, H: int, ell: int, n_layers: int, dtype: int = LIME_BF16, d_ff: int = 0,
                  phi: int = LIME_PHI_SOFTMAX, ln: bool = True, gated_mlp: bool = True, attn_scale: float = 0.0,
-                 cand_scale: float = 0.0, ln_eps: float = 0.0):
-        self.cfg = lime_config(d, H, ell, n_layers, d_ff, dtype, phi, int(ln), int(gated_mlp), attn_scale, cand_scale, ln_eps)
+                 cand_scale: float = 0.0, ln_eps: float = 0.0, cand_heads: int = 0):
+        self.cfg = lime_config(d, H, ell, n_layers, d_ff, dtype, phi, int(ln), int(gated_mlp), attn_scale, cand_scale, ln_eps,
+                               cand_heads)
+        self.ell_c = ell * (H if cand_heads == H and H > 1 else 1)      # weight columns per candidate, link-state rows
         self.ctx = lime_create(self.cfg)
         self.tdtype = torch_dtype(dtype)
         self._keep = []
@@ -303,18 +305,18 @@ class Lime:
     def encode_user_normalized(self, hist_normalized: torch.Tensor, off: torch.Tensor,
                                link_ctx: Optional[torch.Tensor] = None) -> torch.Tensor:
         B = off.numel() - 1
-        ls = torch.empty((B, self.cfg.ell, self.cfg.d), dtype=self.tdtype, device=hist_normalized.device)
+        ls = torch.empty((B, self.ell_c, self.cfg.d), dtype=self.tdtype, device=hist_normalized.device)
         lime_encode_user_normalized(self.ctx, hist_normalized, off, B, link_ctx, ls, self.workspace(B, hist_normalized.shape[0]))
         return ls
 
     def precompute_candidate_links(self, cand_emb: torch.Tensor) -> torch.Tensor:
-        out = torch.empty((cand_emb.shape[0], self.cfg.ell), dtype=self.tdtype, device=cand_emb.device)
+        out = torch.empty((cand_emb.shape[0], self.ell_c), dtype=self.tdtype, device=cand_emb.device)
         lime_precompute_candidate_links(self.ctx, cand_emb, out)
         return out
 
     def encode_user(self, hist: torch.Tensor, off: torch.Tensor, link_ctx: Optional[torch.Tensor] = None) -> torch.Tensor:
         B = off.numel() - 1
-        ls = torch.empty((B, self.cfg.ell, self.cfg.d), dtype=self.tdtype, device=hist.device)
+        ls = torch.empty((B, self.ell_c, self.cfg.d), dtype=self.tdtype, device=hist.device)
         lime_encode_user(self.ctx, hist, off, B, link_ctx, ls, self.workspace(B, hist.shape[0]))
         return ls
 

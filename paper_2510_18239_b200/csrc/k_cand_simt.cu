@@ -7,6 +7,8 @@ namespace lime {
 
 // ----------------------------------------------------------------------------- effective link keys
 // keff[l, i] = scale * sum_j (L Wk)[l, j] * Wq[i, j]   so that <T_c Wq, L_l Wk> * scale = <T_c, keff_l>.
+// With `heads` > 1 (candidate side head by head) there is one key per (head, link): row h * ell + l sums only over
+// head h's columns j, so that <T_c, keff_(h,l)> is head h's score of candidate c against link l.
 template <typename T>
 __global__ void k_keff_stage1(const T* __restrict__ L, const T* __restrict__ Wk, int ell, int d, float* __restrict__ tmp) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -22,91 +24,96 @@ __global__ void k_keff_stage1(const T* __restrict__ L, const T* __restrict__ Wk,
   tmp[i] = acc;
 }
 template <typename T>
-__global__ void k_keff_stage2(const float* __restrict__ tmp, const T* __restrict__ Wq, int ell, int d, float scale,
+__global__ void k_keff_stage2(const float* __restrict__ tmp, const T* __restrict__ Wq, int ell, int d, int heads, float scale,
                               float* __restrict__ keff) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= ell * d) return;
-  const int l = i / d, r = i % d;
+  if (i >= heads * ell * d) return;
+  const int row = i / d, r = i % d;
+  const int h = row / ell, l = row % ell;
+  const int dh = d / heads, j0 = h * dh, j1 = j0 + dh;      // head h's columns (all of them with one head)
   float acc;
   if (Wq) {
     acc = 0.f;
-    for (int j = 0; j < d; ++j) acc = fmaf(tmp[l * d + j], Store<T>::ld(Wq + (int64_t)r * d + j), acc);
+    for (int j = j0; j < j1; ++j) acc = fmaf(tmp[l * d + j], Store<T>::ld(Wq + (int64_t)r * d + j), acc);
   } else {
-    acc = tmp[i];
+    acc = (r >= j0 && r < j1) ? tmp[l * d + r] : 0.f;
   }
   keff[i] = acc * scale;
 }
 
-lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, float scale,
+lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, int heads, float scale,
                         float* keff, cudaStream_t st) {
-  // stage 1 writes into the second half of the keff buffer (the context allocates 2 * ell * d floats)
-  float* tmp = keff + (size_t)ell * d;
-  const int n = ell * d, blocks = (n + 127) / 128;
+  // stage 1 writes behind the keys (the caller provides 2 * heads * ell * d floats)
+  float* tmp = keff + (size_t)heads * ell * d;
+  const int n = ell * d, blocks = (n + 127) / 128, blocks2 = (heads * n + 127) / 128;
   ProfScope _p("k_keff", st);
   if (dtype == LIME_F32) {
     k_keff_stage1<float><<<blocks, 128, 0, st>>>((const float*)L, (const float*)Wk, ell, d, tmp);
-    k_keff_stage2<float><<<blocks, 128, 0, st>>>(tmp, (const float*)Wq, ell, d, scale, keff);
+    k_keff_stage2<float><<<blocks2, 128, 0, st>>>(tmp, (const float*)Wq, ell, d, heads, scale, keff);
   } else {
     k_keff_stage1<__nv_bfloat16><<<blocks, 128, 0, st>>>((const __nv_bfloat16*)L, (const __nv_bfloat16*)Wk, ell, d, tmp);
-    k_keff_stage2<__nv_bfloat16><<<blocks, 128, 0, st>>>(tmp, (const __nv_bfloat16*)Wq, ell, d, scale, keff);
+    k_keff_stage2<__nv_bfloat16><<<blocks2, 128, 0, st>>>(tmp, (const __nv_bfloat16*)Wq, ell, d, heads, scale, keff);
   }
   LIME_LAUNCH_CHECK("k_keff");
   return LIME_OK;
 }
 
 // ----------------------------------------------------------------------------- candidate -> link weights
-// W[c, :] = softmax over links of <T_c, keff_l>.  keff (fp32) sits in shared memory, one warp per candidate.
+// W[c, :] = softmax over links of <T_c, keff_l>.  keff (fp32) sits in shared memory, one warp per candidate.  The
+// `rows` keys form rows / ell groups (one per head of the candidate side); the softmax runs inside each group.
 constexpr int PC_WARPS = 8;
 template <typename T>
 __global__ void __launch_bounds__(PC_WARPS * 32)
-k_precompute(const T* __restrict__ cand, int64_t M, int d, int ell, const float* __restrict__ keff, T* __restrict__ out_w) {
+k_precompute(const T* __restrict__ cand, int64_t M, int d, int rows, int ell, const float* __restrict__ keff, T* __restrict__ out_w) {
   extern __shared__ float smem[];
   const int ldk = d + 1;
   float* Ks = smem;                  // [ell][d+1]
-  float* ts = Ks + ell * ldk;        // [warps][d]
+  float* ts = Ks + rows * ldk;       // [warps][d]
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  for (int i = tid; i < ell * d; i += blockDim.x) Ks[(i / d) * ldk + (i % d)] = keff[i];
+  for (int i = tid; i < rows * d; i += blockDim.x) Ks[(i / d) * ldk + (i % d)] = keff[i];
   __syncthreads();
   float* tw = ts + wid * d;
   constexpr int MAXL = 8;
   for (int64_t c = (int64_t)blockIdx.x * PC_WARPS + wid; c < M; c += (int64_t)gridDim.x * PC_WARPS) {
     for (int k = lane; k < d; k += 32) tw[k] = Store<T>::ld(cand + c * d + k);
     __syncwarp();
-    float p[MAXL];
-    float mx = -INFINITY;
+    for (int g0 = 0; g0 < rows; g0 += ell) {
+      float p[MAXL];
+      float mx = -INFINITY;
 #pragma unroll
-    for (int j = 0; j < MAXL; ++j) {
-      const int l = lane + 32 * j;
-      float sc = -INFINITY;
-      if (l < ell) {
-        sc = 0.f;
-        const float* kr = Ks + l * ldk;
-        for (int k = 0; k < d; ++k) sc = fmaf(tw[k], kr[k], sc);
+      for (int j = 0; j < MAXL; ++j) {
+        const int l = lane + 32 * j;
+        float sc = -INFINITY;
+        if (l < ell) {
+          sc = 0.f;
+          const float* kr = Ks + (g0 + l) * ldk;
+          for (int k = 0; k < d; ++k) sc = fmaf(tw[k], kr[k], sc);
+        }
+        p[j] = sc;
+        mx = fmaxf(mx, sc);
       }
-      p[j] = sc;
-      mx = fmaxf(mx, sc);
-    }
-    mx = warp_max(mx);
-    float sum = 0.f;
+      mx = warp_max(mx);
+      float sum = 0.f;
 #pragma unroll
-    for (int j = 0; j < MAXL; ++j) {
-      p[j] = (lane + 32 * j < ell) ? __expf(p[j] - mx) : 0.f;
-      sum += p[j];
-    }
-    const float inv = 1.f / warp_sum(sum);
+      for (int j = 0; j < MAXL; ++j) {
+        p[j] = (lane + 32 * j < ell) ? __expf(p[j] - mx) : 0.f;
+        sum += p[j];
+      }
+      const float inv = 1.f / warp_sum(sum);
 #pragma unroll
-    for (int j = 0; j < MAXL; ++j) {
-      const int l = lane + 32 * j;
-      if (l < ell) Store<T>::st(out_w + c * ell + l, p[j] * inv);
+      for (int j = 0; j < MAXL; ++j) {
+        const int l = lane + 32 * j;
+        if (l < ell) Store<T>::st(out_w + c * rows + g0 + l, p[j] * inv);
+      }
     }
     __syncwarp();
   }
 }
 
-lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int ell, const float* keff, void* out_w,
+lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int rows, int ell, const float* keff, void* out_w,
                               cudaStream_t st) {
   if (M == 0) return LIME_OK;
-  const size_t smem = sizeof(float) * ((size_t)ell * (d + 1) + (size_t)PC_WARPS * d);
+  const size_t smem = sizeof(float) * ((size_t)rows * (d + 1) + (size_t)PC_WARPS * d);
   if (smem > 200 * 1024) return LIME_UNSUPPORTED_SHAPE;
   int64_t blocks = (M + PC_WARPS - 1) / PC_WARPS;
   const int64_t cap = (int64_t)kSMs * 4;
@@ -114,10 +121,10 @@ lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int
   ProfScope _p("k_precompute", st);
   if (dtype == LIME_F32) {
     LIME_CUDA(cudaFuncSetAttribute(k_precompute<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_precompute<float><<<(int)blocks, PC_WARPS * 32, smem, st>>>((const float*)cand, M, d, ell, keff, (float*)out_w);
+    k_precompute<float><<<(int)blocks, PC_WARPS * 32, smem, st>>>((const float*)cand, M, d, rows, ell, keff, (float*)out_w);
   } else {
     LIME_CUDA(cudaFuncSetAttribute(k_precompute<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_precompute<__nv_bfloat16><<<(int)blocks, PC_WARPS * 32, smem, st>>>((const __nv_bfloat16*)cand, M, d, ell, keff,
+    k_precompute<__nv_bfloat16><<<(int)blocks, PC_WARPS * 32, smem, st>>>((const __nv_bfloat16*)cand, M, d, rows, ell, keff,
                                                                         (__nv_bfloat16*)out_w);
   }
   LIME_LAUNCH_CHECK("k_precompute");

@@ -285,10 +285,35 @@ __global__ void k_axpy(const float* __restrict__ x, float* __restrict__ y, int64
     y[i] = (zero_first ? 0.0f : y[i]) + x[i];
 }
 
+// Link states of the per-head candidate side (Eq. 1 applied to Eq. 4): row (h, l) of a user is L^P row l on head h's
+// columns and zero elsewhere, so that the full-width dot <T_c, row (h, l)> is head h's dot product.
+template <typename T>
+__global__ void k_expand_heads(const float* __restrict__ src, int64_t n_out, int ell, int d, int heads, T* __restrict__ out) {
+  const int dh = d / heads;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_out; i += (int64_t)gridDim.x * blockDim.x) {
+    const int j = (int)(i % d);
+    const int64_t row = i / d;                       // (user, head, link)
+    const int l = (int)(row % ell), h = (int)((row / ell) % heads);
+    const int64_t b = row / ((int64_t)ell * heads);
+    Store<T>::st(out + i, j / dh == h ? src[(b * ell + l) * d + j] : 0.f);
+  }
+}
+
 static inline int ew_blocks(int64_t n) {
   int64_t b = (n + 255) / 256;
   const int64_t cap = (int64_t)kSMs * 8;
   return (int)(b > cap ? cap : (b < 1 ? 1 : b));
+}
+
+lime_status launch_expand_heads(const float* src, int64_t rows_in, int ell, int d, int heads, void* out, int dtype,
+                                cudaStream_t st) {
+  const int64_t n_out = rows_in * heads * d;
+  if (n_out == 0) return LIME_OK;
+  ProfScope _p("k_expand_heads", st);
+  if (dtype == LIME_F32) k_expand_heads<float><<<ew_blocks(n_out), 256, 0, st>>>(src, n_out, ell, d, heads, (float*)out);
+  else k_expand_heads<__nv_bfloat16><<<ew_blocks(n_out), 256, 0, st>>>(src, n_out, ell, d, heads, (__nv_bfloat16*)out);
+  LIME_LAUNCH_CHECK("k_expand_heads");
+  return LIME_OK;
 }
 
 lime_status launch_cast_rows(const float* in, int64_t n, void* out, int dtype, cudaStream_t st) {

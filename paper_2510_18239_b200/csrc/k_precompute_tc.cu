@@ -11,6 +11,7 @@
 //   warp 0    : TMA producer - item tile [128 x d] into a ring of 128B-swizzled stages (keys once, resident)
 //   warp 1    : MMA issuer   - d/16 tcgen05.mma (M=128, N=2 ell, K=16) per tile into one of two TMEM accumulators
 //   warps 2-5 : epilogue     - thread r owns item row r (TMEM lane r): row softmax in registers, bf16 row to global
+//                              (GROUP < ELL: the ELL keys are ELL / GROUP heads' keys and the softmax runs per head)
 // HBM traffic per item is the algorithmic minimum: its embedding row in, its weight row out.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
@@ -51,7 +52,7 @@ __device__ __forceinline__ uint32_t pct_pack(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int ELL>
+template <int ELL, int GROUP>
 __global__ void __launch_bounds__(PCT_THREADS, 1)
 k_precompute_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmK, const PrecomputeTcParams p) {
   using namespace tc;
@@ -175,27 +176,32 @@ k_precompute_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[buf]);
-      float mx = sc[0];
 #pragma unroll
-      for (int j = 1; j < ELL; ++j) mx = fmaxf(mx, sc[j]);
-      float s0 = 0.f, s1 = 0.f;
+      for (int g0 = 0; g0 < ELL; g0 += GROUP) {
+        float mx = sc[g0];
 #pragma unroll
-      for (int j = 0; j < ELL; j += 2) {
-        sc[j] = __expf(sc[j] - mx);
-        sc[j + 1] = __expf(sc[j + 1] - mx);
-        s0 += sc[j];
-        s1 += sc[j + 1];
+        for (int j = 1; j < GROUP; ++j) mx = fmaxf(mx, sc[g0 + j]);
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < GROUP; j += 2) {
+          sc[g0 + j] = __expf(sc[g0 + j] - mx);
+          sc[g0 + j + 1] = __expf(sc[g0 + j + 1] - mx);
+          s0 += sc[g0 + j];
+          s1 += sc[g0 + j + 1];
+        }
+        const float inv = 1.f / (s0 + s1);
+#pragma unroll
+        for (int j = 0; j < GROUP; ++j) sc[g0 + j] *= inv;
       }
-      const float inv = 1.f / (s0 + s1);
       if (row < p.M) {
         uint4* dst = reinterpret_cast<uint4*>(p.out + row * ELL);
 #pragma unroll
         for (int c8 = 0; c8 < ELL / 8; ++c8) {
           uint4 o;
-          o.x = pct_pack(sc[c8 * 8 + 0] * inv, sc[c8 * 8 + 1] * inv);
-          o.y = pct_pack(sc[c8 * 8 + 2] * inv, sc[c8 * 8 + 3] * inv);
-          o.z = pct_pack(sc[c8 * 8 + 4] * inv, sc[c8 * 8 + 5] * inv);
-          o.w = pct_pack(sc[c8 * 8 + 6] * inv, sc[c8 * 8 + 7] * inv);
+          o.x = pct_pack(sc[c8 * 8 + 0], sc[c8 * 8 + 1]);
+          o.y = pct_pack(sc[c8 * 8 + 2], sc[c8 * 8 + 3]);
+          o.z = pct_pack(sc[c8 * 8 + 4], sc[c8 * 8 + 5]);
+          o.w = pct_pack(sc[c8 * 8 + 6], sc[c8 * 8 + 7]);
           __stcs(dst + c8, o);
         }
       }
@@ -221,15 +227,16 @@ static int precompute_tc_stages(int ell, int d, size_t* smem_bytes) {
   return S;
 }
 
-bool precompute_tc_supported(int dtype, int d, int ell) {
+bool precompute_tc_supported(int dtype, int d, int ell, int group) {
   if (dtype != LIME_BF16) return false;
   if (!(ell == 16 || ell == 32 || ell == 64 || ell == 128)) return false;
+  if (!(group == ell || group == 16 || group == 32 || group == 64) || group > ell) return false;
   if (d % 64 != 0 || d > 512) return false;
   size_t smem;
   return precompute_tc_stages(ell, d, &smem) >= 2;
 }
 
-template <int ELL>
+template <int ELL, int GROUP>
 static lime_status launch_precompute_tc_t(const void* cand, int64_t M, int d, const void* keff_hl, void* out_w, int* err,
                                           cudaStream_t st) {
   size_t smem;
@@ -243,22 +250,32 @@ static lime_status launch_precompute_tc_t(const void* cand, int64_t M, int d, co
   p.n_tiles = (int)((M + PCT_TILE - 1) / PCT_TILE);
   p.stages = S; p.err = err;
   const int grid = p.n_tiles < kSMs ? p.n_tiles : kSMs;
-  LIME_CUDA(cudaFuncSetAttribute(k_precompute_tc<ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  LIME_CUDA(cudaFuncSetAttribute(k_precompute_tc<ELL, GROUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   ProfScope _p("k_precompute_tc", st);
-  k_precompute_tc<ELL><<<grid, PCT_THREADS, smem, st>>>(tmT, tmK, p);
+  k_precompute_tc<ELL, GROUP><<<grid, PCT_THREADS, smem, st>>>(tmT, tmK, p);
   LIME_LAUNCH_CHECK("k_precompute_tc");
   return LIME_OK;
 }
 
-lime_status launch_precompute_tc(const void* cand, int64_t M, int d, int ell, const void* keff_hl, void* out_w, int* err,
-                                 cudaStream_t st) {
+template <int ELL>
+static lime_status launch_precompute_tc_g(const void* cand, int64_t M, int d, int group, const void* keff_hl, void* out_w, int* err,
+                                          cudaStream_t st) {
+  if (group == ELL) return launch_precompute_tc_t<ELL, ELL>(cand, M, d, keff_hl, out_w, err, st);
+  if constexpr (ELL > 16) if (group == 16) return launch_precompute_tc_t<ELL, 16>(cand, M, d, keff_hl, out_w, err, st);
+  if constexpr (ELL > 32) if (group == 32) return launch_precompute_tc_t<ELL, 32>(cand, M, d, keff_hl, out_w, err, st);
+  if constexpr (ELL > 64) if (group == 64) return launch_precompute_tc_t<ELL, 64>(cand, M, d, keff_hl, out_w, err, st);
+  return LIME_UNSUPPORTED_SHAPE;
+}
+
+lime_status launch_precompute_tc(const void* cand, int64_t M, int d, int rows, int group, const void* keff_hl, void* out_w,
+                                 int* err, cudaStream_t st) {
   if (M == 0) return LIME_OK;
   if (M > (int64_t)0x7fffffff * PCT_TILE / 2) return LIME_UNSUPPORTED_SHAPE;
-  switch (ell) {
-    case 16: return launch_precompute_tc_t<16>(cand, M, d, keff_hl, out_w, err, st);
-    case 32: return launch_precompute_tc_t<32>(cand, M, d, keff_hl, out_w, err, st);
-    case 64: return launch_precompute_tc_t<64>(cand, M, d, keff_hl, out_w, err, st);
-    case 128: return launch_precompute_tc_t<128>(cand, M, d, keff_hl, out_w, err, st);
+  switch (rows) {
+    case 16: return launch_precompute_tc_g<16>(cand, M, d, group, keff_hl, out_w, err, st);
+    case 32: return launch_precompute_tc_g<32>(cand, M, d, group, keff_hl, out_w, err, st);
+    case 64: return launch_precompute_tc_g<64>(cand, M, d, group, keff_hl, out_w, err, st);
+    case 128: return launch_precompute_tc_g<128>(cand, M, d, group, keff_hl, out_w, err, st);
   }
   return LIME_UNSUPPORTED_SHAPE;
 }

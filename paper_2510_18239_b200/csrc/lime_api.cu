@@ -205,7 +205,7 @@ static lime_status encode_user_tc(Ctx* c, const void* hist, bool hist_normalized
     LinkMlpArgs mlp{};
     mlp.LP = w.LP; mlp.lp_accumulate = j > 0;                                   // L^P = sum_j T^j  (Eq. 8)
     mlp.That_next = last ? nullptr : w.That;
-    mlp.link_states = (last && !c->w.cand_Wv) ? link_states : nullptr;
+    mlp.link_states = (last && !c->w.cand_Wv && c->cand_heads == 1) ? link_states : nullptr;
     s = tc_layer_core(c, j, j == 0 ? hist : w.S, off, B, total, ops, last ? nullptr : w.S, (g.ln && j == 0 && !hist_normalized) ? 1 : 0,
                       (g.ln && !last) ? 1 : 0, mlp, w, st);
     if (s != LIME_OK) return s;
@@ -365,6 +365,9 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   if (g.dtype != LIME_F32 && g.dtype != LIME_BF16) return LIME_INVALID_ARG;
   if (g.phi != LIME_PHI_SOFTMAX && g.phi != LIME_PHI_SILU) return LIME_INVALID_ARG;
   if (g.attn_scale < 0.f || g.cand_scale < 0.f || g.ln_eps < 0.f) return LIME_INVALID_ARG;
+  if (g.cand_heads != 0 && g.cand_heads != 1 && g.cand_heads != g.H) return LIME_INVALID_ARG;
+  const int cand_heads = g.cand_heads == g.H ? g.H : 1;
+  if (cand_heads * g.ell > 256) return LIME_UNSUPPORTED_SHAPE;
   const int d_ff = g.d_ff ? g.d_ff : g.d;
   if (g.d % 8 || d_ff % 8 || g.d % g.H || g.d / g.H > 128 || g.ell > 256 || g.n_layers > LIME_MAX_LAYERS ||
       g.d > 1024 || d_ff > 1024)
@@ -379,14 +382,17 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->d_ff = d_ff;
   c->d_h = g.d / g.H;
   c->attn_scale = g.attn_scale > 0.f ? g.attn_scale : 1.0f / sqrtf((float)c->d_h);
-  c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)g.d);
+  c->cand_heads = cand_heads;
+  c->ell_c = cand_heads * g.ell;
+  // per-head scores are scaled like any head of Eq. 1; the single-row form by the full width
+  c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)(cand_heads > 1 ? c->d_h : g.d));
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = nullptr;
   c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
-  if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)g.ell * g.d);
-  if (e == cudaSuccess) e = cudaMalloc(&c->keff_hl, 2 * (size_t)2 * g.ell * g.d);
+  if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)c->ell_c * g.d);
+  if (e == cudaSuccess) e = cudaMalloc(&c->keff_hl, 2 * (size_t)2 * c->ell_c * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->links32, sizeof(float) * (size_t)g.ell * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->dev_err, sizeof(int));
   if (e == cudaSuccess) e = cudaMemset(c->dev_err, 0, sizeof(int));
@@ -431,9 +437,10 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   lime_status s = launch_widen(w->links, g.dtype, c->links32, (int64_t)g.ell * g.d, st);
   if (s != LIME_OK) return s;
-  s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_scale, c->keff, st);
+  s = launch_keff(g.dtype, w->links, w->cand_Wk, w->cand_Wq, g.ell, g.d, c->cand_heads, c->cand_scale, c->keff, st);
   if (s != LIME_OK) return s;
-  if (precompute_tc_supported(g.dtype, g.d, g.ell) && (s = launch_keff_split(c->keff, g.ell, g.d, c->keff_hl, st)) != LIME_OK)
+  if (precompute_tc_supported(g.dtype, g.d, c->ell_c, g.ell) &&
+      (s = launch_keff_split(c->keff, c->ell_c, g.d, c->keff_hl, st)) != LIME_OK)
     return s;
   // tensor-core path: per layer, W_o as a K-major B operand ([d x d_ff], contraction index contiguous) and the
   // weight-only products that fold the history-side projections into the link rows
@@ -510,10 +517,10 @@ lime_status lime_precompute_candidate_links(lime_ctx* ctx, const void* cand_emb,
   if (!c->have_weights) return LIME_NOT_READY;
   if (M == 0) return LIME_OK;
   if (!cand_emb || !out_w || !aligned16(cand_emb) || !aligned16(out_w)) return LIME_INVALID_ARG;
-  if (precompute_tc_supported(c->cfg.dtype, c->cfg.d, c->cfg.ell))
-    return launch_precompute_tc(cand_emb, M, c->cfg.d, c->cfg.ell, c->keff_hl, out_w, c->dev_err,
+  if (precompute_tc_supported(c->cfg.dtype, c->cfg.d, c->ell_c, c->cfg.ell))
+    return launch_precompute_tc(cand_emb, M, c->cfg.d, c->ell_c, c->cfg.ell, c->keff_hl, out_w, c->dev_err,
                                 static_cast<cudaStream_t>(stream));
-  return launch_precompute(c->cfg.dtype, cand_emb, M, c->cfg.d, c->cfg.ell, c->keff, out_w,
+  return launch_precompute(c->cfg.dtype, cand_emb, M, c->cfg.d, c->ell_c, c->cfg.ell, c->keff, out_w,
                            static_cast<cudaStream_t>(stream));
 }
 
@@ -558,7 +565,7 @@ static lime_status encode_user_impl(lime_ctx* ctx, const void* hist, bool hist_n
   const int64_t BLd = (int64_t)B * g.ell * g.d;
   if (layer_on_tensor_cores(c, 0)) {
     if ((s = encode_user_tc(c, hist, hist_normalized, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;
-    if (!c->w.cand_Wv) return LIME_OK;        // the last layer's kernel wrote the link states
+    if (!c->w.cand_Wv && c->cand_heads == 1) return LIME_OK;        // the last layer's kernel wrote the link states
   } else {
     for (int j = 0; j < g.n_layers; ++j) {
       const bool last = j == g.n_layers - 1;
@@ -579,6 +586,7 @@ static lime_status encode_user_impl(lime_ctx* ctx, const void* hist, bool hist_n
     if ((s = launch_linear_simt(lv, st)) != LIME_OK) return s;
     src = w.LS32;
   }
+  if (c->cand_heads > 1) return launch_expand_heads(src, (int64_t)B * g.ell, g.ell, g.d, c->cand_heads, link_states, g.dtype, st);
   return launch_cast_rows(src, BLd, link_states, g.dtype, st);
 }
 
@@ -603,7 +611,7 @@ lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_
   if (!aligned16(link_states) || !aligned16(cand_w) || !aligned16(cand_emb)) return LIME_INVALID_ARG;
   Ctx* c = reinterpret_cast<Ctx*>(ctx);
   ScoreArgs a{};
-  a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->cfg.ell; a.d = c->cfg.d;
+  a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->ell_c; a.d = c->cfg.d;
   a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
   if (score_tc_supported(a)) return launch_score_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   if (score_gather_tc_supported(a)) return launch_score_gather_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));

@@ -50,6 +50,8 @@ struct Ctx {
   lime_weights w;
   bool have_weights;
   int device;
+  int cand_heads;   // heads of the candidate side: 1 (one weight row per candidate) or H (one per head)
+  int ell_c;        // weight columns per candidate = cand_heads * ell; also the rows of a user's link states
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
   void* keff_hl;    // [2 ell x d] bf16: keff split into a rounded part and its remainder (tensor-core precompute)
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
@@ -148,18 +150,23 @@ lime_status launch_cast_rows(const float* in, int64_t n, void* out, int dtype, c
 lime_status launch_axpy(const float* x, float* y, int64_t n, int zero_first, cudaStream_t st);
 lime_status launch_widen(const void* in, int dtype, float* out, int64_t n, cudaStream_t st);
 
-// candidate -> link weights: W[c, :] = softmax_l( <T_c, keff_l> )  (keff already carries cand_scale)
-lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int ell, const float* keff,
+// candidate -> link weights: W[c, :] = softmax_l( <T_c, keff_l> )  (keff already carries cand_scale); `rows` keys
+// in groups of `ell` (one group per head of the candidate side), the softmax inside each group
+lime_status launch_precompute(int dtype, const void* cand, int64_t M, int d, int rows, int ell, const float* keff,
                               void* out_w, cudaStream_t st);
-// keff = ((L Wk) Wq^T) * scale, fp32 [ell x d]
-lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, float scale,
+// keff = ((L Wk) Wq^T) * scale, fp32 [heads * ell x d]: one key per link, or per (head, link) restricted to the
+// head's columns; the buffer holds 2 * heads * ell * d floats
+lime_status launch_keff(int dtype, const void* L, const void* Wk, const void* Wq, int ell, int d, int heads, float scale,
                         float* keff, cudaStream_t st);
+// link states for the per-head candidate side: out[b, h * ell + l, :] = src[b, l, :] on head h's columns, 0 elsewhere
+lime_status launch_expand_heads(const float* src, int64_t rows_in, int ell, int d, int heads, void* out, int dtype, cudaStream_t st);
 
 // bf16 precompute on tcgen05 tensor cores (ell in {16,32,64,128}, d % 64 == 0); keff_hl from launch_keff_split
-bool precompute_tc_supported(int dtype, int d, int ell);
+// `ell` keys in all, softmax per group of `group` consecutive keys (group == ell: one softmax per row)
+bool precompute_tc_supported(int dtype, int d, int ell, int group);
 lime_status launch_keff_split(const float* keff, int ell, int d, void* keff_hl, cudaStream_t st);
-lime_status launch_precompute_tc(const void* cand, int64_t M, int d, int ell, const void* keff_hl, void* out_w, int* err,
-                                 cudaStream_t st);
+lime_status launch_precompute_tc(const void* cand, int64_t M, int d, int rows, int group, const void* keff_hl, void* out_w,
+                                 int* err, cudaStream_t st);
 
 struct ScoreArgs {
   const void* LS; const void* W; const void* T; int dtype;

@@ -56,6 +56,6 @@ extern "C" lime_status lime_precompute_candidate_links_noalloc(int32_t dtype, in
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float scale = cand_scale > 0.f ? cand_scale : 1.0f / sqrtf((float)d);
   // both halves of the scratch are fully rewritten before they are read, so nothing has to start at zero
-  if ((s = launch_keff(dtype, links, cand_Wk, cand_Wq, ell, d, scale, scratch, st)) != LIME_OK) return s;
-  return launch_precompute(dtype, cand_emb, M, d, ell, scratch, out_w, st);
+  if ((s = launch_keff(dtype, links, cand_Wk, cand_Wq, ell, d, 1, scale, scratch, st)) != LIME_OK) return s;
+  return launch_precompute(dtype, cand_emb, M, d, ell, ell, scratch, out_w, st);
 }

@@ -29,28 +29,28 @@ def oracle_layers(inp: Dict[str, np.ndarray], wl: synth.Workload, gated_mlp=True
 
 
 def oracle_user(inp, wl, b: int, off: np.ndarray, table64: np.ndarray, links64: np.ndarray, layers, cfg,
-                cand_rows: Optional[np.ndarray] = None, cand_w=None):
+                cand_rows: Optional[np.ndarray] = None, cand_w=None, cand_heads: bool = False):
     """Oracle logits / link states / weights for user b (optionally only candidate slots `cand_rows` of that user)."""
     E = O.gather_history(table64, inp["hist_ids"][off[b]:off[b + 1]])
     cids = inp["cand_ids"][b * wl.C:(b + 1) * wl.C]
     if cand_rows is not None:
         cids = cids[cand_rows]
     T = O.gather_history(table64, cids)
-    return O.run_user(E, links64, layers, cfg, T, cand_w=cand_w)
+    return O.run_user(E, links64, layers, cfg, T, cand_w=cand_w, cand_heads=cand_heads)
 
 
 class DeviceBatch:
     """Device-side mirror of one synthetic batch plus a configured library context."""
 
     def __init__(self, wl: synth.Workload, inp: Dict[str, np.ndarray], phi=0, ln=True, gated_mlp=True, cand=None,
-                 attn_scale=0.0):
+                 attn_scale=0.0, cand_heads=0):
         import torch
         from paper_2510_18239_b200 import binding as Bd
         self.Bd = Bd
         self.wl = wl
         dt = Bd.LIME_F32 if wl.dtype == synth.F32 else Bd.LIME_BF16
         self.lime = Bd.Lime(wl.d, wl.H, wl.ell, wl.n_layers, dtype=dt, d_ff=wl.d_ff, phi=phi, ln=ln, gated_mlp=gated_mlp,
-                            attn_scale=attn_scale)
+                            attn_scale=attn_scale, cand_heads=cand_heads)
         self.table = Bd.to_device(inp["table"], wl.dtype)
         self.links = Bd.to_device(inp["links"], wl.dtype)
         self.w = {k: Bd.to_device(inp[k], wl.dtype) for k in LAYER_KEYS}

@@ -46,5 +46,5 @@ def test_version_string_and_host_side_validation():
 
 
 def test_struct_layouts_match_header():
-    assert ctypes.sizeof(binding.lime_config) == 12 * 4
+    assert ctypes.sizeof(binding.lime_config) == 13 * 4          # 12 fields of the paper's model + cand_heads
     assert ctypes.sizeof(binding.lime_weights) == 8 * (1 + 6 * binding.LIME_MAX_LAYERS + 3)

@@ -508,6 +508,40 @@ def test_candidate_side_projections_and_link_context():
         assert np.abs(Hh.to_f64(ls[b]) - LP).max() <= 2e-4 * max(1.0, np.abs(LP).max())
 
 
+@pytest.mark.parametrize("dtype,d,H,ell,proj", [(synth.F32, 32, 2, 8, False), (synth.F32, 64, 4, 5, True),
+                                                 (synth.BF16, 128, 4, 32, False), (synth.BF16, 128, 8, 16, True),
+                                                 (synth.BF16, 128, 2, 32, False), (synth.BF16, 128, 4, 64, False),
+                                                 (synth.BF16, 64, 2, 33, False)])
+def test_candidate_side_head_by_head(dtype, d, H, ell, proj):
+    """Eq. 1 applied to Eq. 4 head by head (cand_heads = H): cached weights [C x H x ell], link states expanded per head,
+    logits against the oracle's per-head form.  H * ell = 128 runs the tensor-core precompute (per-head softmax groups)
+    and scorer; 256 and odd sizes the generic kernels."""
+    Bd = _lib()
+    wl = small(dtype, B=3, n_min=20, n_max=200, d=d, H=H, ell=ell, n_layers=2, C=300, V=2000,
+               table_std=0.05 if dtype == synth.BF16 else 1.0)
+    inp = synth.make_inputs(wl, seed=d + ell)
+    cand_np = None
+    if proj:
+        cand_np = {k: synth.normal_storage(6, "c" + k, (d, d), d ** -0.5, dtype) for k in ("Wq", "Wk", "Wv")}
+    dev = Hh.DeviceBatch(wl, inp, cand=cand_np, cand_heads=H)
+    out = dev.run()
+    assert tuple(out["W"].shape) == (wl.B * wl.C, H * ell) and tuple(out["link_states"].shape) == (wl.B, H * ell, d)
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    table64 = synth.storage_to_f64(inp["table"], dtype)
+    links64 = synth.storage_to_f64(inp["links"], dtype)
+    cw = {k + "_c": synth.storage_to_f64(v, dtype) for k, v in cand_np.items()} if cand_np else None
+    off = O.lengths_to_offsets(inp["lengths"])
+    got_all, want_all = [], []
+    for b in range(wl.B):
+        lg, LS, W = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg, cand_w=cw, cand_heads=True)
+        got_w = Hh.to_f64(out["W"][b * wl.C:(b + 1) * wl.C]).reshape(wl.C, H, ell)
+        assert np.abs(got_w.sum(axis=2) - 1.0).max() <= (1e-5 if dtype == synth.F32 else 2e-2)
+        assert np.abs(got_w - W).max() <= (1e-5 if dtype == synth.F32 else 2.0 ** -8)
+        got_all.append(Hh.to_f64(out["logits"][b * wl.C:(b + 1) * wl.C]))
+        want_all.append(lg)
+    _check_logits(np.concatenate(got_all), np.concatenate(want_all), dtype)
+
+
 # ----------------------------------------------------------------------------- the named workloads
 def test_config1_tiny_fp32_full_parity():
     wl = synth.named_workloads()["tiny_fp32"]
