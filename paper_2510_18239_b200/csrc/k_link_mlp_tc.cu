@@ -73,6 +73,7 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   uint64_t* out_full = wo_full + 3;
   uint64_t* pair_bar = wo_full + 4;      // [4], 2 warps each
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(wo_full + 8);
+  uint64_t* all_bar = wo_full + 9;       // rendezvous of the 8 epilogue warps (tiles staged in shared memory)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m0 = blockIdx.x * 128;
@@ -81,6 +82,7 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     for (int s = 0; s < LM_STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(wo_full, 1); mbar_init(gu_full, 1); mbar_init(u_ready, 8); mbar_init(out_full, 1);
     for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 2);
+    mbar_init(all_bar, 8);
     fence_barrier_init();
     prefetch_tmap(&tmA); prefetch_tmap(&tmB); prefetch_tmap(&tmWo);
   }
@@ -148,8 +150,6 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     const int q = warp & 3;
     const int half = ew >> 2;
     const uint32_t r = (uint32_t)(q * 32 + lane);
-    const int64_t row = (int64_t)m0 + r;
-    const bool valid = row < p.M;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     float* exch = reinterpret_cast<float*>(smem + LM_OFF_EXCH);
     if (mbar_wait(gu_full, 0, p.err, 73)) {
@@ -192,30 +192,31 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
         }
-        const int64_t o64 = row * 128 + half * 64;
-        if (valid && p.T_out) {
+        // T, the running sum of Eq. 8 and (last layer) the link states leave row by row: a thread owns half a row
+        // (256 bytes), so direct accesses would touch 32 lines per instruction.  The tile is staged as fp32 in the
+        // stage ring (free since the first contraction finished) and each warp then moves whole 512-byte rows.
+        constexpr int TS_LD = 132;                                   // floats per staged row (pad: 16-byte aligned, 4-way banks)
+        float* Ts = reinterpret_cast<float*>(smem);
 #pragma unroll
-          for (int j = 0; j < 64; j += 4) *reinterpret_cast<float4*>(p.T_out + o64 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-        }
-        if (valid && p.LP) {
-          // running sum of Eq. 8; on the last layer it also leaves as the link states
-#pragma unroll
-          for (int j = 0; j < 64; j += 8) {
-            float s[8];
-            if (p.lp_accumulate) {
-              const float4 a = *reinterpret_cast<const float4*>(p.LP + o64 + j), b = *reinterpret_cast<const float4*>(p.LP + o64 + j + 4);
-              s[0] = a.x + v[j]; s[1] = a.y + v[j + 1]; s[2] = a.z + v[j + 2]; s[3] = a.w + v[j + 3];
-              s[4] = b.x + v[j + 4]; s[5] = b.y + v[j + 5]; s[6] = b.z + v[j + 6]; s[7] = b.w + v[j + 7];
-            } else {
-#pragma unroll
-              for (int i = 0; i < 8; ++i) s[i] = v[j + i];
-            }
-            *reinterpret_cast<float4*>(p.LP + o64 + j) = make_float4(s[0], s[1], s[2], s[3]);
-            *reinterpret_cast<float4*>(p.LP + o64 + j + 4) = make_float4(s[4], s[5], s[6], s[7]);
-            if (p.link_states) {
-              uint4 o;
-              o.x = lm_pack(s[0], s[1]); o.y = lm_pack(s[2], s[3]); o.z = lm_pack(s[4], s[5]); o.w = lm_pack(s[6], s[7]);
-              *reinterpret_cast<uint4*>(p.link_states + o64 + j) = o;
+        for (int j = 0; j < 64; j += 4)
+          *reinterpret_cast<float4*>(Ts + r * TS_LD + half * 64 + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(all_bar);
+        if (mbar_wait(all_bar, 0, p.err, 79)) {
+#pragma unroll 4
+          for (int i = ew; i < 128; i += 8) {
+            const int64_t grow = (int64_t)m0 + i;
+            if (grow >= p.M) break;
+            float4 t = *reinterpret_cast<const float4*>(Ts + i * TS_LD + lane * 4);
+            const int64_t o = grow * 128 + lane * 4;
+            if (p.T_out) *reinterpret_cast<float4*>(p.T_out + o) = t;
+            if (p.LP) {
+              if (p.lp_accumulate) {
+                const float4 a = *reinterpret_cast<const float4*>(p.LP + o);
+                t.x += a.x; t.y += a.y; t.z += a.z; t.w += a.w;
+              }
+              *reinterpret_cast<float4*>(p.LP + o) = t;
+              if (p.link_states) *reinterpret_cast<uint2*>(p.link_states + o) = make_uint2(lm_pack(t.x, t.y), lm_pack(t.z, t.w));
             }
           }
         }
@@ -246,12 +247,23 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
             for (int j = 0; j < 64; ++j) v[j] *= rstd;
           }
-          if (ok && valid) {
+          // the same way out for the bf16 rows: staged behind the fp32 tile, then whole 256-byte rows per warp
+          constexpr int TH_LD = 136;                                 // bf16 per staged row (272 bytes: 16-byte aligned, spread banks)
+          __nv_bfloat16* Th = reinterpret_cast<__nv_bfloat16*>(smem + 128 * TS_LD * 4);
 #pragma unroll
-            for (int j = 0; j < 64; j += 8) {
-              uint4 o;
-              o.x = lm_pack(v[j], v[j + 1]); o.y = lm_pack(v[j + 2], v[j + 3]); o.z = lm_pack(v[j + 4], v[j + 5]); o.w = lm_pack(v[j + 6], v[j + 7]);
-              *reinterpret_cast<uint4*>(p.That_next + o64 + j) = o;
+          for (int j = 0; j < 64; j += 8) {
+            uint4 o;
+            o.x = lm_pack(v[j], v[j + 1]); o.y = lm_pack(v[j + 2], v[j + 3]); o.z = lm_pack(v[j + 4], v[j + 5]); o.w = lm_pack(v[j + 6], v[j + 7]);
+            *reinterpret_cast<uint4*>(Th + r * TH_LD + half * 64 + j) = o;
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(all_bar);
+          if (ok && mbar_wait(all_bar, 1, p.err, 80)) {
+#pragma unroll 4
+            for (int i = ew; i < 128; i += 8) {
+              const int64_t grow = (int64_t)m0 + i;
+              if (grow >= p.M) break;
+              *reinterpret_cast<uint2*>(p.That_next + grow * 128 + lane * 4) = *reinterpret_cast<const uint2*>(Th + i * TH_LD + lane * 4);
             }
           }
         }
