@@ -89,22 +89,26 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
 
 // Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
 //   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
-// grid (B, H * ell / MERGE_ROWS), 128 threads: each warp takes rows of the block's MERGE_ROWS, a lane four consecutive
+// Blocks of 128 threads walk the (user, group of MERGE_ROWS rows) pairs with a grid stride (a few blocks per SM: when no
+// user has more than one chunk the launch is over as soon as the users have been looked at); within a pair each warp
+// takes rows, a lane four consecutive
 // columns at a time (128-bit reads of the partial accumulators, four chunks in flight).  d is a multiple of 8.  A user
 // without history gets zeros; a user with a single chunk was already written by the attention kernel (its blocks
 // return at once).
 constexpr int MERGE_ROWS = 8;
 __global__ void __launch_bounds__(128)
-k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, int H, const float* __restrict__ part_m,
+k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int B, int ell, int d, int H, const float* __restrict__ part_m,
                        const float* __restrict__ part_s, const float* __restrict__ part_acc,
                        __nv_bfloat16* __restrict__ Ohat) {
   const int HL = H * ell;
-  const int u = blockIdx.x;
-  const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
-  if (c1 - c0 == 1) return;
+  const int groups = (HL + MERGE_ROWS - 1) / MERGE_ROWS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row_end = min(HL, ((int)blockIdx.y + 1) * MERGE_ROWS);
-  for (int row = blockIdx.y * MERGE_ROWS + warp; row < row_end; row += 4) {
+  for (int64_t pair = blockIdx.x; pair < (int64_t)B * groups; pair += gridDim.x) {
+  const int u = (int)(pair / groups), grp = (int)(pair % groups);
+  const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
+  if (c1 - c0 == 1) continue;
+  const int row_end = min(HL, (grp + 1) * MERGE_ROWS);
+  for (int row = grp * MERGE_ROWS + warp; row < row_end; row += 4) {
     const int h = row / ell, l = row % ell;
     __nv_bfloat16* dst = Ohat + ((int64_t)u * ell + l) * (H * d) + h * d;
     float M = -INFINITY;
@@ -141,14 +145,16 @@ k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int ell, int d, 
       *reinterpret_cast<uint2*>(dst + i) = o;
     }
   }
+  }
 }
 
 lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
                                         const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
   if (B == 0) return LIME_OK;
   ProfScope _p("k_link_attn_merge_norm", st);
-  const dim3 grid((unsigned)B, (unsigned)((H * ell + MERGE_ROWS - 1) / MERGE_ROWS));
-  k_link_attn_merge_norm<<<grid, 128, 0, st>>>(chunk_start, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  const int64_t pairs = (int64_t)B * ((H * ell + MERGE_ROWS - 1) / MERGE_ROWS);
+  const int grid = (int)(pairs < (int64_t)kSMs * 8 ? pairs : (int64_t)kSMs * 8);
+  k_link_attn_merge_norm<<<grid, 128, 0, st>>>(chunk_start, B, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }
