@@ -267,7 +267,6 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       const int t = t_begin + g;
       const int b = tu.of(tile_start, p.B, t);
       const int row0 = off[b] + (t - tu.lo) * H2_TILE;
-      const bool valid = row0 + (int)r < off[b + 1];
       // ---- LayerNorm statistics of the tile (two lanes per token, 64 features each), then this row's constants
       float rstd_r = 1.f, mu_r = 0.f;
       if (LN) {
@@ -404,7 +403,7 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(u_ready);
-      // ---- this thread's 64 columns of its S' row -> (LayerNorm) -> bf16 -> global (one 128-byte line per thread)
+      // ---- this thread's 64 columns of its S' row -> (LayerNorm) -> bf16 -> staged in the P/U buffer -> whole rows to global
       if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 34)) { ok = false; break; }
       tc_fence_after();
       float v[64];
@@ -440,15 +439,30 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
 #pragma unroll
         for (int j = 0; j < 64; ++j) v[j] = (v[j] - mu) * rstd;
       }
-      if (valid) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + (int64_t)(row0 + (int)r) * H2_D + half * 64);
+      {
+        // A thread owns half a row (128 bytes): stored directly, every instruction would touch 32 lines.  S'(g) has
+        // consumed U, so the P/U buffer is free until the next tile's first P: the tile is staged there (row r at
+        // r * 256 bytes, 16-byte chunk c at position c ^ (r & 15) to spread the banks) and each warp then writes whole
+        // 256-byte rows.
+        uint8_t* stage = smem + H2_OFF_PU;
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8) {
           uint4 o;
           o.x = h2_pack(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = h2_pack(v[c8 * 8 + 2], v[c8 * 8 + 3]);
           o.z = h2_pack(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = h2_pack(v[c8 * 8 + 6], v[c8 * 8 + 7]);
-          dst[c8] = o;
+          *reinterpret_cast<uint4*>(stage + r * 256u + ((((uint32_t)(half * 8 + c8)) ^ (r & 15u)) << 4)) = o;
         }
+        if (!h2_group_sync(stats_bar, stats_uses, lane, p.err, 38)) { ok = false; break; }
+        const int row_end = off[b + 1];
+#pragma unroll 4
+        for (int i = rw; i < H2_TILE; i += H2_ROW_WARPS) {
+          if (row0 + i >= row_end) break;
+          const uint2 o = *reinterpret_cast<const uint2*>(stage + i * 256 + ((((uint32_t)lane >> 1) ^ ((uint32_t)i & 15u)) << 4) + (lane & 1) * 8);
+          *reinterpret_cast<uint2*>(p.out + (int64_t)(row0 + i) * H2_D + lane * 4) = o;
+        }
+        // the next tile's first P goes into the same buffer: with LayerNorm on the fly its statistics rendezvous comes
+        // first, otherwise wait here until every warp has copied its rows out
+        if (!LN && !h2_group_sync(stats_bar, stats_uses, lane, p.err, 40)) { ok = false; break; }
       }
     }
   }

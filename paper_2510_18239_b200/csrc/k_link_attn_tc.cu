@@ -484,6 +484,20 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
       if (lane == 0) mbar_arrive(o_free);
       const bool single = chunk_start[b + 1] - chunk_start[b] == 1;
       const int64_t prow = (int64_t)w.ci * p.HL + R;            // row of the per-chunk partials
+      // 4 x 4 transpose of 16-byte chunks inside each group of four lanes (two butterfly steps of warp shuffles)
+      auto xchg = [&](uint4& keep_lo, uint4& keep_hi, bool upper, int dist) {
+        // lanes with `upper` clear give away keep_hi and receive into it; lanes with it set give away keep_lo
+        uint4 send = upper ? keep_lo : keep_hi, recv;
+        recv.x = __shfl_xor_sync(0xffffffffu, send.x, dist); recv.y = __shfl_xor_sync(0xffffffffu, send.y, dist);
+        recv.z = __shfl_xor_sync(0xffffffffu, send.z, dist); recv.w = __shfl_xor_sync(0xffffffffu, send.w, dist);
+        if (upper) keep_lo = recv; else keep_hi = recv;
+      };
+      auto transpose4 = [&](uint4 (&t)[4]) {
+        xchg(t[0], t[1], (lane & 1) != 0, 1);
+        xchg(t[2], t[3], (lane & 1) != 0, 1);
+        xchg(t[0], t[2], (lane & 2) != 0, 2);
+        xchg(t[1], t[3], (lane & 2) != 0, 2);
+      };
       if (single) {
         // the whole history of this user was one chunk: normalise and write the attention rows directly
         const float inv = 1.0f / l_tot;
@@ -496,25 +510,27 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           tch[c8].z = la_pack((a[c8 * 8 + 4] - c_tot) * inv, (a[c8 * 8 + 5] - c_tot) * inv);
           tch[c8].w = la_pack((a[c8 * 8 + 6] - c_tot) * inv, (a[c8 * 8 + 7] - c_tot) * inv);
         }
-        auto xchg = [&](uint4& keep_lo, uint4& keep_hi, bool upper, int dist) {
-          // lanes with `upper` clear give away keep_hi and receive into it; lanes with it set give away keep_lo
-          uint4 send = upper ? keep_lo : keep_hi, recv;
-          recv.x = __shfl_xor_sync(0xffffffffu, send.x, dist); recv.y = __shfl_xor_sync(0xffffffffu, send.y, dist);
-          recv.z = __shfl_xor_sync(0xffffffffu, send.z, dist); recv.w = __shfl_xor_sync(0xffffffffu, send.w, dist);
-          if (upper) keep_lo = recv; else keep_hi = recv;
-        };
-        xchg(tch[0], tch[1], (lane & 1) != 0, 1);
-        xchg(tch[2], tch[3], (lane & 1) != 0, 1);
-        xchg(tch[0], tch[2], (lane & 2) != 0, 2);
-        xchg(tch[1], tch[3], (lane & 2) != 0, 2);
+        transpose4(tch);
         __nv_bfloat16* dst = p.Ohat + (int64_t)b * p.ell * (p.H * LA_D) + ohat_off;
 #pragma unroll
         for (int m = 0; m < 4; ++m) *reinterpret_cast<uint4*>(dst + (int64_t)m * (p.H * LA_D)) = tch[m];
       } else {
-        float4* dst = reinterpret_cast<float4*>(p.part_acc + prow * LA_D + col0);
+        // fp32 partial accumulator: this thread's 32 columns are two runs of four 16-byte chunks; after the transposes
+        // lane 4j+i holds chunk i of rows 4j..4j+3, so a store instruction writes whole 64-byte pieces of rows
+        float* dst = p.part_acc + ((int64_t)w.ci * p.HL + R4) * LA_D + col0 + (lane & 3) * 4;
 #pragma unroll
-        for (int j = 0; j < LA_COLS; j += 4)
-          dst[j / 4] = make_float4(a[j] - c_tot, a[j + 1] - c_tot, a[j + 2] - c_tot, a[j + 3] - c_tot);
+        for (int run = 0; run < 2; ++run) {
+          uint4 t[4];
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            const int j = run * 16 + c4 * 4;
+            t[c4] = make_uint4(__float_as_uint(a[j] - c_tot), __float_as_uint(a[j + 1] - c_tot), __float_as_uint(a[j + 2] - c_tot),
+                               __float_as_uint(a[j + 3] - c_tot));
+          }
+          transpose4(t);
+#pragma unroll
+          for (int m = 0; m < 4; ++m) *reinterpret_cast<uint4*>(dst + (int64_t)m * LA_D + run * 16) = t[m];
+        }
         if (part == 0) {
           p.part_m[prow] = p.silu ? 0.f : m_ref;        // log2 domain; equal weights for the chunks in SiLU mode
           p.part_s[prow] = l_tot;
