@@ -203,20 +203,30 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         __syncwarp();
         if (lane == 0) mbar_arrive(all_bar);
         if (mbar_wait(all_bar, 0, p.err, 79)) {
-#pragma unroll 4
-          for (int i = ew; i < 128; i += 8) {
-            const int64_t grow = (int64_t)m0 + i;
-            if (grow >= p.M) break;
-            float4 t = *reinterpret_cast<const float4*>(Ts + i * TS_LD + lane * 4);
-            const int64_t o = grow * 128 + lane * 4;
-            if (p.T_out) *reinterpret_cast<float4*>(p.T_out + o) = t;
-            if (p.LP) {
-              if (p.lp_accumulate) {
-                const float4 a = *reinterpret_cast<const float4*>(p.LP + o);
-                t.x += a.x; t.y += a.y; t.z += a.z; t.w += a.w;
+          // a warp takes rows ew, ew + 8, ...; the reads of the running sum for a batch of rows are issued together
+          constexpr int BATCH = 8;
+          const int n_valid = (int)(p.M - m0 < 128 ? p.M - m0 : 128);
+          const bool acc = p.LP != nullptr && p.lp_accumulate != 0;
+          for (int i0 = ew; i0 < 128; i0 += 8 * BATCH) {
+            float4 prev[BATCH];
+#pragma unroll
+            for (int k = 0; k < BATCH; ++k) {
+              const int i = i0 + 8 * k;
+              prev[k] = (acc && i < n_valid) ? *reinterpret_cast<const float4*>(p.LP + ((int64_t)m0 + i) * 128 + lane * 4)
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < BATCH; ++k) {
+              const int i = i0 + 8 * k;
+              if (i >= n_valid) continue;
+              float4 t = *reinterpret_cast<const float4*>(Ts + i * TS_LD + lane * 4);
+              const int64_t o = ((int64_t)m0 + i) * 128 + lane * 4;
+              if (p.T_out) *reinterpret_cast<float4*>(p.T_out + o) = t;
+              if (p.LP) {
+                t.x += prev[k].x; t.y += prev[k].y; t.z += prev[k].z; t.w += prev[k].w;
+                *reinterpret_cast<float4*>(p.LP + o) = t;
+                if (p.link_states) *reinterpret_cast<uint2*>(p.link_states + o) = make_uint2(lm_pack(t.x, t.y), lm_pack(t.z, t.w));
               }
-              *reinterpret_cast<float4*>(p.LP + o) = t;
-              if (p.link_states) *reinterpret_cast<uint2*>(p.link_states + o) = make_uint2(lm_pack(t.x, t.y), lm_pack(t.z, t.w));
             }
           }
         }
