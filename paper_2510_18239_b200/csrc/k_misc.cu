@@ -128,6 +128,34 @@ k_gather(const uint4* __restrict__ table, int64_t V, int row_vec, const int32_t*
 // its WORDS 16-byte words of the row in registers, the lanes of a row reduce the sum and then the squared
 // deviations with shuffles (two passes: exact mean first), and the normalised row is written once.  The loop runs
 // per warp-wide group of rows so that every lane takes part in the shuffles.
+// a 16-byte word of the storage type <-> floats (bf16: two elements per 32-bit lane, widened with a shift / a mask
+// and narrowed pairwise with one round-to-nearest conversion)
+template <typename T> struct Word16;
+template <> struct Word16<float> {
+  static __device__ __forceinline__ void unpack(const uint4& w, float (&x)[4]) {
+    x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y); x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&x)[4]) {
+    return make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
+  }
+};
+template <> struct Word16<__nv_bfloat16> {
+  static __device__ __forceinline__ void unpack(const uint4& w, float (&x)[8]) {
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) { x[2 * k] = __uint_as_float(u[k] << 16); x[2 * k + 1] = __uint_as_float(u[k] & 0xffff0000u); }
+  }
+  static __device__ __forceinline__ uint4 pack(const float (&x)[8]) {
+    uint32_t u[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const __nv_bfloat162 p2 = __floats2bfloat162_rn(x[2 * k], x[2 * k + 1]);
+      u[k] = *reinterpret_cast<const uint32_t*>(&p2);
+    }
+    return make_uint4(u[0], u[1], u[2], u[3]);
+  }
+};
+
 template <typename T, int LANES, int WORDS>
 __global__ void __launch_bounds__(256)
 k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, float eps, const int32_t* __restrict__ ids,
@@ -162,9 +190,9 @@ k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, floa
       float sum = 0.f;
 #pragma unroll
       for (int i = 0; i < WORDS; ++i) {
-        const T* e = reinterpret_cast<const T*>(&w[k][i]);
+        Word16<T>::unpack(w[k][i], x[i]);
 #pragma unroll
-        for (int j = 0; j < PER; ++j) { x[i][j] = Store<T>::ld(e + j); sum += x[i][j]; }
+        for (int j = 0; j < PER; ++j) sum += x[i][j];
       }
 #pragma unroll
       for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -174,7 +202,7 @@ k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, floa
       for (int i = 0; i < WORDS; ++i) {
         if (sub + i * LANES < row_vec) {
 #pragma unroll
-          for (int j = 0; j < PER; ++j) { const float c = x[i][j] - mu; var = fmaf(c, c, var); }
+          for (int j = 0; j < PER; ++j) { x[i][j] -= mu; var = fmaf(x[i][j], x[i][j], var); }
         }
       }
 #pragma unroll
@@ -187,9 +215,9 @@ k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, floa
           if (v < row_vec) {
             uint4 o4 = make_uint4(0, 0, 0, 0);              // an id outside [0, V) gives a zero row, as in k_gather
             if (ok[k]) {
-              T* e = reinterpret_cast<T*>(&o4);
 #pragma unroll
-              for (int j = 0; j < PER; ++j) Store<T>::st(e + j, (x[i][j] - mu) * rstd);
+              for (int j = 0; j < PER; ++j) x[i][j] *= rstd;
+              o4 = Word16<T>::pack(x[i]);
             }
             out[t[k] * row_vec + v] = o4;
           }
