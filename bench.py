@@ -78,6 +78,10 @@ def kernel_models(wl: synth.Workload, total_tokens: int, cand_heads: int = 1):
     }
 
 
+NOMINAL_HBM_GBS = 8000.0        # B200 HBM3e, vendor figure (7.7 TB/s on HGX boards); context beside the measured copy peak
+NOMINAL_BF16_TFLOPS = 2250.0    # dense bf16, vendor figure
+
+
 def roofline_entry(mdl, ms, pk):
     """Achieved rate of `ms` milliseconds of kernel time against the roofline that bounds it."""
     t = ms * 1e-3
@@ -90,10 +94,14 @@ def roofline_entry(mdl, ms, pk):
     bound = max(floors, key=floors.get)
     if bound == "hbm":
         ach = mdl["bytes"] / t / 1e9
-        return dict(bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"])
+        return dict(bound="hbm", achieved=ach, peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"],
+                    frac_of_nominal=ach / NOMINAL_HBM_GBS)
     peak = FP32_ALU_TFLOPS if bound == "alu" else pk["bf16_tflops_sustained"]
     ach = mdl["flops"] / t / 1e12
-    return dict(bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
+    r = dict(bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak)
+    if bound == "tensor":
+        r["frac_of_nominal"] = ach / NOMINAL_BF16_TFLOPS
+    return r
 
 
 def model_for(name, models):
