@@ -15,6 +15,10 @@
 // second block of the same tokens finds them in L2).  Online softmax whose reference maximum is only raised
 // when the true maximum exceeds it by more than 8 (then the accumulator row is rescaled in TMEM), so most tiles need
 // no correction pass.  With LN = false the rows of X are LayerNorm-ed already and the corrections vanish.
+// With `silu` set the activation is SiLU(s) / N(U) (Algorithms 1-2): one pass per tile, no maximum, no row sums; the
+// divisor is the number of keys, and per-chunk partials are summed with equal weights.
+// Shared memory: three token stages, the folded queries of the current user, two P' buffers (the second MMA of a
+// tile runs while the next tile's P' is written).
 //
 // Persistent CTAs walk (user, chunk-of-history) items.  Warp roles: warp 0 TMA producer (runs ahead across items),
 // warp 1 MMA issuer, warps 2-17 softmax: four threads per (head, link) row, each owning 32 of the tile's 128 token
