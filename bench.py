@@ -252,8 +252,8 @@ NCU_TRAFFIC = {
     # profiles/k_score_tc_bf16_baseline.md: 169.9 MB read + 4.0-4.5 MB written per launch
     ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
     # profiles/xor_layer_kernels_bf16_baseline.md: 33.7 MB (layer 1) and 42.1 MB (layer 2) read + written; average per launch
-    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "8115f5c98cad9cbd"},
-    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.5e6, "source": "k_hist_update_tc.cu", "sha": "5d823b7efc1ff4d8"},
+    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "756d8af8ad9dd54b"},
+    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.5e6, "source": "k_hist_update_tc.cu", "sha": "cbdc6b1690b70517"},
     # profiles/k_score_gather_tc_bf16_baseline.md: 170.0 MB read + 3.9 MB written per launch
     ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 173.9e6, "source": "k_score_gather_tc.cu", "sha": "4daad32675f4aff5"},
 }
