@@ -180,13 +180,14 @@ def mha(Q: np.ndarray, K: np.ndarray, V: np.ndarray, Wq, Wk, Wv, cfg: OracleConf
 # XOR attention: Eq. 6 (dense, masked) and Eq. 7 (two block attentions)
 # --------------------------------------------------------------------------- #
 def xor_mask_and_denominator(i: int, j: int, n_s: int, n_t: int):
-    """Algorithm 1: query i, key j over X = E (+) L^C with n_s source rows then n_t target rows.
-    Attend iff exactly one of them is a source row; normalise by the size of the opposite partition."""
-    is_src_q = i < n_s
-    is_src_k = j < n_s
-    m = is_src_q != is_src_k
-    dnm = n_t if is_src_q else n_s
-    return m, dnm
+    """M_xor under Eq. 6, for X = E (+) L^C: rows 0 .. n_s-1 form the history partition, rows n_s .. n_s+n_t-1 the link
+    partition.  Query row i may attend to key row j exactly when the two lie in different partitions ("attend to one
+    another only"), and the SiLU form divides a query's row by the number of keys it can attend to, i.e. the size of
+    the partition the query is NOT in (Algorithm 1's normaliser)."""
+    sizes = (n_s, n_t)
+    partition = lambda row: 0 if row < n_s else 1
+    attends = partition(i) != partition(j)
+    return attends, sizes[1 - partition(i)]
 
 
 def xora_dense(E: np.ndarray, LC: np.ndarray, Wq, Wk, Wv, cfg: OracleConfig) -> np.ndarray:

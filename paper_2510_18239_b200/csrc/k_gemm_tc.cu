@@ -1,8 +1,9 @@
 // Link-side preparation GEMM of the XOR layers on tcgen05 (bf16 in, fp32 accumulate in TMEM).
 //
-//   PREP   LN(T) [rows x d] . Wprep [d x 4*H*128]  -> folded queries Q2, folded keys K2 (+ their row sums) and the
-//          folded gate / up operands G2t, U2t that the streaming kernels contract against the history (Eq. 7);
-//          weights folded once at set-up, see k_link_prep.cu
+//   PREP   LN(T) [rows x d] . Wprep [d x N]  -> folded queries Q2, folded keys K2 (+ their row sums) and either the
+//          folded gate / up operands G2t, U2t (N = 2*H*d + 2*H*f) or the plain link values V[T], stored transposed
+//          (N = 2*H*d + d), that the streaming kernels contract against the history (Eq. 7); weights folded once at
+//          set-up, see k_link_prep.cu.  d and f are multiples of 128.
 // One CTA per 128-row x 128-column output tile: warp 0 streams K blocks of A and B with TMA through a stage ring,
 // warp 1 issues the MMAs, warps 2-5 (one thread per output row = TMEM lane) run the epilogue.  The GatedMLP on the
 // link rows lives in k_link_mlp_tc.cu.
@@ -22,8 +23,9 @@ struct GemmParams {
   int stages;
   // PREP
   int ell, H, shared_rows;          // rows are (user, link): user = row / ell
-  __nv_bfloat16 *Q2, *K2, *G2t, *U2t;
-  float *cQ, *cK;
+  int d, f, plain_v;                // output widths; plain_v: the third segment is V[T] (d columns) instead of G2 | U2
+  __nv_bfloat16 *Q2, *K2, *G2t, *U2t, *V2t;
+  float *cQ, *cK;                   // row sums of Q2 / K2 (only with d = 128: one n-tile per row)
   int* err;
 };
 
@@ -107,13 +109,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
       tc_fence_after();
       const bool valid = row < p.M;
       if (EPI == GM_EPI_PREP) {
-        // n-tile -> (segment, head); row -> (user, link)
-        const int seg = nt / p.H, h = nt % p.H;
+        // n-tile -> (segment, head, 128-column part); row -> (user, link)
+        const int n0 = nt * 128, qk_cols = 2 * p.H * p.d;
         const int64_t u = row / p.ell;
         const int l = (int)(row % p.ell);
         const int HL = p.H * p.ell;
-        if (seg < 2) {
-          __nv_bfloat16* dst = (seg == 0 ? p.Q2 : p.K2) + ((u * HL) + h * p.ell + l) * 128;
+        if (n0 < qk_cols) {
+          const int seg = n0 / (p.H * p.d), h = (n0 / p.d) % p.H, i0 = n0 % p.d;
+          __nv_bfloat16* dst = (seg == 0 ? p.Q2 : p.K2) + ((u * HL) + h * p.ell + l) * p.d + i0;
           float rs = 0.f;
 #pragma unroll
           for (int c = 0; c < 128; c += 16) {
@@ -130,10 +133,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               *reinterpret_cast<uint4*>(dst + c + 8) = o1;
             }
           }
-          if (valid) (seg == 0 ? p.cQ : p.cK)[u * HL + h * p.ell + l] = rs;
+          float* cs = seg == 0 ? p.cQ : p.cK;
+          if (valid && cs != nullptr) cs[u * HL + h * p.ell + l] = rs;
         } else {
-          // transposed store: out[user][n][(h,l)]
-          __nv_bfloat16* dst = (seg == 2 ? p.G2t : p.U2t) + u * 128 * HL + h * p.ell + l;
+          // transposed stores: G2t / U2t [user][f][(h, l)], or V2t [user][d][l]
+          __nv_bfloat16* dst;
+          int64_t ld;
+          if (p.plain_v) {
+            dst = p.V2t + (u * p.d + (n0 - qk_cols)) * p.ell + l;
+            ld = p.ell;
+          } else {
+            const int n1 = n0 - qk_cols;
+            const int seg = n1 / (p.H * p.f), h = (n1 / p.f) % p.H, i0 = n1 % p.f;
+            dst = (seg == 0 ? p.G2t : p.U2t) + (u * p.f + i0) * HL + h * p.ell + l;
+            ld = HL;
+          }
 #pragma unroll
           for (int c = 0; c < 128; c += 16) {
             float v[16];
@@ -141,7 +155,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             tmem_wait_ld();
             if (valid) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) dst[(int64_t)(c + j) * HL] = __float2bfloat16_rn(v[j]);
+              for (int j = 0; j < 16; ++j) dst[(int64_t)(c + j) * ld] = __float2bfloat16_rn(v[j]);
             }
           }
         }
@@ -179,11 +193,14 @@ static lime_status launch_gemm(const void* A, int64_t M, int K, const void* Bt, 
 
 lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st) {
   GemmParams p{};
-  p.ell = a.ell; p.H = a.H; p.Q2 = (__nv_bfloat16*)a.Q2; p.K2 = (__nv_bfloat16*)a.K2; p.G2t = (__nv_bfloat16*)a.G2t;
-  p.U2t = (__nv_bfloat16*)a.U2t; p.cQ = a.cQ; p.cK = a.cK; p.err = a.err;
-  // segments: Q2 | K2 | G2 | U2, H n-tiles each; the last layer needs only the queries
-  const int n_tiles = (a.need_hist ? 4 : 1) * a.H;
-  return launch_gemm<GM_EPI_PREP, 128>(a.A, a.M, 128, a.Bt, 4 * a.H * 128, n_tiles, p, "k_gemm_tc_prep", st);
+  p.ell = a.ell; p.H = a.H; p.d = a.K; p.f = a.f; p.plain_v = a.plain_v;
+  p.Q2 = (__nv_bfloat16*)a.Q2; p.K2 = (__nv_bfloat16*)a.K2; p.G2t = (__nv_bfloat16*)a.G2t;
+  p.U2t = (__nv_bfloat16*)a.U2t; p.V2t = (__nv_bfloat16*)a.V2t; p.cQ = a.cQ; p.cK = a.cK; p.err = a.err;
+  if (a.K % 128 || a.f % 128 || a.K < 128) return LIME_UNSUPPORTED_SHAPE;
+  // column segments: Q2 | K2 | (G2 | U2, or V); the last layer needs only the queries
+  const int cols_all = 2 * a.H * a.K + (a.plain_v ? a.K : 2 * a.H * a.f);
+  const int n_tiles = (a.need_hist ? cols_all : a.H * a.K) / 128;
+  return launch_gemm<GM_EPI_PREP, 128>(a.A, a.M, a.K, a.Bt, cols_all, n_tiles, p, "k_gemm_tc_prep", st);
 }
 
 }  // namespace lime

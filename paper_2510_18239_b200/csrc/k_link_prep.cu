@@ -18,26 +18,35 @@ __device__ __forceinline__ float w_at(const __nv_bfloat16* W, int r, int c, int 
   return W ? __bfloat162float(W[(int64_t)r * ld + c]) : (r == c ? 1.f : 0.f);
 }
 
-// WprepT [4*H*128 x d]  (B operand of the PREP GEMM: output column major, contraction index j contiguous)
+// WprepT (B operand of the PREP GEMM: one row per output column, contraction index j contiguous), row segments
+//   [H*d] folded queries | [H*d] folded keys | then, with `plain_v` clear, [H*f] folded gate | [H*f] folded up;
+//   with `plain_v` set, [d] rows of W_V^T (the link values V[T] = LN(T) W_V are then formed as they stand, for the
+//   kernels that mix values head by head and apply the GatedMLP weights afterwards)
 // WpostT [2f x H*d]     (B operand of the GLU GEMM on link rows)
 __global__ void k_fold_weights(const __nv_bfloat16* __restrict__ Wq, const __nv_bfloat16* __restrict__ Wk,
                                const __nv_bfloat16* __restrict__ Wv, const __nv_bfloat16* __restrict__ Wg,
-                               const __nv_bfloat16* __restrict__ Wu, int d, int H, int f, float scale,
+                               const __nv_bfloat16* __restrict__ Wu, int d, int H, int f, float scale, int plain_v,
                                __nv_bfloat16* __restrict__ WprepT, __nv_bfloat16* __restrict__ WpostT) {
   const int d_h = d / H;
-  const int n_prep = 4 * H * 128 * d, n_post = 2 * f * H * d;
+  const int rows_qk = 2 * H * d;
+  const int n_prep = (rows_qk + (plain_v ? d : 2 * H * f)) * d, n_post = 2 * f * H * d;
   for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < n_prep + n_post; idx += gridDim.x * blockDim.x) {
     float acc = 0.f;
     if (idx < n_prep) {
       const int R = idx / d, j = idx % d;
-      const int seg = R / (H * 128), h = (R / 128) % H, i = R % 128;
-      for (int k = h * d_h; k < (h + 1) * d_h; ++k) {
-        if (seg == 0) acc = fmaf(w_at(Wq, j, k, d), w_at(Wk, i, k, d), acc);
-        else if (seg == 1) acc = fmaf(w_at(Wk, j, k, d), w_at(Wq, i, k, d), acc);
-        else if (seg == 2) acc = fmaf(w_at(Wv, j, k, d), __bfloat162float(Wg[(int64_t)k * f + i]), acc);
-        else acc = fmaf(w_at(Wv, j, k, d), __bfloat162float(Wu[(int64_t)k * f + i]), acc);
+      if (R < rows_qk) {
+        const int seg = R / (H * d), h = (R / d) % H, i = R % d;
+        for (int k = h * d_h; k < (h + 1) * d_h; ++k)
+          acc = seg == 0 ? fmaf(w_at(Wq, j, k, d), w_at(Wk, i, k, d), acc) : fmaf(w_at(Wk, j, k, d), w_at(Wq, i, k, d), acc);
+        acc *= scale;
+      } else if (plain_v) {
+        acc = w_at(Wv, j, R - rows_qk, d);
+      } else {
+        const int R2 = R - rows_qk;
+        const int seg = R2 / (H * f), h = (R2 / f) % H, i = R2 % f;
+        const __nv_bfloat16* Wx = seg == 0 ? Wg : Wu;
+        for (int k = h * d_h; k < (h + 1) * d_h; ++k) acc = fmaf(w_at(Wv, j, k, d), __bfloat162float(Wx[(int64_t)k * f + i]), acc);
       }
-      if (seg < 2) acc *= scale;
       WprepT[idx] = __float2bfloat16_rn(acc);
     } else {
       const int e = idx - n_prep;
@@ -51,10 +60,10 @@ __global__ void k_fold_weights(const __nv_bfloat16* __restrict__ Wq, const __nv_
 }
 
 lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,
-                                int H, int f, float scale, void* WprepT, void* WpostT, cudaStream_t st) {
+                                int H, int f, float scale, int plain_v, void* WprepT, void* WpostT, cudaStream_t st) {
   ProfScope _p("k_fold_weights", st);
   k_fold_weights<<<kSMs * 2, 256, 0, st>>>((const __nv_bfloat16*)Wq, (const __nv_bfloat16*)Wk, (const __nv_bfloat16*)Wv,
-                                           (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, d, H, f, scale,
+                                           (const __nv_bfloat16*)Wg, (const __nv_bfloat16*)Wu, d, H, f, scale, plain_v,
                                            (__nv_bfloat16*)WprepT, (__nv_bfloat16*)WpostT);
   LIME_LAUNCH_CHECK("k_fold_weights");
   return LIME_OK;

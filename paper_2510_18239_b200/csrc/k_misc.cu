@@ -124,7 +124,8 @@ k_gather(const uint4* __restrict__ table, int64_t V, int row_vec, const int32_t*
   }
 }
 
-// out[t, :] = LayerNorm(table[ids[t], :]) (non-affine), in the storage type.  Same row-per-LANES mapping; a lane keeps
+// out[t, :] = LayerNorm(table[ids[t], :]) (non-affine), in the storage type (ids == NULL: the rows of `table` in order,
+// i.e. a plain LayerNorm pass over V = total rows).  Same row-per-LANES mapping; a lane keeps
 // its WORDS 16-byte words of the row in registers, the lanes of a row reduce the sum and then the squared
 // deviations with shuffles (two passes: exact mean first), and the normalised row is written once.  The loop runs
 // per warp-wide group of rows so that every lane takes part in the shuffles.
@@ -173,7 +174,7 @@ k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, floa
     for (int k = 0; k < ROWS; ++k) {
       t[k] = base + (int64_t)k * rows_per_block + threadIdx.x / LANES;
       live[k] = t[k] < total;
-      id[k] = live[k] ? __ldg(ids + t[k]) : 0;
+      id[k] = live[k] ? (ids != nullptr ? __ldg(ids + t[k]) : (int32_t)t[k]) : 0;   // no ids: row t of `table` itself
       ok[k] = live[k] && id[k] >= 0 && (int64_t)id[k] < V;
     }
     uint4 w[ROWS][WORDS];

@@ -41,11 +41,24 @@ static inline int elem_size(int dtype) { return dtype == LIME_F32 ? 4 : 2; }
 // Tokens per work item of the link<-history attention: a power of two in [lo, 2048] giving about three work items per
 // SM (`row_blocks` items per chunk).  Every chunk of a multi-chunk history costs a set of fp32 partials and a pipeline
 // refill, so long histories take long chunks.
-static int pick_chunk(int64_t total_tokens, int row_blocks, int lo) {
+static int pick_chunk(int64_t total_tokens, int row_blocks, int lo, int hi = 2048) {
   const int64_t target = total_tokens * row_blocks / (3 * kSMs);
   int c = lo;
-  while (c < 2048 && c < target) c <<= 1;
+  while (c < hi && c < target) c <<= 1;
   return c;
+}
+
+// Which kernels serve the XOR layers of this shape: 1 = the tensor-core kernels built for d = d_ff = 128, 2 = those
+// built for d = d_ff = 256, 0 = the generic CUDA-core path.
+static int tensor_core_mode(const lime_config& g, int d_ff) {
+  if (link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi) &&
+      (hist_update_tc_supported(g.dtype, g.d, d_ff, g.H, g.ell, g.phi, g.gated_mlp) ||
+       hist_update2_tc_supported(g.dtype, g.d, d_ff, g.H, g.ell, g.phi, g.gated_mlp)))
+    return 1;
+  if (link_attn_d256_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi) &&
+      hist_update_d256_tc_supported(g.dtype, g.d, d_ff, g.H, g.ell, g.phi, g.gated_mlp))
+    return 2;
+  return 0;
 }
 constexpr int kHistTile = 128;  // tokens per block of the history<-links attention
 
@@ -57,7 +70,7 @@ struct Workspace {
   int32_t *chunk_start, *tile_start, *chunk_user;
   float *part_m, *part_s, *part_acc;
   // tensor-core path: folded link-side operands (bf16) and their row sums
-  void *Q2, *K2, *G2t, *U2t;
+  void *Q2, *K2, *G2t, *U2t, *V2t;
   float *cQ, *cK;
   float2* row_stats;   // LayerNorm {rstd, mean} of the history rows of the layer being processed
   void *That, *Ohat, *UTb;   // LN(T) [B*ell x d], merged attention rows [B*ell x H*d], GLU output [B*ell x d_ff] (bf16)
@@ -79,9 +92,11 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.AT = (float*)take(ld); w.UT = (float*)take(lf); w.LP = (float*)take(ld); w.LS32 = (float*)take(ld);
   w.chunk_start = (int32_t*)take((size_t)(B + 1) * 4);
   w.tile_start = (int32_t*)take((size_t)(B + 1) * 4);
-  const bool tc_link = link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi);
-  // tensor-core path: at least 4 token tiles per work item, one item per 128-row block of H * ell
-  w.chunk = tc_link ? pick_chunk(total, (g.H * g.ell + 127) / 128, 512) : pick_chunk(total, 1, 64);
+  const bool tc_link = c->tc_mode != 0;
+  // tensor-core path: at least 4 token tiles per work item, one item per 128-row block of H * ell (at d = 256 a set of
+  // partials is 4 x larger and the batches served have many users, so chunks may be longer still)
+  w.chunk = c->tc_mode == 2 ? pick_chunk(total, (g.H * g.ell + 127) / 128, 512, 4096)
+                            : (tc_link ? pick_chunk(total, (g.H * g.ell + 127) / 128, 512) : pick_chunk(total, 1, 64));
   w.n_chunk_upper = (int)((total + w.chunk - 1) / w.chunk + B);
   w.n_tile_upper = (int)((total + kHistTile - 1) / kHistTile + B);
   w.chunk_user = (int32_t*)take((size_t)w.n_chunk_upper * 4);
@@ -92,6 +107,7 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   const size_t HL = (size_t)g.H * g.ell;
   w.Q2 = take((size_t)B * HL * g.d * 2); w.K2 = take((size_t)B * HL * g.d * 2);
   w.G2t = take((size_t)B * c->d_ff * HL * 2); w.U2t = take((size_t)B * c->d_ff * HL * 2);
+  w.V2t = take((size_t)B * g.d * g.ell * 2);
   w.cQ = (float*)take((size_t)B * HL * 4); w.cK = (float*)take((size_t)B * HL * 4);
   w.row_stats = (float2*)take((size_t)total * 8);
   w.That = take((size_t)B * g.ell * g.d * 2); w.Ohat = take((size_t)B * g.ell * g.H * g.d * 2);
@@ -100,29 +116,29 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   return w;
 }
 
-// True when the whole layer runs on the tensor-core kernels (bf16, d = d_ff = 128, H * ell = 128, softmax, GatedMLP).
+// True when the whole layer runs on the tensor-core kernels (their set-up data exists for this layer).
 static bool layer_on_tensor_cores(const Ctx* c, int layer) {
-  const lime_config& g = c->cfg;
-  return c->WoT[layer] && c->WprepT[layer] && c->WpostT[layer] && link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi) &&
-         (hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) ||
-          hist_update2_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp));
+  return c->tc_mode != 0 && c->WoT[layer] && c->WprepT[layer] && c->WpostT[layer] && (c->tc_mode == 1 || c->WguT[layer]);
 }
 
 // One XOR layer, tensor-core path: three link-row GEMMs around the two streaming attention kernels.
 // Link-side operands of one layer's two attention directions (folded through the weights, k_link_prep.cu).
 struct LinkOperands {
-  const void *Q2, *K2, *G2t, *U2t;
+  const void *Q2, *K2, *G2t, *U2t, *V2t;   // G2t / U2t with tc_mode 1, V2t with tc_mode 2
   const float *cQ, *cK;
   int shared;                 // one set for every user (T^0 = L) or one per user
 };
 
 // LN(links_in) -> bf16 -> PREP GEMM: the operands of `layer` for `rows` link rows, written to the given buffers.
 static lime_status make_link_operands(Ctx* c, int layer, const void* That, int64_t rows, int need_hist, void* Q2, void* K2,
-                                      void* G2t, void* U2t, float* cQ, float* cK, cudaStream_t st) {
+                                      void* G2t, void* U2t, void* V2t, float* cQ, float* cK, cudaStream_t st) {
   const lime_config& g = c->cfg;
   LinkGemmArgs gp{};
   gp.A = That; gp.M = rows; gp.K = g.d; gp.Bt = c->WprepT[layer]; gp.ell = g.ell; gp.H = g.H;
-  gp.need_hist = need_hist; gp.Q2 = Q2; gp.K2 = K2; gp.G2t = G2t; gp.U2t = U2t; gp.cQ = cQ; gp.cK = cK;
+  gp.f = c->d_ff; gp.plain_v = c->tc_mode == 2;
+  gp.need_hist = need_hist; gp.Q2 = Q2; gp.K2 = K2; gp.G2t = G2t; gp.U2t = U2t; gp.V2t = V2t;
+  // the row sums serve the LayerNorm folded into the d = 128 kernels; the d = 256 kernels read normalised rows
+  gp.cQ = c->tc_mode == 1 ? cQ : nullptr; gp.cK = c->tc_mode == 1 ? cK : nullptr;
   gp.err = c->dev_err;
   return launch_gemm_prep(gp, st);
 }
@@ -135,6 +151,13 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
                                  const Workspace& w, cudaStream_t st) {
   const lime_config& g = c->cfg;
   lime_status s;
+  if (c->tc_mode == 2 && hist_ln && total > 0) {
+    // the d = 256 kernels read LayerNorm-ed rows only: normalise the raw rows once into a scratch copy (what the
+    // fused lookup + LayerNorm would have stored)
+    if ((s = launch_gather_ln(g.dtype, hist_in, total, g.d, c->ln_eps, nullptr, total, w.Q, nullptr, st)) != LIME_OK) return s;
+    hist_in = w.Q;
+    hist_ln = 0;
+  }
   // O[T]: links attend over the stored history (keys = values = history rows), chunks merged and normalised
   LinkAttnArgs la{};
   la.hist = hist_in; la.total = total; la.Q2 = ops.Q2; la.cQ = ops.cQ; la.off = off; la.chunk_start = w.chunk_start; la.chunk_user = w.chunk_user; la.B = B;
@@ -142,17 +165,23 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
   la.ln = hist_ln; la.ln_eps = c->ln_eps; la.silu = g.phi == LIME_PHI_SILU; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
   la.err = c->dev_err;
   // the attention kernel forms the LayerNorm statistics of every history row anyway; the history update reuses them
-  const bool one_block_update = hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
+  const bool one_block_update = c->tc_mode == 1 && hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp);
   const bool pass_stats = hist_ln && hist_out && one_block_update && total > 0;
   la.stats_out = pass_stats ? w.row_stats : nullptr;
-  if ((s = launch_link_attn_tc(la, st)) != LIME_OK) return s;
+  if ((s = c->tc_mode == 2 ? launch_link_attn_d256_tc(la, st) : launch_link_attn_tc(la, st)) != LIME_OK) return s;
   if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
     return s;
   // T^j = GatedMLP(O[T]) with W_V folded into the gate / up weights, and what the next step needs from it
-  mlp.Ohat = w.Ohat; mlp.M = (int64_t)B * g.ell; mlp.K = g.H * g.d; mlp.WpostT = c->WpostT[layer]; mlp.WoT = c->WoT[layer];
+  mlp.Ohat = w.Ohat; mlp.M = (int64_t)B * g.ell; mlp.K = g.H * g.d; mlp.d = g.d; mlp.WpostT = c->WpostT[layer]; mlp.WoT = c->WoT[layer];
   mlp.ln = g.ln; mlp.ln_eps = c->ln_eps; mlp.err = c->dev_err;
   if ((s = launch_link_mlp_tc(mlp, st)) != LIME_OK) return s;
-  if (hist_out) {
+  if (hist_out && c->tc_mode == 2) {
+    HistUpdate256Args hu{};
+    hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = ops.K2; hu.V2t = ops.V2t; hu.WguT = c->WguT[layer];
+    hu.WoT = c->WoT[layer]; hu.off = off; hu.tile_start = w.tile_start; hu.B = B; hu.n_tile_upper = w.n_tile_upper; hu.H = g.H;
+    hu.shared = ops.shared; hu.out_ln = out_ln; hu.silu = g.phi == LIME_PHI_SILU; hu.ln_eps = c->ln_eps; hu.err = c->dev_err;
+    if ((s = launch_hist_update_d256_tc(hu, st)) != LIME_OK) return s;
+  } else if (hist_out) {
     // history attends back over the links; scores, per-head softmax, value mix and GatedMLP in one fused kernel
     HistUpdateArgs hu{};
     hu.hist_in = hist_in; hu.hist_out = hist_out; hu.total = total; hu.K2 = ops.K2; hu.G2t = ops.G2t; hu.U2t = ops.U2t;
@@ -175,9 +204,9 @@ static lime_status xor_layer_tc(Ctx* c, int layer, const void* hist_in, const in
   lime_status s;
   const int64_t link_rows = links_shared ? g.ell : (int64_t)B * g.ell;
   if ((s = launch_ln_rows_bf16(links_in, link_rows, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
-  if ((s = make_link_operands(c, layer, w.That, link_rows, hist_out != nullptr, w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, st)) != LIME_OK)
+  if ((s = make_link_operands(c, layer, w.That, link_rows, hist_out != nullptr, w.Q2, w.K2, w.G2t, w.U2t, w.V2t, w.cQ, w.cK, st)) != LIME_OK)
     return s;
-  LinkOperands ops{w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, links_shared};
+  LinkOperands ops{w.Q2, w.K2, w.G2t, w.U2t, w.V2t, w.cQ, w.cK, links_shared};
   LinkMlpArgs mlp{};
   mlp.T_out = links_out;
   return tc_layer_core(c, layer, hist_in, off, B, total, ops, hist_out, g.ln, 0, mlp, w, st);
@@ -196,11 +225,11 @@ static lime_status encode_user_tc(Ctx* c, const void* hist, bool hist_normalized
     const bool last = j == g.n_layers - 1;
     LinkOperands ops;
     if (j == 0 && !link_ctx) {
-      ops = LinkOperands{c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_cQ, c->sh_cK, 1};
+      ops = LinkOperands{c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_V2t, c->sh_cQ, c->sh_cK, 1};
     } else {
       if (j == 0 && (s = launch_ln_rows_bf16(link_ctx, BL, g.d, g.ln, c->ln_eps, w.That, st)) != LIME_OK) return s;
-      if ((s = make_link_operands(c, j, w.That, BL, !last, w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, st)) != LIME_OK) return s;
-      ops = LinkOperands{w.Q2, w.K2, w.G2t, w.U2t, w.cQ, w.cK, 0};
+      if ((s = make_link_operands(c, j, w.That, BL, !last, w.Q2, w.K2, w.G2t, w.U2t, w.V2t, w.cQ, w.cK, st)) != LIME_OK) return s;
+      ops = LinkOperands{w.Q2, w.K2, w.G2t, w.U2t, w.V2t, w.cQ, w.cK, 0};
     }
     LinkMlpArgs mlp{};
     mlp.LP = w.LP; mlp.lp_accumulate = j > 0;                                   // L^P = sum_j T^j  (Eq. 8)
@@ -388,8 +417,9 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)(cand_heads > 1 ? c->d_h : g.d));
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
-  for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = nullptr;
-  c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
+  c->tc_mode = tensor_core_mode(g, d_ff);
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = c->WguT[j] = nullptr;
+  c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = c->sh_V2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff, sizeof(float) * 2 * (size_t)c->ell_c * g.d);
   if (e == cudaSuccess) e = cudaMalloc(&c->keff_hl, 2 * (size_t)2 * c->ell_c * g.d);
@@ -415,9 +445,9 @@ lime_status lime_destroy(lime_ctx* ctx) {
   cudaFree(c->keff_hl);
   cudaFree(c->links32);
   cudaFree(c->dev_err);
-  for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); }
-  cudaFree(c->sh_That); cudaFree(c->sh_Q2); cudaFree(c->sh_K2); cudaFree(c->sh_G2t); cudaFree(c->sh_U2t); cudaFree(c->sh_cQ);
-  cudaFree(c->sh_cK);
+  for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); cudaFree(c->WguT[j]); }
+  cudaFree(c->sh_That); cudaFree(c->sh_Q2); cudaFree(c->sh_K2); cudaFree(c->sh_G2t); cudaFree(c->sh_U2t); cudaFree(c->sh_V2t);
+  cudaFree(c->sh_cQ); cudaFree(c->sh_cK);
   delete c;
   return LIME_OK;
 }
@@ -444,34 +474,43 @@ lime_status lime_set_weights(lime_ctx* ctx, const lime_weights* w, void* stream)
     return s;
   // tensor-core path: per layer, W_o as a K-major B operand ([d x d_ff], contraction index contiguous) and the
   // weight-only products that fold the history-side projections into the link rows
-  if ((hist_update_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp) ||
-       hist_update2_tc_supported(g.dtype, g.d, c->d_ff, g.H, g.ell, g.phi, g.gated_mlp)) &&
-      link_attn_tc_supported(g.dtype, g.d, g.H, g.ell, g.phi)) {
+  if (c->tc_mode != 0) {
+    const bool plain_v = c->tc_mode == 2;
+    const size_t prep_rows = 2 * (size_t)g.H * g.d + (plain_v ? (size_t)g.d : 2 * (size_t)g.H * c->d_ff);
+    auto need = [](void** p, size_t bytes) -> cudaError_t { return *p ? cudaSuccess : cudaMalloc(p, bytes); };
     for (int j = 0; j < g.n_layers; ++j) {
-      if (!c->WoT[j]) LIME_CUDA(cudaMalloc(&c->WoT[j], (size_t)g.d * c->d_ff * 2));
-      if (!c->WprepT[j]) LIME_CUDA(cudaMalloc(&c->WprepT[j], (size_t)4 * g.H * 128 * g.d * 2));
-      if (!c->WpostT[j]) LIME_CUDA(cudaMalloc(&c->WpostT[j], (size_t)2 * c->d_ff * g.H * g.d * 2));
+      LIME_CUDA(need(&c->WoT[j], (size_t)g.d * c->d_ff * 2));
+      LIME_CUDA(need(&c->WprepT[j], prep_rows * g.d * 2));
+      LIME_CUDA(need(&c->WpostT[j], (size_t)2 * c->d_ff * g.H * g.d * 2));
       if ((s = launch_transpose_bf16(w->Wo[j], c->d_ff, g.d, c->WoT[j], st)) != LIME_OK) return s;
+      if (plain_v) {
+        // [W_g | W_u]^T [2f x d]: the history update applies the GatedMLP weights as they stand
+        LIME_CUDA(need(&c->WguT[j], (size_t)2 * c->d_ff * g.d * 2));
+        if ((s = launch_transpose_bf16(w->Wg[j], g.d, c->d_ff, c->WguT[j], st)) != LIME_OK) return s;
+        if ((s = launch_transpose_bf16(w->Wu[j], g.d, c->d_ff, (char*)c->WguT[j] + (size_t)c->d_ff * g.d * 2, st)) != LIME_OK) return s;
+      }
       if ((s = launch_fold_weights(w->Wq[j], w->Wk[j], w->Wv[j], w->Wg[j], w->Wu[j], g.d, g.H, c->d_ff,
                                    // softmax: scores leave the fold scaled and in the log2 domain; SiLU(s) takes the raw scores
-                                   g.phi == LIME_PHI_SILU ? 1.0f : c->attn_scale * 1.4426950408889634f,
+                                   g.phi == LIME_PHI_SILU ? 1.0f : c->attn_scale * 1.4426950408889634f, plain_v ? 1 : 0,
                                    c->WprepT[j], c->WpostT[j], st)) != LIME_OK)
         return s;
     }
     // first-layer operands for the shared links T^0 = L: LN(L) through the PREP GEMM, once
     const size_t HL = (size_t)g.H * g.ell;
-    if (!c->sh_That) {
-      LIME_CUDA(cudaMalloc(&c->sh_That, (size_t)g.ell * g.d * 2));
-      LIME_CUDA(cudaMalloc(&c->sh_Q2, HL * g.d * 2));
-      LIME_CUDA(cudaMalloc(&c->sh_K2, HL * g.d * 2));
-      LIME_CUDA(cudaMalloc(&c->sh_G2t, (size_t)c->d_ff * HL * 2));
-      LIME_CUDA(cudaMalloc(&c->sh_U2t, (size_t)c->d_ff * HL * 2));
-      LIME_CUDA(cudaMalloc(&c->sh_cQ, HL * 4));
-      LIME_CUDA(cudaMalloc(&c->sh_cK, HL * 4));
+    LIME_CUDA(need(&c->sh_That, (size_t)g.ell * g.d * 2));
+    LIME_CUDA(need(&c->sh_Q2, HL * g.d * 2));
+    LIME_CUDA(need(&c->sh_K2, HL * g.d * 2));
+    if (plain_v) {
+      LIME_CUDA(need(&c->sh_V2t, (size_t)g.d * g.ell * 2));
+    } else {
+      LIME_CUDA(need(&c->sh_G2t, (size_t)c->d_ff * HL * 2));
+      LIME_CUDA(need(&c->sh_U2t, (size_t)c->d_ff * HL * 2));
     }
+    LIME_CUDA(need((void**)&c->sh_cQ, HL * 4));
+    LIME_CUDA(need((void**)&c->sh_cK, HL * 4));
     if ((s = launch_ln_rows_bf16(c->links32, g.ell, g.d, g.ln, c->ln_eps, c->sh_That, st)) != LIME_OK) return s;
-    if ((s = make_link_operands(c, 0, c->sh_That, g.ell, g.n_layers > 1, c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_cQ,
-                                c->sh_cK, st)) != LIME_OK)
+    if ((s = make_link_operands(c, 0, c->sh_That, g.ell, g.n_layers > 1, c->sh_Q2, c->sh_K2, c->sh_G2t, c->sh_U2t, c->sh_V2t,
+                                c->sh_cQ, c->sh_cK, st)) != LIME_OK)
       return s;
   }
   c->have_weights = true;

@@ -55,11 +55,13 @@ struct Ctx {
   float* keff;      // [ell x d] fp32: (L W_K^c) W_Q^c^T * cand_scale, the effective link keys of Eq. 4
   void* keff_hl;    // [2 ell x d] bf16: keff split into a rounded part and its remainder (tensor-core precompute)
   float* links32;   // [ell x d] fp32 copy of L (layer-1 link rows when no L^C is given)
+  int tc_mode;                   // 0: generic kernels; 1: tensor-core layer kernels at d = 128; 2: at d = 256
   void* WoT[LIME_MAX_LAYERS];    // tensor-core path, per layer (NULL otherwise): W_o transposed [d x d_ff] bf16,
-  void* WprepT[LIME_MAX_LAYERS]; //   folded PREP operand [4*H*128 x d], folded link-row GLU operand [2*d_ff x H*d]
-  void* WpostT[LIME_MAX_LAYERS];
+  void* WprepT[LIME_MAX_LAYERS]; //   folded PREP operand (k_link_prep.cu), folded link-row GLU operand [2*d_ff x H*d],
+  void* WpostT[LIME_MAX_LAYERS]; //   and (tc_mode 2) [W_g | W_u] transposed [2*d_ff x d]
+  void* WguT[LIME_MAX_LAYERS];
   // link-side operands of the first layer for the shared links T^0 = L (weights only, formed at lime_set_weights)
-  void *sh_That, *sh_Q2, *sh_K2, *sh_G2t, *sh_U2t;
+  void *sh_That, *sh_Q2, *sh_K2, *sh_G2t, *sh_U2t, *sh_V2t;
   float *sh_cQ, *sh_cK;
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
@@ -184,8 +186,9 @@ bool score_gather_tc_supported(const ScoreArgs& a);
 lime_status launch_score_gather_tc(const ScoreArgs& a, int* err, cudaStream_t st);
 
 // ---- tensor-core XOR layer (bf16, d = d_ff = 128, H * ell = 128) ----------------------------------------------
+// plain_v: WprepT's third segment is W_V^T (link values formed as they stand) instead of the folded gate / up products
 lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,
-                                int H, int f, float scale, void* WprepT, void* WpostT, cudaStream_t st);
+                                int H, int f, float scale, int plain_v, void* WprepT, void* WpostT, cudaStream_t st);
 lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, float eps, void* out, cudaStream_t st);
 lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
                                         const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st);
@@ -193,16 +196,17 @@ lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, c
 
 // link-row GEMMs on tensor cores (k_gemm_tc.cu); A [M x K] bf16 row-major, Bt [N x K] bf16 (weights, pre-folded)
 struct LinkGemmArgs {
-  const void* A; int64_t M; int K; const void* Bt; void* out;
-  int ell, H, need_hist;                       // PREP: rows are (user, link); need_hist = also K2 / G2t / U2t
-  void *Q2, *K2, *G2t, *U2t; float *cQ, *cK;   // PREP outputs
+  const void* A; int64_t M; int K; const void* Bt; void* out;   // K = d
+  int ell, H, need_hist;                       // PREP: rows are (user, link); need_hist = also K2 and G2t / U2t (or V2t)
+  int f, plain_v;                              // GatedMLP width; plain_v: V2t [users x d x ell] instead of G2t / U2t
+  void *Q2, *K2, *G2t, *U2t, *V2t; float *cQ, *cK;   // PREP outputs (cQ / cK nullable; only formed with d = 128)
   int* err;
 };
 lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st);
 
-// GatedMLP on link rows fused with its consumers (k_link_mlp_tc.cu); d = d_ff = 128
+// GatedMLP on link rows fused with its consumers (k_link_mlp_tc.cu); d = d_ff in {128, 256}
 struct LinkMlpArgs {
-  const void* Ohat; int64_t M; int K;          // attention rows [M x K = H*d] bf16
+  const void* Ohat; int64_t M; int K; int d;   // attention rows [M x K = H*d] bf16
   const void* WpostT; const void* WoT;         // folded [2f x H*d] and transposed [d x f] weights, bf16
   float* T_out;                                // nullable: the layer's link rows, fp32 [M x d]
   float* LP; int lp_accumulate;                // nullable running sum of Eq. 8 (0: assign, 1: add)
@@ -243,5 +247,24 @@ lime_status launch_hist_update_tc(const HistUpdateArgs& a, cudaStream_t st);
 // same step for H * ell in {256, 384, 512} (link-side operands streamed per tile, k_hist_update2_tc.cu)
 bool hist_update2_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
 lime_status launch_hist_update2_tc(const HistUpdateArgs& a, int H, cudaStream_t st);
+
+// ---- tensor-core XOR layer at d = d_ff = 256 (bf16, ell = 64, H in {2, 4, 8}; history rows LayerNorm-ed already) ----
+bool link_attn_d256_tc_supported(int dtype, int d, int H, int ell, int phi);
+lime_status launch_link_attn_d256_tc(const LinkAttnArgs& a, cudaStream_t st);   // a.ln must be 0
+
+struct HistUpdate256Args {
+  const void* hist_in; void* hist_out; int64_t total;
+  const void* K2;                       // folded link keys [users x H*ell x d] bf16
+  const void* V2t;                      // link values, transposed [users x d x ell] bf16
+  const void* WguT; const void* WoT;    // [W_g | W_u]^T [2f x d] and W_o^T [d x f], bf16
+  const int32_t* off; const int32_t* tile_start; int B, n_tile_upper;
+  int H, shared;
+  int out_ln;                           // 1: store LayerNorm(S') instead of S'
+  int silu;                             // 1: SiLU(s) / ell instead of the per-head softmax (Algorithm 2)
+  float ln_eps;
+  int* err;
+};
+bool hist_update_d256_tc_supported(int dtype, int d, int f, int H, int ell, int phi, int gated_mlp);
+lime_status launch_hist_update_d256_tc(const HistUpdate256Args& a, cudaStream_t st);
 
 }  // namespace lime

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import lime_oracle as O
 from paper_2510_18239_b200 import synth
 
 pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
@@ -24,7 +25,10 @@ def _both(Bd, dtype, ell, d, M, seed, proj):
     got = torch.empty_like(want)               # the caller owns every buffer, the output included
     Bd.lime_precompute_candidate_links_noalloc(dt, d, ell, 0.0, links, wq, wk, cand, got)
     torch.cuda.synchronize()
-    return got.float().cpu().numpy(), want.float().cpu().numpy()
+    # the expected value proper: the oracle's candidate->link weights (Eq. 4) on the same stored inputs
+    f64 = lambda t: None if t is None else t.float().cpu().numpy().astype(np.float64)
+    oracle = O.precompute_candidate_links(f64(cand), f64(links), O.OracleConfig(d=d, H=1, ell=ell, n_layers=1), f64(wq), f64(wk))
+    return got.float().cpu().numpy(), want.float().cpu().numpy(), oracle
 
 
 @pytest.mark.parametrize("dtype", [synth.BF16, synth.F32])
@@ -32,14 +36,18 @@ def test_noalloc_precompute_matches_context_path_twice_in_a_row(dtype):
     from paper_2510_18239_b200 import binding as Bd
     tol = 2e-5 if dtype == synth.F32 else 4e-3      # the tolerances of the precompute parity test
     # first call: projections present, 32 links; second call straight after: other weights, fewer links, no
-    # projections - stale scratch from the first call would show up here
-    got1, want1 = _both(Bd, dtype, 32, 128, 777, seed=11, proj=True)
+    # projections - stale scratch from the first call would show up here.  Every result is held against the oracle
+    # first, and against the context-based entry point second.
+    got1, want1, oracle1 = _both(Bd, dtype, 32, 128, 777, seed=11, proj=True)
+    assert np.abs(got1 - oracle1).max() <= tol
     assert np.abs(got1 - want1).max() <= tol
-    got2, want2 = _both(Bd, dtype, 16, 64, 300, seed=12, proj=False)
+    got2, want2, oracle2 = _both(Bd, dtype, 16, 64, 300, seed=12, proj=False)
+    assert np.abs(got2 - oracle2).max() <= tol
     assert np.abs(got2 - want2).max() <= tol
     assert np.abs(got2.sum(axis=1) - 1.0).max() <= 1e-2
     # the largest supported shape
-    got3, want3 = _both(Bd, dtype, 64, 256, 129, seed=13, proj=True)
+    got3, want3, oracle3 = _both(Bd, dtype, 64, 256, 129, seed=13, proj=True)
+    assert np.abs(got3 - oracle3).max() <= tol
     assert np.abs(got3 - want3).max() <= tol
 
 
