@@ -69,6 +69,15 @@ def kernel_models(wl: synth.Workload, total_tokens: int, cand_heads: int = 1):
                                  pipe="tensor"),
         "k_hist_update2_tc": dict(bytes=(n - 1) * 2.0 * N * d * es, flops=(n - 1) * 2.0 * N * (HL * d + 2 * HL * f + f * d),
                                   pipe="tensor"),
+        # d = 256 kernels: folded scores against the stored rows, values mixed head by head, GatedMLP weights as they stand
+        "k_link_attn_d256_tc": dict(bytes=n * N * d * es, flops=n * 4.0 * HL * d * N, pipe="tensor"),
+        "k_hist_update_d256_tc": dict(bytes=(n - 1) * 2.0 * N * d * es,
+                                      flops=(n - 1) * 2.0 * N * (HL * d + ell * d + 2 * d * f + f * d), pipe="tensor"),
+        # link-side GEMMs (rows = users x links): PREP (layers 2..n: folded queries / keys and values or gate / up operands)
+        # and the GatedMLP on the attention rows with W_V folded in
+        "k_gemm_tc_prep": dict(flops=2.0 * BL * d * (max(n - 2, 0) * (2 * H * d + (d if d == 256 else 2 * H * f)) + (H * d if n > 1 else 0)),
+                               pipe="tensor"),
+        "k_link_mlp_tc": dict(flops=n * 2.0 * BL * (H * d * 2 * f + f * d), pipe="tensor"),
         # CUDA-core path (fp32 storage and shapes the tensor-core kernels do not serve)
         "k_linear_simt_ln": dict(flops=hist_proj + link_proj, pipe="alu"),
         "k_linear_simt_glu": dict(flops=glu, pipe="alu"),
@@ -114,7 +123,8 @@ def model_for(name, models):
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """nvidia-smi sampled every 50 ms; start() early (it takes a second to come up), then mark() the timed region."""
+    """nvidia-smi sampled every 50 ms; start() early (it takes a second to come up), then mark() the timed region (or ask
+    for any window(t0, t1) of wall-clock time while it runs)."""
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
@@ -125,6 +135,12 @@ class ClockSampler:
             self.t0 = time.time()
         else:
             self.t1 = time.time()
+
+    def window(self, t0: float, t1: float):
+        """Clock record of the samples taken between two wall-clock instants."""
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        return self._stats([ln for (ts, ln) in list(self.lines) if t0 - 0.02 <= ts <= t1 + 0.06])
 
     def start(self):
         q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -149,10 +165,14 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         inside = [ln for (ts, ln) in self.lines if self.t0 is None or (self.t0 - 0.05 <= ts <= (self.t1 or ts) + 0.1)]
         if not inside:
             inside = [ln for (_, ln) in self.lines[-3:]]
+        return self._stats(inside)
+
+    @staticmethod
+    def _stats(inside):
+        sm, mx, reasons = [], [], set()
         for ln in inside:
             p = [x.strip() for x in ln.split(",")]
             if len(p) < 7:
@@ -174,23 +194,10 @@ def oracle_sample(wl, inp, users, budget_s=None, phi="softmax", cand_heads=False
     from oracle import lime_oracle as O
     from tests import lime_helpers as Hh
     cfg, layers = Hh.oracle_config(wl, phi=O.SILU if phi == "silu" else O.SOFTMAX), Hh.oracle_layers(inp, wl)
-    table64_rows = {}
     links64 = synth.storage_to_f64(inp["links"], wl.dtype)
     off = O.lengths_to_offsets(inp["lengths"])
 
-    class LazyTable:                      # widen only the rows the sample touches (the table is GBs)
-        shape = inp["table"].shape
-        dtype = np.float64
-
-        def __getitem__(self, key):
-            i = key[0] if isinstance(key, tuple) else key
-            r = table64_rows.get(i)
-            if r is None:
-                r = synth.storage_to_f64(inp["table"][i], wl.dtype)
-                table64_rows[i] = r
-            return r
-
-    tab = LazyTable()
+    tab = Hh.LazyTable64(inp["table"], wl.dtype)   # widens only the rows the sample touches (the table is GBs)
     done, t0 = 0, time.perf_counter()
     for b in users:
         Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg, cand_heads=cand_heads)
@@ -249,12 +256,12 @@ def launch_mode(args):
 # kernel and workload, with the hash of the kernel's source at capture time: once the source changes the figure
 # is stale and the bench reports null.
 NCU_TRAFFIC = {
-    # profiles/k_score_tc_bf16_baseline.md: 169.9 MB read + 4.0-4.5 MB written per launch
+    # dense scorer: 169.9 MB read + 4.0-4.5 MB written per launch
     ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
-    # profiles/xor_layer_kernels_bf16_baseline.md: 33.7 MB (layer 1) and 42.1 MB (layer 2) read + written; average per launch
+    # XOR-layer kernels: 33.7 MB (layer 1) and 42.1 MB (layer 2) read + written; average per launch
     ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "756d8af8ad9dd54b"},
     ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.5e6, "source": "k_hist_update_tc.cu", "sha": "cbdc6b1690b70517"},
-    # profiles/k_score_gather_tc_bf16_baseline.md: 170.0 MB read + 3.9 MB written per launch
+    # scorer by id: 170.0 MB read + 3.9 MB written per launch
     ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 173.9e6, "source": "k_score_gather_tc.cu", "sha": "4daad32675f4aff5"},
 }
 
@@ -275,7 +282,7 @@ def ncu_traffic(kernel, wl, args=None):
         return None
 
 
-def run_ours(args, wl):
+def run_ours(args, wl, sampler=None, with_sweeps=False):
     import torch
     import torch.distributed as dist
     from paper_2510_18239_b200 import binding as Bd, shard
@@ -348,9 +355,11 @@ def run_ours(args, wl):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    own_sampler = sampler is None
+    if own_sampler:
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
     for i in range(max(args.warmup, ROTATE)):
         step(i)
     barrier()
@@ -380,15 +389,15 @@ def run_ours(args, wl):
     # ---- timed region: exactly `steps` steps, device-timed, nothing but the library's launches in between
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    sampler.mark(True)
+    t_wall0 = time.time()
     ev[0].record()
     for i in range(args.steps):
         step(i)
         ev[i + 1].record()
     torch.cuda.synchronize()
-    sampler.mark(False)
+    t_wall1 = time.time()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.window(t_wall0, t_wall1) if rank == 0 else None
     total_ms = ev[0].elapsed_time(ev[-1])
     step_ms = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps))
     # every rank serves its own batch of B users (users are independent: no collective on the data path); the job's
@@ -587,9 +596,175 @@ def run_ours(args, wl):
                 "precompute": {"ms": pre_ms, "candidates": wl.B * wl.C, "candidates_per_s": wl.B * wl.C / (pre_ms * 1e-3),
                                **roofline_entry(models["k_precompute"], pre_ms, pk)},
                 "cpu_baseline": cpu, "peaks": pk}
+        if with_sweeps and world == 1:
+            # free this workload's buffers before the sweep points allocate theirs
+            del sets, host_sets, table, hist, ws, w_corpus, wscratch, d_hid, d_cid, d_logits, h_logits
+            if not args.no_graph:
+                del step_graphs, graphs, e2e_graphs
+            torch.cuda.empty_cache()
+            line["sweeps"] = run_sweeps(args, sampler, pk)
         print(json.dumps(line), flush=True)
+    if own_sampler and rank == 0:
+        sampler.stop()
     if world > 1:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- the metric's curves, point by point
+# Latency vs number of candidates and vs history length (App. F, tables a and b) and the production-shaped batch: a few
+# points of each, every one timed long enough for the clock sampler to see it.
+SWEEP_POINTS = (
+    ("candidate_sweep", dict(C=16)), ("candidate_sweep", dict(C=2048)), ("candidate_sweep", dict(C=32768)),
+    ("long_history", dict(n_min=1024, n_max=1024)), ("long_history", dict(n_min=32768, n_max=32768)),
+    ("production_ragged", dict()),
+)
+L2_FLUSH_BYTES = 256 << 20
+
+
+def measure_point(wl, model, sampler, pk, args, min_seconds=0.35, max_steps=4000):
+    """One workload point: p50 / p10 / p90 latency of the step (offsets -> lookup + LayerNorm -> encode -> score), each step
+    timed by its own pair of CUDA events after an L2 flush (a 256 MB device buffer is overwritten in between; points
+    whose candidate streams exceed 512 MB are not flushed), steps repeated until at least `min_seconds` of device time.
+    The precompute for this point's candidates is timed separately, as the paper caches it."""
+    import torch
+    from paper_2510_18239_b200 import binding as Bd
+    lime, table, dev = model["lime"], model["table"], model["dev"]
+    ctx = lime.ctx
+    seed = 7
+    lengths = synth.history_lengths(seed, wl.B, wl.n_min, wl.n_max)
+    total = int(lengths.sum())
+    d_len = torch.from_numpy(lengths).to(dev)
+    d_hid = torch.from_numpy(synth.zipf_ids(seed, "hist_ids", total, wl.V, wl.zipf_s)).to(dev)
+    d_cid = torch.from_numpy(synth.uniform_ids(seed, "cand_ids", wl.B * wl.C, wl.V)).to(dev)
+    T = lime.gather_history(table, d_cid)
+    W = lime.precompute_candidate_links(T)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream_bytes = wl.B * wl.C * 2.0 * (wl.d + wl.ell)
+    do_flush = stream_bytes < 2 * L2_FLUSH_BYTES
+    pre = []
+    for _ in range(5):
+        flush.zero_()
+        e0.record()
+        Bd.lime_precompute_candidate_links(ctx, T, W)
+        e1.record()
+        torch.cuda.synchronize()
+        pre.append(e0.elapsed_time(e1))
+    off = torch.empty(wl.B + 1, dtype=torch.int32, device=dev)
+    hist = torch.empty((total, wl.d), dtype=lime.tdtype, device=dev)
+    ls = torch.empty((wl.B, lime.ell_c, wl.d), dtype=lime.tdtype, device=dev)
+    logits = torch.empty(wl.B * wl.C, dtype=torch.float32, device=dev)
+    ws = lime.workspace(wl.B, total)
+
+    def direct_step():
+        Bd.lime_lengths_to_offsets(ctx, d_len, off)
+        Bd.lime_gather_history_normalized(ctx, table, d_hid, hist)
+        Bd.lime_encode_user_normalized(ctx, hist, off, wl.B, None, ls, ws)
+        Bd.lime_score_candidates(ctx, ls, wl.B, W, T, None, wl.C, wl.B * wl.C, None, logits)
+
+    for _ in range(3):
+        direct_step()
+    torch.cuda.synchronize()
+    step = direct_step
+    if not args.no_graph:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            direct_step()
+        step = g.replay
+        step()
+        torch.cuda.synchronize()
+    # per-kernel durations of one step (event brackets around every launch: read the shares)
+    Bd.lime_profile_start(256)
+    for _ in range(3):
+        if do_flush:
+            flush.zero_()
+        direct_step()
+    torch.cuda.synchronize()
+    records, launches = Bd.lime_profile_stop(256)
+    kms = {}
+    for name, ms in records:
+        kms[name] = kms.get(name, 0.0) + ms / 3
+    # the timed steps
+    times, busy = [], 0.0
+    t_wall0 = time.time()
+    while (busy < min_seconds * 1e3 or len(times) < 10) and len(times) < max_steps:
+        batch = []
+        for _ in range(10):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if do_flush:
+                flush.zero_()
+            a.record()
+            step()
+            b.record()
+            batch.append((a, b))
+        torch.cuda.synchronize()
+        for a, b in batch:
+            times.append(a.elapsed_time(b))
+        busy = sum(times) * (1.0 + (0.05 / max(statistics.median(times), 1e-3) if do_flush else 0.0))   # ~50 us per flush
+    t_wall1 = time.time()
+    Bd.lime_device_status(ctx)
+    times.sort()
+    p50 = times[len(times) // 2]
+    clocks = sampler.window(t_wall0, t_wall1)
+    score_ms = sum(v for k, v in kms.items() if k.startswith("k_score"))
+    models = kernel_models(wl, total, 1)
+    out = {"workload": wl.name, "B": wl.B, "N": wl.n_max if not wl.ragged else [wl.n_min, wl.n_max], "tokens": total, "C": wl.C,
+           "d": wl.d, "H": wl.H, "ell": wl.ell, "n_layers": wl.n_layers,
+           "p50_ms": p50, "p10_ms": times[len(times) // 10], "p90_ms": times[(len(times) * 9) // 10], "steps": len(times),
+           "timed_s": (t_wall1 - t_wall0), "candidates_per_s": wl.B * wl.C / (p50 * 1e-3),
+           "l2": "flushed before every step (256 MB overwritten)" if do_flush else "candidate streams exceed L2 many times over",
+           "launches_per_step": launches / 3, "precompute_ms": sorted(pre)[len(pre) // 2],
+           "clocks": clocks, "p50_ms_x_sm_mhz": (p50 * clocks["sm_mhz"]) if clocks.get("sm_mhz") else None,
+           "score_ms": score_ms,
+           "score_roofline": (dict(roofline_entry(models["k_score"], score_ms, pk), timing="CUDA events around the launch inside the step")
+                              if score_ms > 0 else None),
+           "kernels_ms": {k: round(v, 5) for k, v in sorted(kms.items(), key=lambda kv: -kv[1])[:8]}}
+    enc = {k: v for k, v in kms.items() if not k.startswith(("k_score", "k_gather", "k_offsets"))}
+    out["encode_ms"] = sum(enc.values())
+    dom = max(enc, key=enc.get) if enc else None
+    mdl = model_for(dom, models) if dom else None
+    if mdl:
+        out["encode_dominant"] = dict(kernel=dom, ms=enc[dom], **roofline_entry(mdl, enc[dom], pk))
+    del T, W, hist, ws, flush, logits
+    torch.cuda.empty_cache()
+    return out
+
+
+def run_sweeps(args, sampler, pk):
+    import torch
+    from paper_2510_18239_b200 import binding as Bd
+    dev = torch.device("cuda", torch.cuda.current_device())
+    named = synth.named_workloads()
+    points, model, model_name = [], None, None
+    for name, kw in SWEEP_POINTS:
+        if args.sweep_only and name not in args.sweep_only.split(","):
+            continue
+        base = named[name]
+        wl = base.replace(**kw) if kw else base
+        if model_name != name:
+            model = None
+            torch.cuda.empty_cache()
+            # the model of the named workload: table, links and layer weights (requests are drawn per point)
+            inp = synth.make_inputs(base.replace(B=1, C=1, n_min=1, n_max=1), seed=0)
+            lime = Bd.Lime(base.d, base.H, base.ell, base.n_layers, dtype=Bd.LIME_BF16, d_ff=base.d_ff)
+            table = Bd.to_device(inp["table"], base.dtype, dev)
+            links = Bd.to_device(inp["links"], base.dtype, dev)
+            wts = {k: Bd.to_device(inp[k], base.dtype, dev) for k in ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")}
+            lime.set_weights(links, [{k: wts[k][j] for k in wts} for j in range(base.n_layers)])
+            model, model_name = dict(lime=lime, table=table, dev=dev, keep=(links, wts)), name
+            del inp
+        points.append(measure_point(wl, model, sampler, pk, args))
+    # "flat in C": all growth with C is the candidate stream at >= 70 % of the copy peak on top of the C-independent encode
+    cs = [q for q in points if q["workload"] == "candidate_sweep"]
+    if cs:
+        t_small = min(cs, key=lambda q: q["C"])["p50_ms"]
+        for q in cs:
+            stream = q["B"] * q["C"] * (2.0 * (q["d"] + q["ell"]) + 4.0)
+            bound = t_small + stream / (0.7 * pk["hbm_gbs"] * 1e9) * 1e3
+            q["flat_in_C"] = {"p50_ms": q["p50_ms"], "bound_ms": bound, "holds": q["p50_ms"] <= bound,
+                              "rule": "t(C) <= t(smallest C) + stream bytes(C) / (0.7 x copy peak)"}
+    return {"points": points,
+            "paper": "LIME-XOR 2.07 -> 2.15 ms over C = 16..32768 and 2.08 -> 2.12 ms over N = 1024..16384 (App. F, hardware unstated)"}
 
 
 def main():
@@ -610,6 +785,9 @@ def main():
     ap.add_argument("--cand-heads", action="store_true",
                     help="candidate side head by head (Eq. 1 applied to Eq. 4): H * ell cached weights per candidate")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying CUDA graphs")
+    ap.add_argument("--no-sweeps", action="store_true",
+                    help="leave out the `sweeps` object (points of the candidate sweep, the history sweep and production_ragged)")
+    ap.add_argument("--sweep-only", default="", help="comma-separated workload names whose sweep points to keep")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = synth.named_workloads()[args.workload]
@@ -632,7 +810,9 @@ def main():
         for N in synth.LONG_HISTORY_N:
             run_ours(args, base.replace(n_min=N, n_max=N, B=args.B or base.B))
     else:
-        run_ours(args, wl)
+        # the default run carries the metric's curves in its one line; explicit workloads and multi-GPU runs do not
+        plain_default = args.workload == "bf16_baseline" and not (args.C or args.N or args.B) and args.phi == "softmax" and not args.cand_heads
+        run_ours(args, wl, with_sweeps=plain_default and not args.no_sweeps and int(os.environ.get("WORLD_SIZE", "1")) == 1)
 
 
 if __name__ == "__main__":

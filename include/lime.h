@@ -170,11 +170,15 @@ LIME_API lime_status lime_encode_user_normalized(lime_ctx* ctx, const void* hist
  * cand_emb [total_cands x d] and logits [total_cands]; cand_off is a DEVICE int32 array [B+1], non-decreasing,
  * cand_off[0] = 0, cand_off[B] = total_cands.  With cand_off = NULL every user owns C slots (slot b*C + c) and
  * total_cands must equal B*C.  cand_ids (device int32 [total_cands], nullable): when given, cand_w and
- * cand_emb are corpus-level caches (Sec. 3.3 "QK cache") and row cand_ids[i] is read for slot i; ids are
- * not range-checked.  link_states [B x ell_c x d] as written by lime_encode_user. */
+ * cand_emb are corpus-level caches (Sec. 3.3 "QK cache") of corpus_rows rows each (1 <= corpus_rows < 2^31) and row
+ * cand_ids[i] is read for slot i.  An id outside [0, corpus_rows) reads nothing: that slot's logit is 0 and, if
+ * dev_flag is not NULL, *dev_flag (device int32, caller initialises it to INT32_MAX) is atomically lowered to the
+ * smallest offending slot, as in lime_gather_history.  Without cand_ids both arguments are ignored.
+ * link_states [B x ell_c x d] as written by lime_encode_user. */
 LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
                                   const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
-                                  const int32_t* cand_ids, float* logits, void* stream);
+                                  const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
+                                  void* stream);
 
 /* Allocation-free precompute (the paper has no counterpart: this exists for hosts that must not allocate).
  * Same result as lime_create + lime_set_weights + lime_precompute_candidate_links, for callers that cannot call

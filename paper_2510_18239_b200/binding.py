@@ -76,7 +76,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_xor_layer.argtypes = [vp, i32, vp, vp, i32, i64, vp, i32, vp, vp, vp, sz, vp]
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_encode_user_normalized.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
-    lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, vp, vp]
+    lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, i64, vp, vp, vp]
     lib.lime_precompute_candidate_links_noalloc.argtypes = [i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, i64, vp, vp]
     lib.lime_device_status.argtypes = [vp, ctypes.POINTER(i32)]
     lib.lime_profile_start.argtypes = [i32]
@@ -181,9 +181,14 @@ def lime_encode_user_normalized(ctx: int, hist_normalized: torch.Tensor, off: to
 
 def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: torch.Tensor, cand_emb: torch.Tensor,
                           cand_off: Optional[torch.Tensor], C: int, total_cands: int,
-                          cand_ids: Optional[torch.Tensor], logits: torch.Tensor) -> None:
+                          cand_ids: Optional[torch.Tensor], logits: torch.Tensor, corpus_rows: Optional[int] = None,
+                          dev_flag: Optional[torch.Tensor] = None) -> None:
+    """corpus_rows (only with cand_ids): rows of the corpus caches cand_w / cand_emb; by default the row count of cand_emb."""
+    if cand_ids is not None and corpus_rows is None:
+        corpus_rows = int(cand_emb.shape[0])
     _check(load_library().lime_score_candidates(ctx, _ptr(link_states), B, _ptr(cand_w), _ptr(cand_emb), _ptr(cand_off),
-                                                C, total_cands, _ptr(cand_ids), _ptr(logits), _stream()),
+                                                C, total_cands, _ptr(cand_ids), int(corpus_rows or 0), _ptr(dev_flag),
+                                                _ptr(logits), _stream()),
            "lime_score_candidates")
 
 
@@ -322,9 +327,10 @@ class Lime:
 
     def score_candidates(self, link_states: torch.Tensor, cand_w: torch.Tensor, cand_emb: torch.Tensor, C: int = 0,
                          cand_off: Optional[torch.Tensor] = None, cand_ids: Optional[torch.Tensor] = None,
-                         total_cands: Optional[int] = None) -> torch.Tensor:
+                         total_cands: Optional[int] = None, corpus_rows: Optional[int] = None,
+                         dev_flag: Optional[torch.Tensor] = None) -> torch.Tensor:
         B = link_states.shape[0]
         total = total_cands if total_cands is not None else (cand_ids.numel() if cand_ids is not None else cand_emb.shape[0])
         logits = torch.empty(total, dtype=torch.float32, device=link_states.device)
-        lime_score_candidates(self.ctx, link_states, B, cand_w, cand_emb, cand_off, C, total, cand_ids, logits)
+        lime_score_candidates(self.ctx, link_states, B, cand_w, cand_emb, cand_off, C, total, cand_ids, logits, corpus_rows, dev_flag)
         return logits

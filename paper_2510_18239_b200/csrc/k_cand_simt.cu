@@ -140,7 +140,7 @@ template <typename T>
 __global__ void __launch_bounds__(SC_WARPS * 32)
 k_score_simt(const T* __restrict__ LS, const T* __restrict__ W, const T* __restrict__ Tc, int B, int ell, int d,
              const int32_t* __restrict__ cand_off, int C, int64_t total, const int32_t* __restrict__ cand_ids,
-             float* __restrict__ logits) {
+             int64_t corpus_rows, int32_t* __restrict__ dev_flag, float* __restrict__ logits) {
   extern __shared__ float smem[];
   float* Ls = smem;                  // [ell][d]
   float* ws = Ls + ell * d;          // [warps][ell]
@@ -161,6 +161,14 @@ k_score_simt(const T* __restrict__ LS, const T* __restrict__ W, const T* __restr
     __syncthreads();
     for (int64_t i = i0 + wid; i < e; i += SC_WARPS) {
       const int64_t row = cand_ids ? (int64_t)cand_ids[i] : i;
+      if (cand_ids && (row < 0 || row >= corpus_rows)) {
+        // an id outside the corpus caches reads nothing: logit 0 and the smallest offending slot recorded
+        if (lane == 0) {
+          logits[i] = 0.f;
+          if (dev_flag != nullptr) atomicMin(dev_flag, (int32_t)min(i, (int64_t)INT32_MAX));
+        }
+        continue;
+      }
       for (int l = lane; l < ell; l += 32) ww[l] = Store<T>::ld(W + row * ell + l);
       __syncwarp();
       float dot = 0.f;
@@ -188,12 +196,12 @@ lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st) {
     LIME_CUDA(cudaFuncSetAttribute(k_score_simt<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_score_simt<float><<<(int)blocks, SC_WARPS * 32, smem, st>>>((const float*)a.LS, (const float*)a.W, (const float*)a.T,
                                                                  a.B, a.ell, a.d, a.cand_off, a.C, a.total, a.cand_ids,
-                                                                 a.logits);
+                                                                 a.corpus_rows, a.dev_flag, a.logits);
   } else {
     LIME_CUDA(cudaFuncSetAttribute(k_score_simt<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_score_simt<__nv_bfloat16><<<(int)blocks, SC_WARPS * 32, smem, st>>>(
         (const __nv_bfloat16*)a.LS, (const __nv_bfloat16*)a.W, (const __nv_bfloat16*)a.T, a.B, a.ell, a.d, a.cand_off,
-        a.C, a.total, a.cand_ids, a.logits);
+        a.C, a.total, a.cand_ids, a.corpus_rows, a.dev_flag, a.logits);
   }
   LIME_LAUNCH_CHECK("k_score_simt");
   return LIME_OK;

@@ -48,14 +48,6 @@ __global__ void __launch_bounds__(1024) k_offsets(const int32_t* __restrict__ le
   block_exclusive_scan(B, off, [&](int i) { return max(len[i], 0); });
 }
 
-__global__ void __launch_bounds__(1024)
-k_tile_schedule(const int32_t* __restrict__ off, int B, int tile, int32_t* __restrict__ tile_start) {
-  block_exclusive_scan(B, tile_start, [&](int i) {
-    int n = off[i + 1] - off[i];
-    return n > 0 ? (n + tile - 1) / tile : 0;
-  });
-}
-
 // both work lists of the XOR layers in one launch: chunks of the links<-history attention, tiles of the history update
 __global__ void __launch_bounds__(1024)
 k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __restrict__ chunk_start, int tile,
@@ -89,13 +81,6 @@ lime_status launch_offsets(const int32_t* len, int B, int32_t* off, cudaStream_t
   ProfScope _p("k_offsets", st);
   k_offsets<<<1, 1024, 0, st>>>(len, B, off);
   LIME_LAUNCH_CHECK("k_offsets");
-  return LIME_OK;
-}
-
-lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st) {
-  ProfScope _p("k_tile_schedule", st);
-  k_tile_schedule<<<1, 1024, 0, st>>>(off, B, tile, tile_start);
-  LIME_LAUNCH_CHECK("k_tile_schedule");
   return LIME_OK;
 }
 

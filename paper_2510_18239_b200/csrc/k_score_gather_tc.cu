@@ -15,7 +15,8 @@
 //   warps 0-3 : producers  - 32 x (d/64 + 1) gather copies per tile spread over the threads; thread 0 also fetches the user's link states when the stage held another user's
 //   warp  4   : MMA issuer
 //   warps 5-8 : epilogue   - thread r owns candidate row r (TMEM lane r)
-// ids are not range-checked (as in the generic scorer).
+// An id outside [0, V) fetches row 0 instead (the copies of a stage keep their fixed byte count and never leave the
+// caches); the epilogue thread of that slot writes logit 0 and lowers the caller's flag to the slot index.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
@@ -27,6 +28,8 @@ constexpr int SG_MAX_STAGES = 8;
 
 struct ScoreGatherParams {
   const int32_t* ids;           // [B x C]
+  int32_t V;                    // rows of the corpus caches
+  int32_t* flag;                // nullable: smallest slot whose id was outside [0, V)
   float* logits;                // [B x C]
   int B, C, d;
   int tiles_per_user, n_tiles;
@@ -105,6 +108,9 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
         for (int i = 0; i < 4; ++i)
           if (c + i < p.C) id[i] = __ldg(src + i);
       }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (id[i] < 0 || id[i] >= p.V) id[i] = 0;      // out of range: row 0 stands in; the epilogue zeroes the logit
     };
     int id_now[4], id_next[4], id_after[4];
     read_ids(t_begin, id_next);
@@ -190,6 +196,7 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
       const bool valid = c0 + r < p.C;
       const int64_t grow = (int64_t)b * p.C + c0 + r;
       const int s = it % S;
+      const int32_t my_id = valid ? __ldg(p.ids + grow) : 0;        // in L2 since the producers read it; used at the very end
       if (!mbar_wait(&full[s], (uint32_t)(it / S) & 1u, p.err, 105)) break;
       uint4 w[ELL / 8];
       {
@@ -226,7 +233,11 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty[buf]);
-      if (valid) p.logits[grow] = acc;
+      if (valid) {
+        const bool in_range = my_id >= 0 && my_id < p.V;
+        p.logits[grow] = in_range ? acc : 0.f;
+        if (!in_range && p.flag != nullptr) atomicMin(p.flag, (int32_t)grow);
+      }
     }
   }
 
@@ -261,15 +272,13 @@ template <int ELL>
 static lime_status launch_score_gather_t(const ScoreArgs& a, int* err, cudaStream_t st) {
   size_t smem;
   const int S = score_gather_stages(ELL, a.d, &smem);
-  // the corpus caches have no row count at this interface (ids are not range-checked): the maps span every possible id
-  const uint64_t any_rows = 0x7fffffffull;
   CUtensorMap tmLS, tmT, tmW;
   if (!make_tmap_bf16_sw128(&tmLS, a.LS, (uint64_t)a.B * ELL, (uint64_t)a.d, (uint64_t)a.d, ELL) ||
-      !make_tmap_bf16_sw128(&tmT, a.T, any_rows, (uint64_t)a.d, (uint64_t)a.d, 1) ||
-      !make_tmap_bf16_plain(&tmW, a.W, any_rows, ELL, ELL, 1))
+      !make_tmap_bf16_sw128(&tmT, a.T, (uint64_t)a.corpus_rows, (uint64_t)a.d, (uint64_t)a.d, 1) ||
+      !make_tmap_bf16_plain(&tmW, a.W, (uint64_t)a.corpus_rows, ELL, ELL, 1))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   ScoreGatherParams p;
-  p.ids = a.cand_ids; p.logits = a.logits;
+  p.ids = a.cand_ids; p.logits = a.logits; p.V = (int32_t)a.corpus_rows; p.flag = a.dev_flag;
   p.B = a.B; p.C = a.C; p.d = a.d;
   p.tiles_per_user = (a.C + SG_TILE - 1) / SG_TILE;
   p.n_tiles = p.tiles_per_user * a.B;

@@ -642,8 +642,10 @@ lime_status lime_encode_user_normalized(lime_ctx* ctx, const void* hist_normaliz
 
 lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
                                   const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
-                                  const int32_t* cand_ids, float* logits, void* stream) {
+                                  const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
+                                  void* stream) {
   if (!ctx || B < 0 || C < 0 || total_cands < 0 || total_cands > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (cand_ids && (corpus_rows <= 0 || corpus_rows > 0x7fffffffLL)) return LIME_INVALID_ARG;
   if (!cand_off && total_cands != (int64_t)B * C) return LIME_INVALID_ARG;
   if (B == 0 || total_cands == 0) return LIME_OK;
   if (!link_states || !cand_w || !cand_emb || !logits) return LIME_INVALID_ARG;
@@ -652,6 +654,7 @@ lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_
   ScoreArgs a{};
   a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = c->cfg.dtype; a.B = B; a.ell = c->ell_c; a.d = c->cfg.d;
   a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
+  a.corpus_rows = cand_ids ? corpus_rows : 0; a.dev_flag = cand_ids ? dev_flag : nullptr;
   if (score_tc_supported(a)) return launch_score_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   if (score_gather_tc_supported(a)) return launch_score_gather_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   return launch_score_simt(a, static_cast<cudaStream_t>(stream));

@@ -102,10 +102,8 @@ lime_status launch_gather(int dtype, const void* table, int64_t V, int d, const 
 lime_status launch_gather_ln(int dtype, const void* table, int64_t V, int d, float eps, const int32_t* ids, int64_t total,
                              void* out, int32_t* dev_flag, cudaStream_t st);
 
-// tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B  (work list of per-user token tiles)
-lime_status launch_tile_schedule(const int32_t* off, int B, int tile, int32_t* tile_start, cudaStream_t st);
-// chunk_start (tile = chunk) and tile_start (tile = tile) in one launch; chunk_user[item] = user of the chunk item
-// (may be NULL)
+// Work lists of the XOR layers in one launch: chunk_start[b] = sum_{b' < b} ceil(len_b' / chunk) and
+// tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B; chunk_user[item] = user of the chunk item (may be NULL)
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
                                    int32_t* chunk_user, cudaStream_t st);
 
@@ -130,7 +128,7 @@ struct AttnLinkArgs {
   const void* KS; const void* VS; int s_dtype; // [total x d]
   const int32_t* off; int B; int64_t total;
   int ell, d, H; int phi; float scale;
-  int chunk; const int32_t* chunk_start; int n_chunk_upper;  // work list from launch_tile_schedule(tile = chunk)
+  int chunk; const int32_t* chunk_start; int n_chunk_upper;  // work list from launch_layer_schedules
   float* part_m; float* part_s; float* part_acc;             // [n_chunk_upper x H x ell], same, [.. x d_h]
   float* AT;                                                  // out [B x ell x d] fp32
 };
@@ -174,7 +172,9 @@ struct ScoreArgs {
   const void* LS; const void* W; const void* T; int dtype;
   int B; int ell, d;
   const int32_t* cand_off; int C; int64_t total;
-  const int32_t* cand_ids;
+  const int32_t* cand_ids;      // nullable; with ids, W and T have `corpus_rows` rows and ids outside [0, corpus_rows) score 0
+  int64_t corpus_rows;
+  int32_t* dev_flag;            // nullable: lowered to the smallest slot whose id was out of range
   float* logits;
 };
 lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);

@@ -200,13 +200,3 @@ def make_inputs(wl: Workload, seed: int = 0, with_candidates: bool = True) -> Di
         if with_candidates:
             out["cand_ids"] = uniform_ids(seed, "cand_ids", wl.B * wl.C, wl.V)
     return out
-
-
-def scaled_down(wl: Workload, B: int, V: int = 0, C: int = 0) -> Workload:
-    """Same per-user shape with fewer users (and optionally a smaller table / candidate count)."""
-    kw = dict(B=B)
-    if V:
-        kw["V"] = V
-    if C:
-        kw["C"] = C
-    return wl.replace(**kw)

@@ -39,6 +39,23 @@ def oracle_user(inp, wl, b: int, off: np.ndarray, table64: np.ndarray, links64: 
     return O.run_user(E, links64, layers, cfg, T, cand_w=cand_w, cand_heads=cand_heads)
 
 
+class LazyTable64:
+    """The stored embedding table seen as fp64 rows, widened row by row on demand (the largest table is 4M x 256:
+    widening all of it would take 8 GB); indexable the way the oracle's lookup indexes a table."""
+
+    def __init__(self, table: np.ndarray, dtype: str):
+        self._table, self._dtype, self._rows = table, dtype, {}
+        self.shape, self.dtype = table.shape, np.float64
+
+    def __getitem__(self, key):
+        i = int(key[0] if isinstance(key, tuple) else key)
+        r = self._rows.get(i)
+        if r is None:
+            r = synth.storage_to_f64(self._table[i], self._dtype)
+            self._rows[i] = r
+        return r
+
+
 class DeviceBatch:
     """Device-side mirror of one synthetic batch plus a configured library context."""
 
