@@ -131,7 +131,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   uint64_t* x_full = bars;             // [LB_XSTAGES]
   uint64_t* x_empty = bars + 4;        // [LB_XSTAGES]  second MMA of the tile done
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       //      per tile: P in smem (all softmax warps)
+  uint64_t* p_ready = bars + 10;       // [2]  per tile and P buffer: P in smem (all softmax warps)
   uint64_t* p_free = bars + 12;        // [2]  per tile and P buffer: second MMA done reading P (and accumulator up to date)
   uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
   uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the warps that share a TMEM lane quarter
@@ -145,7 +145,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     for (int s = 0; s < LB_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
-    mbar_init(p_ready, LB_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
+    mbar_init(&p_ready[0], LB_SOFTMAX_WARPS); mbar_init(&p_ready[1], LB_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
     mbar_init(o_free, LB_SOFTMAX_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LB_PARTS);
     fence_barrier_init();
@@ -255,7 +255,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
           }
           const int s = g % LB_XSTAGES;
-          if (!mbar_wait(p_ready, (uint32_t)g & 1u, p.err, 52)) { ok = false; break; }
+          if (!mbar_wait(&p_ready[g % LB_PBUFS], (uint32_t)(g / LB_PBUFS) & 1u, p.err, 52)) { ok = false; break; }
           // the first tile of an item overwrites the accumulator: the previous item must have been read out
           if (t == 0 && k > 0 && !mbar_wait(o_free, (uint32_t)(k - 1) & 1u, p.err, 53)) { ok = false; break; }
           tc_fence_after();
@@ -306,7 +306,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
           tc_fence_before();
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(p_ready);
+          if (lane == 0) mbar_arrive(&p_ready[g % LB_PBUFS]);
           continue;
         }
         float mx = -INFINITY;
@@ -346,7 +346,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(p_ready);
+        if (lane == 0) mbar_arrive(&p_ready[g % LB_PBUFS]);
       }
       if (!ok) break;
       // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row

@@ -188,7 +188,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
   uint64_t* q_full = bars + 22;        // [2]  folded queries of a user landed in buffer i
   uint64_t* q_empty = bars + 24;       // [2]  every score MMA that reads buffer i has run
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       //      per tile: P' in smem (all softmax warps)
+  uint64_t* p_ready = bars + 10;       // [2]  per tile and P' buffer: P' in smem (all softmax warps)
   uint64_t* p_free = bars + 12;        // [2]  per tile and P' buffer: second MMA done reading P' (and accumulator up to date)
   uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
   uint64_t* stats_bar = bars + 15;     //      rendezvous of the softmax warps (token statistics written)
@@ -201,7 +201,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     for (int s = 0; s < LA_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 1); mbar_init(&q_empty[i], 1); }
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
-    mbar_init(p_ready, LA_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
+    mbar_init(&p_ready[0], LA_SOFTMAX_WARPS); mbar_init(&p_ready[1], LA_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
     mbar_init(o_free, LA_SOFTMAX_WARPS);
     mbar_init(stats_bar, LA_SOFTMAX_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LA_PARTS);
@@ -318,7 +318,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
             if (t + 2 == n_tiles && next_reloads) mma_commit(&q_empty[(qn - 1) % LA_Q2_BUFS]);
           }
           const int s = g % LA_XSTAGES;
-          if (!mbar_wait(p_ready, (uint32_t)g & 1u, p.err, 52)) { ok = false; break; }
+          if (!mbar_wait(&p_ready[g % LA_PBUFS], (uint32_t)(g / LA_PBUFS) & 1u, p.err, 52)) { ok = false; break; }
           // the first tile of an item overwrites the accumulator: the previous item must have been read out
           if (t == 0 && k > 0 && !mbar_wait(o_free, (uint32_t)(k - 1) & 1u, p.err, 53)) { ok = false; break; }
           tc_fence_after();
@@ -427,7 +427,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
           tc_fence_before();
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(p_ready);
+          if (lane == 0) mbar_arrive(&p_ready[g % LA_PBUFS]);
           continue;
         }
         exch_max[(pb * LA_PARTS + part) * 128 + r] = mx;
@@ -465,7 +465,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(p_ready);
+        if (lane == 0) mbar_arrive(&p_ready[g % LA_PBUFS]);
       }
       if (!ok) break;
       // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
