@@ -27,6 +27,11 @@ the design notes of the repository):
   * XOR layers are stacked: layer j consumes layer j-1's history and link rows; L^P sums the link
     rows of every layer's output (Eq. 8)
   * an empty history gives zero attention output for the link rows
+  * the two small MLPs the paper names without a formula - the link contextualisation of Eq. 2 and the
+    "shallow interaction network" that scores the LIME embedding (Sec. 3.3; widths in App. C's table) - are
+    plain feed-forward networks: x <- ReLU(x W_i + b_i) for every hidden layer, a linear last layer.  Eq. 2's
+    input row is a link row followed by the user's context vector; the interaction network's input row is the
+    LIME embedding O_c followed by the candidate embedding T_c   -- parity unpinned by the paper, see PINS below
 
 PINS (what ties each function to something other than itself; see tests/test_oracle_*.py):
   lengths_to_offsets, gather_history : definition, exact integers / bytes
@@ -44,6 +49,11 @@ PINS (what ties each function to something other than itself; see tests/test_ora
                                      : PARITY UNPINNED by the paper beyond reductions: identity weights
                                        reduce FULL to CORE; n = 1 gives L^P = T^1; the last layer's
                                        history update never reaches the logits
+  ffn, contextualize_links, interaction_head
+                                     : scalar-loop evaluation; a library Linear/ReLU stack in fp64; zero hidden
+                                       weights leave the last bias; bias-free networks are positively
+                                       homogeneous; a context vector of zeros makes every user's L^C equal.
+                                       Their FORM (inputs, activation) is PARITY UNPINNED by the paper
 """
 from __future__ import annotations
 
@@ -314,6 +324,41 @@ def score_candidates_heads(W: np.ndarray, LS: np.ndarray, T: np.ndarray, cfg: Or
     for c in range(T.shape[0]):
         out[c] = float(np.dot(O[c, :], T[c, :]))
     return out
+
+
+# --------------------------------------------------------------------------- #
+# the two small feed-forward networks: Eq. 2 (link contextualisation) and the interaction network of Sec. 3.3
+# --------------------------------------------------------------------------- #
+def ffn(X: np.ndarray, layers) -> np.ndarray:
+    """Feed-forward network on the rows of X: `layers` is a list of (W [in x out], b [out] or None); every layer
+    but the last is followed by ReLU."""
+    Z = np.asarray(X, dtype=np.float64)
+    for i, (W, b) in enumerate(layers):
+        Z = Z @ W
+        if b is not None:
+            Z = Z + b
+        if i + 1 < len(layers):
+            Z = np.maximum(Z, 0.0)
+    return Z
+
+
+def contextualize_links(L: np.ndarray, EC: np.ndarray, layers) -> np.ndarray:
+    """Eq. 2: L^C = MLP(L (+) E^C) for one user.  L [l x d] shared links, EC [d_c] the user's context features;
+    every link row is followed by the same context vector, the MLP maps the (d + d_c)-wide rows back to d."""
+    X = np.concatenate([np.asarray(L, dtype=np.float64), np.tile(np.asarray(EC, dtype=np.float64), (L.shape[0], 1))], axis=1)
+    return ffn(X, layers)
+
+
+def interaction_head(O: np.ndarray, T: np.ndarray, layers) -> np.ndarray:
+    """Sec. 3.3 "Lightweight User-Item Interaction": the LIME embedding O_c is passed to a shallow interaction
+    network for scoring.  Input row = O_c followed by T_c; hidden widths as App. C's "Interaction MLP" row (one
+    96-wide layer on the industrial model); the last layer has one output, the logit."""
+    return ffn(np.concatenate([O, T], axis=1), layers)[:, 0]
+
+
+def score_candidates_head(W: np.ndarray, LS: np.ndarray, T: np.ndarray, layers) -> np.ndarray:
+    """logit[c] = head(O_c, T_c) with O = phi(T L^t) L^P of Eq. 4."""
+    return interaction_head(candidate_outputs(W, LS), T, layers)
 
 
 # --------------------------------------------------------------------------- #

@@ -443,3 +443,107 @@ def test_silu_attention_matches_scalar_loops():
                 for k in range(2):
                     want[i, 2 * h + k] += p * E[j, 2 * h + k]
     assert np.allclose(out, want, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- feed-forward networks (Eq. 2, Sec. 3.3)
+def _ffn_scalar(x, layers):
+    """One row through the network with scalar loops only."""
+    z = [float(v) for v in x]
+    for i, (W, b) in enumerate(layers):
+        out = []
+        for j in range(W.shape[1]):
+            acc = 0.0 if b is None else float(b[j])
+            for k in range(W.shape[0]):
+                acc += z[k] * float(W[k, j])
+            out.append(max(acc, 0.0) if i + 1 < len(layers) else acc)
+        z = out
+    return z
+
+
+def _rand_ffn(g, widths, bias=True):
+    return [(g.normal(size=(a, b)) / math.sqrt(a), g.normal(size=b) * 0.3 if bias else None)
+            for a, b in zip(widths[:-1], widths[1:])]
+
+
+def test_ffn_against_scalar_loops_and_torch():
+    g = rng(31)
+    for widths in ([6, 5, 1], [8, 7, 4, 3], [5, 2]):
+        layers = _rand_ffn(g, widths)
+        X = g.normal(size=(9, widths[0]))
+        got = O.ffn(X, layers)
+        want = np.array([_ffn_scalar(x, layers) for x in X])
+        assert np.allclose(got, want, atol=1e-12)
+        mods = []
+        for i, (W, b) in enumerate(layers):
+            lin = torch.nn.Linear(W.shape[0], W.shape[1]).double()
+            with torch.no_grad():
+                lin.weight.copy_(torch.from_numpy(W.T))
+                lin.bias.copy_(torch.from_numpy(b))
+            mods.append(lin)
+            if i + 1 < len(layers):
+                mods.append(torch.nn.ReLU())
+        with torch.no_grad():
+            ref = torch.nn.Sequential(*mods)(torch.from_numpy(X)).numpy()
+        assert np.allclose(got, ref, atol=1e-12)
+
+
+def test_ffn_reductions():
+    g = rng(32)
+    layers = _rand_ffn(g, [6, 8, 1])
+    X = g.normal(size=(4, 6))
+    # zero hidden weights and bias: the ReLU layer outputs 0, the logit is the last bias
+    zeroed = [(np.zeros_like(layers[0][0]), np.zeros_like(layers[0][1])), layers[1]]
+    assert np.allclose(O.ffn(X, zeroed)[:, 0], layers[1][1][0])
+    # without biases a ReLU network is positively homogeneous
+    nobias = [(W, None) for W, _ in layers]
+    assert np.allclose(O.ffn(3.5 * X, nobias), 3.5 * O.ffn(X, nobias), atol=1e-12)
+    # a hidden layer that passes a non-negative input through (identity weights) leaves a linear map
+    Xp = np.abs(X)
+    ident = [(np.eye(6), None), (layers[1][0][:6], None)]
+    assert np.allclose(O.ffn(Xp, ident), Xp @ layers[1][0][:6], atol=1e-12)
+
+
+def test_interaction_head_inputs_and_permutation():
+    g = rng(33)
+    d, ell, C = 6, 3, 7
+    W = O.softmax_rows(g.normal(size=(C, ell)))
+    LS, T = g.normal(size=(ell, d)), g.normal(size=(C, d))
+    layers = _rand_ffn(g, [2 * d, 5, 1])
+    got = O.score_candidates_head(W, LS, T, layers)
+    # row c of the network's input is (O_c, T_c) with O_c = sum_l W[c, l] LS[l, :]  (Eq. 4), in scalar loops
+    for c in range(C):
+        o = [sum(W[c, l] * LS[l, k] for l in range(ell)) for k in range(d)]
+        assert abs(got[c] - _ffn_scalar(o + list(T[c]), layers)[0]) < 1e-12
+    perm = g.permutation(C)
+    assert np.allclose(O.score_candidates_head(W[perm], LS, T[perm], layers), got[perm], atol=1e-13)
+    # a head whose first layer ignores the O half scores the candidate embedding alone, whatever the user
+    W1 = layers[0][0].copy()
+    W1[:d] = 0.0
+    blind = [(W1, layers[0][1]), layers[1]]
+    assert np.allclose(O.score_candidates_head(W, LS, T, blind), O.score_candidates_head(W, 7.0 * LS + 1.0, T, blind), atol=1e-13)
+
+
+def test_contextualize_links_eq2():
+    g = rng(34)
+    d, d_c, ell = 6, 4, 5
+    L = g.normal(size=(ell, d))
+    layers = _rand_ffn(g, [d + d_c, 7, d])
+    ec = g.normal(size=d_c)
+    LC = O.contextualize_links(L, ec, layers)
+    assert LC.shape == (ell, d)
+    for l in range(ell):
+        assert np.allclose(LC[l], _ffn_scalar(list(L[l]) + list(ec), layers), atol=1e-12)
+    # first layer splits over the concatenation: (L (+) E^C) W = L W[:d] + E^C W[d:]
+    W1, b1 = layers[0]
+    hidden = np.maximum(L @ W1[:d] + ec @ W1[d:] + b1, 0.0)
+    assert np.allclose(LC, hidden @ layers[1][0] + layers[1][1], atol=1e-12)
+    # a first layer that ignores the context columns gives every user the same contextualised links
+    W1z = W1.copy()
+    W1z[d:] = 0.0
+    same = [(W1z, b1), layers[1]]
+    assert np.allclose(O.contextualize_links(L, ec, same), O.contextualize_links(L, g.normal(size=d_c), same), atol=1e-13)
+    # L^C feeds the user side in place of L (Eq. 3 / Eq. 8): encode_user takes it as the link rows
+    cfg = core_cfg(d, 2, ell)
+    E = g.normal(size=(11, d))
+    LP, _ = O.encode_user(E, LC, [dict()], cfg)
+    assert np.allclose(LP, O.mha(LC, E, E, None, None, None, cfg), atol=1e-13)
