@@ -180,6 +180,40 @@ LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_state
                                   const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
                                   void* stream);
 
+/* The two small feed-forward networks the paper names without a formula.  Both are read as x <- ReLU(x W_i + b_i)
+ * for each of n_hidden hidden layers followed by one linear layer; W[i] is [in_i x out_i] row-major in config.dtype,
+ * b[i] fp32 [out_i] or NULL (no bias); all are device pointers, borrowed until replaced or lime_destroy. */
+#define LIME_FFN_MAX_HIDDEN 3
+typedef struct lime_ffn {
+  int32_t n_hidden;                          /* hidden layers: 0..3 (the interaction network needs at least 1)        */
+  int32_t widths[LIME_FFN_MAX_HIDDEN];       /* their widths, each 1..1024                                             */
+  const void* W[LIME_FFN_MAX_HIDDEN + 1];    /* n_hidden + 1 weight matrices                                           */
+  const float* b[LIME_FFN_MAX_HIDDEN + 1];   /* n_hidden + 1 bias vectors (nullable)                                   */
+} lime_ffn;
+
+/* Link contextualisation (Eq. 2): L^C_b = MLP(L (+) E^C_b).  Every link row L_l [d] is followed by the user's context
+ * features E^C_b [d_c]; the network maps the (d + d_c)-wide rows to d: in_0 = d + d_c (rows 0..d-1 of W[0] act on the
+ * link, rows d.. on the context), out of the last layer = d.  lime_set_context_mlp is a set-up call (it allocates a
+ * few KB and launches the weights-only part of the first layer on `stream`); call it after lime_set_weights, and again
+ * after the links change.  lime_contextualize_links writes link_ctx fp32 [B x ell x d], the `link_ctx` argument of
+ * lime_encode_user; user_ctx [B x d_c] in config.dtype.  LIME_NOT_READY without a network. */
+LIME_API lime_status lime_set_context_mlp(lime_ctx* ctx, int32_t d_c, const lime_ffn* mlp, void* stream);
+LIME_API lime_status lime_contextualize_links(lime_ctx* ctx, const void* user_ctx, int32_t B, float* link_ctx, void* stream);
+
+/* Interaction network on the LIME embedding (Sec. 3.3 "Lightweight User-Item Interaction"; hidden widths as the
+ * "Interaction MLP" row of App. C's table, e.g. one 96-wide layer):
+ *   logits[i] = FFN( [O_i | T_i] ),  O_i = sum_l cand_w[i,l] * link_states[b(i),l,:],  T_i = cand_emb[i,:]
+ * in_0 = 2d (rows 0..d-1 of W[0] act on O, rows d..2d-1 on T), out of the last layer = 1, n_hidden >= 1.
+ * lime_set_head is a set-up call (allocates copies of two small operands).  lime_score_candidates_head takes the
+ * arguments of lime_score_candidates plus scratch of lime_head_workspace_bytes(ctx, B) bytes (the per-user product
+ * link_states . W[0][:d], so that O is never formed).  LIME_NOT_READY without a network. */
+LIME_API lime_status lime_set_head(lime_ctx* ctx, const lime_ffn* head, void* stream);
+LIME_API size_t lime_head_workspace_bytes(const lime_ctx* ctx, int32_t B);
+LIME_API lime_status lime_score_candidates_head(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
+                                       const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
+                                       const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
+                                       void* ws, size_t ws_bytes, void* stream);
+
 /* Allocation-free precompute (the paper has no counterpart: this exists for hosts that must not allocate).
  * Same result as lime_create + lime_set_weights + lime_precompute_candidate_links, for callers that cannot call
  * cudaMalloc at this point - a serving process whose device memory pool is frozen after start-up, or code running
@@ -208,6 +242,13 @@ LIME_API lime_status lime_precompute_candidate_links_noalloc(int32_t dtype, int3
  * writes the code to *code (host), clears it, and returns LIME_DEVICE_TIMEOUT if it was set, else LIME_OK.
  * The paper has no counterpart; codes: 1 producer, 2-3 MMA issuer, 4 epilogue waits of the scorer. */
 LIME_API lime_status lime_device_status(lime_ctx* ctx, int32_t* code);
+
+/* Self-test of that mechanism (the paper has no counterpart): launches one thread that waits, for at most limit_us
+ * microseconds (1 .. 1,000,000), on a barrier nothing ever arrives at.  The wait gives up, the kernel returns, and the
+ * next lime_device_status reports LIME_DEVICE_TIMEOUT with code LIME_SELFTEST_WAIT_CODE; the context stays usable.
+ * Nothing faults, traps or spins without a bound. */
+#define LIME_SELFTEST_WAIT_CODE 200
+LIME_API lime_status lime_selftest_wait_expiry(lime_ctx* ctx, int32_t limit_us, void* stream);
 
 /* Per-kernel timing for benchmarks (the paper reports latency only end to end, App. F; this breaks a call down).
  * Between lime_profile_start(capacity) and lime_profile_stop every kernel this library launches is bracketed by two

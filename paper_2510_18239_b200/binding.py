@@ -44,10 +44,19 @@ class lime_weights(ctypes.Structure):
                 ("cand_Wv", ctypes.c_void_p)]
 
 
+LIME_FFN_MAX_HIDDEN = 3
+
+
+class lime_ffn(ctypes.Structure):
+    _fields_ = [("n_hidden", ctypes.c_int32), ("widths", ctypes.c_int32 * LIME_FFN_MAX_HIDDEN),
+                ("W", ctypes.c_void_p * (LIME_FFN_MAX_HIDDEN + 1)), ("b", ctypes.c_void_p * (LIME_FFN_MAX_HIDDEN + 1))]
+
+
 EXPORTS = ("lime_create", "lime_destroy", "lime_set_weights", "lime_workspace_bytes", "lime_lengths_to_offsets",
            "lime_gather_history", "lime_gather_history_normalized", "lime_precompute_candidate_links", "lime_xor_layer",
            "lime_encode_user", "lime_encode_user_normalized",
-           "lime_score_candidates", "lime_precompute_candidate_links_noalloc", "lime_device_status", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
+           "lime_score_candidates", "lime_set_context_mlp", "lime_contextualize_links", "lime_set_head",
+           "lime_head_workspace_bytes", "lime_score_candidates_head", "lime_precompute_candidate_links_noalloc", "lime_device_status", "lime_selftest_wait_expiry", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
            "lime_version")
 
 _lib_handle = None
@@ -77,8 +86,15 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_encode_user_normalized.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, i64, vp, vp, vp]
+    lib.lime_set_context_mlp.argtypes = [vp, i32, ctypes.POINTER(lime_ffn), vp]
+    lib.lime_contextualize_links.argtypes = [vp, vp, i32, vp, vp]
+    lib.lime_set_head.argtypes = [vp, ctypes.POINTER(lime_ffn), vp]
+    lib.lime_head_workspace_bytes.argtypes = [vp, i32]
+    lib.lime_head_workspace_bytes.restype = sz
+    lib.lime_score_candidates_head.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, i64, vp, vp, vp, sz, vp]
     lib.lime_precompute_candidate_links_noalloc.argtypes = [i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, i64, vp, vp]
     lib.lime_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+    lib.lime_selftest_wait_expiry.argtypes = [vp, i32, vp]
     lib.lime_profile_start.argtypes = [i32]
     lib.lime_profile_stop.argtypes = [ctypes.c_char_p, sz, ctypes.POINTER(ctypes.c_float), i32, ctypes.POINTER(i32)]
     for name in EXPORTS:
@@ -86,7 +102,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
         if name in ("lime_last_cuda_error", "lime_version"):
             fn.restype = ctypes.c_char_p
             fn.argtypes = []
-        elif name != "lime_workspace_bytes":
+        elif name not in ("lime_workspace_bytes", "lime_head_workspace_bytes"):
             fn.restype = ctypes.c_int
     if path is None:
         _lib_handle = lib
@@ -192,6 +208,46 @@ def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: t
            "lime_score_candidates")
 
 
+def make_ffn(layers) -> lime_ffn:
+    """layers: list of (W tensor [in x out], b fp32 tensor [out] or None); all but the last are hidden layers."""
+    f = lime_ffn()
+    f.n_hidden = len(layers) - 1
+    for i, (W, b) in enumerate(layers):
+        if i < len(layers) - 1:
+            f.widths[i] = int(W.shape[1])
+        f.W[i] = _ptr(W)
+        f.b[i] = _ptr(b)
+    return f
+
+
+def lime_set_context_mlp(ctx: int, d_c: int, mlp: lime_ffn) -> None:
+    _check(load_library().lime_set_context_mlp(ctx, d_c, ctypes.byref(mlp), _stream()), "lime_set_context_mlp")
+
+
+def lime_contextualize_links(ctx: int, user_ctx: torch.Tensor, B: int, link_ctx: torch.Tensor) -> None:
+    _check(load_library().lime_contextualize_links(ctx, _ptr(user_ctx), B, _ptr(link_ctx), _stream()), "lime_contextualize_links")
+
+
+def lime_set_head(ctx: int, head: lime_ffn) -> None:
+    _check(load_library().lime_set_head(ctx, ctypes.byref(head), _stream()), "lime_set_head")
+
+
+def lime_head_workspace_bytes(ctx: int, B: int) -> int:
+    return int(load_library().lime_head_workspace_bytes(ctx, B))
+
+
+def lime_score_candidates_head(ctx: int, link_states: torch.Tensor, B: int, cand_w: torch.Tensor, cand_emb: torch.Tensor,
+                               cand_off: Optional[torch.Tensor], C: int, total_cands: int, cand_ids: Optional[torch.Tensor],
+                               logits: torch.Tensor, ws: torch.Tensor, corpus_rows: Optional[int] = None,
+                               dev_flag: Optional[torch.Tensor] = None) -> None:
+    if cand_ids is not None and corpus_rows is None:
+        corpus_rows = int(cand_emb.shape[0])
+    _check(load_library().lime_score_candidates_head(ctx, _ptr(link_states), B, _ptr(cand_w), _ptr(cand_emb), _ptr(cand_off),
+                                                     C, total_cands, _ptr(cand_ids), int(corpus_rows or 0), _ptr(dev_flag),
+                                                     _ptr(logits), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "lime_score_candidates_head")
+
+
 def lime_precompute_candidate_links_noalloc(dtype: int, d: int, ell: int, cand_scale: float, links: torch.Tensor,
                                             cand_Wq: Optional[torch.Tensor], cand_Wk: Optional[torch.Tensor],
                                             cand_emb: torch.Tensor, out_w: torch.Tensor) -> None:
@@ -212,6 +268,11 @@ def lime_device_status(ctx: int) -> int:
     if st != 0:
         raise LimeError(st, "lime_device_status", f"wait code {code.value}")
     return int(code.value)
+
+
+def lime_selftest_wait_expiry(ctx: int, limit_us: int) -> None:
+    """Launches a wait that can never be satisfied, bounded by limit_us; lime_device_status then reports the time-out."""
+    _check(load_library().lime_selftest_wait_expiry(ctx, limit_us, _stream()), "lime_selftest_wait_expiry")
 
 
 def lime_profile_start(capacity: int = 4096) -> None:
@@ -333,4 +394,33 @@ class Lime:
         total = total_cands if total_cands is not None else (cand_ids.numel() if cand_ids is not None else cand_emb.shape[0])
         logits = torch.empty(total, dtype=torch.float32, device=link_states.device)
         lime_score_candidates(self.ctx, link_states, B, cand_w, cand_emb, cand_off, C, total, cand_ids, logits, corpus_rows, dev_flag)
+        return logits
+
+    # ---- feed-forward networks (Eq. 2; the interaction network of Sec. 3.3)
+    def set_context_mlp(self, d_c: int, layers) -> None:
+        self._keep_ctx = [t for pair in layers for t in pair if t is not None]
+        lime_set_context_mlp(self.ctx, d_c, make_ffn(layers))
+
+    def contextualize_links(self, user_ctx: torch.Tensor) -> torch.Tensor:
+        B = user_ctx.shape[0]
+        out = torch.empty((B, self.cfg.ell, self.cfg.d), dtype=torch.float32, device=user_ctx.device)
+        lime_contextualize_links(self.ctx, user_ctx, B, out)
+        return out
+
+    def set_head(self, layers) -> None:
+        self._keep_head = [t for pair in layers for t in pair if t is not None]
+        lime_set_head(self.ctx, make_ffn(layers))
+
+    def score_candidates_head(self, link_states: torch.Tensor, cand_w: torch.Tensor, cand_emb: torch.Tensor, C: int = 0,
+                              cand_off: Optional[torch.Tensor] = None, cand_ids: Optional[torch.Tensor] = None,
+                              total_cands: Optional[int] = None, corpus_rows: Optional[int] = None,
+                              dev_flag: Optional[torch.Tensor] = None) -> torch.Tensor:
+        B = link_states.shape[0]
+        total = total_cands if total_cands is not None else (cand_ids.numel() if cand_ids is not None else cand_emb.shape[0])
+        logits = torch.empty(total, dtype=torch.float32, device=link_states.device)
+        need = lime_head_workspace_bytes(self.ctx, B)
+        if getattr(self, "_head_ws", None) is None or self._head_ws.numel() < need:
+            self._head_ws = torch.empty(need, dtype=torch.uint8, device=link_states.device)
+        lime_score_candidates_head(self.ctx, link_states, B, cand_w, cand_emb, cand_off, C, total, cand_ids, logits,
+                                   self._head_ws, corpus_rows, dev_flag)
         return logits

@@ -417,6 +417,8 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->cand_scale = g.cand_scale > 0.f ? g.cand_scale : 1.0f / sqrtf((float)(cand_heads > 1 ? c->d_h : g.d));
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
+  c->have_head = c->have_ctx_mlp = false; c->ctx_dc = 0;
+  c->head_W1bT = nullptr; c->head_w2 = nullptr; c->ctx_first = nullptr;
   c->tc_mode = tensor_core_mode(g, d_ff);
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = c->WguT[j] = nullptr;
   c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = c->sh_V2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
@@ -448,6 +450,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); cudaFree(c->WguT[j]); }
   cudaFree(c->sh_That); cudaFree(c->sh_Q2); cudaFree(c->sh_K2); cudaFree(c->sh_G2t); cudaFree(c->sh_U2t); cudaFree(c->sh_V2t);
   cudaFree(c->sh_cQ); cudaFree(c->sh_cK);
+  cudaFree(c->head_W1bT); cudaFree(c->head_w2); cudaFree(c->ctx_first);
   delete c;
   return LIME_OK;
 }
@@ -658,6 +661,137 @@ lime_status lime_score_candidates(lime_ctx* ctx, const void* link_states, int32_
   if (score_tc_supported(a)) return launch_score_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   if (score_gather_tc_supported(a)) return launch_score_gather_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
   return launch_score_simt(a, static_cast<cudaStream_t>(stream));
+}
+
+// ---- feed-forward networks (Eq. 2; Sec. 3.3 interaction network) ----------------------------------------------------
+static bool ffn_valid(const lime_ffn* f, int min_hidden) {
+  if (!f || f->n_hidden < min_hidden || f->n_hidden > LIME_FFN_MAX_HIDDEN) return false;
+  for (int i = 0; i < f->n_hidden; ++i)
+    if (f->widths[i] < 1 || f->widths[i] > 1024) return false;
+  for (int i = 0; i <= f->n_hidden; ++i)
+    if (!f->W[i] || !aligned16(f->W[i])) return false;
+  return true;
+}
+// layers after the first: layer i maps widths[i-1] to widths[i] (the last one to `out_last`)
+static FfnArgs ffn_tail(const lime_ffn& f, int out_last) {
+  FfnArgs a{};
+  a.n_layers = f.n_hidden;
+  for (int i = 1; i <= f.n_hidden; ++i) {
+    a.in_w[i - 1] = f.widths[i - 1];
+    a.out_w[i - 1] = i < f.n_hidden ? f.widths[i] : out_last;
+    a.W[i - 1] = f.W[i];
+    a.b[i - 1] = f.b[i];
+  }
+  return a;
+}
+
+lime_status lime_set_context_mlp(lime_ctx* ctx, int32_t d_c, const lime_ffn* mlp, void* stream) {
+  if (!ctx || d_c < 1 || d_c > 4096 || !ffn_valid(mlp, 0)) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_weights) return LIME_NOT_READY;
+  const lime_config& g = c->cfg;
+  const int w0 = mlp->n_hidden > 0 ? mlp->widths[0] : g.d;
+  cudaFree(c->ctx_first);
+  c->ctx_first = nullptr;
+  c->have_ctx_mlp = false;
+  LIME_CUDA(cudaMalloc(&c->ctx_first, sizeof(float) * (size_t)g.ell * w0));
+  // weights-only part of the first layer: (L W_0[:d]) + b_0
+  lime_status s = launch_rows_times_w(c->w.links, g.dtype, g.ell, g.d, mlp->W[0], g.dtype, w0, w0, mlp->b[0], c->ctx_first, nullptr,
+                                      1, "k_ctx_first", static_cast<cudaStream_t>(stream));
+  if (s != LIME_OK) return s;
+  c->ctx_mlp = *mlp;
+  c->ctx_dc = d_c;
+  c->have_ctx_mlp = true;
+  return LIME_OK;
+}
+
+lime_status lime_contextualize_links(lime_ctx* ctx, const void* user_ctx, int32_t B, float* link_ctx, void* stream) {
+  if (!ctx || B < 0) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_ctx_mlp) return LIME_NOT_READY;
+  if (B == 0) return LIME_OK;
+  if (!user_ctx || !link_ctx || !aligned16(link_ctx)) return LIME_INVALID_ARG;
+  const lime_config& g = c->cfg;
+  const lime_ffn& f = c->ctx_mlp;
+  const int w0 = f.n_hidden > 0 ? f.widths[0] : g.d;
+  const char* W0c = static_cast<const char*>(f.W[0]) + (size_t)g.d * w0 * elem_size(g.dtype);     // rows d.. act on E^C
+  return launch_link_ctx_mlp(g.dtype, c->ctx_first, user_ctx, c->ctx_dc, W0c, w0, B, g.ell, ffn_tail(f, g.d), link_ctx,
+                             static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_set_head(lime_ctx* ctx, const lime_ffn* head, void* stream) {
+  if (!ctx || !ffn_valid(head, 1)) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  const lime_config& g = c->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int w0 = head->widths[0], w_last = head->widths[head->n_hidden - 1];
+  cudaFree(c->head_W1bT); cudaFree(c->head_w2);
+  c->head_W1bT = nullptr; c->head_w2 = nullptr;
+  c->have_head = false;
+  LIME_CUDA(cudaMalloc(&c->head_w2, sizeof(float) * (size_t)w_last));
+  lime_status s = launch_widen(head->W[head->n_hidden], g.dtype, c->head_w2, w_last, st);
+  if (s != LIME_OK) return s;
+  if (g.dtype == LIME_BF16) {
+    // the T half of the first layer as a K-major B operand [w0 x d]
+    LIME_CUDA(cudaMalloc(&c->head_W1bT, (size_t)w0 * g.d * 2));
+    const char* W0t = static_cast<const char*>(head->W[0]) + (size_t)g.d * w0 * 2;
+    if ((s = launch_transpose_bf16(W0t, g.d, w0, c->head_W1bT, st)) != LIME_OK) return s;
+  }
+  c->head = *head;
+  c->have_head = true;
+  return LIME_OK;
+}
+
+size_t lime_head_workspace_bytes(const lime_ctx* ctx, int32_t B) {
+  if (!ctx || B < 0) return 0;
+  const Ctx* c = reinterpret_cast<const Ctx*>(ctx);
+  if (!c->have_head) return 0;
+  const size_t n = (size_t)B * c->ell_c * c->head.widths[0];
+  return align_up(n * 4) + align_up(n * 2) + 256;
+}
+
+lime_status lime_score_candidates_head(lime_ctx* ctx, const void* link_states, int32_t B, const void* cand_w,
+                                       const void* cand_emb, const int32_t* cand_off, int32_t C, int64_t total_cands,
+                                       const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
+                                       void* ws, size_t ws_bytes, void* stream) {
+  if (!ctx || B < 0 || C < 0 || total_cands < 0 || total_cands > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (cand_ids && (corpus_rows <= 0 || corpus_rows > 0x7fffffffLL)) return LIME_INVALID_ARG;
+  if (!cand_off && total_cands != (int64_t)B * C) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  if (!c->have_head) return LIME_NOT_READY;
+  if (B == 0 || total_cands == 0) return LIME_OK;
+  if (!link_states || !cand_w || !cand_emb || !logits || !ws) return LIME_INVALID_ARG;
+  if (!aligned16(link_states) || !aligned16(cand_w) || !aligned16(cand_emb)) return LIME_INVALID_ARG;
+  const lime_config& g = c->cfg;
+  const lime_ffn& f = c->head;
+  const int w0 = f.widths[0];
+  char* base = reinterpret_cast<char*>(align_up(reinterpret_cast<uintptr_t>(ws)));
+  const size_t n = (size_t)B * c->ell_c * w0;
+  if ((size_t)(base - static_cast<char*>(ws)) + align_up(n * 4) + align_up(n * 2) > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
+  float* LSW = reinterpret_cast<float*>(base);
+  void* LSWt = base + align_up(n * 4);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ScoreArgs a{};
+  a.LS = link_states; a.W = cand_w; a.T = cand_emb; a.dtype = g.dtype; a.B = B; a.ell = c->ell_c; a.d = g.d;
+  a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
+  a.corpus_rows = cand_ids ? corpus_rows : 0; a.dev_flag = cand_ids ? dev_flag : nullptr;
+  const bool tc = f.n_hidden == 1 && c->head_W1bT && score_head_tc_supported(a, w0);
+  // per user: LSW_b = LS_b W_0[:d]  (the O half of the first layer applied to the link states, so O is never formed)
+  lime_status s = launch_rows_times_w(link_states, g.dtype, (int64_t)B * c->ell_c, g.d, f.W[0], g.dtype, w0, w0, nullptr,
+                                      tc ? nullptr : LSW, tc ? LSWt : nullptr, c->ell_c, "k_head_lsw", st);
+  if (s != LIME_OK) return s;
+  if (tc) {
+    ScoreHeadArgs h{LSWt, c->head_W1bT, f.b[0], c->head_w2, f.b[1], w0};
+    return launch_score_head_tc(a, h, c->dev_err, st);
+  }
+  const char* W0t = static_cast<const char*>(f.W[0]) + (size_t)g.d * w0 * elem_size(g.dtype);
+  return launch_score_head_simt(a, LSW, W0t, f.b[0], w0, ffn_tail(f, 1), st);
+}
+
+lime_status lime_selftest_wait_expiry(lime_ctx* ctx, int32_t limit_us, void* stream) {
+  if (!ctx || limit_us < 1 || limit_us > 1000000) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  return launch_wait_expiry(c->dev_err, (uint64_t)limit_us * 1000ull, LIME_SELFTEST_WAIT_CODE, static_cast<cudaStream_t>(stream));
 }
 
 lime_status lime_device_status(lime_ctx* ctx, int32_t* code) {

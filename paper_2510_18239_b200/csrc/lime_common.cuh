@@ -63,6 +63,13 @@ struct Ctx {
   // link-side operands of the first layer for the shared links T^0 = L (weights only, formed at lime_set_weights)
   void *sh_That, *sh_Q2, *sh_K2, *sh_G2t, *sh_U2t, *sh_V2t;
   float *sh_cQ, *sh_cK;
+  // feed-forward networks (k_ffn_simt.cu, k_score_head_tc.cu): the caller's description plus derived device data
+  bool have_head, have_ctx_mlp;
+  lime_ffn head, ctx_mlp;
+  int ctx_dc;            // context features per user
+  void* head_W1bT;       // [w0 x d] bf16: the T half of the head's first layer, transposed (tensor-core path)
+  float* head_w2;        // [w_last] fp32 copy of the head's last layer
+  float* ctx_first;      // [ell x w0] fp32: (L W_0[:d]) + b_0 of the context MLP
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
   float attn_scale, cand_scale, ln_eps;
   int d_ff, d_h;
@@ -184,6 +191,32 @@ lime_status launch_score_tc(const ScoreArgs& a, int* err, cudaStream_t st);
 // the same with rows taken from corpus-level caches by cand_ids (fixed C per user), k_score_gather_tc.cu
 bool score_gather_tc_supported(const ScoreArgs& a);
 lime_status launch_score_gather_tc(const ScoreArgs& a, int* err, cudaStream_t st);
+
+// one-thread kernel whose only wait can never be satisfied (self-test of the bounded waits, tc_host.cu)
+lime_status launch_wait_expiry(int* err, uint64_t limit_ns, int code, cudaStream_t st);
+
+// ---- feed-forward networks: Eq. 2 and the interaction network of Sec. 3.3 ------------------------------------------
+// layers after the first (whose input is a concatenation and is handled split): W[i] [in_w[i] x out_w[i]], b[i] nullable
+struct FfnArgs {
+  int n_layers;
+  int in_w[LIME_FFN_MAX_HIDDEN + 1], out_w[LIME_FFN_MAX_HIDDEN + 1];
+  const void* W[LIME_FFN_MAX_HIDDEN + 1];
+  const float* b[LIME_FFN_MAX_HIDDEN + 1];
+};
+// Y = X . W (+ bias) for a few rows: fp32 [M x N] and / or bf16 transposed per group of rows [M/group][N][group]
+lime_status launch_rows_times_w(const void* X, int x_dtype, int64_t M, int K, const void* W, int w_dtype, int ldw, int N,
+                                const float* bias, float* Y, void* Yt, int group, const char* name, cudaStream_t st);
+lime_status launch_link_ctx_mlp(int dtype, const float* first, const void* user_ctx, int d_c, const void* W0c, int w0, int B,
+                                int ell, const FfnArgs& f, float* out, cudaStream_t st);
+// generic scorer through the interaction network; LSW fp32 [B x ell x w0], W0t = rows d.. of the first layer [d x w0]
+lime_status launch_score_head_simt(const ScoreArgs& a, const float* LSW, const void* W0t, const float* b0, int w0,
+                                   const FfnArgs& f, cudaStream_t st);
+// one hidden layer of n1 units on tensor cores; LSWt bf16 [B x n1 x ell], W1bT bf16 [n1 x d], w2 fp32 [n1]
+struct ScoreHeadArgs {
+  const void* LSWt; const void* W1bT; const float* b1; const float* w2; const float* b2; int n1;
+};
+bool score_head_tc_supported(const ScoreArgs& a, int n1);
+lime_status launch_score_head_tc(const ScoreArgs& a, const ScoreHeadArgs& h, int* err, cudaStream_t st);
 
 // ---- tensor-core XOR layer (bf16, d = d_ff = 128, H * ell = 128) ----------------------------------------------
 // plain_v: WprepT's third segment is W_V^T (link values formed as they stand) instead of the folded gate / up products

@@ -52,19 +52,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // in *err (if not already set) and returns false; callers then leave their loops, so the CTA always reaches its
 // final barrier, frees its TMEM and exits.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err, int where) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, int* err, int where, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0x3ff) == 0) {
-      if (global_timer_ns() - t0 > kWaitLimitNs || *(volatile int*)err != 0) {
+      if (global_timer_ns() - t0 > limit_ns || *(volatile int*)err != 0) {
         atomicCAS(err, 0, where);
         return false;
       }
     }
   }
   return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* err, int where) {
+  return mbar_wait_limit(bar, parity, err, where, kWaitLimitNs);
 }
 
 // Bounded wait that records nothing (used on the way out, when the error word is already set).
@@ -227,6 +230,19 @@ __device__ __forceinline__ uint64_t make_sdesc_k_sw128(uint32_t smem_addr) {
   return d;
 }
 
+// The same for rows of `row_bytes` = 128, 64 or 32 bytes (64, 32 or 16 bf16 of the contraction index per row), laid out
+// by a TMA load whose swizzle span equals the row: 8-row groups are 8 * row_bytes apart and the descriptor names the
+// matching swizzle mode.  Stepping K by 16 elements advances the start address by 32 bytes in every mode.
+__device__ __forceinline__ uint64_t make_sdesc_k_sw(uint32_t smem_addr, uint32_t row_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)((8u * row_bytes) >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)(row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6)) << 61;      // 128-, 64-, 32-byte swizzle
+  return d;
+}
+
 // Shared-memory matrix descriptor for an MN-major bf16 operand held as [K rows x 64 MN elements] 128B-swizzled
 // sub-tiles (a row-major [K x MN] matrix loaded by TMA in 64-column boxes): 8 K-rows are 1024 B apart (stride
 // offset), the next 64 MN elements live `mn_chunk_bytes` further (leading offset = distance between sub-tiles).
@@ -262,6 +278,10 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
 // 128-byte swizzle.  Returns false if the driver entry point is unavailable or the encode fails.
 bool make_tmap_bf16_sw128(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
                           uint32_t box_rows);
+// Row-major bf16 matrix [rows x cols], box [box_rows x box_cols] with box_cols in {64, 32, 16}: rows of the box land
+// box_cols * 2 bytes apart under the swizzle of that span (what make_sdesc_k_sw describes).
+bool make_tmap_bf16_kmajor(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                           uint32_t box_rows, uint32_t box_cols);
 // Kernels that need more than 48 KB of dynamic shared memory must have the limit raised once per device; `done` is
 // the caller's per-kernel record (one flag per device ordinal).
 constexpr int kMaxDeviceOrdinals = 64;

@@ -40,6 +40,22 @@ bool make_tmap_bf16_sw128(CUtensorMap* out, const void* base, uint64_t rows, uin
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_tmap_bf16_kmajor(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_elems,
+                           uint32_t box_rows, uint32_t box_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || rows == 0 || box_rows == 0 || box_rows > 256 || cols < box_cols) return false;
+  if (box_cols != 64 && box_cols != 32 && box_cols != 16) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15u) || (pitch_elems * 2) % 16) return false;
+  const cuuint64_t gdim[2] = {cols, rows};
+  const cuuint64_t gstride[1] = {pitch_elems * 2};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUtensorMapSwizzle sw = box_cols == 64 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                               : (box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 lime_status ensure_dynamic_smem(const void* kernel, int bytes, bool (&done)[kMaxDeviceOrdinals]) {
   int dev = 0;
   LIME_CUDA(cudaGetDevice(&dev));
@@ -64,6 +80,24 @@ bool make_tmap_bf16_plain(CUtensorMap* out, const void* base, uint64_t rows, uin
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Self-test of the bounded waits: one thread waits on an mbarrier that nothing ever arrives at; after `limit_ns` the
+// wait gives up, records `code` in the status word and the kernel returns.
+__global__ void k_wait_expiry(int* err, unsigned long long limit_ns, int code) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    tc::mbar_init(&bar, 1);
+    tc::fence_barrier_init();
+    tc::mbar_wait_limit(&bar, 0, err, code, limit_ns);
+  }
+}
+
+lime_status launch_wait_expiry(int* err, uint64_t limit_ns, int code, cudaStream_t st) {
+  ProfScope _p("k_wait_expiry", st);
+  k_wait_expiry<<<1, 32, 0, st>>>(err, (unsigned long long)limit_ns, code);
+  LIME_LAUNCH_CHECK("k_wait_expiry");
+  return LIME_OK;
 }
 
 }  // namespace lime

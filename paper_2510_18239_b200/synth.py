@@ -174,6 +174,17 @@ def layer_weights(seed: int, wl: Workload) -> Dict[str, np.ndarray]:
     return out
 
 
+def ffn_weights(seed: int, stream: str, widths, dtype: str, bias_std: float = 0.1):
+    """Weights of a feed-forward network with layer widths `widths` = (in, hidden..., out): a list of
+    (W [in_i x out_i] in storage format, variance 1/in_i; b [out_i] fp32, std `bias_std`)."""
+    out = []
+    for i, (a, b) in enumerate(zip(widths[:-1], widths[1:])):
+        W = normal_storage(seed, f"{stream}_W{i}", (int(a), int(b)), float(a) ** -0.5, dtype)
+        bias = normal_storage(seed, f"{stream}_b{i}", (int(b),), bias_std, F32)
+        out.append((W, bias))
+    return out
+
+
 def make_inputs(wl: Workload, seed: int = 0, with_candidates: bool = True) -> Dict[str, np.ndarray]:
     """All inputs of one batch, as stored arrays (fp32, or uint16 bf16 bit patterns) and int32 indices.
 

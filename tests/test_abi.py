@@ -48,3 +48,13 @@ def test_version_string_and_host_side_validation():
 def test_struct_layouts_match_header():
     assert ctypes.sizeof(binding.lime_config) == 13 * 4          # 12 fields of the paper's model + cand_heads
     assert ctypes.sizeof(binding.lime_weights) == 8 * (1 + 6 * binding.LIME_MAX_LAYERS + 3)
+    assert ctypes.sizeof(binding.lime_ffn) == 4 * 4 + 8 * 8      # n_hidden + 3 widths, 4 weight and 4 bias pointers
+
+
+def test_ffn_entry_points_validate_on_the_host():
+    lib = binding.load_library()
+    assert lib.lime_set_head(None, None, None) == 1
+    assert lib.lime_set_context_mlp(None, 4, None, None) == 1
+    assert lib.lime_contextualize_links(None, None, 1, None, None) == 1
+    assert lib.lime_head_workspace_bytes(None, 4) == 0
+    assert lib.lime_score_candidates_head(None, None, 1, None, None, None, 1, 1, None, 0, None, None, None, 0, None) == 1
