@@ -189,7 +189,15 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample(wl, inp, users, budget_s=None, phi="softmax", cand_heads=False):
+HEAD_SEED = 11
+
+
+def head_layers(wl, n1):
+    """The interaction network used with --head: one hidden layer of n1 units (App. C lists [96] for the industrial model)."""
+    return synth.ffn_weights(HEAD_SEED, "head", (2 * wl.d, n1, 1), wl.dtype)
+
+
+def oracle_sample(wl, inp, users, budget_s=None, phi="softmax", cand_heads=False, head=0):
     """Time the fp64 oracle (as it stands) on `users` of the batch: gather + encode + precompute + score."""
     from oracle import lime_oracle as O
     from tests import lime_helpers as Hh
@@ -198,9 +206,10 @@ def oracle_sample(wl, inp, users, budget_s=None, phi="softmax", cand_heads=False
     off = O.lengths_to_offsets(inp["lengths"])
 
     tab = Hh.LazyTable64(inp["table"], wl.dtype)   # widens only the rows the sample touches (the table is GBs)
+    head64 = [(synth.storage_to_f64(W, wl.dtype), b.astype(np.float64)) for W, b in head_layers(wl, head)] if head else None
     done, t0 = 0, time.perf_counter()
     for b in users:
-        Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg, cand_heads=cand_heads)
+        Hh.oracle_user(inp, wl, b, off, tab, links64, layers, cfg, cand_heads=cand_heads, head=head64)
         done += 1
         if budget_s is not None and time.perf_counter() - t0 > budget_s:
             break
@@ -221,14 +230,14 @@ def run_reference(args, wl):
     if rank != 0:
         return
     inp = synth.make_inputs(wl, seed=0)
-    _, t_user = oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads)          # calibrates the per-step sample; also the first warm-up
+    _, t_user = oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads, head=args.head)          # calibrates the per-step sample; also the first warm-up
     users_per_step = 2 if (wl.B >= 2 and 2 * t_user * args.steps < 120.0) else 1
     for _ in range(max(0, args.warmup - 1)):
-        oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads)
+        oracle_sample(wl, inp, range(1), phi=args.phi, cand_heads=args.cand_heads, head=args.head)
     times = []
     for s in range(args.steps):
         users = [(s * users_per_step + u) % wl.B for u in range(users_per_step)]
-        _, dt = oracle_sample(wl, inp, users, phi=args.phi, cand_heads=args.cand_heads)
+        _, dt = oracle_sample(wl, inp, users, phi=args.phi, cand_heads=args.cand_heads, head=args.head)
         times.append(dt)
     total = sum(times)
     value = users_per_step * wl.C * args.steps / total
@@ -306,6 +315,18 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     links = Bd.to_device(inp["links"], wl.dtype, dev)
     wts = {k: Bd.to_device(inp[k], wl.dtype, dev) for k in ("Wq", "Wk", "Wv", "Wg", "Wu", "Wo")}
     lime.set_weights(links, [{k: wts[k][j] for k in wts} for j in range(wl.n_layers)])
+    head_dev = None
+    if args.head:
+        head_dev = [(Bd.to_device(W, wl.dtype, dev), torch.from_numpy(b).to(dev)) for W, b in head_layers(wl, args.head)]
+        lime.set_head(head_dev)
+        head_ws = torch.empty(Bd.lime_head_workspace_bytes(lime.ctx, wl.B), dtype=torch.uint8, device=dev)
+
+    def score(ls_, W_, T_, ids_, out_, corpus=None):
+        # the per-candidate stage: the dot product <O_c, T_c>, or (--head) the interaction network on [O_c | T_c]
+        if args.head:
+            Bd.lime_score_candidates_head(lime.ctx, ls_, wl.B, W_, T_, None, wl.C, wl.B * wl.C, ids_, out_, head_ws, corpus)
+        else:
+            Bd.lime_score_candidates(lime.ctx, ls_, wl.B, W_, T_, None, wl.C, wl.B * wl.C, ids_, out_, corpus)
 
     sets, host_sets = [], []
     pre_ms = []
@@ -348,7 +369,7 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
         # the lookup applies the first layer's LayerNorm on the way (every layer reads the history through it only)
         Bd.lime_gather_history_normalized(ctx, table, s["hist_ids"], h)
         Bd.lime_encode_user_normalized(ctx, h, off, wl.B, None, ls, ws)
-        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+        score(ls, s["W"], s["T"], None, logits)
 
     def barrier():
         if world > 1:
@@ -421,12 +442,12 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     score_reps = max(20, min(200, args.steps))
     for i in range(ROTATE):
         s = sets[i]
-        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+        score(ls, s["W"], s["T"], None, logits)
     torch.cuda.synchronize()
     e0.record()
     for i in range(score_reps):
         s = sets[i % ROTATE]
-        Bd.lime_score_candidates(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits)
+        score(ls, s["W"], s["T"], None, logits)
     e1.record()
     torch.cuda.synchronize()
     score_alone_ms = e0.elapsed_time(e1) / score_reps
@@ -437,6 +458,12 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     #      Three streams pipeline consecutive requests - copies in | kernels | logits out - over two request slots, as
     #      a server would; every step's copies are inside the timed region.
     w_corpus = lime.precompute_candidate_links(table)
+    # a context whose row width is ell_c: the row lookup applied to the cached weights
+    lime_w = Bd.Lime(lime.ell_c, (lime.ell_c + 127) // 128, 1, 1, dtype=dt)
+    Tg = Wg = None
+    if args.head:
+        Tg = torch.empty((wl.B * wl.C, wl.d), dtype=lime.tdtype, device=dev)
+        Wg = torch.empty((wl.B * wl.C, lime.ell_c), dtype=lime.tdtype, device=dev)
     SLOTS = 2
     d_len = [torch.empty(wl.B, dtype=torch.int32, device=dev) for _ in range(SLOTS)]
     d_hid = [torch.empty(max_total, dtype=torch.int32, device=dev) for _ in range(SLOTS)]
@@ -460,7 +487,13 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
         Bd.lime_gather_history_normalized(ctx, table, d_hid[k][:n], h)
         Bd.lime_encode_user_normalized(ctx, h, off, wl.B, None, ls, ws)
         # candidates are scored straight from the corpus caches by id (no gather of their rows)
-        Bd.lime_score_candidates(ctx, ls, wl.B, w_corpus, table, None, wl.C, wl.B * wl.C, d_cid[k], d_logits[k])
+        if args.head:
+            # the tensor-core interaction-network scorer takes dense streams: the candidates' rows are looked up first
+            Bd.lime_gather_history(ctx, table, d_cid[k], Tg)
+            Bd.lime_gather_history(lime_w.ctx, w_corpus, d_cid[k], Wg)
+            score(ls, Wg, Tg, None, d_logits[k])
+        else:
+            score(ls, w_corpus, table, d_cid[k], d_logits[k])
 
     def e2e_copy_out(i):
         k = i % SLOTS
@@ -511,8 +544,8 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     torch.cuda.synchronize()
     eg0, eg1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     eg0.record()
-    for i in range(50):
-        Bd.lime_score_candidates(ctx, ls, wl.B, w_corpus, table, None, wl.C, wl.B * wl.C, d_cid[i % SLOTS], d_logits[i % SLOTS])
+    for i in range(50 if not args.head else 0):
+        score(ls, w_corpus, table, d_cid[i % SLOTS], d_logits[i % SLOTS])
     eg1.record()
     torch.cuda.synchronize()
     score_by_id_ms = eg0.elapsed_time(eg1) / 50
@@ -530,6 +563,10 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     e2e_ms = e0.elapsed_time(e1)
     e2e_ms = shard.max_over_ranks(e2e_ms, dev)
     e2e_value = shard.sum_over_ranks(wl.B * wl.C * args.steps, dev) / (e2e_ms * 1e-3)
+    extras = None
+    if rank == 0 and world == 1 and not args.no_extras:
+        extras = measure_extras(args, wl, lime, dict(table=table, sets=sets, hist=hist, off=off, ls=ls, ws=ws, logits=logits,
+                                                     w_corpus=w_corpus, d_cid=d_cid, lime_w=lime_w), dev)
     Bd.lime_device_status(ctx)          # raises if any bounded in-kernel wait gave up during the run
 
     if rank == 0:
@@ -575,7 +612,7 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget, phi=args.phi, cand_heads=args.cand_heads)
+            n_done, dt_s = oracle_sample(wl, inp, range(wl.B), budget_s=args.cpu_budget, phi=args.phi, cand_heads=args.cand_heads, head=args.head)
             cpu = {"value": n_done * wl.C / dt_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                    "sample": f"first {n_done} users x {wl.C} candidates of the same workload, {dt_s:.1f} s "
                              "(gather+encode+precompute+score, fp64 numpy)"}
@@ -596,9 +633,15 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
                 "precompute": {"ms": pre_ms, "candidates": wl.B * wl.C, "candidates_per_s": wl.B * wl.C / (pre_ms * 1e-3),
                                **roofline_entry(models["k_precompute"], pre_ms, pk)},
                 "cpu_baseline": cpu, "peaks": pk}
+        line["config"]["head"] = args.head or None
+        if extras:
+            if extras.get("head"):
+                hm = dict(bytes=models["k_score"]["bytes"])
+                extras["head"].update(roofline_entry(hm, extras["head"]["ms_alone"], pk))
+            line["extras"] = extras
         if with_sweeps and world == 1:
             # free this workload's buffers before the sweep points allocate theirs
-            del sets, host_sets, table, hist, ws, w_corpus, wscratch, d_hid, d_cid, d_logits, h_logits
+            del sets, host_sets, table, hist, ws, w_corpus, wscratch, d_hid, d_cid, d_logits, h_logits, extras
             if not args.no_graph:
                 del step_graphs, graphs, e2e_graphs
             torch.cuda.empty_cache()
@@ -608,6 +651,99 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
         sampler.stop()
     if world > 1:
         dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- the stages around the core path
+def measure_extras(args, wl, lime, bufs, dev):
+    """Three short measurements on the bench workload, each with CUDA events on the launching stream:
+    head      the per-candidate stage through a one-hidden-layer interaction network (Sec. 3.3; 96 units, App. C) alone;
+    link_ctx  Eq. 2 (L^C = MLP(L (+) E^C), 32 context features, one hidden layer of d units) and the encode that takes
+              per-user link rows, next to the encode on the shared links;
+    overlap   the user side running beside a stand-in for candidate retrieval on a second stream (Sec. 3.3: the user-side
+              computation runs in parallel with retrieval): fetching the candidates' cached weight rows and embedding
+              rows by id into dense streams; alone, alone, and together."""
+    import torch
+    from paper_2510_18239_b200 import binding as Bd
+    ctx, table, sets = lime.ctx, bufs["table"], bufs["sets"]
+    ls, off, ws, logits, hist = bufs["ls"], bufs["off"], bufs["ws"], bufs["logits"], bufs["hist"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps, warm=3):
+        for i in range(warm):
+            fn(i)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(reps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    out = {}
+    # ---- interaction network
+    n1 = args.head or 96
+    hd = [(Bd.to_device(W, wl.dtype, dev), torch.from_numpy(b).to(dev)) for W, b in head_layers(wl, n1)]
+    lime.set_head(hd)
+    hws = torch.empty(Bd.lime_head_workspace_bytes(ctx, wl.B), dtype=torch.uint8, device=dev)
+
+    def head_score(i):
+        s = sets[i % ROTATE]
+        Bd.lime_score_candidates_head(ctx, ls, wl.B, s["W"], s["T"], None, wl.C, wl.B * wl.C, None, logits, hws)
+
+    Bd.lime_profile_start(16)
+    head_score(0)
+    torch.cuda.synchronize()
+    rec, _ = Bd.lime_profile_stop(16)
+    out["head"] = {"hidden": [n1], "ms_alone": timed(head_score, 40), "kernels": [k for k, _ in rec],
+                   "note": "k_head_lsw (per-user link states x W_0[:d]) + the scorer; bytes per candidate as the dot-product scorer"}
+    # ---- Eq. 2 and the encode on per-user link rows
+    d_c = 32
+    mlp = [(Bd.to_device(W, wl.dtype, dev), torch.from_numpy(b).to(dev)) for W, b in
+           synth.ffn_weights(HEAD_SEED, "ctx", (wl.d + d_c, wl.d, wl.d), wl.dtype)]
+    lime.set_context_mlp(d_c, mlp)
+    ec = Bd.to_device(synth.normal_storage(HEAD_SEED, "ec", (wl.B, d_c), 1.0, wl.dtype), wl.dtype, dev)
+    lc = torch.empty((wl.B, wl.ell, wl.d), dtype=torch.float32, device=dev)
+    s0 = sets[0]
+    h0 = hist[: s0["total"]]
+    Bd.lime_lengths_to_offsets(ctx, s0["lengths"], off)
+    Bd.lime_gather_history_normalized(ctx, table, s0["hist_ids"], h0)
+    t_ctx = timed(lambda i: Bd.lime_contextualize_links(ctx, ec, wl.B, lc), 40)
+    t_enc_shared = timed(lambda i: Bd.lime_encode_user_normalized(ctx, h0, off, wl.B, None, ls, ws), 40)
+    t_enc_ctx = timed(lambda i: Bd.lime_encode_user_normalized(ctx, h0, off, wl.B, lc, ls, ws), 40)
+    out["link_ctx"] = {"d_c": d_c, "hidden": [wl.d], "contextualize_ms": t_ctx, "encode_shared_links_ms": t_enc_shared,
+                       "encode_per_user_links_ms": t_enc_ctx}
+    # ---- encode beside the retrieval stand-in
+    cid = bufs["d_cid"][0]
+    Tg = torch.empty((wl.B * wl.C, wl.d), dtype=lime.tdtype, device=dev)
+    Wg = torch.empty((wl.B * wl.C, lime.ell_c), dtype=lime.tdtype, device=dev)
+    w_corpus = bufs["w_corpus"]
+    lime_w = bufs["lime_w"]                     # a context of row width ell_c: the row lookup applied to the cached weights
+
+    def fetch(i):
+        Bd.lime_gather_history(ctx, table, cid, Tg)
+        Bd.lime_gather_history(lime_w.ctx, w_corpus, cid, Wg)
+
+    def encode(i):
+        Bd.lime_encode_user_normalized(ctx, h0, off, wl.B, None, ls, ws)
+
+    t_fetch, t_enc = timed(fetch, 20), timed(encode, 20)
+    side = torch.cuda.Stream(dev)
+    fork, join = torch.cuda.Event(), torch.cuda.Event()
+
+    def both(i):
+        fork.record()
+        side.wait_event(fork)
+        with torch.cuda.stream(side):
+            fetch(i)
+            join.record(side)
+        encode(i)
+        torch.cuda.current_stream().wait_event(join)
+
+    t_both = timed(both, 20)
+    out["overlap"] = {"encode_ms": t_enc, "retrieval_standin_ms": t_fetch, "together_ms": t_both,
+                      "hidden_fraction": max(0.0, (t_enc + t_fetch - t_both) / max(min(t_enc, t_fetch), 1e-9)),
+                      "standin": "lookup of the candidates' cached weight rows and embedding rows by id into dense streams, on a second stream"}
+    return out
 
 
 # ----------------------------------------------------------------------------- the metric's curves, point by point
@@ -784,6 +920,9 @@ def main():
                     help="attention activation of the XOR layers: online softmax (default) or SiLU(s) / n (Algorithms 1-2)")
     ap.add_argument("--cand-heads", action="store_true",
                     help="candidate side head by head (Eq. 1 applied to Eq. 4): H * ell cached weights per candidate")
+    ap.add_argument("--head", type=int, default=0,
+                    help="score through an interaction network with one hidden layer of this many units (Sec. 3.3; 0 = dot product)")
+    ap.add_argument("--no-extras", action="store_true", help="leave out the `extras` object (head, link_ctx, overlap)")
     ap.add_argument("--no-graph", action="store_true", help="launch every step from the host instead of replaying CUDA graphs")
     ap.add_argument("--no-sweeps", action="store_true",
                     help="leave out the `sweeps` object (points of the candidate sweep, the history sweep and production_ragged)")
@@ -811,7 +950,7 @@ def main():
             run_ours(args, base.replace(n_min=N, n_max=N, B=args.B or base.B))
     else:
         # the default run carries the metric's curves in its one line; explicit workloads and multi-GPU runs do not
-        plain_default = args.workload == "bf16_baseline" and not (args.C or args.N or args.B) and args.phi == "softmax" and not args.cand_heads
+        plain_default = args.workload == "bf16_baseline" and not (args.C or args.N or args.B) and args.phi == "softmax" and not args.cand_heads and not args.head
         run_ours(args, wl, with_sweeps=plain_default and not args.no_sweeps and int(os.environ.get("WORLD_SIZE", "1")) == 1)
 
 

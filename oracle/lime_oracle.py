@@ -366,9 +366,10 @@ def score_candidates_head(W: np.ndarray, LS: np.ndarray, T: np.ndarray, layers) 
 # --------------------------------------------------------------------------- #
 def run_user(E: np.ndarray, L: np.ndarray, layers, cfg: OracleConfig, T: np.ndarray,
              LC: Optional[np.ndarray] = None, W: Optional[np.ndarray] = None,
-             cand_w: Optional[Dict[str, np.ndarray]] = None, cand_heads: bool = False):
+             cand_w: Optional[Dict[str, np.ndarray]] = None, cand_heads: bool = False, head=None):
     """Encode one user and score that user's candidates. Returns (logits [C], link states [l x d], W [C x l]);
-    with cand_heads the candidate side runs head by head (W [C x H x l])."""
+    with cand_heads the candidate side runs head by head (W [C x H x l]); with `head` (layers of the interaction
+    network) the LIME embedding is scored by that network instead of the dot product."""
     cand_w = cand_w or {}
     LP, _ = encode_user(E, L if LC is None else LC, layers, cfg)
     LS = link_states(LP, cand_w.get("Wv_c"))
@@ -378,6 +379,8 @@ def run_user(E: np.ndarray, L: np.ndarray, layers, cfg: OracleConfig, T: np.ndar
         return score_candidates_heads(W, LS, T, cfg), LS, W
     if W is None:
         W = precompute_candidate_links(T, L, cfg, cand_w.get("Wq_c"), cand_w.get("Wk_c"))
+    if head is not None:
+        return score_candidates_head(W, LS, T, head), LS, W
     return score_candidates(W, LS, T), LS, W
 
 

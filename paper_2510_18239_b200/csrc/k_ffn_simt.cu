@@ -33,6 +33,7 @@ k_rows_times_w(const TX* __restrict__ X, int64_t M, int K, const TW* __restrict_
     const float b = bias ? bias[j] : 0.f;
 #pragma unroll
     for (int r = 0; r < FR_ROWS; ++r) acc[r] = b;
+#pragma unroll 8
     for (int k = 0; k < K; ++k) {
       const float w = Store<TW>::ld(W + (int64_t)k * ldw + j);
 #pragma unroll

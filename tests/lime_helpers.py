@@ -29,14 +29,14 @@ def oracle_layers(inp: Dict[str, np.ndarray], wl: synth.Workload, gated_mlp=True
 
 
 def oracle_user(inp, wl, b: int, off: np.ndarray, table64: np.ndarray, links64: np.ndarray, layers, cfg,
-                cand_rows: Optional[np.ndarray] = None, cand_w=None, cand_heads: bool = False):
+                cand_rows: Optional[np.ndarray] = None, cand_w=None, cand_heads: bool = False, head=None, LC=None):
     """Oracle logits / link states / weights for user b (optionally only candidate slots `cand_rows` of that user)."""
     E = O.gather_history(table64, inp["hist_ids"][off[b]:off[b + 1]])
     cids = inp["cand_ids"][b * wl.C:(b + 1) * wl.C]
     if cand_rows is not None:
         cids = cids[cand_rows]
     T = O.gather_history(table64, cids)
-    return O.run_user(E, links64, layers, cfg, T, cand_w=cand_w, cand_heads=cand_heads)
+    return O.run_user(E, links64, layers, cfg, T, LC=LC, cand_w=cand_w, cand_heads=cand_heads, head=head)
 
 
 class LazyTable64:
