@@ -458,6 +458,8 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     #      Three streams pipeline consecutive requests - copies in | kernels | logits out - over two request slots, as
     #      a server would; every step's copies are inside the timed region.
     w_corpus = lime.precompute_candidate_links(table)
+    # one record per item: [embedding row | cached weight row], so that scoring by id touches one place per candidate
+    packed = lime.pack_corpus_cache(table, w_corpus)
     # a context whose row width is ell_c: the row lookup applied to the cached weights
     lime_w = Bd.Lime(lime.ell_c, (lime.ell_c + 127) // 128, 1, 1, dtype=dt)
     Tg = Wg = None
@@ -493,7 +495,7 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
             Bd.lime_gather_history(lime_w.ctx, w_corpus, d_cid[k], Wg)
             score(ls, Wg, Tg, None, d_logits[k])
         else:
-            score(ls, w_corpus, table, d_cid[k], d_logits[k])
+            Bd.lime_score_candidates_packed(ctx, ls, wl.B, packed, d_cid[k], None, wl.C, wl.B * wl.C, d_logits[k])
 
     def e2e_copy_out(i):
         k = i % SLOTS
@@ -545,10 +547,16 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
     eg0, eg1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     eg0.record()
     for i in range(50 if not args.head else 0):
-        score(ls, w_corpus, table, d_cid[i % SLOTS], d_logits[i % SLOTS])
+        Bd.lime_score_candidates_packed(ctx, ls, wl.B, packed, d_cid[i % SLOTS], None, wl.C, wl.B * wl.C, d_logits[i % SLOTS])
     eg1.record()
     torch.cuda.synchronize()
     score_by_id_ms = eg0.elapsed_time(eg1) / 50
+    eg0.record()
+    for i in range(50 if not args.head else 0):
+        score(ls, w_corpus, table, d_cid[i % SLOTS], d_logits[i % SLOTS])
+    eg1.record()
+    torch.cuda.synchronize()
+    score_by_id_two_arrays_ms = eg0.elapsed_time(eg1) / 50
     h2d = d2h = 0
     e0.record(s_in)
     t_issue = time.perf_counter()
@@ -622,12 +630,13 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
                 "data": "synthetic", "config": dict(workload_config(wl), launch=launch_mode(args), phi=args.phi, cand_heads=bool(args.cand_heads)), "clocks": clocks,
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d // args.steps, "d2h_bytes_per_step": d2h // args.steps,
                         "ms_per_step": e2e_ms / args.steps, "host_issue_ms_per_step": 1e3 * t_issue / args.steps,
-                        "score_by_id_alone_ms": score_by_id_ms,
+                        "score_by_id_alone_ms": score_by_id_ms, "score_by_id_two_arrays_ms": score_by_id_two_arrays_ms,
                         "score_by_id_roofline": dict(kernel="k_score_gather_tc", **roofline_entry(models["k_score_gather_tc"], score_by_id_ms, pk),
                                                      traffic=ncu_traffic("k_score_gather_tc", wl, args),
-                                                     note="random 128-byte pieces; the copy peak is for contiguous streams"),
+                                                     note="random rows of packed corpus records [embedding | weights] (score_by_id_two_arrays_ms: "
+                                                          "the same from two separate caches); the copy peak is for contiguous streams"),
                         "how": "pinned host ids -> H2D | offsets, history gather, encode, scoring by candidate id from the resident "
-                               "corpus caches | logits D2H; three streams, two request slots"},
+                               "packed corpus records | logits D2H; three streams, two request slots"},
                 "gpu_launches": int(round(launches_per_step * args.steps)), "roofline": roofline, "scoring_roofline": scoring,
                 "kernels": kernels[:14],
                 "precompute": {"ms": pre_ms, "candidates": wl.B * wl.C, "candidates_per_s": wl.B * wl.C / (pre_ms * 1e-3),
@@ -641,7 +650,7 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
             line["extras"] = extras
         if with_sweeps and world == 1:
             # free this workload's buffers before the sweep points allocate theirs
-            del sets, host_sets, table, hist, ws, w_corpus, wscratch, d_hid, d_cid, d_logits, h_logits, extras
+            del sets, host_sets, table, hist, ws, w_corpus, packed, wscratch, d_hid, d_cid, d_logits, h_logits, extras
             if not args.no_graph:
                 del step_graphs, graphs, e2e_graphs
             torch.cuda.empty_cache()

@@ -180,6 +180,17 @@ LIME_API lime_status lime_score_candidates(lime_ctx* ctx, const void* link_state
                                   const int32_t* cand_ids, int64_t corpus_rows, int32_t* dev_flag, float* logits,
                                   void* stream);
 
+/* Corpus caches as one record per item (Sec. 3.3: the cached weights sit beside the item embedding): packed [corpus_rows x
+ * (d + ell_c)] in config.dtype, record v = [ cand_emb[v, 0..d) | cand_w[v, 0..ell_c) ].  lime_pack_corpus_cache builds it
+ * from the two separate caches (offline, whenever they change).  lime_score_candidates_packed is lime_score_candidates
+ * with cand_ids over such records: a candidate's embedding and weights then come from one place in memory instead of
+ * two.  Same logits, same treatment of ids outside [0, corpus_rows), same meaning of cand_off / C / total_cands. */
+LIME_API lime_status lime_pack_corpus_cache(lime_ctx* ctx, const void* cand_emb, const void* cand_w, int64_t corpus_rows,
+                                   void* packed, void* stream);
+LIME_API lime_status lime_score_candidates_packed(lime_ctx* ctx, const void* link_states, int32_t B, const void* packed,
+                                         int64_t corpus_rows, const int32_t* cand_ids, const int32_t* cand_off, int32_t C,
+                                         int64_t total_cands, int32_t* dev_flag, float* logits, void* stream);
+
 /* The two small feed-forward networks the paper names without a formula.  Both are read as x <- ReLU(x W_i + b_i)
  * for each of n_hidden hidden layers followed by one linear layer; W[i] is [in_i x out_i] row-major in config.dtype,
  * b[i] fp32 [out_i] or NULL (no bias); all are device pointers, borrowed until replaced or lime_destroy. */

@@ -55,7 +55,7 @@ class lime_ffn(ctypes.Structure):
 EXPORTS = ("lime_create", "lime_destroy", "lime_set_weights", "lime_workspace_bytes", "lime_lengths_to_offsets",
            "lime_gather_history", "lime_gather_history_normalized", "lime_precompute_candidate_links", "lime_xor_layer",
            "lime_encode_user", "lime_encode_user_normalized",
-           "lime_score_candidates", "lime_set_context_mlp", "lime_contextualize_links", "lime_set_head",
+           "lime_score_candidates", "lime_pack_corpus_cache", "lime_score_candidates_packed", "lime_set_context_mlp", "lime_contextualize_links", "lime_set_head",
            "lime_head_workspace_bytes", "lime_score_candidates_head", "lime_precompute_candidate_links_noalloc", "lime_device_status", "lime_selftest_wait_expiry", "lime_profile_start", "lime_profile_stop", "lime_last_cuda_error",
            "lime_version")
 
@@ -86,6 +86,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.lime_encode_user.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_encode_user_normalized.argtypes = [vp, vp, vp, i32, i64, vp, vp, vp, sz, vp]
     lib.lime_score_candidates.argtypes = [vp, vp, i32, vp, vp, vp, i32, i64, vp, i64, vp, vp, vp]
+    lib.lime_pack_corpus_cache.argtypes = [vp, vp, vp, i64, vp, vp]
+    lib.lime_score_candidates_packed.argtypes = [vp, vp, i32, vp, i64, vp, vp, i32, i64, vp, vp, vp]
     lib.lime_set_context_mlp.argtypes = [vp, i32, ctypes.POINTER(lime_ffn), vp]
     lib.lime_contextualize_links.argtypes = [vp, vp, i32, vp, vp]
     lib.lime_set_head.argtypes = [vp, ctypes.POINTER(lime_ffn), vp]
@@ -206,6 +208,19 @@ def lime_score_candidates(ctx: int, link_states: torch.Tensor, B: int, cand_w: t
                                                 C, total_cands, _ptr(cand_ids), int(corpus_rows or 0), _ptr(dev_flag),
                                                 _ptr(logits), _stream()),
            "lime_score_candidates")
+
+
+def lime_pack_corpus_cache(ctx: int, cand_emb: torch.Tensor, cand_w: torch.Tensor, packed: torch.Tensor) -> None:
+    _check(load_library().lime_pack_corpus_cache(ctx, _ptr(cand_emb), _ptr(cand_w), cand_emb.shape[0], _ptr(packed), _stream()),
+           "lime_pack_corpus_cache")
+
+
+def lime_score_candidates_packed(ctx: int, link_states: torch.Tensor, B: int, packed: torch.Tensor, cand_ids: torch.Tensor,
+                                 cand_off: Optional[torch.Tensor], C: int, total_cands: int, logits: torch.Tensor,
+                                 dev_flag: Optional[torch.Tensor] = None) -> None:
+    _check(load_library().lime_score_candidates_packed(ctx, _ptr(link_states), B, _ptr(packed), packed.shape[0], _ptr(cand_ids),
+                                                       _ptr(cand_off), C, total_cands, _ptr(dev_flag), _ptr(logits), _stream()),
+           "lime_score_candidates_packed")
 
 
 def make_ffn(layers) -> lime_ffn:
@@ -394,6 +409,18 @@ class Lime:
         total = total_cands if total_cands is not None else (cand_ids.numel() if cand_ids is not None else cand_emb.shape[0])
         logits = torch.empty(total, dtype=torch.float32, device=link_states.device)
         lime_score_candidates(self.ctx, link_states, B, cand_w, cand_emb, cand_off, C, total, cand_ids, logits, corpus_rows, dev_flag)
+        return logits
+
+    def pack_corpus_cache(self, cand_emb: torch.Tensor, cand_w: torch.Tensor) -> torch.Tensor:
+        packed = torch.empty((cand_emb.shape[0], self.cfg.d + self.ell_c), dtype=self.tdtype, device=cand_emb.device)
+        lime_pack_corpus_cache(self.ctx, cand_emb, cand_w, packed)
+        return packed
+
+    def score_candidates_packed(self, link_states: torch.Tensor, packed: torch.Tensor, cand_ids: torch.Tensor, C: int = 0,
+                                cand_off: Optional[torch.Tensor] = None, dev_flag: Optional[torch.Tensor] = None) -> torch.Tensor:
+        logits = torch.empty(cand_ids.numel(), dtype=torch.float32, device=link_states.device)
+        lime_score_candidates_packed(self.ctx, link_states, link_states.shape[0], packed, cand_ids, cand_off, C, cand_ids.numel(),
+                                     logits, dev_flag)
         return logits
 
     # ---- feed-forward networks (Eq. 2; the interaction network of Sec. 3.3)

@@ -140,7 +140,7 @@ template <typename T>
 __global__ void __launch_bounds__(SC_WARPS * 32)
 k_score_simt(const T* __restrict__ LS, const T* __restrict__ W, const T* __restrict__ Tc, int B, int ell, int d,
              const int32_t* __restrict__ cand_off, int C, int64_t total, const int32_t* __restrict__ cand_ids,
-             int64_t corpus_rows, int32_t* __restrict__ dev_flag, float* __restrict__ logits) {
+             int64_t corpus_rows, int32_t* __restrict__ dev_flag, float* __restrict__ logits, int64_t ldw, int64_t ldt) {
   extern __shared__ float smem[];
   float* Ls = smem;                  // [ell][d]
   float* ws = Ls + ell * d;          // [warps][ell]
@@ -169,13 +169,13 @@ k_score_simt(const T* __restrict__ LS, const T* __restrict__ W, const T* __restr
         }
         continue;
       }
-      for (int l = lane; l < ell; l += 32) ww[l] = Store<T>::ld(W + row * ell + l);
+      for (int l = lane; l < ell; l += 32) ww[l] = Store<T>::ld(W + row * ldw + l);
       __syncwarp();
       float dot = 0.f;
       for (int k = lane; k < d; k += 32) {
         float o = 0.f;
         for (int l = 0; l < ell; ++l) o = fmaf(ww[l], Ls[l * d + k], o);
-        dot = fmaf(o, Store<T>::ld(Tc + row * d + k), dot);
+        dot = fmaf(o, Store<T>::ld(Tc + row * ldt + k), dot);
       }
       dot = warp_sum(dot);
       if (lane == 0) logits[i] = dot;
@@ -191,19 +191,44 @@ lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st) {
   if (smem > 200 * 1024) return LIME_UNSUPPORTED_SHAPE;
   const int64_t blocks = (a.total + SC_SLOTS - 1) / SC_SLOTS;
   if (blocks > 0x7fffffffLL) return LIME_UNSUPPORTED_SHAPE;
+  const int64_t ldw = a.ldw ? a.ldw : a.ell, ldt = a.ldt ? a.ldt : a.d;
   ProfScope _p("k_score_simt", st);
   if (a.dtype == LIME_F32) {
     LIME_CUDA(cudaFuncSetAttribute(k_score_simt<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_score_simt<float><<<(int)blocks, SC_WARPS * 32, smem, st>>>((const float*)a.LS, (const float*)a.W, (const float*)a.T,
                                                                  a.B, a.ell, a.d, a.cand_off, a.C, a.total, a.cand_ids,
-                                                                 a.corpus_rows, a.dev_flag, a.logits);
+                                                                 a.corpus_rows, a.dev_flag, a.logits, ldw, ldt);
   } else {
     LIME_CUDA(cudaFuncSetAttribute(k_score_simt<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k_score_simt<__nv_bfloat16><<<(int)blocks, SC_WARPS * 32, smem, st>>>(
         (const __nv_bfloat16*)a.LS, (const __nv_bfloat16*)a.W, (const __nv_bfloat16*)a.T, a.B, a.ell, a.d, a.cand_off,
-        a.C, a.total, a.cand_ids, a.corpus_rows, a.dev_flag, a.logits);
+        a.C, a.total, a.cand_ids, a.corpus_rows, a.dev_flag, a.logits, ldw, ldt);
   }
   LIME_LAUNCH_CHECK("k_score_simt");
+  return LIME_OK;
+}
+
+// ----------------------------------------------------------------------------- packed corpus records
+// One record per item: its embedding row followed by its cached candidate->link weights (Sec. 3.3: the "QK cache" sits
+// beside the item embedding), so that scoring by id touches one place in memory per candidate instead of two.
+template <typename T>
+__global__ void __launch_bounds__(256)
+k_pack_corpus(const T* __restrict__ emb, const T* __restrict__ w, int64_t V, int d, int ell, T* __restrict__ out) {
+  const int rec = d + ell;
+  const int64_t n = V * rec;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t v = i / rec;
+    const int c = (int)(i % rec);
+    out[i] = c < d ? emb[v * d + c] : w[v * ell + (c - d)];
+  }
+}
+
+lime_status launch_pack_corpus(int dtype, const void* emb, const void* w, int64_t V, int d, int ell, void* out, cudaStream_t st) {
+  if (V == 0) return LIME_OK;
+  ProfScope _p("k_pack_corpus", st);
+  if (dtype == LIME_F32) k_pack_corpus<float><<<kSMs * 8, 256, 0, st>>>((const float*)emb, (const float*)w, V, d, ell, (float*)out);
+  else k_pack_corpus<__nv_bfloat16><<<kSMs * 8, 256, 0, st>>>((const __nv_bfloat16*)emb, (const __nv_bfloat16*)w, V, d, ell, (__nv_bfloat16*)out);
+  LIME_LAUNCH_CHECK("k_pack_corpus");
   return LIME_OK;
 }
 

@@ -1,4 +1,4 @@
-// Links attend over the history on the 5th-generation tensor cores at d = 256 (bf16 storage, rows LayerNorm-ed already):
+// Links attend over the history on the 5th-generation tensor cores, 64-token tiles (bf16 storage, rows LayerNorm-ed already):
 //
 //   O[T]_h = phi( Q[T]_h K[S]_h^T * scale ) V[S]_h,  K[S] = X W_K,  V[S] = X W_V,  X = LN(S)                (Eq. 3 / Eq. 7)
 //
@@ -7,42 +7,52 @@
 // once by TMA and used as keys and as values:
 //   scores [128 x 64]   = Q2_block [128 x d] . X_tile^T          (one block of 128 stacked (head, link) rows per work item)
 //   acc    [128 x d]   += P [128 x 64] . X_tile
-// What changes with d = 256 is the budget: the accumulator takes 256 TMEM columns and a block of folded queries 64 KB of
-// shared memory, so the history is walked in tiles of 64 tokens (32 KB per stage, three stages; two score buffers of
-// 64 columns; two P buffers of 16 KB).  The rows read must be LayerNorm-ed already (the lookup or the previous layer's
-// history update stores them so); there is no on-the-fly LayerNorm in this kernel.
+// The history is walked in tiles of 64 tokens, which halves every per-tile buffer against k_link_attn_tc.cu: at d = 256
+// the accumulator takes 256 TMEM columns and a block of folded queries 64 KB of shared memory, which only fits with the
+// small tile (32 KB per stage, three stages; two score buffers of 64 columns; two P buffers of 16 KB).  The geometry is a
+// template parameter (LbCfg).  A d = 128 build with two CTAs per SM (16 KB stages, two threads per row) was measured
+// and dropped: with only two token stages per CTA the tile period is bound by the latency of the copies (31 us per
+// launch on 256 users x 512 tokens against 25 us for k_link_attn_tc.cu).
+// The rows read must be LayerNorm-ed already (the lookup or the previous layer's history update stores them so); there is
+// no on-the-fly LayerNorm in this kernel.
 // Online softmax in the log2 domain with lazy rescale, or SiLU(s) / N(U) with `silu` (Algorithms 1-2), as in
 // k_link_attn_tc.cu.  Persistent CTAs walk (user, chunk) x row-block items; warp 0 TMA producer, warp 1 MMA issuer,
-// warps 2-17 softmax: four threads per stacked row, 16 of the tile's 64 token columns each, and 64 of the 256
-// accumulator columns when a row is rescaled or read out.
+// the other warps softmax: PARTS threads per stacked row, 64 / PARTS of the tile's token columns each, and d / PARTS of
+// the accumulator columns when a row is rescaled or read out.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
 
-constexpr int LB_D = 256, LB_TILE = 64, LB_XSTAGES = 3;
-constexpr int LB_PARTS = 4;
-constexpr int LB_COLS = LB_TILE / LB_PARTS;                   // token columns per thread
-constexpr int LB_OUT = LB_D / LB_PARTS;                       // accumulator columns per thread
-constexpr int LB_SOFTMAX_WARPS = 4 * LB_PARTS, LB_THREADS = 64 + 32 * LB_SOFTMAX_WARPS;
-constexpr uint32_t LB_XSUB = 64 * 128;                        // [64 tokens x 64 features]
-constexpr uint32_t LB_X_STAGE = (LB_D / 64) * LB_XSUB;
-constexpr uint32_t LB_QSUB = 128 * 128;                       // [128 rows x 64 features]
-constexpr uint32_t LB_Q_BUF = (LB_D / 64) * LB_QSUB;
-constexpr int LB_PBUFS = 2;
-constexpr uint32_t LB_P_BUF = 128 * 128;                      // [128 rows x 64 tokens]
-constexpr uint32_t LB_OFF_X = 0;
-constexpr uint32_t LB_OFF_Q2 = LB_XSTAGES * LB_X_STAGE;
-constexpr uint32_t LB_OFF_P = LB_OFF_Q2 + LB_Q_BUF;
-constexpr uint32_t LB_OFF_EXCH = LB_OFF_P + LB_PBUFS * LB_P_BUF;        // [2 tile parities][PARTS][128] maxima, [PARTS][128] sums
-constexpr uint32_t LB_OFF_BAR = LB_OFF_EXCH + 3 * LB_PARTS * 128 * 4;
-constexpr int LB_IDX_CAP = 1025;                              // users + 1 whose offsets are staged in shared memory
-constexpr uint32_t LB_OFF_IDX = LB_OFF_BAR + 256;
-constexpr uint32_t LB_SMEM = LB_OFF_IDX + 2 * LB_IDX_CAP * 4 + 8;
-static_assert(LB_SMEM <= 232448, "shared memory budget of one CTA");
+// Geometry of one build: D features per row, PARTS threads per stacked row, XSTAGES token stages, MINB CTAs per SM.
+template <int D_, int PARTS_, int XSTAGES_, int MINB_>
+struct LbCfg {
+  static constexpr int D = D_, TILE = 64, PARTS = PARTS_, XSTAGES = XSTAGES_, MINB = MINB_;
+  static constexpr int COLS = TILE / PARTS;                     // token columns per thread
+  static constexpr int OUT = D / PARTS;                         // accumulator columns per thread
+  static constexpr int SOFTMAX_WARPS = 4 * PARTS, THREADS = 64 + 32 * SOFTMAX_WARPS;
+  static constexpr uint32_t XSUB = 64 * 128;                    // [64 tokens x 64 features]
+  static constexpr uint32_t X_STAGE = (D / 64) * XSUB;
+  static constexpr uint32_t QSUB = 128 * 128;                   // [128 rows x 64 features]
+  static constexpr uint32_t Q_BUF = (D / 64) * QSUB;
+  static constexpr int PBUFS = 2;
+  static constexpr uint32_t P_BUF = 128 * 128;                  // [128 rows x 64 tokens]
+  static constexpr uint32_t OFF_X = 0;
+  static constexpr uint32_t OFF_Q2 = XSTAGES * X_STAGE;
+  static constexpr uint32_t OFF_P = OFF_Q2 + Q_BUF;
+  static constexpr uint32_t OFF_EXCH = OFF_P + PBUFS * P_BUF;   // [2 tile parities][PARTS][128] maxima, [PARTS][128] sums
+  static constexpr uint32_t OFF_BAR = OFF_EXCH + 3 * PARTS * 128 * 4;
+  static constexpr int IDX_CAP = 1025;                          // users + 1 whose offsets are staged in shared memory
+  static constexpr uint32_t OFF_IDX = OFF_BAR + 256;
+  static constexpr uint32_t SMEM = OFF_IDX + 2 * IDX_CAP * 4 + 8 + 1024;     // + slack to align the base to 1024 bytes
+  static constexpr uint32_t TMEM_COLS = D > 128 ? 512 : 256;    // scores: 2 x 64 columns; accumulator: D columns
+  static_assert(OUT % 32 == 0 && (COLS == 16 || COLS == 32), "column split of a row");
+  static_assert(MINB * (SMEM + 1024) <= 232448, "shared memory budget of the CTAs on one SM");
+  static_assert(MINB * TMEM_COLS <= 512, "TMEM budget of the CTAs on one SM");
+};
 constexpr float LB_RESCALE_THRESHOLD = 8.0f;                  // in log2 units
 
-struct LinkAttn256Params {
+struct LinkAttn64Params {
   const int32_t* off;
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
   const int32_t* chunk_user;      // [chunk items] user of each (user, chunk) item
@@ -78,13 +88,13 @@ __device__ __forceinline__ bool lb_group_sync(uint64_t* bar, uint32_t& uses, int
   return ok;
 }
 
-// p = 2^(s - m_ref) (or SiLU(s)) for this thread's 16 token columns, as bf16 into the A-operand buffer (K-major over
+// p = 2^(s - m_ref) (or SiLU(s)) for this thread's COLS token columns, as bf16 into the A-operand buffer (K-major over
 // the tile's tokens, 128-byte swizzle: one K-block of 64 tokens); columns at or past nvalid give 0.  Returns the sum.
-template <bool SILU>
-__device__ __forceinline__ float lb_probabilities(const float (&v)[LB_COLS], float m_ref, int col0, int nvalid, uint8_t* pbuf, uint32_t r) {
+template <bool SILU, int COLS>
+__device__ __forceinline__ float lb_probabilities(const float (&v)[COLS], float m_ref, int col0, int nvalid, uint8_t* pbuf, uint32_t r) {
   float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
-  for (int c8 = 0; c8 < LB_COLS / 8; ++c8) {
+  for (int c8 = 0; c8 < COLS / 8; ++c8) {
     uint32_t packed[4];
 #pragma unroll
     for (int j2 = 0; j2 < 4; ++j2) {
@@ -117,19 +127,18 @@ struct LbItemWalk {
   __device__ __forceinline__ void advance() { ci += stride; b0 = b1; b1 = b2; }
 };
 
-__global__ void __launch_bounds__(LB_THREADS, 1)
-k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttn256Params p) {
+template <class G>
+__global__ void __launch_bounds__(G::THREADS, G::MINB)
+k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttn64Params p) {
   using namespace tc;
+  constexpr int D = G::D, TILE = G::TILE, PARTS = G::PARTS, COLS = G::COLS, OUT = G::OUT, XSTAGES = G::XSTAGES, PBUFS = G::PBUFS;
   const int n_items = p.chunk_start[p.B] * p.RB;          // work items: (user, chunk) x row block; gridDim % RB == 0, so
   if ((int)blockIdx.x >= n_items) return;                  // a CTA keeps one row block for its whole life
-  extern __shared__ __align__(1024) uint8_t smem[];
-  if ((smem_u32(smem) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicCAS(p.err, 0, 95);
-    return;
-  }
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + LB_OFF_BAR);
-  uint64_t* x_full = bars;             // [LB_XSTAGES]
-  uint64_t* x_empty = bars + 4;        // [LB_XSTAGES]  second MMA of the tile done
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G::OFF_BAR);
+  uint64_t* x_full = bars;             // [XSTAGES]
+  uint64_t* x_empty = bars + 4;        // [XSTAGES]  second MMA of the tile done
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
   uint64_t* p_ready = bars + 10;       // [2]  per tile and P buffer: P in smem (all softmax warps)
   uint64_t* p_free = bars + 12;        // [2]  per tile and P buffer: second MMA done reading P (and accumulator up to date)
@@ -142,29 +151,29 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < LB_XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
+    for (int s = 0; s < XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
-    mbar_init(&p_ready[0], LB_SOFTMAX_WARPS); mbar_init(&p_ready[1], LB_SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
-    mbar_init(o_free, LB_SOFTMAX_WARPS);
-    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], LB_PARTS);
+    mbar_init(&p_ready[0], G::SOFTMAX_WARPS); mbar_init(&p_ready[1], G::SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
+    mbar_init(o_free, G::SOFTMAX_WARPS);
+    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], PARTS);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, G::TMEM_COLS); tmem_relinquish(); }
   const int32_t* chunk_start = p.chunk_start;
   const int32_t* off = p.off;
-  if (p.B + 1 <= LB_IDX_CAP) {
-    int32_t* idx = reinterpret_cast<int32_t*>(smem + LB_OFF_IDX);
-    for (int i = threadIdx.x; i <= p.B; i += LB_THREADS) { idx[i] = p.chunk_start[i]; idx[LB_IDX_CAP + i] = p.off[i]; }
+  if (p.B + 1 <= G::IDX_CAP) {
+    int32_t* idx = reinterpret_cast<int32_t*>(smem + G::OFF_IDX);
+    for (int i = threadIdx.x; i <= p.B; i += G::THREADS) { idx[i] = p.chunk_start[i]; idx[G::IDX_CAP + i] = p.off[i]; }
     chunk_start = idx;
-    off = idx + LB_IDX_CAP;
+    off = idx + G::IDX_CAP;
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_S = 0, COL_O = 128;      // scores: 2 x 64 columns; accumulator: d columns
+  constexpr uint32_t COL_S = 0, COL_O = 128;      // scores: 2 x 64 columns; accumulator: D columns
 
   const int rb = (int)blockIdx.x % p.RB;
   const int ci_first = (int)blockIdx.x / p.RB, ci_step = (int)gridDim.x / p.RB, n_ci = n_items / p.RB;
@@ -189,42 +198,42 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         prev_user = b;
         if (load_q) {
           if (!mbar_wait(q_empty, ((uint32_t)qn & 1u) ^ 1u, p.err, 42)) { ok = false; break; }
-          mbar_arrive_expect_tx(q_full, LB_Q_BUF);
-          for (int kb = 0; kb < LB_D / 64; ++kb)
-            tma_load_2d_hint(smem + LB_OFF_Q2 + kb * LB_QSUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128, q_full, pol_keep);
+          mbar_arrive_expect_tx(q_full, G::Q_BUF);
+          for (int kb = 0; kb < D / 64; ++kb)
+            tma_load_2d_hint(smem + G::OFF_Q2 + kb * G::QSUB, &tmQ2, kb * 64, (p.shared ? 0 : b) * p.HL + rb * 128, q_full, pol_keep);
           ++qn;
         }
-        const int n_tiles = (tok1 - tok0 + LB_TILE - 1) / LB_TILE;
+        const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
         for (int t = 0; t < n_tiles; ++t, ++g) {
-          const int s = g % LB_XSTAGES;
-          if (!mbar_wait(&x_empty[s], ((uint32_t)(g / LB_XSTAGES) & 1u) ^ 1u, p.err, 41)) { ok = false; break; }
-          mbar_arrive_expect_tx(&x_full[s], LB_X_STAGE);
-          for (int kb = 0; kb < LB_D / 64; ++kb)
-            tma_load_2d_hint(smem + LB_OFF_X + s * LB_X_STAGE + kb * LB_XSUB, &tmX, kb * 64, tok0 + t * LB_TILE, &x_full[s], pol_stream);
+          const int s = g % XSTAGES;
+          if (!mbar_wait(&x_empty[s], ((uint32_t)(g / XSTAGES) & 1u) ^ 1u, p.err, 41)) { ok = false; break; }
+          mbar_arrive_expect_tx(&x_full[s], G::X_STAGE);
+          for (int kb = 0; kb < D / 64; ++kb)
+            tma_load_2d_hint(smem + G::OFF_X + s * G::X_STAGE + kb * G::XSUB, &tmX, kb * 64, tok0 + t * TILE, &x_full[s], pol_stream);
         }
       }
       if (!ok || *(volatile int*)p.err != 0) {
         // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
-        for (int j = 0; j < g && j < LB_XSTAGES; ++j)
-          mbar_wait_quiet(&x_full[(g - 1 - j) % LB_XSTAGES], (uint32_t)((g - 1 - j) / LB_XSTAGES) & 1u);
+        for (int j = 0; j < g && j < XSTAGES; ++j)
+          mbar_wait_quiet(&x_full[(g - 1 - j) % XSTAGES], (uint32_t)((g - 1 - j) / XSTAGES) & 1u);
         if (qn > 0) mbar_wait_quiet(q_full, (uint32_t)(qn - 1) & 1u);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(128, LB_TILE);                 // Q2 . X^T  : both K-major
-      constexpr uint32_t idesc_o = make_idesc_bf16(128, LB_D, false, true);      // P . X     : B is MN-major
+      constexpr uint32_t idesc_s = make_idesc_bf16(128, TILE);               // Q2 . X^T  : both K-major
+      constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);     // P . X     : B is MN-major
       const uint32_t sbase = smem_u32(smem);
       auto issue_scores = [&](int g) -> bool {
-        const int s = g % LB_XSTAGES;
-        if (!mbar_wait(&x_full[s], (uint32_t)(g / LB_XSTAGES) & 1u, p.err, 51)) return false;
+        const int s = g % XSTAGES;
+        if (!mbar_wait(&x_full[s], (uint32_t)(g / XSTAGES) & 1u, p.err, 51)) return false;
         tc_fence_after();
-        for (int kk = 0; kk < LB_D / 16; ++kk) {
-          const uint32_t oa = (uint32_t)(kk >> 2) * LB_QSUB + (uint32_t)(kk & 3) * 32;
-          const uint32_t ob = (uint32_t)(kk >> 2) * LB_XSUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * LB_TILE, make_sdesc_k_sw128(sbase + LB_OFF_Q2 + oa),
-                      make_sdesc_k_sw128(sbase + LB_OFF_X + s * LB_X_STAGE + ob), idesc_s, kk != 0);
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t oa = (uint32_t)(kk >> 2) * G::QSUB + (uint32_t)(kk & 3) * 32;
+          const uint32_t ob = (uint32_t)(kk >> 2) * G::XSUB + (uint32_t)(kk & 3) * 32;
+          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * TILE, make_sdesc_k_sw128(sbase + G::OFF_Q2 + oa),
+                      make_sdesc_k_sw128(sbase + G::OFF_X + s * G::X_STAGE + ob), idesc_s, kk != 0);
         }
         mma_commit(&s_full[g & 1]);
         return true;
@@ -245,7 +254,7 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
         // will the producer replace the queries after this item?
         const bool next_reloads = !p.shared && w.b1 >= 0 && w.b1 != b;
-        const int n_tiles = (tok1 - tok0 + LB_TILE - 1) / LB_TILE;
+        const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
         if (!issue_scores(g)) { ok = false; break; }
         if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
         for (int t = 0; t < n_tiles; ++t, ++g) {
@@ -254,31 +263,31 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
             if (!issue_scores(g + 1)) { ok = false; break; }
             if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
           }
-          const int s = g % LB_XSTAGES;
-          if (!mbar_wait(&p_ready[g % LB_PBUFS], (uint32_t)(g / LB_PBUFS) & 1u, p.err, 52)) { ok = false; break; }
+          const int s = g % XSTAGES;
+          if (!mbar_wait(&p_ready[g % PBUFS], (uint32_t)(g / PBUFS) & 1u, p.err, 52)) { ok = false; break; }
           // the first tile of an item overwrites the accumulator: the previous item must have been read out
           if (t == 0 && k > 0 && !mbar_wait(o_free, (uint32_t)(k - 1) & 1u, p.err, 53)) { ok = false; break; }
           tc_fence_after();
-          for (int kk = 0; kk < LB_TILE / 16; ++kk)      // contraction over the tile's 64 tokens, 16 per instruction
-            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + LB_OFF_P + (uint32_t)(g % LB_PBUFS) * LB_P_BUF + (uint32_t)kk * 32),
-                        make_sdesc_mn_sw128(sbase + LB_OFF_X + s * LB_X_STAGE + (uint32_t)kk * 2048, LB_XSUB), idesc_o, (t | kk) != 0);
+          for (int kk = 0; kk < TILE / 16; ++kk)      // contraction over the tile's 64 tokens, 16 per instruction
+            mma_bf16_ss(tmem_base + COL_O, make_sdesc_k_sw128(sbase + G::OFF_P + (uint32_t)(g % PBUFS) * G::P_BUF + (uint32_t)kk * 32),
+                        make_sdesc_mn_sw128(sbase + G::OFF_X + s * G::X_STAGE + (uint32_t)kk * 2048, G::XSUB), idesc_o, (t | kk) != 0);
           mma_commit(&x_empty[s]);
-          mma_commit(&p_free[g % LB_PBUFS]);
+          mma_commit(&p_free[g % PBUFS]);
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax warps (2..17)
-    const int sw = warp - 2;                                   // 0..15
+    // ------------------------------------------------------------------ softmax warps
+    const int sw = warp - 2;
     const int q = warp & 3;                                    // TMEM lane quarter of this warp
-    const int part = sw >> 2;                                  // which 16 token columns of the tile / 64 accumulator columns
-    const int col0 = part * LB_COLS;
+    const int part = sw >> 2;                                  // which COLS token columns of the tile / OUT accumulator columns
+    const int col0 = part * COLS;
     const uint32_t r = (uint32_t)(q * 32 + lane);              // (head, link) row == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    float* exch_max = reinterpret_cast<float*>(smem + LB_OFF_EXCH);          // [2 tile parities][PARTS][128]
-    float* exch_sum = exch_max + 2 * LB_PARTS * 128;                         // [PARTS][128]
+    float* exch_max = reinterpret_cast<float*>(smem + G::OFF_EXCH);          // [2 tile parities][PARTS][128]
+    float* exch_sum = exch_max + 2 * PARTS * 128;                            // [PARTS][128]
     const int R = rb * 128 + (int)r;                            // row among all H * ell
-    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * LB_D) + (R / p.ell) * LB_D + part * LB_OUT;
+    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * D) + (R / p.ell) * D + part * OUT;
     bool ok = true;
     int g = 0, k = 0;
     uint32_t row_uses = 0;
@@ -288,35 +297,36 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
       const int b = w.b0;
       int tok0, tok1;
       item_range(w.ci, b, tok0, tok1);
-      const int n_tiles = (tok1 - tok0 + LB_TILE - 1) / LB_TILE;
+      const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
       float m_ref = -INFINITY, l_sum = 0.f;
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         const int pb = g & 1;
-        const int nvalid = min(LB_TILE, tok1 - tok0 - t * LB_TILE);
+        const int nvalid = min(TILE, tok1 - tok0 - t * TILE);
         if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
         tc_fence_after();
-        float v[LB_COLS];
-        tmem_ld_32x16(lane_addr + COL_S + pb * LB_TILE + col0, v);
+        float v[COLS];
+        if constexpr (COLS == 16) tmem_ld_32x16(lane_addr + COL_S + pb * TILE + col0, v);
+        else tmem_ld_32x32(lane_addr + COL_S + pb * TILE + col0, v);
         tmem_wait_ld();
-        uint8_t* pbuf = smem + LB_OFF_P + (g % LB_PBUFS) * LB_P_BUF;
+        uint8_t* pbuf = smem + G::OFF_P + (g % PBUFS) * G::P_BUF;
         if (p.silu) {
           // SiLU(s) / N(U) needs neither a reference maximum nor row sums: one pass, no exchange between the row's threads
-          if (g >= LB_PBUFS && !mbar_wait(&p_free[g % LB_PBUFS], (uint32_t)((g - LB_PBUFS) / LB_PBUFS) & 1u, p.err, 65)) { ok = false; break; }
-          lb_probabilities<true>(v, 0.f, col0, nvalid, pbuf, r);
+          if (g >= PBUFS && !mbar_wait(&p_free[g % PBUFS], (uint32_t)((g - PBUFS) / PBUFS) & 1u, p.err, 65)) { ok = false; break; }
+          lb_probabilities<true, COLS>(v, 0.f, col0, nvalid, pbuf, r);
           tc_fence_before();
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&p_ready[g % LB_PBUFS]);
+          if (lane == 0) mbar_arrive(&p_ready[g % PBUFS]);
           continue;
         }
         float mx = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < LB_COLS; ++j)
+        for (int j = 0; j < COLS; ++j)
           if (col0 + j < nvalid) mx = fmaxf(mx, v[j]);
-        exch_max[(pb * LB_PARTS + part) * 128 + r] = mx;
+        exch_max[(pb * PARTS + part) * 128 + r] = mx;
         if (!lb_group_sync(&row_bar[q], row_uses, lane, p.err, 67)) { ok = false; break; }
 #pragma unroll
-        for (int i = 1; i < LB_PARTS; ++i) mx = fmaxf(mx, exch_max[(pb * LB_PARTS + ((part + i) & (LB_PARTS - 1))) * 128 + r]);
+        for (int i = 1; i < PARTS; ++i) mx = fmaxf(mx, exch_max[(pb * PARTS + ((part + i) & (PARTS - 1))) * 128 + r]);
 
         // raise the reference maximum only when it is exceeded by more than the threshold (or unset)
         const bool need = mx > m_ref + LB_RESCALE_THRESHOLD;
@@ -324,16 +334,16 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         const float factor = (need && m_ref != -INFINITY) ? lb_ex2(m_ref - m_new) : 1.0f;
         if (__any_sync(0xffffffffu, need && t > 0)) {
           // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this part of the row
-          if (!mbar_wait(&p_free[(g - 1) % LB_PBUFS], (uint32_t)((g - 1) / LB_PBUFS) & 1u, p.err, 64)) { ok = false; break; }
+          if (!mbar_wait(&p_free[(g - 1) % PBUFS], (uint32_t)((g - 1) / PBUFS) & 1u, p.err, 64)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
-          for (int c = 0; c < LB_OUT; c += 32) {
+          for (int c = 0; c < OUT; c += 32) {
             float a[32];
-            tmem_ld_32x32(lane_addr + COL_O + part * LB_OUT + c, a);
+            tmem_ld_32x32(lane_addr + COL_O + part * OUT + c, a);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 32; ++j) a[j] *= factor;
-            tmem_st_32x32(lane_addr + COL_O + part * LB_OUT + c, a);
+            tmem_st_32x32(lane_addr + COL_O + part * OUT + c, a);
           }
           tmem_wait_st();
         }
@@ -341,33 +351,33 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         m_ref = m_new;
 
         // the P that last sat in this buffer must have been consumed
-        if (g >= LB_PBUFS && !mbar_wait(&p_free[g % LB_PBUFS], (uint32_t)((g - LB_PBUFS) / LB_PBUFS) & 1u, p.err, 65)) { ok = false; break; }
-        l_sum += lb_probabilities<false>(v, m_ref, col0, nvalid, pbuf, r);
+        if (g >= PBUFS && !mbar_wait(&p_free[g % PBUFS], (uint32_t)((g - PBUFS) / PBUFS) & 1u, p.err, 65)) { ok = false; break; }
+        l_sum += lb_probabilities<false, COLS>(v, m_ref, col0, nvalid, pbuf, r);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_ready[g % LB_PBUFS]);
+        if (lane == 0) mbar_arrive(&p_ready[g % PBUFS]);
       }
       if (!ok) break;
       // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
       const int gl = g - 1;
-      if (!mbar_wait(&p_free[gl % LB_PBUFS], (uint32_t)(gl / LB_PBUFS) & 1u, p.err, 66)) { ok = false; break; }
+      if (!mbar_wait(&p_free[gl % PBUFS], (uint32_t)(gl / PBUFS) & 1u, p.err, 66)) { ok = false; break; }
       tc_fence_after();
       exch_sum[part * 128 + r] = l_sum;
       if (!lb_group_sync(&row_bar[q], row_uses, lane, p.err, 68)) { ok = false; break; }
       float l_tot = 0.f;
 #pragma unroll
-      for (int i = 0; i < LB_PARTS; ++i) l_tot += exch_sum[i * 128 + r];
+      for (int i = 0; i < PARTS; ++i) l_tot += exch_sum[i * 128 + r];
       // SiLU mode normalises by the number of keys (Algorithm 1): this chunk's tokens, summed over the chunks by the merge
       if (p.silu) l_tot = (float)(tok1 - tok0);
       const bool single = chunk_start[b + 1] - chunk_start[b] == 1;
       const float inv = 1.0f / l_tot;
-      __nv_bfloat16* dst_o = p.Ohat + (int64_t)b * p.ell * (p.H * LB_D) + ohat_off;
-      float* dst_p = p.part_acc + ((int64_t)w.ci * p.HL + R) * LB_D + part * LB_OUT;
+      __nv_bfloat16* dst_o = p.Ohat + (int64_t)b * p.ell * (p.H * D) + ohat_off;
+      float* dst_p = p.part_acc + ((int64_t)w.ci * p.HL + R) * D + part * OUT;
 #pragma unroll
-      for (int c = 0; c < LB_OUT; c += 32) {
+      for (int c = 0; c < OUT; c += 32) {
         float a[32];
-        tmem_ld_32x32(lane_addr + COL_O + part * LB_OUT + c, a);
+        tmem_ld_32x32(lane_addr + COL_O + part * OUT + c, a);
         tmem_wait_ld();
         if (single) {
           // the whole history of this user was one chunk: normalise and write the attention row directly
@@ -398,36 +408,44 @@ k_link_attn_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_consta
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, G::TMEM_COLS);
   }
 }
 
+using LbD256 = LbCfg<256, 4, 3, 1>;       // d = 256: four threads per stacked row, three token stages, one CTA per SM
+
 bool link_attn_d256_tc_supported(int dtype, int d, int H, int ell, int phi) {
-  return dtype == LIME_BF16 && d == LB_D && (H * ell) % 128 == 0 && H * ell <= 512 && ell % 4 == 0 &&
+  return dtype == LIME_BF16 && d == 256 && (H * ell) % 128 == 0 && H * ell <= 512 && ell % 4 == 0 &&
          (phi == LIME_PHI_SOFTMAX || phi == LIME_PHI_SILU);
 }
 
-lime_status launch_link_attn_d256_tc(const LinkAttnArgs& a, cudaStream_t st) {
+template <class G>
+static lime_status launch_link_attn_t64(const LinkAttnArgs& a, cudaStream_t st, const char* name, bool (&smem_set)[kMaxDeviceOrdinals]) {
   if (a.n_chunk_upper <= 0 || a.total == 0) return LIME_OK;   // no history: the merge step writes zeros
   if (a.ln) return LIME_INVALID_ARG;                           // rows must arrive LayerNorm-ed
   CUtensorMap tmX, tmQ2;
   const uint64_t users = a.shared ? 1 : (uint64_t)a.B;
-  if (!make_tmap_bf16_sw128(&tmX, a.hist, (uint64_t)a.total, LB_D, LB_D, LB_TILE) ||
-      !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), LB_D, LB_D, 128))
+  if (!make_tmap_bf16_sw128(&tmX, a.hist, (uint64_t)a.total, G::D, G::D, G::TILE) ||
+      !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), G::D, G::D, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
-  LinkAttn256Params p;
+  LinkAttn64Params p;
   p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.silu = a.silu; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
-  int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;
+  const int slots = kSMs * G::MINB;
+  int grid = a.n_chunk_upper * p.RB < slots ? a.n_chunk_upper * p.RB : slots;
   grid -= grid % p.RB;                              // a CTA's work items then all share its row block
-  static bool smem_set[kMaxDeviceOrdinals] = {};
-  lime_status es = ensure_dynamic_smem((const void*)k_link_attn_d256_tc, (int)LB_SMEM, smem_set);
+  lime_status es = ensure_dynamic_smem((const void*)k_link_attn_t64_tc<G>, (int)G::SMEM, smem_set);
   if (es != LIME_OK) return es;
-  ProfScope _p("k_link_attn_d256_tc", st);
-  k_link_attn_d256_tc<<<grid, LB_THREADS, LB_SMEM, st>>>(tmX, tmQ2, p);
-  LIME_LAUNCH_CHECK("k_link_attn_d256_tc");
+  ProfScope _p(name, st);
+  k_link_attn_t64_tc<G><<<grid, G::THREADS, G::SMEM, st>>>(tmX, tmQ2, p);
+  LIME_LAUNCH_CHECK(name);
   return LIME_OK;
+}
+
+lime_status launch_link_attn_d256_tc(const LinkAttnArgs& a, cudaStream_t st) {
+  static bool smem_set[kMaxDeviceOrdinals] = {};
+  return launch_link_attn_t64<LbD256>(a, st, "k_link_attn_d256_tc", smem_set);
 }
 
 }  // namespace lime

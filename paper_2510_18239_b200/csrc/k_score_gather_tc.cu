@@ -15,6 +15,8 @@
 //   warps 0-3 : producers  - 32 x (d/64 + 1) gather copies per tile spread over the threads; thread 0 also fetches the user's link states when the stage held another user's
 //   warp  4   : MMA issuer
 //   warps 5-8 : epilogue   - thread r owns candidate row r (TMEM lane r)
+// With packed corpus records ([embedding row | weight row] per item, row pitch d + ell: lime_pack_corpus_cache) the
+// same copies run over two views of the one array, and a candidate's embedding and weights come from one place in DRAM.
 // An id outside [0, V) fetches row 0 instead (the copies of a stage keep their fixed byte count and never leave the
 // caches); the epilogue thread of that slot writes logit 0 and lowers the caller's flag to the slot index.
 #include "lime_common.cuh"
@@ -274,8 +276,8 @@ static lime_status launch_score_gather_t(const ScoreArgs& a, int* err, cudaStrea
   const int S = score_gather_stages(ELL, a.d, &smem);
   CUtensorMap tmLS, tmT, tmW;
   if (!make_tmap_bf16_sw128(&tmLS, a.LS, (uint64_t)a.B * ELL, (uint64_t)a.d, (uint64_t)a.d, ELL) ||
-      !make_tmap_bf16_sw128(&tmT, a.T, (uint64_t)a.corpus_rows, (uint64_t)a.d, (uint64_t)a.d, 1) ||
-      !make_tmap_bf16_plain(&tmW, a.W, (uint64_t)a.corpus_rows, ELL, ELL, 1))
+      !make_tmap_bf16_sw128(&tmT, a.T, (uint64_t)a.corpus_rows, (uint64_t)a.d, (uint64_t)(a.ldt ? a.ldt : a.d), 1) ||
+      !make_tmap_bf16_plain(&tmW, a.W, (uint64_t)a.corpus_rows, ELL, (uint64_t)(a.ldw ? a.ldw : ELL), 1))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   ScoreGatherParams p;
   p.ids = a.cand_ids; p.logits = a.logits; p.V = (int32_t)a.corpus_rows; p.flag = a.dev_flag;

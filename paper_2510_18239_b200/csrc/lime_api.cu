@@ -788,6 +788,35 @@ lime_status lime_score_candidates_head(lime_ctx* ctx, const void* link_states, i
   return launch_score_head_simt(a, LSW, W0t, f.b[0], w0, ffn_tail(f, 1), st);
 }
 
+lime_status lime_pack_corpus_cache(lime_ctx* ctx, const void* cand_emb, const void* cand_w, int64_t corpus_rows, void* packed,
+                                   void* stream) {
+  if (!ctx || corpus_rows < 0 || corpus_rows > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (corpus_rows == 0) return LIME_OK;
+  if (!cand_emb || !cand_w || !packed || !aligned16(cand_emb) || !aligned16(cand_w) || !aligned16(packed)) return LIME_INVALID_ARG;
+  const Ctx* c = reinterpret_cast<const Ctx*>(ctx);
+  return launch_pack_corpus(c->cfg.dtype, cand_emb, cand_w, corpus_rows, c->cfg.d, c->ell_c, packed, static_cast<cudaStream_t>(stream));
+}
+
+lime_status lime_score_candidates_packed(lime_ctx* ctx, const void* link_states, int32_t B, const void* packed,
+                                         int64_t corpus_rows, const int32_t* cand_ids, const int32_t* cand_off, int32_t C,
+                                         int64_t total_cands, int32_t* dev_flag, float* logits, void* stream) {
+  if (!ctx || B < 0 || C < 0 || total_cands < 0 || total_cands > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (corpus_rows <= 0 || corpus_rows > 0x7fffffffLL) return LIME_INVALID_ARG;
+  if (!cand_off && total_cands != (int64_t)B * C) return LIME_INVALID_ARG;
+  if (B == 0 || total_cands == 0) return LIME_OK;
+  if (!link_states || !packed || !cand_ids || !logits || !aligned16(link_states) || !aligned16(packed)) return LIME_INVALID_ARG;
+  Ctx* c = reinterpret_cast<Ctx*>(ctx);
+  const int es = elem_size(c->cfg.dtype);
+  ScoreArgs a{};
+  a.LS = link_states; a.T = packed; a.W = static_cast<const char*>(packed) + (size_t)c->cfg.d * es;
+  a.ldt = a.ldw = c->cfg.d + c->ell_c;
+  a.dtype = c->cfg.dtype; a.B = B; a.ell = c->ell_c; a.d = c->cfg.d;
+  a.cand_off = cand_off; a.C = C; a.total = total_cands; a.cand_ids = cand_ids; a.logits = logits;
+  a.corpus_rows = corpus_rows; a.dev_flag = dev_flag;
+  if (score_gather_tc_supported(a)) return launch_score_gather_tc(a, c->dev_err, static_cast<cudaStream_t>(stream));
+  return launch_score_simt(a, static_cast<cudaStream_t>(stream));
+}
+
 lime_status lime_selftest_wait_expiry(lime_ctx* ctx, int32_t limit_us, void* stream) {
   if (!ctx || limit_us < 1 || limit_us > 1000000) return LIME_INVALID_ARG;
   Ctx* c = reinterpret_cast<Ctx*>(ctx);

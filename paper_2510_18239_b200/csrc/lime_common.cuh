@@ -183,7 +183,10 @@ struct ScoreArgs {
   int64_t corpus_rows;
   int32_t* dev_flag;            // nullable: lowered to the smallest slot whose id was out of range
   float* logits;
+  int64_t ldw, ldt;             // row pitch of W and T in elements; 0 = dense (ell, d).  Packed corpus records: d + ell both
 };
+// out[v, :] = [ emb[v, 0..d) | w[v, 0..ell) ]: one record per item of the corpus caches (k_cand_simt.cu)
+lime_status launch_pack_corpus(int dtype, const void* emb, const void* w, int64_t V, int d, int ell, void* out, cudaStream_t st);
 lime_status launch_score_simt(const ScoreArgs& a, cudaStream_t st);
 // bf16 streaming scorer on tcgen05 tensor cores (fixed C per user, dense rows, ell in {16,32,64,128}, d % 64 == 0)
 bool score_tc_supported(const ScoreArgs& a);

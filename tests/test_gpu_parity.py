@@ -236,6 +236,49 @@ def test_score_from_corpus_caches_by_ids(B, C, ell, d, corpus):
     assert err <= 1e-4 * max(1.0, np.abs(want).max()), err
 
 
+@pytest.mark.parametrize("dtype,B,C,ell,d,corpus,ragged", [(synth.BF16, 3, 2048, 32, 128, 5000, False), (synth.BF16, 2, 129, 64, 256, 300, False),
+                                                           (synth.BF16, 150, 1000, 32, 128, 100000, False), (synth.BF16, 5, 300, 128, 64, 999, False),
+                                                           (synth.BF16, 4, 50, 33, 40, 257, False), (synth.F32, 3, 70, 8, 64, 257, False),
+                                                           (synth.BF16, 3, 0, 16, 64, 257, True)])
+def test_score_from_packed_corpus_records(dtype, B, C, ell, d, corpus, ragged):
+    """Corpus caches packed as one record per item ([embedding row | weight row], Sec. 3.3): the records are the two
+    caches bit for bit, and scoring by id over them gives the oracle's logits (tensor-core scorer with its own gather
+    over two views of the one array; generic scorer for the other shapes); ids outside the corpus score 0."""
+    Bd = _lib()
+    dt = Bd.LIME_F32 if dtype == synth.F32 else Bd.LIME_BF16
+    lime = Bd.Lime(d, max(1, d // 128), ell, 1, dtype=dt, gated_mlp=False)
+    if ragged:
+        counts = np.array([40, 0, 91], dtype=np.int64)
+        off = O.lengths_to_offsets(counts)
+        total = int(counts.sum())
+    else:
+        off = np.arange(B + 1, dtype=np.int64) * C
+        total = B * C
+    LS = synth.normal_storage(41, "ls", (B, ell, d), 1.0, dtype)
+    Tc = synth.normal_storage(41, "t", (corpus, d), 1.0, dtype)
+    Wc = synth.to_storage(O.softmax_rows(np.random.default_rng(41).normal(size=(corpus, ell))), dtype)
+    ids = synth.uniform_ids(41, "ids", total, corpus)
+    bad = {3: -1, total - 1: corpus} if total > 8 else {}
+    for slot, v in bad.items():
+        ids[slot] = v
+    packed = lime.pack_corpus_cache(Bd.to_device(Tc, dtype), Bd.to_device(Wc, dtype))
+    raw = packed.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == synth.BF16 else packed.cpu().numpy()
+    assert np.array_equal(raw[:, :d], Tc) and np.array_equal(raw[:, d:], Wc)
+    flag = torch.full((1,), 2 ** 31 - 1, dtype=torch.int32, device="cuda")
+    logits = lime.score_candidates_packed(Bd.to_device(LS, dtype), packed, torch.from_numpy(ids).cuda(), C=C,
+                                          cand_off=torch.from_numpy(off.astype(np.int32)).cuda() if ragged else None, dev_flag=flag)
+    assert Bd.lime_device_status(lime.ctx) == 0
+    got = Hh.to_f64(logits)
+    W64, T64, LS64 = (synth.storage_to_f64(x, dtype) for x in (Wc, Tc, LS))
+    ok_ids = np.clip(ids, 0, corpus - 1)
+    want = np.concatenate([O.score_candidates(W64[ok_ids[off[b]:off[b + 1]]], LS64[b], T64[ok_ids[off[b]:off[b + 1]]])
+                           for b in range(B)])
+    want[list(bad)] = 0.0
+    assert np.abs(got - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+    assert np.all(got[list(bad)] == 0.0)
+    assert int(flag.item()) == (min(bad) if bad else 2 ** 31 - 1)
+
+
 @pytest.mark.parametrize("dtype,B,C,ell,d,ragged", [(synth.BF16, 3, 300, 32, 128, False),     # tensor-core scorer with its own gather
                                                     (synth.BF16, 2, 129, 64, 256, False),
                                                     (synth.BF16, 4, 50, 33, 40, False),       # generic scorer, fixed C
