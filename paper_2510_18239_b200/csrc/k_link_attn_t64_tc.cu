@@ -1,4 +1,5 @@
-// Links attend over the history on the 5th-generation tensor cores, 64-token tiles (bf16 storage, rows LayerNorm-ed already):
+// Links attend over the history on the 5th-generation tensor cores at d = 256, 64-token tiles (bf16 storage, rows
+// LayerNorm-ed already):
 //
 //   O[T]_h = phi( Q[T]_h K[S]_h^T * scale ) V[S]_h,  K[S] = X W_K,  V[S] = X W_V,  X = LN(S)                (Eq. 3 / Eq. 7)
 //
@@ -7,48 +8,57 @@
 // once by TMA and used as keys and as values:
 //   scores [128 x 64]   = Q2_block [128 x d] . X_tile^T          (one block of 128 stacked (head, link) rows per work item)
 //   acc    [128 x d]   += P [128 x 64] . X_tile
-// The history is walked in tiles of 64 tokens, which halves every per-tile buffer against k_link_attn_tc.cu: at d = 256
-// the accumulator takes 256 TMEM columns and a block of folded queries 64 KB of shared memory, which only fits with the
-// small tile (32 KB per stage, three stages; two score buffers of 64 columns; two P buffers of 16 KB).  The geometry is a
-// template parameter (LbCfg).  A d = 128 build with two CTAs per SM (16 KB stages, two threads per row) was measured
-// and dropped: with only two token stages per CTA the tile period is bound by the latency of the copies (31 us per
-// launch on 256 users x 512 tokens against 25 us for k_link_attn_tc.cu).
-// The rows read must be LayerNorm-ed already (the lookup or the previous layer's history update stores them so); there is
-// no on-the-fly LayerNorm in this kernel.
-// Online softmax in the log2 domain with lazy rescale, or SiLU(s) / N(U) with `silu` (Algorithms 1-2), as in
-// k_link_attn_tc.cu.  Persistent CTAs walk (user, chunk) x row-block items; warp 0 TMA producer, warp 1 MMA issuer,
-// the other warps softmax: PARTS threads per stacked row, 64 / PARTS of the tile's token columns each, and d / PARTS of
-// the accumulator columns when a row is rescaled or read out.
+// At d = 256 the accumulator takes 256 TMEM columns and a block of folded queries 64 KB of shared memory, which only fits
+// with a 64-token tile (32 KB per stage, three stages; two score buffers of 64 columns; two P buffers of 16 KB).  The rows
+// read must be LayerNorm-ed already (the lookup or the previous layer's history update stores them so); there is no
+// on-the-fly LayerNorm in this kernel.  Online softmax in the log2 domain with lazy rescale, or SiLU(s) / N(U) with `silu`
+// (Algorithms 1-2).
+//
+// Persistent CTAs walk (user, chunk) x row-block items; warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 softmax.  What
+// a softmax warp does for a tile is a chain of waits (scores in TMEM -> TMEM load -> row maximum -> exponentials -> P in
+// shared memory -> fence -> signal) whose latency, not its arithmetic, sets the tile period, so the eight warps form TWO
+// GROUPS that take alternate tiles: while one group is in the middle of its chain the other starts the next tile's.  A
+// group is four warps, ONE thread per stacked row (the row's 64 scores of the tile in registers: no exchange between
+// threads for the maximum, and with 320 threads per CTA no register spills - with shared memory configured to its
+// maximum a spill is a round trip to L2), and owns the score buffer and the P buffer of its tile parity.  The running
+// reference maximum of a row is shared by both groups: the group that handles tile g publishes it (after its own decision
+// whether to raise it) and the other group picks it up for tile g + 1; each group keeps the partial row sums of its own
+// tiles, relative to the last reference it saw, and the two threads of a row combine them when the item ends.
+// A d = 128 build of this kernel with two CTAs per SM (16 KB stages, two threads per row) was measured and dropped: with
+// only two token stages per CTA the tile period is bound by the latency of the copies (31 us per launch on 256 users x
+// 512 tokens against 25 us for k_link_attn_tc.cu).
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
 
-// Geometry of one build: D features per row, PARTS threads per stacked row, XSTAGES token stages, MINB CTAs per SM.
-template <int D_, int PARTS_, int XSTAGES_, int MINB_>
+// Geometry: D features per row, XSTAGES token stages.
+template <int D_, int XSTAGES_>
 struct LbCfg {
-  static constexpr int D = D_, TILE = 64, PARTS = PARTS_, XSTAGES = XSTAGES_, MINB = MINB_;
-  static constexpr int COLS = TILE / PARTS;                     // token columns per thread
-  static constexpr int OUT = D / PARTS;                         // accumulator columns per thread
-  static constexpr int SOFTMAX_WARPS = 4 * PARTS, THREADS = 64 + 32 * SOFTMAX_WARPS;
+  static constexpr int D = D_, TILE = 64, XSTAGES = XSTAGES_;
+  static constexpr int GROUPS = 2;                              // softmax groups (alternate tiles), one thread per row in each
+  static constexpr int COLS = TILE;                             // token columns per thread: the whole row of the tile
+  static constexpr int OUT = D / GROUPS;                        // accumulator columns a thread reads out (the two threads of a row)
+  static constexpr int SOFTMAX_WARPS = 4 * GROUPS, GROUP_WARPS = 4, THREADS = 64 + 32 * SOFTMAX_WARPS;
   static constexpr uint32_t XSUB = 64 * 128;                    // [64 tokens x 64 features]
   static constexpr uint32_t X_STAGE = (D / 64) * XSUB;
   static constexpr uint32_t QSUB = 128 * 128;                   // [128 rows x 64 features]
   static constexpr uint32_t Q_BUF = (D / 64) * QSUB;
-  static constexpr int PBUFS = 2;
+  static constexpr int PBUFS = 2;                               // one per group
   static constexpr uint32_t P_BUF = 128 * 128;                  // [128 rows x 64 tokens]
   static constexpr uint32_t OFF_X = 0;
   static constexpr uint32_t OFF_Q2 = XSTAGES * X_STAGE;
   static constexpr uint32_t OFF_P = OFF_Q2 + Q_BUF;
-  static constexpr uint32_t OFF_EXCH = OFF_P + PBUFS * P_BUF;   // [2 tile parities][PARTS][128] maxima, [PARTS][128] sums
-  static constexpr uint32_t OFF_BAR = OFF_EXCH + 3 * PARTS * 128 * 4;
+  // exchange area (floats): published reference maxima [2 tile parities][128], row sums [GROUPS][128]
+  static constexpr uint32_t OFF_EXCH = OFF_P + PBUFS * P_BUF;
+  static constexpr uint32_t EXCH_FLOATS = (2 + GROUPS) * 128;
+  static constexpr uint32_t OFF_BAR = OFF_EXCH + EXCH_FLOATS * 4;
   static constexpr int IDX_CAP = 1025;                          // users + 1 whose offsets are staged in shared memory
   static constexpr uint32_t OFF_IDX = OFF_BAR + 256;
   static constexpr uint32_t SMEM = OFF_IDX + 2 * IDX_CAP * 4 + 8 + 1024;     // + slack to align the base to 1024 bytes
   static constexpr uint32_t TMEM_COLS = D > 128 ? 512 : 256;    // scores: 2 x 64 columns; accumulator: D columns
-  static_assert(OUT % 32 == 0 && (COLS == 16 || COLS == 32), "column split of a row");
-  static_assert(MINB * (SMEM + 1024) <= 232448, "shared memory budget of the CTAs on one SM");
-  static_assert(MINB * TMEM_COLS <= 512, "TMEM budget of the CTAs on one SM");
+  static_assert(OUT % 32 == 0 && COLS == 64, "column split of a row");
+  static_assert(SMEM + 1024 <= 232448, "shared memory budget of one CTA");
 };
 constexpr float LB_RESCALE_THRESHOLD = 8.0f;                  // in log2 units
 
@@ -128,10 +138,10 @@ struct LbItemWalk {
 };
 
 template <class G>
-__global__ void __launch_bounds__(G::THREADS, G::MINB)
+__global__ void __launch_bounds__(G::THREADS, 1)
 k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttn64Params p) {
   using namespace tc;
-  constexpr int D = G::D, TILE = G::TILE, PARTS = G::PARTS, COLS = G::COLS, OUT = G::OUT, XSTAGES = G::XSTAGES, PBUFS = G::PBUFS;
+  constexpr int D = G::D, TILE = G::TILE, COLS = G::COLS, OUT = G::OUT, XSTAGES = G::XSTAGES, PBUFS = G::PBUFS;
   const int n_items = p.chunk_start[p.B] * p.RB;          // work items: (user, chunk) x row block; gridDim % RB == 0, so
   if ((int)blockIdx.x >= n_items) return;                  // a CTA keeps one row block for its whole life
   extern __shared__ uint8_t smem_raw[];
@@ -140,13 +150,15 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   uint64_t* x_full = bars;             // [XSTAGES]
   uint64_t* x_empty = bars + 4;        // [XSTAGES]  second MMA of the tile done
   uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       // [2]  per tile and P buffer: P in smem (all softmax warps)
+  uint64_t* p_ready = bars + 10;       // [2]  per tile and P buffer: P in smem (the four warps of that buffer's group)
   uint64_t* p_free = bars + 12;        // [2]  per tile and P buffer: second MMA done reading P (and accumulator up to date)
   uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
-  uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the warps that share a TMEM lane quarter
+  uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the two warps that share a TMEM lane quarter (end of an item)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
   uint64_t* q_full = bars + 22;        //      folded queries of a user landed
   uint64_t* q_empty = bars + 23;       //      every score MMA that reads them has run
+  uint64_t* mref_bar = bars + 24;      // [2 tile parities][4 quarters]  reference maxima after the tile published (and the
+                                       //                                previous ones read) by the handling group's warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -154,9 +166,10 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     for (int s = 0; s < XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
     for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
-    mbar_init(&p_ready[0], G::SOFTMAX_WARPS); mbar_init(&p_ready[1], G::SOFTMAX_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
+    mbar_init(&p_ready[0], G::GROUP_WARPS); mbar_init(&p_ready[1], G::GROUP_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
     mbar_init(o_free, G::SOFTMAX_WARPS);
-    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], PARTS);
+    for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], G::GROUPS);
+    for (int i = 0; i < 8; ++i) mbar_init(&mref_bar[i], 1);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
@@ -277,17 +290,15 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       }
     }
   } else {
-    // ------------------------------------------------------------------ softmax warps
-    const int sw = warp - 2;
+    // ------------------------------------------------------------------ softmax warps (2..9), two groups of four
     const int q = warp & 3;                                    // TMEM lane quarter of this warp
-    const int part = sw >> 2;                                  // which COLS token columns of the tile / OUT accumulator columns
-    const int col0 = part * COLS;
-    const uint32_t r = (uint32_t)(q * 32 + lane);              // (head, link) row == TMEM lane
+    const int grp = (warp - 2) >> 2;                           // handles the tiles with g % 2 == grp
+    const uint32_t r = (uint32_t)(q * 32 + lane);              // (head, link) row == TMEM lane; the thread owns the whole row
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    float* exch_max = reinterpret_cast<float*>(smem + G::OFF_EXCH);          // [2 tile parities][PARTS][128]
-    float* exch_sum = exch_max + 2 * PARTS * 128;                            // [PARTS][128]
+    float* mref = reinterpret_cast<float*>(smem + G::OFF_EXCH);              // [2 tile parities][128]
+    float* exch_sum = mref + 2 * 128;                                        // [GROUPS][128]
     const int R = rb * 128 + (int)r;                            // row among all H * ell
-    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * D) + (R / p.ell) * D + part * OUT;
+    const int64_t ohat_off = (int64_t)(R % p.ell) * (p.H * D) + (R / p.ell) * D + grp * OUT;
     bool ok = true;
     int g = 0, k = 0;
     uint32_t row_uses = 0;
@@ -298,86 +309,105 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       int tok0, tok1;
       item_range(w.ci, b, tok0, tok1);
       const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
-      float m_ref = -INFINITY, l_sum = 0.f;
+      // m_own: the reference maximum this thread's row sum is relative to; l_sum: sum over the tiles of this group
+      float m_own = -INFINITY, l_sum = 0.f;
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
-        const int pb = g & 1;
+        if ((g & 1) != grp) continue;                          // the other group's tile
+        const int pb = grp;                                    // score buffer and P buffer of this group
         const int nvalid = min(TILE, tok1 - tok0 - t * TILE);
         if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
         tc_fence_after();
         float v[COLS];
-        if constexpr (COLS == 16) tmem_ld_32x16(lane_addr + COL_S + pb * TILE + col0, v);
-        else tmem_ld_32x32(lane_addr + COL_S + pb * TILE + col0, v);
-        tmem_wait_ld();
-        uint8_t* pbuf = smem + G::OFF_P + (g % PBUFS) * G::P_BUF;
+        {
+          float v0[32], v1[32];
+          tmem_ld_32x32(lane_addr + COL_S + pb * TILE, v0);
+          tmem_ld_32x32(lane_addr + COL_S + pb * TILE + 32, v1);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
+        }
+        uint8_t* pbuf = smem + G::OFF_P + pb * G::P_BUF;
         if (p.silu) {
-          // SiLU(s) / N(U) needs neither a reference maximum nor row sums: one pass, no exchange between the row's threads
-          if (g >= PBUFS && !mbar_wait(&p_free[g % PBUFS], (uint32_t)((g - PBUFS) / PBUFS) & 1u, p.err, 65)) { ok = false; break; }
-          lb_probabilities<true, COLS>(v, 0.f, col0, nvalid, pbuf, r);
+          // SiLU(s) / N(U) needs neither a reference maximum nor row sums: one pass, nothing shared between threads
+          if (g >= PBUFS && !mbar_wait(&p_free[pb], (uint32_t)((g - PBUFS) >> 1) & 1u, p.err, 65)) { ok = false; break; }
+          lb_probabilities<true, COLS>(v, 0.f, 0, nvalid, pbuf, r);
           tc_fence_before();
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&p_ready[g % PBUFS]);
+          if (lane == 0) mbar_arrive(&p_ready[pb]);
           continue;
         }
         float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < COLS; ++j)
-          if (col0 + j < nvalid) mx = fmaxf(mx, v[j]);
-        exch_max[(pb * PARTS + part) * 128 + r] = mx;
-        if (!lb_group_sync(&row_bar[q], row_uses, lane, p.err, 67)) { ok = false; break; }
-#pragma unroll
-        for (int i = 1; i < PARTS; ++i) mx = fmaxf(mx, exch_max[(pb * PARTS + ((part + i) & (PARTS - 1))) * 128 + r]);
-
+          if (j < nvalid) mx = fmaxf(mx, v[j]);
+        // the reference the other group left after the previous tile (every tile but the very first waits, whether or
+        // not it uses the value: the two groups then never drift more than one tile apart)
+        float m_prev = -INFINITY;
+        if (g > 0) {
+          if (!mbar_wait(&mref_bar[((g - 1) & 1) * 4 + q], (uint32_t)((g - 1) >> 1) & 1u, p.err, 69)) { ok = false; break; }
+          if (t > 0) m_prev = mref[((g - 1) & 1) * 128 + r];
+        }
+        if (m_prev != m_own && l_sum != 0.f) l_sum *= lb_ex2(m_own - m_prev);       // bring this group's sum up to date
         // raise the reference maximum only when it is exceeded by more than the threshold (or unset)
-        const bool need = mx > m_ref + LB_RESCALE_THRESHOLD;
-        const float m_new = need ? mx : m_ref;
-        const float factor = (need && m_ref != -INFINITY) ? lb_ex2(m_ref - m_new) : 1.0f;
+        const bool need = mx > m_prev + LB_RESCALE_THRESHOLD;
+        const float m_new = need ? mx : m_prev;
+        const float factor = (need && m_prev != -INFINITY) ? lb_ex2(m_prev - m_new) : 1.0f;
+        mref[(g & 1) * 128 + r] = m_new;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&mref_bar[(g & 1) * 4 + q]);
         if (__any_sync(0xffffffffu, need && t > 0)) {
-          // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale this part of the row
-          if (!mbar_wait(&p_free[(g - 1) % PBUFS], (uint32_t)((g - 1) / PBUFS) & 1u, p.err, 64)) { ok = false; break; }
+          // the accumulator must be quiescent: wait for the previous tile's second MMA, then scale the row
+          if (!mbar_wait(&p_free[(g - 1) & 1], (uint32_t)((g - 1) >> 1) & 1u, p.err, 64)) { ok = false; break; }
           tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < OUT; c += 32) {
+#pragma unroll 1
+          for (int c = 0; c < D; c += 32) {
             float a[32];
-            tmem_ld_32x32(lane_addr + COL_O + part * OUT + c, a);
+            tmem_ld_32x32(lane_addr + COL_O + c, a);
             tmem_wait_ld();
 #pragma unroll
             for (int j = 0; j < 32; ++j) a[j] *= factor;
-            tmem_st_32x32(lane_addr + COL_O + part * OUT + c, a);
+            tmem_st_32x32(lane_addr + COL_O + c, a);
           }
           tmem_wait_st();
         }
         l_sum *= factor;
-        m_ref = m_new;
+        m_own = m_new;
 
-        // the P that last sat in this buffer must have been consumed
-        if (g >= PBUFS && !mbar_wait(&p_free[g % PBUFS], (uint32_t)((g - PBUFS) / PBUFS) & 1u, p.err, 65)) { ok = false; break; }
-        l_sum += lb_probabilities<false, COLS>(v, m_ref, col0, nvalid, pbuf, r);
+        // the P that last sat in this group's buffer must have been consumed
+        if (g >= PBUFS && !mbar_wait(&p_free[pb], (uint32_t)((g - PBUFS) >> 1) & 1u, p.err, 65)) { ok = false; break; }
+        l_sum += lb_probabilities<false, COLS>(v, m_own, 0, nvalid, pbuf, r);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&p_ready[g % PBUFS]);
+        if (lane == 0) mbar_arrive(&p_ready[pb]);
       }
       if (!ok) break;
-      // item result: wait for the last second MMA, combine the parts' sums, read this part of the accumulator row
+      // item result: the final reference (published with the last tile), the two partial sums, then the accumulator
       const int gl = g - 1;
-      if (!mbar_wait(&p_free[gl % PBUFS], (uint32_t)(gl / PBUFS) & 1u, p.err, 66)) { ok = false; break; }
-      tc_fence_after();
-      exch_sum[part * 128 + r] = l_sum;
+      if (!p.silu) {
+        if ((gl & 1) != grp) {
+          if (!mbar_wait(&mref_bar[(gl & 1) * 4 + q], (uint32_t)(gl >> 1) & 1u, p.err, 70)) { ok = false; break; }
+          const float m_fin = mref[(gl & 1) * 128 + r];
+          if (m_fin != m_own && l_sum != 0.f) l_sum *= lb_ex2(m_own - m_fin);
+          m_own = m_fin;
+        }
+        exch_sum[grp * 128 + r] = l_sum;
+      }
       if (!lb_group_sync(&row_bar[q], row_uses, lane, p.err, 68)) { ok = false; break; }
-      float l_tot = 0.f;
-#pragma unroll
-      for (int i = 0; i < PARTS; ++i) l_tot += exch_sum[i * 128 + r];
-      // SiLU mode normalises by the number of keys (Algorithm 1): this chunk's tokens, summed over the chunks by the merge
-      if (p.silu) l_tot = (float)(tok1 - tok0);
+      float l_tot;
+      if (!p.silu) l_tot = exch_sum[r] + exch_sum[128 + r];
+      else l_tot = (float)(tok1 - tok0);   // SiLU mode normalises by the number of keys (Algorithm 1): this chunk's tokens, summed over the chunks by the merge
+      if (!mbar_wait(&p_free[gl & 1], (uint32_t)(gl >> 1) & 1u, p.err, 66)) { ok = false; break; }
+      tc_fence_after();
       const bool single = chunk_start[b + 1] - chunk_start[b] == 1;
       const float inv = 1.0f / l_tot;
       __nv_bfloat16* dst_o = p.Ohat + (int64_t)b * p.ell * (p.H * D) + ohat_off;
-      float* dst_p = p.part_acc + ((int64_t)w.ci * p.HL + R) * D + part * OUT;
-#pragma unroll
+      float* dst_p = p.part_acc + ((int64_t)w.ci * p.HL + R) * D + grp * OUT;
+#pragma unroll 1
       for (int c = 0; c < OUT; c += 32) {
         float a[32];
-        tmem_ld_32x32(lane_addr + COL_O + part * OUT + c, a);
+        tmem_ld_32x32(lane_addr + COL_O + grp * OUT + c, a);
         tmem_wait_ld();
         if (single) {
           // the whole history of this user was one chunk: normalise and write the attention row directly
@@ -396,9 +426,9 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
-      if (!single && part == 0) {
+      if (!single && grp == 0) {
         const int64_t prow = (int64_t)w.ci * p.HL + R;
-        p.part_m[prow] = p.silu ? 0.f : m_ref;        // log2 domain; equal weights for the chunks in SiLU mode
+        p.part_m[prow] = p.silu ? 0.f : m_own;        // log2 domain; equal weights for the chunks in SiLU mode
         p.part_s[prow] = l_tot;
       }
     }
@@ -412,7 +442,7 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   }
 }
 
-using LbD256 = LbCfg<256, 4, 3, 1>;       // d = 256: four threads per stacked row, three token stages, one CTA per SM
+using LbD256 = LbCfg<256, 3>;             // d = 256, three token stages
 
 bool link_attn_d256_tc_supported(int dtype, int d, int H, int ell, int phi) {
   return dtype == LIME_BF16 && d == 256 && (H * ell) % 128 == 0 && H * ell <= 512 && ell % 4 == 0 &&
@@ -432,8 +462,7 @@ static lime_status launch_link_attn_t64(const LinkAttnArgs& a, cudaStream_t st, 
   p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.silu = a.silu; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
-  const int slots = kSMs * G::MINB;
-  int grid = a.n_chunk_upper * p.RB < slots ? a.n_chunk_upper * p.RB : slots;
+  int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;
   grid -= grid % p.RB;                              // a CTA's work items then all share its row block
   lime_status es = ensure_dynamic_smem((const void*)k_link_attn_t64_tc<G>, (int)G::SMEM, smem_set);
   if (es != LIME_OK) return es;
