@@ -168,6 +168,13 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         const int t = t_begin + g;
         const int b = tu.of(tile_start, p.B, t);
         const int urow = p.shared ? 0 : b;
+        // Operand slabs go out in the order of use.  The first ring-load of this tile's K2 slabs is requested BEFORE the
+        // wait for the X / O buffer: the slabs only need free ring slots (which the previous tile's last contractions
+        // release one by one), so they travel while that tile is still being finished and stored.
+        int k2_done = 0;
+        for (; k2_done < HC_RING && k2_done < NG * 4 && ok; ++k2_done)
+          ok = slab(&tmK2, (k2_done & 3) * 64, urow * p.HL + (k2_done >> 2) * 128);
+        if (!ok) break;
         // the X / O buffer and (on a change of user) the value buffer are free once the previous tile's last
         // contraction over O has run: every MMA issued before it, the value mixes included, has then finished
         if (g > 0 && !mbar_wait(x_free, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
@@ -180,10 +187,10 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
           ++vn;
         }
         prev_user = b;
-        // operand slabs in the order of use: K2 of every group; then per half of the hidden columns the gate and up
-        // columns of W_g / W_u (contraction over d) and that half's rows of W_o (both halves of the output columns)
-        for (int c = 0; c < NG && ok; ++c)
-          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab(&tmK2, kb * 64, urow * p.HL + c * 128);
+        // the rest: K2 of the remaining groups; then per half of the hidden columns the gate and up columns of
+        // W_g / W_u (contraction over d) and that half's rows of W_o (both halves of the output columns)
+        for (; k2_done < NG * 4 && ok; ++k2_done)
+          ok = slab(&tmK2, (k2_done & 3) * 64, urow * p.HL + (k2_done >> 2) * 128);
         for (int hf = 0; hf < 2 && ok; ++hf) {
           if (hf == 1) {
             for (int nh = 0; nh < 2 && ok; ++nh)
