@@ -11,38 +11,55 @@
 
 namespace lime {
 
-// ----------------------------------------------------------------------------- Y[r, :] = X[r, :] . W[row0 .. row0+K, :] (+ b)
-// Small dense product with fp32 accumulation: a block takes FR_ROWS rows of X into shared memory, a thread one output
-// column at a time (weight reads coalesced over the columns).  Outputs: fp32 [M x N] and / or bf16 transposed per group
-// of `group` rows ([M/group][N][group], the K-major operand layout of k_score_head_tc.cu).
-constexpr int FR_ROWS = 16, FR_THREADS = 128;
+// ----------------------------------------------------------------------------- Y[r, :] = X[r, :] . W (+ b)
+// Small dense product with fp32 accumulation.  A block takes FR_ROWS rows of X and FR_COLS output columns; the rows sit in
+// shared memory, the block's slice of W is staged there too in pieces of FR_KC contraction indices (read once, coalesced
+// over the columns), and a thread forms FR_ROWS / 4 x 1 outputs per piece from shared memory only.  Outputs: fp32 [M x N]
+// and / or bf16 transposed per group of `group` rows ([M/group][N][group], the K-major operand layout of
+// k_score_head_tc.cu).
+constexpr int FR_ROWS = 32, FR_COLS = 32, FR_KC = 64, FR_THREADS = 128;      // thread (ty, tx): rows ty*8..ty*8+7, column tx
 template <typename TX, typename TW>
 __global__ void __launch_bounds__(FR_THREADS)
 k_rows_times_w(const TX* __restrict__ X, int64_t M, int K, const TW* __restrict__ W, int ldw, int N, const float* __restrict__ bias,
                float* __restrict__ Y, __nv_bfloat16* __restrict__ Yt, int group) {
-  extern __shared__ float xs[];                     // [FR_ROWS][K]
+  extern __shared__ float fr_sm[];
+  float* xs = fr_sm;                                 // [FR_ROWS][K + 1]
+  float* wsm = xs + FR_ROWS * (K + 1);               // [FR_KC][FR_COLS]
   const int64_t r0 = (int64_t)blockIdx.x * FR_ROWS;
+  const int c0 = blockIdx.y * FR_COLS;
   const int nr = (int)min((int64_t)FR_ROWS, M - r0);
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   for (int i = threadIdx.x; i < FR_ROWS * K; i += FR_THREADS) {
     const int r = i / K, k = i % K;
-    xs[i] = r < nr ? Store<TX>::ld(X + (r0 + r) * K + k) : 0.f;
+    xs[r * (K + 1) + k] = r < nr ? Store<TX>::ld(X + (r0 + r) * K + k) : 0.f;
   }
-  __syncthreads();
-  for (int j = threadIdx.x; j < N; j += FR_THREADS) {
-    float acc[FR_ROWS];
-    const float b = bias ? bias[j] : 0.f;
+  constexpr int RPT = FR_ROWS / 4;                   // rows per thread
+  float acc[RPT];
+  const int col = c0 + tx;
+  const float b = (bias && col < N) ? bias[col] : 0.f;
 #pragma unroll
-    for (int r = 0; r < FR_ROWS; ++r) acc[r] = b;
-#pragma unroll 8
-    for (int k = 0; k < K; ++k) {
-      const float w = Store<TW>::ld(W + (int64_t)k * ldw + j);
-#pragma unroll
-      for (int r = 0; r < FR_ROWS; ++r) acc[r] = fmaf(xs[r * K + k], w, acc[r]);
+  for (int r = 0; r < RPT; ++r) acc[r] = b;
+  for (int k0 = 0; k0 < K; k0 += FR_KC) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < FR_KC * FR_COLS; i += FR_THREADS) {
+      const int kk = i / FR_COLS, c = i % FR_COLS;
+      wsm[i] = (k0 + kk < K && c0 + c < N) ? Store<TW>::ld(W + (int64_t)(k0 + kk) * ldw + c0 + c) : 0.f;
     }
-    for (int r = 0; r < nr; ++r) {
-      const int64_t row = r0 + r;
-      if (Y) Y[row * N + j] = acc[r];
-      if (Yt) Yt[((row / group) * N + j) * group + (row % group)] = __float2bfloat16_rn(acc[r]);
+    __syncthreads();
+    const int kn = min(FR_KC, K - k0);
+    for (int kk = 0; kk < kn; ++kk) {
+      const float w = wsm[kk * FR_COLS + tx];
+#pragma unroll
+      for (int r = 0; r < RPT; ++r) acc[r] = fmaf(xs[(ty * RPT + r) * (K + 1) + k0 + kk], w, acc[r]);
+    }
+  }
+  if (col < N) {
+    for (int r = 0; r < RPT; ++r) {
+      const int rr = ty * RPT + r;
+      if (rr >= nr) break;
+      const int64_t row = r0 + rr;
+      if (Y) Y[row * N + col] = acc[r];
+      if (Yt) Yt[((row / group) * N + col) * group + (row % group)] = __float2bfloat16_rn(acc[r]);
     }
   }
 }
@@ -50,9 +67,9 @@ k_rows_times_w(const TX* __restrict__ X, int64_t M, int K, const TW* __restrict_
 lime_status launch_rows_times_w(const void* X, int x_dtype, int64_t M, int K, const void* W, int w_dtype, int ldw, int N,
                                 const float* bias, float* Y, void* Yt, int group, const char* name, cudaStream_t st) {
   if (M == 0 || N == 0) return LIME_OK;
-  const size_t smem = sizeof(float) * FR_ROWS * (size_t)K;
-  if (smem > 96 * 1024) return LIME_UNSUPPORTED_SHAPE;
-  const unsigned grid = (unsigned)((M + FR_ROWS - 1) / FR_ROWS);
+  const size_t smem = sizeof(float) * (FR_ROWS * ((size_t)K + 1) + FR_KC * FR_COLS);
+  if (smem > 200 * 1024) return LIME_UNSUPPORTED_SHAPE;
+  const dim3 grid((unsigned)((M + FR_ROWS - 1) / FR_ROWS), (unsigned)((N + FR_COLS - 1) / FR_COLS));
   ProfScope _p(name, st);
 #define LIME_RTW(TX, TW)                                                                                                  \
   do {                                                                                                                    \
