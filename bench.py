@@ -267,11 +267,17 @@ def launch_mode(args):
 NCU_TRAFFIC = {
     # dense scorer: 169.9 MB read + 4.0-4.5 MB written per launch
     ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
-    # XOR-layer kernels: 33.7 MB (layer 1) and 42.1 MB (layer 2) read + written; average per launch
-    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "756d8af8ad9dd54b"},
-    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.5e6, "source": "k_hist_update_tc.cu", "sha": "cbdc6b1690b70517"},
-    # scorer by id: 170.0 MB read + 3.9 MB written per launch
-    ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 173.9e6, "source": "k_score_gather_tc.cu", "sha": "4daad32675f4aff5"},
+    # XOR-layer kernels: 33.7 MB (layer 1) and 42.2 MB (layer 2) read + written; average per launch
+    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "186136fa777f8d53"},
+    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.6e6, "source": "k_hist_update_tc.cu", "sha": "cbdc6b1690b70517"},
+    # scorer by id over packed corpus records: 174.5 MB read + 4.1 MB written per launch
+    ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 178.6e6, "source": "k_score_gather_tc.cu", "sha": "2b14f0762b275cd7"},
+    # scorer through the interaction network (--head 96): 169.4 MB read + 4.4 MB written per launch
+    ("k_score_head_tc", "bf16_baseline", 256, 2048): {"bytes": 173.8e6, "source": "k_score_head_tc.cu", "sha": "614556b96c1342b2"},
+    # d = 256 kernels: captured on 128 users of the same model and length mix (327,693 tokens) and scaled by the tokens of
+    # a launch (persistent kernels, identical tiles: traffic grows in proportion): bytes per token, average of the layers
+    ("k_link_attn_d256_tc", "production_ragged", 1024, 8192): {"bytes_per_token": 560.0, "source": "k_link_attn_t64_tc.cu", "sha": "a9c8341ced1c82f4"},
+    ("k_hist_update_d256_tc", "production_ragged", 1024, 8192): {"bytes_per_token": 880.0, "source": "k_hist_update_d256_tc.cu", "sha": "0627bdad4ab0a4bd"},
 }
 
 
@@ -281,14 +287,18 @@ def source_hash(rel):
         return hashlib.sha256(f.read()).hexdigest()[:16]
 
 
-def ncu_traffic(kernel, wl, args=None):
+def ncu_traffic(kernel, wl, args=None, tokens=None):
     rec = NCU_TRAFFIC.get((kernel, wl.name, wl.B, wl.C))
     if not rec or (args is not None and (args.cand_heads or args.phi != "softmax")):
         return None          # the captures were taken in the default mode
     try:
-        return rec["bytes"] if source_hash(rec["source"]) == rec["sha"] else None
+        if source_hash(rec["source"]) != rec["sha"]:
+            return None
     except OSError:
         return None
+    if "bytes_per_token" in rec:
+        return rec["bytes_per_token"] * tokens if tokens else None
+    return rec["bytes"]
 
 
 def run_ours(args, wl, sampler=None, with_sweeps=False):
@@ -599,7 +609,7 @@ def run_ours(args, wl, sampler=None, with_sweeps=False):
         def roof(k, ms=None, how="CUDA events around each launch inside the step"):
             mdl = model_for(k["kernel"], models)
             r = dict(kernel=k["kernel"], **roofline_entry(mdl, ms if ms is not None else k["ms_per_step"], pk))
-            r["traffic"] = ncu_traffic(k["kernel"], wl, args)
+            r["traffic"] = ncu_traffic(k["kernel"], wl, args, avg_tokens)
             r["peak_source"] = ("derived: 148 SM x 128 lanes x 2 x 1.965 GHz" if r["bound"] == "alu" else
                                 f"{pk['source']} ({'copy bandwidth' if r['bound'] == 'hbm' else 'sustained bf16 GEMM'})")
             r["timing"] = how
