@@ -15,7 +15,7 @@ namespace lime {
 constexpr int GM_THREADS = 192, GM_MAX_STAGES = 6;
 constexpr uint32_t GM_SUB = 128 * 128;    // [128 rows x 64 bf16]
 
-enum { GM_EPI_PREP = 0 };
+enum { GM_EPI_PREP = 0, GM_EPI_ROWS_T = 1 };
 
 struct GemmParams {
   int64_t M;            // valid rows of A / C
@@ -26,6 +26,9 @@ struct GemmParams {
   int d, f, plain_v;                // output widths; plain_v: the third segment is V[T] (d columns) instead of G2 | U2
   __nv_bfloat16 *Q2, *K2, *G2t, *U2t, *V2t;
   float *cQ, *cK;                   // row sums of Q2 / K2 (only with d = 128: one n-tile per row)
+  // ROWS_T: out[(row / group) * n_cols + col][row % group] for col < n_cols (bf16): the product transposed per group of rows
+  __nv_bfloat16* out_t;
+  int group, n_cols;
   int* err;
 };
 
@@ -159,6 +162,21 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             }
           }
         }
+      } else if (EPI == GM_EPI_ROWS_T) {
+        const int64_t u = row / p.group;
+        const int l = (int)(row % p.group);
+        __nv_bfloat16* dst = p.out_t + (u * p.n_cols + (int64_t)nt * NT) * p.group + l;
+#pragma unroll
+        for (int c = 0; c < NT; c += 16) {
+          float v[16];
+          tmem_ld_32x16(lane_addr + c, v);
+          tmem_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (nt * NT + c + j < p.n_cols) dst[(int64_t)(c + j) * p.group] = __float2bfloat16_rn(v[j]);
+          }
+        }
       }
     }
   }
@@ -201,6 +219,16 @@ lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st) {
   const int cols_all = 2 * a.H * a.K + (a.plain_v ? a.K : 2 * a.H * a.f);
   const int n_tiles = (a.need_hist ? cols_all : a.H * a.K) / 128;
   return launch_gemm<GM_EPI_PREP, 128>(a.A, a.M, a.K, a.Bt, cols_all, n_tiles, p, "k_gemm_tc_prep", st);
+}
+
+// A [M x K] . Bt^T with Bt [n_cols x K] (bf16, K a multiple of 64): the product as bf16, transposed per group of `group`
+// consecutive rows: out_t [M / group][n_cols][group]
+lime_status launch_gemm_rows_t(const void* A, int64_t M, int K, const void* Bt, int n_cols, int group, void* out_t, int* err,
+                               const char* name, cudaStream_t st) {
+  if (K % 64 || K < 64 || n_cols < 1 || group < 1) return LIME_UNSUPPORTED_SHAPE;
+  GemmParams p{};
+  p.out_t = (__nv_bfloat16*)out_t; p.group = group; p.n_cols = n_cols; p.err = err;
+  return launch_gemm<GM_EPI_ROWS_T, 128>(A, M, K, Bt, n_cols, (n_cols + 127) / 128, p, name, st);
 }
 
 }  // namespace lime

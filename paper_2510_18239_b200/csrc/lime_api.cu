@@ -418,7 +418,7 @@ lime_status lime_create(const lime_config* cfg, lime_ctx** out) {
   c->ln_eps = g.ln_eps > 0.f ? g.ln_eps : 1e-5f;
   c->keff = nullptr; c->keff_hl = nullptr; c->links32 = nullptr; c->dev_err = nullptr;
   c->have_head = c->have_ctx_mlp = false; c->ctx_dc = 0;
-  c->head_W1bT = nullptr; c->head_w2 = nullptr; c->ctx_first = nullptr;
+  c->head_W1bT = nullptr; c->head_W1aT = nullptr; c->head_w2 = nullptr; c->ctx_first = nullptr;
   c->tc_mode = tensor_core_mode(g, d_ff);
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) c->WoT[j] = c->WprepT[j] = c->WpostT[j] = c->WguT[j] = nullptr;
   c->sh_That = c->sh_Q2 = c->sh_K2 = c->sh_G2t = c->sh_U2t = c->sh_V2t = nullptr; c->sh_cQ = c->sh_cK = nullptr;
@@ -450,7 +450,7 @@ lime_status lime_destroy(lime_ctx* ctx) {
   for (int j = 0; j < LIME_MAX_LAYERS; ++j) { cudaFree(c->WoT[j]); cudaFree(c->WprepT[j]); cudaFree(c->WpostT[j]); cudaFree(c->WguT[j]); }
   cudaFree(c->sh_That); cudaFree(c->sh_Q2); cudaFree(c->sh_K2); cudaFree(c->sh_G2t); cudaFree(c->sh_U2t); cudaFree(c->sh_V2t);
   cudaFree(c->sh_cQ); cudaFree(c->sh_cK);
-  cudaFree(c->head_W1bT); cudaFree(c->head_w2); cudaFree(c->ctx_first);
+  cudaFree(c->head_W1bT); cudaFree(c->head_W1aT); cudaFree(c->head_w2); cudaFree(c->ctx_first);
   delete c;
   return LIME_OK;
 }
@@ -725,8 +725,8 @@ lime_status lime_set_head(lime_ctx* ctx, const lime_ffn* head, void* stream) {
   const lime_config& g = c->cfg;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int w0 = head->widths[0], w_last = head->widths[head->n_hidden - 1];
-  cudaFree(c->head_W1bT); cudaFree(c->head_w2);
-  c->head_W1bT = nullptr; c->head_w2 = nullptr;
+  cudaFree(c->head_W1bT); cudaFree(c->head_W1aT); cudaFree(c->head_w2);
+  c->head_W1bT = nullptr; c->head_W1aT = nullptr; c->head_w2 = nullptr;
   c->have_head = false;
   LIME_CUDA(cudaMalloc(&c->head_w2, sizeof(float) * (size_t)w_last));
   lime_status s = launch_widen(head->W[head->n_hidden], g.dtype, c->head_w2, w_last, st);
@@ -736,6 +736,8 @@ lime_status lime_set_head(lime_ctx* ctx, const lime_ffn* head, void* stream) {
     LIME_CUDA(cudaMalloc(&c->head_W1bT, (size_t)w0 * g.d * 2));
     const char* W0t = static_cast<const char*>(head->W[0]) + (size_t)g.d * w0 * 2;
     if ((s = launch_transpose_bf16(W0t, g.d, w0, c->head_W1bT, st)) != LIME_OK) return s;
+    LIME_CUDA(cudaMalloc(&c->head_W1aT, (size_t)w0 * g.d * 2));
+    if ((s = launch_transpose_bf16(head->W[0], g.d, w0, c->head_W1aT, st)) != LIME_OK) return s;
   }
   c->head = *head;
   c->have_head = true;
@@ -777,8 +779,12 @@ lime_status lime_score_candidates_head(lime_ctx* ctx, const void* link_states, i
   a.corpus_rows = cand_ids ? corpus_rows : 0; a.dev_flag = cand_ids ? dev_flag : nullptr;
   const bool tc = f.n_hidden == 1 && c->head_W1bT && score_head_tc_supported(a, w0);
   // per user: LSW_b = LS_b W_0[:d]  (the O half of the first layer applied to the link states, so O is never formed)
-  lime_status s = launch_rows_times_w(link_states, g.dtype, (int64_t)B * c->ell_c, g.d, f.W[0], g.dtype, w0, w0, nullptr,
-                                      tc ? nullptr : LSW, tc ? LSWt : nullptr, c->ell_c, "k_head_lsw", st);
+  lime_status s;
+  if (tc && c->head_W1aT && g.d % 64 == 0)      // on tensor cores when the scorer is (link states and W_0 are bf16)
+    s = launch_gemm_rows_t(link_states, (int64_t)B * c->ell_c, g.d, c->head_W1aT, w0, c->ell_c, LSWt, c->dev_err, "k_gemm_tc_lsw", st);
+  else
+    s = launch_rows_times_w(link_states, g.dtype, (int64_t)B * c->ell_c, g.d, f.W[0], g.dtype, w0, w0, nullptr,
+                            tc ? nullptr : LSW, tc ? LSWt : nullptr, c->ell_c, "k_head_lsw", st);
   if (s != LIME_OK) return s;
   if (tc) {
     ScoreHeadArgs h{LSWt, c->head_W1bT, f.b[0], c->head_w2, f.b[1], w0};

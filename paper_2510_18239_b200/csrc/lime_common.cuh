@@ -68,6 +68,7 @@ struct Ctx {
   lime_ffn head, ctx_mlp;
   int ctx_dc;            // context features per user
   void* head_W1bT;       // [w0 x d] bf16: the T half of the head's first layer, transposed (tensor-core path)
+  void* head_W1aT;       // [w0 x d] bf16: its O half, transposed (B operand of the per-user link-state product)
   float* head_w2;        // [w_last] fp32 copy of the head's last layer
   float* ctx_first;      // [ell x w0] fp32: (L W_0[:d]) + b_0 of the context MLP
   int* dev_err;     // device word: 0, or the code of the first bounded wait that gave up in a kernel of this context
@@ -239,6 +240,10 @@ struct LinkGemmArgs {
   int* err;
 };
 lime_status launch_gemm_prep(const LinkGemmArgs& a, cudaStream_t st);
+// A [M x K] . Bt^T, Bt [n_cols x K] (bf16, K % 64 == 0, 16-byte aligned): bf16 result transposed per group of rows,
+// out_t [M / group][n_cols][group]
+lime_status launch_gemm_rows_t(const void* A, int64_t M, int K, const void* Bt, int n_cols, int group, void* out_t, int* err,
+                               const char* name, cudaStream_t st);
 
 // GatedMLP on link rows fused with its consumers (k_link_mlp_tc.cu); d = d_ff in {128, 256}
 struct LinkMlpArgs {
