@@ -376,6 +376,8 @@ def run_user(E: np.ndarray, L: np.ndarray, layers, cfg: OracleConfig, T: np.ndar
     if cand_heads:
         if W is None:
             W = precompute_candidate_links_heads(T, L, cfg, cand_w.get("Wq_c"), cand_w.get("Wk_c"))
+        if head is not None:
+            return interaction_head(candidate_outputs_heads(W, LS, cfg), T, head), LS, W
         return score_candidates_heads(W, LS, T, cfg), LS, W
     if W is None:
         W = precompute_candidate_links(T, L, cfg, cand_w.get("Wq_c"), cand_w.get("Wk_c"))

@@ -195,3 +195,36 @@ def test_bounded_wait_expires_and_reports():
     assert off.cpu().tolist() == [0, 3, 3, 7]
     with pytest.raises(Bd.LimeError):
         Bd.lime_selftest_wait_expiry(lime.ctx, 0)
+
+
+@pytest.mark.parametrize("dtype,d,H,ell,n1", [(synth.BF16, 128, 2, 16, 64), (synth.F32, 32, 2, 8, 24)])
+def test_interaction_head_after_the_whole_path_with_head_wise_candidate_side(dtype, d, H, ell, n1):
+    """offsets -> lookup -> XOR layers -> link states -> precompute -> interaction network, with the candidate side run
+    head by head (H * ell weight columns per candidate, link states expanded per head): every logit against the oracle."""
+    Bd = _lib()
+    wl = synth.Workload("headwise", B=3, n_min=20, n_max=150, d=d, H=H, ell=ell, n_layers=2, C=70, dtype=dtype, V=900,
+                        zipf_s=1.1, table_std=0.5, link_std=1.0)
+    inp = synth.make_inputs(wl, seed=5)
+    dev = Hh.DeviceBatch(wl, inp, cand_heads=H)
+    lime = dev.lime
+    layers = synth.ffn_weights(9, "head", (2 * d, n1, 1), dtype)
+    lime.set_head(_dev_ffn(Bd, layers, dtype))
+    off = lime.lengths_to_offsets(dev.lengths)
+    ls = lime.encode_user(lime.gather_history(dev.table, dev.hist_ids), off)
+    cand = lime.gather_history(dev.table, dev.cand_ids)
+    W = lime.precompute_candidate_links(cand)
+    assert tuple(W.shape) == (wl.B * wl.C, H * ell) and tuple(ls.shape) == (wl.B, H * ell, d)
+    got = Hh.to_f64(lime.score_candidates_head(ls, W, cand, C=wl.C))
+    Bd.lime_device_status(lime.ctx)
+    cfg, lay, L64 = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl), _ffn64(layers, dtype)
+    table64, links64 = synth.storage_to_f64(inp["table"], dtype), synth.storage_to_f64(inp["links"], dtype)
+    offs = O.lengths_to_offsets(inp["lengths"])
+    worst, spread = 0.0, 0.0
+    for b in range(wl.B):
+        want, _, _ = Hh.oracle_user(inp, wl, b, offs, table64, links64, lay, cfg, cand_heads=True, head=L64)
+        worst = max(worst, float(np.abs(got[b * wl.C:(b + 1) * wl.C] - want).max()))
+        spread = max(spread, float(want.std()))
+    if dtype == synth.F32:
+        assert worst <= 1e-4 * max(1.0, spread), (worst, spread)
+    else:
+        assert worst <= 2e-2 and worst <= 6e-2 * spread + 1e-3, (worst, spread)
