@@ -98,32 +98,34 @@ lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, flo
 
 // Combine the chunks of a user with log-sum-exp weights and normalise (maxima are kept in the log2 domain):
 //   Ohat[(u*ell + l), h*d + i] = sum_c w_c acc_c[(h,l), i] / sum_c w_c s_c,   w_c = 2^(m_c - max_c m_c)
-// Blocks of 128 threads walk the (user, group of MERGE_ROWS rows) pairs with a grid stride (a few blocks per SM: when no
-// user has more than one chunk the launch is over as soon as the users have been looked at); within a pair each warp
-// takes rows, a lane four consecutive
-// columns at a time (128-bit reads of the partial accumulators, four chunks in flight).  d is a multiple of 8.  A user
-// without history gets zeros; a user with a single chunk was already written by the attention kernel (its blocks
-// return at once).
-constexpr int MERGE_ROWS = 8;
-__global__ void __launch_bounds__(128)
-k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int B, int ell, int d, int H, const float* __restrict__ part_m,
-                       const float* __restrict__ part_s, const float* __restrict__ part_acc,
-                       __nv_bfloat16* __restrict__ Ohat) {
+// One warp per (user, stacked row), walked with a grid stride: lane c first takes chunk c's (m, s) (32 chunks at a time),
+// the warp reduces the maximum and the weighted sum with shuffles, then every lane owns four consecutive columns per
+// 128-column piece of the row and reads the chunks' partial accumulators as 128-bit words, four chunks in flight.
+// d is a multiple of 4.  A user without history gets zeros; a user with a single chunk was already written by the
+// attention kernel (its warps move on at once); when the schedule says that every user is such a user (*merge_needed == 0)
+// the whole grid returns after one read.
+__global__ void __launch_bounds__(256)
+k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, const int32_t* __restrict__ merge_needed, int B, int ell, int d,
+                       int H, const float* __restrict__ part_m, const float* __restrict__ part_s,
+                       const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
+  if (merge_needed != nullptr && *merge_needed == 0) return;
   const int HL = H * ell;
-  const int groups = (HL + MERGE_ROWS - 1) / MERGE_ROWS;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int64_t pair = blockIdx.x; pair < (int64_t)B * groups; pair += gridDim.x) {
-  const int u = (int)(pair / groups), grp = (int)(pair % groups);
-  const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
-  if (c1 - c0 == 1) continue;
-  const int row_end = min(HL, (grp + 1) * MERGE_ROWS);
-  for (int row = grp * MERGE_ROWS + warp; row < row_end; row += 4) {
+  const int lane = threadIdx.x & 31;
+  const int64_t n_rows = (int64_t)B * HL;
+  const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t wr = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wr < n_rows; wr += warps) {
+    const int u = (int)(wr / HL), row = (int)(wr % HL);
+    const int c0 = chunk_start[u], c1 = chunk_start[u + 1];
+    if (c1 - c0 == 1) continue;
     const int h = row / ell, l = row % ell;
     __nv_bfloat16* dst = Ohat + ((int64_t)u * ell + l) * (H * d) + h * d;
+    // maximum over the chunks, then the normaliser
     float M = -INFINITY;
-    for (int c = c0; c < c1; ++c) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
+    for (int c = c0 + lane; c < c1; c += 32) M = fmaxf(M, part_m[(int64_t)c * HL + row]);
+    M = warp_max(M);
     float S = 0.f;
-    for (int c = c0; c < c1; ++c) S = fmaf(part_s[(int64_t)c * HL + row], exp2f(part_m[(int64_t)c * HL + row] - M), S);
+    for (int c = c0 + lane; c < c1; c += 32) S = fmaf(part_s[(int64_t)c * HL + row], exp2f(part_m[(int64_t)c * HL + row] - M), S);
+    S = warp_sum(S);
     const float inv = c1 > c0 ? 1.0f / S : 0.f;
     for (int i = lane * 4; i < d; i += 128) {
       float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -154,16 +156,15 @@ k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, int B, int ell, 
       *reinterpret_cast<uint2*>(dst + i) = o;
     }
   }
-  }
 }
 
-lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
-                                        const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
+lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, const int32_t* merge_needed, int B, int ell, int d, int H,
+                                        const float* part_m, const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st) {
   if (B == 0) return LIME_OK;
   ProfScope _p("k_link_attn_merge_norm", st);
-  const int64_t pairs = (int64_t)B * ((H * ell + MERGE_ROWS - 1) / MERGE_ROWS);
-  const int grid = (int)(pairs < (int64_t)kSMs * 8 ? pairs : (int64_t)kSMs * 8);
-  k_link_attn_merge_norm<<<grid, 128, 0, st>>>(chunk_start, B, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  const int64_t blocks_needed = ((int64_t)B * H * ell + 7) / 8;           // 8 warps (rows) per block
+  const int grid = (int)(blocks_needed < (int64_t)kSMs * 8 ? blocks_needed : (int64_t)kSMs * 8);
+  k_link_attn_merge_norm<<<grid, 256, 0, st>>>(chunk_start, merge_needed, B, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }

@@ -51,7 +51,15 @@ __global__ void __launch_bounds__(1024) k_offsets(const int32_t* __restrict__ le
 // both work lists of the XOR layers in one launch: chunks of the links<-history attention, tiles of the history update
 __global__ void __launch_bounds__(1024)
 k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __restrict__ chunk_start, int tile,
-                  int32_t* __restrict__ tile_start, int32_t* __restrict__ chunk_user) {
+                  int32_t* __restrict__ tile_start, int32_t* __restrict__ chunk_user, int32_t* __restrict__ merge_needed) {
+  // does any user's attention output need the merge step (several chunks to combine, or no history: a zero row)?
+  __shared__ int any_merge;
+  if (threadIdx.x == 0) any_merge = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < B; b += blockDim.x)
+    if (off[b + 1] - off[b] <= 0 || off[b + 1] - off[b] > chunk) any_merge = 1;
+  __syncthreads();
+  if (threadIdx.x == 0 && merge_needed != nullptr) *merge_needed = any_merge;
   block_exclusive_scan(B, chunk_start, [&](int i) {
     int n = off[i + 1] - off[i];
     return n > 0 ? (n + chunk - 1) / chunk : 0;
@@ -70,9 +78,9 @@ k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __
 }
 
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
-                                   int32_t* chunk_user, cudaStream_t st) {
+                                   int32_t* chunk_user, int32_t* merge_needed, cudaStream_t st) {
   ProfScope _p("k_layer_schedules", st);
-  k_layer_schedules<<<1, 1024, 0, st>>>(off, B, chunk, chunk_start, tile, tile_start, chunk_user);
+  k_layer_schedules<<<1, 1024, 0, st>>>(off, B, chunk, chunk_start, tile, tile_start, chunk_user, merge_needed);
   LIME_LAUNCH_CHECK("k_layer_schedules");
   return LIME_OK;
 }

@@ -67,7 +67,7 @@ struct Workspace {
   void *S, *Q, *K, *V, *U;
   // link rows, fp32
   float *T, *QT, *KT, *VT, *AT, *UT, *LP, *LS32;
-  int32_t *chunk_start, *tile_start, *chunk_user;
+  int32_t *chunk_start, *tile_start, *chunk_user, *merge_needed;
   float *part_m, *part_s, *part_acc;
   // tensor-core path: folded link-side operands (bf16) and their row sums
   void *Q2, *K2, *G2t, *U2t, *V2t;
@@ -92,6 +92,7 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.AT = (float*)take(ld); w.UT = (float*)take(lf); w.LP = (float*)take(ld); w.LS32 = (float*)take(ld);
   w.chunk_start = (int32_t*)take((size_t)(B + 1) * 4);
   w.tile_start = (int32_t*)take((size_t)(B + 1) * 4);
+  w.merge_needed = (int32_t*)take(4);
   const bool tc_link = c->tc_mode != 0;
   // tensor-core path: at least 4 token tiles per work item, one item per 128-row block of H * ell (at d = 256 a set of
   // partials is 4 x larger and the batches served have many users, so chunks may be longer still)
@@ -169,7 +170,7 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
   const bool pass_stats = hist_ln && hist_out && one_block_update && total > 0;
   la.stats_out = pass_stats ? w.row_stats : nullptr;
   if ((s = c->tc_mode == 2 ? launch_link_attn_d256_tc(la, st) : launch_link_attn_tc(la, st)) != LIME_OK) return s;
-  if ((s = launch_link_attn_merge_norm(w.chunk_start, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
+  if ((s = launch_link_attn_merge_norm(w.chunk_start, w.merge_needed, B, g.ell, g.d, g.H, w.part_m, w.part_s, w.part_acc, w.Ohat, st)) != LIME_OK)
     return s;
   // T^j = GatedMLP(O[T]) with W_V folded into the gate / up weights, and what the next step needs from it
   mlp.Ohat = w.Ohat; mlp.M = (int64_t)B * g.ell; mlp.K = g.H * g.d; mlp.d = g.d; mlp.WpostT = c->WpostT[layer]; mlp.WoT = c->WoT[layer];
@@ -251,7 +252,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   const lime_config& g = c->cfg;
   lime_status s;
   if (!schedules_ready) {
-    if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, st)) != LIME_OK) return s;
+    if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, st)) != LIME_OK) return s;
   }
   if (layer_on_tensor_cores(c, layer))
     return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, st);
@@ -603,7 +604,7 @@ static lime_status encode_user_impl(lime_ctx* ctx, const void* hist, bool hist_n
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   lime_status s;
-  if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, st)) != LIME_OK) return s;
+  if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, st)) != LIME_OK) return s;
   const int64_t BLd = (int64_t)B * g.ell * g.d;
   if (layer_on_tensor_cores(c, 0)) {
     if ((s = encode_user_tc(c, hist, hist_normalized, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;

@@ -111,9 +111,10 @@ lime_status launch_gather_ln(int dtype, const void* table, int64_t V, int d, flo
                              void* out, int32_t* dev_flag, cudaStream_t st);
 
 // Work lists of the XOR layers in one launch: chunk_start[b] = sum_{b' < b} ceil(len_b' / chunk) and
-// tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B; chunk_user[item] = user of the chunk item (may be NULL)
+// tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B; chunk_user[item] = user of the chunk item (may be NULL);
+// *merge_needed (may be NULL) = 1 if any user has several chunks or none (its attention rows come from the merge step)
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
-                                   int32_t* chunk_user, cudaStream_t st);
+                                   int32_t* chunk_user, int32_t* merge_needed, cudaStream_t st);
 
 // Y[r, n] (+)= epilogue( LN?(X[r, :]) . W[:, n] ) for up to three weight matrices sharing X.
 struct LinearArgs {
@@ -227,8 +228,8 @@ lime_status launch_score_head_tc(const ScoreArgs& a, const ScoreHeadArgs& h, int
 lime_status launch_fold_weights(const void* Wq, const void* Wk, const void* Wv, const void* Wg, const void* Wu, int d,
                                 int H, int f, float scale, int plain_v, void* WprepT, void* WpostT, cudaStream_t st);
 lime_status launch_ln_rows_bf16(const float* T, int64_t rows, int d, int ln, float eps, void* out, cudaStream_t st);
-lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, int B, int ell, int d, int H, const float* part_m,
-                                        const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st);
+lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, const int32_t* merge_needed, int B, int ell, int d, int H,
+                                        const float* part_m, const float* part_s, const float* part_acc, void* Ohat, cudaStream_t st);
 lime_status launch_transpose_bf16(const void* W, int rows, int cols, void* WT, cudaStream_t st);
 
 // link-row GEMMs on tensor cores (k_gemm_tc.cu); A [M x K] bf16 row-major, Bt [N x K] bf16 (weights, pre-folded)
