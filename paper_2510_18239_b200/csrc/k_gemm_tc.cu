@@ -4,15 +4,16 @@
 //          folded gate / up operands G2t, U2t (N = 2*H*d + 2*H*f) or the plain link values V[T], stored transposed
 //          (N = 2*H*d + d), that the streaming kernels contract against the history (Eq. 7); weights folded once at
 //          set-up, see k_link_prep.cu.  d and f are multiples of 128.
-// One CTA per 128-row x 128-column output tile: warp 0 streams K blocks of A and B with TMA through a stage ring,
-// warp 1 issues the MMAs, warps 2-5 (one thread per output row = TMEM lane) run the epilogue.  The GatedMLP on the
+// Persistent CTAs walk the 128-row x 128-column output tiles: warp 0 streams K blocks of A and B with TMA through a stage
+// ring that runs on across tiles, warp 1 issues the MMAs into one of two TMEM accumulators, warps 2-9 (two threads per
+// output row = TMEM lane, half of the tile's columns each) run the epilogue of a tile while the next tile's copies and MMAs proceed.  The GatedMLP on the
 // link rows lives in k_link_mlp_tc.cu.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
 namespace lime {
 
-constexpr int GM_THREADS = 192, GM_MAX_STAGES = 6;
+constexpr int GM_THREADS = 64 + 256, GM_MAX_STAGES = 6;   // producer, MMA issuer, eight epilogue warps
 constexpr uint32_t GM_SUB = 128 * 128;    // [128 rows x 64 bf16]
 
 enum { GM_EPI_PREP = 0, GM_EPI_ROWS_T = 1 };
@@ -21,6 +22,7 @@ struct GemmParams {
   int64_t M;            // valid rows of A / C
   int kblocks;          // K / 64
   int stages;
+  int m_tiles, n_tiles; // output tiles of 128 rows x NT columns
   // PREP
   int ell, H, shared_rows;          // rows are (user, link): user = row / ell
   int d, f, plain_v;                // output widths; plain_v: the third segment is V[T] (d columns) instead of G2 | U2
@@ -41,30 +43,31 @@ template <int EPI, int NT>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
   using namespace tc;
-  extern __shared__ __align__(1024) uint8_t smem[];
-  if ((smem_u32(smem) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicCAS(p.err, 0, 92);
-    return;
-  }
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   constexpr uint32_t B_SUB = (uint32_t)NT * 128;
   constexpr uint32_t STAGE = GM_SUB + B_SUB;
   const int S = p.stages;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)S * STAGE);
   uint64_t* full = bars;
   uint64_t* empty = bars + GM_MAX_STAGES;
-  uint64_t* acc_full = bars + 2 * GM_MAX_STAGES;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * GM_MAX_STAGES + 1);
+  uint64_t* acc_full = bars + 2 * GM_MAX_STAGES;          // [2] accumulator of a tile complete
+  uint64_t* acc_empty = acc_full + 2;                      // [2] read out by the four epilogue warps
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.x * 128, nt = blockIdx.y;
+  // persistent: output tiles (m-tile, n-tile), n fastest, dealt round-robin to the CTAs; the stage ring and the two
+  // accumulators run on across tiles, so the copies and MMAs of the next tile overlap this tile's epilogue
+  const int n_tiles = p.m_tiles * p.n_tiles;
+  const int KB = p.kblocks;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    mbar_init(acc_full, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 8); }
     fence_barrier_init();
     prefetch_tmap(&tmA); prefetch_tmap(&tmB);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, NT); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, 2 * NT); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -74,41 +77,56 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     if (lane == 0) {
       const uint64_t pol = policy_evict_last();
       bool ok = true;
-      int kb = 0;
-      for (; kb < p.kblocks; ++kb) {
-        const int s = kb % S;
-        if (!mbar_wait(&empty[s], ((uint32_t)(kb / S) & 1u) ^ 1u, p.err, 71)) { ok = false; break; }
-        uint8_t* st = smem + (size_t)s * STAGE;
-        mbar_arrive_expect_tx(&full[s], STAGE);
-        tma_load_2d_hint(st, &tmA, kb * 64, m0, &full[s], pol);
-        tma_load_2d_hint(st + GM_SUB, &tmB, kb * 64, nt * NT, &full[s], pol);
+      int it = 0;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const int m0 = (t / p.n_tiles) * 128, nt = t % p.n_tiles;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % S;
+          if (!mbar_wait(&empty[s], ((uint32_t)(it / S) & 1u) ^ 1u, p.err, 71)) { ok = false; break; }
+          uint8_t* st = smem + (size_t)s * STAGE;
+          mbar_arrive_expect_tx(&full[s], STAGE);
+          tma_load_2d_hint(st, &tmA, kb * 64, m0, &full[s], pol);
+          tma_load_2d_hint(st + GM_SUB, &tmB, kb * 64, nt * NT, &full[s], pol);
+        }
       }
       if (!ok || *(volatile int*)p.err != 0)
-        for (int j = 0; j < kb && j < S; ++j) mbar_wait_quiet(&full[(kb - 1 - j) % S], (uint32_t)((kb - 1 - j) / S) & 1u);
+        for (int j = 0; j < it && j < S; ++j) mbar_wait_quiet(&full[(it - 1 - j) % S], (uint32_t)((it - 1 - j) / S) & 1u);
     }
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc_bf16(128, NT);
       const uint32_t sbase = smem_u32(smem);
       bool ok = true;
-      for (int kb = 0; kb < p.kblocks && ok; ++kb) {
-        const int s = kb % S;
-        if (!mbar_wait(&full[s], (uint32_t)(kb / S) & 1u, p.err, 72)) { ok = false; break; }
+      int it = 0, n = 0;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++n) {
+        const int buf = n & 1;
+        if (!mbar_wait(&acc_empty[buf], ((uint32_t)(n >> 1) & 1u) ^ 1u, p.err, 74)) { ok = false; break; }
         tc_fence_after();
+        for (int kb = 0; kb < KB && ok; ++kb, ++it) {
+          const int s = it % S;
+          if (!mbar_wait(&full[s], (uint32_t)(it / S) & 1u, p.err, 72)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          mma_bf16_ss(tmem_base, make_sdesc_k_sw128(sbase + s * STAGE + k * 32),
-                      make_sdesc_k_sw128(sbase + s * STAGE + GM_SUB + k * 32), idesc, (kb | k) != 0);
-        mma_commit(&empty[s]);
+          for (int k = 0; k < 4; ++k)
+            mma_bf16_ss(tmem_base + (uint32_t)buf * NT, make_sdesc_k_sw128(sbase + s * STAGE + k * 32),
+                        make_sdesc_k_sw128(sbase + s * STAGE + GM_SUB + k * 32), idesc, (kb | k) != 0);
+          mma_commit(&empty[s]);
+        }
+        if (ok) mma_commit(&acc_full[buf]);
       }
-      if (ok) mma_commit(acc_full);
     }
   } else {
     const int q = warp & 3;
     const int r = q * 32 + lane;
-    const int64_t row = (int64_t)m0 + r;
-    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-    if (mbar_wait(acc_full, 0, p.err, 73)) {
+    const int half = (warp - 2) >> 2;                  // which half of the tile's columns this warp reads out
+    const int cb = half * (NT / 2), ce = cb + NT / 2;
+    int n = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++n) {
+      const int buf = n & 1;
+      const int m0 = (t / p.n_tiles) * 128, nt = t % p.n_tiles;
+      const int64_t row = (int64_t)m0 + r;
+      const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * NT;
+      if (!mbar_wait(&acc_full[buf], (uint32_t)(n >> 1) & 1u, p.err, 73)) break;
       tc_fence_after();
       const bool valid = row < p.M;
       if (EPI == GM_EPI_PREP) {
@@ -120,9 +138,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         if (n0 < qk_cols) {
           const int seg = n0 / (p.H * p.d), h = (n0 / p.d) % p.H, i0 = n0 % p.d;
           __nv_bfloat16* dst = (seg == 0 ? p.Q2 : p.K2) + ((u * HL) + h * p.ell + l) * p.d + i0;
+          float* cs = seg == 0 ? p.cQ : p.cK;
           float rs = 0.f;
 #pragma unroll
-          for (int c = 0; c < 128; c += 16) {
+          for (int c = cb; c < ce; c += 16) {
             float v[16];
             tmem_ld_32x16(lane_addr + c, v);
             tmem_wait_ld();
@@ -136,8 +155,18 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
               *reinterpret_cast<uint4*>(dst + c + 8) = o1;
             }
           }
-          float* cs = seg == 0 ? p.cQ : p.cK;
-          if (valid && cs != nullptr) cs[u * HL + h * p.ell + l] = rs;
+          if (cs != nullptr && half == 0) {
+            // the row sum spans the whole tile: this warp also reads the other half's columns for it
+#pragma unroll
+            for (int c = ce; c < NT; c += 16) {
+              float v[16];
+              tmem_ld_32x16(lane_addr + c, v);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 16; ++j) rs += __bfloat162float(__float2bfloat16_rn(v[j]));
+            }
+            if (valid) cs[u * HL + h * p.ell + l] = rs;
+          }
         } else {
           // transposed stores: G2t / U2t [user][f][(h, l)], or V2t [user][d][l]
           __nv_bfloat16* dst;
@@ -152,7 +181,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
             ld = HL;
           }
 #pragma unroll
-          for (int c = 0; c < 128; c += 16) {
+          for (int c = cb; c < ce; c += 16) {
             float v[16];
             tmem_ld_32x16(lane_addr + c, v);
             tmem_wait_ld();
@@ -167,7 +196,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         const int l = (int)(row % p.group);
         __nv_bfloat16* dst = p.out_t + (u * p.n_cols + (int64_t)nt * NT) * p.group + l;
 #pragma unroll
-        for (int c = 0; c < NT; c += 16) {
+        for (int c = cb; c < ce; c += 16) {
           float v[16];
           tmem_ld_32x16(lane_addr + c, v);
           tmem_wait_ld();
@@ -178,6 +207,10 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
           }
         }
       }
+      // the accumulator has been read: the MMA issuer may reuse it for the tile after next
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
   }
 
@@ -185,7 +218,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, NT);
+    tmem_dealloc(tmem_base, 2 * NT);
   }
 }
 
@@ -198,12 +231,15 @@ static lime_status launch_gemm(const void* A, int64_t M, int K, const void* Bt, 
       !make_tmap_bf16_sw128(&tmB, Bt, (uint64_t)n_rows_b, (uint64_t)K, (uint64_t)K, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
   constexpr size_t stage = GM_SUB + (size_t)NT * 128;
-  p.M = M; p.kblocks = K / 64;
-  p.stages = p.kblocks < 4 ? p.kblocks : 4;
-  const size_t smem = p.stages * stage + 256;
+  const int64_t m_tiles = (M + 127) / 128;
+  if (m_tiles * n_tiles > 0x7fffffffLL) return LIME_UNSUPPORTED_SHAPE;
+  p.M = M; p.kblocks = K / 64; p.m_tiles = (int)m_tiles; p.n_tiles = n_tiles;
+  p.stages = GM_MAX_STAGES;
+  const size_t smem = p.stages * stage + 256 + 1024;
   LIME_CUDA(cudaFuncSetAttribute(k_gemm_tc<EPI, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   ProfScope _p(name, st);
-  dim3 grid((unsigned)((M + 127) / 128), (unsigned)n_tiles);
+  const int64_t tiles = m_tiles * n_tiles;
+  const unsigned grid = (unsigned)(tiles < kSMs ? tiles : kSMs);
   k_gemm_tc<EPI, NT><<<grid, GM_THREADS, smem, st>>>(tmA, tmB, p);
   LIME_LAUNCH_CHECK(name);
   return LIME_OK;
