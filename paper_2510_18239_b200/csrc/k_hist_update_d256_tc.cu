@@ -16,9 +16,10 @@
 //                                        S' (+)= U . W_o[hf rows, :]
 //   S' -> (LayerNorm) -> bf16 -> whole rows to global memory
 // TMEM (512 columns): [0, 256) two score buffers, later [gate | up] of one half; [256, 512) O, later S'.
-// Shared memory: X / O tile 64 KB, P / U / output staging 32 KB, the user's V[T]^T 32 KB, and a ring of 16 KB operand
-// slabs ([128 rows x 64 of the contraction index]) through which K2, W_g, W_u and W_o stream from L2 in the order the
-// MMA issuer consumes them (40 slabs per tile).
+// Shared memory: X / O tile 64 KB, P / U 32 KB, and a ring of seven 16 KB operand slabs ([128 rows x 64
+// of the contraction index]) through which K2, the link values of each group of two heads, W_g, W_u and W_o stream from
+// L2 in the order the MMA issuer consumes them (44 slabs per tile with 8 heads).  What bounds the kernel is how many
+// operand bytes are in flight from L2 per SM, so everything that is not the token tile or the P / U buffer is ring.
 // Warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 token rows: four threads per token (TMEM lane), a quarter of the
 // columns of every step each; the two threads that share a head of the softmax exchange (max, sum) once per group.
 #include "lime_common.cuh"
@@ -28,12 +29,11 @@ namespace lime {
 
 constexpr int HC_D = 256, HC_F = 256, HC_TILE = 128, HC_ELL = 64;
 constexpr int HC_PARTS = 4, HC_ROW_WARPS = 4 * HC_PARTS, HC_THREADS = 64 + 32 * HC_ROW_WARPS;
-constexpr int HC_RING = 5;
+constexpr int HC_RING = 7;
 constexpr uint32_t HC_SUB = 128 * 128;                          // bytes of one [128 rows x 64 bf16] swizzled sub-tile
 constexpr uint32_t HC_OFF_XO = 0;                               // token tile, later O: 4 K-blocks
-constexpr uint32_t HC_OFF_PU = HC_OFF_XO + 4 * HC_SUB;          // P_c, later U, later the output staging: 2 K-blocks
-constexpr uint32_t HC_OFF_V = HC_OFF_PU + 2 * HC_SUB;           // V[T]^T of the user: [256 features x 64 links]
-constexpr uint32_t HC_OFF_RING = HC_OFF_V + 2 * HC_SUB;
+constexpr uint32_t HC_OFF_PU = HC_OFF_XO + 4 * HC_SUB;          // P_c, later U: 2 K-blocks
+constexpr uint32_t HC_OFF_RING = HC_OFF_PU + 2 * HC_SUB;
 constexpr uint32_t HC_OFF_EXCH = HC_OFF_RING + HC_RING * HC_SUB;      // [2 parities][PARTS][128] float2
 constexpr uint32_t HC_OFF_BAR = HC_OFF_EXCH + 2 * HC_PARTS * 128 * 8;
 constexpr int HC_IDX_CAP = 1025;                                // users + 1 whose offsets are staged in shared memory
@@ -99,22 +99,21 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HC_OFF_BAR);
   uint64_t* full = bars;              // [HC_RING] operand slab landed
-  uint64_t* empty = bars + 5;         // [HC_RING] the MMAs that read the slab have run
-  uint64_t* x_full = bars + 10;       // per tile
-  uint64_t* x_free = bars + 11;       // per tile: the last contraction that reads the X / O buffer has run
-  uint64_t* v_full = bars + 12;       // per user change
-  uint64_t* s_full = bars + 13;       // [2] per group, by parity of the group counter: scores in TMEM
-  uint64_t* p_ready = bars + 15;      // per group: P_c in smem (16 warps)
-  uint64_t* pv_done = bars + 16;      // per group: value mix done (P buffer free)
-  uint64_t* o_full = bars + 17;       // per tile: O complete in TMEM
-  uint64_t* o_ready = bars + 18;      // per tile: O as bf16 in smem (16 warps)
-  uint64_t* gu_full = bars + 19;      // per (tile, half): [gate | up] complete
-  uint64_t* u_ready = bars + 20;      // per (tile, half): U in smem, [gate | up] read (16 warps)
-  uint64_t* sp_full = bars + 21;      // per tile: S' complete
-  uint64_t* sp_read = bars + 22;      // per tile: S' read out (16 warps)
-  uint64_t* all_bar = bars + 23;      // rendezvous of the 16 row warps
-  uint64_t* row_bar = bars + 24;      // [4] rendezvous of the four warps sharing a TMEM lane quarter
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 28);
+  uint64_t* empty = bars + 7;         // [HC_RING] the MMAs that read the slab have run
+  uint64_t* x_full = bars + 14;       // per tile
+  uint64_t* x_free = bars + 15;       // per tile: the last contraction that reads the X / O buffer has run
+  uint64_t* s_full = bars + 16;       // [2] per group, by parity of the group counter: scores in TMEM
+  uint64_t* p_ready = bars + 18;      // per group: P_c in smem (16 warps)
+  uint64_t* pv_done = bars + 19;      // per group: value mix done (P buffer free)
+  uint64_t* o_full = bars + 20;       // per tile: O complete in TMEM
+  uint64_t* o_ready = bars + 21;      // per tile: O as bf16 in smem (16 warps)
+  uint64_t* gu_full = bars + 22;      // per (tile, half): [gate | up] complete
+  uint64_t* u_ready = bars + 23;      // per (tile, half): U in smem, [gate | up] read (16 warps)
+  uint64_t* sp_full = bars + 24;      // per tile: S' complete
+  uint64_t* sp_read = bars + 25;      // per tile: S' read out (16 warps)
+  uint64_t* row_bar = bars + 27;      // [4] rendezvous of the four warps sharing a TMEM lane quarter
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 31);
+  static_assert(HC_RING == 7, "barrier table above");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_all = p.tile_start[p.B];
@@ -123,13 +122,16 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   const int n = t_end - t_begin;
   const int NG = p.NG;
   const int d_h = HC_D / p.H;
+  // link values of a group of two heads: 2 * d_h feature rows of V[T]^T, in slabs of up to 128 rows
+  const int v_rows = 2 * d_h < 128 ? 2 * d_h : 128;
+  const int v_slabs = (2 * d_h + 127) / 128;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < HC_RING; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    mbar_init(x_full, 1); mbar_init(x_free, 1); mbar_init(v_full, 1);
+    mbar_init(x_full, 1); mbar_init(x_free, 1);
     mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1); mbar_init(p_ready, HC_ROW_WARPS); mbar_init(pv_done, 1);
     mbar_init(o_full, 1); mbar_init(o_ready, HC_ROW_WARPS); mbar_init(gu_full, 1); mbar_init(u_ready, HC_ROW_WARPS);
-    mbar_init(sp_full, 1); mbar_init(sp_read, HC_ROW_WARPS); mbar_init(all_bar, HC_ROW_WARPS);
+    mbar_init(sp_full, 1); mbar_init(sp_read, HC_ROW_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], HC_PARTS);
     fence_barrier_init();
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmV); prefetch_tmap(&tmWgu); prefetch_tmap(&tmWo);
@@ -154,43 +156,42 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     if (lane == 0 && n > 0) {
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
       bool ok = true;
-      int g = 0, sl = 0, vn = 0, prev_user = -1;
-      auto slab = [&](const CUtensorMap* m, int x, int y) -> bool {
+      int g = 0, sl = 0;
+      auto slab_n = [&](const CUtensorMap* m, int x, int y, uint32_t bytes) -> bool {
         const int s = sl % HC_RING;
         if (!mbar_wait(&empty[s], ((uint32_t)(sl / HC_RING) & 1u) ^ 1u, p.err, 11)) return false;
-        mbar_arrive_expect_tx(&full[s], HC_SUB);
+        mbar_arrive_expect_tx(&full[s], bytes);
         tma_load_2d_hint(smem + HC_OFF_RING + s * HC_SUB, m, x, y, &full[s], pol_keep);
         ++sl;
         return true;
       };
+      auto slab = [&](const CUtensorMap* m, int x, int y) -> bool { return slab_n(m, x, y, HC_SUB); };
       HcTileUser tu;
       for (; g < n && ok; ++g) {
         const int t = t_begin + g;
         const int b = tu.of(tile_start, p.B, t);
         const int urow = p.shared ? 0 : b;
-        // Operand slabs go out in the order of use.  The first ring-load of this tile's K2 slabs is requested BEFORE the
-        // wait for the X / O buffer: the slabs only need free ring slots (which the previous tile's last contractions
-        // release one by one), so they travel while that tile is still being finished and stored.
-        int k2_done = 0;
-        for (; k2_done < HC_RING && k2_done < NG * 4 && ok; ++k2_done)
-          ok = slab(&tmK2, (k2_done & 3) * 64, urow * p.HL + (k2_done >> 2) * 128);
+        auto k2_group = [&](int c) {
+          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab(&tmK2, kb * 64, urow * p.HL + c * 128);
+        };
+        // Operand slabs go out in the order of use.  The first group's K2 slabs are requested BEFORE the wait for the
+        // X / O buffer: they only need free ring slots (which the previous tile's last contractions release one by one),
+        // so they travel while that tile is still being finished and stored.
+        k2_group(0);
         if (!ok) break;
-        // the X / O buffer and (on a change of user) the value buffer are free once the previous tile's last
-        // contraction over O has run: every MMA issued before it, the value mixes included, has then finished
+        // the X / O buffer is free once the previous tile's last contraction over O has run
         if (g > 0 && !mbar_wait(x_free, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
         const int row0 = off[b] + (t - tu.lo) * HC_TILE;
         mbar_arrive_expect_tx(x_full, 4 * HC_SUB);
         for (int kb = 0; kb < 4; ++kb) tma_load_2d_hint(smem + HC_OFF_XO + kb * HC_SUB, &tmX, kb * 64, row0, x_full, pol_stream);
-        if (p.shared ? (vn == 0) : (b != prev_user)) {
-          mbar_arrive_expect_tx(v_full, 2 * HC_SUB);
-          tma_load_2d_hint(smem + HC_OFF_V, &tmV, 0, urow * HC_D, v_full, pol_keep);
-          ++vn;
+        // per group: the next group's K2 (its scores are formed under this group's softmax), then this group's values
+        for (int c = 0; c < NG && ok; ++c) {
+          if (c + 1 < NG) k2_group(c + 1);
+          for (int j = 0; j < v_slabs && ok; ++j)
+            ok = slab_n(&tmV, 0, urow * HC_D + c * 2 * d_h + j * 128, (uint32_t)v_rows * 128u);
         }
-        prev_user = b;
-        // the rest: K2 of the remaining groups; then per half of the hidden columns the gate and up columns of
-        // W_g / W_u (contraction over d) and that half's rows of W_o (both halves of the output columns)
-        for (; k2_done < NG * 4 && ok; ++k2_done)
-          ok = slab(&tmK2, (k2_done & 3) * 64, urow * p.HL + (k2_done >> 2) * 128);
+        // then per half of the hidden columns the gate and up columns of W_g / W_u (contraction over d) and that half's
+        // rows of W_o (both halves of the output columns)
         for (int hf = 0; hf < 2 && ok; ++hf) {
           if (hf == 1) {
             for (int nh = 0; nh < 2 && ok; ++nh)
@@ -207,7 +208,6 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       if (!ok || *(volatile int*)p.err != 0) {
         // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
         if (g > 0 || sl > 0) mbar_wait_quiet(x_full, (uint32_t)(g < n ? g : n - 1) & 1u);
-        if (vn > 0) mbar_wait_quiet(v_full, (uint32_t)(vn - 1) & 1u);
         for (int j = 0; j < sl && j < HC_RING; ++j) mbar_wait_quiet(&full[(sl - 1 - j) % HC_RING], (uint32_t)((sl - 1 - j) / HC_RING) & 1u);
       }
     }
@@ -219,7 +219,7 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       const uint32_t sbase = smem_u32(smem);
       const uint32_t xo = sbase + HC_OFF_XO, pu = sbase + HC_OFF_PU;
       bool ok = true;
-      int sl = 0, q = 0, vn = 0, prev_user = -1;
+      int sl = 0, q = 0;
       // one operand slab (64 of the contraction index): D[128 x 128] (+)= A_kblock . slab^T
       auto slab_mma = [&](uint32_t d_col, uint32_t a_kblock, bool first) -> bool {
         const int s = sl % HC_RING;
@@ -239,15 +239,8 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         mma_commit(&s_full[qq & 1]);
         return true;
       };
-      HcTileUser tu;
       for (int g = 0; g < n && ok; ++g) {
-        const int b = tu.of(tile_start, p.B, t_begin + g);
         if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 23)) break;
-        if (p.shared ? (vn == 0) : (b != prev_user)) {
-          if (!mbar_wait(v_full, (uint32_t)vn & 1u, p.err, 28)) break;
-          ++vn;
-        }
-        prev_user = b;
         // 1. scores of the first group (both score buffers were last read as [gate | up] of the previous tile: u_ready waited)
         if (!issue_scores(q)) { ok = false; break; }
         for (int c = 0; c < NG && ok; ++c, ++q) {
@@ -255,14 +248,23 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
           if (!mbar_wait(p_ready, (uint32_t)q & 1u, p.err, 24)) { ok = false; break; }
           // the O columns last held S' of the previous tile
           if (c == 0 && g > 0 && !mbar_wait(sp_read, (uint32_t)(g - 1) & 1u, p.err, 26)) { ok = false; break; }
+          // the group's link values: one or two ring slabs
+          const int sv = sl;
+          for (int j = 0; j < v_slabs && ok; ++j)
+            ok = mbar_wait(&full[(sv + j) % HC_RING], (uint32_t)((sv + j) / HC_RING) & 1u, p.err, 28);
+          if (!ok) break;
           tc_fence_after();
           // 2. value mix, head by head: O[:, head] = P_head . V_head  (contraction over the 64 links of the head)
           for (int hl = 0; hl < 2; ++hl) {
             const int h = c * 2 + hl;
+            const int fo = hl * d_h;                         // the head's first feature row among the group's rows
+            const uint32_t vb = sbase + HC_OFF_RING + (uint32_t)((sv + fo / 128) % HC_RING) * HC_SUB + (uint32_t)(fo % 128) * 128u;
             for (int kk = 0; kk < 4; ++kk)
               mma_bf16_ss(tmem_base + COL_O + (uint32_t)(h * d_h), make_sdesc_k_sw128(pu + hl * HC_SUB + kk * 32),
-                          make_sdesc_k_sw128(sbase + HC_OFF_V + (uint32_t)(h * d_h) * 128 + kk * 32), idesc_v, kk != 0);
+                          make_sdesc_k_sw128(vb + kk * 32), idesc_v, kk != 0);
           }
+          for (int j = 0; j < v_slabs; ++j) mma_commit(&empty[(sv + j) % HC_RING]);
+          sl += v_slabs;
           mma_commit(pv_done);
           if (c == NG - 1) mma_commit(o_full);
         }
@@ -302,7 +304,7 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     float2* exch = reinterpret_cast<float2*>(smem + HC_OFF_EXCH);         // [2][PARTS][128]
     uint8_t* pu_part = smem + HC_OFF_PU + (part >> 1) * HC_SUB;           // K-block part / 2, chunks (part % 2) * 4 ..
     const uint32_t pu_chunk0 = (uint32_t)(part & 1) * 4;
-    uint32_t row_uses = 0, all_uses = 0;
+    uint32_t row_uses = 0;
     int q = 0;
     bool ok = true;
     HcTileUser tu;
@@ -405,17 +407,21 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (lane == 0) mbar_arrive(u_ready);
       }
       if (!ok) break;
-      // ---- S': this thread's 64 columns of its row -> (LayerNorm) -> bf16 -> staged -> whole rows to global
+      // ---- S': this thread's 64 columns of its row -> (LayerNorm) -> bf16 -> global, straight from registers
       if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 37)) { ok = false; break; }
       tc_fence_after();
+      float a0[32], a1[32];
+      tmem_ld_32x32(lane_addr + COL_SP + part * 64, a0);
+      tmem_ld_32x32(lane_addr + COL_SP + part * 64 + 32, a1);
+      tmem_wait_ld();
+      // S' is in registers: the columns may take the next tile's value mix while this tile is normalised and stored
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sp_read);
       float mu = 0.f, rstd = 1.f;
       if (p.out_ln) {
         // each quarter sends the mean of its 64 columns and their squared deviations from it; the four combine exactly
         float s = 0.f;
-        float a0[32], a1[32];
-        tmem_ld_32x32(lane_addr + COL_SP + part * 64, a0);
-        tmem_ld_32x32(lane_addr + COL_SP + part * 64 + 32, a1);
-        tmem_wait_ld();
 #pragma unroll
         for (int j = 0; j < 32; ++j) s += a0[j] + a1[j];
         const float m_q = s * (1.0f / 64);
@@ -438,44 +444,40 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         for (int i = 0; i < HC_PARTS; ++i) { const float dm = e[i].x - mu; tot += e[i].y + 64.0f * dm * dm; }
         rstd = rsqrtf(tot * (1.0f / HC_D) + p.ln_eps);
       }
-      // Two rounds through the 32 KB P / U buffer (free: S' has consumed U): the threads of the round's two quarters stage
-      // their 64 columns (row r at r * 256 bytes, 16-byte chunk c at position c ^ (r & 15) to spread the banks), then
-      // every warp writes 256-byte half rows.
-      const int row_end = off[b + 1];
-      uint8_t* stage = smem + HC_OFF_PU;
-      for (int round = 0; round < 2 && ok; ++round) {
-        if ((part >> 1) == round) {
+      // Out through a 2 KB patch of the P / U buffer that belongs to this warp alone (S' has consumed U): the warp stages
+      // 32 columns of its 32 rows (row R at R * 64 bytes, 16-byte chunk c at position c ^ ((R >> 1) & 3): conflict-free
+      // both ways), then writes them with four lanes per row, 64 contiguous bytes each.  Only the warp itself has to
+      // rendezvous; the patch lies inside the rows of the P / U buffer that this warp and its column neighbour write.
+      {
+        uint8_t* patch = smem + HC_OFF_PU + (part >> 1) * HC_SUB + q4 * 4096 + (part & 1) * 2048;
+        const int row_end = off[b + 1];
+        const uint32_t rr = (uint32_t)lane >> 2, rc = (uint32_t)lane & 3u;
 #pragma unroll
-          for (int c = 0; c < 64; c += 32) {
-            float a[32];
-            tmem_ld_32x32(lane_addr + COL_SP + part * 64 + c, a);
-            tmem_wait_ld();
+        for (int hcol = 0; hcol < 2; ++hcol) {
+          const float* a = hcol ? a1 : a0;
 #pragma unroll
-            for (int c8 = 0; c8 < 4; ++c8) {
-              uint4 o;
-              o.x = hc_pack((a[c8 * 8 + 0] - mu) * rstd, (a[c8 * 8 + 1] - mu) * rstd);
-              o.y = hc_pack((a[c8 * 8 + 2] - mu) * rstd, (a[c8 * 8 + 3] - mu) * rstd);
-              o.z = hc_pack((a[c8 * 8 + 4] - mu) * rstd, (a[c8 * 8 + 5] - mu) * rstd);
-              o.w = hc_pack((a[c8 * 8 + 6] - mu) * rstd, (a[c8 * 8 + 7] - mu) * rstd);
-              const uint32_t ch = (uint32_t)(part & 1) * 8 + (uint32_t)(c >> 3) + c8;
-              *reinterpret_cast<uint4*>(stage + r * 256u + ((ch ^ (r & 15u)) << 4)) = o;
-            }
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint4 o;
+            o.x = hc_pack((a[c8 * 8 + 0] - mu) * rstd, (a[c8 * 8 + 1] - mu) * rstd);
+            o.y = hc_pack((a[c8 * 8 + 2] - mu) * rstd, (a[c8 * 8 + 3] - mu) * rstd);
+            o.z = hc_pack((a[c8 * 8 + 4] - mu) * rstd, (a[c8 * 8 + 5] - mu) * rstd);
+            o.w = hc_pack((a[c8 * 8 + 6] - mu) * rstd, (a[c8 * 8 + 7] - mu) * rstd);
+            *reinterpret_cast<uint4*>(patch + lane * 64 + (((uint32_t)c8 ^ (((uint32_t)lane >> 1) & 3u)) << 4)) = o;
           }
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t R = (uint32_t)i * 8 + rr;
+            const uint4 o = *reinterpret_cast<const uint4*>(patch + R * 64 + ((rc ^ ((R >> 1) & 3u)) << 4));
+            const int grow = row0 + q4 * 32 + (int)R;
+            if (grow < row_end)
+              *reinterpret_cast<uint4*>(p.out + (int64_t)grow * HC_D + part * 64 + hcol * 32 + rc * 8) = o;
+          }
+          __syncwarp();
         }
-        if (!hc_group_sync(all_bar, all_uses, lane, p.err, 39)) { ok = false; break; }
-#pragma unroll 4
-        for (int i = rw; i < HC_TILE; i += HC_ROW_WARPS) {
-          if (row0 + i >= row_end) break;
-          const uint2 o = *reinterpret_cast<const uint2*>(stage + i * 256 + ((((uint32_t)lane >> 1) ^ ((uint32_t)i & 15u)) << 4) + (lane & 1) * 8);
-          *reinterpret_cast<uint2*>(p.out + (int64_t)(row0 + i) * HC_D + round * 128 + lane * 4) = o;
-        }
-        // the buffer is rewritten next (second round, or the next tile's first P): every warp must have copied its rows out
-        if (!hc_group_sync(all_bar, all_uses, lane, p.err, 40)) { ok = false; break; }
       }
-      if (!ok) break;
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(sp_read);
+      // without the softmax exchange nothing else keeps the column neighbour from writing the next P over this patch
+      if (p.silu && !hc_group_sync(&row_bar[q4], row_uses, lane, p.err, 39)) { ok = false; break; }
     }
   }
 
@@ -497,9 +499,10 @@ lime_status launch_hist_update_d256_tc(const HistUpdate256Args& a, cudaStream_t 
   const int HL = a.H * HC_ELL;
   CUtensorMap tmX, tmK2, tmV, tmWgu, tmWo;
   const uint64_t users = a.shared ? 1 : (uint64_t)a.B;
+  const int v_rows = 2 * (HC_D / a.H) < 128 ? 2 * (HC_D / a.H) : 128;      // value rows of one slab: a group of two heads
   if (!make_tmap_bf16_sw128(&tmX, a.hist_in, (uint64_t)a.total, HC_D, HC_D, HC_TILE) ||
       !make_tmap_bf16_sw128(&tmK2, a.K2, users * HL, HC_D, HC_D, 128) ||
-      !make_tmap_bf16_sw128(&tmV, a.V2t, users * HC_D, HC_ELL, HC_ELL, 256) ||
+      !make_tmap_bf16_sw128(&tmV, a.V2t, users * HC_D, HC_ELL, HC_ELL, v_rows) ||
       !make_tmap_bf16_sw128(&tmWgu, a.WguT, 2 * HC_F, HC_D, HC_D, 128) ||
       !make_tmap_bf16_sw128(&tmWo, a.WoT, HC_D, HC_F, HC_F, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
