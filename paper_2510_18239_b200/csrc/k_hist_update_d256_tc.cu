@@ -8,20 +8,25 @@
 // (k_link_prep.cu: Q[S] is never formed), the value mix is done head by head against the plain link values V[T], and
 // the GatedMLP weights follow unfolded - at this width folding W_V W_g into the link side (as the d = 128 kernels do)
 // would cost twice the tensor work and twice the operand traffic:
-//   per group c of 128 stacked (head, link) rows = 2 heads:
-//     scores_c [128 x 128] = X . K2_c^T            -> per-head softmax over the 64 links (or SiLU(s) / 64) -> P_c (bf16)
-//     O[:, head]           = P_head [128 x 64] . V_head [64 x d_h]          (both heads of the group)
-//   O -> bf16 (over the X tile, which nothing reads any more)
+//   scores [128 x H*64] = X . K2^T, 256 stacked (head, link) rows = four heads per contraction
+//   per group c of two heads: per-head softmax over the 64 links, unnormalised (or SiLU(s) / 64) -> P_c (bf16);
+//                             O[:, head] = P_head [128 x 64] . V_head [64 x d_h]
+//   O * 1 / (row sum of the head) -> bf16
 //   per half hf of the hidden columns:   [gate | up] = O . [W_g | W_u][:, hf]  ->  U = SiLU(gate) * up (bf16)
 //                                        S' (+)= U . W_o[hf rows, :]
-//   S' -> (LayerNorm) -> bf16 -> whole rows to global memory
-// TMEM (512 columns): [0, 256) two score buffers, later [gate | up] of one half; [256, 512) O, later S'.
-// Shared memory: X / O tile 64 KB, P / U 32 KB, and a ring of seven 16 KB operand slabs ([128 rows x 64
-// of the contraction index]) through which K2, the link values of each group of two heads, W_g, W_u and W_o stream from
-// L2 in the order the MMA issuer consumes them (44 slabs per tile with 8 heads).  What bounds the kernel is how many
-// operand bytes are in flight from L2 per SM, so everything that is not the token tile or the P / U buffer is ring.
-// Warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 token rows: four threads per token (TMEM lane), a quarter of the
-// columns of every step each; the two threads that share a head of the softmax exchange (max, sum) once per group.
+//   S' -> (LayerNorm) -> bf16 -> global memory
+// Every contraction but the value mix is issued 256 columns wide: at 128 columns an MMA re-reads its A operand from
+// shared memory twice as often per flop, and shared-memory bandwidth (operands in, TMA writes, the row warps) is what
+// the tensor pipe waits for here.
+// TMEM (512 columns) as two regions that swap roles every tile.  R0: scores of heads 0-3, overwritten head by head by
+// O as its scores are consumed, later S'.  R1: scores of heads 4-7, later [gate | up] of one half.  The next tile's
+// R0 is this tile's R1, which is free before S' is even complete.
+// Shared memory: X tile 64 KB (dead once the scores are formed: then the two P buffers, then O); V[T]^T of the user, later
+// U, later the patches S' leaves through, 32 KB; a ring of three 32 KB operand slabs ([256 rows x 64 of the contraction
+// index]) through which K2, [W_g | W_u] and W_o stream from L2 in the order the MMA issuer consumes them.
+// Warp 0 TMA producer, warp 1 MMA issuer, warps 2-17 token rows.  For the softmax the row warps form two groups that
+// take alternate groups of two heads, one thread per (token, head): no exchange between threads, and one group's
+// exponentials overlap the other group's value mix.  Elsewhere four threads share a token, a quarter of the columns each.
 #include "lime_common.cuh"
 #include "tc_common.cuh"
 
@@ -29,13 +34,15 @@ namespace lime {
 
 constexpr int HC_D = 256, HC_F = 256, HC_TILE = 128, HC_ELL = 64;
 constexpr int HC_PARTS = 4, HC_ROW_WARPS = 4 * HC_PARTS, HC_THREADS = 64 + 32 * HC_ROW_WARPS;
-constexpr int HC_RING = 7;
+constexpr int HC_RING = 3;
 constexpr uint32_t HC_SUB = 128 * 128;                          // bytes of one [128 rows x 64 bf16] swizzled sub-tile
-constexpr uint32_t HC_OFF_XO = 0;                               // token tile, later O: 4 K-blocks
-constexpr uint32_t HC_OFF_PU = HC_OFF_XO + 4 * HC_SUB;          // P_c, later U: 2 K-blocks
+constexpr uint32_t HC_SLAB = 2 * HC_SUB;                        // one ring slot: [256 rows x 64 bf16]
+constexpr uint32_t HC_OFF_XO = 0;                               // token tile, then P of two groups, then O: 4 K-blocks
+constexpr uint32_t HC_OFF_PU = HC_OFF_XO + 4 * HC_SUB;          // V[T]^T [256 features x 64 links], later U: 2 K-blocks
 constexpr uint32_t HC_OFF_RING = HC_OFF_PU + 2 * HC_SUB;
-constexpr uint32_t HC_OFF_EXCH = HC_OFF_RING + HC_RING * HC_SUB;      // [2 parities][PARTS][128] float2
-constexpr uint32_t HC_OFF_BAR = HC_OFF_EXCH + 2 * HC_PARTS * 128 * 8;
+constexpr uint32_t HC_OFF_EXCH = HC_OFF_RING + HC_RING * HC_SLAB;     // [2 parities][PARTS][128] float2
+constexpr uint32_t HC_OFF_INV = HC_OFF_EXCH + 2 * HC_PARTS * 128 * 8; // [8 heads][128 rows] 1 / softmax row sum
+constexpr uint32_t HC_OFF_BAR = HC_OFF_INV + 8 * 128 * 4;
 constexpr int HC_IDX_CAP = 1025;                                // users + 1 whose offsets are staged in shared memory
 constexpr uint32_t HC_OFF_IDX = HC_OFF_BAR + 512;
 constexpr uint32_t HC_SMEM = HC_OFF_IDX + 2 * HC_IDX_CAP * 4 + 8;
@@ -99,37 +106,38 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + HC_OFF_BAR);
   uint64_t* full = bars;              // [HC_RING] operand slab landed
-  uint64_t* empty = bars + 7;         // [HC_RING] the MMAs that read the slab have run
-  uint64_t* x_full = bars + 14;       // per tile
-  uint64_t* x_free = bars + 15;       // per tile: the last contraction that reads the X / O buffer has run
-  uint64_t* s_full = bars + 16;       // [2] per group, by parity of the group counter: scores in TMEM
-  uint64_t* p_ready = bars + 18;      // per group: P_c in smem (16 warps)
-  uint64_t* pv_done = bars + 19;      // per group: value mix done (P buffer free)
-  uint64_t* o_full = bars + 20;       // per tile: O complete in TMEM
-  uint64_t* o_ready = bars + 21;      // per tile: O as bf16 in smem (16 warps)
-  uint64_t* gu_full = bars + 22;      // per (tile, half): [gate | up] complete
-  uint64_t* u_ready = bars + 23;      // per (tile, half): U in smem, [gate | up] read (16 warps)
-  uint64_t* sp_full = bars + 24;      // per tile: S' complete
-  uint64_t* sp_read = bars + 25;      // per tile: S' read out (16 warps)
-  uint64_t* row_bar = bars + 27;      // [4] rendezvous of the four warps sharing a TMEM lane quarter
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 31);
-  static_assert(HC_RING == 7, "barrier table above");
+  uint64_t* empty = bars + 3;         // [HC_RING] the MMAs that read the slab have run
+  uint64_t* x_full = bars + 6;        // per tile
+  uint64_t* x_free = bars + 7;        // per tile: the last contraction that reads the X / P / O buffer has run
+  uint64_t* v_full = bars + 8;        // per tile: V[T]^T of the tile's user landed
+  uint64_t* pu_free = bars + 9;       // per tile: every row warp is done with its patch of the V / U buffer (16 warps)
+  uint64_t* s_full = bars + 10;       // [2] per tile: scores of heads 0-3 / 4-7 in TMEM
+  uint64_t* p_ready = bars + 12;      // [2] per group, by row-warp group: P_c in smem (8 warps)
+  uint64_t* pv_done = bars + 14;      // [2] per group: value mix done (that P buffer free)
+  uint64_t* o_full = bars + 16;       // per tile: O complete in TMEM
+  uint64_t* o_ready = bars + 17;      // per tile: O as bf16 in smem (16 warps)
+  uint64_t* gu_full = bars + 18;      // per (tile, half): [gate | up] complete
+  uint64_t* u_ready = bars + 19;      // per (tile, half): U in smem, [gate | up] read (16 warps)
+  uint64_t* sp_full = bars + 20;      // per tile: S' complete
+  uint64_t* sp_read = bars + 21;      // per tile: S' read out of TMEM (16 warps)
+  uint64_t* row_bar = bars + 22;      // [4] rendezvous of the four warps sharing a TMEM lane quarter
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 26);
+  static_assert(HC_RING == 3, "barrier table above");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles_all = p.tile_start[p.B];
   const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
   const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
   const int n = t_end - t_begin;
-  const int NG = p.NG;
+  const int NG = p.NG;                                       // groups of two heads
   const int d_h = HC_D / p.H;
-  // link values of a group of two heads: 2 * d_h feature rows of V[T]^T, in slabs of up to 128 rows
-  const int v_rows = 2 * d_h < 128 ? 2 * d_h : 128;
-  const int v_slabs = (2 * d_h + 127) / 128;
+  const int n_sg = (p.HL + 255) / 256;                       // score contractions per tile (four heads each)
+  const int sc_boxes = p.HL >= 256 ? 2 : 1;                  // 128-row boxes of K2 per score slab
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < HC_RING; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    mbar_init(x_full, 1); mbar_init(x_free, 1);
-    mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1); mbar_init(p_ready, HC_ROW_WARPS); mbar_init(pv_done, 1);
+    mbar_init(x_full, 1); mbar_init(x_free, 1); mbar_init(v_full, 1); mbar_init(pu_free, HC_ROW_WARPS);
+    for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], HC_ROW_WARPS / 2); mbar_init(&pv_done[i], 1); }
     mbar_init(o_full, 1); mbar_init(o_ready, HC_ROW_WARPS); mbar_init(gu_full, 1); mbar_init(u_ready, HC_ROW_WARPS);
     mbar_init(sp_full, 1); mbar_init(sp_read, HC_ROW_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], HC_PARTS);
@@ -149,7 +157,6 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_SC = 0, COL_GU = 0, COL_O = 256, COL_SP = 256;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -157,130 +164,127 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
       bool ok = true;
       int g = 0, sl = 0;
-      auto slab_n = [&](const CUtensorMap* m, int x, int y, uint32_t bytes) -> bool {
+      bool v_sent = false;
+      // one ring slab: one or two boxes of 128 rows at contraction offset x
+      auto slab = [&](const CUtensorMap* m, int x, int y0, int y1, int boxes) -> bool {
         const int s = sl % HC_RING;
         if (!mbar_wait(&empty[s], ((uint32_t)(sl / HC_RING) & 1u) ^ 1u, p.err, 11)) return false;
-        mbar_arrive_expect_tx(&full[s], bytes);
-        tma_load_2d_hint(smem + HC_OFF_RING + s * HC_SUB, m, x, y, &full[s], pol_keep);
+        mbar_arrive_expect_tx(&full[s], (uint32_t)boxes * HC_SUB);
+        tma_load_2d_hint(smem + HC_OFF_RING + s * HC_SLAB, m, x, y0, &full[s], pol_keep);
+        if (boxes == 2) tma_load_2d_hint(smem + HC_OFF_RING + s * HC_SLAB + HC_SUB, m, x, y1, &full[s], pol_keep);
         ++sl;
         return true;
       };
-      auto slab = [&](const CUtensorMap* m, int x, int y) -> bool { return slab_n(m, x, y, HC_SUB); };
       HcTileUser tu;
       for (; g < n && ok; ++g) {
         const int t = t_begin + g;
         const int b = tu.of(tile_start, p.B, t);
         const int urow = p.shared ? 0 : b;
-        auto k2_group = [&](int c) {
-          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab(&tmK2, kb * 64, urow * p.HL + c * 128);
+        auto k2_slab = [&](int sg, int kb) -> bool {
+          const int y = urow * p.HL + sg * 256;
+          return slab(&tmK2, kb * 64, y, y + 128, sc_boxes);
         };
-        // Operand slabs go out in the order of use.  The first group's K2 slabs are requested BEFORE the wait for the
-        // X / O buffer: they only need free ring slots (which the previous tile's last contractions release one by one),
-        // so they travel while that tile is still being finished and stored.
-        k2_group(0);
+        // Operand slabs go out in the order of use.  The first K2 slab is requested BEFORE the wait for the X buffer: it
+        // only needs a free ring slot, so it travels while the previous tile is still being finished.
+        ok = k2_slab(0, 0);
         if (!ok) break;
-        // the X / O buffer is free once the previous tile's last contraction over O has run
+        // the X / P / O buffer is free once the previous tile's last contraction over O has run
         if (g > 0 && !mbar_wait(x_free, (uint32_t)(g - 1) & 1u, p.err, 12)) { ok = false; break; }
         const int row0 = off[b] + (t - tu.lo) * HC_TILE;
         mbar_arrive_expect_tx(x_full, 4 * HC_SUB);
         for (int kb = 0; kb < 4; ++kb) tma_load_2d_hint(smem + HC_OFF_XO + kb * HC_SUB, &tmX, kb * 64, row0, x_full, pol_stream);
-        // per group: the next group's K2 (its scores are formed under this group's softmax), then this group's values
-        for (int c = 0; c < NG && ok; ++c) {
-          if (c + 1 < NG) k2_group(c + 1);
-          for (int j = 0; j < v_slabs && ok; ++j)
-            ok = slab_n(&tmV, 0, urow * HC_D + c * 2 * d_h + j * 128, (uint32_t)v_rows * 128u);
-        }
+        for (int kb = 1; kb < 4 && ok; ++kb) ok = k2_slab(0, kb);
+        for (int sg = 1; sg < n_sg && ok; ++sg)
+          for (int kb = 0; kb < 4 && ok; ++kb) ok = k2_slab(sg, kb);
+        if (!ok) break;
+        // the user's link values go where U of the previous tile was and where its rows left through
+        if (g > 0 && !mbar_wait(pu_free, (uint32_t)(g - 1) & 1u, p.err, 13)) { ok = false; break; }
+        mbar_arrive_expect_tx(v_full, 2 * HC_SUB);
+        tma_load_2d_hint(smem + HC_OFF_PU, &tmV, 0, urow * HC_D, v_full, pol_keep);
+        v_sent = true;
         // then per half of the hidden columns the gate and up columns of W_g / W_u (contraction over d) and that half's
-        // rows of W_o (both halves of the output columns)
+        // rows of W_o (all output columns)
         for (int hf = 0; hf < 2 && ok; ++hf) {
-          if (hf == 1) {
-            for (int nh = 0; nh < 2 && ok; ++nh)
-              for (int kb = 0; kb < 2 && ok; ++kb) ok = slab(&tmWo, kb * 64, nh * 128);            // S'(0): hidden columns 0..127
-          }
-          for (int kb = 0; kb < 4 && ok; ++kb) {
-            ok = slab(&tmWgu, kb * 64, hf * 128);
-            ok = ok && slab(&tmWgu, kb * 64, HC_F + hf * 128);
-          }
+          if (hf == 1)
+            for (int kb = 0; kb < 2 && ok; ++kb) ok = slab(&tmWo, kb * 64, 0, 128, 2);             // S'(0): hidden columns 0..127
+          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab(&tmWgu, kb * 64, hf * 128, HC_F + hf * 128, 2);
         }
-        for (int nh = 0; nh < 2 && ok; ++nh)
-          for (int kb = 0; kb < 2 && ok; ++kb) ok = slab(&tmWo, 128 + kb * 64, nh * 128);          // S'(1): hidden columns 128..255
+        for (int kb = 0; kb < 2 && ok; ++kb) ok = slab(&tmWo, 128 + kb * 64, 0, 128, 2);           // S'(1): hidden columns 128..255
       }
       if (!ok || *(volatile int*)p.err != 0) {
         // giving up: let the copies already issued land (bounded) before this CTA's shared memory goes away
-        if (g > 0 || sl > 0) mbar_wait_quiet(x_full, (uint32_t)(g < n ? g : n - 1) & 1u);
+        const int gl = g < n ? g : n - 1;
+        if (g > 0 || sl > 0) mbar_wait_quiet(x_full, (uint32_t)gl & 1u);
+        if (v_sent) mbar_wait_quiet(v_full, (uint32_t)gl & 1u);
         for (int j = 0; j < sl && j < HC_RING; ++j) mbar_wait_quiet(&full[(sl - 1 - j) % HC_RING], (uint32_t)((sl - 1 - j) / HC_RING) & 1u);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && n > 0) {
-      constexpr uint32_t idesc_128 = make_idesc_bf16(128, 128);
+      constexpr uint32_t idesc_256 = make_idesc_bf16(128, 256);
+      const uint32_t idesc_sc = p.HL >= 256 ? idesc_256 : make_idesc_bf16(128, 128);
       const uint32_t idesc_v = make_idesc_bf16(128, d_h);
       const uint32_t sbase = smem_u32(smem);
       const uint32_t xo = sbase + HC_OFF_XO, pu = sbase + HC_OFF_PU;
       bool ok = true;
-      int sl = 0, q = 0;
-      // one operand slab (64 of the contraction index): D[128 x 128] (+)= A_kblock . slab^T
-      auto slab_mma = [&](uint32_t d_col, uint32_t a_kblock, bool first) -> bool {
+      int sl = 0;
+      uint32_t p_uses[2] = {0u, 0u};
+      // one operand slab (64 of the contraction index): D[128 x N] (+)= A_kblock . slab^T
+      auto slab_mma = [&](uint32_t d_col, uint32_t a_kblock, uint32_t idesc, bool first) -> bool {
         const int s = sl % HC_RING;
         if (!mbar_wait(&full[s], (uint32_t)(sl / HC_RING) & 1u, p.err, 22)) return false;
         tc_fence_after();
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-          mma_bf16_ss(tmem_base + d_col, make_sdesc_k_sw128(a_kblock + k * 32), make_sdesc_k_sw128(sbase + HC_OFF_RING + s * HC_SUB + k * 32),
-                      idesc_128, (first && k == 0) ? 0u : 1u);
+          mma_bf16_ss(tmem_base + d_col, make_sdesc_k_sw128(a_kblock + k * 32), make_sdesc_k_sw128(sbase + HC_OFF_RING + s * HC_SLAB + k * 32),
+                      idesc, (first && k == 0) ? 0u : 1u);
         mma_commit(&empty[s]);
         ++sl;
         return true;
       };
-      auto issue_scores = [&](int qq) -> bool {
-        for (int kb = 0; kb < 4; ++kb)
-          if (!slab_mma(COL_SC + (uint32_t)(qq & 1) * 128, xo + kb * HC_SUB, kb == 0)) return false;
-        mma_commit(&s_full[qq & 1]);
-        return true;
-      };
       for (int g = 0; g < n && ok; ++g) {
+        const uint32_t R0 = (uint32_t)(g & 1) * 256u, R1 = 256u - R0;
         if (!mbar_wait(x_full, (uint32_t)g & 1u, p.err, 23)) break;
-        // 1. scores of the first group (both score buffers were last read as [gate | up] of the previous tile: u_ready waited)
-        if (!issue_scores(q)) { ok = false; break; }
-        for (int c = 0; c < NG && ok; ++c, ++q) {
-          if (c + 1 < NG && !issue_scores(q + 1)) { ok = false; break; }
-          if (!mbar_wait(p_ready, (uint32_t)q & 1u, p.err, 24)) { ok = false; break; }
-          // the O columns last held S' of the previous tile
-          if (c == 0 && g > 0 && !mbar_wait(sp_read, (uint32_t)(g - 1) & 1u, p.err, 26)) { ok = false; break; }
-          // the group's link values: one or two ring slabs
-          const int sv = sl;
-          for (int j = 0; j < v_slabs && ok; ++j)
-            ok = mbar_wait(&full[(sv + j) % HC_RING], (uint32_t)((sv + j) / HC_RING) & 1u, p.err, 28);
+        // 1. scores.  R0 was [gate | up] of the previous tile (u_ready waited); R1 was its S'.
+        for (int kb = 0; kb < 4 && ok; ++kb) ok = slab_mma(R0, xo + kb * HC_SUB, idesc_sc, kb == 0);
+        if (!ok) break;
+        mma_commit(&s_full[0]);
+        if (g > 0 && !mbar_wait(sp_read, (uint32_t)(g - 1) & 1u, p.err, 26)) break;
+        tc_fence_after();
+        if (n_sg == 2) {
+          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab_mma(R1, xo + kb * HC_SUB, idesc_256, kb == 0);
           if (!ok) break;
+          mma_commit(&s_full[1]);
+        }
+        if (!mbar_wait(v_full, (uint32_t)g & 1u, p.err, 28)) break;
+        // 2. value mix, head by head: O[:, head] = P_head . V_head  (contraction over the 64 links of the head).  The O
+        //    columns of group c lie inside score columns that groups <= c / 2 held, all consumed once P_c exists and the
+        //    groups are taken in order.
+        for (int c = 0; c < NG && ok; ++c) {
+          const int rg = c & 1;
+          if (!mbar_wait(&p_ready[rg], p_uses[rg] & 1u, p.err, 24)) { ok = false; break; }
+          ++p_uses[rg];
           tc_fence_after();
-          // 2. value mix, head by head: O[:, head] = P_head . V_head  (contraction over the 64 links of the head)
           for (int hl = 0; hl < 2; ++hl) {
             const int h = c * 2 + hl;
-            const int fo = hl * d_h;                         // the head's first feature row among the group's rows
-            const uint32_t vb = sbase + HC_OFF_RING + (uint32_t)((sv + fo / 128) % HC_RING) * HC_SUB + (uint32_t)(fo % 128) * 128u;
             for (int kk = 0; kk < 4; ++kk)
-              mma_bf16_ss(tmem_base + COL_O + (uint32_t)(h * d_h), make_sdesc_k_sw128(pu + hl * HC_SUB + kk * 32),
-                          make_sdesc_k_sw128(vb + kk * 32), idesc_v, kk != 0);
+              mma_bf16_ss(tmem_base + R0 + (uint32_t)(h * d_h), make_sdesc_k_sw128(xo + (uint32_t)(rg * 2 + hl) * HC_SUB + kk * 32),
+                          make_sdesc_k_sw128(pu + (uint32_t)(h * d_h) * 128 + kk * 32), idesc_v, kk != 0);
           }
-          for (int j = 0; j < v_slabs; ++j) mma_commit(&empty[(sv + j) % HC_RING]);
-          sl += v_slabs;
-          mma_commit(pv_done);
+          mma_commit(&pv_done[rg]);
           if (c == NG - 1) mma_commit(o_full);
         }
         if (!ok) break;
-        // 3. GatedMLP on O (bf16 in the X / O buffer), the hidden columns in two halves
+        // 3. GatedMLP on O (bf16 in the X / P / O buffer), the hidden columns in two halves
         if (!mbar_wait(o_ready, (uint32_t)g & 1u, p.err, 25)) break;
+        tc_fence_after();
         for (int hf = 0; hf < 2 && ok; ++hf) {
           if (hf == 1) {
             // S' = U(0) . W_o[0..127, :] first: it frees the U buffer for the second half
-            for (int nh = 0; nh < 2 && ok; ++nh)
-              for (int kb = 0; kb < 2 && ok; ++kb) ok = slab_mma(COL_SP + (uint32_t)nh * 128, pu + kb * HC_SUB, kb == 0);
+            for (int kb = 0; kb < 2 && ok; ++kb) ok = slab_mma(R0, pu + kb * HC_SUB, idesc_256, kb == 0);
           }
-          for (int kb = 0; kb < 4 && ok; ++kb) {
-            ok = slab_mma(COL_GU, xo + kb * HC_SUB, kb == 0);
-            ok = ok && slab_mma(COL_GU + 128, xo + kb * HC_SUB, kb == 0);
-          }
+          for (int kb = 0; kb < 4 && ok; ++kb) ok = slab_mma(R1, xo + kb * HC_SUB, idesc_256, kb == 0);
           if (!ok) break;
           mma_commit(gu_full);
           if (hf == 1) mma_commit(x_free);
@@ -288,8 +292,7 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
           tc_fence_after();
         }
         if (!ok) break;
-        for (int nh = 0; nh < 2 && ok; ++nh)
-          for (int kb = 0; kb < 2 && ok; ++kb) ok = slab_mma(COL_SP + (uint32_t)nh * 128, pu + kb * HC_SUB, false);
+        for (int kb = 0; kb < 2 && ok; ++kb) ok = slab_mma(R0, pu + kb * HC_SUB, idesc_256, false);
         if (!ok) break;
         mma_commit(sp_full);
       }
@@ -299,81 +302,94 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
     const int rw = warp - 2;                                 // 0..15
     const int q4 = warp & 3;                                 // TMEM lane quarter of this warp
     const int part = rw >> 2;                                // which quarter of the columns of every step
+    const int rg = part >> 1, hh = part & 1;                 // softmax: row-warp group, head within a group of two
     const uint32_t r = (uint32_t)(q4 * 32 + lane);           // token row of the tile == TMEM lane
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q4 * 32) << 16);
     float2* exch = reinterpret_cast<float2*>(smem + HC_OFF_EXCH);         // [2][PARTS][128]
-    uint8_t* pu_part = smem + HC_OFF_PU + (part >> 1) * HC_SUB;           // K-block part / 2, chunks (part % 2) * 4 ..
+    float* inv_sum = reinterpret_cast<float*>(smem + HC_OFF_INV);         // [8][128]
+    uint8_t* p_head = smem + HC_OFF_XO + (uint32_t)(rg * 2 + hh) * HC_SUB;   // P of this thread's head: one K-block
+    uint8_t* pu_part = smem + HC_OFF_PU + (part >> 1) * HC_SUB;           // U: K-block part / 2, chunks (part % 2) * 4 ..
     const uint32_t pu_chunk0 = (uint32_t)(part & 1) * 4;
-    uint32_t row_uses = 0;
-    int q = 0;
+    uint32_t row_uses = 0, my_p = 0;
     bool ok = true;
     HcTileUser tu;
     for (int g = 0; g < n && ok; ++g) {
       const int t = t_begin + g;
       const int b = tu.of(tile_start, p.B, t);
       const int row0 = off[b] + (t - tu.lo) * HC_TILE;
-      // ---- per group: softmax over the 64 links of a head (two threads per head), P_c -> smem
-      for (int c = 0; c < NG && ok; ++c, ++q) {
-        if (!mbar_wait(&s_full[q & 1], (uint32_t)(q >> 1) & 1u, p.err, 32)) { ok = false; break; }
+      const uint32_t R0 = (uint32_t)(g & 1) * 256u, R1 = 256u - R0;
+      // ---- this row-warp group's groups of two heads: softmax over the 64 links of this thread's head, P_c -> smem
+      for (int c = rg; c < NG && ok; c += 2, ++my_p) {
+        const int sg = c >> 1;
+        if (!mbar_wait(&s_full[sg], (uint32_t)g & 1u, p.err, 32)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t col = lane_addr + (sg ? R1 : R0) + (uint32_t)(c & 1) * 128u + (uint32_t)hh * 64u;
         float v[32];
-        tmem_ld_32x32(lane_addr + COL_SC + (uint32_t)(q & 1) * 128 + part * 32, v);
-        tmem_wait_ld();
-        if (p.silu) {
-          // SiLU(s) / ell: every history query attends to the ell links of the head (Algorithm 1)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) { const float hx = 0.5f * v[j]; v[j] = fmaf(hx, hc_tanh(hx), hx) * (1.0f / HC_ELL); }
-        } else {
-          float mx = v[0];
+        float mx = 0.f, sum = 0.f;
+        if (!p.silu) {
+          tmem_ld_32x32(col, v);
+          tmem_wait_ld();
+          mx = v[0];
 #pragma unroll
           for (int j = 1; j < 32; ++j) mx = fmaxf(mx, v[j]);
-          float s0 = 0.f, s1 = 0.f;
+          tmem_ld_32x32(col + 32, v);
+          tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            v[j] = hc_ex2(v[j] - mx);
-            v[j + 1] = hc_ex2(v[j + 1] - mx);
-            s0 += v[j];
-            s1 += v[j + 1];
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, v[j]);
+        }
+        // the P buffers lie over the token tile: every score contraction of the tile must have read it, and the value mix
+        // that read this buffer last must have run
+        if (!mbar_wait(&s_full[n_sg - 1], (uint32_t)g & 1u, p.err, 35)) { ok = false; break; }
+        if (my_p > 0 && !mbar_wait(&pv_done[rg], (my_p - 1) & 1u, p.err, 36)) { ok = false; break; }
+#pragma unroll
+        for (int hv = 0; hv < 2; ++hv) {
+          tmem_ld_32x32(col + hv * 32, v);
+          tmem_wait_ld();
+          if (p.silu) {
+            // SiLU(s) / ell: every history query attends to the ell links of the head (Algorithm 1)
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { const float hx = 0.5f * v[j]; v[j] = fmaf(hx, hc_tanh(hx), hx) * (1.0f / HC_ELL); }
+          } else {
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              v[j] = hc_ex2(v[j] - mx);
+              v[j + 1] = hc_ex2(v[j + 1] - mx);
+              s0 += v[j];
+              s1 += v[j + 1];
+            }
+            sum += s0 + s1;
           }
-          // one exchange with the thread that holds the other half of the head
-          float2* ex = exch + (row_uses & 1u) * (HC_PARTS * 128);
-          ex[part * 128 + r] = make_float2(mx, s0 + s1);
-          if (!hc_group_sync(&row_bar[q4], row_uses, lane, p.err, 35)) { ok = false; break; }
-          const float2 other = ex[(part ^ 1) * 128 + r];
-          const float M = fmaxf(mx, other.x);
-          const float mine = hc_ex2(mx - M);
-          const float scale = __fdividef(mine, fmaf(s0 + s1, mine, other.y * hc_ex2(other.x - M)));
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] *= scale;
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint4 o;
+            o.x = hc_pack(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = hc_pack(v[c8 * 8 + 2], v[c8 * 8 + 3]);
+            o.z = hc_pack(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = hc_pack(v[c8 * 8 + 6], v[c8 * 8 + 7]);
+            *reinterpret_cast<uint4*>(p_head + hc_chunk(r, (uint32_t)(hv * 4 + c8))) = o;
+          }
         }
-        // P_{q-1} must have been consumed by its value mix before the buffer is rewritten
-        if (q > 0 && !mbar_wait(pv_done, (uint32_t)(q - 1) & 1u, p.err, 36)) { ok = false; break; }
-#pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
-          uint4 o;
-          o.x = hc_pack(v[c8 * 8 + 0], v[c8 * 8 + 1]); o.y = hc_pack(v[c8 * 8 + 2], v[c8 * 8 + 3]);
-          o.z = hc_pack(v[c8 * 8 + 4], v[c8 * 8 + 5]); o.w = hc_pack(v[c8 * 8 + 6], v[c8 * 8 + 7]);
-          *reinterpret_cast<uint4*>(pu_part + hc_chunk(r, pu_chunk0 + (uint32_t)c8)) = o;
-        }
+        // the exponentials go to the value mix unnormalised; O is divided by the row sum of its head afterwards
+        inv_sum[(c * 2 + hh) * 128 + (int)r] = p.silu ? 1.0f : __fdividef(1.0f, sum);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(p_ready);
+        if (lane == 0) mbar_arrive(&p_ready[rg]);
       }
       if (!ok) break;
-      // ---- O: this thread's 64 columns -> bf16 -> K-block `part` of the X / O buffer (every scores MMA has run)
+      // ---- O: this thread's 64 columns / row sum of their heads -> bf16 -> K-block `part` of the X / P / O buffer
       if (!mbar_wait(o_full, (uint32_t)g & 1u, p.err, 33)) { ok = false; break; }
       tc_fence_after();
 #pragma unroll
       for (int c = 0; c < 64; c += 32) {
         float a[32];
-        tmem_ld_32x32(lane_addr + COL_O + part * 64 + c, a);
+        tmem_ld_32x32(lane_addr + R0 + part * 64 + c, a);
+        const float sc = inv_sum[((part * 64 + c) / d_h) * 128 + (int)r];
         tmem_wait_ld();
 #pragma unroll
         for (int c8 = 0; c8 < 4; ++c8) {
           uint4 o;
-          o.x = hc_pack(a[c8 * 8 + 0], a[c8 * 8 + 1]); o.y = hc_pack(a[c8 * 8 + 2], a[c8 * 8 + 3]);
-          o.z = hc_pack(a[c8 * 8 + 4], a[c8 * 8 + 5]); o.w = hc_pack(a[c8 * 8 + 6], a[c8 * 8 + 7]);
+          o.x = hc_pack(a[c8 * 8 + 0] * sc, a[c8 * 8 + 1] * sc); o.y = hc_pack(a[c8 * 8 + 2] * sc, a[c8 * 8 + 3] * sc);
+          o.z = hc_pack(a[c8 * 8 + 4] * sc, a[c8 * 8 + 5] * sc); o.w = hc_pack(a[c8 * 8 + 6] * sc, a[c8 * 8 + 7] * sc);
           *reinterpret_cast<uint4*>(smem + HC_OFF_XO + part * HC_SUB + hc_chunk(r, (uint32_t)(c >> 3) + c8)) = o;
         }
       }
@@ -386,8 +402,8 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         if (!mbar_wait(gu_full, (uint32_t)(2 * g + hf) & 1u, p.err, 34)) { ok = false; break; }
         tc_fence_after();
         float gt[32], up[32];
-        tmem_ld_32x32(lane_addr + COL_GU + part * 32, gt);
-        tmem_ld_32x32(lane_addr + COL_GU + 128 + part * 32, up);
+        tmem_ld_32x32(lane_addr + R1 + part * 32, gt);
+        tmem_ld_32x32(lane_addr + R1 + 128 + part * 32, up);
         tmem_wait_ld();
 #pragma unroll
         for (int c8 = 0; c8 < 4; ++c8) {
@@ -411,8 +427,8 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
       if (!mbar_wait(sp_full, (uint32_t)g & 1u, p.err, 37)) { ok = false; break; }
       tc_fence_after();
       float a0[32], a1[32];
-      tmem_ld_32x32(lane_addr + COL_SP + part * 64, a0);
-      tmem_ld_32x32(lane_addr + COL_SP + part * 64 + 32, a1);
+      tmem_ld_32x32(lane_addr + R0 + part * 64, a0);
+      tmem_ld_32x32(lane_addr + R0 + part * 64 + 32, a1);
       tmem_wait_ld();
       // S' is in registers: the columns may take the next tile's value mix while this tile is normalised and stored
       tc_fence_before();
@@ -444,10 +460,10 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
         for (int i = 0; i < HC_PARTS; ++i) { const float dm = e[i].x - mu; tot += e[i].y + 64.0f * dm * dm; }
         rstd = rsqrtf(tot * (1.0f / HC_D) + p.ln_eps);
       }
-      // Out through a 2 KB patch of the P / U buffer that belongs to this warp alone (S' has consumed U): the warp stages
+      // Out through a 2 KB patch of the V / U buffer that belongs to this warp alone (S' has consumed U): the warp stages
       // 32 columns of its 32 rows (row R at R * 64 bytes, 16-byte chunk c at position c ^ ((R >> 1) & 3): conflict-free
       // both ways), then writes them with four lanes per row, 64 contiguous bytes each.  Only the warp itself has to
-      // rendezvous; the patch lies inside the rows of the P / U buffer that this warp and its column neighbour write.
+      // rendezvous.
       {
         uint8_t* patch = smem + HC_OFF_PU + (part >> 1) * HC_SUB + q4 * 4096 + (part & 1) * 2048;
         const int row_end = off[b + 1];
@@ -476,8 +492,8 @@ k_hist_update_d256_tc(const __grid_constant__ CUtensorMap tmX, const __grid_cons
           __syncwarp();
         }
       }
-      // without the softmax exchange nothing else keeps the column neighbour from writing the next P over this patch
-      if (p.silu && !hc_group_sync(&row_bar[q4], row_uses, lane, p.err, 39)) { ok = false; break; }
+      // the V / U buffer may take the next tile's link values
+      if (lane == 0) mbar_arrive(pu_free);
     }
   }
 
@@ -499,10 +515,9 @@ lime_status launch_hist_update_d256_tc(const HistUpdate256Args& a, cudaStream_t 
   const int HL = a.H * HC_ELL;
   CUtensorMap tmX, tmK2, tmV, tmWgu, tmWo;
   const uint64_t users = a.shared ? 1 : (uint64_t)a.B;
-  const int v_rows = 2 * (HC_D / a.H) < 128 ? 2 * (HC_D / a.H) : 128;      // value rows of one slab: a group of two heads
   if (!make_tmap_bf16_sw128(&tmX, a.hist_in, (uint64_t)a.total, HC_D, HC_D, HC_TILE) ||
       !make_tmap_bf16_sw128(&tmK2, a.K2, users * HL, HC_D, HC_D, 128) ||
-      !make_tmap_bf16_sw128(&tmV, a.V2t, users * HC_D, HC_ELL, HC_ELL, v_rows) ||
+      !make_tmap_bf16_sw128(&tmV, a.V2t, users * HC_D, HC_ELL, HC_ELL, 256) ||
       !make_tmap_bf16_sw128(&tmWgu, a.WguT, 2 * HC_F, HC_D, HC_D, 128) ||
       !make_tmap_bf16_sw128(&tmWo, a.WoT, HC_D, HC_F, HC_F, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
