@@ -46,6 +46,7 @@ struct LbCfg {
   static constexpr uint32_t QSUB = 128 * 128;                   // [128 rows x 64 features]
   static constexpr uint32_t Q_BUF = (D / 64) * QSUB;
   static constexpr int PBUFS = 2;                               // one per group
+  static constexpr int SBUFS = 3;                               // score buffers in TMEM: tile g uses buffer g % 3
   static constexpr uint32_t P_BUF = 128 * 128;                  // [128 rows x 64 tokens]
   static constexpr uint32_t OFF_X = 0;
   static constexpr uint32_t OFF_Q2 = XSTAGES * X_STAGE;
@@ -54,12 +55,11 @@ struct LbCfg {
   static constexpr uint32_t OFF_EXCH = OFF_P + PBUFS * P_BUF;
   static constexpr uint32_t EXCH_FLOATS = (2 + GROUPS) * 128;
   static constexpr uint32_t OFF_BAR = OFF_EXCH + EXCH_FLOATS * 4;
-  static constexpr int IDX_CAP = 1025;                          // users + 1 whose offsets are staged in shared memory
-  static constexpr uint32_t OFF_IDX = OFF_BAR + 256;
-  static constexpr uint32_t SMEM = OFF_IDX + 2 * IDX_CAP * 4 + 8 + 1024;     // + slack to align the base to 1024 bytes
-  static constexpr uint32_t TMEM_COLS = D > 128 ? 512 : 256;    // scores: 2 x 64 columns; accumulator: D columns
-  static_assert(OUT % 32 == 0 && COLS == 64, "column split of a row");
-  static_assert(SMEM + 1024 <= 232448, "shared memory budget of one CTA");
+  static constexpr uint32_t SMEM = OFF_BAR + 256;
+  static constexpr uint32_t COL_S = 0, COL_O = 256;             // scores: 3 x 64 columns; accumulator: D columns
+  static constexpr uint32_t TMEM_COLS = 512;
+  static_assert(OUT % 32 == 0 && COLS == 64 && D <= 256, "column split of a row");
+  static_assert(SMEM <= 232448, "shared memory budget of one CTA");
 };
 constexpr float LB_RESCALE_THRESHOLD = 8.0f;                  // in log2 units
 
@@ -67,6 +67,8 @@ struct LinkAttn64Params {
   const int32_t* off;
   const int32_t* chunk_start;     // [B+1] prefix of per-user chunk counts
   const int32_t* chunk_user;      // [chunk items] user of each (user, chunk) item
+  const int32_t* group_start;     // [groups + 1] the items of a group of CTAs (one CTA per row block) are
+  const int32_t* group_items;     //              group_items[group_start[j] .. group_start[j + 1])
   int B, chunk, shared, ell, H;
   int silu;
   int HL, RB;                     // stacked (head, link) rows in all, and 128-row blocks of them (one per work item)
@@ -122,51 +124,83 @@ __device__ __forceinline__ float lb_probabilities(const float (&v)[COLS], float 
   return ls0 + ls1;
 }
 
+// Walk over the (user, chunk) items of a CTA's group, in the order the schedule dealt them (even token counts across
+// the groups).  The index arrays stay in global memory (shared memory is all tiles), so the items and users of the
+// next two steps and the token range of the next item are fetched an item ahead.
 struct LbItemWalk {
-  int ci, stride, n_ci;     // (user, chunk) index of the current item, its step, and the number of such items
-  int b0, b1, b2;           // users of the current item, the next, and the one after (-1: none)
-  __device__ __forceinline__ void init(const int32_t* __restrict__ chunk_user, int first, int step, int n) {
-    ci = first; stride = step; n_ci = n;
-    b0 = ci < n ? __ldg(chunk_user + ci) : -1;
-    b1 = ci + step < n ? __ldg(chunk_user + ci + step) : -1;
+  int pos, end;             // position in group_items of the current item, and of the group's end
+  int ci, ci1, ci2;         // (user, chunk) index of the current item, the next, and the one after
+  int b0, b1, b2;           // their users (-1: none)
+  int tok0, tok1, single;   // token range of the current item; 1 if its user has this chunk only
+  int ntok0, ntok1, nsingle;
+  const int32_t* items; const int32_t* chunk_user; const int32_t* chunk_start; const int32_t* off;
+  int chunk;
+  __device__ __forceinline__ void range(int ci_, int b, int& t0, int& t1, int& sg) const {
+    const int c0 = __ldg(chunk_start + b), c1 = __ldg(chunk_start + b + 1), o0 = __ldg(off + b), o1 = __ldg(off + b + 1);
+    t0 = o0 + (ci_ - c0) * chunk;
+    t1 = min(o1, t0 + chunk);
+    sg = (c1 - c0 == 1) ? 1 : 0;
+  }
+  __device__ __forceinline__ void init(const int32_t* it, const int32_t* cu, const int32_t* cs, const int32_t* of, int ch, int first, int last) {
+    items = it; chunk_user = cu; chunk_start = cs; off = of; chunk = ch;
+    pos = first; end = last;
+    ci = pos < end ? __ldg(items + pos) : -1;
+    ci1 = pos + 1 < end ? __ldg(items + pos + 1) : -1;
+    ci2 = -1;
+    b0 = ci >= 0 ? __ldg(chunk_user + ci) : -1;
+    b1 = ci1 >= 0 ? __ldg(chunk_user + ci1) : -1;
     b2 = -1;
+    tok0 = tok1 = single = ntok0 = ntok1 = nsingle = 0;
+    if (b0 >= 0) range(ci, b0, tok0, tok1, single);
+    if (b1 >= 0) range(ci1, b1, ntok0, ntok1, nsingle);
   }
-  __device__ __forceinline__ bool valid() const { return ci < n_ci; }
-  __device__ __forceinline__ void prefetch(const int32_t* __restrict__ chunk_user) {
-    b2 = ci + 2 * stride < n_ci ? __ldg(chunk_user + ci + 2 * stride) : -1;
+  __device__ __forceinline__ bool valid() const { return pos < end; }
+  __device__ __forceinline__ void prefetch() {
+    ci2 = pos + 2 < end ? __ldg(items + pos + 2) : -1;
+    b2 = ci2 >= 0 ? __ldg(chunk_user + ci2) : -1;
   }
-  __device__ __forceinline__ void advance() { ci += stride; b0 = b1; b1 = b2; }
+  __device__ __forceinline__ void advance() {
+    ++pos; ci = ci1; ci1 = ci2; b0 = b1; b1 = b2;
+    tok0 = ntok0; tok1 = ntok1; single = nsingle;
+    if (b1 >= 0) range(ci1, b1, ntok0, ntok1, nsingle);
+  }
 };
 
 template <class G>
 __global__ void __launch_bounds__(G::THREADS, 1)
 k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttn64Params p) {
   using namespace tc;
-  constexpr int D = G::D, TILE = G::TILE, COLS = G::COLS, OUT = G::OUT, XSTAGES = G::XSTAGES, PBUFS = G::PBUFS;
-  const int n_items = p.chunk_start[p.B] * p.RB;          // work items: (user, chunk) x row block; gridDim % RB == 0, so
-  if ((int)blockIdx.x >= n_items) return;                  // a CTA keeps one row block for its whole life
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  constexpr int D = G::D, TILE = G::TILE, COLS = G::COLS, OUT = G::OUT, XSTAGES = G::XSTAGES, PBUFS = G::PBUFS, SBUFS = G::SBUFS;
+  // work items: (user, chunk) x row block.  gridDim % RB == 0: a CTA keeps one row block for its whole life, and the RB
+  // CTAs of a group walk the same items, so the history rows they share meet in L2.
+  const int grp_first = __ldg(p.group_start + (int)blockIdx.x / p.RB), grp_end = __ldg(p.group_start + (int)blockIdx.x / p.RB + 1);
+  if (grp_first >= grp_end) return;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  if ((smem_u32(smem) & 1023u) != 0) {                     // the swizzled tiles need a 1024-byte aligned base
+    if (threadIdx.x == 0) atomicCAS(p.err, 0, 97);
+    return;
+  }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + G::OFF_BAR);
   uint64_t* x_full = bars;             // [XSTAGES]
   uint64_t* x_empty = bars + 4;        // [XSTAGES]  second MMA of the tile done
-  uint64_t* s_full = bars + 8;         // [2]  score tile in TMEM
-  uint64_t* p_ready = bars + 10;       // [2]  per tile and P buffer: P in smem (the four warps of that buffer's group)
-  uint64_t* p_free = bars + 12;        // [2]  per tile and P buffer: second MMA done reading P (and accumulator up to date)
-  uint64_t* o_free = bars + 14;        //      accumulator of the item read out (all softmax warps)
+  uint64_t* s_full = bars + 8;         // [SBUFS]  score tile in TMEM
+  uint64_t* p_ready = bars + 11;       // [2]  per tile and P buffer: P in smem (the four warps of that buffer's group)
+  uint64_t* p_free = bars + 13;        // [2]  per tile and P buffer: second MMA done reading P (and accumulator up to date)
+  uint64_t* o_free = bars + 15;        //      accumulator of the item read out (all softmax warps)
   uint64_t* row_bar = bars + 16;       // [4]  rendezvous of the two warps that share a TMEM lane quarter (end of an item)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 20);
-  uint64_t* q_full = bars + 22;        //      folded queries of a user landed
-  uint64_t* q_empty = bars + 23;       //      every score MMA that reads them has run
-  uint64_t* mref_bar = bars + 24;      // [2 tile parities][4 quarters]  reference maxima after the tile published (and the
+  uint64_t* q_full = bars + 21;        //      folded queries of a user landed
+  uint64_t* q_empty = bars + 22;       //      every score MMA that reads them has run
+  uint64_t* mref_bar = bars + 23;      // [2 tile parities][4 quarters]  reference maxima after the tile published (and the
                                        //                                previous ones read) by the handling group's warp
+  static_assert(XSTAGES <= 4 && SBUFS == 3 && PBUFS == 2, "barrier table above");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < XSTAGES; ++s) { mbar_init(&x_full[s], 1); mbar_init(&x_empty[s], 1); }
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
-    for (int i = 0; i < 2; ++i) mbar_init(&s_full[i], 1);
+    for (int i = 0; i < SBUFS; ++i) mbar_init(&s_full[i], 1);
     mbar_init(&p_ready[0], G::GROUP_WARPS); mbar_init(&p_ready[1], G::GROUP_WARPS); mbar_init(&p_free[0], 1); mbar_init(&p_free[1], 1);
     mbar_init(o_free, G::SOFTMAX_WARPS);
     for (int i = 0; i < 4; ++i) mbar_init(&row_bar[i], G::GROUPS);
@@ -175,26 +209,13 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, G::TMEM_COLS); tmem_relinquish(); }
-  const int32_t* chunk_start = p.chunk_start;
-  const int32_t* off = p.off;
-  if (p.B + 1 <= G::IDX_CAP) {
-    int32_t* idx = reinterpret_cast<int32_t*>(smem + G::OFF_IDX);
-    for (int i = threadIdx.x; i <= p.B; i += G::THREADS) { idx[i] = p.chunk_start[i]; idx[G::IDX_CAP + i] = p.off[i]; }
-    chunk_start = idx;
-    off = idx + G::IDX_CAP;
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  constexpr uint32_t COL_S = 0, COL_O = 128;      // scores: 2 x 64 columns; accumulator: D columns
+  constexpr uint32_t COL_S = G::COL_S, COL_O = G::COL_O;
 
   const int rb = (int)blockIdx.x % p.RB;
-  const int ci_first = (int)blockIdx.x / p.RB, ci_step = (int)gridDim.x / p.RB, n_ci = n_items / p.RB;
-  auto item_range = [&](int ci, int b, int& tok0, int& tok1) {
-    tok0 = off[b] + (ci - chunk_start[b]) * p.chunk;
-    tok1 = min(off[b + 1], tok0 + p.chunk);
-  };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -203,11 +224,10 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       bool ok = true;
       int g = 0, qn = 0, prev_user = -1;
       LbItemWalk w;
-      for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance()) {
-        w.prefetch(p.chunk_user);
+      for (w.init(p.group_items, p.chunk_user, p.chunk_start, p.off, p.chunk, grp_first, grp_end); w.valid() && ok; w.advance()) {
+        w.prefetch();
         const int b = w.b0;
-        int tok0, tok1;
-        item_range(w.ci, b, tok0, tok1);
+        const int tok0 = w.tok0, tok1 = w.tok1;
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
@@ -246,20 +266,19 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t oa = (uint32_t)(kk >> 2) * G::QSUB + (uint32_t)(kk & 3) * 32;
           const uint32_t ob = (uint32_t)(kk >> 2) * G::XSUB + (uint32_t)(kk & 3) * 32;
-          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g & 1) * TILE, make_sdesc_k_sw128(sbase + G::OFF_Q2 + oa),
+          mma_bf16_ss(tmem_base + COL_S + (uint32_t)(g % SBUFS) * TILE, make_sdesc_k_sw128(sbase + G::OFF_Q2 + oa),
                       make_sdesc_k_sw128(sbase + G::OFF_X + s * G::X_STAGE + ob), idesc_s, kk != 0);
         }
-        mma_commit(&s_full[g & 1]);
+        mma_commit(&s_full[g % SBUFS]);
         return true;
       };
       bool ok = true;
       int g = 0, qn = 0, k = 0, prev_user = -1;
       LbItemWalk w;
-      for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance(), ++k) {
-        w.prefetch(p.chunk_user);
+      for (w.init(p.group_items, p.chunk_user, p.chunk_start, p.off, p.chunk, grp_first, grp_end); w.valid() && ok; w.advance(), ++k) {
+        w.prefetch();
         const int b = w.b0;
-        int tok0, tok1;
-        item_range(w.ci, b, tok0, tok1);
+        const int tok0 = w.tok0, tok1 = w.tok1;
         const bool load_q = p.shared ? (qn == 0) : (b != prev_user);
         prev_user = b;
         if (load_q) {
@@ -269,14 +288,13 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         // will the producer replace the queries after this item?
         const bool next_reloads = !p.shared && w.b1 >= 0 && w.b1 != b;
         const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
+        // The scores run two tiles ahead of the second contraction: while the group of tile g is in its chain, the
+        // tensor pipe holds the value contraction of tile g - 1 and the scores of tile g + 1, so it never waits for a
+        // chain that has not even started.  Score buffer (g + 2) % 3 was read before p_ready(g - 1).
         if (!issue_scores(g)) { ok = false; break; }
-        if (n_tiles == 1 && next_reloads) mma_commit(q_empty);
+        if (n_tiles > 1 && !issue_scores(g + 1)) { ok = false; break; }
+        if (n_tiles <= 2 && next_reloads) mma_commit(q_empty);
         for (int t = 0; t < n_tiles; ++t, ++g) {
-          // the next tile's scores overlap this tile's softmax (its score buffer was read before p_ready(g-1))
-          if (t + 1 < n_tiles) {
-            if (!issue_scores(g + 1)) { ok = false; break; }
-            if (t + 2 == n_tiles && next_reloads) mma_commit(q_empty);
-          }
           const int s = g % XSTAGES;
           if (!mbar_wait(&p_ready[g % PBUFS], (uint32_t)(g / PBUFS) & 1u, p.err, 52)) { ok = false; break; }
           // the first tile of an item overwrites the accumulator: the previous item must have been read out
@@ -287,6 +305,10 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                         make_sdesc_mn_sw128(sbase + G::OFF_X + s * G::X_STAGE + (uint32_t)kk * 2048, G::XSUB), idesc_o, (t | kk) != 0);
           mma_commit(&x_empty[s]);
           mma_commit(&p_free[g % PBUFS]);
+          if (t + 2 < n_tiles) {
+            if (!issue_scores(g + 2)) { ok = false; break; }
+            if (t + 3 == n_tiles && next_reloads) mma_commit(q_empty);
+          }
         }
       }
     }
@@ -304,25 +326,25 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     int g = 0, k = 0;
     uint32_t row_uses = 0;
     LbItemWalk w;
-    for (w.init(p.chunk_user, ci_first, ci_step, n_ci); w.valid() && ok; w.advance(), ++k) {
-      w.prefetch(p.chunk_user);
+    for (w.init(p.group_items, p.chunk_user, p.chunk_start, p.off, p.chunk, grp_first, grp_end); w.valid() && ok; w.advance(), ++k) {
+      w.prefetch();
       const int b = w.b0;
-      int tok0, tok1;
-      item_range(w.ci, b, tok0, tok1);
+      const int tok0 = w.tok0, tok1 = w.tok1;
       const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
       // m_own: the reference maximum this thread's row sum is relative to; l_sum: sum over the tiles of this group
       float m_own = -INFINITY, l_sum = 0.f;
       for (int t = 0; t < n_tiles && ok; ++t, ++g) {
         if ((g & 1) != grp) continue;                          // the other group's tile
-        const int pb = grp;                                    // score buffer and P buffer of this group
+        const int pb = grp;                                    // P buffer of this group
+        const int sb = g % SBUFS;                              // score buffer of the tile
         const int nvalid = min(TILE, tok1 - tok0 - t * TILE);
-        if (!mbar_wait(&s_full[pb], (uint32_t)(g >> 1) & 1u, p.err, 63)) { ok = false; break; }
+        if (!mbar_wait(&s_full[sb], (uint32_t)(g / SBUFS) & 1u, p.err, 63)) { ok = false; break; }
         tc_fence_after();
         float v[COLS];
         {
           float v0[32], v1[32];
-          tmem_ld_32x32(lane_addr + COL_S + pb * TILE, v0);
-          tmem_ld_32x32(lane_addr + COL_S + pb * TILE + 32, v1);
+          tmem_ld_32x32(lane_addr + COL_S + sb * TILE, v0);
+          tmem_ld_32x32(lane_addr + COL_S + sb * TILE + 32, v1);
           tmem_wait_ld();
 #pragma unroll
           for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
@@ -401,7 +423,7 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       else l_tot = (float)(tok1 - tok0);   // SiLU mode normalises by the number of keys (Algorithm 1): this chunk's tokens, summed over the chunks by the merge
       if (!mbar_wait(&p_free[gl & 1], (uint32_t)(gl >> 1) & 1u, p.err, 66)) { ok = false; break; }
       tc_fence_after();
-      const bool single = chunk_start[b + 1] - chunk_start[b] == 1;
+      const bool single = w.single != 0;
       const float inv = 1.0f / l_tot;
       __nv_bfloat16* dst_o = p.Ohat + (int64_t)b * p.ell * (p.H * D) + ohat_off;
       float* dst_p = p.part_acc + ((int64_t)w.ci * p.HL + R) * D + grp * OUT;
@@ -443,11 +465,18 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   }
 }
 
-using LbD256 = LbCfg<256, 3>;             // d = 256, three token stages
+using LbD256 = LbCfg<256, 4>;             // d = 256, four token stages
 
 bool link_attn_d256_tc_supported(int dtype, int d, int H, int ell, int phi) {
   return dtype == LIME_BF16 && d == 256 && (H * ell) % 128 == 0 && H * ell <= 512 && ell % 4 == 0 &&
          (phi == LIME_PHI_SOFTMAX || phi == LIME_PHI_SILU);
+}
+
+int link_attn_d256_groups(int n_chunk_upper, int H, int ell) {
+  const int RB = H * ell / 128;
+  if (RB < 1) return 0;
+  const int grid = n_chunk_upper * RB < kSMs ? n_chunk_upper * RB : kSMs;
+  return grid / RB;
 }
 
 template <class G>
@@ -459,12 +488,14 @@ static lime_status launch_link_attn_t64(const LinkAttnArgs& a, cudaStream_t st, 
   if (!make_tmap_bf16_sw128(&tmX, a.hist, (uint64_t)a.total, G::D, G::D, G::TILE) ||
       !make_tmap_bf16_sw128(&tmQ2, a.Q2, users * (uint64_t)(a.H * a.ell), G::D, G::D, 128))
     return cuda_fail(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+  if (a.group_start == nullptr || a.group_items == nullptr) return LIME_INVALID_ARG;
   LinkAttn64Params p;
+  p.group_start = a.group_start; p.group_items = a.group_items;
   p.off = a.off; p.chunk_start = a.chunk_start; p.chunk_user = a.chunk_user; p.silu = a.silu; p.B = a.B; p.chunk = a.chunk; p.shared = a.shared;
   p.ell = a.ell; p.H = a.H; p.HL = a.H * a.ell; p.RB = p.HL / 128; p.part_m = a.part_m; p.part_s = a.part_s; p.part_acc = a.part_acc;
   p.Ohat = (__nv_bfloat16*)a.Ohat; p.err = a.err;
-  int grid = a.n_chunk_upper * p.RB < kSMs ? a.n_chunk_upper * p.RB : kSMs;
-  grid -= grid % p.RB;                              // a CTA's work items then all share its row block
+  const int grid = link_attn_d256_groups(a.n_chunk_upper, a.H, a.ell) * p.RB;
+  if (a.n_groups * p.RB != grid) return LIME_INVALID_ARG;      // the schedule was dealt for another grid
   lime_status es = ensure_dynamic_smem((const void*)k_link_attn_t64_tc<G>, (int)G::SMEM, smem_set);
   if (es != LIME_OK) return es;
   ProfScope _p(name, st);

@@ -68,6 +68,7 @@ struct Workspace {
   // link rows, fp32
   float *T, *QT, *KT, *VT, *AT, *UT, *LP, *LS32;
   int32_t *chunk_start, *tile_start, *chunk_user, *merge_needed;
+  GroupSchedule groups;          // balanced deal of the chunk items (d = 256 kernels only)
   float *part_m, *part_s, *part_acc;
   // tensor-core path: folded link-side operands (bf16) and their row sums
   void *Q2, *K2, *G2t, *U2t, *V2t;
@@ -101,6 +102,13 @@ static Workspace carve(const Ctx* c, void* base, int32_t B, int64_t total) {
   w.n_chunk_upper = (int)((total + w.chunk - 1) / w.chunk + B);
   w.n_tile_upper = (int)((total + kHistTile - 1) / kHistTile + B);
   w.chunk_user = (int32_t*)take((size_t)w.n_chunk_upper * 4);
+  if (c->tc_mode == 2) {
+    w.groups.n_groups = link_attn_d256_groups(w.n_chunk_upper, g.H, g.ell);
+    w.groups.att_tile = 64;
+    w.groups.group_start = (int32_t*)take((size_t)(w.groups.n_groups + 1) * 4);
+    w.groups.group_items = (int32_t*)take((size_t)w.n_chunk_upper * 4);
+    w.groups.scratch = (int32_t*)take((size_t)w.n_chunk_upper * 16);
+  }
   const size_t rows = (size_t)w.n_chunk_upper * g.H * g.ell;
   w.part_m = (float*)take(rows * 4);
   w.part_s = (float*)take(rows * 4);
@@ -162,6 +170,7 @@ static lime_status tc_layer_core(Ctx* c, int layer, const void* hist_in, const i
   // O[T]: links attend over the stored history (keys = values = history rows), chunks merged and normalised
   LinkAttnArgs la{};
   la.hist = hist_in; la.total = total; la.Q2 = ops.Q2; la.cQ = ops.cQ; la.off = off; la.chunk_start = w.chunk_start; la.chunk_user = w.chunk_user; la.B = B;
+  la.group_start = w.groups.group_start; la.group_items = w.groups.group_items; la.n_groups = w.groups.n_groups;
   la.chunk = w.chunk; la.n_chunk_upper = w.n_chunk_upper; la.ell = g.ell; la.d = g.d; la.H = g.H; la.shared = ops.shared;
   la.ln = hist_ln; la.ln_eps = c->ln_eps; la.silu = g.phi == LIME_PHI_SILU; la.part_m = w.part_m; la.part_s = w.part_s; la.part_acc = w.part_acc; la.Ohat = w.Ohat;
   la.err = c->dev_err;
@@ -252,7 +261,7 @@ static lime_status xor_layer_impl(Ctx* c, int layer, const void* hist_in, const 
   const lime_config& g = c->cfg;
   lime_status s;
   if (!schedules_ready) {
-    if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, st)) != LIME_OK) return s;
+    if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, w.groups, st)) != LIME_OK) return s;
   }
   if (layer_on_tensor_cores(c, layer))
     return xor_layer_tc(c, layer, hist_in, off, B, total, links_in, links_shared, hist_out, links_out, w, st);
@@ -604,7 +613,7 @@ static lime_status encode_user_impl(lime_ctx* ctx, const void* hist, bool hist_n
   if (w.bytes + pad > ws_bytes) return LIME_WORKSPACE_TOO_SMALL;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   lime_status s;
-  if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, st)) != LIME_OK) return s;
+  if ((s = launch_layer_schedules(off, B, w.chunk, w.chunk_start, kHistTile, w.tile_start, w.chunk_user, w.merge_needed, w.groups, st)) != LIME_OK) return s;
   const int64_t BLd = (int64_t)B * g.ell * g.d;
   if (layer_on_tensor_cores(c, 0)) {
     if ((s = encode_user_tc(c, hist, hist_normalized, off, B, total_tokens, link_ctx, link_states, w, st)) != LIME_OK) return s;

@@ -113,8 +113,14 @@ lime_status launch_gather_ln(int dtype, const void* table, int64_t V, int d, flo
 // Work lists of the XOR layers in one launch: chunk_start[b] = sum_{b' < b} ceil(len_b' / chunk) and
 // tile_start[b] = sum_{b' < b} ceil(len_b' / tile) for b = 0..B; chunk_user[item] = user of the chunk item (may be NULL);
 // *merge_needed (may be NULL) = 1 if any user has several chunks or none (its attention rows come from the merge step)
+// Optional: the chunk items dealt to n_groups groups of CTAs with even token-tile counts (tiles of att_tile tokens);
+// group_start == NULL: not wanted.  group_start[n_groups + 1], group_items[items], scratch[4 x items].
+struct GroupSchedule {
+  int n_groups = 0, att_tile = 0;
+  int32_t* group_start = nullptr; int32_t* group_items = nullptr; int32_t* scratch = nullptr;
+};
 lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t* chunk_start, int tile, int32_t* tile_start,
-                                   int32_t* chunk_user, int32_t* merge_needed, cudaStream_t st);
+                                   int32_t* chunk_user, int32_t* merge_needed, const GroupSchedule& gs, cudaStream_t st);
 
 // Y[r, n] (+)= epilogue( LN?(X[r, :]) . W[:, n] ) for up to three weight matrices sharing X.
 struct LinearArgs {
@@ -264,6 +270,7 @@ struct LinkAttnArgs {
   const void* Q2; const float* cQ;          // folded link queries [users x H*ell x d] bf16 and their row sums
   const int32_t* off; const int32_t* chunk_start; int B, chunk, n_chunk_upper;
   const int32_t* chunk_user;                // [items] user of each (user, chunk) work item
+  const int32_t* group_start; const int32_t* group_items; int n_groups;   // balanced deal of the items (d = 256 kernel)
   int ell, d, H, shared, ln; float ln_eps;
   int silu;                                 // 1: SiLU(s) / N(U) instead of softmax (Algorithm 2)
   float *part_m, *part_s, *part_acc;        // scratch: [items x H*ell], same, [items x H*ell x d]
@@ -272,6 +279,7 @@ struct LinkAttnArgs {
   int* err;
 };
 bool link_attn_tc_supported(int dtype, int d, int H, int ell, int phi);
+int link_attn_d256_groups(int n_chunk_upper, int H, int ell);   // groups of CTAs (one CTA per 128-row block) of that kernel
 lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st);
 
 struct HistUpdateArgs {
