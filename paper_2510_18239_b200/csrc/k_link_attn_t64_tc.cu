@@ -290,7 +290,9 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         const int n_tiles = (tok1 - tok0 + TILE - 1) / TILE;
         // The scores run two tiles ahead of the second contraction: while the group of tile g is in its chain, the
         // tensor pipe holds the value contraction of tile g - 1 and the scores of tile g + 1, so it never waits for a
-        // chain that has not even started.  Score buffer (g + 2) % 3 was read before p_ready(g - 1).
+        // chain that has not even started.  Score buffer (g + 2) % 3 was read before p_ready(g - 1).  (Measured and
+        // dropped: the next scores issued before the wait for P, two tiles ahead - the fourth token stage then has no slack
+        // and the issuer waits for the copy - or one tile ahead - the chain is then exposed again.)
         if (!issue_scores(g)) { ok = false; break; }
         if (n_tiles > 1 && !issue_scores(g + 1)) { ok = false; break; }
         if (n_tiles <= 2 && next_reloads) mma_commit(q_empty);
