@@ -9,18 +9,21 @@
 //   scores [128 x 64]   = Q2_block [128 x d] . X_tile^T          (one block of 128 stacked (head, link) rows per work item)
 //   acc    [128 x d]   += P [128 x 64] . X_tile
 // At d = 256 the accumulator takes 256 TMEM columns and a block of folded queries 64 KB of shared memory, which only fits
-// with a 64-token tile (32 KB per stage, three stages; two score buffers of 64 columns; two P buffers of 16 KB).  The rows
+// with a 64-token tile (32 KB per stage, four stages; three score buffers of 64 columns; two P buffers of 16 KB: all of
+// the CTA's shared memory but 1 KB, so the index arrays stay in global memory and are read an item ahead).  The rows
 // read must be LayerNorm-ed already (the lookup or the previous layer's history update stores them so); there is no
 // on-the-fly LayerNorm in this kernel.  Online softmax in the log2 domain with lazy rescale, or SiLU(s) / N(U) with `silu`
 // (Algorithms 1-2).
 //
-// Persistent CTAs walk (user, chunk) x row-block items; warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 softmax.  What
+// Persistent CTAs walk (user, chunk) x row-block items - the four CTAs of a group take the same items, one row block
+// each, in the order the schedule kernel dealt them so that every group gets the same number of token tiles; warp 0 TMA producer, warp 1 MMA issuer, warps 2-9 softmax.  What
 // a softmax warp does for a tile is a chain of waits (scores in TMEM -> TMEM load -> row maximum -> exponentials -> P in
 // shared memory -> fence -> signal) whose latency, not its arithmetic, sets the tile period, so the eight warps form TWO
 // GROUPS that take alternate tiles: while one group is in the middle of its chain the other starts the next tile's.  A
 // group is four warps, ONE thread per stacked row (the row's 64 scores of the tile in registers: no exchange between
 // threads for the maximum, and with 320 threads per CTA no register spills - with shared memory configured to its
-// maximum a spill is a round trip to L2), and owns the score buffer and the P buffer of its tile parity.  The running
+// maximum a spill is a round trip to L2), and owns the P buffer of its tile parity; tile g's scores sit in buffer g % 3
+// and are issued two tiles ahead of its value contraction.  The running
 // reference maximum of a row is shared by both groups: the group that handles tile g publishes it (after its own decision
 // whether to raise it) and the other group picks it up for tile g + 1; each group keeps the partial row sums of its own
 // tiles, relative to the last reference it saw, and the two threads of a row combine them when the item ends.
