@@ -72,6 +72,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -240,7 +243,7 @@ static lime_status launch_gemm(const void* A, int64_t M, int K, const void* Bt, 
   ProfScope _p(name, st);
   const int64_t tiles = m_tiles * n_tiles;
   const unsigned grid = (unsigned)(tiles < kSMs ? tiles : kSMs);
-  k_gemm_tc<EPI, NT><<<grid, GM_THREADS, smem, st>>>(tmA, tmB, p);
+  launch_pdl(k_gemm_tc<EPI, NT>, dim3(grid), dim3(GM_THREADS), smem, st, tmA, tmB, p);
   LIME_LAUNCH_CHECK(name);
   return LIME_OK;
 }

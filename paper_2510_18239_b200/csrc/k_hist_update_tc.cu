@@ -148,10 +148,6 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tiles_all = p.tile_start[p.B];
-  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
-  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
-  const int n = t_end - t_begin;                            // tiles of this CTA, g = 0..n-1
 
   if (threadIdx.x == 0) {
     mbar_init(x_full, 1); mbar_init(x_empty, 1 + HU_ROW_WARPS);
@@ -163,6 +159,17 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n_tiles_all = p.tile_start[p.B];
+  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
+  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
+  const int n = t_end - t_begin;                            // tiles of this CTA, g = 0..n-1
   const int32_t* tile_start = p.tile_start;
   const int32_t* off = p.off;
   if (p.B + 1 <= HU_IDX_CAP) {
@@ -170,11 +177,8 @@ k_hist_update_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     for (int i = threadIdx.x; i <= p.B; i += HU_THREADS) { idx[i] = p.tile_start[i]; idx[HU_IDX_CAP + i] = p.off[i]; }
     tile_start = idx;
     off = idx + HU_IDX_CAP;
+    __syncthreads();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
   constexpr uint32_t COL_SS = 0, COL_GU = 256;      // scores / S' buffer of tile g: COL_SS + (g & 1) * 128
 
   if (warp == 0) {
@@ -569,8 +573,8 @@ static lime_status launch_hu(const HistUpdateArgs& a, cudaStream_t st) {
                         : ensure_dynamic_smem((const void*)k_hist_update_tc<ELL, false>, (int)HU_SMEM, smem_plain);
   if (es != LIME_OK) return es;
   ProfScope _p("k_hist_update_tc", st);
-  if (a.ln) k_hist_update_tc<ELL, true><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
-  else k_hist_update_tc<ELL, false><<<grid, HU_THREADS, HU_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  if (a.ln) launch_pdl(k_hist_update_tc<ELL, true>, dim3(grid), dim3(HU_THREADS), HU_SMEM, st, tmX, tmK2, tmG, tmU, tmWo, p);
+  else launch_pdl(k_hist_update_tc<ELL, false>, dim3(grid), dim3(HU_THREADS), HU_SMEM, st, tmX, tmK2, tmG, tmU, tmWo, p);
   LIME_LAUNCH_CHECK("k_hist_update_tc");
   return LIME_OK;
 }

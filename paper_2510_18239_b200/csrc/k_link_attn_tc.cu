@@ -175,8 +175,6 @@ template <bool LN>
 __global__ void __launch_bounds__(LA_THREADS, 1)
 k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmQ2, const LinkAttnParams p) {
   using namespace tc;
-  const int n_items = p.chunk_start[p.B] * p.RB;          // work items: (user, chunk) x row block; gridDim % RB == 0, so
-  if ((int)blockIdx.x >= n_items) return;                  // a CTA keeps one row block for its whole life
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {
     if (threadIdx.x == 0) atomicCAS(p.err, 0, 91);
@@ -209,6 +207,16 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     prefetch_tmap(&tmX); prefetch_tmap(&tmQ2);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
+  // work items: (user, chunk) x row block; gridDim % RB == 0, so a CTA keeps one row block for its whole life
+  const int n_items = p.chunk_start[p.B] * p.RB;
+  const bool active = (int)blockIdx.x < n_items;           // a CTA without items goes straight to the end
   const int32_t* chunk_start = p.chunk_start;
   const int32_t* off = p.off;
   if (p.B + 1 <= LA_IDX_CAP) {
@@ -216,11 +224,8 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     for (int i = threadIdx.x; i <= p.B; i += LA_THREADS) { idx[i] = p.chunk_start[i]; idx[LA_IDX_CAP + i] = p.off[i]; }
     chunk_start = idx;
     off = idx + LA_IDX_CAP;
+    __syncthreads();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
   constexpr uint32_t COL_S = 0, COL_O = 256;      // scores: 2 x 128 columns; accumulator: d columns
 
   // item -> token range; identical in every role
@@ -233,7 +238,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && active) {
       const uint64_t pol_stream = policy_evict_first(), pol_keep = policy_evict_last();
       bool ok = true;
       int g = 0, qn = 0, prev_user = -1;
@@ -274,7 +279,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && active) {
       constexpr uint32_t idesc_s = make_idesc_bf16(128, 128);                 // Q2 . X^T  : both K-major
       constexpr uint32_t idesc_o = make_idesc_bf16(128, 128, false, true);    // P' . X    : B is MN-major
       const uint32_t sbase = smem_u32(smem);
@@ -333,7 +338,7 @@ k_link_attn_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ 
         }
       }
     }
-  } else {
+  } else if (active) {
     // ------------------------------------------------------------------ softmax warps (2..17)
     const int sw = warp - 2;                                   // 0..15
     const int q = warp & 3;                                    // TMEM lane quarter of this warp
@@ -574,8 +579,8 @@ lime_status launch_link_attn_tc(const LinkAttnArgs& a, cudaStream_t st) {
                         : ensure_dynamic_smem((const void*)k_link_attn_tc<false>, (int)LA_SMEM, smem_plain);
   if (es != LIME_OK) return es;
   ProfScope _p("k_link_attn_tc", st);
-  if (a.ln) k_link_attn_tc<true><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
-  else k_link_attn_tc<false><<<grid, LA_THREADS, LA_SMEM, st>>>(tmX, tmQ2, p);
+  if (a.ln) launch_pdl(k_link_attn_tc<true>, dim3(grid), dim3(LA_THREADS), LA_SMEM, st, tmX, tmQ2, p);
+  else launch_pdl(k_link_attn_tc<false>, dim3(grid), dim3(LA_THREADS), LA_SMEM, st, tmX, tmQ2, p);
   LIME_LAUNCH_CHECK("k_link_attn_tc");
   return LIME_OK;
 }

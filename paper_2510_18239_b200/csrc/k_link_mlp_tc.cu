@@ -109,6 +109,9 @@ k_link_mlp_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   constexpr uint32_t COL_GU = 0, COL_OUT = 256;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -361,7 +364,7 @@ static lime_status launch_lm(const LinkMlpArgs& a, cudaStream_t st) {
   lime_status es = ensure_dynamic_smem((const void*)k_link_mlp_tc<D>, (int)Lay::SMEM, smem_set);
   if (es != LIME_OK) return es;
   ProfScope _p("k_link_mlp_tc", st);
-  k_link_mlp_tc<D><<<(unsigned)((a.M + 127) / 128), LM_THREADS, Lay::SMEM, st>>>(tmA, tmB, tmWo, p);
+  launch_pdl(k_link_mlp_tc<D>, dim3((unsigned)((a.M + 127) / 128)), dim3(LM_THREADS), Lay::SMEM, st, tmA, tmB, tmWo, p);
   LIME_LAUNCH_CHECK("k_link_mlp_tc");
   return LIME_OK;
 }

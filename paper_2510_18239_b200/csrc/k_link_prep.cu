@@ -108,6 +108,8 @@ __global__ void __launch_bounds__(256)
 k_link_attn_merge_norm(const int32_t* __restrict__ chunk_start, const int32_t* __restrict__ merge_needed, int B, int ell, int d,
                        int H, const float* __restrict__ part_m, const float* __restrict__ part_s,
                        const float* __restrict__ part_acc, __nv_bfloat16* __restrict__ Ohat) {
+  pdl_launch_dependents();     // simple kernel: the next one may set itself up beside it
+  pdl_wait();                  // nothing is read or written before the previous kernel is complete
   if (merge_needed != nullptr && *merge_needed == 0) return;
   const int HL = H * ell;
   const int lane = threadIdx.x & 31;
@@ -164,7 +166,8 @@ lime_status launch_link_attn_merge_norm(const int32_t* chunk_start, const int32_
   ProfScope _p("k_link_attn_merge_norm", st);
   const int64_t blocks_needed = ((int64_t)B * H * ell + 7) / 8;           // 8 warps (rows) per block
   const int grid = (int)(blocks_needed < (int64_t)kSMs * 8 ? blocks_needed : (int64_t)kSMs * 8);
-  k_link_attn_merge_norm<<<grid, 256, 0, st>>>(chunk_start, merge_needed, B, ell, d, H, part_m, part_s, part_acc, (__nv_bfloat16*)Ohat);
+  launch_pdl(k_link_attn_merge_norm, dim3(grid), dim3(256), 0, st, chunk_start, merge_needed, B, ell, d, H, part_m, part_s, part_acc,
+             (__nv_bfloat16*)Ohat);
   LIME_LAUNCH_CHECK("k_link_attn_merge_norm");
   return LIME_OK;
 }

@@ -45,6 +45,8 @@ __device__ __forceinline__ void block_exclusive_scan(int n, int32_t* out, F valu
 }
 
 __global__ void __launch_bounds__(1024) k_offsets(const int32_t* __restrict__ len, int B, int32_t* __restrict__ off) {
+  pdl_launch_dependents();     // simple kernel: the next one may set itself up beside it
+  pdl_wait();                  // nothing is read or written before the previous kernel is complete
   block_exclusive_scan(B, off, [&](int i) { return max(len[i], 0); });
 }
 
@@ -125,6 +127,8 @@ k_layer_schedules(const int32_t* __restrict__ off, int B, int chunk, int32_t* __
                   int32_t* __restrict__ tile_start, int32_t* __restrict__ chunk_user, int32_t* __restrict__ merge_needed,
                   int G, int att_tile, int32_t* __restrict__ group_start, int32_t* __restrict__ group_items,
                   int32_t* __restrict__ scratch) {
+  pdl_launch_dependents();     // simple kernel: the next one may set itself up beside it
+  pdl_wait();                  // nothing is read or written before the previous kernel is complete
   // does any user's attention output need the merge step (several chunks to combine, or no history: a zero row)?
   __shared__ int any_merge;
   if (threadIdx.x == 0) any_merge = 0;
@@ -158,15 +162,15 @@ lime_status launch_layer_schedules(const int32_t* off, int B, int chunk, int32_t
                                    int32_t* chunk_user, int32_t* merge_needed, const GroupSchedule& gs, cudaStream_t st) {
   if (gs.group_start != nullptr && (gs.n_groups < 1 || gs.n_groups > 160 || gs.att_tile < 1)) return LIME_INVALID_ARG;
   ProfScope _p("k_layer_schedules", st);
-  k_layer_schedules<<<1, 1024, 0, st>>>(off, B, chunk, chunk_start, tile, tile_start, chunk_user, merge_needed, gs.n_groups,
-                                        gs.att_tile, gs.group_start, gs.group_items, gs.scratch);
+  launch_pdl(k_layer_schedules, dim3(1), dim3(1024), 0, st, off, B, chunk, chunk_start, tile, tile_start, chunk_user, merge_needed,
+             gs.n_groups, gs.att_tile, gs.group_start, gs.group_items, gs.scratch);
   LIME_LAUNCH_CHECK("k_layer_schedules");
   return LIME_OK;
 }
 
 lime_status launch_offsets(const int32_t* len, int B, int32_t* off, cudaStream_t st) {
   ProfScope _p("k_offsets", st);
-  k_offsets<<<1, 1024, 0, st>>>(len, B, off);
+  launch_pdl(k_offsets, dim3(1), dim3(1024), 0, st, len, B, off);
   LIME_LAUNCH_CHECK("k_offsets");
   return LIME_OK;
 }
@@ -233,6 +237,8 @@ template <typename T, int LANES, int WORDS>
 __global__ void __launch_bounds__(256)
 k_gather_ln(const uint4* __restrict__ table, int64_t V, int row_vec, int d, float eps, const int32_t* __restrict__ ids,
             int64_t total, uint4* __restrict__ out, int32_t* __restrict__ dev_flag) {
+  pdl_launch_dependents();     // simple kernel: the next one may set itself up beside it
+  pdl_wait();                  // nothing is read or written before the previous kernel is complete
   constexpr int PER = 16 / (int)sizeof(T);                 // elements per 16-byte word
   constexpr int ROWS = 1;   // rows per lane group and pass (more in flight measured slower: the grid already covers the latency)
   const int rows_per_block = blockDim.x / LANES;
@@ -305,10 +311,10 @@ template <typename T, int WORDS>
 static void launch_gather_ln_w(int lanes, int blocks, const uint4* tb, int64_t V, int row_vec, int d, float eps,
                                const int32_t* ids, int64_t total, uint4* o, int32_t* dev_flag, cudaStream_t st) {
   switch (lanes) {
-    case 32: k_gather_ln<T, 32, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
-    case 16: k_gather_ln<T, 16, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
-    case 8:  k_gather_ln<T, 8, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
-    default: k_gather_ln<T, 4, WORDS><<<blocks, 256, 0, st>>>(tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    case 32: launch_pdl(k_gather_ln<T, 32, WORDS>, dim3((unsigned)blocks), dim3(256), 0, st, tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    case 16: launch_pdl(k_gather_ln<T, 16, WORDS>, dim3((unsigned)blocks), dim3(256), 0, st, tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    case 8:  launch_pdl(k_gather_ln<T, 8, WORDS>, dim3((unsigned)blocks), dim3(256), 0, st, tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
+    default: launch_pdl(k_gather_ln<T, 4, WORDS>, dim3((unsigned)blocks), dim3(256), 0, st, tb, V, row_vec, d, eps, ids, total, o, dev_flag); break;
   }
 }
 template <typename T>

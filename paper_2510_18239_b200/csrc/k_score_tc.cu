@@ -73,6 +73,9 @@ k_score_tc(const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUte
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -237,7 +240,7 @@ static lime_status launch_score_tc_t(const ScoreArgs& a, int* err, cudaStream_t 
   int grid = p.n_tiles < kSMs ? p.n_tiles : kSMs;
   LIME_CUDA(cudaFuncSetAttribute(k_score_tc<ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   ProfScope _p("k_score_tc", st);
-  k_score_tc<ELL><<<grid, SCT_THREADS, smem, st>>>(tmT, tmLS, tmW, p);
+  launch_pdl(k_score_tc<ELL>, dim3(grid), dim3(SCT_THREADS), smem, st, tmT, tmLS, tmW, p);
   LIME_LAUNCH_CHECK("k_score_tc");
   return LIME_OK;
 }

@@ -89,6 +89,35 @@ lime_status cuda_fail(cudaError_t e, const char* where);
     if (_e != cudaSuccess) return ::lime::cuda_fail(_e, name);   \
   } while (0)
 
+// ----------------------------------------------------------------------------- programmatic dependent launch
+// The kernels of one step run back to back on one stream.  Launched with the programmatic-serialization attribute, a
+// kernel's CTAs may become resident while its predecessor still runs (as soon as every CTA of the predecessor has
+// executed pdl_launch_dependents() or exited), set up their barriers and tensor memory, and then block in pdl_wait()
+// until the predecessor has completed and its writes are visible.  Rules kept by every kernel launched this way:
+//  - nothing produced by an earlier kernel is read, and no global memory is written, before pdl_wait();
+//  - a kernel that allocates tensor memory calls pdl_launch_dependents() only after its allocation, so a dependent CTA
+//    that shares the SM can never hold the columns a CTA of the running kernel still waits for.
+// A kernel launched the ordinary way after such a kernel still waits for its completion, as always.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+bool pdl_enabled();      // environment LIME_PDL=0 turns the attribute off (every launch then serialises fully)
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ----------------------------------------------------------------------------- per-kernel event timing
 // While a profile is open (lime_profile_start .. lime_profile_stop) every launcher brackets its kernel with two
 // CUDA events on the launching stream.  Closed, a scope costs one predictable branch.

@@ -2,6 +2,7 @@
 // (resolved at run time, so the library does not link against libcuda).
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <cstdlib>
 
 #include "lime_common.cuh"
 #include "tc_common.cuh"
@@ -54,6 +55,14 @@ bool make_tmap_bf16_kmajor(CUtensorMap* out, const void* base, uint64_t rows, ui
                                                : (box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
   return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char* e = std::getenv("LIME_PDL");
+    return !(e != nullptr && e[0] == '0');
+  }();
+  return on;
 }
 
 lime_status ensure_dynamic_smem(const void* kernel, int bytes, bool (&done)[kMaxDeviceOrdinals]) {
