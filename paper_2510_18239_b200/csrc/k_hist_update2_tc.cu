@@ -116,10 +116,6 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 19);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_tiles_all = p.tile_start[p.B];
-  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
-  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
-  const int n = t_end - t_begin;
   const int NG = p.NG;
 
   if (threadIdx.x == 0) {
@@ -132,6 +128,17 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     prefetch_tmap(&tmX); prefetch_tmap(&tmK2); prefetch_tmap(&tmG); prefetch_tmap(&tmU); prefetch_tmap(&tmWo);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
+  const int n_tiles_all = p.tile_start[p.B];
+  const int t_begin = (int)(((int64_t)blockIdx.x * n_tiles_all) / gridDim.x);
+  const int t_end = (int)(((int64_t)(blockIdx.x + 1) * n_tiles_all) / gridDim.x);
+  const int n = t_end - t_begin;
   const int32_t* tile_start = p.tile_start;
   const int32_t* off = p.off;
   if (p.B + 1 <= H2_IDX_CAP) {
@@ -139,11 +146,8 @@ k_hist_update2_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     for (int i = threadIdx.x; i <= p.B; i += H2_THREADS) { idx[i] = p.tile_start[i]; idx[H2_IDX_CAP + i] = p.off[i]; }
     tile_start = idx;
     off = idx + H2_IDX_CAP;
+    __syncthreads();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
   // Two 128-column buffers take the scores of the groups and S' in rotation: use u of this CTA (per tile NG score uses,
   // then S') goes to buffer u & 1, so the scores of the next group are formed while the row warps still read this one's.
   constexpr uint32_t COL_A = 0, COL_GU = 128, COL_B = 384;
@@ -501,8 +505,8 @@ static lime_status launch_hu2(const HistUpdateArgs& a, int HL, cudaStream_t st) 
                         : ensure_dynamic_smem((const void*)k_hist_update2_tc<ELL, false>, (int)H2_SMEM, smem_plain);
   if (es != LIME_OK) return es;
   ProfScope _p("k_hist_update2_tc", st);
-  if (a.ln) k_hist_update2_tc<ELL, true><<<grid, H2_THREADS, H2_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
-  else k_hist_update2_tc<ELL, false><<<grid, H2_THREADS, H2_SMEM, st>>>(tmX, tmK2, tmG, tmU, tmWo, p);
+  if (a.ln) launch_pdl(k_hist_update2_tc<ELL, true>, dim3(grid), dim3(H2_THREADS), H2_SMEM, st, tmX, tmK2, tmG, tmU, tmWo, p);
+  else launch_pdl(k_hist_update2_tc<ELL, false>, dim3(grid), dim3(H2_THREADS), H2_SMEM, st, tmX, tmK2, tmG, tmU, tmWo, p);
   LIME_LAUNCH_CHECK("k_hist_update2_tc");
   return LIME_OK;
 }

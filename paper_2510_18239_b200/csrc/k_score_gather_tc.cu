@@ -82,6 +82,9 @@ k_score_gather_tc(const __grid_constant__ CUtensorMap tmLS, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done: the next kernel's CTAs may become resident; nothing an earlier kernel wrote is read before this wait
+  pdl_launch_dependents();
+  pdl_wait();
 
   if (warp < 4) {
     // ------------------------------------------------------------------ producers: thread r fetches row r of the tile
@@ -288,7 +291,7 @@ static lime_status launch_score_gather_t(const ScoreArgs& a, int* err, cudaStrea
   const int grid = p.n_tiles < kSMs ? p.n_tiles : kSMs;
   LIME_CUDA(cudaFuncSetAttribute(k_score_gather_tc<ELL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   ProfScope _p("k_score_gather_tc", st);
-  k_score_gather_tc<ELL><<<grid, SG_THREADS, smem, st>>>(tmLS, tmT, tmW, p);
+  launch_pdl(k_score_gather_tc<ELL>, dim3(grid), dim3(SG_THREADS), smem, st, tmLS, tmT, tmW, p);
   LIME_LAUNCH_CHECK("k_score_gather_tc");
   return LIME_OK;
 }
