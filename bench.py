@@ -266,12 +266,12 @@ def launch_mode(args):
 # is stale and the bench reports null.
 NCU_TRAFFIC = {
     # dense scorer: 169.9 MB read + 4.0-4.5 MB written per launch
-    ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "8accb4a67cfefc46"},
+    ("k_score_tc", "bf16_baseline", 256, 2048): {"bytes": 174.2e6, "source": "k_score_tc.cu", "sha": "823248ada31d3d04"},
     # XOR-layer kernels: 33.7 MB (layer 1) and 42.2 MB (layer 2) read + written; average per launch
-    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "186136fa777f8d53"},
-    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.6e6, "source": "k_hist_update_tc.cu", "sha": "cbdc6b1690b70517"},
+    ("k_link_attn_tc", "bf16_baseline", 256, 2048): {"bytes": 37.9e6, "source": "k_link_attn_tc.cu", "sha": "81680b45282491ef"},
+    ("k_hist_update_tc", "bf16_baseline", 256, 2048): {"bytes": 34.6e6, "source": "k_hist_update_tc.cu", "sha": "a47ccfb7ddd4247f"},
     # scorer by id over packed corpus records: 174.5 MB read + 4.1 MB written per launch
-    ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 178.6e6, "source": "k_score_gather_tc.cu", "sha": "2b14f0762b275cd7"},
+    ("k_score_gather_tc", "bf16_baseline", 256, 2048): {"bytes": 178.6e6, "source": "k_score_gather_tc.cu", "sha": "580e539a2d79f57c"},
     # scorer through the interaction network (--head 96): 169.4 MB read + 4.4 MB written per launch
     ("k_score_head_tc", "bf16_baseline", 256, 2048): {"bytes": 173.8e6, "source": "k_score_head_tc.cu", "sha": "614556b96c1342b2"},
     # d = 256 kernels: captured on 128 users of the same model and length mix (327,693 tokens) and scaled by the tokens of
