@@ -105,9 +105,10 @@ __device__ __forceinline__ bool lb_group_sync(uint64_t* bar, uint32_t& uses, int
 }
 
 // p = 2^(s - m_ref) (or SiLU(s)) for this thread's COLS token columns, as bf16 into the A-operand buffer (K-major over
-// the tile's tokens, 128-byte swizzle: one K-block of 64 tokens); columns at or past nvalid give 0.  Returns the sum.
+// the tile's tokens, 128-byte swizzle: one K-block of 64 tokens).  Columns past the end of a ragged last tile were set to
+// -inf (0 for SiLU) by the caller and give 0.  Returns the sum.
 template <bool SILU, int COLS>
-__device__ __forceinline__ float lb_probabilities(const float (&v)[COLS], float m_ref, int col0, int nvalid, uint8_t* pbuf, uint32_t r) {
+__device__ __forceinline__ float lb_probabilities(const float (&v)[COLS], float m_ref, int col0, uint8_t* pbuf, uint32_t r) {
   float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
   for (int c8 = 0; c8 < COLS / 8; ++c8) {
@@ -116,8 +117,6 @@ __device__ __forceinline__ float lb_probabilities(const float (&v)[COLS], float 
     for (int j2 = 0; j2 < 4; ++j2) {
       const int j = c8 * 8 + 2 * j2;
       float e0 = SILU ? lb_silu(v[j]) : lb_ex2(v[j] - m_ref), e1 = SILU ? lb_silu(v[j + 1]) : lb_ex2(v[j + 1] - m_ref);
-      if (col0 + j >= nvalid) e0 = 0.f;
-      if (col0 + j + 1 >= nvalid) e1 = 0.f;
       ls0 += e0;
       ls1 += e1;
       packed[j2] = lb_pack(e0, e1);
@@ -354,21 +353,31 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 32; ++j) { v[j] = v0[j]; v[32 + j] = v1[j]; }
         }
+        if (nvalid < TILE) {
+          // ragged last tile of the item: the columns past its end (rows of the next user, or the fill value) drop out
+          const float dead = p.silu ? 0.f : -INFINITY;
+#pragma unroll
+          for (int j = 0; j < COLS; ++j)
+            if (j >= nvalid) v[j] = dead;
+        }
         uint8_t* pbuf = smem + G::OFF_P + pb * G::P_BUF;
         if (p.silu) {
           // SiLU(s) / N(U) needs neither a reference maximum nor row sums: one pass, nothing shared between threads
           if (g >= PBUFS && !mbar_wait(&p_free[pb], (uint32_t)((g - PBUFS) >> 1) & 1u, p.err, 65)) { ok = false; break; }
-          lb_probabilities<true, COLS>(v, 0.f, 0, nvalid, pbuf, r);
+          lb_probabilities<true, COLS>(v, 0.f, 0, pbuf, r);
           tc_fence_before();
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(&p_ready[pb]);
           continue;
         }
-        float mx = -INFINITY;
+        // four independent chains for the row maximum (a ragged tile's dead columns hold -inf)
+        float mx0 = v[0], mx1 = v[1], mx2 = v[2], mx3 = v[3];
 #pragma unroll
-        for (int j = 0; j < COLS; ++j)
-          if (j < nvalid) mx = fmaxf(mx, v[j]);
+        for (int j = 4; j < COLS; j += 4) {
+          mx0 = fmaxf(mx0, v[j]); mx1 = fmaxf(mx1, v[j + 1]); mx2 = fmaxf(mx2, v[j + 2]); mx3 = fmaxf(mx3, v[j + 3]);
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
         // the reference the other group left after the previous tile (every tile but the very first waits, whether or
         // not it uses the value: the two groups then never drift more than one tile apart)
         float m_prev = -INFINITY;
@@ -404,7 +413,7 @@ k_link_attn_t64_tc(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
         // the P that last sat in this group's buffer must have been consumed
         if (g >= PBUFS && !mbar_wait(&p_free[pb], (uint32_t)((g - PBUFS) >> 1) & 1u, p.err, 65)) { ok = false; break; }
-        l_sum += lb_probabilities<false, COLS>(v, m_own, 0, nvalid, pbuf, r);
+        l_sum += lb_probabilities<false, COLS>(v, m_own, 0, pbuf, r);
         tc_fence_before();
         fence_proxy_async_smem();
         __syncwarp();
