@@ -816,6 +816,58 @@ def test_config2_bf16_baseline_every_logit(normalized):
     assert per_user.max() <= REL_BF16 * want.std() + 1e-4, int(np.argmax(per_user))
 
 
+def test_config2_step_replayed_from_a_cuda_graph_matches_the_eager_run():
+    """The bench workload's step (offsets -> lookup + LayerNorm -> encode -> score) captured once into a CUDA graph and
+    replayed back to back, as bench.py times it: in a replay the kernels follow one another without the host between
+    them, and those launched for programmatic dependent launch start their set-up while the previous kernel still
+    runs.  Every replay must give the eager run's logits bit for bit (the kernels are deterministic), and the eager run
+    is checked against the oracle on a few users."""
+    wl = synth.named_workloads()["bf16_baseline"]
+    inp = synth.make_inputs(wl, seed=7)
+    db = Hh.DeviceBatch(wl, inp)
+    L = db.lime
+
+    def step():
+        off = L.lengths_to_offsets(db.lengths)
+        hist = L.gather_history_normalized(db.table, db.hist_ids)
+        ls = L.encode_user_normalized(hist, off)
+        return L.score_candidates(ls, W, cand, C=wl.C)
+
+    cand = L.gather_history(db.table, db.cand_ids)
+    W = L.precompute_candidate_links(cand)
+    eager = step().clone()
+    db.Bd.lime_device_status(L.ctx)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            step()                                   # warm-up on the capture stream: sizes shared-memory attributes
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        out = step()
+    for _ in range(25):
+        g.replay()
+    torch.cuda.synchronize()
+    db.Bd.lime_device_status(L.ctx)
+    assert torch.equal(out, eager)
+    # between replays, with the output cleared: a kernel that ran ahead of its input would leave zeros or stale rows
+    for _ in range(5):
+        out.zero_()
+        g.replay()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+    off = O.lengths_to_offsets(inp["lengths"])
+    table64, links64 = Hh.LazyTable64(inp["table"], wl.dtype), synth.storage_to_f64(inp["links"], wl.dtype)
+    cfg, layers = Hh.oracle_config(wl), Hh.oracle_layers(inp, wl)
+    got = Hh.to_f64(eager).reshape(wl.B, wl.C)
+    for b in (0, 77, 255):
+        want = Hh.oracle_user(inp, wl, b, off, table64, links64, layers, cfg)[0]
+        _check_logits(got[b], want, wl.dtype)
+
+
 def test_config2_bf16_baseline_normalized_lookup_sampled():
     # the launch sequence bench.py times: lookup fused with the first layer's LayerNorm, encode on normalised rows
     wl = synth.named_workloads()["bf16_baseline"]
