@@ -276,7 +276,7 @@ NCU_TRAFFIC = {
     ("k_score_head_tc", "bf16_baseline", 256, 2048): {"bytes": 173.8e6, "source": "k_score_head_tc.cu", "sha": "614556b96c1342b2"},
     # d = 256 kernels: captured on 128 users of the same model and length mix (327,693 tokens) and scaled by the tokens of
     # a launch (persistent kernels, identical tiles: traffic grows in proportion): bytes per token, average of the layers
-    ("k_link_attn_d256_tc", "production_ragged", 1024, 8192): {"bytes_per_token": 560.0, "source": "k_link_attn_t64_tc.cu", "sha": "ac15f599de0d51f5"},
+    ("k_link_attn_d256_tc", "production_ragged", 1024, 8192): {"bytes_per_token": 560.0, "source": "k_link_attn_t64_tc.cu", "sha": "b26d676843314aed"},
     ("k_hist_update_d256_tc", "production_ragged", 1024, 8192): {"bytes_per_token": 893.0, "source": "k_hist_update_d256_tc.cu", "sha": "b84060b13975253c"},
 }
 
